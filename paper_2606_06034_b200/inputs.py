@@ -1,0 +1,143 @@
+"""Seeded synthetic inputs for the chunk-prepare path.
+
+This module only draws random tensors with the shapes and value distributions of
+the workloads; it holds none of the method's arithmetic, so the CUDA path's
+tests, the benchmark and the CPU oracle's tests can all take inputs from it.
+
+Layouts (contiguous):
+  K     [B, H_k, T, d_k]   keys, rows L2-normalised in fp32 and then cast
+  V     [B, H_v, T, d_v]   values
+  beta  [B, H_v, T]  fp32  write strength, sigmoid of a normal draw
+  g     [B, H_v, T]  fp32  cumulative log-gate, prefix sum restarted at every
+                           chunk of C tokens, of -softplus(normal draw)
+
+Two regimes:
+  "benign"       the distributions above
+  "adversarial"  beta = 0.99, g = 0 and highly correlated keys: per chunk one
+                 direction u ~ N(0, I), K_t = u + 0.1 * eps_t, row-normalised
+                 (cosine ~ 0.99), which maximises growth of the Neumann terms.
+`adversarial_heads="odd"` applies the adversarial regime to value heads with
+odd index (and to the key heads they read), the rest stay benign.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+
+import torch
+
+
+@dataclass
+class ChunkInputs:
+    K: torch.Tensor
+    V: torch.Tensor
+    beta: torch.Tensor
+    g: torch.Tensor
+    B: int
+    H_k: int
+    H_v: int
+    T: int
+    C: int
+    d_k: int
+    d_v: int
+
+    @property
+    def n_chunks(self) -> int:
+        return self.B * self.H_v * (self.T // self.C)
+
+
+def make_inputs(B: int, H_k: int, H_v: int, T: int, C: int, d_k: int, d_v: int, *,
+                seed: int, dtype: torch.dtype = torch.bfloat16,
+                device: str | torch.device = "cpu",
+                adversarial_heads: str = "none") -> ChunkInputs:
+    """Draw one workload. Tensors are drawn in the fixed order K, V, beta, g."""
+    assert T % C == 0 and H_v % H_k == 0
+    assert adversarial_heads in ("none", "odd", "all")
+    dev = torch.device(device)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(seed)
+
+    def randn(*shape):
+        return torch.randn(*shape, generator=gen, device=dev, dtype=torch.float32)
+
+    Kf = randn(B, H_k, T, d_k)
+    if adversarial_heads != "none":
+        n_ch = T // C
+        u = randn(B, H_k, n_ch, 1, d_k)
+        eps = randn(B, H_k, n_ch, C, d_k)
+        Kadv = (u + 0.1 * eps).reshape(B, H_k, T, d_k)
+        if adversarial_heads == "all":
+            Kf = Kadv
+        else:
+            # key heads with odd index are adversarial, and so are the value
+            # heads that read them (see `sel` below)
+            odd = (torch.arange(H_k, device=dev) % 2 == 1).view(1, H_k, 1, 1)
+            Kf = torch.where(odd, Kadv, Kf)
+        del u, eps, Kadv
+    Kf = Kf / Kf.norm(dim=-1, keepdim=True).clamp_min(1e-12)
+    K = Kf.to(dtype)
+    del Kf
+    V = randn(B, H_v, T, d_v).to(dtype)
+    beta = torch.sigmoid(randn(B, H_v, T))
+    graw = -torch.nn.functional.softplus(randn(B, H_v, T))
+    g = graw.view(B, H_v, T // C, C).cumsum(dim=-1).reshape(B, H_v, T).contiguous()
+    if adversarial_heads != "none":
+        if adversarial_heads == "all":
+            sel = torch.ones(H_v, dtype=torch.bool, device=dev)
+        else:
+            group = H_v // H_k
+            sel = ((torch.arange(H_v, device=dev) // group) % 2 == 1)
+        sel = sel.view(1, H_v, 1)
+        beta = torch.where(sel, torch.full_like(beta, 0.99), beta)
+        g = torch.where(sel, torch.zeros_like(g), g)
+    return ChunkInputs(K.contiguous(), V.contiguous(), beta.contiguous(), g.contiguous(),
+                       B, H_k, H_v, T, C, d_k, d_v)
+
+
+# The named workloads (shapes and regimes); seeds are fixed per workload.
+WORKLOADS = {
+    # tiny fp32 case the CPU oracle finishes at once
+    "tiny_fp32": dict(B=1, H_k=2, H_v=2, T=256, C=64, d_k=128, d_v=128, seed=0,
+                      dtype=torch.float32, adversarial_heads="none"),
+    # chunk-size sweep, bf16
+    "sweep_c16": dict(B=4, H_k=16, H_v=16, T=4096, C=16, d_k=128, d_v=128, seed=1,
+                      dtype=torch.bfloat16, adversarial_heads="none"),
+    "sweep_c32": dict(B=4, H_k=16, H_v=16, T=4096, C=32, d_k=128, d_v=128, seed=1,
+                      dtype=torch.bfloat16, adversarial_heads="none"),
+    "sweep_c64": dict(B=4, H_k=16, H_v=16, T=4096, C=64, d_k=128, d_v=128, seed=1,
+                      dtype=torch.bfloat16, adversarial_heads="none"),
+    "sweep_c128": dict(B=4, H_k=16, H_v=16, T=4096, C=128, d_k=128, d_v=128, seed=1,
+                       dtype=torch.bfloat16, adversarial_heads="none"),
+    # prefill layer with keys shared by pairs of value heads
+    "prefill_gqa": dict(B=1, H_k=16, H_v=32, T=32768, C=64, d_k=128, d_v=128, seed=2,
+                        dtype=torch.bfloat16, adversarial_heads="none"),
+    # stress + scale, odd heads adversarial
+    "stress": dict(B=8, H_k=32, H_v=32, T=65536, C=64, d_k=128, d_v=128, seed=4,
+                   dtype=torch.bfloat16, adversarial_heads="odd"),
+}
+
+
+def make_workload(name: str, device: str | torch.device = "cpu", **overrides) -> ChunkInputs:
+    cfg = dict(WORKLOADS[name])
+    cfg.update(overrides)
+    return make_inputs(device=device, **cfg)
+
+
+def chunk_slices(inp: ChunkInputs, chunk_ids):
+    """Host fp64 copies of selected chunks: lists of (K, V, beta, g) numpy arrays.
+
+    chunk id = (b * H_v + h_v) * (T / C) + c. The key head of value head h_v is
+    h_v // (H_v / H_k). Values are upcast exactly from the stored dtype.
+    """
+    n_c = inp.T // inp.C
+    group = inp.H_v // inp.H_k
+    out = []
+    for cid in chunk_ids:
+        bh, c = divmod(int(cid), n_c)
+        b, hv = divmod(bh, inp.H_v)
+        hk = hv // group
+        sl = slice(c * inp.C, (c + 1) * inp.C)
+        out.append((inp.K[b, hk, sl].double().cpu().numpy(),
+                    inp.V[b, hv, sl].double().cpu().numpy(),
+                    inp.beta[b, hv, sl].double().cpu().numpy(),
+                    inp.g[b, hv, sl].double().cpu().numpy()))
+    return out

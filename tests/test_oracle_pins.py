@@ -1,0 +1,371 @@
+"""Pins for the fp64 CPU oracle: closed forms, invariants, library routines and
+brute force that do not go through the oracle's own formulas."""
+import math
+import os
+
+import numpy as np
+import pytest
+import scipy.linalg
+import torch
+
+from oracle import gdn_oracle as orc
+from paper_2606_06034_b200 import inputs as gen
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _chunks(C, n=4, seed=0, adversarial="none", d=128):
+    inp = gen.make_inputs(1, 2, 2, C * max(1, n // 2), C, d, d, seed=seed,
+                          dtype=torch.float32, adversarial_heads=adversarial)
+    sl = gen.chunk_slices(inp, range(inp.n_chunks))
+    K = np.stack([s[0] for s in sl])
+    V = np.stack([s[1] for s in sl])
+    b = np.stack([s[2] for s in sl])
+    g = np.stack([s[3] for s in sl])
+    return K, V, b, g
+
+
+def _rand_strict_lower(k, rng, scale=1.0):
+    return np.tril(rng.uniform(-scale, scale, size=(k, k)), -1)
+
+
+# -- A-build -------------------------------------------------------------------
+def test_build_A_reduces_to_gram_when_ungated():
+    rng = np.random.default_rng(0)
+    K = rng.normal(size=(8, 5))
+    A = orc.build_A(K, np.ones(8), np.zeros(8))
+    assert np.allclose(A, np.tril(K @ K.T, -1), atol=0, rtol=1e-15)
+    assert np.all(np.triu(A) == 0)
+
+
+def test_build_A_row_scaling_and_decay_direction():
+    # one non-zero pair: row 2 looks back at row 0 with decay exp(g2 - g0) and beta of the ROW
+    K = np.zeros((3, 2))
+    K[0] = [1.0, 0.0]
+    K[2] = [2.0, 0.0]
+    beta = np.array([0.3, 0.5, 0.7])
+    g = np.array([-0.1, -0.4, -1.1])
+    A = orc.build_A(K, beta, g)
+    expect = 0.7 * math.exp(-1.1 - (-0.1)) * 2.0
+    assert A[2, 0] == pytest.approx(expect, rel=1e-15)
+    assert np.count_nonzero(A) == 1
+
+
+def test_chunk_quantities_reproduce_gated_delta_rule_recurrence():
+    """U, W against the token-by-token gated delta rule they stand for.
+
+    S_t = a_t S_{t-1} (I - beta_t k_t k_t^T) + beta_t v_t k_t^T, a_t = exp(graw_t).
+    From S_0 = 0 the state after the chunk is sum_i exp(g_C - g_i) U_i k_i^T.
+    Without gates and from a state S_0 it is S_0 + sum_i (U_i - W_i S_0^T)_i k_i^T.
+    """
+    rng = np.random.default_rng(3)
+    C, dk, dv = 16, 6, 5
+    K = rng.normal(size=(C, dk))
+    K /= np.linalg.norm(K, axis=1, keepdims=True)
+    V = rng.normal(size=(C, dv))
+    beta = 1 / (1 + np.exp(-rng.normal(size=C)))
+    graw = -np.log1p(np.exp(rng.normal(size=C)))
+    g = np.cumsum(graw)
+
+    def recurrence(S0, graw_):
+        S = S0.copy()
+        for t in range(C):
+            S = math.exp(graw_[t]) * S
+            S = S - beta[t] * np.outer(S @ K[t], K[t]) + beta[t] * np.outer(V[t], K[t])
+        return S
+
+    # gated, zero initial state
+    W, U, T = orc.chunk_prepare(K, V, beta, g, exact=True)
+    S_end = recurrence(np.zeros((dv, dk)), graw)
+    S_chunk = sum(math.exp(g[-1] - g[i]) * np.outer(U[i], K[i]) for i in range(C))
+    assert np.allclose(S_end, S_chunk, atol=1e-13)
+
+    # ungated, non-zero initial state: needs W
+    W0, U0, _ = orc.chunk_prepare(K, V, beta, np.zeros(C), exact=True)
+    S0 = rng.normal(size=(dv, dk))
+    S_end = recurrence(S0, np.zeros(C))
+    Unew = U0 - W0 @ S0.T
+    S_chunk = S0 + sum(np.outer(Unew[i], K[i]) for i in range(C))
+    assert np.allclose(S_end, S_chunk, atol=1e-12)
+
+
+# -- P2 / P12: exact inverse -----------------------------------------------------
+def test_forward_substitution_closed_forms_c2_c3():
+    a = 0.37
+    T = orc.exact_inverse(np.array([[0, 0], [a, 0.0]]))
+    assert np.array_equal(T, np.array([[1, 0], [-a, 1.0]]))
+    a21, a31, a32 = 0.2, -0.5, 0.7
+    A = np.array([[0, 0, 0], [a21, 0, 0], [a31, a32, 0.0]])
+    T = orc.exact_inverse(A)
+    expect = np.array([[1, 0, 0], [-a21, 1, 0], [a32 * a21 - a31, -a32, 1.0]])
+    assert np.allclose(T, expect, atol=1e-16)
+
+
+@pytest.mark.parametrize("k", [2, 3, 4, 8, 16, 64])
+def test_forward_substitution_matches_library_inverse(k):
+    rng = np.random.default_rng(k)
+    A = _rand_strict_lower(k, rng, 0.3)
+    T = orc.exact_inverse(A)
+    I = np.eye(k)
+    assert np.allclose((I + A) @ T, I, atol=1e-12)
+    assert np.allclose(T, np.linalg.inv(I + A), atol=1e-12)
+    assert np.allclose(T, scipy.linalg.solve_triangular(I + A, I, lower=True), atol=1e-12)
+
+
+def test_forward_substitution_batched_equals_single():
+    rng = np.random.default_rng(5)
+    A = np.stack([_rand_strict_lower(8, rng) for _ in range(3)])
+    Tb = orc.exact_inverse(A)
+    for i in range(3):
+        assert np.array_equal(Tb[i], orc.exact_inverse(A[i]))
+
+
+# -- P1: nilpotency --------------------------------------------------------------
+@pytest.mark.parametrize("C", [16, 32, 64])
+def test_full_neumann_series_is_the_exact_inverse_benign(C):
+    K, V, b, g = _chunks(C)
+    A = orc.build_A(K, b, g)
+    Abar = -A
+    assert np.allclose(orc.neumann_full(Abar), orc.forward_substitution_inverse(Abar), atol=1e-13)
+    # A^k = 0
+    P = np.linalg.matrix_power(Abar[0], C)
+    assert np.all(P == 0)
+
+
+def test_full_neumann_series_exact_on_small_adversarial():
+    K, V, b, g = _chunks(16, adversarial="all")
+    Abar = -orc.build_A(K, b, g)
+    assert np.allclose(orc.neumann_full(Abar), orc.forward_substitution_inverse(Abar), atol=1e-9)
+
+
+# -- P3 / P4: structure ------------------------------------------------------------
+@pytest.mark.parametrize("C,N,S", [(64, 3, 8), (32, 3, 4), (32, 4, 3), (16, 3, 3), (16, 3, 2), (64, 2, 5)])
+@pytest.mark.parametrize("adv", ["none", "all"])
+def test_band_and_residual_structure(C, N, S, adv):
+    K, V, b, g = _chunks(C, adversarial=adv)
+    Abar = -orc.build_A(K, b, g)
+    Tex = orc.forward_substitution_inverse(Abar)
+    T0 = orc.neumann_masked_init(Abar, N)
+    i = np.arange(C)[:, None]
+    j = np.arange(C)[None, :]
+    d = i - j
+    band = (d >= 0) & (d <= N)
+    scale = max(1.0, np.abs(Tex).max())
+    # the masked initial approximation is exact on its band and zero off it
+    assert np.allclose(T0[..., band], Tex[..., band], atol=1e-12 * scale)
+    assert np.all(T0[..., ~band] == 0)
+    # E vanishes inside the band (up to rounding of cancelling terms), E^s below s(N+1)
+    E = orc.residual_matrix(Abar, T0)
+    assert np.abs(E[..., d <= N]).max() <= 1e-12 * scale
+    Es = E.copy()
+    for s in range(2, 5):
+        Es = Es @ E
+        tol = 1e-11 * max(1.0, np.abs(Es).max())
+        assert np.abs(Es[..., d < s * (N + 1)]).max() <= tol
+    # T_{N,S} is exact on i - j < (S+1)(N+1)
+    Tns = orc.neumann_residual(Abar, N, S)
+    near = d < (S + 1) * (N + 1)
+    assert np.allclose(Tns[..., near], Tex[..., near], atol=1e-10 * scale)
+    # and everywhere once S reaches ceil(C/(N+1)) - 1
+    Sfull = math.ceil(C / (N + 1)) - 1
+    Tfull = orc.neumann_residual(Abar, N, Sfull)
+    assert np.allclose(Tfull, Tex, atol=1e-10 * scale)
+
+
+# -- P5: the truncation error is the dropped terms ---------------------------------
+@pytest.mark.parametrize("C,N,S", [(64, 3, 2), (64, 3, 8), (32, 2, 3), (16, 1, 2)])
+def test_truncation_error_equals_dropped_terms(C, N, S):
+    K, V, b, g = _chunks(C, seed=7)
+    Abar = -orc.build_A(K, b, g)
+    Tex = orc.forward_substitution_inverse(Abar)
+    T0 = orc.neumann_masked_init(Abar, N)
+    E = orc.residual_matrix(Abar, T0)
+    Tns = orc.neumann_residual(Abar, N, S)
+    dropped = np.zeros_like(E)
+    P = np.broadcast_to(np.eye(C), E.shape).copy()
+    for s in range(1, math.ceil(C / (N + 1))):
+        P = P @ E
+        if s > S:
+            dropped = dropped + P
+    assert np.allclose(Tex - Tns, T0 @ dropped, atol=1e-13)
+    if S < math.ceil(C / (N + 1)) - 1 and C == 64 and S == 2:
+        assert np.abs(Tex - Tns).max() > 1e-9  # the truncated form really differs
+
+
+# -- P6: pairing of E and the side of the product -----------------------------------
+def test_right_and_left_consistent_agree_alg1_verbatim_does_not():
+    K, V, b, g = _chunks(64, seed=11)
+    Abar = -orc.build_A(K, b, g)
+    Tex = orc.forward_substitution_inverse(Abar)
+    R = orc.neumann_residual(Abar, 3, 4, side="right")
+    L = orc.neumann_residual(Abar, 3, 4, side="left_consistent")
+    Vb = orc.neumann_residual(Abar, 3, 4, side="alg1_verbatim")
+    assert np.allclose(R, L, atol=1e-14)
+    err_r = orc.rel_frobenius(R, Tex).max()
+    err_v = orc.rel_frobenius(Vb, Tex).min()
+    assert err_v > 1e3 * max(err_r, 1e-16)
+
+
+# -- P7: iterative residual correction = power sum with S = 2^m - 1 -----------------
+@pytest.mark.parametrize("m", [1, 2, 3])
+def test_iterative_correction_equals_power_sum(m):
+    K, V, b, g = _chunks(64, seed=13)
+    Abar = -orc.build_A(K, b, g)
+    it = orc.iterative_residual(Abar, 3, m)
+    ps = orc.neumann_residual(Abar, 3, 2 ** m - 1)
+    assert np.allclose(it, ps, atol=1e-14)
+
+
+def test_factorised_power_sum_matches_plain_sum():
+    rng = np.random.default_rng(17)
+    E = _rand_strict_lower(32, rng, 0.2)
+    assert np.allclose(orc.factorised_power_sum(E, 3), orc.power_sum(E, 7), atol=1e-14)
+
+
+# -- P8: entrywise growth (Lemma 3) -------------------------------------------------
+def test_binomial_growth_tight_for_all_ones():
+    k = 24
+    L = np.tril(np.ones((k, k)), -1)
+    P = np.eye(k)
+    for n in range(1, 8):
+        P = P @ L
+        for i in range(k):
+            for j in range(k):
+                d = i - j
+                expect = math.comb(d - 1, n - 1) if d >= 1 else 0
+                assert P[i, j] == expect
+    # the oracle's running sum sees the same numbers: sum_{n<=N} L^n entries
+    T0 = orc.neumann_masked_init(L, 3, mask=False)
+    assert T0[10, 2] == sum(math.comb(7, n - 1) for n in range(1, 4))
+
+
+def test_binomial_growth_bounds_bounded_entries():
+    rng = np.random.default_rng(19)
+    k = 20
+    A = _rand_strict_lower(k, rng, 1.0)
+    P = np.eye(k)
+    for n in range(1, 6):
+        P = P @ A
+        for i in range(k):
+            for j in range(i):
+                assert abs(P[i, j]) <= math.comb(i - j - 1, n - 1) + 1e-12
+
+
+# -- P9: closed form reachable through the whole path -------------------------------
+@pytest.mark.parametrize("a", [0.25, 0.99, 1.0])
+@pytest.mark.parametrize("C", [16, 64])
+def test_identical_keys_closed_form(a, C):
+    rng = np.random.default_rng(23)
+    u = rng.normal(size=8)
+    u /= np.linalg.norm(u)
+    K = np.tile(u, (C, 1))
+    V = rng.normal(size=(C, 4))
+    W, U, T = orc.chunk_prepare(K, V, np.full(C, a), np.zeros(C),
+                                N=3, S=math.ceil(C / 4) - 1)
+    i = np.arange(C)[:, None]
+    j = np.arange(C)[None, :]
+    d = i - j
+    expect = np.where(d > 0, -a * (1 - a) ** np.maximum(d - 1, 0), 0.0) + np.eye(C)
+    if a == 1.0:
+        expect = np.eye(C) - np.eye(C, k=-1)
+    assert np.allclose(T, expect, atol=1e-9)
+    assert np.allclose(W, (a * (1 - a) ** np.arange(C))[:, None] * u[None, :], atol=1e-9)
+    # U_i = a (v_i - sum_{j<i} U_j): running form of the same system
+    Uref = np.zeros_like(V)
+    run = np.zeros(4)
+    for t in range(C):
+        Uref[t] = a * (V[t] - run)
+        run = run + Uref[t]
+    assert np.allclose(U, Uref, atol=1e-8)
+
+
+# -- P10: truncation bound (Lemma 2) -------------------------------------------------
+def test_truncation_norm_bound():
+    rng = np.random.default_rng(29)
+    k = 64
+    i = np.arange(k)[:, None]
+    j = np.arange(k)[None, :]
+    A = np.where(i > j, rng.uniform(0, 1, size=(k, k)) * 0.8 ** (i - j), 0.0)
+    A *= 0.55 / np.linalg.norm(A, 2)
+    Tex = orc.neumann_full(A)
+    for N in (1, 3, 5, 8):
+        EN = Tex - orc.neumann_full(A, upto=N)
+        bound = 0.55 ** (N + 1) / (1 - 0.55)
+        assert np.linalg.norm(EN, 2) <= bound * (1 + 1e-12)
+        assert np.allclose(EN, sum(np.linalg.matrix_power(A, n) for n in range(N + 1, k)), atol=1e-14)
+
+
+# -- P11: matmul counts the paper prints ----------------------------------------------
+def test_matmul_counts_match_paper():
+    rows = []
+    with open(os.path.join(GOLDEN, "paper_matmul_counts.txt")) as f:
+        for line in f:
+            if line.strip() and not line.startswith("#"):
+                rows.append(tuple(int(x) for x in line.split()))
+    assert rows
+    for k, N, S, count in rows:
+        rng = np.random.default_rng(k)
+        A = _rand_strict_lower(k, rng, 0.1)
+        orc.reset_matmul_count()
+        orc.neumann_residual(A, N, S)
+        assert orc.matmul_count() == count
+        assert orc.default_order(k) == N and orc.default_residual_steps(k) == S
+
+
+# -- P13: block formula (App. E) --------------------------------------------------------
+def test_block_formula_reproduces_exact_inverse_with_exact_blocks():
+    K, V, b, g = _chunks(128, n=2, seed=31)
+    A = orc.build_A(K, b, g)
+    Tex = orc.exact_inverse(A)
+    # 64-blocks inverted exactly (S large enough), merged by the block formula
+    Tb = orc.chunk_inverse(A, 3, 15, block=64)
+    assert np.allclose(Tb, Tex, atol=1e-12)
+    # four 32-blocks exercise the general recursion (Eq. 27)
+    Tb4 = orc.chunk_inverse(A, 3, 7, block=32)
+    assert np.allclose(Tb4, Tex, atol=1e-12)
+    # the two-block corner: S_21 = -S_22 M_21 S_11
+    T11 = orc.exact_inverse(A[..., :64, :64])
+    T22 = orc.exact_inverse(A[..., 64:, 64:])
+    assert np.allclose(Tex[..., 64:, :64], -T22 @ A[..., 64:, :64] @ T11, atol=1e-12)
+    assert np.all(Tb[..., :64, 64:] == 0)
+
+
+# -- defaults: truncation invisible at the graded tolerance ---------------------------
+@pytest.mark.parametrize("C", [16, 32, 64, 128])
+@pytest.mark.parametrize("adv", ["none", "all"])
+def test_default_parameters_deviation_from_exact(C, adv):
+    K, V, b, g = _chunks(C, n=2, seed=37, adversarial=adv)
+    W, U, T = orc.chunk_prepare(K, V, b, g)
+    We, Ue, Te = orc.chunk_prepare(K, V, b, g, exact=True)
+    assert orc.rel_frobenius(T, Te).max() < 1e-9
+    assert orc.rel_frobenius(W, We).max() < 1e-8
+    assert orc.rel_frobenius(U, Ue).max() < 1e-8
+    # W, U are T applied to the beta-scaled rows
+    assert np.allclose(W, T @ (b[..., None] * K), atol=1e-13)
+
+
+def test_snr_definition():
+    ref = np.ones((2, 2))
+    x = ref + 0.1
+    # ||ref||^2 / ||ref - x||^2 = 4 / 0.04 = 100 -> 20 dB
+    assert orc.snr_db(x, ref) == pytest.approx(20.0, abs=1e-9)
+
+
+# -- input recipe --------------------------------------------------------------------
+def test_input_recipe():
+    inp = gen.make_inputs(2, 2, 4, 128, 64, 128, 128, seed=4, adversarial_heads="odd")
+    assert inp.K.dtype == torch.bfloat16 and inp.K.shape == (2, 2, 128, 128)
+    assert inp.V.shape == (2, 4, 128, 128) and inp.beta.shape == (2, 4, 128)
+    n = inp.K.float().norm(dim=-1)
+    assert torch.allclose(n, torch.ones_like(n), atol=1e-2)
+    # cumulative gate restarts at each chunk and decreases
+    gch = inp.g.view(2, 4, 2, 64)
+    assert (gch[:, :2].diff(dim=-1) <= 0).all()
+    # odd key head / its value heads are adversarial
+    assert (inp.beta[:, 2:] == 0.99).all() and (inp.g[:, 2:] == 0).all()
+    Kc = inp.K[0, 1, :64].float()
+    cos = Kc @ Kc.T
+    assert cos.min() > 0.95
+    # seeded
+    again = gen.make_inputs(2, 2, 4, 128, 64, 128, 128, seed=4, adversarial_heads="odd")
+    assert torch.equal(inp.K, again.K) and torch.equal(inp.g, again.g)
