@@ -1,0 +1,127 @@
+/*
+ * gdnprep - chunk preparation for chunk-wise Gated DeltaNet on NVIDIA B200 (sm_100a).
+ *
+ * For every chunk of C consecutive tokens of every (batch, head) this library
+ * builds the strictly lower-triangular matrix
+ *
+ *     A_ij = beta_i * exp(g_i - g_j) * <K_i, K_j>      (i > j, 0 otherwise),
+ *
+ * the "scaled inner product of the keys" of the paper's Sec. 2.1 with the Gated
+ * DeltaNet write strength beta and gate decay, and computes
+ *
+ *     T = (I + A)^-1,      W = T diag(beta) K,      U = T diag(beta) V.
+ *
+ * The paper writes the system as (I - A)^-1 (Eq. 1); its A is -A here.
+ *
+ * T is obtained with the paper's multiplication-only scheme (Sec. 3, Alg. 1):
+ * a Neumann series truncated at order N and masked to the band 0 <= i-j <= N
+ * (Eq. 7, 10, 11), followed by the parallel residual correction
+ * T = T0 * sum_{s=0..S} E^s with E = I - (I + A) T0 (Eq. 13). For C = 128 the
+ * two 64 x 64 diagonal blocks are inverted this way and the lower-left block
+ * follows from the block formula of App. E (Eq. 28).
+ *
+ * Common conventions
+ *   - Every pointer is a DEVICE pointer owned by the caller. The library
+ *     allocates no device memory for the caller's data, never synchronises
+ *     (except gdn_device_status) and enqueues its work on `stream`.
+ *   - Layouts are contiguous:  K [B, H_k, T, d_k],  V [B, H_v, T, d_v],
+ *     beta, g [B, H_v, T] (fp32),  W [B, H_v, T, d_k],  U [B, H_v, T, d_v],
+ *     Tinv [B, H_v, T/C, C, C] (the full matrix, unit diagonal included, zeros
+ *     above it). K, V, W, U, Tinv have the element type selected by `dtype`.
+ *   - g is the CUMULATIVE log-gate. Only differences inside a chunk are used,
+ *     so a chunk-local or a global prefix sum give the same result.
+ *   - Value head h reads key head h / (H_v / H_k); H_v must be a multiple of H_k.
+ *   - order = N >= 1 and residual_steps = S >= 0; -1 selects the paper's value
+ *     for the chunk size (gdn_default_order, gdn_default_residual_steps).
+ *   - Return value: GDN_OK or a negative gdn_status. On any error nothing is
+ *     launched. No exception crosses this boundary.
+ *   - Pointers must be 16-byte aligned; T must be a multiple of C.
+ *   - The device must be compute capability 10.x (B200); anything else gives
+ *     GDN_ERR_ARCH. There is no CPU fallback.
+ */
+#ifndef GDNPREP_H_
+#define GDNPREP_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    GDN_OK = 0,
+    GDN_ERR_INVALID_ARG = -1, /* a size or parameter is out of range (e.g. T % C != 0, order < 1) */
+    GDN_ERR_UNSUPPORTED = -2, /* valid in principle, not implemented by the kernels (e.g. d_k = 96) */
+    GDN_ERR_NULL = -3,        /* a required pointer is NULL */
+    GDN_ERR_ALIGN = -4,       /* a pointer is not 16-byte aligned */
+    GDN_ERR_LAUNCH = -5,      /* the CUDA runtime refused the launch or a set-up call */
+    GDN_ERR_TIMEOUT = -6,     /* a bounded wait inside a kernel ran out (reported by gdn_device_status) */
+    GDN_ERR_ARCH = -7         /* the current device is not sm_100 */
+} gdn_status;
+
+enum { GDN_DTYPE_FP32 = 0, GDN_DTYPE_BF16 = 1 };
+
+/* variants of the forward-substitution comparison kernel */
+enum { GDN_FWDSUBST_ROWS = 0, GDN_FWDSUBST_BLOCKED = 1 };
+
+/* A CUDA stream handle (cudaStream_t) passed as an opaque pointer. */
+typedef void* gdn_stream_t;
+
+/*
+ * The hot path (Sec. 3, Alg. 1, Eq. 7-13; App. E for C = 128): A-build, masked
+ * truncated Neumann series, residual power sum, W and U.
+ *   dtype GDN_DTYPE_BF16: bf16 K, V, W, U, Tinv; tensor-core kernel; C in {16, 32, 64, 128},
+ *                         d_k, d_v = 128, 1 <= order <= 7. fp32 accumulation.
+ *   dtype GDN_DTYPE_FP32: fp32 everywhere, plain FMA kernel; 2 <= C <= 128, d_k, d_v <= 256.
+ * Tinv_out may be NULL (the store is skipped). H = H_k = H_v.
+ */
+int gdn_chunk_prepare(const void* K, const void* V, const float* beta, const float* g,
+                      int B, int H, int T, int C, int d_k, int d_v,
+                      int order, int residual_steps, int dtype,
+                      void* W_out, void* U_out, void* Tinv_out, gdn_stream_t stream);
+
+/*
+ * Same operation with grouped heads: H_k key heads shared by H_v value heads
+ * (beta, g, W, U, Tinv are per value head; only K is shared).
+ */
+int gdn_chunk_prepare_gqa(const void* K, const void* V, const float* beta, const float* g,
+                          int B, int H_k, int H_v, int T, int C, int d_k, int d_v,
+                          int order, int residual_steps, int dtype,
+                          void* W_out, void* U_out, void* Tinv_out, gdn_stream_t stream);
+
+/*
+ * The comparison the paper's speed-up is measured against: the same A-build, W
+ * and U, with T computed exactly by forward substitution (Eq. 2-3;
+ * variant GDN_FWDSUBST_ROWS) or by 16 x 16 diagonal blocks merged with the
+ * block recursion of App. E (Eq. 25-27; variant GDN_FWDSUBST_BLOCKED).
+ */
+int gdn_chunk_prepare_fwdsubst(const void* K, const void* V, const float* beta, const float* g,
+                               int B, int H_k, int H_v, int T, int C, int d_k, int d_v,
+                               int dtype, int variant,
+                               void* W_out, void* U_out, void* Tinv_out, gdn_stream_t stream);
+
+/*
+ * Waits for `stream`, then returns and clears the status word the kernels of
+ * this library write on the current device: GDN_OK, or GDN_ERR_TIMEOUT when a
+ * bounded wait inside a kernel gave up (its outputs are then undefined).
+ * This is the only call that synchronises.
+ */
+int gdn_device_status(gdn_stream_t stream);
+
+/* Paper's parameters per chunk size: N = 3; S = 8 for C = 64 (Sec. 4.1) and for the
+ * 64-blocks of C = 128 (App. H), S = 4 for C = 32 (Sec. 4.3); C = 16 is not in the
+ * paper: S = 3, which makes the result exact. Other C: S = ceil(C/4) - 1. */
+int gdn_default_order(int C);
+int gdn_default_residual_steps(int C);
+
+/* Human-readable name of a gdn_status value (static storage). */
+const char* gdn_status_string(int status);
+
+/* Number of kernels this library has launched in this process (for benchmarks that
+ * must report how many of the library's own kernels ran inside a timed region). */
+long long gdn_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GDNPREP_H_ */

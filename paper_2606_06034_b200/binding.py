@@ -1,0 +1,185 @@
+"""Python binding of the C-ABI library `libgdnprep.so` (argument marshalling only).
+
+Every function has the name and the argument order of its C entry point in
+`include/gdnprep.h`; tensors are passed as raw device pointers on torch's
+current CUDA stream. All arithmetic runs inside the library's CUDA kernels; if
+the library is missing the import of a function raises, there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libgdnprep.so")
+
+GDN_OK = 0
+GDN_ERR_INVALID_ARG = -1
+GDN_ERR_UNSUPPORTED = -2
+GDN_ERR_NULL = -3
+GDN_ERR_ALIGN = -4
+GDN_ERR_LAUNCH = -5
+GDN_ERR_TIMEOUT = -6
+GDN_ERR_ARCH = -7
+GDN_DTYPE_FP32 = 0
+GDN_DTYPE_BF16 = 1
+GDN_FWDSUBST_ROWS = 0
+GDN_FWDSUBST_BLOCKED = 1
+
+EXPORTS = (
+    "gdn_chunk_prepare", "gdn_chunk_prepare_gqa", "gdn_chunk_prepare_fwdsubst",
+    "gdn_device_status", "gdn_default_order", "gdn_default_residual_steps",
+    "gdn_status_string", "gdn_launch_count",
+)
+
+_lib = None
+
+
+class GdnError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+def load_library() -> ctypes.CDLL:
+    """Loads the shared library (built in-tree by `paper_2606_06034_b200.build`)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise FileNotFoundError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2606_06034_b200.build` "
+            "(the CUDA path has no fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, ip = ctypes.c_void_p, ctypes.c_int
+    lib.gdn_chunk_prepare.restype = ip
+    lib.gdn_chunk_prepare.argtypes = [vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ip, ip, ip, vp, vp, vp, vp]
+    lib.gdn_chunk_prepare_gqa.restype = ip
+    lib.gdn_chunk_prepare_gqa.argtypes = [vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ip, ip, ip, ip, vp, vp, vp, vp]
+    lib.gdn_chunk_prepare_fwdsubst.restype = ip
+    lib.gdn_chunk_prepare_fwdsubst.argtypes = [vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ip, ip, ip, vp, vp, vp, vp]
+    lib.gdn_device_status.restype = ip
+    lib.gdn_device_status.argtypes = [vp]
+    lib.gdn_default_order.restype = ip
+    lib.gdn_default_order.argtypes = [ip]
+    lib.gdn_default_residual_steps.restype = ip
+    lib.gdn_default_residual_steps.argtypes = [ip]
+    lib.gdn_status_string.restype = ctypes.c_char_p
+    lib.gdn_status_string.argtypes = [ip]
+    lib.gdn_launch_count.restype = ctypes.c_longlong
+    lib.gdn_launch_count.argtypes = []
+    _lib = lib
+    return lib
+
+
+def status_string(status: int) -> str:
+    return load_library().gdn_status_string(int(status)).decode()
+
+
+def gdn_default_order(C: int) -> int:
+    return load_library().gdn_default_order(int(C))
+
+
+def gdn_default_residual_steps(C: int) -> int:
+    return load_library().gdn_default_residual_steps(int(C))
+
+
+def gdn_launch_count() -> int:
+    return int(load_library().gdn_launch_count())
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return GDN_DTYPE_FP32
+    if t.dtype == torch.bfloat16:
+        return GDN_DTYPE_BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check_inputs(K, V, beta, g, outs):
+    for t in (K, V, beta, g, *[o for o in outs if o is not None]):
+        if not t.is_cuda:
+            raise ValueError("all tensors must live on a CUDA device (there is no CPU path)")
+        if not t.is_contiguous():
+            raise ValueError("all tensors must be contiguous")
+    if V.dtype != K.dtype or beta.dtype != torch.float32 or g.dtype != torch.float32:
+        raise TypeError("K and V share a dtype; beta and g are fp32")
+
+
+def alloc_outputs(K, V, C, want_tinv=True):
+    """Allocates W [B,H_v,T,d_k], U [B,H_v,T,d_v], Tinv [B,H_v,T/C,C,C] with torch."""
+    B, H_v, T, d_v = V.shape
+    d_k = K.shape[-1]
+    W = torch.empty(B, H_v, T, d_k, dtype=K.dtype, device=K.device)
+    U = torch.empty(B, H_v, T, d_v, dtype=K.dtype, device=K.device)
+    Tinv = torch.empty(B, H_v, T // C, C, C, dtype=K.dtype, device=K.device) if want_tinv else None
+    return W, U, Tinv
+
+
+def gdn_chunk_prepare(K, V, beta, g, B, H, T, C, d_k, d_v, order, residual_steps, dtype, W_out, U_out, Tinv_out,
+                      *, check=True):
+    """Raw call (same argument list as the C function, tensors instead of pointers)."""
+    _check_inputs(K, V, beta, g, (W_out, U_out, Tinv_out))
+    rc = load_library().gdn_chunk_prepare(_ptr(K), _ptr(V), _ptr(beta), _ptr(g), B, H, T, C, d_k, d_v, order,
+                                          residual_steps, dtype, _ptr(W_out), _ptr(U_out), _ptr(Tinv_out), _stream())
+    if check and rc != GDN_OK:
+        raise GdnError(rc, "gdn_chunk_prepare")
+    return rc
+
+
+def gdn_chunk_prepare_gqa(K, V, beta, g, B, H_k, H_v, T, C, d_k, d_v, order, residual_steps, dtype, W_out, U_out,
+                          Tinv_out, *, check=True):
+    _check_inputs(K, V, beta, g, (W_out, U_out, Tinv_out))
+    rc = load_library().gdn_chunk_prepare_gqa(_ptr(K), _ptr(V), _ptr(beta), _ptr(g), B, H_k, H_v, T, C, d_k, d_v,
+                                              order, residual_steps, dtype, _ptr(W_out), _ptr(U_out), _ptr(Tinv_out),
+                                              _stream())
+    if check and rc != GDN_OK:
+        raise GdnError(rc, "gdn_chunk_prepare_gqa")
+    return rc
+
+
+def gdn_chunk_prepare_fwdsubst(K, V, beta, g, B, H_k, H_v, T, C, d_k, d_v, dtype, variant, W_out, U_out, Tinv_out,
+                               *, check=True):
+    _check_inputs(K, V, beta, g, (W_out, U_out, Tinv_out))
+    rc = load_library().gdn_chunk_prepare_fwdsubst(_ptr(K), _ptr(V), _ptr(beta), _ptr(g), B, H_k, H_v, T, C, d_k,
+                                                   d_v, dtype, variant, _ptr(W_out), _ptr(U_out), _ptr(Tinv_out),
+                                                   _stream())
+    if check and rc != GDN_OK:
+        raise GdnError(rc, "gdn_chunk_prepare_fwdsubst")
+    return rc
+
+
+def gdn_device_status() -> int:
+    """Synchronises torch's current stream and returns (and clears) the kernels' status word."""
+    return load_library().gdn_device_status(_stream())
+
+
+def chunk_prepare(K, V, beta, g, C, order=-1, residual_steps=-1, *, want_tinv=True, outputs=None,
+                  method="neumann", variant=GDN_FWDSUBST_ROWS):
+    """Convenience wrapper: shapes from the tensors, outputs allocated with torch.
+
+    K [B,H_k,T,d_k], V [B,H_v,T,d_v], beta, g [B,H_v,T]. Returns (W, U, Tinv).
+    """
+    B, H_k, T, d_k = K.shape
+    _, H_v, _, d_v = V.shape
+    if outputs is None:
+        outputs = alloc_outputs(K, V, C, want_tinv)
+    W, U, Tinv = outputs
+    dt = _dtype_code(K)
+    if method == "neumann":
+        gdn_chunk_prepare_gqa(K, V, beta, g, B, H_k, H_v, T, C, d_k, d_v, order, residual_steps, dt, W, U, Tinv)
+    elif method == "fwdsubst":
+        gdn_chunk_prepare_fwdsubst(K, V, beta, g, B, H_k, H_v, T, C, d_k, d_v, dt, variant, W, U, Tinv)
+    else:
+        raise ValueError(method)
+    return W, U, Tinv

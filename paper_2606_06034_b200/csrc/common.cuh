@@ -1,0 +1,36 @@
+// Shared declarations of the library's translation units (host side).
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+
+#include "../../include/gdnprep.h"
+
+namespace gdn {
+
+// Problem description shared by all kernels.
+struct Problem {
+    const void* K;
+    const void* V;
+    const float* beta;
+    const float* g;
+    void* W;
+    void* U;
+    void* Tinv;  // may be null
+    int B, H_k, H_v, T, C, d_k, d_v;
+    int order;   // N
+    int steps;   // S
+    int dtype;   // GDN_DTYPE_*
+};
+
+enum InverseMode { INV_NEUMANN = 0, INV_FWDSUBST_ROWS = 1, INV_FWDSUBST_BLOCKED = 2 };
+
+// Status word written by kernels (one per device, static device memory).
+int* device_status_word();  // device address for the current device (nullptr on failure)
+void count_launch();
+
+// Kernel launchers. Each returns a gdn_status and launches on `stream`.
+int launch_simt(const Problem& p, InverseMode mode, cudaStream_t stream);
+int launch_tc_bf16(const Problem& p, InverseMode mode, cudaStream_t stream);
+
+}  // namespace gdn

@@ -1,0 +1,167 @@
+// C-ABI entry points: argument validation, kernel selection, status word.
+#include <atomic>
+#include <cstdint>
+
+#include "common.cuh"
+
+namespace gdn {
+
+// One status word per device that loads this library; kernels write GDN_ERR_TIMEOUT here
+// when a bounded wait gives up.
+__device__ int g_status_word = 0;
+
+namespace {
+std::atomic<long long> g_launches{0};
+constexpr int kMaxDevices = 64;
+int* g_status_addr[kMaxDevices] = {nullptr};
+int g_arch_ok[kMaxDevices] = {0};  // 0 unknown, 1 yes, -1 no
+}  // namespace
+
+void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+
+int* device_status_word() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    if (g_status_addr[dev] == nullptr) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_status_word) != cudaSuccess) return nullptr;
+        g_status_addr[dev] = static_cast<int*>(ptr);
+    }
+    return g_status_addr[dev];
+}
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_arch() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        cudaGetLastError();
+        return GDN_ERR_ARCH;
+    }
+    if (g_arch_ok[dev] == 0) {
+        int major = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
+            cudaGetLastError();
+            return GDN_ERR_ARCH;
+        }
+        g_arch_ok[dev] = (major == 10) ? 1 : -1;
+    }
+    return g_arch_ok[dev] == 1 ? GDN_OK : GDN_ERR_ARCH;
+}
+
+// Validation shared by every entry point. Order: NULL, sizes, alignment, architecture.
+int validate(const Problem& p, bool neumann) {
+    if (p.K == nullptr || p.V == nullptr || p.beta == nullptr || p.g == nullptr || p.W == nullptr || p.U == nullptr)
+        return GDN_ERR_NULL;
+    if (p.B < 0 || p.H_k <= 0 || p.H_v <= 0 || p.T < 0 || p.C < 2 || p.d_k <= 0 || p.d_v <= 0) return GDN_ERR_INVALID_ARG;
+    if (p.H_v % p.H_k != 0) return GDN_ERR_INVALID_ARG;
+    if (p.T % p.C != 0) return GDN_ERR_INVALID_ARG;
+    if (p.dtype != GDN_DTYPE_FP32 && p.dtype != GDN_DTYPE_BF16) return GDN_ERR_INVALID_ARG;
+    if (neumann) {
+        const int blk = (p.C == 128) ? 64 : p.C;
+        if (p.order < 1 || p.order >= blk || p.steps < 0) return GDN_ERR_INVALID_ARG;
+    }
+    if (p.C > 128) return GDN_ERR_UNSUPPORTED;
+    if (p.d_k % 8 != 0 || p.d_v % 8 != 0) return GDN_ERR_UNSUPPORTED;
+    if (!aligned16(p.K) || !aligned16(p.V) || !aligned16(p.beta) || !aligned16(p.g) || !aligned16(p.W) || !aligned16(p.U) ||
+        !aligned16(p.Tinv))
+        return GDN_ERR_ALIGN;
+    return GDN_OK;
+}
+
+int run(Problem p, InverseMode mode, cudaStream_t stream) {
+    const bool neumann = (mode == INV_NEUMANN);
+    if (neumann) {
+        if (p.order == -1) p.order = gdn_default_order(p.C);
+        if (p.steps == -1) p.steps = gdn_default_residual_steps(p.C);
+    }
+    int rc = validate(p, neumann);
+    if (rc != GDN_OK) return rc;
+    rc = check_arch();
+    if (rc != GDN_OK) return rc;
+    if (p.dtype == GDN_DTYPE_FP32) return launch_simt(p, mode, stream);
+    return launch_tc_bf16(p, mode, stream);
+}
+
+}  // namespace
+}  // namespace gdn
+
+using namespace gdn;
+
+extern "C" {
+
+int gdn_chunk_prepare(const void* K, const void* V, const float* beta, const float* g, int B, int H, int T, int C, int d_k,
+                      int d_v, int order, int residual_steps, int dtype, void* W_out, void* U_out, void* Tinv_out,
+                      gdn_stream_t stream) {
+    Problem p{K, V, beta, g, W_out, U_out, Tinv_out, B, H, H, T, C, d_k, d_v, order, residual_steps, dtype};
+    return run(p, INV_NEUMANN, static_cast<cudaStream_t>(stream));
+}
+
+int gdn_chunk_prepare_gqa(const void* K, const void* V, const float* beta, const float* g, int B, int H_k, int H_v, int T, int C,
+                          int d_k, int d_v, int order, int residual_steps, int dtype, void* W_out, void* U_out, void* Tinv_out,
+                          gdn_stream_t stream) {
+    Problem p{K, V, beta, g, W_out, U_out, Tinv_out, B, H_k, H_v, T, C, d_k, d_v, order, residual_steps, dtype};
+    return run(p, INV_NEUMANN, static_cast<cudaStream_t>(stream));
+}
+
+int gdn_chunk_prepare_fwdsubst(const void* K, const void* V, const float* beta, const float* g, int B, int H_k, int H_v, int T,
+                               int C, int d_k, int d_v, int dtype, int variant, void* W_out, void* U_out, void* Tinv_out,
+                               gdn_stream_t stream) {
+    if (variant != GDN_FWDSUBST_ROWS && variant != GDN_FWDSUBST_BLOCKED) return GDN_ERR_INVALID_ARG;
+    Problem p{K, V, beta, g, W_out, U_out, Tinv_out, B, H_k, H_v, T, C, d_k, d_v, 0, 0, dtype};
+    return run(p, variant == GDN_FWDSUBST_ROWS ? INV_FWDSUBST_ROWS : INV_FWDSUBST_BLOCKED, static_cast<cudaStream_t>(stream));
+}
+
+int gdn_device_status(gdn_stream_t stream) {
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+        cudaGetLastError();
+        return GDN_ERR_LAUNCH;
+    }
+    int* addr = device_status_word();
+    if (addr == nullptr) return GDN_ERR_LAUNCH;
+    int value = 0;
+    if (cudaMemcpy(&value, addr, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return GDN_ERR_LAUNCH;
+    if (value != 0) {
+        const int zero = 0;
+        if (cudaMemcpy(addr, &zero, sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) return GDN_ERR_LAUNCH;
+    }
+    return value;
+}
+
+int gdn_default_order(int C) {
+    (void)C;
+    return 3;
+}
+
+int gdn_default_residual_steps(int C) {
+    switch (C) {
+        case 16: return 3;
+        case 32: return 4;
+        case 64: return 8;
+        case 128: return 8;
+        default: {
+            const int s = (C + 3) / 4 - 1;
+            return s < 0 ? 0 : s;
+        }
+    }
+}
+
+const char* gdn_status_string(int status) {
+    switch (status) {
+        case GDN_OK: return "ok";
+        case GDN_ERR_INVALID_ARG: return "invalid argument";
+        case GDN_ERR_UNSUPPORTED: return "unsupported configuration";
+        case GDN_ERR_NULL: return "null pointer";
+        case GDN_ERR_ALIGN: return "pointer not 16-byte aligned";
+        case GDN_ERR_LAUNCH: return "CUDA launch or set-up failed";
+        case GDN_ERR_TIMEOUT: return "bounded wait inside a kernel ran out";
+        case GDN_ERR_ARCH: return "device is not sm_100";
+        default: return "unknown status";
+    }
+}
+
+long long gdn_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

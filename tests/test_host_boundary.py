@@ -1,0 +1,81 @@
+"""Host-side checks that need no GPU: the library loads, exports what the header declares,
+and rejects bad arguments before touching the device."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2606_06034_b200 import binding as gdn
+from paper_2606_06034_b200 import build as gdn_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    gdn_build.build()
+    return gdn.load_library()
+
+
+def _declared_functions():
+    text = open(os.path.join(ROOT, "include", "gdnprep.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(gdn_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol(lib):
+    names = _declared_functions()
+    assert "gdn_chunk_prepare" in names and "gdn_device_status" in names
+    for name in names:
+        assert hasattr(lib, name), name
+    assert set(names) == set(gdn.EXPORTS)
+
+
+def test_defaults_follow_the_paper(lib):
+    assert [lib.gdn_default_order(c) for c in (16, 32, 64, 128)] == [3, 3, 3, 3]
+    assert [lib.gdn_default_residual_steps(c) for c in (16, 32, 64, 128)] == [3, 4, 8, 8]
+
+
+def test_status_strings(lib):
+    for code in range(0, -8, -1):
+        assert lib.gdn_status_string(code)
+    assert gdn.status_string(gdn.GDN_ERR_TIMEOUT).startswith("bounded wait")
+
+
+def test_bad_arguments_are_rejected_without_a_device(lib):
+    buf = ctypes.create_string_buffer(4096)
+    base = ctypes.addressof(buf)
+    base += (-base) % 16
+    p = ctypes.c_void_p(base)
+    mis = ctypes.c_void_p(base + 4)
+
+    def call(K=p, V=p, beta=p, g=p, B=1, H=1, T=128, C=64, dk=128, dv=128, N=-1, S=-1, dt=1, W=p, U=p, Ti=p):
+        return lib.gdn_chunk_prepare(K, V, beta, g, B, H, T, C, dk, dv, N, S, dt, W, U, Ti, None)
+
+    assert call(K=None) == gdn.GDN_ERR_NULL
+    assert call(W=None) == gdn.GDN_ERR_NULL
+    assert call(T=100) == gdn.GDN_ERR_INVALID_ARG
+    assert call(C=1, T=128) == gdn.GDN_ERR_INVALID_ARG
+    assert call(N=0) == gdn.GDN_ERR_INVALID_ARG
+    assert call(N=64) == gdn.GDN_ERR_INVALID_ARG
+    assert call(S=-2) == gdn.GDN_ERR_INVALID_ARG
+    assert call(dt=7) == gdn.GDN_ERR_INVALID_ARG
+    assert call(C=256, T=256) == gdn.GDN_ERR_UNSUPPORTED
+    assert call(g=mis) == gdn.GDN_ERR_ALIGN
+    assert call(Ti=mis) == gdn.GDN_ERR_ALIGN
+    assert lib.gdn_chunk_prepare_gqa(p, p, p, p, 1, 2, 3, 128, 64, 128, 128, -1, -1, 1, p, p, p, None) == gdn.GDN_ERR_INVALID_ARG
+    assert lib.gdn_chunk_prepare_fwdsubst(p, p, p, p, 1, 1, 1, 128, 64, 128, 128, 1, 5, p, p, p, None) == gdn.GDN_ERR_INVALID_ARG
+    # valid arguments but no sm_100 device in this process: refused, nothing launched
+    import torch
+    if not torch.cuda.is_available():
+        assert call() == gdn.GDN_ERR_ARCH
+        assert lib.gdn_launch_count() == 0
+
+
+def test_binding_refuses_host_tensors():
+    import torch
+    K = torch.zeros(1, 1, 64, 128, dtype=torch.bfloat16)
+    b = torch.zeros(1, 1, 64)
+    with pytest.raises(ValueError):
+        gdn.chunk_prepare(K, K, b, b, 64)
