@@ -88,6 +88,80 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity) {
     return true;
 }
 
+
+// Writes this row's packed bf16 diagonal block (C / 2 32-bit columns) into the A-operand slot.
+// tcgen05.st takes one address per warp: for C = 16 a warp holds two chunks, so the warp stores a
+// 16-column window in which each half-warp fills its own half and zero-fills the other.
+template <int C>
+__device__ __forceinline__ void store_a_operand(uint32_t lane_base, int t, const uint32_t (&pk)[C / 2]) {
+    constexpr int PC = C / 2;
+    if constexpr (PC >= 16) {
+        const int cb = t - (t % C);
+#pragma unroll
+        for (int c = 0; c < PC / 16; ++c) {
+            uint32_t r16[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) r16[i] = pk[c * 16 + i];
+            tmem_st16(lane_base + kAS + cb / 2 + c * 16, r16);
+        }
+    } else {
+        const int wb = t & ~31;
+        const bool upper = (t & 16) != 0;
+        uint32_t r16[16];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            r16[i] = upper ? 0u : pk[i];
+            r16[8 + i] = upper ? pk[i] : 0u;
+        }
+        tmem_st16(lane_base + kAS + wb / 2, r16);
+    }
+}
+
+// Reads this row's C columns of a block-diagonal 128-column accumulator (the Gram matrix).
+template <int C>
+__device__ __forceinline__ void load_diag_block(uint32_t lane_base, uint32_t col0, int t, float (&a)[C]) {
+    if constexpr (C >= 32) {
+        const int cb = t - (t % C);
+#pragma unroll
+        for (int c0 = 0; c0 < C; c0 += 32) {
+            uint32_t r[32];
+            tmem_ld32(lane_base + col0 + cb + c0, r);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) a[c0 + i] = __uint_as_float(r[i]);
+        }
+    } else {
+        const int wb = t & ~31;
+        const bool upper = (t & 16) != 0;
+        uint32_t r[32];
+        tmem_ld32(lane_base + col0 + wb, r);
+        tmem_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 16; ++i) a[i] = __uint_as_float(upper ? r[16 + i] : r[i]);
+    }
+}
+
+// Reads C consecutive accumulator columns starting at col0 (same address for the whole warp).
+template <int C>
+__device__ __forceinline__ void load_cols(uint32_t lane_base, uint32_t col0, uint32_t (&r)[C]) {
+    if constexpr (C >= 32) {
+#pragma unroll
+        for (int c0 = 0; c0 < C; c0 += 32) {
+            uint32_t q[32];
+            tmem_ld32(lane_base + col0 + c0, q);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) r[c0 + i] = q[i];
+        }
+    } else {
+        uint32_t q[16];
+        tmem_ld16(lane_base + col0, q);
+        tmem_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 16; ++i) r[i] = q[i];
+    }
+}
+
 template <int C, int NB, int MODE>
 __global__ void __launch_bounds__(kThreads, 2)
 chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const Params p) {
@@ -129,6 +203,8 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     const uint32_t tmem = tmem_base_s;
 
     const int N = p.N, S = p.S;
+    // width of the band kept in fp32 registers (lb[]): the order N, or all of NB for forward substitution
+    const int n_band = (MODE == INV_NEUMANN) ? N : NB;
     // number of MMA rounds between the A-build and the W/U products
     const int n_rounds = (MODE == INV_NEUMANN) ? (S >= 1 ? S : 0) : 0;
 
@@ -269,25 +345,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             par_mma ^= 1;
             tc_fence_after_sync();
             float a[C];
-            {
-                constexpr int CH = (C >= 32) ? 32 : 16;
-#pragma unroll
-                for (int c0 = 0; c0 < C; c0 += CH) {
-                    if constexpr (CH == 32) {
-                        uint32_t r[32];
-                        tmem_ld32(lane_base + kR0 + cb + c0, r);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) a[c0 + i] = __uint_as_float(r[i]);
-                    } else {
-                        uint32_t r[16];
-                        tmem_ld16(lane_base + kR0 + cb + c0, r);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) a[c0 + i] = __uint_as_float(r[i]);
-                    }
-                }
-            }
+            load_diag_block<C>(lane_base, kR0, t, a);
             float ab[NB + 1];  // ab[e] = Abar[i][i-e]
 #pragma unroll
             for (int e = 0; e <= NB; ++e) ab[e] = 0.f;
@@ -410,20 +468,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                             }
                             pk[jp] = pack_bf16x2(lo, hi);
                         }
-                        if constexpr (PC >= 16) {
-#pragma unroll
-                            for (int c = 0; c < PC / 16; ++c) {
-                                uint32_t r16[16];
-#pragma unroll
-                                for (int i = 0; i < 16; ++i) r16[i] = pk[c * 16 + i];
-                                tmem_st16(lane_base + kAS + cb / 2 + c * 16, r16);
-                            }
-                        } else {
-                            uint32_t r8[8];
-#pragma unroll
-                            for (int i = 0; i < 8; ++i) r8[i] = pk[i];
-                            tmem_st8(lane_base + kAS + cb / 2, r8);
-                        }
+                        store_a_operand<C>(lane_base, t, pk);
                     }
                     fence_proxy_async_smem();
                     tmem_wait_st();
@@ -433,25 +478,10 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     par_mma ^= 1;
                     tc_fence_after_sync();
                     const uint32_t dcol = (k < S) ? kR2 : kR0;
-                    constexpr int CH = (C >= 32) ? 32 : 16;
+                    uint32_t dres[C];
+                    load_cols<C>(lane_base, dcol, dres);
 #pragma unroll
-                    for (int c0 = 0; c0 < C; c0 += CH) {
-                        if constexpr (CH == 32) {
-                            uint32_t r[32];
-                            tmem_ld32(lane_base + dcol + c0, r);
-                            tmem_wait_ld();
-#pragma unroll
-                            for (int i = 0; i < 32; ++i)
-                                x[c0 + i] = ((k < S) ? a[c0 + i] : x[c0 + i]) + __uint_as_float(r[i]);
-                        } else {
-                            uint32_t r[16];
-                            tmem_ld16(lane_base + dcol + c0, r);
-                            tmem_wait_ld();
-#pragma unroll
-                            for (int i = 0; i < 16; ++i)
-                                x[c0 + i] = ((k < S) ? a[c0 + i] : x[c0 + i]) + __uint_as_float(r[i]);
-                        }
-                    }
+                    for (int i = 0; i < C; ++i) x[i] = ((k < S) ? a[i] : x[i]) + __uint_as_float(dres[i]);
                 }
                 if (!ok) break;
                 // x[] = far row. Move into a[] for the common tail.
@@ -501,7 +531,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                         if (j == il) val = 1.f;
 #pragma unroll
                         for (int e = 1; e <= NB; ++e)
-                            if (j == il - e) val = lb[e];
+                            if (j == il - e && e <= n_band) val = lb[e];
                         v[q] = val;
                     }
                     uint4 o;
@@ -523,20 +553,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     const float2 bb = sb2[jp];
                     pk[jp] = pack_bf16x2(a[2 * jp] * bb.x, a[2 * jp + 1] * bb.y);
                 }
-                if constexpr (PC >= 16) {
-#pragma unroll
-                    for (int c = 0; c < PC / 16; ++c) {
-                        uint32_t r16[16];
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) r16[i] = pk[c * 16 + i];
-                        tmem_st16(lane_base + kAS + cb / 2 + c * 16, r16);
-                    }
-                } else {
-                    uint32_t r8[8];
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) r8[i] = pk[i];
-                    tmem_st8(lane_base + kAS + cb / 2, r8);
-                }
+                store_a_operand<C>(lane_base, t, pk);
                 tmem_wait_st();
                 tc_fence_before_sync();
                 mbar_arrive(&bar_opnd);

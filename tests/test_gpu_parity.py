@@ -25,6 +25,10 @@ def _oracle(inp, N=None, S=None, exact=False, chunk_ids=None):
     return orc.chunk_prepare(K, V, b, g, N, S, exact=exact)
 
 
+def _bf16_round(x):
+    return torch.from_numpy(np.ascontiguousarray(x)).to(torch.bfloat16).double().numpy()
+
+
 def _gpu_chunks(W, U, Tinv, inp, chunk_ids=None):
     C = inp.C
     n = inp.n_chunks
@@ -42,9 +46,16 @@ def _check(inp, tol, N=-1, S=-1, method="neumann", exact=False, chunk_ids=None):
     Wg, Ug, Tg = _gpu_chunks(W, U, Tinv, inp, chunk_ids)
     Wo, Uo, To = _oracle(inp, None if N < 0 else N, None if S < 0 else S, exact=exact, chunk_ids=chunk_ids)
     eT = orc.rel_frobenius(Tg, To); eW = orc.rel_frobenius(Wg, Wo); eU = orc.rel_frobenius(Ug, Uo)
-    assert eT.max() <= tol, f"Tinv rel-F max {eT.max():.3e} at chunk {eT.argmax()}"
-    assert eW.max() <= tol, f"W rel-F max {eW.max():.3e} at chunk {eW.argmax()}"
-    assert eU.max() <= tol, f"U rel-F max {eU.max():.3e} at chunk {eU.argmax()}"
+    for name, err, ref in (("Tinv", eT, To), ("W", eW, Wo), ("U", eU, Uo)):
+        bound = np.full_like(err, tol)
+        if inp.K.dtype == torch.bfloat16:
+            # Rounding the exact result to bf16 already costs ~1.7e-3 and, on strongly correlated keys
+            # with C <= 32, up to 2.2e-3 on a few chunks. Where that floor is within 10% of the
+            # tolerance or above it, the bar is the floor plus 2e-4.
+            floor = orc.rel_frobenius(_bf16_round(ref), ref)
+            bound = np.where(floor > 0.9 * tol, np.maximum(tol, floor + 2e-4), tol)
+        worst = int(np.argmax(err - bound))
+        assert np.all(err <= bound), f"{name} rel-F {err[worst]:.3e} > {bound[worst]:.3e} at chunk {worst}"
     # structure: strictly upper triangle exactly zero, unit diagonal
     assert np.all(np.triu(Tg, 1) == 0)
     assert np.all(np.diagonal(Tg, axis1=-2, axis2=-1) == 1)
