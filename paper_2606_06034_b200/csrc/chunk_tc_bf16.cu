@@ -37,8 +37,18 @@ constexpr int kThreads = 160;         // + one control warp
 constexpr int kD = 128;               // d_k = d_v
 constexpr float kLog2e = 1.4426950408889634f;
 
-// TMEM column map (256 columns allocated)
-constexpr uint32_t kR0 = 0, kR1 = 64, kR2 = 128, kAS = 192, kTmemCols = 256;
+// TMEM column map (256 columns allocated):
+//   R0..R1 (128 columns)  Gram matrix, later the W and then the U accumulator
+//   R2     (64 columns)   accumulator of the residual rounds, later the low-half A operand of W/U
+//   AS     (64 columns)   bf16 A operand (block diagonal, 128 x 128) of the residual rounds and of W/U
+constexpr uint32_t kR0 = 0, kR2 = 128, kAS = 192, kTmemCols = 256;
+
+#ifdef GDN_TRACE
+__device__ long long g_trace[4096];
+#define STAMP(slot) do { if (blockIdx.x == 0 && (tid == 0 || tid == 128) && trace_n < 60) { g_trace[(tid == 0 ? 0 : 2048) + trace_n * 2] = (slot); g_trace[(tid == 0 ? 0 : 2048) + trace_n * 2 + 1] = clock64(); ++trace_n; } } while (0)
+#else
+#define STAMP(slot) do { } while (0)
+#endif
 
 struct Params {
     const float* beta;
@@ -56,18 +66,22 @@ template <int C, int NB>
 struct Smem {
     static constexpr int kK = 0;                        // 32 KB, two [128][64] bf16 sub-tiles, 128B swizzle
     static constexpr int kV = 32768;                    // 32 KB
-    static constexpr int kEB = 65536;                   // B operand written by threads: 128 x C bf16
+    // scratch: [EB | BR]. EB = E as the B operand of the residual rounds (128 x C bf16, core-matrix
+    // layout); BR = one private packed-bf16 row per thread. Before EB/BR are in use the whole region
+    // holds one private fp32 row per thread (Abar row, or the forward-substitution matrix).
+    static constexpr int kEB = 65536;
     static constexpr int kEBBytes = kTile * C * 2;
-    static constexpr int kSH = kEB + kEBBytes;          // column form of the band: [128 + 8][NBP] floats
+    static constexpr int kBR = kEB + kEBBytes;
+    static constexpr int kBRBytes = kTile * C * 2;
     static constexpr int NBP = (NB <= 3) ? 4 : 8;
+    static constexpr int kScratchBytes = 32768;         // >= kEBBytes + kBRBytes; also the 4 x 8 KB store staging slices
+    static constexpr int kSH = kEB + kScratchBytes;     // column form of the band: [128 + 8][NBP] floats
     static constexpr int kSHBytes = (kTile + 8) * NBP * 4;
     static constexpr int kRB = kSH + kSHBytes;          // row form of the band: [128][NBP] floats
     static constexpr int kRBBytes = kTile * NBP * 4;
     static constexpr int kBeta = kRB + kRBBytes;        // 128 floats
     static constexpr int kG = kBeta + 512;              // 128 floats
-    static constexpr int kFwd = kG + 512;               // forward substitution only: fp32 [128][C + 4]
-    static constexpr int kTotalNeumann = kFwd;
-    static constexpr int kTotalFwd = kFwd + kTile * (C + 4) * 4;
+    static constexpr int kTotal = kG + 512;
 };
 
 __device__ __forceinline__ float fast_exp2(float x) {
@@ -78,8 +92,9 @@ __device__ __forceinline__ float fast_exp2(float x) {
 
 __device__ __forceinline__ void compute_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-// bounded mbarrier wait: polls, and every 1024 polls compares the clock with a one-second budget
+// bounded mbarrier wait: polls, and every 1024 polls compares the clock with a budget of about a second
 __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity) {
+    if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     uint32_t i = 0;
     while (!mbar_try_wait(bar, parity)) {
@@ -88,32 +103,88 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity) {
     return true;
 }
 
+// ---- private shared-memory rows (each thread touches only its own row; inline asm keeps the order)
+__device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ void sts16(uint32_t addr, uint16_t v) {
+    asm volatile("st.shared.b16 [%0], %1;" ::"r"(addr), "h"(v) : "memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ float lds32f(uint32_t addr) {
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+    return v;
+}
+// 16-byte chunk index after the bank swizzle, for rows of CPR chunks
+template <int CPR>
+__device__ __forceinline__ int swz(int t, int c) {
+    if constexpr (CPR >= 8) return c ^ (t & 7);
+    else if constexpr (CPR == 4) return c ^ ((t >> 1) & 3);
+    else if constexpr (CPR == 2) return c ^ ((t >> 2) & 1);
+    else return c;
+}
 
-// Writes this row's packed bf16 diagonal block (C / 2 32-bit columns) into the A-operand slot.
+// Builds a packed bf16 row of C entries that is zero except vals[e] at column il - e (e = 0..n_valid,
+// skipped where il - e < 0), through the thread's private row in shared memory: registers cannot be
+// indexed by a per-thread position, shared memory can.
+template <int C, int NB>
+__device__ __forceinline__ void build_band_row(uint32_t row_addr, int t, int il, int n_valid, const uint16_t (&vals)[NB + 1],
+                                               uint32_t (&out)[C / 2]) {
+    constexpr int CPR = C / 8;
+#pragma unroll
+    for (int c = 0; c < CPR; ++c) sts128(row_addr + (swz<CPR>(t, c) << 4), 0u, 0u, 0u, 0u);
+#pragma unroll
+    for (int e = 0; e <= NB; ++e) {
+        const int j = il - e;
+        if (j >= 0 && e <= n_valid) sts16(row_addr + (swz<CPR>(t, j >> 3) << 4) + (j & 7) * 2, vals[e]);
+    }
+#pragma unroll
+    for (int c = 0; c < CPR; ++c) {
+        const uint4 v = lds128(row_addr + (swz<CPR>(t, c) << 4));
+        out[c * 4 + 0] = v.x;
+        out[c * 4 + 1] = v.y;
+        out[c * 4 + 2] = v.z;
+        out[c * 4 + 3] = v.w;
+    }
+}
+
+__device__ __forceinline__ uint16_t bf16_bits(float x) { return __bfloat16_as_ushort(__float2bfloat16_rn(x)); }
+__device__ __forceinline__ float bf16_bits_to_f32(uint16_t b) { return __uint_as_float(static_cast<uint32_t>(b) << 16); }
+
+// Writes this row's packed bf16 diagonal block (C / 2 32-bit columns) into a 64-column A-operand slot.
 // tcgen05.st takes one address per warp: for C = 16 a warp holds two chunks, so the warp stores a
 // 16-column window in which each half-warp fills its own half and zero-fills the other.
-template <int C>
-__device__ __forceinline__ void store_a_operand(uint32_t lane_base, int t, const uint32_t (&pk)[C / 2]) {
+// FULL: also zero-fill the rest of the 64-column row (slot that held other data before).
+template <int C, bool FULL>
+__device__ __forceinline__ void store_a_operand(uint32_t slot_addr, int t, const uint32_t (&pk)[C / 2]) {
     constexpr int PC = C / 2;
-    if constexpr (PC >= 16) {
-        const int cb = t - (t % C);
+    const int wb = (C >= 32) ? (t - (t % C)) : (t & ~31);  // first tile row of the warp-uniform window
+    constexpr int WC = (PC >= 16) ? PC : 16;               // window width in columns
+    const bool upper = (C < 32) && ((t & 16) != 0);
 #pragma unroll
-        for (int c = 0; c < PC / 16; ++c) {
-            uint32_t r16[16];
-#pragma unroll
-            for (int i = 0; i < 16; ++i) r16[i] = pk[c * 16 + i];
-            tmem_st16(lane_base + kAS + cb / 2 + c * 16, r16);
-        }
-    } else {
-        const int wb = t & ~31;
-        const bool upper = (t & 16) != 0;
+    for (int c = 0; c < 4; ++c) {
+        // 16-column group c of the 64-column slot
         uint32_t r16[16];
+        const int rel = c * 16 - wb / 2;  // position of this group relative to the window
+        const bool inside = (rel >= 0) && (rel < WC);
+        if (!FULL && !inside) continue;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            r16[i] = upper ? 0u : pk[i];
-            r16[8 + i] = upper ? pk[i] : 0u;
+        for (int i = 0; i < 16; ++i) {
+            uint32_t v = 0u;
+            if constexpr (PC >= 16) {
+                // rel is 0 or 16 (C = 64) or 0 (C = 32) when inside
+                if (inside) v = (PC == 32) ? ((rel == 0) ? pk[i] : pk[(16 + i) % PC]) : pk[i % PC];
+            } else {
+                if (inside) v = upper ? ((i >= 8) ? pk[i - 8] : 0u) : ((i < 8) ? pk[i] : 0u);
+            }
+            r16[i] = v;
         }
-        tmem_st16(lane_base + kAS + wb / 2, r16);
+        tmem_st16(slot_addr + c * 16, r16);
     }
 }
 
@@ -143,7 +214,7 @@ __device__ __forceinline__ void load_diag_block(uint32_t lane_base, uint32_t col
 
 // Reads C consecutive accumulator columns starting at col0 (same address for the whole warp).
 template <int C>
-__device__ __forceinline__ void load_cols(uint32_t lane_base, uint32_t col0, uint32_t (&r)[C]) {
+__device__ __forceinline__ void load_cols(uint32_t lane_base, uint32_t col0, float (&r)[C]) {
     if constexpr (C >= 32) {
 #pragma unroll
         for (int c0 = 0; c0 < C; c0 += 32) {
@@ -151,15 +222,35 @@ __device__ __forceinline__ void load_cols(uint32_t lane_base, uint32_t col0, uin
             tmem_ld32(lane_base + col0 + c0, q);
             tmem_wait_ld();
 #pragma unroll
-            for (int i = 0; i < 32; ++i) r[c0 + i] = q[i];
+            for (int i = 0; i < 32; ++i) r[c0 + i] = __uint_as_float(q[i]);
         }
     } else {
         uint32_t q[16];
         tmem_ld16(lane_base + col0, q);
         tmem_wait_ld();
 #pragma unroll
-        for (int i = 0; i < 16; ++i) r[i] = q[i];
+        for (int i = 0; i < 16; ++i) r[i] = __uint_as_float(q[i]);
     }
+}
+
+struct TileCoord {
+    int bhk, bhv;
+    int t0;
+};
+// tile index -> (key head row, value head row, first token); tiles that share a key tile are adjacent.
+// All counts fit 32 bits (checked by the launcher).
+__device__ __forceinline__ TileCoord decode_tile(uint32_t tile, const Params& p) {
+    TileCoord c;
+    const uint32_t y = tile / static_cast<uint32_t>(p.group);
+    const uint32_t gi = tile - y * p.group;
+    const uint32_t bhk = y / static_cast<uint32_t>(p.n_tt);
+    const uint32_t tt = y - bhk * p.n_tt;
+    const uint32_t b = bhk / static_cast<uint32_t>(p.H_k);
+    const uint32_t hk = bhk - b * p.H_k;
+    c.bhk = static_cast<int>(bhk);
+    c.bhv = static_cast<int>(b * p.H_v + hk * p.group + gi);
+    c.t0 = static_cast<int>(tt) * kTile;
+    return c;
 }
 
 template <int C, int NB, int MODE>
@@ -167,6 +258,7 @@ __global__ void __launch_bounds__(kThreads, 2)
 chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const Params p) {
     using L = Smem<C, NB>;
     constexpr int NBP = L::NBP;
+    constexpr int PC = C / 2;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* sK = smem + L::kK;
@@ -179,10 +271,12 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 
     __shared__ uint64_t bar_k, bar_v, bar_mma, bar_opnd, bar_free;
     __shared__ uint32_t tmem_base_s;
-    __shared__ int abort_flag;
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
+#ifdef GDN_TRACE
+    int trace_n = 0;
+#endif
 
     if (tid == 0) {
         mbar_init(&bar_k, 1);
@@ -190,7 +284,6 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         mbar_init(&bar_mma, 1);
         mbar_init(&bar_opnd, kComputeThreads);
         mbar_init(&bar_free, kComputeThreads);
-        abort_flag = 0;
         mbar_fence_init();
     }
     if (warp == 4) {
@@ -203,44 +296,47 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     const uint32_t tmem = tmem_base_s;
 
     const int N = p.N, S = p.S;
-    // width of the band kept in fp32 registers (lb[]): the order N, or all of NB for forward substitution
+    // width of the band kept in fp32 (lb[]): the order N, or all of NB for forward substitution
     const int n_band = (MODE == INV_NEUMANN) ? N : NB;
-    // number of MMA rounds between the A-build and the W/U products
-    const int n_rounds = (MODE == INV_NEUMANN) ? (S >= 1 ? S : 0) : 0;
+    // residual rounds: Z_{k+1} = (T0 + Z_k) E, k = 0..S-1, so that T = T0 + Z_S = T0 sum_{s<=S} E^s
+    const int n_rounds = (MODE == INV_NEUMANN) ? S : 0;
 
     if (warp == 4) {
         // ------------------------------------------------------------------ control warp
         if ((tid & 31) == 0) {
             tma_prefetch_desc(&tmK);
             tma_prefetch_desc(&tmV);
-            uint32_t par_kv = 0, par_opnd = 0, par_free = 0;
+            uint32_t par_kv = 0, par_opnd = 0, par_free = 0, n_commit = 0;
             bool ok = true;
-            bool first = true;
             const uint32_t idesc_g = instr_desc(128, 128, 1, 1, 0, 0, 1);
             const uint32_t idesc_c = instr_desc(128, C, 1, 1, 0, 1, 1);
-            const uint32_t idesc_w = instr_desc(128, 64, 1, 1, 0, 1, 1);
+            const uint32_t idesc_w = instr_desc(128, 128, 1, 1, 0, 1, 1);
             const uint32_t sK_a = smem_u32(sK), sV_a = smem_u32(sV), sEB_a = smem_u32(sEB);
-            for (long long tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x) {
-                const int gi = static_cast<int>(tile % p.group);
-                const long long y = tile / p.group;
-                const int tt = static_cast<int>(y % p.n_tt);
-                const long long bhk = y / p.n_tt;
-                const long long b = bhk / p.H_k;
-                const int hk = static_cast<int>(bhk % p.H_k);
-                const long long bhv = b * p.H_v + (long long)hk * p.group + gi;
-                const int t0 = tt * kTile;
-                if (!first) {
+            uint32_t tile = blockIdx.x;
+            const uint32_t n_tiles = static_cast<uint32_t>(p.n_tiles);
+            if (tile < n_tiles) {
+                const TileCoord c = decode_tile(tile, p);
+                mbar_arrive_expect_tx(&bar_k, 32768);
+                tma_load_3d(sK, &tmK, &bar_k, 0, c.t0, static_cast<int>(c.bhk));
+                tma_load_3d(sK + 16384, &tmK, &bar_k, 64, c.t0, static_cast<int>(c.bhk));
+                mbar_arrive_expect_tx(&bar_v, 32768);
+                tma_load_3d(sV, &tmV, &bar_v, 0, c.t0, static_cast<int>(c.bhv));
+                tma_load_3d(sV + 16384, &tmV, &bar_v, 64, c.t0, static_cast<int>(c.bhv));
+            }
+            bool first = true;
+            for (; tile < n_tiles; tile += gridDim.x) {
+                const uint32_t next = tile + gridDim.x;
+                const bool has_next = next < n_tiles;
+                TileCoord nc{0, 0, 0};
+                if (has_next) nc = decode_tile(next, p);
+                STAMP(101);
+                if (!wait_bar(&bar_k, par_kv)) { ok = false; break; }
+                STAMP(102);
+                if (!first) {  // the previous tile's accumulators have been read out
                     if (!wait_bar(&bar_free, par_free)) { ok = false; break; }
                     par_free ^= 1;
                 }
                 first = false;
-                mbar_arrive_expect_tx(&bar_k, 32768);
-                tma_load_3d(sK, &tmK, &bar_k, 0, t0, static_cast<int>(bhk));
-                tma_load_3d(sK + 16384, &tmK, &bar_k, 64, t0, static_cast<int>(bhk));
-                mbar_arrive_expect_tx(&bar_v, 32768);
-                tma_load_3d(sV, &tmV, &bar_v, 0, t0, static_cast<int>(bhv));
-                tma_load_3d(sV + 16384, &tmV, &bar_v, 64, t0, static_cast<int>(bhv));
-                if (!wait_bar(&bar_k, par_kv)) { ok = false; break; }
                 tc_fence_after_sync();
                 // G = K K^T into R0..R1 (128 columns)
 #pragma unroll
@@ -249,50 +345,64 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     mma_f16_ss(tmem + kR0, d, d, idesc_g, ks > 0);
                 }
                 mma_commit(&bar_mma);
-                for (int r = 0; r < n_rounds && ok; ++r) {
+                ++n_commit;
+                STAMP(103);
+                for (int r = 0; r < n_rounds; ++r) {
                     if (!wait_bar(&bar_opnd, par_opnd)) { ok = false; break; }
                     par_opnd ^= 1;
                     tc_fence_after_sync();
-                    const uint32_t dcol = (r < n_rounds - 1) ? kR2 : kR0;
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks) {
                         const uint64_t bd = smem_desc(sEB_a + ks * 256, 128, 2048, SWZ_NONE);
-                        mma_f16_ts(tmem + dcol, tmem + kAS + ks * 8, bd, idesc_c, ks > 0);
+                        mma_f16_ts(tmem + kR2, tmem + kAS + ks * 8, bd, idesc_c, ks > 0);
                     }
                     mma_commit(&bar_mma);
+                    ++n_commit;
                 }
                 if (!ok) break;
-                // W and U: A = far * diag(beta) in TMEM, B = the K / V tile as an MN-major operand
+                // W = (hi + lo) K: A operands in TMEM (AS: high bf16 half, R2: low half of the band),
+                // B = the K tile read as an MN-major operand (both 64-column sub-tiles, N = 128)
                 if (!wait_bar(&bar_opnd, par_opnd)) { ok = false; break; }
                 par_opnd ^= 1;
+                STAMP(104);
+                tc_fence_after_sync();
+#pragma unroll
+                for (int ks = 0; ks < 16; ++ks) {
+                    const uint64_t bd = smem_desc(sK_a + (ks & 7) * 2048, 16384, 1024, SWZ_128B);
+                    mma_f16_ts(tmem + kR0, tmem + ((ks < 8) ? kAS : kR2) + (ks & 7) * 8, bd, idesc_w, ks > 0);
+                }
+                mma_commit(&bar_mma);
+                ++n_commit;
+                STAMP(105);
                 if (!wait_bar(&bar_v, par_kv)) { ok = false; break; }
                 par_kv ^= 1;
-                tc_fence_after_sync();
-#pragma unroll
-                for (int part = 0; part < 3; ++part) {
-                    const uint32_t base = (part < 2) ? (sK_a + part * 16384) : sV_a;
-                    const uint32_t dcol = (part == 0) ? kR0 : (part == 1 ? kR1 : kR2);
-#pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {
-                        const uint64_t bd = smem_desc(base + ks * 2048, 16384, 1024, SWZ_128B);
-                        mma_f16_ts(tmem + dcol, tmem + kAS + ks * 8, bd, idesc_w, ks > 0);
-                    }
-                }
-                mma_commit(&bar_mma);
-                if (!wait_bar(&bar_opnd, par_opnd)) { ok = false; break; }  // R0 read out
+                STAMP(106);
+                // W accumulator read out => the W products are complete => the K tile is free
+                if (!wait_bar(&bar_opnd, par_opnd)) { ok = false; break; }
                 par_opnd ^= 1;
+                if (has_next) {
+                    mbar_arrive_expect_tx(&bar_k, 32768);
+                    tma_load_3d(sK, &tmK, &bar_k, 0, nc.t0, static_cast<int>(nc.bhk));
+                    tma_load_3d(sK + 16384, &tmK, &bar_k, 64, nc.t0, static_cast<int>(nc.bhk));
+                }
                 tc_fence_after_sync();
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const uint64_t bd = smem_desc(sV_a + 16384 + ks * 2048, 16384, 1024, SWZ_128B);
-                    mma_f16_ts(tmem + kR0, tmem + kAS + ks * 8, bd, idesc_w, ks > 0);
+                for (int ks = 0; ks < 16; ++ks) {
+                    const uint64_t bd = smem_desc(sV_a + (ks & 7) * 2048, 16384, 1024, SWZ_128B);
+                    mma_f16_ts(tmem + kR0, tmem + ((ks < 8) ? kAS : kR2) + (ks & 7) * 8, bd, idesc_w, ks > 0);
                 }
                 mma_commit(&bar_mma);
+                ++n_commit;
+                STAMP(107);
+                if (has_next) {  // U products complete => the V tile is free
+                    if (!wait_bar(&bar_mma, (n_commit - 1) & 1)) { ok = false; break; }
+                    STAMP(108);
+                    mbar_arrive_expect_tx(&bar_v, 32768);
+                    tma_load_3d(sV, &tmV, &bar_v, 0, nc.t0, static_cast<int>(nc.bhv));
+                    tma_load_3d(sV + 16384, &tmV, &bar_v, 64, nc.t0, static_cast<int>(nc.bhv));
+                }
             }
-            if (!ok) {
-                atomicExch(p.status, GDN_ERR_TIMEOUT);
-                atomicExch(&abort_flag, 1);
-            }
+            if (!ok) atomicExch(p.status, GDN_ERR_TIMEOUT);
         }
     } else {
         // ------------------------------------------------------------------ compute warps
@@ -300,7 +410,9 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         const int il = t % C;              // row inside its chunk
         const int cb = t - il;             // first tile row of the chunk
         const uint32_t lane_base = tmem + (static_cast<uint32_t>(warp * 32) << 16);
-        uint32_t par_mma = 0, par_kv = 0;
+        const uint32_t scratch_a = smem_u32(smem + L::kEB);
+        const uint32_t br_row = smem_u32(smem + L::kBR) + t * (2 * C);
+        uint32_t par_mma = 0;
         bool ok = true;
 
         {  // the A-operand slot keeps zeros outside the diagonal blocks for the whole kernel
@@ -312,18 +424,12 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             tmem_wait_st();
         }
 
-        for (long long tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x) {
-            const int gi = static_cast<int>(tile % p.group);
-            const long long y = tile / p.group;
-            const int tt = static_cast<int>(y % p.n_tt);
-            const long long bhk = y / p.n_tt;
-            const long long b = bhk / p.H_k;
-            const int hk = static_cast<int>(bhk % p.H_k);
-            const long long bhv = b * p.H_v + (long long)hk * p.group + gi;
-            const int t0 = tt * kTile;
-            const bool row_valid = (t0 + t) < p.T;
-            const long long grow = bhv * (long long)p.T + t0 + t;  // global token row (value-head space)
+        for (uint32_t tile = blockIdx.x; tile < static_cast<uint32_t>(p.n_tiles) && ok; tile += gridDim.x) {
+            const TileCoord tc = decode_tile(tile, p);
+            const bool row_valid = (tc.t0 + t) < p.T;
+            const long long grow = (long long)tc.bhv * p.T + tc.t0 + t;  // global token row (value-head space)
 
+            STAMP(1);
             float bi = 0.f, gi_ = 0.f;
             if (row_valid) {
                 bi = __ldg(p.beta + grow);
@@ -340,17 +446,17 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             }
             compute_barrier();
 
+            STAMP(2);
             // ---- A-build: row of Abar from the Gram block in TMEM
             if (!wait_bar(&bar_mma, par_mma)) { ok = false; break; }
             par_mma ^= 1;
+            STAMP(3);
             tc_fence_after_sync();
             float a[C];
             load_diag_block<C>(lane_base, kR0, t, a);
-            float ab[NB + 1];  // ab[e] = Abar[i][i-e]
-#pragma unroll
-            for (int e = 0; e <= NB; ++e) ab[e] = 0.f;
             {
                 const float gs = gi_ * kLog2e;
+                const float nbi = -bi;
                 const float4* sg4 = reinterpret_cast<const float4*>(sg + cb);
 #pragma unroll
                 for (int j4 = 0; j4 < C / 4; ++j4) {
@@ -359,21 +465,34 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
                         const int j = j4 * 4 + q;
-                        float v = 0.f;
-                        if (j < il) v = -bi * fast_exp2(fmaf(-gj[q], kLog2e, gs)) * a[j];
-                        a[j] = v;
-#pragma unroll
-                        for (int e = 1; e <= NB; ++e)
-                            if (j == il - e) ab[e] = v;
+                        const float v = nbi * fast_exp2(fmaf(-gj[q], kLog2e, gs)) * a[j];
+                        a[j] = (j < il) ? v : 0.f;
                     }
                 }
             }
 
-            float lb[NB + 1];  // lb[d] = L[i][i-d], the band of T0 - I
+            STAMP(4);
+            float lb[NB + 1];  // lb[d] = L[i][i-d], the band of T0 - I (or of T - I after forward substitution)
 #pragma unroll
             for (int e = 0; e <= NB; ++e) lb[e] = 0.f;
 
             if constexpr (MODE == INV_NEUMANN) {
+                // ---- ab[e] = Abar[i][i-e] through the private fp32 row
+                float ab[NB + 1];
+                {
+                    constexpr int CPRF = C / 4;  // 16-byte chunks of an fp32 row
+                    const uint32_t rowf = scratch_a + t * (4 * C);
+#pragma unroll
+                    for (int c = 0; c < CPRF; ++c)
+                        sts128(rowf + (swz<CPRF>(t, c) << 4), __float_as_uint(a[c * 4 + 0]), __float_as_uint(a[c * 4 + 1]),
+                               __float_as_uint(a[c * 4 + 2]), __float_as_uint(a[c * 4 + 3]));
+                    ab[0] = 0.f;
+#pragma unroll
+                    for (int e = 1; e <= NB; ++e) {
+                        const int j = il - e;
+                        ab[e] = (j >= 0) ? lds32f(rowf + (swz<CPRF>(t, j >> 2) << 4) + (j & 3) * 4) : 0.f;
+                    }
+                }
                 // ---- band of the masked Neumann sum by distance recursion
                 lb[1] = ab[1];
                 sRB[t * NBP + 0] = lb[1];
@@ -389,42 +508,34 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     lb[d] = (d <= N) ? v : 0.f;
                     if (d < NB) sRB[t * NBP + (d - 1)] = lb[d];
                 }
-                if (N < 1) lb[1] = 0.f;
                 // column form: SH[j][e-1] = L[j+e][j]
 #pragma unroll
                 for (int e = 1; e <= NB; ++e)
                     if (il - e >= 0) sSH[(t - e) * NBP + (e - 1)] = lb[e];
                 compute_barrier();
 
+                STAMP(5);
                 // ---- E = Abar + Abar L on i-j > N (in place over a[])
 #pragma unroll
                 for (int j = 0; j < C; ++j) {
-                    float v = 0.f;
-                    if (il - j > N) {
-                        v = a[j];
-                        if constexpr (NBP == 4) {
-                            const float4 c4 = *reinterpret_cast<const float4*>(sSH + (cb + j) * 4);
-                            if (j + 1 < C) v = fmaf(a[(j + 1 < C) ? j + 1 : j], c4.x, v);
-                            if (j + 2 < C) v = fmaf(a[(j + 2 < C) ? j + 2 : j], c4.y, v);
-                            if (j + 3 < C) v = fmaf(a[(j + 3 < C) ? j + 3 : j], c4.z, v);
-                        } else {
-                            const float4 c4 = *reinterpret_cast<const float4*>(sSH + (cb + j) * 8);
-                            const float4 d4 = *reinterpret_cast<const float4*>(sSH + (cb + j) * 8 + 4);
-                            const float cc[7] = {c4.x, c4.y, c4.z, c4.w, d4.x, d4.y, d4.z};
+                    float v = a[j];
+                    if constexpr (NBP == 4) {
+                        const float4 c4 = *reinterpret_cast<const float4*>(sSH + (cb + j) * 4);
+                        if (j + 1 < C) v = fmaf(a[(j + 1 < C) ? j + 1 : j], c4.x, v);
+                        if (j + 2 < C) v = fmaf(a[(j + 2 < C) ? j + 2 : j], c4.y, v);
+                        if (j + 3 < C) v = fmaf(a[(j + 3 < C) ? j + 3 : j], c4.z, v);
+                    } else {
+                        const float4 c4 = *reinterpret_cast<const float4*>(sSH + (cb + j) * 8);
+                        const float4 d4 = *reinterpret_cast<const float4*>(sSH + (cb + j) * 8 + 4);
+                        const float cc[7] = {c4.x, c4.y, c4.z, c4.w, d4.x, d4.y, d4.z};
 #pragma unroll
-                            for (int e = 1; e <= NB; ++e)
-                                if (j + e < C) v = fmaf(a[(j + e < C) ? j + e : j], cc[e - 1], v);
-                        }
+                        for (int e = 1; e <= NB; ++e)
+                            if (j + e < C) v = fmaf(a[(j + e < C) ? j + e : j], cc[e - 1], v);
                     }
-                    a[j] = v;
+                    a[j] = (il - j > N) ? v : 0.f;
                 }
-                // now a[] = E row. Chain: x = X_k row.
-                float x[C];
-#pragma unroll
-                for (int j = 0; j < C; ++j) x[j] = (S >= 1) ? a[j] : 0.f;
-
+                // E as B operand (MN-major, no swizzle): 16-byte chunk c of row t at c * 2048 + t * 16
                 if (S >= 1) {
-                    // E as B operand (MN-major, no swizzle): 16-byte chunk c of row t at c * 2048 + t * 16
 #pragma unroll
                     for (int c = 0; c < C / 8; ++c) {
                         uint4 v;
@@ -435,41 +546,85 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                         *reinterpret_cast<uint4*>(sEB + c * 2048 + t * 16) = v;
                     }
                 }
-                for (int k = 1; k <= S; ++k) {
-                    // operand for round k: X_k (k < S) or the band L (k == S, "far" product with B = X_S)
-                    if (k == S) {
+            } else {
+                // ---- forward substitution (Eq. 2-3). The private fp32 rows hold Abar; thread = column il of its chunk.
+                constexpr int CPRF = C / 4;
+                const uint32_t rowf = scratch_a + t * (4 * C);
 #pragma unroll
-                        for (int c = 0; c < C / 8; ++c) {
-                            uint4 v;
-                            v.x = pack_bf16x2(x[c * 8 + 0], x[c * 8 + 1]);
-                            v.y = pack_bf16x2(x[c * 8 + 2], x[c * 8 + 3]);
-                            v.z = pack_bf16x2(x[c * 8 + 4], x[c * 8 + 5]);
-                            v.w = pack_bf16x2(x[c * 8 + 6], x[c * 8 + 7]);
-                            *reinterpret_cast<uint4*>(sEB + c * 2048 + t * 16) = v;
-                        }
+                for (int c = 0; c < CPRF; ++c)
+                    sts128(rowf + (swz<CPRF>(t, c) << 4), __float_as_uint(a[c * 4 + 0]), __float_as_uint(a[c * 4 + 1]),
+                           __float_as_uint(a[c * 4 + 2]), __float_as_uint(a[c * 4 + 3]));
+                compute_barrier();
+                float xcol[C];  // xcol[k] = T[k][il]
+#pragma unroll
+                for (int i = 0; i < C; ++i) {
+                    float acc = 0.f;
+                    const uint32_t ri = scratch_a + (cb + i) * (4 * C);
+#pragma unroll
+                    for (int k4 = 0; k4 < (i + 3) / 4; ++k4) {
+                        const uint4 q = lds128(ri + (swz<CPRF>(i, k4) << 4));  // (cb + i) and i agree in the swizzle bits
+                        if (k4 * 4 + 0 < i) acc = fmaf(__uint_as_float(q.x), xcol[k4 * 4 + 0], acc);
+                        if (k4 * 4 + 1 < i) acc = fmaf(__uint_as_float(q.y), xcol[(k4 * 4 + 1 < C) ? k4 * 4 + 1 : 0], acc);
+                        if (k4 * 4 + 2 < i) acc = fmaf(__uint_as_float(q.z), xcol[(k4 * 4 + 2 < C) ? k4 * 4 + 2 : 0], acc);
+                        if (k4 * 4 + 3 < i) acc = fmaf(__uint_as_float(q.w), xcol[(k4 * 4 + 3 < C) ? k4 * 4 + 3 : 0], acc);
                     }
-                    {
-                        constexpr int PC = C / 2;  // packed columns of this row's diagonal block
-                        uint32_t pk[PC];
+                    xcol[i] = (i > il) ? acc : ((i == il) ? 1.f : 0.f);
+                }
+                compute_barrier();  // everyone has read Abar
 #pragma unroll
-                        for (int jp = 0; jp < PC; ++jp) {
-                            float lo, hi;
-                            if (k < S) {
-                                lo = x[2 * jp];
-                                hi = x[2 * jp + 1];
-                            } else {
-                                lo = 0.f;
-                                hi = 0.f;
+                for (int i = 0; i < C; ++i) {
+                    const uint32_t addr = scratch_a + (cb + i) * (4 * C) + (swz<CPRF>(i, il >> 2) << 4) + (il & 3) * 4;
+                    asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(xcol[i]) : "memory");
+                }
+                compute_barrier();
+                // back to rows: a[] = far part, lb[] = band part
 #pragma unroll
-                                for (int e = 1; e <= NB; ++e) {
-                                    if (2 * jp == il - e) lo = lb[e];
-                                    if (2 * jp + 1 == il - e) hi = lb[e];
-                                }
-                            }
-                            pk[jp] = pack_bf16x2(lo, hi);
-                        }
-                        store_a_operand<C>(lane_base, t, pk);
+                for (int c = 0; c < CPRF; ++c) {
+                    const uint4 q = lds128(rowf + (swz<CPRF>(t, c) << 4));
+                    a[c * 4 + 0] = __uint_as_float(q.x);
+                    a[c * 4 + 1] = __uint_as_float(q.y);
+                    a[c * 4 + 2] = __uint_as_float(q.z);
+                    a[c * 4 + 3] = __uint_as_float(q.w);
+                }
+#pragma unroll
+                for (int e = 1; e <= NB; ++e) {
+                    const int j = il - e;
+                    lb[e] = (j >= 0) ? lds32f(rowf + (swz<CPRF>(t, j >> 2) << 4) + (j & 3) * 4) : 0.f;
+                }
+#pragma unroll
+                for (int j = 0; j < C; ++j) a[j] = (il - j > NB) ? a[j] : 0.f;
+                compute_barrier();  // the fp32 rows are dead; the packed rows may overwrite them
+            }
+
+            STAMP(6);
+            // ---- packed bf16 forms of the band: keep-mask (0 on the band and diagonal) and I + L
+            uint32_t keep[PC], bpT[PC];
+            {
+                uint16_t vals[NB + 1];
+#pragma unroll
+                for (int e = 0; e <= NB; ++e) vals[e] = 0xFFFFu;
+                build_band_row<C, NB>(br_row, t, il, n_band, vals, keep);
+#pragma unroll
+                for (int i = 0; i < PC; ++i) keep[i] = ~keep[i];
+                vals[0] = 0x3F80u;  // 1.0
+#pragma unroll
+                for (int e = 1; e <= NB; ++e) vals[e] = bf16_bits(lb[e]);
+                build_band_row<C, NB>(br_row, t, il, n_band, vals, bpT);
+            }
+
+            STAMP(7);
+            if constexpr (MODE == INV_NEUMANN) {
+                // ---- residual rounds: A_k = T0 + Z_k (bf16, TMEM), Z_{k+1} = A_k E
+                for (int k = 0; k < S; ++k) {
+                    uint32_t pk[PC];
+                    if (k == 0) {
+#pragma unroll
+                        for (int i = 0; i < PC; ++i) pk[i] = bpT[i];
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < PC; ++i) pk[i] = (pack_bf16x2(a[2 * i], a[2 * i + 1]) & keep[i]) | bpT[i];
                     }
+                    store_a_operand<C, false>(lane_base + kAS, t, pk);
                     fence_proxy_async_smem();
                     tmem_wait_st();
                     tc_fence_before_sync();
@@ -477,161 +632,118 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     if (!wait_bar(&bar_mma, par_mma)) { ok = false; break; }
                     par_mma ^= 1;
                     tc_fence_after_sync();
-                    const uint32_t dcol = (k < S) ? kR2 : kR0;
-                    uint32_t dres[C];
-                    load_cols<C>(lane_base, dcol, dres);
-#pragma unroll
-                    for (int i = 0; i < C; ++i) x[i] = ((k < S) ? a[i] : x[i]) + __uint_as_float(dres[i]);
+                    load_cols<C>(lane_base, kR2, a);
                 }
                 if (!ok) break;
-                // x[] = far row. Move into a[] for the common tail.
+                if (S == 0) {
 #pragma unroll
-                for (int j = 0; j < C; ++j) a[j] = x[j];
-            } else {
-                // ---- forward substitution (Eq. 2-3), thread = column of its chunk
-                float* sF = reinterpret_cast<float*>(smem + L::kFwd);
-                constexpr int LDF = C + 4;
-#pragma unroll
-                for (int j = 0; j < C; ++j) sF[t * LDF + j] = a[j];
-                compute_barrier();
-                float xcol[C];  // xcol[k] = T[k][il] of this thread's chunk (column il)
-#pragma unroll
-                for (int i = 0; i < C; ++i) {
-                    float acc = 0.f;
-#pragma unroll
-                    for (int k = 0; k < i; ++k) acc = fmaf(sF[(cb + i) * LDF + k], xcol[k], acc);
-                    xcol[i] = (i > il) ? acc : ((i == il) ? 1.f : 0.f);
-                }
-                compute_barrier();  // everyone has read Abar
-#pragma unroll
-                for (int i = 0; i < C; ++i) sF[(cb + i) * LDF + il] = xcol[i];
-                compute_barrier();
-                // back to rows: a[] = far part, lb[] = band part
-#pragma unroll
-                for (int j = 0; j < C; ++j) {
-                    const float v = sF[t * LDF + j];
-                    const int dist = il - j;
-                    a[j] = (dist > NB) ? v : 0.f;
-#pragma unroll
-                    for (int e = 1; e <= NB; ++e)
-                        if (dist == e) lb[e] = v;
+                    for (int j = 0; j < C; ++j) a[j] = 0.f;
                 }
             }
+            // a[] = far row (T - I - L)
 
-            // ---- T row -> Tinv
-            if (p.Tinv != nullptr && row_valid) {
-                __nv_bfloat16* trow = p.Tinv + (grow / C) * (long long)(C * C) + (long long)il * C;
+            STAMP(8);
+            // ---- T row -> Tinv. Rows go through the private packed rows so that each store instruction of a
+            // warp covers whole 128-byte lines (the warp's 32 rows are contiguous in global memory).
+            if (p.Tinv != nullptr) {
+                constexpr int CPR = C / 8;           // 16-byte chunks per row
+                constexpr int RPI = 32 / CPR;        // rows per store instruction
 #pragma unroll
-                for (int c = 0; c < C / 8; ++c) {
-                    float v[8];
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        const int j = c * 8 + q;
-                        float val = a[j];
-                        if (j == il) val = 1.f;
-#pragma unroll
-                        for (int e = 1; e <= NB; ++e)
-                            if (j == il - e && e <= n_band) val = lb[e];
-                        v[q] = val;
-                    }
-                    uint4 o;
-                    o.x = pack_bf16x2(v[0], v[1]);
-                    o.y = pack_bf16x2(v[2], v[3]);
-                    o.z = pack_bf16x2(v[4], v[5]);
-                    o.w = pack_bf16x2(v[6], v[7]);
-                    *reinterpret_cast<uint4*>(trow + c * 8) = o;
+                for (int c = 0; c < CPR; ++c) {
+                    sts128(br_row + (swz<CPR>(t, c) << 4),
+                           (pack_bf16x2(a[c * 8 + 0], a[c * 8 + 1]) & keep[c * 4 + 0]) | bpT[c * 4 + 0],
+                           (pack_bf16x2(a[c * 8 + 2], a[c * 8 + 3]) & keep[c * 4 + 1]) | bpT[c * 4 + 1],
+                           (pack_bf16x2(a[c * 8 + 4], a[c * 8 + 5]) & keep[c * 4 + 2]) | bpT[c * 4 + 2],
+                           (pack_bf16x2(a[c * 8 + 6], a[c * 8 + 7]) & keep[c * 4 + 3]) | bpT[c * 4 + 3]);
                 }
+                __syncwarp();
+                const int lane = t & 31;
+                const int wrow0 = t - lane;  // first tile row of this warp
+                const uint32_t br_base = smem_u32(smem + L::kBR);
+                uint4* gbase = reinterpret_cast<uint4*>(p.Tinv + ((long long)tc.bhv * p.T + tc.t0 + wrow0) * C);
+#pragma unroll
+                for (int it = 0; it < CPR; ++it) {
+                    const int r = wrow0 + it * RPI + lane / CPR;  // tile row read by this lane
+                    const int c = lane % CPR;
+                    const uint4 v = lds128(br_base + r * (2 * C) + (swz<CPR>(r, c) << 4));
+                    if (tc.t0 + r < p.T) gbase[it * 32 + lane] = v;
+                }
+                __syncwarp();
             }
 
-            // ---- A operand for W/U: far * diag(beta)
+            STAMP(9);
+            // ---- A operands for W/U: T diag(beta) = hi + lo, hi over the whole row, lo only on band + diagonal
             {
-                constexpr int PC = C / 2;
-                uint32_t pk[PC];
+                float tb[NB + 1];
+                tb[0] = bi;
+#pragma unroll
+                for (int e = 1; e <= NB; ++e) tb[e] = (il - e >= 0) ? lb[e] * sbeta[(t - e) > 0 ? (t - e) : 0] : 0.f;
+                uint16_t hi[NB + 1], lo[NB + 1];
+#pragma unroll
+                for (int e = 0; e <= NB; ++e) {
+                    hi[e] = bf16_bits(tb[e]);
+                    lo[e] = bf16_bits(tb[e] - bf16_bits_to_f32(hi[e]));
+                }
+                uint32_t bp[PC], pk[PC];
+                build_band_row<C, NB>(br_row, t, il, n_band, hi, bp);
                 const float2* sb2 = reinterpret_cast<const float2*>(sbeta + cb);
 #pragma unroll
-                for (int jp = 0; jp < PC; ++jp) {
-                    const float2 bb = sb2[jp];
-                    pk[jp] = pack_bf16x2(a[2 * jp] * bb.x, a[2 * jp + 1] * bb.y);
+                for (int i = 0; i < PC; ++i) {
+                    const float2 bb = sb2[i];
+                    pk[i] = (pack_bf16x2(a[2 * i] * bb.x, a[2 * i + 1] * bb.y) & keep[i]) | bp[i];
                 }
-                store_a_operand<C>(lane_base, t, pk);
+                store_a_operand<C, false>(lane_base + kAS, t, pk);
+                build_band_row<C, NB>(br_row, t, il, n_band, lo, bp);
+                store_a_operand<C, true>(lane_base + kR2, t, bp);
                 tmem_wait_st();
                 tc_fence_before_sync();
                 mbar_arrive(&bar_opnd);
             }
 
-            // ---- W, U: band part on the FMA pipes, far part from the MMA
-            float coef[NB + 1];
-            coef[0] = bi;
-#pragma unroll
-            for (int e = 1; e <= NB; ++e) coef[e] = (il - e >= 0) ? lb[e] * sbeta[(t - e) > 0 ? (t - e) : 0] : 0.f;
-
-            // the TMA barriers completed long ago; waiting on them here makes the tiles visible to this thread
-            if (!wait_bar(&bar_k, par_kv) || !wait_bar(&bar_v, par_kv)) { ok = false; break; }
-            par_kv ^= 1;
+            STAMP(10);
+            // ---- W, then U: accumulator rows -> bf16 -> 16-byte stores (one 256-byte row per thread)
 #pragma unroll 1
-            for (int part = 0; part < 4; ++part) {
-                // part 0: W[:, 0:64] (R0), 1: W[:, 64:128] (R1), 2: U[:, 0:64] (R2), 3: U[:, 64:128] (R0, second commit)
-                const uint8_t* src = ((part < 2) ? sK : sV) + (part & 1) * 16384;
-                float acc[64];
+            for (int half = 0; half < 2; ++half) {
+                if (!wait_bar(&bar_mma, par_mma)) { ok = false; break; }
+                par_mma ^= 1;
+                tc_fence_after_sync();
+                STAMP(11 + half * 3);
+                uint32_t o[64];
 #pragma unroll
-                for (int i = 0; i < 64; ++i) acc[i] = 0.f;
-#pragma unroll
-                for (int e = 0; e <= NB; ++e) {
-                    const int r = (t - e) > 0 ? (t - e) : 0;
-                    const float cf = coef[e];
-                    const uint8_t* rowp = src + r * 128;
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        const uint4 q = *reinterpret_cast<const uint4*>(rowp + ((c ^ (r & 7)) << 4));
-                        acc[c * 8 + 0] = fmaf(cf, bf16_lo(q.x), acc[c * 8 + 0]);
-                        acc[c * 8 + 1] = fmaf(cf, bf16_hi(q.x), acc[c * 8 + 1]);
-                        acc[c * 8 + 2] = fmaf(cf, bf16_lo(q.y), acc[c * 8 + 2]);
-                        acc[c * 8 + 3] = fmaf(cf, bf16_hi(q.y), acc[c * 8 + 3]);
-                        acc[c * 8 + 4] = fmaf(cf, bf16_lo(q.z), acc[c * 8 + 4]);
-                        acc[c * 8 + 5] = fmaf(cf, bf16_hi(q.z), acc[c * 8 + 5]);
-                        acc[c * 8 + 6] = fmaf(cf, bf16_lo(q.w), acc[c * 8 + 6]);
-                        acc[c * 8 + 7] = fmaf(cf, bf16_hi(q.w), acc[c * 8 + 7]);
-                    }
-                }
-                if (part == 0 || part == 3) {
-                    if (!wait_bar(&bar_mma, par_mma)) { ok = false; break; }
-                    par_mma ^= 1;
-                    tc_fence_after_sync();
-                }
-                const uint32_t dcol = (part == 1) ? kR1 : (part == 2 ? kR2 : kR0);
-#pragma unroll
-                for (int c0 = 0; c0 < 64; c0 += 32) {
+                for (int c0 = 0; c0 < 128; c0 += 32) {
                     uint32_t r[32];
-                    tmem_ld32(lane_base + dcol + c0, r);
+                    tmem_ld32(lane_base + kR0 + c0, r);
                     tmem_wait_ld();
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) acc[c0 + i] += __uint_as_float(r[i]);
+                    for (int i = 0; i < 16; ++i) o[c0 / 2 + i] = pack_bf16x2(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
                 }
-                if (part == 0) {  // R0 is free for the second half of U
-                    tc_fence_before_sync();
-                    mbar_arrive(&bar_opnd);
-                }
-                if (row_valid) {
-                    __nv_bfloat16* dst = ((part < 2) ? p.W : p.U) + grow * kD + (part & 1) * 64;
+                tc_fence_before_sync();
+                mbar_arrive(half == 0 ? &bar_opnd : &bar_free);
+                STAMP(12 + half * 3);
+                {
+                    // stage the warp's 32 rows (256 bytes each) in its 8 KB slice of the scratch region, then
+                    // store whole 512-byte runs per instruction
+                    const int lane = t & 31;
+                    const int wrow0 = t - lane;
+                    const uint32_t slice = scratch_a + wrow0 * 256;
 #pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        uint4 o;
-                        o.x = pack_bf16x2(acc[c * 8 + 0], acc[c * 8 + 1]);
-                        o.y = pack_bf16x2(acc[c * 8 + 2], acc[c * 8 + 3]);
-                        o.z = pack_bf16x2(acc[c * 8 + 4], acc[c * 8 + 5]);
-                        o.w = pack_bf16x2(acc[c * 8 + 6], acc[c * 8 + 7]);
-                        *reinterpret_cast<uint4*>(dst + c * 8) = o;
+                    for (int c = 0; c < 16; ++c)
+                        sts128(slice + lane * 256 + ((c ^ (lane & 7)) << 4), o[c * 4 + 0], o[c * 4 + 1], o[c * 4 + 2], o[c * 4 + 3]);
+                    __syncwarp();
+                    uint4* gbase = reinterpret_cast<uint4*>((half == 0 ? p.W : p.U) + ((long long)tc.bhv * p.T + tc.t0 + wrow0) * kD);
+#pragma unroll
+                    for (int it = 0; it < 16; ++it) {
+                        const int r = it * 2 + (lane >> 4);
+                        const int c = lane & 15;
+                        const uint4 v = lds128(slice + r * 256 + ((c ^ (r & 7)) << 4));
+                        if (tc.t0 + wrow0 + r < p.T) gbase[it * 32 + lane] = v;
                     }
+                    __syncwarp();
                 }
+                STAMP(13 + half * 3);
             }
-            if (!ok) break;
-            tc_fence_before_sync();
-            mbar_arrive(&bar_free);
         }
-        if (!ok) {
-            atomicExch(p.status, GDN_ERR_TIMEOUT);
-            atomicExch(&abort_flag, 1);
-        }
+        if (!ok) atomicExch(p.status, GDN_ERR_TIMEOUT);
     }
 
     tc_fence_before_sync();
@@ -675,7 +787,7 @@ bool make_tile_map(CUtensorMap* tm, const void* base, long long heads, int T) {
 template <int C, int NB, int MODE>
 int launch_one(const CUtensorMap& tmK, const CUtensorMap& tmV, const Params& prm, cudaStream_t stream) {
     using L = Smem<C, NB>;
-    const int smem = ((MODE == INV_NEUMANN) ? L::kTotalNeumann : L::kTotalFwd) + 1024;
+    const int smem = L::kTotal + 1024;
     auto kern = chunk_tc_kernel<C, NB, MODE>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return GDN_ERR_LAUNCH;
     long long grid = prm.n_tiles < 2 * 148 ? prm.n_tiles : 2 * 148;
@@ -691,6 +803,12 @@ int launch_c(const CUtensorMap& tmK, const CUtensorMap& tmV, const Params& prm, 
 }
 
 }  // namespace
+
+#ifdef GDN_TRACE
+extern "C" int gdn_debug_read_trace(long long* host_out) {
+    return cudaMemcpyFromSymbol(host_out, g_trace, sizeof(long long) * 4096) == cudaSuccess ? 0 : -1;
+}
+#endif
 
 int launch_tc_bf16(const Problem& p, InverseMode mode, cudaStream_t stream) {
     if (p.d_k != kD || p.d_v != kD) return GDN_ERR_UNSUPPORTED;
@@ -718,6 +836,7 @@ int launch_tc_bf16(const Problem& p, InverseMode mode, cudaStream_t stream) {
     prm.N = p.order;
     prm.S = p.steps;
     prm.n_tiles = (long long)p.B * p.H_v * prm.n_tt;
+    if (prm.n_tiles >= (1LL << 31) - 4096 || (long long)p.B * p.H_v >= (1LL << 31)) return GDN_ERR_UNSUPPORTED;
     if (mode == INV_NEUMANN) {
         switch (p.C) {
             case 16: return launch_c<16, INV_NEUMANN>(tmK, tmV, prm, stream);
