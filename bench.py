@@ -1,0 +1,358 @@
+#!/usr/bin/env python
+"""Benchmark of the chunk-prepare hot path (A-build, multiplication-only inverse, W and U).
+
+One "step" = one pass of the whole path over one batch of synthetic chunks, i.e. one call of
+`gdn_chunk_prepare_gqa` through the C-ABI library. Prints ONE JSON line (rank 0).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+  python -m torch.distributed.run --nnodes=1 --nproc-per-node N ... bench.py --gpus N ...
+
+N > 1: every rank runs the same workload on its own GPU (chunks are independent, there is no
+exchange step), the timed region is bracketed by a barrier and the slowest rank's time counts.
+`--impl reference` times the fp64 CPU oracle on the host cores instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+METRIC = "chunk_prepare_throughput"
+UNIT = "chunks/s"
+DEFAULT_WORKLOAD = "sweep_c64"
+
+
+# ----------------------------------------------------------------------------- bookkeeping
+def matmuls_per_inverse(C: int) -> tuple[int, int]:
+    """(number of c x c products, c) the paper's scheme needs per chunk with its default (N, S)."""
+    return {16: (6, 16), 32: (7, 32), 64: (11, 64), 128: (24, 64)}[C]
+
+
+def nominal_flops_per_chunk(C: int, d_k: int, d_v: int) -> float:
+    """Dense count as the paper counts matmuls: K K^T, the inverse's products, W and U."""
+    m, c = matmuls_per_inverse(C)
+    return 2.0 * C * C * d_k + m * 2.0 * c ** 3 + 2.0 * C * C * d_k + 2.0 * C * C * d_v
+
+
+def algorithmic_bytes_per_chunk(C: int, d_k: int, d_v: int, group: int, esize: int = 2) -> float:
+    """What the method must move per chunk: K (once per group of value heads), V, W, U tiles,
+    the full Tinv block, beta and g."""
+    return (C * d_k * esize) / group + C * d_v * esize + C * d_k * esize + C * d_v * esize + C * C * esize + 8 * C
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), float(d.get("bf16_tflops", 1590.0)), "measured"
+    return 6650.0, 1590.0, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and clock-event reasons of one GPU through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.004):
+        super().__init__(daemon=True)
+        self.index = index
+        self.period = period_s
+        self.samples = []
+        self.reasons = set()
+        self.max_mhz = None
+        self._halt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            self.nv = pynvml
+            pynvml.nvmlInit()
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def _reason_names(self, mask: int):
+        nv = self.nv
+        table = {
+            "sw_power_cap": getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4),
+            "hw_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
+            "hw_power_brake_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwPowerBrakeSlowdown", 0x80),
+            "applications_clocks_setting": getattr(nv, "nvmlClocksThrottleReasonApplicationsClocksSetting", 0x2),
+        }
+        return [k for k, bit in table.items() if mask & bit]
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        while not self._halt.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                self.reasons.update(self._reason_names(mask))
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._halt.set()
+        self.join(timeout=1.0)
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ----------------------------------------------------------------------------- CPU oracle leg
+def time_oracle(workload: str, budget_s: float, seed_offset: int = 0):
+    """Times the fp64 oracle, as it stands, on a bounded sample of the workload's chunks."""
+    from oracle import gdn_oracle as orc
+    from paper_2606_06034_b200 import inputs as gen
+
+    cfg = dict(gen.WORKLOADS[workload])
+    # a small instance with the same per-chunk shapes and distributions
+    small = dict(cfg, B=1, H_k=min(cfg["H_k"], 2), H_v=min(cfg["H_k"], 2) * (cfg["H_v"] // cfg["H_k"]), T=max(cfg["C"] * 16, 1024))
+    inp = gen.make_inputs(device="cpu", **small)
+    ids = list(range(inp.n_chunks))
+    sl = gen.chunk_slices(inp, ids)
+    K = np.stack([s[0] for s in sl]); V = np.stack([s[1] for s in sl])
+    b = np.stack([s[2] for s in sl]); g = np.stack([s[3] for s in sl])
+    n0 = min(64, len(ids))
+    t0 = time.perf_counter()
+    orc.chunk_prepare(K[:n0], V[:n0], b[:n0], g[:n0])
+    per_chunk = (time.perf_counter() - t0) / n0
+    n = int(max(n0, budget_s / max(per_chunk, 1e-9)))
+    reps = (n + len(ids) - 1) // len(ids)
+    done = 0
+    w0 = time.perf_counter(); c0 = time.process_time()
+    for r in range(reps):
+        m = min(len(ids), n - done)
+        if m <= 0:
+            break
+        orc.chunk_prepare(K[:m], V[:m], b[:m], g[:m])
+        done += m
+    wall = time.perf_counter() - w0
+    cpu = time.process_time() - c0
+    return {"value": done / wall, "unit": UNIT, "cores": max(1, int(round(cpu / max(wall, 1e-9)))), "kind": "oracle",
+            "sample": f"{done} chunks of the {workload} shapes (C={cfg['C']}, d={cfg['d_k']}), fp64 numpy oracle, "
+                      f"{wall:.1f} s wall, host has {os.cpu_count()} logical cores"}, wall
+
+
+# ----------------------------------------------------------------------------- GPU legs
+def device_time_steps(fn, steps: int, warmup: int, dist_ctx):
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    if dist_ctx is not None:
+        dist_ctx.barrier()
+    torch.cuda.synchronize()
+    stream = torch.cuda.current_stream()
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    evs[0].record(stream)
+    for i in range(steps):
+        fn()
+        evs[i + 1].record(stream)
+    torch.cuda.synchronize()
+    if dist_ctx is not None:
+        dist_ctx.barrier()
+    total_ms = evs[0].elapsed_time(evs[-1])
+    per = [evs[i].elapsed_time(evs[i + 1]) for i in range(steps)]
+    return total_ms, per
+
+
+def run_ours(args, rank, world, dist_ctx):
+    from paper_2606_06034_b200 import binding as gdn
+    from paper_2606_06034_b200 import inputs as gen
+
+    dev = torch.device("cuda", torch.cuda.current_device())
+    inp = gen.make_workload(args.workload, device=dev)
+    C, group = inp.C, inp.H_v // inp.H_k
+    outs = gdn.alloc_outputs(inp.K, inp.V, C)
+    n_chunks = inp.n_chunks
+
+    def step():
+        gdn.chunk_prepare(inp.K, inp.V, inp.beta, inp.g, C, outputs=outs)
+
+    sampler = ClockSampler(torch.cuda.current_device())
+    launches0 = gdn.gdn_launch_count()
+    # warm-up happens inside device_time_steps; the sampler only runs during the timed steps
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    launches0 = gdn.gdn_launch_count()
+    sampler.start()
+    total_ms, per = device_time_steps(step, args.steps, 0, dist_ctx)
+    clocks = sampler.stop()
+    launches = gdn.gdn_launch_count() - launches0
+    status = gdn.gdn_device_status()
+    if status != gdn.GDN_OK:
+        raise RuntimeError(f"kernel status {status}")
+
+    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+    if dist_ctx is not None:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * n_chunks / (ms_per_step * 1e-3)
+
+    bytes_chunk = algorithmic_bytes_per_chunk(C, inp.d_k, inp.d_v, group)
+    flops_chunk = nominal_flops_per_chunk(C, inp.d_k, inp.d_v)
+    hbm_peak, bf16_peak, peak_kind = measured_peaks()
+    launch_ms = float(np.mean(per))
+    achieved = n_chunks * bytes_chunk / (launch_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak,
+                "traffic": TRAFFIC_PER_LAUNCH.get(args.workload), "peak_kind": peak_kind,
+                "algorithmic_bytes_per_launch": n_chunks * bytes_chunk,
+                "kernel": "chunk_tc_kernel<C=%d>" % C,
+                "effective_tflops": n_chunks * flops_chunk / (launch_ms * 1e-3) / 1e12,
+                "tensor_time_frac_of_bf16_peak": (n_chunks * flops_chunk / (launch_ms * 1e-3) / 1e12) / bf16_peak}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic", "impl": "ours",
+        "config": {"workload": args.workload, "B": inp.B, "H_k": inp.H_k, "H_v": inp.H_v, "T": inp.T, "C": C, "d_k": inp.d_k,
+                   "d_v": inp.d_v, "order": gdn.gdn_default_order(C), "residual_steps": gdn.gdn_default_residual_steps(C),
+                   "chunks_per_gpu": n_chunks, "parallelism": f"independent shards x{world}, no collective",
+                   "l2_policy": "inputs+outputs %.0f MB per step, larger than the 126 MB L2" % (n_chunks * bytes_chunk / 1e6)},
+        "effective_tflops": world * n_chunks * flops_chunk / (ms_per_step * 1e-3) / 1e12,
+        "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline,
+    }
+
+    if rank == 0 and not args.no_e2e:
+        line["e2e"] = run_e2e(inp, outs, gdn, args, world, n_chunks)
+    if rank == 0 and not args.no_extras:
+        line["extras"] = run_extras(gdn, gen, dev, args)
+    if rank == 0 and not args.no_cpu and world == 1:
+        line["cpu_baseline"], _ = time_oracle(args.workload, args.cpu_seconds)
+    return line
+
+
+# per-launch DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under profiles/
+TRAFFIC_PER_LAUNCH: dict = {}
+
+
+def run_e2e(inp, outs, gdn, args, world, n_chunks):
+    """Same metric through the C-ABI with HOST buffers: pinned host -> device copies of K, V, beta, g and a
+    device -> host read of W, U, Tinv inside the timed region, every step."""
+    host_in = [t.cpu().pin_memory() for t in (inp.K, inp.V, inp.beta, inp.g)]
+    dev_in = [torch.empty_like(t) for t in (inp.K, inp.V, inp.beta, inp.g)]
+    host_out = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in outs]
+    h2d = sum(t.numel() * t.element_size() for t in host_in)
+    d2h = sum(t.numel() * t.element_size() for t in host_out)
+    steps = max(3, min(args.steps, 10))
+
+    def step():
+        for h, d in zip(host_in, dev_in):
+            d.copy_(h, non_blocking=True)
+        gdn.chunk_prepare(dev_in[0], dev_in[1], dev_in[2], dev_in[3], inp.C, outputs=outs)
+        for h, d in zip(host_out, outs):
+            h.copy_(d, non_blocking=True)
+
+    total_ms, _ = device_time_steps(step, steps, 2, None)
+    return {"value": world * n_chunks / (total_ms / steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+            "d2h_bytes_per_step": d2h, "steps": steps, "ms_per_step": total_ms / steps}
+
+
+def run_extras(gdn, gen, dev, args):
+    """Other workloads and the forward-substitution comparison, timed the same way (not the headline)."""
+    out = {}
+    hbm_peak, _, _ = measured_peaks()
+    plan = [("sweep_c16", "neumann"), ("sweep_c32", "neumann"), ("sweep_c64", "neumann"), ("sweep_c64", "fwdsubst"),
+            ("sweep_c32", "fwdsubst"), ("sweep_c16", "fwdsubst"), ("prefill_gqa", "neumann")]
+    for name, method in plan:
+        try:
+            inp = gen.make_workload(name, device=dev)
+            outs = gdn.alloc_outputs(inp.K, inp.V, inp.C)
+            fn = lambda: gdn.chunk_prepare(inp.K, inp.V, inp.beta, inp.g, inp.C, outputs=outs, method=method)
+            total_ms, _ = device_time_steps(fn, 20, 3, None)
+            ms = total_ms / 20
+            by = algorithmic_bytes_per_chunk(inp.C, inp.d_k, inp.d_v, inp.H_v // inp.H_k)
+            out[f"{name}:{method}"] = {"chunks_per_s": inp.n_chunks / (ms * 1e-3), "ms": ms,
+                                       "hbm_frac": inp.n_chunks * by / (ms * 1e-3) / 1e9 / hbm_peak}
+            del inp, outs
+        except Exception as exc:  # an unsupported extra must not lose the headline
+            out[f"{name}:{method}"] = {"error": repr(exc)}
+    return out
+
+
+def run_reference(args):
+    """The base contract's reference arm: the CPU oracle, as it stands, on the host cores."""
+    steps, warm = args.steps, args.warmup
+    budget_per_step = max(0.2, min(10.0, 120.0 / max(1, steps + warm)))
+    vals = []
+    info = None
+    for i in range(warm + steps):
+        info, wall = time_oracle(args.workload, budget_per_step)
+        if i >= warm:
+            vals.append((info["value"], wall))
+    value = float(np.mean([v for v, _ in vals]))
+    from paper_2606_06034_b200 import inputs as gen
+    cfg = gen.WORKLOADS[args.workload]
+    info["value"] = value
+    return {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps, "warmup": warm,
+        "ms_per_step": float(np.mean([w for _, w in vals])) * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic", "impl": "reference",
+        "config": {"workload": args.workload, "C": cfg["C"], "d_k": cfg["d_k"], "d_v": cfg["d_v"],
+                   "note": "each step is a bounded sample of the workload's chunks run through the fp64 CPU oracle"},
+        "cpu_baseline": info,
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=50)
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-extras", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        if rank == 0:
+            print(json.dumps(run_reference(args)), flush=True)
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (the library has no CPU path)")
+    torch.cuda.set_device(local_rank)
+    dist_ctx = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group(backend="nccl", device_id=torch.device("cuda", local_rank))
+        dist_ctx = dist
+    line = run_ours(args, rank, world, dist_ctx)
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if dist_ctx is not None:
+        dist_ctx.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
