@@ -33,7 +33,7 @@ using namespace sm100;
 
 constexpr int kTile = 128;            // rows per work item
 constexpr int kComputeThreads = 128;  // one per tile row
-constexpr int kThreads = 160;         // + one control warp
+constexpr int kThreads = 128;
 constexpr int kD = 128;               // d_k = d_v
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -45,7 +45,7 @@ constexpr uint32_t kR0 = 0, kR2 = 128, kAS = 192, kTmemCols = 256;
 
 #ifdef GDN_TRACE
 __device__ long long g_trace[4096];
-#define STAMP(slot) do { if (blockIdx.x == 0 && (tid == 0 || tid == 128) && trace_n < 60) { g_trace[(tid == 0 ? 0 : 2048) + trace_n * 2] = (slot); g_trace[(tid == 0 ? 0 : 2048) + trace_n * 2 + 1] = clock64(); ++trace_n; } } while (0)
+#define STAMP(slot) do { if (blockIdx.x == 0 && tid == 32 && trace_n < 100) { g_trace[trace_n * 2] = (slot); g_trace[trace_n * 2 + 1] = clock64(); ++trace_n; } } while (0)
 #else
 #define STAMP(slot) do { } while (0)
 #endif
@@ -255,10 +255,14 @@ __device__ __forceinline__ TileCoord decode_tile(uint32_t tile, const Params& p)
 
 template <int C, int NB, int MODE>
 __global__ void __launch_bounds__(kThreads, 2)
-chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const Params p) {
+chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmU,
+                const __grid_constant__ CUtensorMap tmT, const Params p) {
     using L = Smem<C, NB>;
     constexpr int NBP = L::NBP;
     constexpr int PC = C / 2;
+    constexpr int CPR = C / 8;   // 16-byte chunks of a packed bf16 row
+    constexpr int CPRF = C / 4;  // 16-byte chunks of an fp32 row
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* sK = smem + L::kK;
@@ -269,11 +273,12 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     float* sbeta = reinterpret_cast<float*>(smem + L::kBeta);
     float* sg = reinterpret_cast<float*>(smem + L::kG);
 
-    __shared__ uint64_t bar_k, bar_v, bar_mma, bar_opnd, bar_free;
+    __shared__ uint64_t bar_k, bar_v, bar_mma;
     __shared__ uint32_t tmem_base_s;
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
+    const int lane = tid & 31;
 #ifdef GDN_TRACE
     int trace_n = 0;
 #endif
@@ -282,11 +287,14 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         mbar_init(&bar_k, 1);
         mbar_init(&bar_v, 1);
         mbar_init(&bar_mma, 1);
-        mbar_init(&bar_opnd, kComputeThreads);
-        mbar_init(&bar_free, kComputeThreads);
         mbar_fence_init();
+        tma_prefetch_desc(&tmK);
+        tma_prefetch_desc(&tmV);
+        tma_prefetch_desc(&tmW);
+        tma_prefetch_desc(&tmU);
+        tma_prefetch_desc(&tmT);
     }
-    if (warp == 4) {
+    if (warp == 0) {
         tmem_alloc(&tmem_base_s, kTmemCols);
         tmem_relinquish();
     }
@@ -298,58 +306,261 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     const int N = p.N, S = p.S;
     // width of the band kept in fp32 (lb[]): the order N, or all of NB for forward substitution
     const int n_band = (MODE == INV_NEUMANN) ? N : NB;
-    // residual rounds: Z_{k+1} = (T0 + Z_k) E, k = 0..S-1, so that T = T0 + Z_S = T0 sum_{s<=S} E^s
-    const int n_rounds = (MODE == INV_NEUMANN) ? S : 0;
+    const uint32_t n_tiles = static_cast<uint32_t>(p.n_tiles);
 
-    if (warp == 4) {
-        // ------------------------------------------------------------------ control warp
-        if ((tid & 31) == 0) {
-            tma_prefetch_desc(&tmK);
-            tma_prefetch_desc(&tmV);
-            uint32_t par_kv = 0, par_opnd = 0, par_free = 0, n_commit = 0;
-            bool ok = true;
-            const uint32_t idesc_g = instr_desc(128, 128, 1, 1, 0, 0, 1);
-            const uint32_t idesc_c = instr_desc(128, C, 1, 1, 0, 1, 1);
-            const uint32_t idesc_w = instr_desc(128, 128, 1, 1, 0, 1, 1);
-            const uint32_t sK_a = smem_u32(sK), sV_a = smem_u32(sV), sEB_a = smem_u32(sEB);
-            uint32_t tile = blockIdx.x;
-            const uint32_t n_tiles = static_cast<uint32_t>(p.n_tiles);
-            if (tile < n_tiles) {
-                const TileCoord c = decode_tile(tile, p);
-                mbar_arrive_expect_tx(&bar_k, 32768);
-                tma_load_3d(sK, &tmK, &bar_k, 0, c.t0, static_cast<int>(c.bhk));
-                tma_load_3d(sK + 16384, &tmK, &bar_k, 64, c.t0, static_cast<int>(c.bhk));
-                mbar_arrive_expect_tx(&bar_v, 32768);
-                tma_load_3d(sV, &tmV, &bar_v, 0, c.t0, static_cast<int>(c.bhv));
-                tma_load_3d(sV + 16384, &tmV, &bar_v, 64, c.t0, static_cast<int>(c.bhv));
-            }
-            bool first = true;
-            for (; tile < n_tiles; tile += gridDim.x) {
-                const uint32_t next = tile + gridDim.x;
-                const bool has_next = next < n_tiles;
-                TileCoord nc{0, 0, 0};
-                if (has_next) nc = decode_tile(next, p);
-                STAMP(101);
-                if (!wait_bar(&bar_k, par_kv)) { ok = false; break; }
-                STAMP(102);
-                if (!first) {  // the previous tile's accumulators have been read out
-                    if (!wait_bar(&bar_free, par_free)) { ok = false; break; }
-                    par_free ^= 1;
-                }
-                first = false;
+    // Thread t owns tile row t. Thread 0 also issues every TMA load and every tcgen05.mma, right after the
+    // CTA barrier that says all rows of the operand are in place.
+    const int t = tid;
+    const int il = t % C;   // row inside its chunk
+    const int cb = t - il;  // first tile row of the chunk
+    const int wrow0 = t - lane;
+    const uint32_t lane_base = tmem + (static_cast<uint32_t>(warp * 32) << 16);
+    const uint32_t scratch_a = smem_u32(smem + L::kEB);
+    const uint32_t br_row = smem_u32(smem + L::kBR) + t * (2 * C);
+    const uint32_t sK_a = smem_u32(sK), sV_a = smem_u32(sV), sEB_a = smem_u32(sEB);
+    const uint32_t idesc_g = instr_desc(128, 128, 1, 1, 0, 0, 1);
+    const uint32_t idesc_c = instr_desc(128, C, 1, 1, 0, 1, 1);
+    const uint32_t idesc_w = instr_desc(128, 128, 1, 1, 0, 1, 1);
+    uint32_t par_mma = 0, par_kv = 0;
+    bool ok = true;
+
+    {  // the A-operand slot keeps zeros outside the diagonal blocks for the whole kernel
+        uint32_t z[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) z[i] = 0u;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) tmem_st16(lane_base + kAS + c * 16, z);
+        tmem_wait_st();
+    }
+    if (t == 0 && blockIdx.x < n_tiles) {
+        const TileCoord c = decode_tile(blockIdx.x, p);
+        mbar_arrive_expect_tx(&bar_k, 32768);
+        tma_load_3d(sK, &tmK, &bar_k, 0, c.t0, c.bhk);
+        tma_load_3d(sK + 16384, &tmK, &bar_k, 64, c.t0, c.bhk);
+        mbar_arrive_expect_tx(&bar_v, 32768);
+        tma_load_3d(sV, &tmV, &bar_v, 0, c.t0, c.bhv);
+        tma_load_3d(sV + 16384, &tmV, &bar_v, 64, c.t0, c.bhv);
+    }
+
+    for (uint32_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        const TileCoord tc = decode_tile(tile, p);
+        const uint32_t next = tile + gridDim.x;
+        const bool has_next = next < n_tiles;
+        const bool row_valid = (tc.t0 + t) < p.T;
+        const long long grow = (long long)tc.bhv * p.T + tc.t0 + t;  // global token row (value-head space)
+
+        STAMP(1);
+        float bi = 0.f, gi_ = 0.f;
+        if (row_valid) {
+            bi = __ldg(p.beta + grow);
+            gi_ = __ldg(p.g + grow);
+        }
+        // the previous tile's bulk stores have finished reading the staging slices
+        if (lane == 0) tma_store_wait_read<0>();
+        tc_fence_before_sync();
+        compute_barrier();  // everyone is done with the previous tile's shared arrays and accumulators
+        if (t == 0) {
+            // G = K K^T into R0..R1 (128 columns)
+            if (!wait_bar(&bar_k, par_kv)) ok = false;
+            if (ok) {
                 tc_fence_after_sync();
-                // G = K K^T into R0..R1 (128 columns)
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
                     const uint64_t d = smem_desc(sK_a + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024, SWZ_128B);
                     mma_f16_ss(tmem + kR0, d, d, idesc_g, ks > 0);
                 }
                 mma_commit(&bar_mma);
-                ++n_commit;
-                STAMP(103);
-                for (int r = 0; r < n_rounds; ++r) {
-                    if (!wait_bar(&bar_opnd, par_opnd)) { ok = false; break; }
-                    par_opnd ^= 1;
+            }
+        }
+        sbeta[t] = bi;
+        sg[t] = gi_;
+#pragma unroll
+        for (int e = 0; e < NBP; ++e) sSH[t * NBP + e] = 0.f;
+        if (t < 8) {
+#pragma unroll
+            for (int e = 0; e < NBP; ++e) sSH[(kTile + t) * NBP + e] = 0.f;
+        }
+        compute_barrier();
+
+        STAMP(2);
+        // ---- A-build: row of Abar from the Gram block in TMEM
+        if (!wait_bar(&bar_mma, par_mma)) { ok = false; break; }
+        par_mma ^= 1;
+        STAMP(3);
+        tc_fence_after_sync();
+        float a[C];
+        load_diag_block<C>(lane_base, kR0, t, a);
+        {
+            const float gs = gi_ * kLog2e;
+            const float nbi = -bi;
+            const float4* sg4 = reinterpret_cast<const float4*>(sg + cb);
+#pragma unroll
+            for (int j4 = 0; j4 < C / 4; ++j4) {
+                const float4 gq = sg4[j4];
+                const float gj[4] = {gq.x, gq.y, gq.z, gq.w};
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int j = j4 * 4 + q;
+                    const float v = nbi * fast_exp2(fmaf(-gj[q], kLog2e, gs)) * a[j];
+                    a[j] = (j < il) ? v : 0.f;
+                }
+            }
+        }
+
+        STAMP(4);
+        float lb[NB + 1];  // lb[d] = L[i][i-d], the band of T0 - I (or of T - I after forward substitution)
+#pragma unroll
+        for (int e = 0; e <= NB; ++e) lb[e] = 0.f;
+
+        const uint32_t rowf = scratch_a + t * (4 * C);  // private fp32 row
+        if constexpr (MODE == INV_NEUMANN) {
+            // ---- ab[e] = Abar[i][i-e] through the private fp32 row
+            float ab[NB + 1];
+#pragma unroll
+            for (int c = 0; c < CPRF; ++c)
+                sts128(rowf + (swz<CPRF>(t, c) << 4), __float_as_uint(a[c * 4 + 0]), __float_as_uint(a[c * 4 + 1]),
+                       __float_as_uint(a[c * 4 + 2]), __float_as_uint(a[c * 4 + 3]));
+            ab[0] = 0.f;
+#pragma unroll
+            for (int e = 1; e <= NB; ++e) {
+                const int j = il - e;
+                ab[e] = (j >= 0) ? lds32f(rowf + (swz<CPRF>(t, j >> 2) << 4) + (j & 3) * 4) : 0.f;
+            }
+            // ---- band of the masked Neumann sum by distance recursion
+            lb[1] = ab[1];
+            sRB[t * NBP + 0] = lb[1];
+#pragma unroll
+            for (int d = 2; d <= NB; ++d) {
+                compute_barrier();
+                float v = ab[d];
+#pragma unroll
+                for (int e = 1; e < d; ++e) {
+                    const int r = (t - e) > 0 ? (t - e) : 0;
+                    v = fmaf(ab[e], sRB[r * NBP + (d - e - 1)], v);
+                }
+                lb[d] = (d <= N) ? v : 0.f;
+                if (d < NB) sRB[t * NBP + (d - 1)] = lb[d];
+            }
+            // column form: SH[j][e-1] = L[j+e][j]
+#pragma unroll
+            for (int e = 1; e <= NB; ++e)
+                if (il - e >= 0) sSH[(t - e) * NBP + (e - 1)] = lb[e];
+            compute_barrier();
+
+            STAMP(5);
+            // ---- E = Abar + Abar L on i-j > N (in place over a[])
+#pragma unroll
+            for (int j = 0; j < C; ++j) {
+                float v = a[j];
+                if constexpr (NBP == 4) {
+                    const float4 c4 = *reinterpret_cast<const float4*>(sSH + (cb + j) * 4);
+                    if (j + 1 < C) v = fmaf(a[(j + 1 < C) ? j + 1 : j], c4.x, v);
+                    if (j + 2 < C) v = fmaf(a[(j + 2 < C) ? j + 2 : j], c4.y, v);
+                    if (j + 3 < C) v = fmaf(a[(j + 3 < C) ? j + 3 : j], c4.z, v);
+                } else {
+                    const float4 c4 = *reinterpret_cast<const float4*>(sSH + (cb + j) * 8);
+                    const float4 d4 = *reinterpret_cast<const float4*>(sSH + (cb + j) * 8 + 4);
+                    const float cc[7] = {c4.x, c4.y, c4.z, c4.w, d4.x, d4.y, d4.z};
+#pragma unroll
+                    for (int e = 1; e <= NB; ++e)
+                        if (j + e < C) v = fmaf(a[(j + e < C) ? j + e : j], cc[e - 1], v);
+                }
+                a[j] = (il - j > N) ? v : 0.f;
+            }
+            // E as B operand (MN-major, no swizzle): 16-byte chunk c of row t at c * 2048 + t * 16
+            if (S >= 1) {
+#pragma unroll
+                for (int c = 0; c < C / 8; ++c) {
+                    uint4 v;
+                    v.x = pack_bf16x2(a[c * 8 + 0], a[c * 8 + 1]);
+                    v.y = pack_bf16x2(a[c * 8 + 2], a[c * 8 + 3]);
+                    v.z = pack_bf16x2(a[c * 8 + 4], a[c * 8 + 5]);
+                    v.w = pack_bf16x2(a[c * 8 + 6], a[c * 8 + 7]);
+                    *reinterpret_cast<uint4*>(sEB + c * 2048 + t * 16) = v;
+                }
+            }
+        } else {
+            // ---- forward substitution (Eq. 2-3). The private fp32 rows hold Abar; thread = column il of its chunk.
+#pragma unroll
+            for (int c = 0; c < CPRF; ++c)
+                sts128(rowf + (swz<CPRF>(t, c) << 4), __float_as_uint(a[c * 4 + 0]), __float_as_uint(a[c * 4 + 1]),
+                       __float_as_uint(a[c * 4 + 2]), __float_as_uint(a[c * 4 + 3]));
+            compute_barrier();
+            float xcol[C];  // xcol[k] = T[k][il]
+#pragma unroll
+            for (int i = 0; i < C; ++i) {
+                float acc = 0.f;
+                const uint32_t ri = scratch_a + (cb + i) * (4 * C);
+#pragma unroll
+                for (int k4 = 0; k4 < (i + 3) / 4; ++k4) {
+                    const uint4 q = lds128(ri + (swz<CPRF>(i, k4) << 4));  // (cb + i) and i agree in the swizzle bits
+                    if (k4 * 4 + 0 < i) acc = fmaf(__uint_as_float(q.x), xcol[k4 * 4 + 0], acc);
+                    if (k4 * 4 + 1 < i) acc = fmaf(__uint_as_float(q.y), xcol[(k4 * 4 + 1 < C) ? k4 * 4 + 1 : 0], acc);
+                    if (k4 * 4 + 2 < i) acc = fmaf(__uint_as_float(q.z), xcol[(k4 * 4 + 2 < C) ? k4 * 4 + 2 : 0], acc);
+                    if (k4 * 4 + 3 < i) acc = fmaf(__uint_as_float(q.w), xcol[(k4 * 4 + 3 < C) ? k4 * 4 + 3 : 0], acc);
+                }
+                xcol[i] = (i > il) ? acc : ((i == il) ? 1.f : 0.f);
+            }
+            compute_barrier();  // everyone has read Abar
+#pragma unroll
+            for (int i = 0; i < C; ++i) {
+                const uint32_t addr = scratch_a + (cb + i) * (4 * C) + (swz<CPRF>(i, il >> 2) << 4) + (il & 3) * 4;
+                asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(xcol[i]) : "memory");
+            }
+            compute_barrier();
+            // back to rows: a[] = far part, lb[] = band part
+#pragma unroll
+            for (int c = 0; c < CPRF; ++c) {
+                const uint4 q = lds128(rowf + (swz<CPRF>(t, c) << 4));
+                a[c * 4 + 0] = __uint_as_float(q.x);
+                a[c * 4 + 1] = __uint_as_float(q.y);
+                a[c * 4 + 2] = __uint_as_float(q.z);
+                a[c * 4 + 3] = __uint_as_float(q.w);
+            }
+#pragma unroll
+            for (int e = 1; e <= NB; ++e) {
+                const int j = il - e;
+                lb[e] = (j >= 0) ? lds32f(rowf + (swz<CPRF>(t, j >> 2) << 4) + (j & 3) * 4) : 0.f;
+            }
+#pragma unroll
+            for (int j = 0; j < C; ++j) a[j] = (il - j > NB) ? a[j] : 0.f;
+            compute_barrier();  // the fp32 rows are dead; the packed rows may overwrite them
+        }
+
+        STAMP(6);
+        // ---- packed bf16 forms of the band: keep-mask (0 on the band and diagonal) and I + L
+        uint32_t keep[PC], bpT[PC];
+        {
+            uint16_t vals[NB + 1];
+#pragma unroll
+            for (int e = 0; e <= NB; ++e) vals[e] = 0xFFFFu;
+            build_band_row<C, NB>(br_row, t, il, n_band, vals, keep);
+#pragma unroll
+            for (int i = 0; i < PC; ++i) keep[i] = ~keep[i];
+            vals[0] = 0x3F80u;  // 1.0
+#pragma unroll
+            for (int e = 1; e <= NB; ++e) vals[e] = bf16_bits(lb[e]);
+            build_band_row<C, NB>(br_row, t, il, n_band, vals, bpT);
+        }
+
+        STAMP(7);
+        if constexpr (MODE == INV_NEUMANN) {
+            // ---- residual rounds: A_k = T0 + Z_k (bf16, TMEM), Z_{k+1} = A_k E, so that T = T0 + Z_S
+            for (int k = 0; k < S; ++k) {
+                uint32_t pk[PC];
+                if (k == 0) {
+#pragma unroll
+                    for (int i = 0; i < PC; ++i) pk[i] = bpT[i];
+                } else {
+#pragma unroll
+                    for (int i = 0; i < PC; ++i) pk[i] = (pack_bf16x2(a[2 * i], a[2 * i + 1]) & keep[i]) | bpT[i];
+                }
+                store_a_operand<C, false>(lane_base + kAS, t, pk);
+                fence_proxy_async_smem();
+                tmem_wait_st();
+                tc_fence_before_sync();
+                compute_barrier();
+                if (t == 0) {
                     tc_fence_after_sync();
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks) {
@@ -357,398 +568,158 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                         mma_f16_ts(tmem + kR2, tmem + kAS + ks * 8, bd, idesc_c, ks > 0);
                     }
                     mma_commit(&bar_mma);
-                    ++n_commit;
                 }
-                if (!ok) break;
-                // W = (hi + lo) K: A operands in TMEM (AS: high bf16 half, R2: low half of the band),
-                // B = the K tile read as an MN-major operand (both 64-column sub-tiles, N = 128)
-                if (!wait_bar(&bar_opnd, par_opnd)) { ok = false; break; }
-                par_opnd ^= 1;
-                STAMP(104);
-                tc_fence_after_sync();
-#pragma unroll
-                for (int ks = 0; ks < 16; ++ks) {
-                    const uint64_t bd = smem_desc(sK_a + (ks & 7) * 2048, 16384, 1024, SWZ_128B);
-                    mma_f16_ts(tmem + kR0, tmem + ((ks < 8) ? kAS : kR2) + (ks & 7) * 8, bd, idesc_w, ks > 0);
-                }
-                mma_commit(&bar_mma);
-                ++n_commit;
-                STAMP(105);
-                if (!wait_bar(&bar_v, par_kv)) { ok = false; break; }
-                par_kv ^= 1;
-                STAMP(106);
-                // W accumulator read out => the W products are complete => the K tile is free
-                if (!wait_bar(&bar_opnd, par_opnd)) { ok = false; break; }
-                par_opnd ^= 1;
-                if (has_next) {
-                    mbar_arrive_expect_tx(&bar_k, 32768);
-                    tma_load_3d(sK, &tmK, &bar_k, 0, nc.t0, static_cast<int>(nc.bhk));
-                    tma_load_3d(sK + 16384, &tmK, &bar_k, 64, nc.t0, static_cast<int>(nc.bhk));
-                }
-                tc_fence_after_sync();
-#pragma unroll
-                for (int ks = 0; ks < 16; ++ks) {
-                    const uint64_t bd = smem_desc(sV_a + (ks & 7) * 2048, 16384, 1024, SWZ_128B);
-                    mma_f16_ts(tmem + kR0, tmem + ((ks < 8) ? kAS : kR2) + (ks & 7) * 8, bd, idesc_w, ks > 0);
-                }
-                mma_commit(&bar_mma);
-                ++n_commit;
-                STAMP(107);
-                if (has_next) {  // U products complete => the V tile is free
-                    if (!wait_bar(&bar_mma, (n_commit - 1) & 1)) { ok = false; break; }
-                    STAMP(108);
-                    mbar_arrive_expect_tx(&bar_v, 32768);
-                    tma_load_3d(sV, &tmV, &bar_v, 0, nc.t0, static_cast<int>(nc.bhv));
-                    tma_load_3d(sV + 16384, &tmV, &bar_v, 64, nc.t0, static_cast<int>(nc.bhv));
-                }
-            }
-            if (!ok) atomicExch(p.status, GDN_ERR_TIMEOUT);
-        }
-    } else {
-        // ------------------------------------------------------------------ compute warps
-        const int t = tid;                 // tile row
-        const int il = t % C;              // row inside its chunk
-        const int cb = t - il;             // first tile row of the chunk
-        const uint32_t lane_base = tmem + (static_cast<uint32_t>(warp * 32) << 16);
-        const uint32_t scratch_a = smem_u32(smem + L::kEB);
-        const uint32_t br_row = smem_u32(smem + L::kBR) + t * (2 * C);
-        uint32_t par_mma = 0;
-        bool ok = true;
-
-        {  // the A-operand slot keeps zeros outside the diagonal blocks for the whole kernel
-            uint32_t z[16];
-#pragma unroll
-            for (int i = 0; i < 16; ++i) z[i] = 0u;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) tmem_st16(lane_base + kAS + c * 16, z);
-            tmem_wait_st();
-        }
-
-        for (uint32_t tile = blockIdx.x; tile < static_cast<uint32_t>(p.n_tiles) && ok; tile += gridDim.x) {
-            const TileCoord tc = decode_tile(tile, p);
-            const bool row_valid = (tc.t0 + t) < p.T;
-            const long long grow = (long long)tc.bhv * p.T + tc.t0 + t;  // global token row (value-head space)
-
-            STAMP(1);
-            float bi = 0.f, gi_ = 0.f;
-            if (row_valid) {
-                bi = __ldg(p.beta + grow);
-                gi_ = __ldg(p.g + grow);
-            }
-            compute_barrier();  // everyone is done with the previous tile's shared arrays
-            sbeta[t] = bi;
-            sg[t] = gi_;
-#pragma unroll
-            for (int e = 0; e < NBP; ++e) sSH[t * NBP + e] = 0.f;
-            if (t < 8) {
-#pragma unroll
-                for (int e = 0; e < NBP; ++e) sSH[(kTile + t) * NBP + e] = 0.f;
-            }
-            compute_barrier();
-
-            STAMP(2);
-            // ---- A-build: row of Abar from the Gram block in TMEM
-            if (!wait_bar(&bar_mma, par_mma)) { ok = false; break; }
-            par_mma ^= 1;
-            STAMP(3);
-            tc_fence_after_sync();
-            float a[C];
-            load_diag_block<C>(lane_base, kR0, t, a);
-            {
-                const float gs = gi_ * kLog2e;
-                const float nbi = -bi;
-                const float4* sg4 = reinterpret_cast<const float4*>(sg + cb);
-#pragma unroll
-                for (int j4 = 0; j4 < C / 4; ++j4) {
-                    const float4 gq = sg4[j4];
-                    const float gj[4] = {gq.x, gq.y, gq.z, gq.w};
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const int j = j4 * 4 + q;
-                        const float v = nbi * fast_exp2(fmaf(-gj[q], kLog2e, gs)) * a[j];
-                        a[j] = (j < il) ? v : 0.f;
-                    }
-                }
-            }
-
-            STAMP(4);
-            float lb[NB + 1];  // lb[d] = L[i][i-d], the band of T0 - I (or of T - I after forward substitution)
-#pragma unroll
-            for (int e = 0; e <= NB; ++e) lb[e] = 0.f;
-
-            if constexpr (MODE == INV_NEUMANN) {
-                // ---- ab[e] = Abar[i][i-e] through the private fp32 row
-                float ab[NB + 1];
-                {
-                    constexpr int CPRF = C / 4;  // 16-byte chunks of an fp32 row
-                    const uint32_t rowf = scratch_a + t * (4 * C);
-#pragma unroll
-                    for (int c = 0; c < CPRF; ++c)
-                        sts128(rowf + (swz<CPRF>(t, c) << 4), __float_as_uint(a[c * 4 + 0]), __float_as_uint(a[c * 4 + 1]),
-                               __float_as_uint(a[c * 4 + 2]), __float_as_uint(a[c * 4 + 3]));
-                    ab[0] = 0.f;
-#pragma unroll
-                    for (int e = 1; e <= NB; ++e) {
-                        const int j = il - e;
-                        ab[e] = (j >= 0) ? lds32f(rowf + (swz<CPRF>(t, j >> 2) << 4) + (j & 3) * 4) : 0.f;
-                    }
-                }
-                // ---- band of the masked Neumann sum by distance recursion
-                lb[1] = ab[1];
-                sRB[t * NBP + 0] = lb[1];
-#pragma unroll
-                for (int d = 2; d <= NB; ++d) {
-                    compute_barrier();
-                    float v = ab[d];
-#pragma unroll
-                    for (int e = 1; e < d; ++e) {
-                        const int r = (t - e) > 0 ? (t - e) : 0;
-                        v = fmaf(ab[e], sRB[r * NBP + (d - e - 1)], v);
-                    }
-                    lb[d] = (d <= N) ? v : 0.f;
-                    if (d < NB) sRB[t * NBP + (d - 1)] = lb[d];
-                }
-                // column form: SH[j][e-1] = L[j+e][j]
-#pragma unroll
-                for (int e = 1; e <= NB; ++e)
-                    if (il - e >= 0) sSH[(t - e) * NBP + (e - 1)] = lb[e];
-                compute_barrier();
-
-                STAMP(5);
-                // ---- E = Abar + Abar L on i-j > N (in place over a[])
-#pragma unroll
-                for (int j = 0; j < C; ++j) {
-                    float v = a[j];
-                    if constexpr (NBP == 4) {
-                        const float4 c4 = *reinterpret_cast<const float4*>(sSH + (cb + j) * 4);
-                        if (j + 1 < C) v = fmaf(a[(j + 1 < C) ? j + 1 : j], c4.x, v);
-                        if (j + 2 < C) v = fmaf(a[(j + 2 < C) ? j + 2 : j], c4.y, v);
-                        if (j + 3 < C) v = fmaf(a[(j + 3 < C) ? j + 3 : j], c4.z, v);
-                    } else {
-                        const float4 c4 = *reinterpret_cast<const float4*>(sSH + (cb + j) * 8);
-                        const float4 d4 = *reinterpret_cast<const float4*>(sSH + (cb + j) * 8 + 4);
-                        const float cc[7] = {c4.x, c4.y, c4.z, c4.w, d4.x, d4.y, d4.z};
-#pragma unroll
-                        for (int e = 1; e <= NB; ++e)
-                            if (j + e < C) v = fmaf(a[(j + e < C) ? j + e : j], cc[e - 1], v);
-                    }
-                    a[j] = (il - j > N) ? v : 0.f;
-                }
-                // E as B operand (MN-major, no swizzle): 16-byte chunk c of row t at c * 2048 + t * 16
-                if (S >= 1) {
-#pragma unroll
-                    for (int c = 0; c < C / 8; ++c) {
-                        uint4 v;
-                        v.x = pack_bf16x2(a[c * 8 + 0], a[c * 8 + 1]);
-                        v.y = pack_bf16x2(a[c * 8 + 2], a[c * 8 + 3]);
-                        v.z = pack_bf16x2(a[c * 8 + 4], a[c * 8 + 5]);
-                        v.w = pack_bf16x2(a[c * 8 + 6], a[c * 8 + 7]);
-                        *reinterpret_cast<uint4*>(sEB + c * 2048 + t * 16) = v;
-                    }
-                }
-            } else {
-                // ---- forward substitution (Eq. 2-3). The private fp32 rows hold Abar; thread = column il of its chunk.
-                constexpr int CPRF = C / 4;
-                const uint32_t rowf = scratch_a + t * (4 * C);
-#pragma unroll
-                for (int c = 0; c < CPRF; ++c)
-                    sts128(rowf + (swz<CPRF>(t, c) << 4), __float_as_uint(a[c * 4 + 0]), __float_as_uint(a[c * 4 + 1]),
-                           __float_as_uint(a[c * 4 + 2]), __float_as_uint(a[c * 4 + 3]));
-                compute_barrier();
-                float xcol[C];  // xcol[k] = T[k][il]
-#pragma unroll
-                for (int i = 0; i < C; ++i) {
-                    float acc = 0.f;
-                    const uint32_t ri = scratch_a + (cb + i) * (4 * C);
-#pragma unroll
-                    for (int k4 = 0; k4 < (i + 3) / 4; ++k4) {
-                        const uint4 q = lds128(ri + (swz<CPRF>(i, k4) << 4));  // (cb + i) and i agree in the swizzle bits
-                        if (k4 * 4 + 0 < i) acc = fmaf(__uint_as_float(q.x), xcol[k4 * 4 + 0], acc);
-                        if (k4 * 4 + 1 < i) acc = fmaf(__uint_as_float(q.y), xcol[(k4 * 4 + 1 < C) ? k4 * 4 + 1 : 0], acc);
-                        if (k4 * 4 + 2 < i) acc = fmaf(__uint_as_float(q.z), xcol[(k4 * 4 + 2 < C) ? k4 * 4 + 2 : 0], acc);
-                        if (k4 * 4 + 3 < i) acc = fmaf(__uint_as_float(q.w), xcol[(k4 * 4 + 3 < C) ? k4 * 4 + 3 : 0], acc);
-                    }
-                    xcol[i] = (i > il) ? acc : ((i == il) ? 1.f : 0.f);
-                }
-                compute_barrier();  // everyone has read Abar
-#pragma unroll
-                for (int i = 0; i < C; ++i) {
-                    const uint32_t addr = scratch_a + (cb + i) * (4 * C) + (swz<CPRF>(i, il >> 2) << 4) + (il & 3) * 4;
-                    asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(xcol[i]) : "memory");
-                }
-                compute_barrier();
-                // back to rows: a[] = far part, lb[] = band part
-#pragma unroll
-                for (int c = 0; c < CPRF; ++c) {
-                    const uint4 q = lds128(rowf + (swz<CPRF>(t, c) << 4));
-                    a[c * 4 + 0] = __uint_as_float(q.x);
-                    a[c * 4 + 1] = __uint_as_float(q.y);
-                    a[c * 4 + 2] = __uint_as_float(q.z);
-                    a[c * 4 + 3] = __uint_as_float(q.w);
-                }
-#pragma unroll
-                for (int e = 1; e <= NB; ++e) {
-                    const int j = il - e;
-                    lb[e] = (j >= 0) ? lds32f(rowf + (swz<CPRF>(t, j >> 2) << 4) + (j & 3) * 4) : 0.f;
-                }
-#pragma unroll
-                for (int j = 0; j < C; ++j) a[j] = (il - j > NB) ? a[j] : 0.f;
-                compute_barrier();  // the fp32 rows are dead; the packed rows may overwrite them
-            }
-
-            STAMP(6);
-            // ---- packed bf16 forms of the band: keep-mask (0 on the band and diagonal) and I + L
-            uint32_t keep[PC], bpT[PC];
-            {
-                uint16_t vals[NB + 1];
-#pragma unroll
-                for (int e = 0; e <= NB; ++e) vals[e] = 0xFFFFu;
-                build_band_row<C, NB>(br_row, t, il, n_band, vals, keep);
-#pragma unroll
-                for (int i = 0; i < PC; ++i) keep[i] = ~keep[i];
-                vals[0] = 0x3F80u;  // 1.0
-#pragma unroll
-                for (int e = 1; e <= NB; ++e) vals[e] = bf16_bits(lb[e]);
-                build_band_row<C, NB>(br_row, t, il, n_band, vals, bpT);
-            }
-
-            STAMP(7);
-            if constexpr (MODE == INV_NEUMANN) {
-                // ---- residual rounds: A_k = T0 + Z_k (bf16, TMEM), Z_{k+1} = A_k E
-                for (int k = 0; k < S; ++k) {
-                    uint32_t pk[PC];
-                    if (k == 0) {
-#pragma unroll
-                        for (int i = 0; i < PC; ++i) pk[i] = bpT[i];
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < PC; ++i) pk[i] = (pack_bf16x2(a[2 * i], a[2 * i + 1]) & keep[i]) | bpT[i];
-                    }
-                    store_a_operand<C, false>(lane_base + kAS, t, pk);
-                    fence_proxy_async_smem();
-                    tmem_wait_st();
-                    tc_fence_before_sync();
-                    mbar_arrive(&bar_opnd);
-                    if (!wait_bar(&bar_mma, par_mma)) { ok = false; break; }
-                    par_mma ^= 1;
-                    tc_fence_after_sync();
-                    load_cols<C>(lane_base, kR2, a);
-                }
-                if (!ok) break;
-                if (S == 0) {
-#pragma unroll
-                    for (int j = 0; j < C; ++j) a[j] = 0.f;
-                }
-            }
-            // a[] = far row (T - I - L)
-
-            STAMP(8);
-            // ---- T row -> Tinv. Rows go through the private packed rows so that each store instruction of a
-            // warp covers whole 128-byte lines (the warp's 32 rows are contiguous in global memory).
-            if (p.Tinv != nullptr) {
-                constexpr int CPR = C / 8;           // 16-byte chunks per row
-                constexpr int RPI = 32 / CPR;        // rows per store instruction
-#pragma unroll
-                for (int c = 0; c < CPR; ++c) {
-                    sts128(br_row + (swz<CPR>(t, c) << 4),
-                           (pack_bf16x2(a[c * 8 + 0], a[c * 8 + 1]) & keep[c * 4 + 0]) | bpT[c * 4 + 0],
-                           (pack_bf16x2(a[c * 8 + 2], a[c * 8 + 3]) & keep[c * 4 + 1]) | bpT[c * 4 + 1],
-                           (pack_bf16x2(a[c * 8 + 4], a[c * 8 + 5]) & keep[c * 4 + 2]) | bpT[c * 4 + 2],
-                           (pack_bf16x2(a[c * 8 + 6], a[c * 8 + 7]) & keep[c * 4 + 3]) | bpT[c * 4 + 3]);
-                }
-                __syncwarp();
-                const int lane = t & 31;
-                const int wrow0 = t - lane;  // first tile row of this warp
-                const uint32_t br_base = smem_u32(smem + L::kBR);
-                uint4* gbase = reinterpret_cast<uint4*>(p.Tinv + ((long long)tc.bhv * p.T + tc.t0 + wrow0) * C);
-#pragma unroll
-                for (int it = 0; it < CPR; ++it) {
-                    const int r = wrow0 + it * RPI + lane / CPR;  // tile row read by this lane
-                    const int c = lane % CPR;
-                    const uint4 v = lds128(br_base + r * (2 * C) + (swz<CPR>(r, c) << 4));
-                    if (tc.t0 + r < p.T) gbase[it * 32 + lane] = v;
-                }
-                __syncwarp();
-            }
-
-            STAMP(9);
-            // ---- A operands for W/U: T diag(beta) = hi + lo, hi over the whole row, lo only on band + diagonal
-            {
-                float tb[NB + 1];
-                tb[0] = bi;
-#pragma unroll
-                for (int e = 1; e <= NB; ++e) tb[e] = (il - e >= 0) ? lb[e] * sbeta[(t - e) > 0 ? (t - e) : 0] : 0.f;
-                uint16_t hi[NB + 1], lo[NB + 1];
-#pragma unroll
-                for (int e = 0; e <= NB; ++e) {
-                    hi[e] = bf16_bits(tb[e]);
-                    lo[e] = bf16_bits(tb[e] - bf16_bits_to_f32(hi[e]));
-                }
-                uint32_t bp[PC], pk[PC];
-                build_band_row<C, NB>(br_row, t, il, n_band, hi, bp);
-                const float2* sb2 = reinterpret_cast<const float2*>(sbeta + cb);
-#pragma unroll
-                for (int i = 0; i < PC; ++i) {
-                    const float2 bb = sb2[i];
-                    pk[i] = (pack_bf16x2(a[2 * i] * bb.x, a[2 * i + 1] * bb.y) & keep[i]) | bp[i];
-                }
-                store_a_operand<C, false>(lane_base + kAS, t, pk);
-                build_band_row<C, NB>(br_row, t, il, n_band, lo, bp);
-                store_a_operand<C, true>(lane_base + kR2, t, bp);
-                tmem_wait_st();
-                tc_fence_before_sync();
-                mbar_arrive(&bar_opnd);
-            }
-
-            STAMP(10);
-            // ---- W, then U: accumulator rows -> bf16 -> 16-byte stores (one 256-byte row per thread)
-#pragma unroll 1
-            for (int half = 0; half < 2; ++half) {
                 if (!wait_bar(&bar_mma, par_mma)) { ok = false; break; }
                 par_mma ^= 1;
                 tc_fence_after_sync();
-                STAMP(11 + half * 3);
-                uint32_t o[64];
+                load_cols<C>(lane_base, kR2, a);
+            }
+            if (!ok) break;
+            if (S == 0) {
 #pragma unroll
-                for (int c0 = 0; c0 < 128; c0 += 32) {
-                    uint32_t r[32];
-                    tmem_ld32(lane_base + kR0 + c0, r);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) o[c0 / 2 + i] = pack_bf16x2(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
-                }
-                tc_fence_before_sync();
-                mbar_arrive(half == 0 ? &bar_opnd : &bar_free);
-                STAMP(12 + half * 3);
-                {
-                    // stage the warp's 32 rows (256 bytes each) in its 8 KB slice of the scratch region, then
-                    // store whole 512-byte runs per instruction
-                    const int lane = t & 31;
-                    const int wrow0 = t - lane;
-                    const uint32_t slice = scratch_a + wrow0 * 256;
-#pragma unroll
-                    for (int c = 0; c < 16; ++c)
-                        sts128(slice + lane * 256 + ((c ^ (lane & 7)) << 4), o[c * 4 + 0], o[c * 4 + 1], o[c * 4 + 2], o[c * 4 + 3]);
-                    __syncwarp();
-                    uint4* gbase = reinterpret_cast<uint4*>((half == 0 ? p.W : p.U) + ((long long)tc.bhv * p.T + tc.t0 + wrow0) * kD);
-#pragma unroll
-                    for (int it = 0; it < 16; ++it) {
-                        const int r = it * 2 + (lane >> 4);
-                        const int c = lane & 15;
-                        const uint4 v = lds128(slice + r * 256 + ((c ^ (r & 7)) << 4));
-                        if (tc.t0 + wrow0 + r < p.T) gbase[it * 32 + lane] = v;
-                    }
-                    __syncwarp();
-                }
-                STAMP(13 + half * 3);
+                for (int j = 0; j < C; ++j) a[j] = 0.f;
             }
         }
-        if (!ok) atomicExch(p.status, GDN_ERR_TIMEOUT);
+        // a[] = far row (T - I - L)
+
+        STAMP(9);
+        // ---- A operands for W/U: T diag(beta) = hi + lo, hi over the whole row, lo only on band + diagonal
+        {
+            float tb[NB + 1];
+            tb[0] = bi;
+#pragma unroll
+            for (int e = 1; e <= NB; ++e) tb[e] = (il - e >= 0) ? lb[e] * sbeta[(t - e) > 0 ? (t - e) : 0] : 0.f;
+            uint16_t hi[NB + 1], lo[NB + 1];
+#pragma unroll
+            for (int e = 0; e <= NB; ++e) {
+                hi[e] = bf16_bits(tb[e]);
+                lo[e] = bf16_bits(tb[e] - bf16_bits_to_f32(hi[e]));
+            }
+            uint32_t bp[PC], pk[PC];
+            build_band_row<C, NB>(br_row, t, il, n_band, hi, bp);
+            const float2* sb2 = reinterpret_cast<const float2*>(sbeta + cb);
+#pragma unroll
+            for (int i = 0; i < PC; ++i) {
+                const float2 bb = sb2[i];
+                pk[i] = (pack_bf16x2(a[2 * i] * bb.x, a[2 * i + 1] * bb.y) & keep[i]) | bp[i];
+            }
+            store_a_operand<C, false>(lane_base + kAS, t, pk);
+            build_band_row<C, NB>(br_row, t, il, n_band, lo, bp);
+            store_a_operand<C, true>(lane_base + kR2, t, bp);
+            tmem_wait_st();
+            tc_fence_before_sync();
+            compute_barrier();
+        }
+        if (t == 0) {
+            // W = (hi + lo) K: A operands in TMEM (AS: high bf16 half, R2: low half of the band),
+            // B = the K tile read as an MN-major operand (both 64-column sub-tiles, N = 128)
+            tc_fence_after_sync();
+#pragma unroll
+            for (int ks = 0; ks < 16; ++ks) {
+                const uint64_t bd = smem_desc(sK_a + (ks & 7) * 2048, 16384, 1024, SWZ_128B);
+                mma_f16_ts(tmem + kR0, tmem + ((ks < 8) ? kAS : kR2) + (ks & 7) * 8, bd, idesc_w, ks > 0);
+            }
+            mma_commit(&bar_mma);
+        }
+
+        STAMP(8);
+        // ---- T row -> Tinv: the thread's private packed row already has the TMA swizzle layout; one bulk
+        // tensor store of 32 rows per warp, overlapping the W products
+        if (p.Tinv != nullptr) {
+#pragma unroll
+            for (int c = 0; c < CPR; ++c) {
+                sts128(br_row + (swz<CPR>(t, c) << 4),
+                       (pack_bf16x2(a[c * 8 + 0], a[c * 8 + 1]) & keep[c * 4 + 0]) | bpT[c * 4 + 0],
+                       (pack_bf16x2(a[c * 8 + 2], a[c * 8 + 3]) & keep[c * 4 + 1]) | bpT[c * 4 + 1],
+                       (pack_bf16x2(a[c * 8 + 4], a[c * 8 + 5]) & keep[c * 4 + 2]) | bpT[c * 4 + 2],
+                       (pack_bf16x2(a[c * 8 + 6], a[c * 8 + 7]) & keep[c * 4 + 3]) | bpT[c * 4 + 3]);
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                tma_store_3d(&tmT, smem + L::kBR + wrow0 * (2 * C), 0, tc.t0 + wrow0, tc.bhv);
+                tma_store_commit();
+            }
+        }
+
+        STAMP(10);
+        // ---- W, then U: accumulator rows -> bf16 -> swizzled staging slice of the warp -> bulk tensor store
+#pragma unroll 1
+        for (int half = 0; half < 2; ++half) {
+            if (!wait_bar(&bar_mma, par_mma)) { ok = false; break; }
+            par_mma ^= 1;
+            tc_fence_after_sync();
+            STAMP(11 + half * 3);
+            if (t == 0 && has_next) {
+                // the products that read this tile's K (half 0) or V (half 1) are complete: prefetch the next tile's
+                const TileCoord nc = decode_tile(next, p);
+                if (half == 0) {
+                    mbar_arrive_expect_tx(&bar_k, 32768);
+                    tma_load_3d(sK, &tmK, &bar_k, 0, nc.t0, nc.bhk);
+                    tma_load_3d(sK + 16384, &tmK, &bar_k, 64, nc.t0, nc.bhk);
+                } else {
+                    mbar_arrive_expect_tx(&bar_v, 32768);
+                    tma_load_3d(sV, &tmV, &bar_v, 0, nc.t0, nc.bhv);
+                    tma_load_3d(sV + 16384, &tmV, &bar_v, 64, nc.t0, nc.bhv);
+                }
+            }
+            uint32_t o[64];
+#pragma unroll
+            for (int c0 = 0; c0 < 128; c0 += 32) {
+                uint32_t r[32];
+                tmem_ld32(lane_base + kR0 + c0, r);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 16; ++i) o[c0 / 2 + i] = pack_bf16x2(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
+            }
+            if (half == 0) {
+                // the Tinv store of this warp has been read (the staging slices below overlap other warps' rows)
+                if (lane == 0) tma_store_wait_read<0>();
+                tc_fence_before_sync();
+                compute_barrier();  // every row of the W accumulator has been read
+                if (t == 0) {
+                    if (!wait_bar(&bar_v, par_kv)) ok = false;
+                    if (ok) {
+                        tc_fence_after_sync();
+#pragma unroll
+                        for (int ks = 0; ks < 16; ++ks) {
+                            const uint64_t bd = smem_desc(sV_a + (ks & 7) * 2048, 16384, 1024, SWZ_128B);
+                            mma_f16_ts(tmem + kR0, tmem + ((ks < 8) ? kAS : kR2) + (ks & 7) * 8, bd, idesc_w, ks > 0);
+                        }
+                        mma_commit(&bar_mma);
+                    }
+                }
+            }
+            STAMP(12 + half * 3);
+            {
+                // the warp's 32 rows as two [32][64] sub-tiles in the 128-byte TMA swizzle, 8 KB per warp
+                const uint32_t slice = scratch_a + warp * 8192;
+                if (lane == 0) tma_store_wait_read<0>();  // earlier stores from this slice have been read
+                __syncwarp();
+#pragma unroll
+                for (int c = 0; c < 16; ++c)
+                    sts128(slice + (c >> 3) * 4096 + lane * 128 + (((c & 7) ^ (lane & 7)) << 4), o[c * 4 + 0], o[c * 4 + 1],
+                           o[c * 4 + 2], o[c * 4 + 3]);
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    const CUtensorMap* tm = (half == 0) ? &tmW : &tmU;
+                    uint8_t* src = smem + L::kEB + warp * 8192;
+                    tma_store_3d(tm, src, 0, tc.t0 + wrow0, tc.bhv);
+                    tma_store_3d(tm, src + 4096, 64, tc.t0 + wrow0, tc.bhv);
+                    tma_store_commit();
+                }
+            }
+            STAMP(13 + half * 3);
+        }
+        par_kv ^= 1;
     }
+    if (lane == 0) tma_store_wait_all<0>();
+    if (!ok) atomicExch(p.status, GDN_ERR_TIMEOUT);
 
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 4) {
+    if (warp == 0) {
         tc_fence_after_sync();
         tmem_dealloc(tmem, kTmemCols);
     }
@@ -771,35 +742,40 @@ EncodeTiledFn get_encode_fn() {
     return fn;
 }
 
-// [heads][T][128] bf16 tensor, boxes of 128 rows x 64 columns, 128-byte swizzle
-bool make_tile_map(CUtensorMap* tm, const void* base, long long heads, int T) {
+// [heads][T][cols] bf16 tensor, boxes of `box_rows` rows x `box_cols` columns with the given swizzle
+bool make_map(CUtensorMap* tm, const void* base, long long heads, int T, int cols, int box_cols, int box_rows,
+              CUtensorMapSwizzle swizzle) {
     EncodeTiledFn enc = get_encode_fn();
     if (enc == nullptr) return false;
-    cuuint64_t dims[3] = {static_cast<cuuint64_t>(kD), static_cast<cuuint64_t>(T), static_cast<cuuint64_t>(heads)};
-    cuuint64_t strides[2] = {static_cast<cuuint64_t>(kD) * 2, static_cast<cuuint64_t>(T) * kD * 2};
-    cuuint32_t box[3] = {64, 128, 1};
+    cuuint64_t dims[3] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(T), static_cast<cuuint64_t>(heads)};
+    cuuint64_t strides[2] = {static_cast<cuuint64_t>(cols) * 2, static_cast<cuuint64_t>(T) * cols * 2};
+    cuuint32_t box[3] = {static_cast<cuuint32_t>(box_cols), static_cast<cuuint32_t>(box_rows), 1};
     cuuint32_t estr[3] = {1, 1, 1};
     return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+struct Maps {
+    CUtensorMap K, V, W, U, T;
+};
+
 template <int C, int NB, int MODE>
-int launch_one(const CUtensorMap& tmK, const CUtensorMap& tmV, const Params& prm, cudaStream_t stream) {
+int launch_one(const Maps& m, const Params& prm, cudaStream_t stream) {
     using L = Smem<C, NB>;
     const int smem = L::kTotal + 1024;
     auto kern = chunk_tc_kernel<C, NB, MODE>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return GDN_ERR_LAUNCH;
     long long grid = prm.n_tiles < 2 * 148 ? prm.n_tiles : 2 * 148;
-    kern<<<static_cast<int>(grid), kThreads, smem, stream>>>(tmK, tmV, prm);
+    kern<<<static_cast<int>(grid), kThreads, smem, stream>>>(m.K, m.V, m.W, m.U, m.T, prm);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? GDN_OK : GDN_ERR_LAUNCH;
 }
 
 template <int C, int MODE>
-int launch_c(const CUtensorMap& tmK, const CUtensorMap& tmV, const Params& prm, cudaStream_t stream) {
-    if (MODE != INV_NEUMANN || prm.N <= 3) return launch_one<C, 3, MODE>(tmK, tmV, prm, stream);
-    return launch_one<C, 7, MODE>(tmK, tmV, prm, stream);
+int launch_c(const Maps& m, const Params& prm, cudaStream_t stream) {
+    if (MODE != INV_NEUMANN || prm.N <= 3) return launch_one<C, 3, MODE>(m, prm, stream);
+    return launch_one<C, 7, MODE>(m, prm, stream);
 }
 
 }  // namespace
@@ -818,9 +794,18 @@ int launch_tc_bf16(const Problem& p, InverseMode mode, cudaStream_t stream) {
     if ((long long)p.B * p.H_v * p.T == 0) return GDN_OK;
     int* status = device_status_word();
     if (status == nullptr) return GDN_ERR_LAUNCH;
-    CUtensorMap tmK, tmV;
-    if (!make_tile_map(&tmK, p.K, (long long)p.B * p.H_k, p.T)) return GDN_ERR_LAUNCH;
-    if (!make_tile_map(&tmV, p.V, (long long)p.B * p.H_v, p.T)) return GDN_ERR_LAUNCH;
+    Maps m;
+    const long long hk = (long long)p.B * p.H_k, hv = (long long)p.B * p.H_v;
+    const CUtensorMapSwizzle tsw = (p.C == 64) ? CU_TENSOR_MAP_SWIZZLE_128B
+                                  : (p.C == 32) ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
+    if (!make_map(&m.K, p.K, hk, p.T, kD, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
+    if (!make_map(&m.V, p.V, hv, p.T, kD, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
+    if (!make_map(&m.W, p.W, hv, p.T, kD, 64, 32, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
+    if (!make_map(&m.U, p.U, hv, p.T, kD, 64, 32, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
+    // Tinv rows are C wide; without a Tinv output the map points at W (never used by the kernel then)
+    if (!make_map(&m.T, p.Tinv != nullptr ? p.Tinv : p.W, hv, p.T, p.Tinv != nullptr ? p.C : kD, p.Tinv != nullptr ? p.C : 64, 32,
+                  p.Tinv != nullptr ? tsw : CU_TENSOR_MAP_SWIZZLE_128B))
+        return GDN_ERR_LAUNCH;
     Params prm;
     prm.beta = p.beta;
     prm.g = p.g;
@@ -839,15 +824,15 @@ int launch_tc_bf16(const Problem& p, InverseMode mode, cudaStream_t stream) {
     if (prm.n_tiles >= (1LL << 31) - 4096 || (long long)p.B * p.H_v >= (1LL << 31)) return GDN_ERR_UNSUPPORTED;
     if (mode == INV_NEUMANN) {
         switch (p.C) {
-            case 16: return launch_c<16, INV_NEUMANN>(tmK, tmV, prm, stream);
-            case 32: return launch_c<32, INV_NEUMANN>(tmK, tmV, prm, stream);
-            default: return launch_c<64, INV_NEUMANN>(tmK, tmV, prm, stream);
+            case 16: return launch_c<16, INV_NEUMANN>(m, prm, stream);
+            case 32: return launch_c<32, INV_NEUMANN>(m, prm, stream);
+            default: return launch_c<64, INV_NEUMANN>(m, prm, stream);
         }
     }
     switch (p.C) {
-        case 16: return launch_c<16, INV_FWDSUBST_ROWS>(tmK, tmV, prm, stream);
-        case 32: return launch_c<32, INV_FWDSUBST_ROWS>(tmK, tmV, prm, stream);
-        default: return launch_c<64, INV_FWDSUBST_ROWS>(tmK, tmV, prm, stream);
+        case 16: return launch_c<16, INV_FWDSUBST_ROWS>(m, prm, stream);
+        case 32: return launch_c<32, INV_FWDSUBST_ROWS>(m, prm, stream);
+        default: return launch_c<64, INV_FWDSUBST_ROWS>(m, prm, stream);
     }
 }
 
