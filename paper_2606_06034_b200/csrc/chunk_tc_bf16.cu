@@ -342,6 +342,17 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         tma_load_3d(sV + 16384, &tmV, &bar_v, 64, c.t0, c.bhv);
     }
 
+    // beta and g of the row are fetched one tile ahead
+    float bi_next = 0.f, gi_next = 0.f;
+    if (blockIdx.x < n_tiles) {
+        const TileCoord c = decode_tile(blockIdx.x, p);
+        if (c.t0 + t < p.T) {
+            const long long r = (long long)c.bhv * p.T + c.t0 + t;
+            bi_next = __ldg(p.beta + r);
+            gi_next = __ldg(p.g + r);
+        }
+    }
+
     for (uint32_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
         const TileCoord tc = decode_tile(tile, p);
         const uint32_t next = tile + gridDim.x;
@@ -350,11 +361,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         const long long grow = (long long)tc.bhv * p.T + tc.t0 + t;  // global token row (value-head space)
 
         STAMP(1);
-        float bi = 0.f, gi_ = 0.f;
-        if (row_valid) {
-            bi = __ldg(p.beta + grow);
-            gi_ = __ldg(p.g + grow);
-        }
+        const float bi = bi_next, gi_ = gi_next;  // loaded during the previous tile
         // the previous tile's bulk stores have finished reading the staging slices
         if (lane == 0) tma_store_wait_read<0>();
         tc_fence_before_sync();
@@ -407,6 +414,16 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             }
         }
 
+        bi_next = 0.f;
+        gi_next = 0.f;
+        if (has_next) {
+            const TileCoord nc = decode_tile(next, p);
+            if (nc.t0 + t < p.T) {
+                const long long r = (long long)nc.bhv * p.T + nc.t0 + t;
+                bi_next = __ldg(p.beta + r);
+                gi_next = __ldg(p.g + r);
+            }
+        }
         STAMP(4);
         float lb[NB + 1];  // lb[d] = L[i][i-d], the band of T0 - I (or of T - I after forward substitution)
 #pragma unroll
