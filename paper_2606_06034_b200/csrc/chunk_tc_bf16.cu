@@ -32,8 +32,7 @@ namespace {
 using namespace sm100;
 
 constexpr int kTile = 128;            // rows per work item
-constexpr int kComputeThreads = 128;  // one per tile row
-constexpr int kThreads = 128;
+constexpr int kThreads = 256;            // two threads per tile row
 constexpr int kD = 128;               // d_k = d_v
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -45,7 +44,7 @@ constexpr uint32_t kR0 = 0, kR2 = 128, kAS = 192, kTmemCols = 256;
 
 #ifdef GDN_TRACE
 __device__ long long g_trace[4096];
-#define STAMP(slot) do { if (blockIdx.x == 0 && tid == 32 && trace_n < 100) { g_trace[trace_n * 2] = (slot); g_trace[trace_n * 2 + 1] = clock64(); ++trace_n; } } while (0)
+#define STAMP(slot) do { if (blockIdx.x == 0 && (tid == 0 || tid == 160) && trace_n < 120) { g_trace[(tid == 0 ? 0 : 2048) + trace_n * 2] = (slot); g_trace[(tid == 0 ? 0 : 2048) + trace_n * 2 + 1] = clock64(); ++trace_n; } } while (0)
 #else
 #define STAMP(slot) do { } while (0)
 #endif
@@ -90,7 +89,7 @@ __device__ __forceinline__ float fast_exp2(float x) {
     return y;
 }
 
-__device__ __forceinline__ void compute_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ void compute_barrier() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 // bounded mbarrier wait: polls, and every 1024 polls compares the clock with a budget of about a second
 __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity) {
@@ -129,23 +128,36 @@ __device__ __forceinline__ int swz(int t, int c) {
     else return c;
 }
 
-// Builds a packed bf16 row of C entries that is zero except vals[e] at column il - e (e = 0..n_valid,
-// skipped where il - e < 0), through the thread's private row in shared memory: registers cannot be
-// indexed by a per-thread position, shared memory can.
+// Column split: for C >= 32 two threads share a tile row, thread half h owns the chunk-local columns
+// [h * C/2, (h+1) * C/2); for C = 16 only the h = 0 thread works on the row (h = 1 joins for W/U).
+template <int C>
+struct Split {
+    static constexpr bool kSplit = (C >= 32);
+    static constexpr int HC = kSplit ? C / 2 : C;  // columns per thread
+    static constexpr int PCH = HC / 2;             // packed bf16x2 words per thread
+};
+
+// Builds the thread's part of a packed bf16 row that is zero except vals[e] at column il - e
+// (e = 0..n_valid, skipped where the column is negative or outside [col0, col0 + HC)), through the row's
+// private shared-memory line: registers cannot be indexed by a per-thread position, shared memory can.
+// The two halves of a row own disjoint 16-byte chunks of the line, so they never race.
 template <int C, int NB>
-__device__ __forceinline__ void build_band_row(uint32_t row_addr, int t, int il, int n_valid, const uint16_t (&vals)[NB + 1],
-                                               uint32_t (&out)[C / 2]) {
-    constexpr int CPR = C / 8;
+__device__ __forceinline__ void build_band_row(uint32_t row_addr, int t, int il, int col0, int n_valid,
+                                               const uint16_t (&vals)[NB + 1], uint32_t (&out)[Split<C>::PCH]) {
+    constexpr int CPR = C / 8;                 // chunks of the full row
+    constexpr int CPT = Split<C>::HC / 8;      // chunks owned by this thread
+    const int c0 = col0 >> 3;
 #pragma unroll
-    for (int c = 0; c < CPR; ++c) sts128(row_addr + (swz<CPR>(t, c) << 4), 0u, 0u, 0u, 0u);
+    for (int c = 0; c < CPT; ++c) sts128(row_addr + (swz<CPR>(t, c0 + c) << 4), 0u, 0u, 0u, 0u);
 #pragma unroll
     for (int e = 0; e <= NB; ++e) {
         const int j = il - e;
-        if (j >= 0 && e <= n_valid) sts16(row_addr + (swz<CPR>(t, j >> 3) << 4) + (j & 7) * 2, vals[e]);
+        if (j >= col0 && j < col0 + Split<C>::HC && e <= n_valid)
+            sts16(row_addr + (swz<CPR>(t, j >> 3) << 4) + (j & 7) * 2, vals[e]);
     }
 #pragma unroll
-    for (int c = 0; c < CPR; ++c) {
-        const uint4 v = lds128(row_addr + (swz<CPR>(t, c) << 4));
+    for (int c = 0; c < CPT; ++c) {
+        const uint4 v = lds128(row_addr + (swz<CPR>(t, c0 + c) << 4));
         out[c * 4 + 0] = v.x;
         out[c * 4 + 1] = v.y;
         out[c * 4 + 2] = v.z;
@@ -156,51 +168,73 @@ __device__ __forceinline__ void build_band_row(uint32_t row_addr, int t, int il,
 __device__ __forceinline__ uint16_t bf16_bits(float x) { return __bfloat16_as_ushort(__float2bfloat16_rn(x)); }
 __device__ __forceinline__ float bf16_bits_to_f32(uint16_t b) { return __uint_as_float(static_cast<uint32_t>(b) << 16); }
 
-// Writes this row's packed bf16 diagonal block (C / 2 32-bit columns) into a 64-column A-operand slot.
-// tcgen05.st takes one address per warp: for C = 16 a warp holds two chunks, so the warp stores a
-// 16-column window in which each half-warp fills its own half and zero-fills the other.
-// FULL: also zero-fill the rest of the 64-column row (slot that held other data before).
+// Writes the thread's packed bf16 part of its row's diagonal block into a 64-column A-operand slot
+// (block of row t: columns [cb/2, cb/2 + C/2)). tcgen05.st takes one address per warp; for C = 16 a warp
+// holds two chunks, so the warp stores a 16-column window in which each half-warp fills its own half
+// and zero-fills the other. FULL: the h = 0 thread also zero-fills the columns outside the block.
 template <int C, bool FULL>
-__device__ __forceinline__ void store_a_operand(uint32_t slot_addr, int t, const uint32_t (&pk)[C / 2]) {
-    constexpr int PC = C / 2;
-    const int wb = (C >= 32) ? (t - (t % C)) : (t & ~31);  // first tile row of the warp-uniform window
-    constexpr int WC = (PC >= 16) ? PC : 16;               // window width in columns
-    const bool upper = (C < 32) && ((t & 16) != 0);
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-        // 16-column group c of the 64-column slot
+__device__ __forceinline__ void store_a_operand(uint32_t slot_addr, int t, int h, const uint32_t (&pk)[Split<C>::PCH]) {
+    if constexpr (C == 64) {
+        const int cb = t & 64;
         uint32_t r16[16];
-        const int rel = c * 16 - wb / 2;  // position of this group relative to the window
-        const bool inside = (rel >= 0) && (rel < WC);
-        if (!FULL && !inside) continue;
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            uint32_t v = 0u;
-            if constexpr (PC >= 16) {
-                // rel is 0 or 16 (C = 64) or 0 (C = 32) when inside
-                if (inside) v = (PC == 32) ? ((rel == 0) ? pk[i] : pk[(16 + i) % PC]) : pk[i % PC];
-            } else {
-                if (inside) v = upper ? ((i >= 8) ? pk[i - 8] : 0u) : ((i < 8) ? pk[i] : 0u);
-            }
-            r16[i] = v;
+        for (int i = 0; i < 16; ++i) r16[i] = pk[i];
+        tmem_st16(slot_addr + cb / 2 + h * 16, r16);
+        if (FULL && h == 0) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) r16[i] = 0u;
+            tmem_st16(slot_addr + (32 - cb / 2), r16);
+            tmem_st16(slot_addr + (32 - cb / 2) + 16, r16);
         }
-        tmem_st16(slot_addr + c * 16, r16);
+    } else if constexpr (C == 32) {
+        const int cb = t & 96;
+        uint32_t r8[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) r8[i] = pk[i];
+        tmem_st8(slot_addr + cb / 2 + h * 8, r8);
+        if (FULL && h == 0) {
+            uint32_t z[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) z[i] = 0u;
+#pragma unroll
+            for (int g = 1; g < 4; ++g) tmem_st16(slot_addr + ((cb / 2 + g * 16) & 63), z);
+        }
+    } else {
+        if (h == 0) {
+            const int wb = t & ~31;
+            const bool upper = (t & 16) != 0;
+            uint32_t r16[16];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                r16[i] = upper ? 0u : pk[i];
+                r16[8 + i] = upper ? pk[i] : 0u;
+            }
+            tmem_st16(slot_addr + wb / 2, r16);
+            if (FULL) {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) r16[i] = 0u;
+#pragma unroll
+                for (int g = 1; g < 4; ++g) tmem_st16(slot_addr + ((wb / 2 + g * 16) & 63), r16);
+            }
+        }
     }
 }
 
-// Reads this row's C columns of a block-diagonal 128-column accumulator (the Gram matrix).
+// Reads the thread's columns of its row's diagonal block of a 128-column accumulator (the Gram matrix).
 template <int C>
-__device__ __forceinline__ void load_diag_block(uint32_t lane_base, uint32_t col0, int t, float (&a)[C]) {
-    if constexpr (C >= 32) {
-        const int cb = t - (t % C);
+__device__ __forceinline__ void load_diag_block(uint32_t lane_base, uint32_t col0, int t, int h, float (&a)[Split<C>::HC]) {
+    if constexpr (C == 64) {
+        uint32_t r[32];
+        tmem_ld32(lane_base + col0 + (t & 64) + h * 32, r);
+        tmem_wait_ld();
 #pragma unroll
-        for (int c0 = 0; c0 < C; c0 += 32) {
-            uint32_t r[32];
-            tmem_ld32(lane_base + col0 + cb + c0, r);
-            tmem_wait_ld();
+        for (int i = 0; i < 32; ++i) a[i] = __uint_as_float(r[i]);
+    } else if constexpr (C == 32) {
+        uint32_t r[16];
+        tmem_ld16(lane_base + col0 + (t & 96) + h * 16, r);
+        tmem_wait_ld();
 #pragma unroll
-            for (int i = 0; i < 32; ++i) a[c0 + i] = __uint_as_float(r[i]);
-        }
+        for (int i = 0; i < 16; ++i) a[i] = __uint_as_float(r[i]);
     } else {
         const int wb = t & ~31;
         const bool upper = (t & 16) != 0;
@@ -212,21 +246,18 @@ __device__ __forceinline__ void load_diag_block(uint32_t lane_base, uint32_t col
     }
 }
 
-// Reads C consecutive accumulator columns starting at col0 (same address for the whole warp).
+// Reads the thread's columns of a 128 x C accumulator (same address for the whole warp).
 template <int C>
-__device__ __forceinline__ void load_cols(uint32_t lane_base, uint32_t col0, float (&r)[C]) {
-    if constexpr (C >= 32) {
+__device__ __forceinline__ void load_cols(uint32_t lane_base, uint32_t col0, int h, float (&r)[Split<C>::HC]) {
+    if constexpr (C == 64) {
+        uint32_t q[32];
+        tmem_ld32(lane_base + col0 + h * 32, q);
+        tmem_wait_ld();
 #pragma unroll
-        for (int c0 = 0; c0 < C; c0 += 32) {
-            uint32_t q[32];
-            tmem_ld32(lane_base + col0 + c0, q);
-            tmem_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) r[c0 + i] = __uint_as_float(q[i]);
-        }
+        for (int i = 0; i < 32; ++i) r[i] = __uint_as_float(q[i]);
     } else {
         uint32_t q[16];
-        tmem_ld16(lane_base + col0, q);
+        tmem_ld16(lane_base + col0 + ((C == 32) ? h * 16 : 0), q);
         tmem_wait_ld();
 #pragma unroll
         for (int i = 0; i < 16; ++i) r[i] = __uint_as_float(q[i]);
@@ -259,10 +290,14 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmU,
                 const __grid_constant__ CUtensorMap tmT, const Params p) {
     using L = Smem<C, NB>;
+    using SP = Split<C>;
     constexpr int NBP = L::NBP;
-    constexpr int PC = C / 2;
-    constexpr int CPR = C / 8;   // 16-byte chunks of a packed bf16 row
-    constexpr int CPRF = C / 4;  // 16-byte chunks of an fp32 row
+    constexpr int HC = SP::HC;     // columns of the chunk handled by this thread
+    constexpr int PCH = SP::PCH;   // packed words handled by this thread
+    constexpr int CPR = C / 8;     // 16-byte chunks of a packed bf16 row
+    constexpr int CPRF = C / 4;    // 16-byte chunks of an fp32 row
+    constexpr int CPT = HC / 8;    // packed chunks owned by this thread
+    constexpr int CPTF = HC / 4;   // fp32 chunks owned by this thread
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* sK = smem + L::kK;
@@ -308,15 +343,22 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     const int n_band = (MODE == INV_NEUMANN) ? N : NB;
     const uint32_t n_tiles = static_cast<uint32_t>(p.n_tiles);
 
-    // Thread t owns tile row t. Thread 0 also issues every TMA load and every tcgen05.mma, right after the
-    // CTA barrier that says all rows of the operand are in place.
-    const int t = tid;
-    const int il = t % C;   // row inside its chunk
-    const int cb = t - il;  // first tile row of the chunk
-    const int wrow0 = t - lane;
-    const uint32_t lane_base = tmem + (static_cast<uint32_t>(warp * 32) << 16);
+    // Threads t and t + 128 share tile row t (TMEM lane t): half h owns the chunk-local columns
+    // [h * HC, (h + 1) * HC) when C >= 32; for C = 16 only h = 0 works on the row (h = 1 joins for W/U).
+    // Thread 0 also issues every TMA load and every tcgen05.mma, right after the CTA barrier that says
+    // all rows of the operand are in place.
+    const int t = tid & 127;
+    const int h = tid >> 7;
+    const bool active = SP::kSplit || (h == 0);
+    const int col0 = SP::kSplit ? h * HC : 0;  // first chunk-local column of this thread
+    const int il = t % C;                      // row inside its chunk
+    const int cb = t - il;                     // first tile row of the chunk
+    const int wq = warp & 3;                   // TMEM lane quadrant of the warp
+    const int wrow0 = wq * 32;                 // first tile row of the warp
+    const uint32_t lane_base = tmem + (static_cast<uint32_t>(wq * 32) << 16);
     const uint32_t scratch_a = smem_u32(smem + L::kEB);
     const uint32_t br_row = smem_u32(smem + L::kBR) + t * (2 * C);
+    const uint32_t rowf = scratch_a + t * (4 * C);  // private fp32 row (shared by the two halves)
     const uint32_t sK_a = smem_u32(sK), sV_a = smem_u32(sV), sEB_a = smem_u32(sEB);
     const uint32_t idesc_g = instr_desc(128, 128, 1, 1, 0, 0, 1);
     const uint32_t idesc_c = instr_desc(128, C, 1, 1, 0, 1, 1);
@@ -328,11 +370,11 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         uint32_t z[16];
 #pragma unroll
         for (int i = 0; i < 16; ++i) z[i] = 0u;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) tmem_st16(lane_base + kAS + c * 16, z);
+        tmem_st16(lane_base + kAS + h * 32, z);
+        tmem_st16(lane_base + kAS + h * 32 + 16, z);
         tmem_wait_st();
     }
-    if (t == 0 && blockIdx.x < n_tiles) {
+    if (tid == 0 && blockIdx.x < n_tiles) {
         const TileCoord c = decode_tile(blockIdx.x, p);
         mbar_arrive_expect_tx(&bar_k, 32768);
         tma_load_3d(sK, &tmK, &bar_k, 0, c.t0, c.bhk);
@@ -341,7 +383,6 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         tma_load_3d(sV, &tmV, &bar_v, 0, c.t0, c.bhv);
         tma_load_3d(sV + 16384, &tmV, &bar_v, 64, c.t0, c.bhv);
     }
-
     // beta and g of the row are fetched one tile ahead
     float bi_next = 0.f, gi_next = 0.f;
     if (blockIdx.x < n_tiles) {
@@ -357,8 +398,6 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         const TileCoord tc = decode_tile(tile, p);
         const uint32_t next = tile + gridDim.x;
         const bool has_next = next < n_tiles;
-        const bool row_valid = (tc.t0 + t) < p.T;
-        const long long grow = (long long)tc.bhv * p.T + tc.t0 + t;  // global token row (value-head space)
 
         STAMP(1);
         const float bi = bi_next, gi_ = gi_next;  // loaded during the previous tile
@@ -366,9 +405,11 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         if (lane == 0) tma_store_wait_read<0>();
         tc_fence_before_sync();
         compute_barrier();  // everyone is done with the previous tile's shared arrays and accumulators
-        if (t == 0) {
+        if (tid == 0) {
             // G = K K^T into R0..R1 (128 columns)
+            STAMP(20);
             if (!wait_bar(&bar_k, par_kv)) ok = false;
+            STAMP(21);
             if (ok) {
                 tc_fence_after_sync();
 #pragma unroll
@@ -379,41 +420,51 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 mma_commit(&bar_mma);
             }
         }
-        sbeta[t] = bi;
-        sg[t] = gi_;
+        if (h == 0) {
+            sbeta[t] = bi;
+            sg[t] = gi_;
 #pragma unroll
-        for (int e = 0; e < NBP; ++e) sSH[t * NBP + e] = 0.f;
-        if (t < 8) {
+            for (int e = 0; e < NBP; ++e) sSH[t * NBP + e] = 0.f;
+            if (t < 8) {
 #pragma unroll
-            for (int e = 0; e < NBP; ++e) sSH[(kTile + t) * NBP + e] = 0.f;
+                for (int e = 0; e < NBP; ++e) sSH[(kTile + t) * NBP + e] = 0.f;
+            }
         }
         compute_barrier();
 
         STAMP(2);
-        // ---- A-build: row of Abar from the Gram block in TMEM
+        // ---- A-build: this thread's part of the row of Abar, from the Gram block in TMEM
         if (!wait_bar(&bar_mma, par_mma)) { ok = false; break; }
         par_mma ^= 1;
         STAMP(3);
         tc_fence_after_sync();
-        float a[C];
-        load_diag_block<C>(lane_base, kR0, t, a);
-        {
+        float a[HC];
+        if (active) {
+            load_diag_block<C>(lane_base, kR0, t, h, a);
             const float gs = gi_ * kLog2e;
             const float nbi = -bi;
-            const float4* sg4 = reinterpret_cast<const float4*>(sg + cb);
+            const float4* sg4 = reinterpret_cast<const float4*>(sg + cb + col0);
 #pragma unroll
-            for (int j4 = 0; j4 < C / 4; ++j4) {
+            for (int j4 = 0; j4 < HC / 4; ++j4) {
                 const float4 gq = sg4[j4];
                 const float gj[4] = {gq.x, gq.y, gq.z, gq.w};
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
-                    const int j = j4 * 4 + q;
-                    const float v = nbi * fast_exp2(fmaf(-gj[q], kLog2e, gs)) * a[j];
-                    a[j] = (j < il) ? v : 0.f;
+                    const int jl = j4 * 4 + q;
+                    const float v = nbi * fast_exp2(fmaf(-gj[q], kLog2e, gs)) * a[jl];
+                    a[jl] = (col0 + jl < il) ? v : 0.f;
                 }
             }
+            // the row of Abar goes to its private fp32 line: entries next to the diagonal (and, for the
+            // left half, the first entries of the right half) are read back from there
+#pragma unroll
+            for (int c = 0; c < CPTF; ++c)
+                sts128(rowf + (swz<CPRF>(t, (col0 >> 2) + c) << 4), __float_as_uint(a[c * 4 + 0]), __float_as_uint(a[c * 4 + 1]),
+                       __float_as_uint(a[c * 4 + 2]), __float_as_uint(a[c * 4 + 3]));
+        } else {
+#pragma unroll
+            for (int j = 0; j < HC; ++j) a[j] = 0.f;
         }
-
         bi_next = 0.f;
         gi_next = 0.f;
         if (has_next) {
@@ -424,28 +475,31 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 gi_next = __ldg(p.g + r);
             }
         }
+        compute_barrier();  // both halves of every fp32 row are written
+
         STAMP(4);
         float lb[NB + 1];  // lb[d] = L[i][i-d], the band of T0 - I (or of T - I after forward substitution)
 #pragma unroll
         for (int e = 0; e <= NB; ++e) lb[e] = 0.f;
 
-        const uint32_t rowf = scratch_a + t * (4 * C);  // private fp32 row
         if constexpr (MODE == INV_NEUMANN) {
-            // ---- ab[e] = Abar[i][i-e] through the private fp32 row
-            float ab[NB + 1];
-#pragma unroll
-            for (int c = 0; c < CPRF; ++c)
-                sts128(rowf + (swz<CPRF>(t, c) << 4), __float_as_uint(a[c * 4 + 0]), __float_as_uint(a[c * 4 + 1]),
-                       __float_as_uint(a[c * 4 + 2]), __float_as_uint(a[c * 4 + 3]));
+            float ab[NB + 1];     // ab[e] = Abar[i][i-e]
+            float anext[NB + 1];  // anext[e] = Abar[i][col0 + HC + e]: the entries just right of this thread's part
             ab[0] = 0.f;
 #pragma unroll
             for (int e = 1; e <= NB; ++e) {
                 const int j = il - e;
                 ab[e] = (j >= 0) ? lds32f(rowf + (swz<CPRF>(t, j >> 2) << 4) + (j & 3) * 4) : 0.f;
             }
-            // ---- band of the masked Neumann sum by distance recursion
+#pragma unroll
+            for (int e = 0; e < NB; ++e) {
+                const int j = col0 + HC + e;
+                anext[e] = (SP::kSplit && j < C) ? lds32f(rowf + (swz<CPRF>(t, j >> 2) << 4) + (j & 3) * 4) : 0.f;
+            }
+            anext[NB] = 0.f;
+            // ---- band of the masked Neumann sum by distance recursion (both halves compute it, h = 0 publishes it)
             lb[1] = ab[1];
-            sRB[t * NBP + 0] = lb[1];
+            if (h == 0) sRB[t * NBP + 0] = lb[1];
 #pragma unroll
             for (int d = 2; d <= NB; ++d) {
                 compute_barrier();
@@ -456,128 +510,142 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     v = fmaf(ab[e], sRB[r * NBP + (d - e - 1)], v);
                 }
                 lb[d] = (d <= N) ? v : 0.f;
-                if (d < NB) sRB[t * NBP + (d - 1)] = lb[d];
+                if (d < NB && h == 0) sRB[t * NBP + (d - 1)] = lb[d];
             }
             // column form: SH[j][e-1] = L[j+e][j]
+            if (h == 0) {
 #pragma unroll
-            for (int e = 1; e <= NB; ++e)
-                if (il - e >= 0) sSH[(t - e) * NBP + (e - 1)] = lb[e];
+                for (int e = 1; e <= NB; ++e)
+                    if (il - e >= 0) sSH[(t - e) * NBP + (e - 1)] = lb[e];
+            }
             compute_barrier();
 
             STAMP(5);
-            // ---- E = Abar + Abar L on i-j > N (in place over a[])
+            if (active) {
+                // ---- E = Abar + Abar L on i-j > N (in place over a[])
 #pragma unroll
-            for (int j = 0; j < C; ++j) {
-                float v = a[j];
-                if constexpr (NBP == 4) {
-                    const float4 c4 = *reinterpret_cast<const float4*>(sSH + (cb + j) * 4);
-                    if (j + 1 < C) v = fmaf(a[(j + 1 < C) ? j + 1 : j], c4.x, v);
-                    if (j + 2 < C) v = fmaf(a[(j + 2 < C) ? j + 2 : j], c4.y, v);
-                    if (j + 3 < C) v = fmaf(a[(j + 3 < C) ? j + 3 : j], c4.z, v);
-                } else {
-                    const float4 c4 = *reinterpret_cast<const float4*>(sSH + (cb + j) * 8);
-                    const float4 d4 = *reinterpret_cast<const float4*>(sSH + (cb + j) * 8 + 4);
-                    const float cc[7] = {c4.x, c4.y, c4.z, c4.w, d4.x, d4.y, d4.z};
+                for (int jl = 0; jl < HC; ++jl) {
+                    float v = a[jl];
+                    float cc[NBP];
+                    if constexpr (NBP == 4) {
+                        const float4 c4 = *reinterpret_cast<const float4*>(sSH + (cb + col0 + jl) * 4);
+                        cc[0] = c4.x; cc[1] = c4.y; cc[2] = c4.z; cc[3] = c4.w;
+                    } else {
+                        const float4 c4 = *reinterpret_cast<const float4*>(sSH + (cb + col0 + jl) * 8);
+                        const float4 d4 = *reinterpret_cast<const float4*>(sSH + (cb + col0 + jl) * 8 + 4);
+                        cc[0] = c4.x; cc[1] = c4.y; cc[2] = c4.z; cc[3] = c4.w;
+                        cc[4] = d4.x; cc[5] = d4.y; cc[6] = d4.z; cc[7] = d4.w;
+                    }
 #pragma unroll
-                    for (int e = 1; e <= NB; ++e)
-                        if (j + e < C) v = fmaf(a[(j + e < C) ? j + e : j], cc[e - 1], v);
+                    for (int e = 1; e <= NB; ++e) {
+                        const int k = jl + e;
+                        const float ak = (k < HC) ? a[(k < HC) ? k : 0] : anext[(k >= HC) ? k - HC : 0];
+                        v = fmaf(ak, cc[e - 1], v);
+                    }
+                    a[jl] = (il - (col0 + jl) > N) ? v : 0.f;
                 }
-                a[j] = (il - j > N) ? v : 0.f;
-            }
-            // E as B operand (MN-major, no swizzle): 16-byte chunk c of row t at c * 2048 + t * 16
-            if (S >= 1) {
+                // E as B operand (MN-major, no swizzle): 16-byte chunk c of row t at c * 2048 + t * 16
+                if (S >= 1) {
 #pragma unroll
-                for (int c = 0; c < C / 8; ++c) {
-                    uint4 v;
-                    v.x = pack_bf16x2(a[c * 8 + 0], a[c * 8 + 1]);
-                    v.y = pack_bf16x2(a[c * 8 + 2], a[c * 8 + 3]);
-                    v.z = pack_bf16x2(a[c * 8 + 4], a[c * 8 + 5]);
-                    v.w = pack_bf16x2(a[c * 8 + 6], a[c * 8 + 7]);
-                    *reinterpret_cast<uint4*>(sEB + c * 2048 + t * 16) = v;
+                    for (int c = 0; c < CPT; ++c) {
+                        uint4 v;
+                        v.x = pack_bf16x2(a[c * 8 + 0], a[c * 8 + 1]);
+                        v.y = pack_bf16x2(a[c * 8 + 2], a[c * 8 + 3]);
+                        v.z = pack_bf16x2(a[c * 8 + 4], a[c * 8 + 5]);
+                        v.w = pack_bf16x2(a[c * 8 + 6], a[c * 8 + 7]);
+                        *reinterpret_cast<uint4*>(sEB + ((col0 >> 3) + c) * 2048 + t * 16) = v;
+                    }
                 }
             }
         } else {
-            // ---- forward substitution (Eq. 2-3). The private fp32 rows hold Abar; thread = column il of its chunk.
+            // ---- forward substitution (Eq. 2-3). The private fp32 rows hold Abar; thread (h = 0, t) solves
+            // column il of its chunk, which has no dependence on other columns.
+            if (h == 0) {
+                float xcol[C];  // xcol[k] = T[k][il]
 #pragma unroll
-            for (int c = 0; c < CPRF; ++c)
-                sts128(rowf + (swz<CPRF>(t, c) << 4), __float_as_uint(a[c * 4 + 0]), __float_as_uint(a[c * 4 + 1]),
-                       __float_as_uint(a[c * 4 + 2]), __float_as_uint(a[c * 4 + 3]));
-            compute_barrier();
-            float xcol[C];  // xcol[k] = T[k][il]
+                for (int i = 0; i < C; ++i) {
+                    float acc = 0.f;
+                    const uint32_t ri = scratch_a + (cb + i) * (4 * C);
 #pragma unroll
-            for (int i = 0; i < C; ++i) {
-                float acc = 0.f;
-                const uint32_t ri = scratch_a + (cb + i) * (4 * C);
-#pragma unroll
-                for (int k4 = 0; k4 < (i + 3) / 4; ++k4) {
-                    const uint4 q = lds128(ri + (swz<CPRF>(i, k4) << 4));  // (cb + i) and i agree in the swizzle bits
-                    if (k4 * 4 + 0 < i) acc = fmaf(__uint_as_float(q.x), xcol[k4 * 4 + 0], acc);
-                    if (k4 * 4 + 1 < i) acc = fmaf(__uint_as_float(q.y), xcol[(k4 * 4 + 1 < C) ? k4 * 4 + 1 : 0], acc);
-                    if (k4 * 4 + 2 < i) acc = fmaf(__uint_as_float(q.z), xcol[(k4 * 4 + 2 < C) ? k4 * 4 + 2 : 0], acc);
-                    if (k4 * 4 + 3 < i) acc = fmaf(__uint_as_float(q.w), xcol[(k4 * 4 + 3 < C) ? k4 * 4 + 3 : 0], acc);
+                    for (int k4 = 0; k4 < (i + 3) / 4; ++k4) {
+                        const uint4 q = lds128(ri + (swz<CPRF>(i, k4) << 4));  // (cb + i) and i agree in the swizzle bits
+                        if (k4 * 4 + 0 < i) acc = fmaf(__uint_as_float(q.x), xcol[k4 * 4 + 0], acc);
+                        if (k4 * 4 + 1 < i) acc = fmaf(__uint_as_float(q.y), xcol[(k4 * 4 + 1 < C) ? k4 * 4 + 1 : 0], acc);
+                        if (k4 * 4 + 2 < i) acc = fmaf(__uint_as_float(q.z), xcol[(k4 * 4 + 2 < C) ? k4 * 4 + 2 : 0], acc);
+                        if (k4 * 4 + 3 < i) acc = fmaf(__uint_as_float(q.w), xcol[(k4 * 4 + 3 < C) ? k4 * 4 + 3 : 0], acc);
+                    }
+                    xcol[i] = (i > il) ? acc : ((i == il) ? 1.f : 0.f);
                 }
-                xcol[i] = (i > il) ? acc : ((i == il) ? 1.f : 0.f);
-            }
-            compute_barrier();  // everyone has read Abar
+                compute_barrier();  // everyone has read Abar
 #pragma unroll
-            for (int i = 0; i < C; ++i) {
-                const uint32_t addr = scratch_a + (cb + i) * (4 * C) + (swz<CPRF>(i, il >> 2) << 4) + (il & 3) * 4;
-                asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(xcol[i]) : "memory");
+                for (int i = 0; i < C; ++i) {
+                    const uint32_t addr = scratch_a + (cb + i) * (4 * C) + (swz<CPRF>(i, il >> 2) << 4) + (il & 3) * 4;
+                    asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(xcol[i]) : "memory");
+                }
+            } else {
+                compute_barrier();
             }
             compute_barrier();
-            // back to rows: a[] = far part, lb[] = band part
+            // back to rows: a[] = far part of this thread's columns, lb[] = band part
+            if (active) {
 #pragma unroll
-            for (int c = 0; c < CPRF; ++c) {
-                const uint4 q = lds128(rowf + (swz<CPRF>(t, c) << 4));
-                a[c * 4 + 0] = __uint_as_float(q.x);
-                a[c * 4 + 1] = __uint_as_float(q.y);
-                a[c * 4 + 2] = __uint_as_float(q.z);
-                a[c * 4 + 3] = __uint_as_float(q.w);
+                for (int c = 0; c < CPTF; ++c) {
+                    const uint4 q = lds128(rowf + (swz<CPRF>(t, (col0 >> 2) + c) << 4));
+                    a[c * 4 + 0] = __uint_as_float(q.x);
+                    a[c * 4 + 1] = __uint_as_float(q.y);
+                    a[c * 4 + 2] = __uint_as_float(q.z);
+                    a[c * 4 + 3] = __uint_as_float(q.w);
+                }
+#pragma unroll
+                for (int jl = 0; jl < HC; ++jl) a[jl] = (il - (col0 + jl) > NB) ? a[jl] : 0.f;
             }
 #pragma unroll
             for (int e = 1; e <= NB; ++e) {
                 const int j = il - e;
                 lb[e] = (j >= 0) ? lds32f(rowf + (swz<CPRF>(t, j >> 2) << 4) + (j & 3) * 4) : 0.f;
             }
-#pragma unroll
-            for (int j = 0; j < C; ++j) a[j] = (il - j > NB) ? a[j] : 0.f;
             compute_barrier();  // the fp32 rows are dead; the packed rows may overwrite them
         }
 
         STAMP(6);
         // ---- packed bf16 forms of the band: keep-mask (0 on the band and diagonal) and I + L
-        uint32_t keep[PC], bpT[PC];
-        {
+        uint32_t keep[PCH], bpT[PCH];
+        if (active) {
             uint16_t vals[NB + 1];
 #pragma unroll
             for (int e = 0; e <= NB; ++e) vals[e] = 0xFFFFu;
-            build_band_row<C, NB>(br_row, t, il, n_band, vals, keep);
+            build_band_row<C, NB>(br_row, t, il, col0, n_band, vals, keep);
 #pragma unroll
-            for (int i = 0; i < PC; ++i) keep[i] = ~keep[i];
+            for (int i = 0; i < PCH; ++i) keep[i] = ~keep[i];
             vals[0] = 0x3F80u;  // 1.0
 #pragma unroll
             for (int e = 1; e <= NB; ++e) vals[e] = bf16_bits(lb[e]);
-            build_band_row<C, NB>(br_row, t, il, n_band, vals, bpT);
+            build_band_row<C, NB>(br_row, t, il, col0, n_band, vals, bpT);
+        } else {
+#pragma unroll
+            for (int i = 0; i < PCH; ++i) { keep[i] = 0u; bpT[i] = 0u; }
         }
 
         STAMP(7);
         if constexpr (MODE == INV_NEUMANN) {
             // ---- residual rounds: A_k = T0 + Z_k (bf16, TMEM), Z_{k+1} = A_k E, so that T = T0 + Z_S
             for (int k = 0; k < S; ++k) {
-                uint32_t pk[PC];
-                if (k == 0) {
+                if (active) {
+                    uint32_t pk[PCH];
+                    if (k == 0) {
 #pragma unroll
-                    for (int i = 0; i < PC; ++i) pk[i] = bpT[i];
-                } else {
+                        for (int i = 0; i < PCH; ++i) pk[i] = bpT[i];
+                    } else {
 #pragma unroll
-                    for (int i = 0; i < PC; ++i) pk[i] = (pack_bf16x2(a[2 * i], a[2 * i + 1]) & keep[i]) | bpT[i];
+                        for (int i = 0; i < PCH; ++i) pk[i] = (pack_bf16x2(a[2 * i], a[2 * i + 1]) & keep[i]) | bpT[i];
+                    }
+                    store_a_operand<C, false>(lane_base + kAS, t, h, pk);
+                    fence_proxy_async_smem();
+                    tmem_wait_st();
                 }
-                store_a_operand<C, false>(lane_base + kAS, t, pk);
-                fence_proxy_async_smem();
-                tmem_wait_st();
                 tc_fence_before_sync();
                 compute_barrier();
-                if (t == 0) {
+                if (tid == 0) {
                     tc_fence_after_sync();
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks) {
@@ -589,19 +657,19 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 if (!wait_bar(&bar_mma, par_mma)) { ok = false; break; }
                 par_mma ^= 1;
                 tc_fence_after_sync();
-                load_cols<C>(lane_base, kR2, a);
+                if (active) load_cols<C>(lane_base, kR2, h, a);
             }
             if (!ok) break;
             if (S == 0) {
 #pragma unroll
-                for (int j = 0; j < C; ++j) a[j] = 0.f;
+                for (int j = 0; j < HC; ++j) a[j] = 0.f;
             }
         }
-        // a[] = far row (T - I - L)
+        // a[] = this thread's part of the far row (T - I - L)
 
         STAMP(9);
         // ---- A operands for W/U: T diag(beta) = hi + lo, hi over the whole row, lo only on band + diagonal
-        {
+        if (active) {
             float tb[NB + 1];
             tb[0] = bi;
 #pragma unroll
@@ -612,22 +680,22 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 hi[e] = bf16_bits(tb[e]);
                 lo[e] = bf16_bits(tb[e] - bf16_bits_to_f32(hi[e]));
             }
-            uint32_t bp[PC], pk[PC];
-            build_band_row<C, NB>(br_row, t, il, n_band, hi, bp);
-            const float2* sb2 = reinterpret_cast<const float2*>(sbeta + cb);
+            uint32_t bp[PCH], pk[PCH];
+            build_band_row<C, NB>(br_row, t, il, col0, n_band, hi, bp);
+            const float2* sb2 = reinterpret_cast<const float2*>(sbeta + cb + col0);
 #pragma unroll
-            for (int i = 0; i < PC; ++i) {
+            for (int i = 0; i < PCH; ++i) {
                 const float2 bb = sb2[i];
                 pk[i] = (pack_bf16x2(a[2 * i] * bb.x, a[2 * i + 1] * bb.y) & keep[i]) | bp[i];
             }
-            store_a_operand<C, false>(lane_base + kAS, t, pk);
-            build_band_row<C, NB>(br_row, t, il, n_band, lo, bp);
-            store_a_operand<C, true>(lane_base + kR2, t, bp);
+            store_a_operand<C, false>(lane_base + kAS, t, h, pk);
+            build_band_row<C, NB>(br_row, t, il, col0, n_band, lo, bp);
+            store_a_operand<C, true>(lane_base + kR2, t, h, bp);
             tmem_wait_st();
-            tc_fence_before_sync();
-            compute_barrier();
         }
-        if (t == 0) {
+        tc_fence_before_sync();
+        compute_barrier();
+        if (tid == 0) {
             // W = (hi + lo) K: A operands in TMEM (AS: high bf16 half, R2: low half of the band),
             // B = the K tile read as an MN-major operand (both 64-column sub-tiles, N = 128)
             tc_fence_after_sync();
@@ -640,12 +708,15 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         }
 
         STAMP(8);
-        // ---- T row -> Tinv: the thread's private packed row already has the TMA swizzle layout; one bulk
-        // tensor store of 32 rows per warp, overlapping the W products
-        if (p.Tinv != nullptr) {
+        // ---- T row -> Tinv: each half-row goes to a staging line in the TMA swizzle layout (the band-row
+        // region is free now); one bulk tensor store of 32 rows x HC columns per warp, overlapping the W products
+        if (p.Tinv != nullptr && active) {
+            constexpr int RB = HC * 2;  // bytes per staged half-row
+            const uint32_t stage = smem_u32(smem + L::kBR) + h * (kTile * RB);
+            const uint32_t trow = stage + t * RB;
 #pragma unroll
-            for (int c = 0; c < CPR; ++c) {
-                sts128(br_row + (swz<CPR>(t, c) << 4),
+            for (int c = 0; c < CPT; ++c) {
+                sts128(trow + (swz<CPT>(t, c) << 4),
                        (pack_bf16x2(a[c * 8 + 0], a[c * 8 + 1]) & keep[c * 4 + 0]) | bpT[c * 4 + 0],
                        (pack_bf16x2(a[c * 8 + 2], a[c * 8 + 3]) & keep[c * 4 + 1]) | bpT[c * 4 + 1],
                        (pack_bf16x2(a[c * 8 + 4], a[c * 8 + 5]) & keep[c * 4 + 2]) | bpT[c * 4 + 2],
@@ -654,20 +725,21 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) {
-                tma_store_3d(&tmT, smem + L::kBR + wrow0 * (2 * C), 0, tc.t0 + wrow0, tc.bhv);
+                tma_store_3d(&tmT, smem + L::kBR + h * (kTile * RB) + wrow0 * RB, col0, tc.t0 + wrow0, tc.bhv);
                 tma_store_commit();
             }
         }
 
         STAMP(10);
-        // ---- W, then U: accumulator rows -> bf16 -> swizzled staging slice of the warp -> bulk tensor store
+        // ---- W, then U: each thread reads 64 accumulator columns of its row -> bf16 -> swizzled staging
+        // sub-tile of its warp -> one bulk tensor store (32 rows x 64 columns) per warp
 #pragma unroll 1
         for (int half = 0; half < 2; ++half) {
             if (!wait_bar(&bar_mma, par_mma)) { ok = false; break; }
             par_mma ^= 1;
             tc_fence_after_sync();
             STAMP(11 + half * 3);
-            if (t == 0 && has_next) {
+            if (tid == 0 && has_next) {
                 // the products that read this tile's K (half 0) or V (half 1) are complete: prefetch the next tile's
                 const TileCoord nc = decode_tile(next, p);
                 if (half == 0) {
@@ -680,22 +752,24 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     tma_load_3d(sV + 16384, &tmV, &bar_v, 64, nc.t0, nc.bhv);
                 }
             }
-            uint32_t o[64];
+            uint32_t o[32];
 #pragma unroll
-            for (int c0 = 0; c0 < 128; c0 += 32) {
+            for (int c0 = 0; c0 < 64; c0 += 32) {
                 uint32_t r[32];
-                tmem_ld32(lane_base + kR0 + c0, r);
+                tmem_ld32(lane_base + kR0 + h * 64 + c0, r);
                 tmem_wait_ld();
 #pragma unroll
                 for (int i = 0; i < 16; ++i) o[c0 / 2 + i] = pack_bf16x2(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
             }
             if (half == 0) {
-                // the Tinv store of this warp has been read (the staging slices below overlap other warps' rows)
+                // this warp's Tinv store has been read (the staging slices below overlap other warps' lines)
                 if (lane == 0) tma_store_wait_read<0>();
                 tc_fence_before_sync();
                 compute_barrier();  // every row of the W accumulator has been read
-                if (t == 0) {
+                if (tid == 0) {
+                    STAMP(22);
                     if (!wait_bar(&bar_v, par_kv)) ok = false;
+                    STAMP(23);
                     if (ok) {
                         tc_fence_after_sync();
 #pragma unroll
@@ -709,21 +783,17 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             }
             STAMP(12 + half * 3);
             {
-                // the warp's 32 rows as two [32][64] sub-tiles in the 128-byte TMA swizzle, 8 KB per warp
-                const uint32_t slice = scratch_a + warp * 8192;
-                if (lane == 0) tma_store_wait_read<0>();  // earlier stores from this slice have been read
+                // 32 rows x 64 columns of this warp in the 128-byte TMA swizzle: 4 KB at slice(wq) + h * 4 KB
+                const uint32_t sub = scratch_a + wq * 8192 + h * 4096;
+                if (lane == 0) tma_store_wait_read<0>();  // earlier stores from this sub-tile have been read
                 __syncwarp();
 #pragma unroll
-                for (int c = 0; c < 16; ++c)
-                    sts128(slice + (c >> 3) * 4096 + lane * 128 + (((c & 7) ^ (lane & 7)) << 4), o[c * 4 + 0], o[c * 4 + 1],
-                           o[c * 4 + 2], o[c * 4 + 3]);
+                for (int c = 0; c < 8; ++c)
+                    sts128(sub + lane * 128 + ((c ^ (lane & 7)) << 4), o[c * 4 + 0], o[c * 4 + 1], o[c * 4 + 2], o[c * 4 + 3]);
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) {
-                    const CUtensorMap* tm = (half == 0) ? &tmW : &tmU;
-                    uint8_t* src = smem + L::kEB + warp * 8192;
-                    tma_store_3d(tm, src, 0, tc.t0 + wrow0, tc.bhv);
-                    tma_store_3d(tm, src + 4096, 64, tc.t0 + wrow0, tc.bhv);
+                    tma_store_3d((half == 0) ? &tmW : &tmU, smem + L::kEB + wq * 8192 + h * 4096, h * 64, tc.t0 + wrow0, tc.bhv);
                     tma_store_commit();
                 }
             }
@@ -813,14 +883,15 @@ int launch_tc_bf16(const Problem& p, InverseMode mode, cudaStream_t stream) {
     if (status == nullptr) return GDN_ERR_LAUNCH;
     Maps m;
     const long long hk = (long long)p.B * p.H_k, hv = (long long)p.B * p.H_v;
-    const CUtensorMapSwizzle tsw = (p.C == 64) ? CU_TENSOR_MAP_SWIZZLE_128B
-                                  : (p.C == 32) ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
+    // Tinv leaves in boxes of 32 rows x (C/2 columns for C >= 32, else C columns): 64-, 32- and 32-byte lines
+    const int tbox = (p.C >= 32) ? p.C / 2 : p.C;
+    const CUtensorMapSwizzle tsw = (tbox * 2 == 64) ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
     if (!make_map(&m.K, p.K, hk, p.T, kD, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
     if (!make_map(&m.V, p.V, hv, p.T, kD, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
     if (!make_map(&m.W, p.W, hv, p.T, kD, 64, 32, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
     if (!make_map(&m.U, p.U, hv, p.T, kD, 64, 32, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
     // Tinv rows are C wide; without a Tinv output the map points at W (never used by the kernel then)
-    if (!make_map(&m.T, p.Tinv != nullptr ? p.Tinv : p.W, hv, p.T, p.Tinv != nullptr ? p.C : kD, p.Tinv != nullptr ? p.C : 64, 32,
+    if (!make_map(&m.T, p.Tinv != nullptr ? p.Tinv : p.W, hv, p.T, p.Tinv != nullptr ? p.C : kD, p.Tinv != nullptr ? tbox : 64, 32,
                   p.Tinv != nullptr ? tsw : CU_TENSOR_MAP_SWIZZLE_128B))
         return GDN_ERR_LAUNCH;
     Params prm;
