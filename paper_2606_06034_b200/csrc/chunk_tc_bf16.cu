@@ -37,9 +37,10 @@ constexpr int kD = 128;               // d_k = d_v
 constexpr float kLog2e = 1.4426950408889634f;
 
 // TMEM column map (256 columns allocated):
-//   R0..R1 (128 columns)  Gram matrix, later the W and then the U accumulator
-//   R2     (64 columns)   accumulator of the residual rounds, later the low-half A operand of W/U
-//   AS     (64 columns)   bf16 A operand (block diagonal, 128 x 128) of the residual rounds and of W/U
+//   R0..R1 (128 columns)  Gram matrix, then the accumulator of the residual rounds, of W and of U
+//   R2     (64 columns)   low-half bf16 A operand of W/U (block diagonal)
+//   AS     (64 columns)   bf16 A operand of the residual rounds (chunks stacked along M) and of W/U
+//                         (high half, block diagonal)
 constexpr uint32_t kR0 = 0, kR2 = 128, kAS = 192, kTmemCols = 256;
 
 #ifdef GDN_TRACE
@@ -220,6 +221,23 @@ __device__ __forceinline__ void store_a_operand(uint32_t slot_addr, int t, int h
     }
 }
 
+// Writes the thread's packed bf16 part of its row at its chunk-local position (columns [col0/2, col0/2 + PCH)
+// of the slot): the A operand of the residual rounds, where the chunks of a tile are stacked along M.
+template <int C>
+__device__ __forceinline__ void store_stacked_operand(uint32_t slot_addr, int h, const uint32_t (&pk)[Split<C>::PCH]) {
+    if constexpr (C == 64) {
+        uint32_t r16[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) r16[i] = pk[i];
+        tmem_st16(slot_addr + h * 16, r16);
+    } else {
+        uint32_t r8[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) r8[i] = pk[i];
+        tmem_st8(slot_addr + ((C == 32) ? h * 8 : 0), r8);
+    }
+}
+
 // Reads the thread's columns of its row's diagonal block of a 128-column accumulator (the Gram matrix).
 template <int C>
 __device__ __forceinline__ void load_diag_block(uint32_t lane_base, uint32_t col0, int t, int h, float (&a)[Split<C>::HC]) {
@@ -361,19 +379,11 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     const uint32_t rowf = scratch_a + t * (4 * C);  // private fp32 row (shared by the two halves)
     const uint32_t sK_a = smem_u32(sK), sV_a = smem_u32(sV), sEB_a = smem_u32(sEB);
     const uint32_t idesc_g = instr_desc(128, 128, 1, 1, 0, 0, 1);
-    const uint32_t idesc_c = instr_desc(128, C, 1, 1, 0, 1, 1);
+    const uint32_t idesc_c = instr_desc(128, 128, 1, 1, 0, 1, 1);
     const uint32_t idesc_w = instr_desc(128, 128, 1, 1, 0, 1, 1);
     uint32_t par_mma = 0, par_kv = 0;
     bool ok = true;
 
-    {  // the A-operand slot keeps zeros outside the diagonal blocks for the whole kernel
-        uint32_t z[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) z[i] = 0u;
-        tmem_st16(lane_base + kAS + h * 32, z);
-        tmem_st16(lane_base + kAS + h * 32 + 16, z);
-        tmem_wait_st();
-    }
     if (tid == 0 && blockIdx.x < n_tiles) {
         const TileCoord c = decode_tile(blockIdx.x, p);
         mbar_arrive_expect_tx(&bar_k, 32768);
@@ -544,7 +554,8 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     }
                     a[jl] = (il - (col0 + jl) > N) ? v : 0.f;
                 }
-                // E as B operand (MN-major, no swizzle): 16-byte chunk c of row t at c * 2048 + t * 16
+                // E as B operand [E_1 | E_2 | ...] (C x 128, MN-major, no swizzle): the 16-byte piece of chunk-row il
+                // for global column group n8 sits at n8 * (16 C) + il * 16
                 if (S >= 1) {
 #pragma unroll
                     for (int c = 0; c < CPT; ++c) {
@@ -553,7 +564,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                         v.y = pack_bf16x2(a[c * 8 + 2], a[c * 8 + 3]);
                         v.z = pack_bf16x2(a[c * 8 + 4], a[c * 8 + 5]);
                         v.w = pack_bf16x2(a[c * 8 + 6], a[c * 8 + 7]);
-                        *reinterpret_cast<uint4*>(sEB + ((col0 >> 3) + c) * 2048 + t * 16) = v;
+                        *reinterpret_cast<uint4*>(sEB + (((cb + col0) >> 3) + c) * (16 * C) + il * 16) = v;
                     }
                 }
             }
@@ -639,25 +650,27 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 #pragma unroll
                         for (int i = 0; i < PCH; ++i) pk[i] = (pack_bf16x2(a[2 * i], a[2 * i + 1]) & keep[i]) | bpT[i];
                     }
-                    store_a_operand<C, false>(lane_base + kAS, t, h, pk);
+                    store_stacked_operand<C>(lane_base + kAS, h, pk);
                     fence_proxy_async_smem();
                     tmem_wait_st();
                 }
                 tc_fence_before_sync();
                 compute_barrier();
                 if (tid == 0) {
+                    // [Z_1; Z_2; ...] <- [A_1; A_2; ...] [E_1 | E_2 | ...]: M = 128, N = 128, K = C; row t keeps
+                    // the C columns of its own chunk
                     tc_fence_after_sync();
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {
-                        const uint64_t bd = smem_desc(sEB_a + ks * 256, 128, 2048, SWZ_NONE);
-                        mma_f16_ts(tmem + kR2, tmem + kAS + ks * 8, bd, idesc_c, ks > 0);
+                    for (int ks = 0; ks < C / 16; ++ks) {
+                        const uint64_t bd = smem_desc(sEB_a + ks * 256, 128, 16 * C, SWZ_NONE);
+                        mma_f16_ts(tmem + kR0, tmem + kAS + ks * 8, bd, idesc_c, ks > 0);
                     }
                     mma_commit(&bar_mma);
                 }
                 if (!wait_bar(&bar_mma, par_mma)) { ok = false; break; }
                 par_mma ^= 1;
                 tc_fence_after_sync();
-                if (active) load_cols<C>(lane_base, kR2, h, a);
+                if (active) load_diag_block<C>(lane_base, kR0, t, h, a);
             }
             if (!ok) break;
             if (S == 0) {
@@ -688,7 +701,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 const float2 bb = sb2[i];
                 pk[i] = (pack_bf16x2(a[2 * i] * bb.x, a[2 * i + 1] * bb.y) & keep[i]) | bp[i];
             }
-            store_a_operand<C, false>(lane_base + kAS, t, h, pk);
+            store_a_operand<C, true>(lane_base + kAS, t, h, pk);
             build_band_row<C, NB>(br_row, t, il, col0, n_band, lo, bp);
             store_a_operand<C, true>(lane_base + kR2, t, h, bp);
             tmem_wait_st();
