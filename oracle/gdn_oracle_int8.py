@@ -1,0 +1,334 @@
+"""CPU oracle for the INT8 variant of the chunk-prepare path (exact integer arithmetic).
+
+TEST INFRASTRUCTURE ONLY: only the tests, the smoke check and the benchmark's CPU-baseline leg may
+import this file; it shares no code with the CUDA sources.
+
+The paper fixes little about its low-bit variant: a uniform symmetric quantiser
+q(x) = clip(round(x / Delta), qmin, qmax) (App. G, Eq. 32), one scale per tensor for the inverse
+(App. G table), a truncation order N <= 3 compensated by residual correction (Sec. 3.5), the band
+mask that removes the outliers min-max scales are sensitive to (Sec. 3.3), and the remark that the
+chain re-applies quantisation at every step (Sec. 3.5). Everything else is a reading of this build,
+chosen so that both sides can evaluate it bit for bit ("block floating point, 8-bit mantissas"):
+
+  * every tensor is int8 mantissas in [-127, 127] with ONE power-of-two exponent per chunk
+    (Delta = 2^e, chosen from the tensor's own maximum: dynamic per-tensor scale);
+  * the identity is never quantised (T = I + Toff), the structural mask is applied BEFORE each
+    requantisation (only the structurally non-zero support decides the scale);
+  * round = round half away from zero, range +-127;
+  * the gate decay exp(g_i - g_j) is a 256-entry table of 2^(-f/256) in 1.15 fixed point plus a shift.
+
+Definitions (Python integers or int64; every product that a tensor-core MMA would form fits int32):
+
+  rsr(x, r)    = sign(x) * ((|x| + 2^(r-1)) >> r),  rsr(x, 0) = x
+  Q8(acc, e)   : m = max|acc| over the support, r = max(0, bitlen(m) - 7),
+                 q = clamp(rsr(acc, r), -127, 127), exponent e + r
+  align(terms) : e_ref = max(min e, max e - 24); x_i shifted left by e_i - e_ref (rsr if negative); summed
+
+Steps per chunk (C <= 64), inputs Kq, Vq int8 with exponents k_exp, v_exp, beta_q = rne(beta 2^15) (u16),
+decay_q = rne(-g log2(e) 2^8) (non-decreasing inside a chunk):
+
+  I1  G = Kq Kq^T
+  I2  d = decay_q_i - decay_q_j; Gam = LUT[d & 255] >> (d >> 8) if (d >> 8) < 16 else 0; c = (beta_q_i Gam + 2^14) >> 15
+  I3  (Aq, eA)   = Q8(-(G o c) on i > j, 2 k_exp - 15)                      [Abar, Sec. 2.1]
+  I4  P_1 = band_N(Aq); (P_n, e_n) = Q8(band_N(P_{n-1} band_N(Aq)), e_{n-1} + eA), n = 2..N   [Eq. 7, 10]
+  I5  (T0q, eT0) = Q8(align(P_1..P_N))  on 1 <= i-j <= N                    [T0 - I, Eq. 11]
+  I6  (Eq, eE)   = Q8(align(Aq, Aq T0q)) on i-j > N                         [Eq. 13]
+  I7  R_1 = Eq; (R_s, e_s) = Q8(R_{s-1} Eq, e_{s-1} + eE) on i-j >= s(N+1), s = 2..S while s(N+1) < C;
+      (Sq, eS) = Q8(align(R_1..))                                           [sum_{s>=1} E^s]
+  I8  (Toffq, eT) = Q8(align(T0q, Sq, T0q Sq)) on i > j                     [T - I = T0 sum E^s - I]
+  I9  (Tbq, eTb) = Q8(Toffq_ij beta_q_j, eT - 15) on i > j
+  I10 (Wq, eW)   = Q8(align(Tbq Kq [eTb + k_exp], beta_q_i Kq_i [k_exp - 15])); same for U with Vq, v_exp
+
+Two evaluators are given: `chunk_prepare_int8_ref` (plain Python integers, loops) and
+`chunk_prepare_int8` (numpy int64, with assertions that MMA accumulators fit int32). They are
+written separately and compared with each other in the tests, together with closed forms.
+"""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+
+QMAX = 127
+
+
+def decay_lut() -> list[int]:
+    """LUT[f] = rne(2^15 * 2^(-f/256)), f = 0..255 (unsigned 16 bit; LUT[0] = 32768)."""
+    return [int(math.floor(32768.0 * 2.0 ** (-f / 256.0) + 0.5)) for f in range(256)]
+
+
+def lut_checksum(lut=None) -> int:
+    lut = decay_lut() if lut is None else lut
+    s = 0
+    for f, v in enumerate(lut):
+        s = (s * 31 + int(v) + f) % 1000000007
+    return s
+
+
+# --------------------------------------------------------------------------- plain Python evaluator
+def _rsr(x: int, r: int) -> int:
+    if r <= 0:
+        return x << (-r)
+    a = (abs(x) + (1 << (r - 1))) >> r
+    return a if x >= 0 else -a
+
+
+def _q8(acc, e, support):
+    """acc: dict {(i, j): int} or nested lists; support: iterable of index pairs. Returns (dict, e_out)."""
+    m = 0
+    for idx in support:
+        m = max(m, abs(acc[idx]))
+    r = max(0, m.bit_length() - 7)
+    out = {}
+    for idx in support:
+        q = _rsr(acc[idx], r)
+        out[idx] = max(-QMAX, min(QMAX, q))
+    return out, e + r
+
+
+def _align(terms, support):
+    """terms: list of (dict, exponent). Returns (dict over support, e_ref)."""
+    es = [e for _, e in terms]
+    e_ref = max(min(es), max(es) - 24)
+    out = {}
+    for idx in support:
+        s = 0
+        for x, e in terms:
+            s += _rsr(x.get(idx, 0), -(e - e_ref))
+        out[idx] = s
+    return out, e_ref
+
+
+def _matmul_sparse(X, Y, n, support):
+    out = {}
+    for (i, j) in support:
+        s = 0
+        for k in range(n):
+            a = X.get((i, k), 0)
+            if a:
+                b = Y.get((k, j), 0)
+                if b:
+                    s += a * b
+        out[(i, j)] = s
+    return out
+
+
+def chunk_prepare_int8_ref(Kq, Vq, k_exp, v_exp, beta_q, decay_q, N, S):
+    """One chunk, plain Python integers. Kq [C][dk], Vq [C][dv] lists of ints. Returns a dict of results."""
+    C = len(Kq)
+    dk = len(Kq[0])
+    dv = len(Vq[0])
+    lut = decay_lut()
+    lower = [(i, j) for i in range(C) for j in range(i)]
+    band = [(i, j) for (i, j) in lower if i - j <= N]
+    far = [(i, j) for (i, j) in lower if i - j > N]
+    # I1-I3
+    accA = {}
+    for (i, j) in lower:
+        G = sum(int(Kq[i][d]) * int(Kq[j][d]) for d in range(dk))
+        dlt = int(decay_q[i]) - int(decay_q[j])
+        assert dlt >= 0
+        sh = dlt >> 8
+        gam = (lut[dlt & 255] >> sh) if sh < 16 else 0
+        c = (int(beta_q[i]) * gam + (1 << 14)) >> 15
+        accA[(i, j)] = -G * c
+    Aq, eA = _q8(accA, 2 * int(k_exp) - 15, lower)
+    # I4
+    Aband = {idx: Aq[idx] for idx in band}
+    P = [(Aband, eA)]
+    for n in range(2, N + 1):
+        prev, eprev = P[-1]
+        sup_n = [(i, j) for (i, j) in band if i - j >= n]
+        acc = _matmul_sparse(prev, Aband, C, sup_n)
+        Pn, en = _q8(acc, eprev + eA, sup_n)
+        P.append((Pn, en))
+    # I5
+    accT0, eref = _align(P, band)
+    T0q, eT0 = _q8(accT0, eref, band)
+    # I6
+    AT0 = _matmul_sparse(Aq, T0q, C, far)
+    accE, eref = _align([(Aq, eA), (AT0, eA + eT0)], far)
+    Eq, eE = _q8(accE, eref, far)
+    # I7
+    R = []
+    if S >= 1:
+        R.append((Eq, eE))
+        for s in range(2, S + 1):
+            if s * (N + 1) >= C:
+                break
+            sup_s = [(i, j) for (i, j) in lower if i - j >= s * (N + 1)]
+            prev, eprev = R[-1]
+            acc = _matmul_sparse(prev, Eq, C, sup_s)
+            Rs, es = _q8(acc, eprev + eE, sup_s)
+            R.append((Rs, es))
+    if R:
+        accS, eref = _align(R, far)
+        Sq, eS = _q8(accS, eref, far)
+    else:
+        Sq, eS = {idx: 0 for idx in far}, 0
+    # I8
+    T0S = _matmul_sparse(T0q, Sq, C, lower)
+    accT, eref = _align([(T0q, eT0), (Sq, eS), (T0S, eT0 + eS)], lower)
+    Toffq, eT = _q8(accT, eref, lower)
+    # I9
+    accTb = {(i, j): Toffq[(i, j)] * int(beta_q[j]) for (i, j) in lower}
+    Tbq, eTb = _q8(accTb, eT - 15, lower)
+
+    # I10
+    def out_rows(Xq, x_exp, d):
+        full = [(i, c) for i in range(C) for c in range(d)]
+        prod = {}
+        diag = {}
+        for (i, c) in full:
+            s = 0
+            for j in range(i):
+                t = Tbq[(i, j)]
+                if t:
+                    s += t * int(Xq[j][c])
+            prod[(i, c)] = s
+            diag[(i, c)] = int(beta_q[i]) * int(Xq[i][c])
+        acc, eref = _align([(prod, eTb + int(x_exp)), (diag, int(x_exp) - 15)], full)
+        q, e = _q8(acc, eref, full)
+        return [[q[(i, c)] for c in range(d)] for i in range(C)], e
+
+    Wq, eW = out_rows(Kq, k_exp, dk)
+    Uq, eU = out_rows(Vq, v_exp, dv)
+    Toff = [[Toffq.get((i, j), 0) for j in range(C)] for i in range(C)]
+    return {"Wq": Wq, "w_exp": eW, "Uq": Uq, "u_exp": eU, "Toffq": Toff, "t_exp": eT,
+            "Aq": [[Aq.get((i, j), 0) for j in range(C)] for i in range(C)], "a_exp": eA,
+            "Eq": [[Eq.get((i, j), 0) for j in range(C)] for i in range(C)], "e_exp": eE,
+            "T0q": [[T0q.get((i, j), 0) for j in range(C)] for i in range(C)], "t0_exp": eT0}
+
+
+# --------------------------------------------------------------------------- numpy int64 evaluator (batched)
+def _bitlen(m: np.ndarray) -> np.ndarray:
+    """bit length of non-negative int64 values."""
+    m = m.astype(np.int64)
+    out = np.zeros(m.shape, dtype=np.int64)
+    v = m.copy()
+    for sh in (32, 16, 8, 4, 2, 1):
+        big = v >= (np.int64(1) << sh)
+        out = out + np.where(big, sh, 0)
+        v = np.where(big, v >> sh, v)
+    return out + (v > 0)
+
+
+def _rsr_np(x: np.ndarray, r: np.ndarray) -> np.ndarray:
+    """Round-half-away right shift by r >= 0 (r broadcastable); r == 0 leaves x unchanged."""
+    r = np.asarray(r, dtype=np.int64)
+    half = np.where(r > 0, np.int64(1) << np.maximum(r - 1, 0), 0)
+    a = (np.abs(x) + half) >> r
+    return np.where(x >= 0, a, -a)
+
+
+def _shift_np(x: np.ndarray, s: np.ndarray) -> np.ndarray:
+    """x * 2^s for s >= 0, rsr for s < 0 (s per chunk, broadcast over the last two axes)."""
+    s = np.asarray(s, dtype=np.int64)[..., None, None]
+    return np.where(s >= 0, x << np.maximum(s, 0), _rsr_np(x, np.maximum(-s, 0)))
+
+
+def _q8_np(acc: np.ndarray, e: np.ndarray, support: np.ndarray):
+    acc = np.where(support, acc, 0).astype(np.int64)
+    m = np.abs(acc).max(axis=(-1, -2))
+    r = np.maximum(0, _bitlen(m) - 7)
+    q = np.clip(_rsr_np(acc, r[..., None, None]), -QMAX, QMAX)
+    return np.where(support, q, 0).astype(np.int64), np.asarray(e, dtype=np.int64) + r
+
+
+def _align_np(terms, support):
+    es = np.stack([np.asarray(e, dtype=np.int64) for _, e in terms])
+    e_ref = np.maximum(es.min(axis=0), es.max(axis=0) - 24)
+    total = 0
+    for x, e in terms:
+        total = total + _shift_np(np.where(support, x, 0).astype(np.int64), np.asarray(e, dtype=np.int64) - e_ref)
+    return total, e_ref
+
+
+def _mm_i32(a: np.ndarray, b: np.ndarray) -> np.ndarray:
+    out = np.matmul(a.astype(np.int64), b.astype(np.int64))
+    assert np.abs(out).max(initial=0) < 2 ** 31, "an MMA accumulator would overflow int32"
+    return out
+
+
+def chunk_prepare_int8(Kq, Vq, k_exp, v_exp, beta_q, decay_q, N: int, S: int):
+    """Batched exact evaluation. Kq [n, C, dk], Vq [n, C, dv] (int), k_exp, v_exp [n], beta_q, decay_q [n, C].
+
+    Returns dict with Wq, Uq (int8 arrays), w_exp, u_exp, Toffq [n, C, C] int8, t_exp and the
+    intermediate tensors Aq, Eq, T0q with their exponents.
+    """
+    Kq = np.asarray(Kq).astype(np.int64)
+    Vq = np.asarray(Vq).astype(np.int64)
+    k_exp = np.asarray(k_exp).astype(np.int64)
+    v_exp = np.asarray(v_exp).astype(np.int64)
+    beta_q = np.asarray(beta_q).astype(np.int64)
+    decay_q = np.asarray(decay_q).astype(np.int64)
+    n, C, dk = Kq.shape
+    lut = np.asarray(decay_lut(), dtype=np.int64)
+    i = np.arange(C)[:, None]
+    j = np.arange(C)[None, :]
+    d = i - j
+    lower = d > 0
+    band = lower & (d <= N)
+    far = d > N
+    # I1-I3
+    G = _mm_i32(Kq, np.swapaxes(Kq, -1, -2))
+    dlt = np.where(lower, decay_q[:, :, None] - decay_q[:, None, :], 0)
+    assert dlt.min() >= 0, "decay_q must be non-decreasing inside a chunk"
+    sh = dlt >> 8
+    gam = np.where(sh < 16, lut[dlt & 255] >> np.minimum(sh, 15), 0)
+    c = (beta_q[:, :, None] * gam + (1 << 14)) >> 15
+    Aq, eA = _q8_np(-(G * c), 2 * k_exp - 15, lower)
+    # I4
+    Aband = np.where(band, Aq, 0)
+    P = [(Aband, eA)]
+    for nn in range(2, N + 1):
+        prev, eprev = P[-1]
+        sup = band & (d >= nn)
+        Pn, en = _q8_np(_mm_i32(prev, Aband), eprev + eA, sup)
+        P.append((Pn, en))
+    # I5
+    accT0, eref = _align_np(P, band)
+    T0q, eT0 = _q8_np(accT0, eref, band)
+    # I6
+    accE, eref = _align_np([(Aq, eA), (_mm_i32(Aq, T0q), eA + eT0)], far)
+    Eq, eE = _q8_np(accE, eref, far)
+    # I7
+    R = []
+    if S >= 1:
+        R.append((Eq, eE))
+        for s in range(2, S + 1):
+            if s * (N + 1) >= C:
+                break
+            sup = d >= s * (N + 1)
+            prev, eprev = R[-1]
+            Rs, es = _q8_np(_mm_i32(prev, Eq), eprev + eE, sup)
+            R.append((Rs, es))
+    if R:
+        accS, eref = _align_np(R, far)
+        Sq, eS = _q8_np(accS, eref, far)
+    else:
+        Sq, eS = np.zeros_like(Aq), np.zeros_like(eA)
+    # I8
+    accT, eref = _align_np([(T0q, eT0), (Sq, eS), (_mm_i32(T0q, Sq), eT0 + eS)], lower)
+    Toffq, eT = _q8_np(accT, eref, lower)
+    # I9
+    Tbq, eTb = _q8_np(Toffq * beta_q[:, None, :], eT - 15, lower)
+
+    # I10
+    def out_rows(Xq, x_exp):
+        full = np.ones((1, 1), dtype=bool)
+        prod = _mm_i32(Tbq, Xq)
+        diag = beta_q[:, :, None] * Xq
+        acc, er = _align_np([(prod, eTb + x_exp), (diag, x_exp - 15)], full)
+        return _q8_np(acc, er, full)
+
+    Wq, eW = out_rows(Kq, k_exp)
+    Uq, eU = out_rows(Vq, v_exp)
+    return {"Wq": Wq.astype(np.int8), "w_exp": eW, "Uq": Uq.astype(np.int8), "u_exp": eU,
+            "Toffq": Toffq.astype(np.int8), "t_exp": eT, "Aq": Aq.astype(np.int8), "a_exp": eA,
+            "Eq": Eq.astype(np.int8), "e_exp": eE, "T0q": T0q.astype(np.int8), "t0_exp": eT0}
+
+
+def dequantise(q: np.ndarray, e: np.ndarray) -> np.ndarray:
+    """q * 2^e per chunk, fp64."""
+    return q.astype(np.float64) * np.exp2(np.asarray(e, dtype=np.float64))[..., None, None]

@@ -141,3 +141,71 @@ def chunk_slices(inp: ChunkInputs, chunk_ids):
                     inp.beta[b, hv, sl].double().cpu().numpy(),
                     inp.g[b, hv, sl].double().cpu().numpy()))
     return out
+
+
+# ----------------------------------------------------------------------------- integer inputs
+@dataclass
+class Int8Inputs:
+    """Integer buffers of the INT8 entry point (prepared once; both the CUDA path and the CPU oracle read them).
+
+    Kq [B,H_k,T,d_k], Vq [B,H_v,T,d_v] int8 with one power-of-two exponent per chunk (k_exp [B,H_k,T/C],
+    v_exp [B,H_v,T/C] int32: value = q * 2^exp); beta_q [B,H_v,T] = round(beta * 2^15) in [0, 32767] stored as
+    int16; decay_q [B,H_v,T] int32 = round(-g * log2(e) * 2^8), non-decreasing inside a chunk.
+    """
+    Kq: torch.Tensor
+    Vq: torch.Tensor
+    k_exp: torch.Tensor
+    v_exp: torch.Tensor
+    beta_q: torch.Tensor
+    decay_q: torch.Tensor
+    B: int
+    H_k: int
+    H_v: int
+    T: int
+    C: int
+    d_k: int
+    d_v: int
+
+    @property
+    def n_chunks(self) -> int:
+        return self.B * self.H_v * (self.T // self.C)
+
+
+def _quantise_per_chunk(x: torch.Tensor, C: int):
+    """Symmetric int8 with the smallest power-of-two scale that keeps max|x| / 2^e <= 127 per chunk."""
+    B, H, T, d = x.shape
+    xf = x.float().view(B, H, T // C, C * d)
+    m = xf.abs().amax(dim=-1).clamp_min(1e-30)
+    e = torch.ceil(torch.log2(m / 127.0)).to(torch.int32)
+    # guard against log2 rounding: raise e where the scaled maximum still exceeds 127
+    e = torch.where(m / torch.exp2(e.float()) > 127.0, e + 1, e)
+    q = torch.round(xf / torch.exp2(e.float()).unsqueeze(-1)).clamp_(-127, 127).to(torch.int8)
+    return q.view(B, H, T, d).contiguous(), e.contiguous()
+
+
+def make_int8_inputs(inp: ChunkInputs) -> Int8Inputs:
+    Kq, k_exp = _quantise_per_chunk(inp.K, inp.C)
+    Vq, v_exp = _quantise_per_chunk(inp.V, inp.C)
+    beta_q = torch.round(inp.beta.float() * 32768.0).clamp_(0, 32767).to(torch.int16).contiguous()
+    decay_q = torch.round(-inp.g.double() * (1.4426950408889634 * 256.0)).to(torch.int32).contiguous()
+    return Int8Inputs(Kq, Vq, k_exp, v_exp, beta_q, decay_q, inp.B, inp.H_k, inp.H_v, inp.T, inp.C, inp.d_k, inp.d_v)
+
+
+def int8_chunk_slices(q: Int8Inputs, chunk_ids):
+    """Host numpy copies of selected chunks: (Kq, Vq, k_exp, v_exp, beta_q, decay_q) stacked over the chunks."""
+    import numpy as np
+    n_c = q.T // q.C
+    group = q.H_v // q.H_k
+    Ks, Vs, ke, ve, bq, dq = [], [], [], [], [], []
+    for cid in chunk_ids:
+        bh, c = divmod(int(cid), n_c)
+        b, hv = divmod(bh, q.H_v)
+        hk = hv // group
+        sl = slice(c * q.C, (c + 1) * q.C)
+        Ks.append(q.Kq[b, hk, sl].cpu().numpy().astype(np.int64))
+        Vs.append(q.Vq[b, hv, sl].cpu().numpy().astype(np.int64))
+        ke.append(int(q.k_exp[b, hk, c]))
+        ve.append(int(q.v_exp[b, hv, c]))
+        bq.append(q.beta_q[b, hv, sl].cpu().numpy().astype(np.int64))
+        dq.append(q.decay_q[b, hv, sl].cpu().numpy().astype(np.int64))
+    return (np.stack(Ks), np.stack(Vs), np.asarray(ke), np.asarray(ve), np.stack(bq), np.stack(dq))

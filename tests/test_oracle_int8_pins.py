@@ -1,0 +1,130 @@
+"""Pins for the exact-integer INT8 oracle: two separately written evaluators, closed forms, the
+quantiser's defining properties and a sanity band against the fp64 definition."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import gdn_oracle as orc
+from oracle import gdn_oracle_int8 as orq
+from paper_2606_06034_b200 import inputs as gen
+
+
+def _int8_chunks(C, n_heads=2, T=None, seed=0, adversarial="none", d=32):
+    T = T or 2 * C
+    inp = gen.make_inputs(1, n_heads, n_heads, T, C, d, d, seed=seed, dtype=torch.float32, adversarial_heads=adversarial)
+    q = gen.make_int8_inputs(inp)
+    return inp, q, gen.int8_chunk_slices(q, range(q.n_chunks))
+
+
+def test_rsr_rounds_half_away_from_zero():
+    assert [orq._rsr(x, 1) for x in (1, -1, 3, -3, 2, -2, 5)] == [1, -1, 2, -2, 1, -1, 3]
+    assert orq._rsr(7, 0) == 7 and orq._rsr(-40, 3) == -5 and orq._rsr(44, 3) == 6 and orq._rsr(43, 3) == 5
+    x = np.array([1, -1, 3, -3, 2, -2, 5, -40, 44, 43])
+    assert list(orq._rsr_np(x, np.array([1, 1, 1, 1, 1, 1, 1, 3, 3, 3]))) == [1, -1, 2, -2, 1, -1, 3, -5, 6, 5]
+
+
+def test_q8_definition():
+    # maximum 1000 has bit length 10 -> shift 3; 1000/8 = 125; the scale comes from the support only
+    acc = {(1, 0): 1000, (2, 0): -1000, (2, 1): 4, (0, 1): 10 ** 9}
+    q, e = orq._q8(acc, -5, [(1, 0), (2, 0), (2, 1)])
+    assert e == -2 and q == {(1, 0): 125, (2, 0): -125, (2, 1): 1}
+    # 1023 -> shift 3 -> 128 -> clamped to 127
+    q, e = orq._q8({(0, 0): 1023}, 0, [(0, 0)])
+    assert q[(0, 0)] == 127 and e == 3
+    # small values are not scaled up
+    q, e = orq._q8({(0, 0): 5}, 7, [(0, 0)])
+    assert q[(0, 0)] == 5 and e == 7
+    for m in (0, 1, 127, 128, 255, 256, 2 ** 40 + 3):
+        assert orq._bitlen(np.array([m]))[0] == m.bit_length()
+
+
+def test_decay_lut():
+    lut = orq.decay_lut()
+    assert len(lut) == 256 and lut[0] == 32768 and lut[255] == round(32768 * 2 ** (-255 / 256))
+    assert all(lut[i] > lut[i + 1] for i in range(255))
+    assert all(abs(lut[f] / 32768 - 2 ** (-f / 256)) <= 0.5 / 32768 + 1e-12 for f in range(256))
+    assert orq.lut_checksum() == orq.lut_checksum(list(lut))
+
+
+@pytest.mark.parametrize("C,N,S,adv", [(8, 2, 1, "none"), (16, 3, 2, "none"), (16, 3, 3, "all"), (32, 3, 4, "none"),
+                                       (64, 3, 8, "none"), (64, 3, 8, "all"), (64, 2, 3, "none"), (32, 1, 0, "none")])
+def test_two_evaluators_agree_bit_for_bit(C, N, S, adv):
+    d = 16 if C >= 64 else 8
+    inp, q, (Kq, Vq, ke, ve, bq, dq) = _int8_chunks(C, T=2 * C if C < 64 else C, seed=C + N + S, adversarial=adv, d=d)
+    fast = orq.chunk_prepare_int8(Kq, Vq, ke, ve, bq, dq, N, S)
+    for c in range(Kq.shape[0]):
+        ref = orq.chunk_prepare_int8_ref(Kq[c].tolist(), Vq[c].tolist(), int(ke[c]), int(ve[c]), bq[c].tolist(), dq[c].tolist(), N, S)
+        for key in ("Wq", "Uq", "Toffq", "Aq", "Eq", "T0q"):
+            assert np.array_equal(np.asarray(ref[key]), fast[key][c]), key
+        for key in ("w_exp", "u_exp", "t_exp", "a_exp", "e_exp", "t0_exp"):
+            assert int(ref[key]) == int(fast[key][c]), key
+
+
+def test_structure_and_ranges():
+    inp, q, (Kq, Vq, ke, ve, bq, dq) = _int8_chunks(64, seed=5, adversarial="all", d=32)
+    out = orq.chunk_prepare_int8(Kq, Vq, ke, ve, bq, dq, 3, 8)
+    i = np.arange(64)[:, None]; j = np.arange(64)[None, :]
+    for key in ("Wq", "Uq", "Toffq", "Aq", "Eq", "T0q"):
+        assert np.abs(out[key].astype(int)).max() <= 127
+    assert np.all(out["Toffq"][:, i <= j] == 0)
+    assert np.all(out["Eq"][:, (i - j) <= 3] == 0)
+    assert np.all(out["T0q"][:, ((i - j) > 3) | (i <= j)] == 0)
+    # the largest mantissa of a requantised tensor uses the top bit range (scale is tight)
+    assert np.all(np.abs(out["Aq"].astype(int)).max(axis=(-1, -2)) >= 64)
+
+
+def test_identical_keys_closed_form_in_integers():
+    """All keys equal to one power-of-two-friendly vector, beta = 1/2, no decay: A = (1/2) L exactly, and the
+    integer pipeline must reproduce T - I = -(1/2)^(i-j) on the entries the 8-bit mantissas can hold."""
+    C, d = 16, 4
+    Kq = np.zeros((1, C, d), dtype=np.int64); Kq[:, :, 0] = 64      # K = e_0 (64 * 2^-6)
+    Vq = np.zeros((1, C, d), dtype=np.int64); Vq[:, :, 1] = 32
+    ke = np.array([-6]); ve = np.array([-5])
+    bq = np.full((1, C), 16384); dq = np.zeros((1, C), dtype=np.int64)
+    out = orq.chunk_prepare_int8(Kq, Vq, ke, ve, bq, dq, 3, 3)
+    A = orq.dequantise(out["Aq"], out["a_exp"])[0]
+    assert np.array_equal(A, -0.5 * np.tril(np.ones((C, C)), -1))
+    T = orq.dequantise(out["Toffq"], out["t_exp"])[0]
+    i = np.arange(C)[:, None]; j = np.arange(C)[None, :]
+    exact = np.where(i > j, -(0.5 ** np.maximum(i - j, 1)), 0.0)
+    step = 2.0 ** float(out["t_exp"][0])
+    assert np.abs(T - exact).max() <= 1.5 * step          # within the final mantissa's resolution (+ chain rounding)
+    assert np.array_equal(T[(i - j == 1)], exact[(i - j == 1)])
+    # W_i = beta (1-beta)^i K_i on the first column
+    W = orq.dequantise(out["Wq"], out["w_exp"])[0]
+    expect = 0.5 * 0.5 ** np.arange(C)
+    assert np.abs(W[:, 0] - expect).max() <= 2.0 ** float(out["w_exp"][0]) * 1.5 + 2 * step
+
+
+@pytest.mark.parametrize("adv,lo_T,lo_WU", [("none", 25.0, 28.0), ("all", 20.0, 20.0)])
+def test_dequantised_result_tracks_the_fp64_definition(adv, lo_T, lo_WU):
+    """Sanity band: the integer pipeline, dequantised, stays within an 8-bit SNR band of the fp64 inverse of the
+    same (dequantised) inputs. Guards against a wrong exponent or a dropped term, not a precision claim."""
+    inp, q, (Kq, Vq, ke, ve, bq, dq) = _int8_chunks(64, n_heads=2, T=128, seed=9, adversarial=adv, d=64)
+    out = orq.chunk_prepare_int8(Kq, Vq, ke, ve, bq, dq, 3, 8)
+    K = Kq * np.exp2(ke.astype(float))[:, None, None]
+    V = Vq * np.exp2(ve.astype(float))[:, None, None]
+    beta = bq / 32768.0
+    g = -dq / (256.0 * 1.4426950408889634)
+    We, Ue, Te = orc.chunk_prepare(K, V, beta, g, exact=True)
+    T = orq.dequantise(out["Toffq"], out["t_exp"])
+    W = orq.dequantise(out["Wq"], out["w_exp"])
+    U = orq.dequantise(out["Uq"], out["u_exp"])
+    eye = np.eye(64)
+    assert orc.snr_db(T, Te - eye).min() > lo_T
+    assert orc.snr_db(W, We).min() > lo_WU
+    assert orc.snr_db(U, Ue).min() > lo_WU
+
+
+def test_int8_input_recipe():
+    inp = gen.make_inputs(1, 2, 4, 128, 64, 32, 32, seed=3)
+    q = gen.make_int8_inputs(inp)
+    assert q.Kq.dtype == torch.int8 and q.k_exp.shape == (1, 2, 2) and q.v_exp.shape == (1, 4, 2)
+    assert int(q.Kq.abs().max()) <= 127 and int(q.Kq.view(1, 2, 2, -1).abs().amax(-1).min()) >= 64
+    assert int(q.beta_q.min()) >= 0
+    dd = q.decay_q.view(1, 4, 2, 64).diff(dim=-1)
+    assert (dd >= 0).all()
+    back = q.Kq.float().view(1, 2, 2, 64, 32) * torch.exp2(q.k_exp.float())[..., None, None]
+    assert (back.view_as(inp.K) - inp.K.float()).abs().max() <= torch.exp2(q.k_exp.float()).max() * 0.5 + 1e-6
