@@ -101,6 +101,28 @@ int gdn_chunk_prepare_fwdsubst(const void* K, const void* V, const float* beta, 
                                void* W_out, void* U_out, void* Tinv_out, gdn_stream_t stream);
 
 /*
+ * INT8 variant (Sec. 3.5 "good enough under low-bit quantization"; quantiser of App. G, Eq. 32): every tensor of
+ * the chain is int8 mantissas in [-127, 127] with one power-of-two exponent per chunk, int32 accumulation on the
+ * tensor cores, requantisation after every product and sum with the structural mask applied first. The outputs
+ * are a pure function of the integer inputs (bit-exact against an exact-integer evaluation).
+ *   Kq [B,H_k,T,d_k], Vq [B,H_v,T,d_v] int8; k_exp [B,H_k,T/C], v_exp [B,H_v,T/C]: value = q * 2^exp;
+ *   beta_q [B,H_v,T] = round(beta * 2^15) in [0, 32767]; decay_q [B,H_v,T] = round(-g * log2(e) * 2^8),
+ *   non-decreasing inside every chunk (not checked).
+ *   Wq_out [B,H_v,T,d_k], Uq_out [B,H_v,T,d_v] int8 with w_exp_out, u_exp_out [B,H_v,T/C];
+ *   Toff_q_out [B,H_v,T/C,C,C] int8 (may be NULL) with t_exp_out [B,H_v,T/C]: T = I + Toff_q * 2^t_exp.
+ * Supported: C = 64, d_k = d_v = 128, 1 <= order <= 3 (the paper's low-bit limit), residual_steps <= 8.
+ */
+int gdn_chunk_prepare_int8(const int8_t* Kq, const int8_t* Vq, const int32_t* k_exp, const int32_t* v_exp,
+                           const uint16_t* beta_q, const int32_t* decay_q,
+                           int B, int H_k, int H_v, int T, int C, int d_k, int d_v, int order, int residual_steps,
+                           int8_t* Wq_out, int8_t* Uq_out, int32_t* w_exp_out, int32_t* u_exp_out,
+                           int8_t* Toff_q_out, int32_t* t_exp_out, gdn_stream_t stream);
+
+/* Checksum of the 256-entry gate-decay table round(2^15 * 2^(-f/256)) the INT8 kernel uses
+ * (sum_f: s = (31 s + table[f] + f) mod 1000000007), so that a CPU evaluation can confirm it holds the same table. */
+unsigned int gdn_int8_lut_checksum(void);
+
+/*
  * Waits for `stream`, then returns and clears the status word the kernels of
  * this library write on the current device: GDN_OK, or GDN_ERR_TIMEOUT when a
  * bounded wait inside a kernel gave up (its outputs are then undefined).

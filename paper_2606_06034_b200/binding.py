@@ -29,7 +29,8 @@ GDN_FWDSUBST_ROWS = 0
 GDN_FWDSUBST_BLOCKED = 1
 
 EXPORTS = (
-    "gdn_chunk_prepare", "gdn_chunk_prepare_gqa", "gdn_chunk_prepare_fwdsubst",
+    "gdn_chunk_prepare", "gdn_chunk_prepare_gqa", "gdn_chunk_prepare_fwdsubst", "gdn_chunk_prepare_int8",
+    "gdn_int8_lut_checksum",
     "gdn_device_status", "gdn_default_order", "gdn_default_residual_steps",
     "gdn_status_string", "gdn_launch_count",
 )
@@ -60,6 +61,10 @@ def load_library() -> ctypes.CDLL:
     lib.gdn_chunk_prepare_gqa.argtypes = [vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ip, ip, ip, ip, vp, vp, vp, vp]
     lib.gdn_chunk_prepare_fwdsubst.restype = ip
     lib.gdn_chunk_prepare_fwdsubst.argtypes = [vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ip, ip, ip, vp, vp, vp, vp]
+    lib.gdn_chunk_prepare_int8.restype = ip
+    lib.gdn_chunk_prepare_int8.argtypes = [vp, vp, vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ip, ip, ip, vp, vp, vp, vp, vp, vp, vp]
+    lib.gdn_int8_lut_checksum.restype = ctypes.c_uint
+    lib.gdn_int8_lut_checksum.argtypes = []
     lib.gdn_device_status.restype = ip
     lib.gdn_device_status.argtypes = [vp]
     lib.gdn_default_order.restype = ip
@@ -157,6 +162,46 @@ def gdn_chunk_prepare_fwdsubst(K, V, beta, g, B, H_k, H_v, T, C, d_k, d_v, dtype
     if check and rc != GDN_OK:
         raise GdnError(rc, "gdn_chunk_prepare_fwdsubst")
     return rc
+
+
+def gdn_int8_lut_checksum() -> int:
+    return int(load_library().gdn_int8_lut_checksum())
+
+
+def gdn_chunk_prepare_int8(Kq, Vq, k_exp, v_exp, beta_q, decay_q, B, H_k, H_v, T, C, d_k, d_v, order, residual_steps,
+                           Wq_out, Uq_out, w_exp_out, u_exp_out, Toff_q_out, t_exp_out, *, check=True):
+    """Raw call of the INT8 entry point (tensors instead of pointers, torch's current stream)."""
+    for t in (Kq, Vq, k_exp, v_exp, beta_q, decay_q, Wq_out, Uq_out, w_exp_out, u_exp_out, t_exp_out):
+        if not t.is_cuda or not t.is_contiguous():
+            raise ValueError("all tensors must be contiguous CUDA tensors (there is no CPU path)")
+    rc = load_library().gdn_chunk_prepare_int8(_ptr(Kq), _ptr(Vq), _ptr(k_exp), _ptr(v_exp), _ptr(beta_q), _ptr(decay_q),
+                                               B, H_k, H_v, T, C, d_k, d_v, order, residual_steps, _ptr(Wq_out),
+                                               _ptr(Uq_out), _ptr(w_exp_out), _ptr(u_exp_out), _ptr(Toff_q_out),
+                                               _ptr(t_exp_out), _stream())
+    if check and rc != GDN_OK:
+        raise GdnError(rc, "gdn_chunk_prepare_int8")
+    return rc
+
+
+def chunk_prepare_int8(q, order=-1, residual_steps=-1, *, want_toff=True, outputs=None):
+    """Convenience wrapper over integer inputs (an `inputs.Int8Inputs` whose tensors live on the GPU).
+
+    Returns (Wq, Uq, w_exp, u_exp, Toff_q, t_exp).
+    """
+    dev = q.Kq.device
+    n_c = q.T // q.C
+    if outputs is None:
+        Wq = torch.empty(q.B, q.H_v, q.T, q.d_k, dtype=torch.int8, device=dev)
+        Uq = torch.empty(q.B, q.H_v, q.T, q.d_v, dtype=torch.int8, device=dev)
+        w_exp = torch.empty(q.B, q.H_v, n_c, dtype=torch.int32, device=dev)
+        u_exp = torch.empty_like(w_exp)
+        t_exp = torch.empty_like(w_exp)
+        Toff = torch.empty(q.B, q.H_v, n_c, q.C, q.C, dtype=torch.int8, device=dev) if want_toff else None
+        outputs = (Wq, Uq, w_exp, u_exp, Toff, t_exp)
+    Wq, Uq, w_exp, u_exp, Toff, t_exp = outputs
+    gdn_chunk_prepare_int8(q.Kq, q.Vq, q.k_exp, q.v_exp, q.beta_q, q.decay_q, q.B, q.H_k, q.H_v, q.T, q.C, q.d_k, q.d_v,
+                           order, residual_steps, Wq, Uq, w_exp, u_exp, Toff, t_exp)
+    return outputs
 
 
 def gdn_device_status() -> int:

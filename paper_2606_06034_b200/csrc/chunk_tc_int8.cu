@@ -1,0 +1,776 @@
+// INT8 variant of the chunk-prepare path on the tensor cores (tcgen05 kind::i8, int32 accumulators in TMEM).
+//
+// Every tensor of the chain is int8 mantissas in [-127, 127] with one power-of-two exponent per chunk; the
+// exponent of each requantised tensor comes from the bit length of the largest magnitude on its structural
+// support (CTA-wide OR reduction per chunk), so the result is a pure function of the integer inputs and can be
+// compared bit for bit with an exact-integer evaluation on the CPU. The paper fixes the uniform symmetric
+// quantiser (App. G, Eq. 32), one scale per tensor, N <= 3 with residual correction (Sec. 3.5) and the band
+// mask (Sec. 3.3); where quantisation is re-applied and how scales are chosen is this build's reading:
+//
+//   rsr(x, r)  = sign(x) ((|x| + 2^(r-1)) >> r)
+//   Q8(acc, e) : r = max(0, bitlen(max |acc| on the support) - 7); q = clamp(rsr(acc, r), +-127); exponent e + r
+//   align(..)  : e_ref = max(min e, max e - 24); terms shifted to e_ref (left shift, or rsr) and summed in int64
+//
+//   G = Kq Kq^T                                   MMA (K tile by TMA, 128-byte swizzle)
+//   Aq   = Q8(-(G o c), 2 k_exp - 15),  c = (beta_q_i Gam_ij + 2^14) >> 15, Gam from a 256-entry table of 2^(-f/256)
+//   P_n  = Q8(band(P_{n-1} band(Aq))), n = 2..N;  T0q = Q8(align(P_1..P_N))                      integer ALU, band only
+//   Eq   = Q8(align(Aq, Aq T0q)) on i-j > N                                                       integer ALU
+//   R_1 = Eq, R_s = Q8(R_{s-1} Eq) on i-j >= s(N+1)                                               MMA per power
+//   Sq   = Q8(align(R_1..));  Toffq = Q8(align(T0q, Sq, T0q Sq));  Tbq = Q8(Toffq_ij beta_q_j)    integer ALU
+//   Wq   = Q8(align(Tbq Kq, beta_q_i Kq_i)), Uq likewise                                          MMA + ALU
+//
+// Work item, thread mapping, barriers and stores follow the bf16 kernel: tile of 128 tokens (two 64-chunks),
+// threads t and t + 128 share tile row t and split its 64 chunk columns, thread 0 issues TMA and MMAs.
+#include <cuda.h>
+
+#include "common.cuh"
+#include "sm100_ptx.cuh"
+
+namespace gdn {
+namespace {
+
+using namespace sm100;
+
+constexpr int kTile = 128;
+constexpr int kThreads = 256;
+constexpr int kD = 128;
+constexpr int kC = 64;     // chunk size handled by this kernel
+constexpr int kHC = 32;    // chunk columns per thread
+constexpr int kSMax = 8;   // largest number of residual terms held in registers
+constexpr uint32_t kR0 = 0, kAS = 128, kTmemCols = 256;
+
+struct ParamsI8 {
+    const int16_t* beta_q;
+    const int32_t* decay_q;
+    const int32_t* k_exp;
+    const int32_t* v_exp;
+    int32_t* w_exp;
+    int32_t* u_exp;
+    int32_t* t_exp;
+    int8_t* Toff;  // may be null
+    int* status;
+    int H_k, H_v, T, group, n_tt;
+    int N, S;
+    long long n_tiles;
+    uint16_t lut[256];
+};
+
+// shared memory map (bytes)
+constexpr int kOffK = 0;                 // 16 KB int8 K tile, 128-byte swizzle
+constexpr int kOffV = 16384;             // 16 KB int8 V tile
+constexpr int kOffEB = 32768;            // 8 KB: Eq as B operand [64 x 128] (MN-major, no swizzle)
+constexpr int kOffRowA = 40960;          // 8 KB: one private 64-byte row per tile row (Aq bytes, later Sq bytes)
+constexpr int kOffStage = 49152;         // 24 KB: staging of Toff (8 KB) and of W / U (4 warps x 2 halves x 2 KB)
+constexpr int kOffSH = 73728;            // column form of T0q: [128 + 8][4] int
+constexpr int kOffAB = kOffSH + 136 * 16;  // row form: Aq next to the diagonal / P2q: [128][8] int
+constexpr int kOffBeta = kOffAB + 128 * 32;
+constexpr int kOffDecay = kOffBeta + 512;
+constexpr int kOffLut = kOffDecay + 512;
+constexpr int kOffRed = kOffLut + 512;     // OR-reduction slots: [24][2 chunks][2 words]
+constexpr int kNumRed = 24;
+constexpr int kSmemTotal = kOffRed + kNumRed * 16;
+
+__device__ __forceinline__ void cta_barrier() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+
+__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    uint32_t i = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++i & 1023u) == 0 && clock64() - t0 > 2000000000LL) return false;
+    }
+    return true;
+}
+
+__device__ __forceinline__ long long rsr64(long long x, int r) {
+    if (r <= 0) return x;
+    const long long a = ((x < 0 ? -x : x) + (1LL << (r - 1))) >> r;
+    return x < 0 ? -a : a;
+}
+// x * 2^s for s >= 0, rounded right shift otherwise
+__device__ __forceinline__ long long shift64(long long x, int s) { return s >= 0 ? (x << s) : rsr64(x, -s); }
+__device__ __forceinline__ int clamp127(long long q) { return q > 127 ? 127 : (q < -127 ? -127 : static_cast<int>(q)); }
+__device__ __forceinline__ int q8_shift(int bitlen) { return bitlen > 7 ? bitlen - 7 : 0; }
+__device__ __forceinline__ int align_ref2(int e0, int e1) {
+    const int lo = e0 < e1 ? e0 : e1, hi = e0 < e1 ? e1 : e0;
+    return lo > hi - 24 ? lo : hi - 24;
+}
+__device__ __forceinline__ uint32_t pack4(int a, int b, int c, int d) {
+    return (static_cast<uint32_t>(a) & 0xFFu) | ((static_cast<uint32_t>(b) & 0xFFu) << 8) | ((static_cast<uint32_t>(c) & 0xFFu) << 16) |
+           ((static_cast<uint32_t>(d) & 0xFFu) << 24);
+}
+__device__ __forceinline__ int byte_at(uint32_t w, int i) { return static_cast<int>(static_cast<int8_t>((w >> (8 * i)) & 0xFFu)); }
+
+struct TileCoord {
+    int bhk, bhv, t0;
+};
+__device__ __forceinline__ TileCoord decode_tile(uint32_t tile, const ParamsI8& p) {
+    TileCoord c;
+    const uint32_t y = tile / static_cast<uint32_t>(p.group);
+    const uint32_t gi = tile - y * p.group;
+    const uint32_t bhk = y / static_cast<uint32_t>(p.n_tt);
+    const uint32_t tt = y - bhk * p.n_tt;
+    const uint32_t b = bhk / static_cast<uint32_t>(p.H_k);
+    const uint32_t hk = bhk - b * p.H_k;
+    c.bhk = static_cast<int>(bhk);
+    c.bhv = static_cast<int>(b * p.H_v + hk * p.group + gi);
+    c.t0 = static_cast<int>(tt) * kTile;
+    return c;
+}
+
+__global__ void __launch_bounds__(kThreads, 2)
+chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                     const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmU,
+                     const __grid_constant__ CUtensorMap tmT, const __grid_constant__ ParamsI8 p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* sK = smem + kOffK;
+    uint8_t* sV = smem + kOffV;
+    uint8_t* sEB = smem + kOffEB;
+    uint8_t* sRowA = smem + kOffRowA;
+    int* sSH = reinterpret_cast<int*>(smem + kOffSH);
+    int* sAB = reinterpret_cast<int*>(smem + kOffAB);
+    int* sbeta = reinterpret_cast<int*>(smem + kOffBeta);
+    int* sdecay = reinterpret_cast<int*>(smem + kOffDecay);
+    uint16_t* slut = reinterpret_cast<uint16_t*>(smem + kOffLut);
+    uint32_t* sred = reinterpret_cast<uint32_t*>(smem + kOffRed);
+
+    __shared__ uint64_t bar_k, bar_v, bar_mma;
+    __shared__ uint32_t tmem_base_s;
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    const int lane = tid & 31;
+
+    if (tid == 0) {
+        mbar_init(&bar_k, 1);
+        mbar_init(&bar_v, 1);
+        mbar_init(&bar_mma, 1);
+        mbar_fence_init();
+        tma_prefetch_desc(&tmK);
+        tma_prefetch_desc(&tmV);
+        tma_prefetch_desc(&tmW);
+        tma_prefetch_desc(&tmU);
+        tma_prefetch_desc(&tmT);
+    }
+    slut[tid] = p.lut[tid];
+    if (warp == 0) {
+        tmem_alloc(&tmem_base_s, kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = tmem_base_s;
+
+    const int N = p.N, S = p.S;
+    const uint32_t n_tiles = static_cast<uint32_t>(p.n_tiles);
+    const int n_c = p.T / kC;  // chunks per head
+
+    const int t = tid & 127;        // tile row
+    const int h = tid >> 7;         // column half
+    const int col0 = h * kHC;       // first chunk column of this thread
+    const int il = t & (kC - 1);    // row inside the chunk
+    const int cb = t - il;          // first tile row of the chunk
+    const int ci = t >> 6;          // chunk of the tile
+    const int wq = warp & 3;
+    const int wrow0 = wq * 32;
+    const uint32_t lane_base = tmem + (static_cast<uint32_t>(wq * 32) << 16);
+    const uint32_t sK_a = smem_u32(sK), sV_a = smem_u32(sV), sEB_a = smem_u32(sEB);
+    const uint32_t idesc_g = instr_desc(128, 128, 1, 1, 0, 0, 2);  // s8 x s8 -> s32, both K-major
+    const uint32_t idesc_m = instr_desc(128, 128, 1, 1, 0, 1, 2);  // B MN-major
+    uint32_t par_mma = 0, par_kv = 0;
+    bool ok = true;
+
+    // bit length of the OR of |values| over the chunk; `slot` is a fresh reduction slot of this tile
+    auto chunk_bitlen = [&](unsigned long long m, int slot) -> int {
+        uint32_t lo = __reduce_or_sync(0xFFFFFFFFu, static_cast<uint32_t>(m));
+        uint32_t hi = __reduce_or_sync(0xFFFFFFFFu, static_cast<uint32_t>(m >> 32));
+        if (lane == 0) {
+            if (lo) atomicOr(&sred[(slot * 2 + ci) * 2 + 0], lo);
+            if (hi) atomicOr(&sred[(slot * 2 + ci) * 2 + 1], hi);
+        }
+        cta_barrier();
+        const unsigned long long all =
+            (static_cast<unsigned long long>(sred[(slot * 2 + ci) * 2 + 1]) << 32) | sred[(slot * 2 + ci) * 2 + 0];
+        return all ? 64 - __clzll(static_cast<long long>(all)) : 0;
+    };
+    auto absll = [](long long x) -> unsigned long long { return static_cast<unsigned long long>(x < 0 ? -x : x); };
+
+    if (tid == 0 && blockIdx.x < n_tiles) {
+        const TileCoord c = decode_tile(blockIdx.x, p);
+        mbar_arrive_expect_tx(&bar_k, 16384);
+        tma_load_3d(sK, &tmK, &bar_k, 0, c.t0, c.bhk);
+        mbar_arrive_expect_tx(&bar_v, 16384);
+        tma_load_3d(sV, &tmV, &bar_v, 0, c.t0, c.bhv);
+    }
+
+    for (uint32_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        const TileCoord tc = decode_tile(tile, p);
+        const uint32_t next = tile + gridDim.x;
+        const bool has_next = next < n_tiles;
+        const bool row_valid = (tc.t0 + t) < p.T;
+        const long long grow = (long long)tc.bhv * p.T + tc.t0 + t;
+        const int chunk_in_head = (tc.t0 + cb) / kC;
+        const bool chunk_valid = (tc.t0 + cb) < p.T;
+
+        int bq = 0, dq = 0, kexp = 0, vexp = 0;
+        if (row_valid) {
+            bq = static_cast<int>(static_cast<uint16_t>(p.beta_q[grow]));
+            dq = p.decay_q[grow];
+        }
+        if (chunk_valid) {
+            kexp = p.k_exp[(long long)tc.bhk * n_c + chunk_in_head];
+            vexp = p.v_exp[(long long)tc.bhv * n_c + chunk_in_head];
+        }
+        if (lane == 0) tma_store_wait_read<0>();
+        tc_fence_before_sync();
+        cta_barrier();  // previous tile finished with shared arrays and accumulators
+        if (tid == 0) {
+            if (!wait_bar(&bar_k, par_kv)) ok = false;
+            if (ok) {
+                tc_fence_after_sync();
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) {
+                    const uint64_t d = smem_desc(sK_a + ks * 32, 16, 1024, SWZ_128B);
+                    mma_i8_ss(tmem + kR0, d, d, idesc_g, ks > 0);
+                }
+                mma_commit(&bar_mma);
+            }
+        }
+        if (h == 0) {
+            sbeta[t] = bq;
+            sdecay[t] = dq;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) sSH[t * 4 + e] = 0;
+            if (t < 8) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) sSH[(kTile + t) * 4 + e] = 0;
+            }
+        }
+        if (tid < kNumRed * 4) sred[tid] = 0u;
+        cta_barrier();
+        int slot = 0;
+
+        // ---- I1-I3: Aq = Q8(-(G o c))
+        if (!wait_bar(&bar_mma, par_mma)) { ok = false; break; }
+        par_mma ^= 1;
+        tc_fence_after_sync();
+        int aq[kHC];
+        int eA;
+        {
+            uint32_t g[kHC];
+            tmem_ld32(lane_base + kR0 + cb + col0, g);
+            tmem_wait_ld();
+            // the products are formed twice (once for the scale, once for the mantissas) instead of kept in registers
+            auto acc_a = [&](int jl) -> long long {
+                const int j = col0 + jl;
+                if (j >= il) return 0;
+                const int dlt = dq - sdecay[cb + j];
+                const int sh = dlt >> 8;
+                const int gam = (sh < 16) ? (static_cast<int>(slut[dlt & 255]) >> sh) : 0;
+                const int c = (bq * gam + (1 << 14)) >> 15;
+                return -static_cast<long long>(static_cast<int>(g[jl])) * c;
+            };
+            unsigned long long m = 0;
+#pragma unroll
+            for (int jl = 0; jl < kHC; ++jl) m |= absll(acc_a(jl));
+            const int r = q8_shift(chunk_bitlen(m, slot++));
+#pragma unroll
+            for (int jl = 0; jl < kHC; ++jl) aq[jl] = clamp127(rsr64(acc_a(jl), r));
+            eA = 2 * kexp - 15 + r;
+        }
+        // Aq bytes to the private row; entries next to the diagonal and right of this half come back from there
+        uint8_t* rowa = sRowA + t * 64;
+        {
+            uint4 v0, v1;
+            v0.x = pack4(aq[0], aq[1], aq[2], aq[3]);     v0.y = pack4(aq[4], aq[5], aq[6], aq[7]);
+            v0.z = pack4(aq[8], aq[9], aq[10], aq[11]);   v0.w = pack4(aq[12], aq[13], aq[14], aq[15]);
+            v1.x = pack4(aq[16], aq[17], aq[18], aq[19]); v1.y = pack4(aq[20], aq[21], aq[22], aq[23]);
+            v1.z = pack4(aq[24], aq[25], aq[26], aq[27]); v1.w = pack4(aq[28], aq[29], aq[30], aq[31]);
+            *reinterpret_cast<uint4*>(rowa + col0) = v0;
+            *reinterpret_cast<uint4*>(rowa + col0 + 16) = v1;
+        }
+        cta_barrier();
+        int ab[4], anext[4];
+        ab[0] = 0;
+#pragma unroll
+        for (int e = 1; e <= 3; ++e) ab[e] = (il - e >= 0) ? static_cast<int>(static_cast<int8_t>(rowa[il - e])) : 0;
+#pragma unroll
+        for (int e = 0; e < 3; ++e) anext[e] = (h == 0) ? static_cast<int>(static_cast<int8_t>(rowa[kHC + e])) : 0;
+        anext[3] = 0;
+        // P_1 = band of Aq: zero beyond distance N
+        int p1[4];
+#pragma unroll
+        for (int e = 0; e <= 3; ++e) p1[e] = (e >= 1 && e <= N) ? ab[e] : 0;
+        if (h == 0) {
+            sAB[t * 8 + 1] = p1[1];
+            sAB[t * 8 + 2] = p1[2];
+            sAB[t * 8 + 3] = p1[3];
+        }
+        cta_barrier();
+
+        // ---- I4: P_2, P_3 (band only), I5: T0q
+        int t0q[4] = {0, 0, 0, 0};
+        int eT0;
+        {
+            const int r1 = (t - 1) > 0 ? (t - 1) : 0, r2 = (t - 2) > 0 ? (t - 2) : 0;
+            // P_2 on distances 2..N
+            int acc2[4] = {0, 0, 0, 0};
+            acc2[2] = p1[1] * sAB[r1 * 8 + 1];
+            acc2[3] = p1[1] * sAB[r1 * 8 + 2] + p1[2] * sAB[r2 * 8 + 1];
+            if (N < 2) acc2[2] = 0;
+            if (N < 3) acc2[3] = 0;
+            int p2[4] = {0, 0, 0, 0}, p3 = 0;
+            int e2 = 0, e3 = 0;
+            if (N >= 2) {
+                unsigned long long m = (h == 0) ? (absll(acc2[2]) | absll(acc2[3])) : 0ull;
+                const int r = q8_shift(chunk_bitlen(m, slot++));
+                p2[2] = clamp127(rsr64(acc2[2], r));
+                p2[3] = clamp127(rsr64(acc2[3], r));
+                e2 = eA + eA + r;
+            }
+            if (N >= 3) {
+                // P_3 at distance 3: P_2[i][i-2] * Aq[i-2][i-3]
+                const int acc3 = p2[2] * sAB[r2 * 8 + 1];
+                const int r = q8_shift(chunk_bitlen((h == 0) ? absll(acc3) : 0ull, slot++));
+                p3 = clamp127(rsr64(acc3, r));
+                e3 = e2 + eA + r;
+            }
+            // align(P_1..P_N)
+            int emin = eA, emax = eA;
+            if (N >= 2) { emin = min(emin, e2); emax = max(emax, e2); }
+            if (N >= 3) { emin = min(emin, e3); emax = max(emax, e3); }
+            const int eref = max(emin, emax - 24);
+            long long accT[4] = {0, 0, 0, 0};
+#pragma unroll
+            for (int d = 1; d <= 3; ++d) {
+                long long s = shift64(p1[d], eA - eref);
+                if (N >= 2 && d >= 2) s += shift64(p2[d], e2 - eref);
+                if (N >= 3 && d >= 3) s += shift64(p3, e3 - eref);
+                accT[d] = (d <= N && il - d >= 0) ? s : 0;
+            }
+            unsigned long long m = (h == 0) ? (absll(accT[1]) | absll(accT[2]) | absll(accT[3])) : 0ull;
+            const int r = q8_shift(chunk_bitlen(m, slot++));
+#pragma unroll
+            for (int d = 1; d <= 3; ++d) t0q[d] = clamp127(rsr64(accT[d], r));
+            eT0 = eref + r;
+            if (h == 0) {
+#pragma unroll
+                for (int e = 1; e <= 3; ++e)
+                    if (il - e >= 0) sSH[(t - e) * 4 + (e - 1)] = t0q[e];
+            }
+            cta_barrier();
+        }
+
+        // ---- I6: Eq = Q8(align(Aq, Aq T0q)) on i-j > N
+        int eq[kHC];
+        int eE;
+        {
+            const int eref = align_ref2(eA, eA + eT0);
+            auto acc_e = [&](int jl) -> long long {
+                if (il - (col0 + jl) <= N) return 0;
+                const int4 c4 = *reinterpret_cast<const int4*>(sSH + (cb + col0 + jl) * 4);
+                const int cc[3] = {c4.x, c4.y, c4.z};
+                int prod = 0;
+#pragma unroll
+                for (int e = 1; e <= 3; ++e) {
+                    const int k = jl + e;
+                    const int ak = (k < kHC) ? aq[(k < kHC) ? k : 0] : anext[(k >= kHC) ? k - kHC : 0];
+                    prod += ak * cc[e - 1];
+                }
+                return shift64(aq[jl], eA - eref) + shift64(prod, eA + eT0 - eref);
+            };
+            unsigned long long m = 0;
+#pragma unroll
+            for (int jl = 0; jl < kHC; ++jl) m |= absll(acc_e(jl));
+            const int r = q8_shift(chunk_bitlen(m, slot++));
+#pragma unroll
+            for (int jl = 0; jl < kHC; ++jl) eq[jl] = clamp127(rsr64(acc_e(jl), r));
+            eE = eref + r;
+        }
+        // packed rows of the powers R_s (R_1 = Eq) and their exponents
+        uint32_t rpk[kSMax][kHC / 4];
+        int er[kSMax];
+        int n_terms = 0;
+        if (S >= 1) {
+#pragma unroll
+            for (int w = 0; w < kHC / 4; ++w) rpk[0][w] = pack4(eq[4 * w], eq[4 * w + 1], eq[4 * w + 2], eq[4 * w + 3]);
+            er[0] = eE;
+            n_terms = 1;
+            // B operand [E_1 | E_2] (64 x 128 int8, MN-major, no swizzle): 16 columns of chunk-row il per 16-byte piece
+#pragma unroll
+            for (int c = 0; c < kHC / 16; ++c) {
+                const uint4 v = make_uint4(rpk[0][4 * c], rpk[0][4 * c + 1], rpk[0][4 * c + 2], rpk[0][4 * c + 3]);
+                *reinterpret_cast<uint4*>(sEB + (((cb + col0) >> 4) + c) * (16 * kC) + il * 16) = v;
+            }
+        }
+        // ---- I7: R_s = Q8(R_{s-1} Eq) while s (N+1) < C
+#pragma unroll
+        for (int s = 2; s <= kSMax; ++s) {
+            if (s > S || s * (N + 1) >= kC) break;
+            {
+                uint32_t r8[8];
+#pragma unroll
+                for (int w = 0; w < 8; ++w) r8[w] = rpk[s - 2][w];
+                tmem_st8(lane_base + kAS + h * 8, r8);
+            }
+            fence_proxy_async_smem();
+            tmem_wait_st();
+            tc_fence_before_sync();
+            cta_barrier();
+            if (tid == 0) {
+                tc_fence_after_sync();
+#pragma unroll
+                for (int ks = 0; ks < kC / 32; ++ks) {
+                    const uint64_t bd = smem_desc(sEB_a + ks * 512, 128, 16 * kC, SWZ_NONE);
+                    mma_i8_ts(tmem + kR0, tmem + kAS + ks * 8, bd, idesc_m, ks > 0);
+                }
+                mma_commit(&bar_mma);
+            }
+            if (!wait_bar(&bar_mma, par_mma)) { ok = false; break; }
+            par_mma ^= 1;
+            tc_fence_after_sync();
+            uint32_t dres[kHC];
+            tmem_ld32(lane_base + kR0 + cb + col0, dres);
+            tmem_wait_ld();
+            unsigned long long m = 0;
+#pragma unroll
+            for (int jl = 0; jl < kHC; ++jl) {
+                int v = static_cast<int>(dres[jl]);
+                if (il - (col0 + jl) < s * (N + 1)) v = 0;
+                dres[jl] = static_cast<uint32_t>(v);
+                m |= absll(v);
+            }
+            const int r = q8_shift(chunk_bitlen(m, slot++));
+#pragma unroll
+            for (int w = 0; w < kHC / 4; ++w)
+                rpk[s - 1][w] = pack4(clamp127(rsr64(static_cast<int>(dres[4 * w]), r)), clamp127(rsr64(static_cast<int>(dres[4 * w + 1]), r)),
+                                      clamp127(rsr64(static_cast<int>(dres[4 * w + 2]), r)), clamp127(rsr64(static_cast<int>(dres[4 * w + 3]), r)));
+            er[s - 1] = er[s - 2] + eE + r;
+            n_terms = s;
+        }
+        if (!ok) break;
+
+        // ---- Sq = Q8(align(R_1..))
+        int sq[kHC];
+        int eS = 0;
+        if (n_terms > 0) {
+            int emin = er[0], emax = er[0];
+#pragma unroll
+            for (int s = 1; s < kSMax; ++s)
+                if (s < n_terms) { emin = min(emin, er[s]); emax = max(emax, er[s]); }
+            const int eref = max(emin, emax - 24);
+            auto acc_s = [&](int jl) -> long long {
+                long long a = 0;
+#pragma unroll
+                for (int s = 0; s < kSMax; ++s)
+                    if (s < n_terms) a += shift64(byte_at(rpk[s][jl >> 2], jl & 3), er[s] - eref);
+                return a;
+            };
+            unsigned long long m = 0;
+#pragma unroll
+            for (int jl = 0; jl < kHC; ++jl) m |= absll(acc_s(jl));
+            const int r = q8_shift(chunk_bitlen(m, slot++));
+#pragma unroll
+            for (int jl = 0; jl < kHC; ++jl) sq[jl] = clamp127(rsr64(acc_s(jl), r));
+            eS = eref + r;
+        } else {
+#pragma unroll
+            for (int jl = 0; jl < kHC; ++jl) sq[jl] = 0;
+        }
+        // Sq bytes to the private rows (the rows above are needed for T0q Sq)
+        {
+            uint4 v0, v1;
+            v0.x = pack4(sq[0], sq[1], sq[2], sq[3]);     v0.y = pack4(sq[4], sq[5], sq[6], sq[7]);
+            v0.z = pack4(sq[8], sq[9], sq[10], sq[11]);   v0.w = pack4(sq[12], sq[13], sq[14], sq[15]);
+            v1.x = pack4(sq[16], sq[17], sq[18], sq[19]); v1.y = pack4(sq[20], sq[21], sq[22], sq[23]);
+            v1.z = pack4(sq[24], sq[25], sq[26], sq[27]); v1.w = pack4(sq[28], sq[29], sq[30], sq[31]);
+            *reinterpret_cast<uint4*>(rowa + col0) = v0;
+            *reinterpret_cast<uint4*>(rowa + col0 + 16) = v1;
+        }
+        cta_barrier();
+
+        // ---- I8: Toffq = Q8(align(T0q, Sq, T0q Sq)) on i > j
+        int toff[kHC];
+        int eT;
+        {
+            int prod[kHC];
+#pragma unroll
+            for (int jl = 0; jl < kHC; ++jl) prod[jl] = 0;
+#pragma unroll
+            for (int e = 1; e <= 3; ++e) {
+                const int r = (t - e) > 0 ? (t - e) : 0;
+                const int cf = (il - e >= 0) ? t0q[e] : 0;
+                const uint4 a0 = *reinterpret_cast<const uint4*>(sRowA + r * 64 + col0);
+                const uint4 a1 = *reinterpret_cast<const uint4*>(sRowA + r * 64 + col0 + 16);
+                const uint32_t w[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+#pragma unroll
+                for (int jl = 0; jl < kHC; ++jl) prod[jl] += cf * byte_at(w[jl >> 2], jl & 3);
+            }
+            const int e0 = eT0, e1 = eS, e2 = eT0 + eS;
+            const int emin = min(e0, min(e1, e2)), emax = max(e0, max(e1, e2));
+            const int eref = max(emin, emax - 24);
+            auto acc_t = [&](int jl) -> long long {
+                const int d = il - (col0 + jl);
+                if (d <= 0) return 0;
+                int band = 0;
+#pragma unroll
+                for (int e = 1; e <= 3; ++e)
+                    if (d == e) band = t0q[e];
+                return shift64(band, e0 - eref) + shift64(sq[jl], e1 - eref) + shift64(prod[jl], e2 - eref);
+            };
+            unsigned long long m = 0;
+#pragma unroll
+            for (int jl = 0; jl < kHC; ++jl) m |= absll(acc_t(jl));
+            const int r = q8_shift(chunk_bitlen(m, slot++));
+#pragma unroll
+            for (int jl = 0; jl < kHC; ++jl) toff[jl] = clamp127(rsr64(acc_t(jl), r));
+            eT = eref + r;
+        }
+
+        // ---- I9: Tbq = Q8(Toffq_ij beta_q_j); A operand of W/U (block diagonal, int8 in TMEM)
+        int eTb;
+        {
+            int acc[kHC];
+            unsigned long long m = 0;
+#pragma unroll
+            for (int jl = 0; jl < kHC; ++jl) {
+                acc[jl] = toff[jl] * sbeta[cb + col0 + jl];
+                m |= absll(acc[jl]);
+            }
+            const int r = q8_shift(chunk_bitlen(m, slot++));
+            uint32_t r8[8];
+#pragma unroll
+            for (int w = 0; w < 8; ++w)
+                r8[w] = pack4(clamp127(rsr64(acc[4 * w], r)), clamp127(rsr64(acc[4 * w + 1], r)), clamp127(rsr64(acc[4 * w + 2], r)),
+                              clamp127(rsr64(acc[4 * w + 3], r)));
+            eTb = eT - 15 + r;
+            // row t's block occupies packed columns [cb/4, cb/4 + 16) of a 32-column operand; the other 16 are zero
+            tmem_st8(lane_base + kAS + cb / 4 + h * 8, r8);
+#pragma unroll
+            for (int w = 0; w < 8; ++w) r8[w] = 0u;
+            tmem_st8(lane_base + kAS + (16 - cb / 4) + h * 8, r8);
+            tmem_wait_st();
+        }
+        // Toffq row -> staging (64-byte lines, 64-byte TMA swizzle) -> bulk tensor store of 32 rows per warp (h = 0 issues)
+        uint8_t* stage = smem + kOffStage;
+        if (p.Toff != nullptr) {
+            uint8_t* line = stage + t * 64;
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                const int cc = (col0 >> 4) + c;
+                const uint4 v = make_uint4(pack4(toff[16 * c + 0], toff[16 * c + 1], toff[16 * c + 2], toff[16 * c + 3]),
+                                           pack4(toff[16 * c + 4], toff[16 * c + 5], toff[16 * c + 6], toff[16 * c + 7]),
+                                           pack4(toff[16 * c + 8], toff[16 * c + 9], toff[16 * c + 10], toff[16 * c + 11]),
+                                           pack4(toff[16 * c + 12], toff[16 * c + 13], toff[16 * c + 14], toff[16 * c + 15]));
+                *reinterpret_cast<uint4*>(line + ((cc ^ ((t >> 1) & 3)) << 4)) = v;
+            }
+        }
+        if (row_valid && il == 0 && h == 0) p.t_exp[(long long)tc.bhv * n_c + chunk_in_head] = eT;
+        fence_proxy_async_smem();
+        tc_fence_before_sync();
+        cta_barrier();
+        if (p.Toff != nullptr && h == 0 && lane == 0) {
+            tma_store_3d(&tmT, stage + wrow0 * 64, 0, tc.t0 + wrow0, tc.bhv);
+            tma_store_commit();
+        }
+        if (tid == 0) {
+            // W accumulator = blockdiag(Tbq) Kq: M = 128, N = 128, K = 128 (4 steps of 32)
+            tc_fence_after_sync();
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+                const uint64_t bd = smem_desc(sK_a + ks * 4096, 16384, 1024, SWZ_128B);
+                mma_i8_ts(tmem + kR0, tmem + kAS + ks * 8, bd, idesc_m, ks > 0);
+            }
+            mma_commit(&bar_mma);
+        }
+
+        // ---- I10: W, then U
+#pragma unroll 1
+        for (int half = 0; half < 2; ++half) {
+            const int xexp = (half == 0) ? kexp : vexp;
+            const uint8_t* xtile = (half == 0) ? sK : sV;
+            // own row of the int8 tile (64 columns of this thread): diagonal term beta_q_i * Xq_i
+            uint32_t xr[16];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const uint4 v = *reinterpret_cast<const uint4*>(xtile + t * 128 + (((h * 4 + c) ^ (t & 7)) << 4));
+                xr[4 * c + 0] = v.x; xr[4 * c + 1] = v.y; xr[4 * c + 2] = v.z; xr[4 * c + 3] = v.w;
+            }
+            if (!wait_bar(&bar_mma, par_mma)) { ok = false; break; }
+            par_mma ^= 1;
+            tc_fence_after_sync();
+            const int ep = eTb + xexp, ed = xexp - 15;
+            const int eref = align_ref2(ep, ed);
+            auto acc_w = [&](uint32_t raw, int col) -> long long {
+                return shift64(static_cast<int>(raw), ep - eref) +
+                       shift64(static_cast<long long>(bq) * byte_at(xr[col >> 2], col & 3), ed - eref);
+            };
+            // pass 1: the scale (bit length of the largest magnitude over the chunk's C x d block)
+            unsigned long long m = 0;
+#pragma unroll
+            for (int c0 = 0; c0 < 64; c0 += 32) {
+                uint32_t r[32];
+                tmem_ld32(lane_base + kR0 + h * 64 + c0, r);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) m |= absll(acc_w(r[i], c0 + i));
+            }
+            const int rr = q8_shift(chunk_bitlen(m, slot++));
+            // after that barrier every thread holds its own row of the K (V) tile in registers, and the products that
+            // read the tile are complete: the next tile's K (V) may land
+            if (tid == 0 && has_next) {
+                const TileCoord nc = decode_tile(next, p);
+                if (half == 0) {
+                    mbar_arrive_expect_tx(&bar_k, 16384);
+                    tma_load_3d(sK, &tmK, &bar_k, 0, nc.t0, nc.bhk);
+                } else {
+                    mbar_arrive_expect_tx(&bar_v, 16384);
+                    tma_load_3d(sV, &tmV, &bar_v, 0, nc.t0, nc.bhv);
+                }
+            }
+            if (row_valid && il == 0 && h == 0)
+                ((half == 0) ? p.w_exp : p.u_exp)[(long long)tc.bhv * n_c + chunk_in_head] = eref + rr;
+            // pass 2: mantissas -> 32 rows x 64 int8 columns of this warp in the 64-byte TMA swizzle:
+            // 2 KB at stage + 8 KB + (wq * 2 + h) * 2 KB
+            uint8_t* sub = stage + 8192 + (wq * 2 + h) * 2048;
+            if (lane == 0) tma_store_wait_read<0>();
+            __syncwarp();
+#pragma unroll
+            for (int c0 = 0; c0 < 64; c0 += 32) {
+                uint32_t r[32];
+                tmem_ld32(lane_base + kR0 + h * 64 + c0, r);
+                tmem_wait_ld();
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t w4[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int i = c * 16 + q * 4;
+                        w4[q] = pack4(clamp127(rsr64(acc_w(r[i], c0 + i), rr)), clamp127(rsr64(acc_w(r[i + 1], c0 + i + 1), rr)),
+                                      clamp127(rsr64(acc_w(r[i + 2], c0 + i + 2), rr)), clamp127(rsr64(acc_w(r[i + 3], c0 + i + 3), rr)));
+                    }
+                    const int cc = c0 / 16 + c;
+                    *reinterpret_cast<uint4*>(sub + lane * 64 + ((cc ^ ((lane >> 1) & 3)) << 4)) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+                }
+            }
+            if (half == 0) {
+                tc_fence_before_sync();
+                cta_barrier();  // every row of the W accumulator has been read twice
+                if (tid == 0) {
+                    if (!wait_bar(&bar_v, par_kv)) ok = false;
+                    if (ok) {
+                        tc_fence_after_sync();
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks) {
+                            const uint64_t bd = smem_desc(sV_a + ks * 4096, 16384, 1024, SWZ_128B);
+                            mma_i8_ts(tmem + kR0, tmem + kAS + ks * 8, bd, idesc_m, ks > 0);
+                        }
+                        mma_commit(&bar_mma);
+                    }
+                }
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                tma_store_3d((half == 0) ? &tmW : &tmU, sub, h * 64, tc.t0 + wrow0, tc.bhv);
+                tma_store_commit();
+            }
+        }
+        par_kv ^= 1;
+    }
+    if (lane == 0) tma_store_wait_all<0>();
+    if (!ok) atomicExch(p.status, GDN_ERR_TIMEOUT);
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem, kTmemCols);
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (fn == nullptr) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess)
+            return nullptr;
+        fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+// [heads][T][cols] int8 tensor
+bool make_map(CUtensorMap* tm, const void* base, long long heads, int T, int cols, int box_cols, int box_rows,
+              CUtensorMapSwizzle swizzle) {
+    EncodeTiledFn enc = get_encode_fn();
+    if (enc == nullptr) return false;
+    cuuint64_t dims[3] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(T), static_cast<cuuint64_t>(heads)};
+    cuuint64_t strides[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(T) * cols};
+    cuuint32_t box[3] = {static_cast<cuuint32_t>(box_cols), static_cast<cuuint32_t>(box_rows), 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+void int8_decay_lut(uint16_t* out) {
+    for (int f = 0; f < 256; ++f) out[f] = static_cast<uint16_t>(floor(32768.0 * exp2(-static_cast<double>(f) / 256.0) + 0.5));
+}
+
+int launch_tc_int8(const ProblemI8& q, cudaStream_t stream) {
+    if (q.d_k != kD || q.d_v != kD) return GDN_ERR_UNSUPPORTED;
+    if (q.C != kC) return GDN_ERR_UNSUPPORTED;
+    if (q.order < 1 || q.order > 3) return GDN_ERR_UNSUPPORTED;  // the paper limits the low-bit order to N <= 3
+    if (q.steps > kSMax) return GDN_ERR_UNSUPPORTED;
+    if ((long long)q.B * q.H_v * q.T == 0) return GDN_OK;
+    int* status = device_status_word();
+    if (status == nullptr) return GDN_ERR_LAUNCH;
+    const long long hk = (long long)q.B * q.H_k, hv = (long long)q.B * q.H_v;
+    CUtensorMap mK, mV, mW, mU, mT;
+    if (!make_map(&mK, q.Kq, hk, q.T, kD, 128, 128, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
+    if (!make_map(&mV, q.Vq, hv, q.T, kD, 128, 128, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
+    if (!make_map(&mW, q.Wq, hv, q.T, kD, 64, 32, CU_TENSOR_MAP_SWIZZLE_64B)) return GDN_ERR_LAUNCH;
+    if (!make_map(&mU, q.Uq, hv, q.T, kD, 64, 32, CU_TENSOR_MAP_SWIZZLE_64B)) return GDN_ERR_LAUNCH;
+    if (!make_map(&mT, q.Toff != nullptr ? q.Toff : q.Wq, hv, q.T, q.Toff != nullptr ? kC : kD, 64, 32, CU_TENSOR_MAP_SWIZZLE_64B))
+        return GDN_ERR_LAUNCH;
+    ParamsI8 prm;
+    prm.beta_q = q.beta_q;
+    prm.decay_q = q.decay_q;
+    prm.k_exp = q.k_exp;
+    prm.v_exp = q.v_exp;
+    prm.w_exp = q.w_exp;
+    prm.u_exp = q.u_exp;
+    prm.t_exp = q.t_exp;
+    prm.Toff = q.Toff;
+    prm.status = status;
+    prm.H_k = q.H_k;
+    prm.H_v = q.H_v;
+    prm.T = q.T;
+    prm.group = q.H_v / q.H_k;
+    prm.n_tt = (q.T + kTile - 1) / kTile;
+    prm.N = q.order;
+    prm.S = q.steps;
+    prm.n_tiles = hv * prm.n_tt;
+    if (prm.n_tiles >= (1LL << 31) - 4096) return GDN_ERR_UNSUPPORTED;
+    int8_decay_lut(prm.lut);
+    const int smem = kSmemTotal + 1024;
+    if (cudaFuncSetAttribute(chunk_tc_int8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+        return GDN_ERR_LAUNCH;
+    const long long grid = prm.n_tiles < 2 * 148 ? prm.n_tiles : 2 * 148;
+    chunk_tc_int8_kernel<<<static_cast<int>(grid), kThreads, smem, stream>>>(mK, mV, mW, mU, mT, prm);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? GDN_OK : GDN_ERR_LAUNCH;
+}
+
+}  // namespace gdn

@@ -23,6 +23,24 @@ struct Problem {
     int dtype;   // GDN_DTYPE_*
 };
 
+// INT8 entry point's problem description
+struct ProblemI8 {
+    const int8_t* Kq;
+    const int8_t* Vq;
+    const int32_t* k_exp;
+    const int32_t* v_exp;
+    const int16_t* beta_q;
+    const int32_t* decay_q;
+    int8_t* Wq;
+    int8_t* Uq;
+    int32_t* w_exp;
+    int32_t* u_exp;
+    int8_t* Toff;  // may be null
+    int32_t* t_exp;
+    int B, H_k, H_v, T, C, d_k, d_v;
+    int order, steps;
+};
+
 enum InverseMode { INV_NEUMANN = 0, INV_FWDSUBST_ROWS = 1, INV_FWDSUBST_BLOCKED = 2 };
 
 // Status word written by kernels (one per device, static device memory).
@@ -32,5 +50,7 @@ void count_launch();
 // Kernel launchers. Each returns a gdn_status and launches on `stream`.
 int launch_simt(const Problem& p, InverseMode mode, cudaStream_t stream);
 int launch_tc_bf16(const Problem& p, InverseMode mode, cudaStream_t stream);
+int launch_tc_int8(const ProblemI8& p, cudaStream_t stream);
+void int8_decay_lut(uint16_t* out256);  // table of round(2^15 * 2^(-f/256))
 
 }  // namespace gdn

@@ -114,6 +114,35 @@ int gdn_chunk_prepare_fwdsubst(const void* K, const void* V, const float* beta, 
     return run(p, variant == GDN_FWDSUBST_ROWS ? INV_FWDSUBST_ROWS : INV_FWDSUBST_BLOCKED, static_cast<cudaStream_t>(stream));
 }
 
+int gdn_chunk_prepare_int8(const int8_t* Kq, const int8_t* Vq, const int32_t* k_exp, const int32_t* v_exp, const uint16_t* beta_q,
+                           const int32_t* decay_q, int B, int H_k, int H_v, int T, int C, int d_k, int d_v, int order,
+                           int residual_steps, int8_t* Wq_out, int8_t* Uq_out, int32_t* w_exp_out, int32_t* u_exp_out,
+                           int8_t* Toff_q_out, int32_t* t_exp_out, gdn_stream_t stream) {
+    if (order == -1) order = gdn_default_order(C);
+    if (residual_steps == -1) residual_steps = gdn_default_residual_steps(C);
+    if (Kq == nullptr || Vq == nullptr || k_exp == nullptr || v_exp == nullptr || beta_q == nullptr || decay_q == nullptr ||
+        Wq_out == nullptr || Uq_out == nullptr || w_exp_out == nullptr || u_exp_out == nullptr || t_exp_out == nullptr)
+        return GDN_ERR_NULL;
+    if (B < 0 || H_k <= 0 || H_v <= 0 || T < 0 || C < 2 || d_k <= 0 || d_v <= 0) return GDN_ERR_INVALID_ARG;
+    if (H_v % H_k != 0 || T % C != 0) return GDN_ERR_INVALID_ARG;
+    if (order < 1 || order >= C || residual_steps < 0) return GDN_ERR_INVALID_ARG;
+    if (!aligned16(Kq) || !aligned16(Vq) || !aligned16(Wq_out) || !aligned16(Uq_out) || !aligned16(Toff_q_out))
+        return GDN_ERR_ALIGN;
+    const int rc = check_arch();
+    if (rc != GDN_OK) return rc;
+    ProblemI8 q{Kq, Vq, k_exp, v_exp, reinterpret_cast<const int16_t*>(beta_q), decay_q, Wq_out, Uq_out, w_exp_out, u_exp_out,
+                Toff_q_out, t_exp_out, B, H_k, H_v, T, C, d_k, d_v, order, residual_steps};
+    return launch_tc_int8(q, static_cast<cudaStream_t>(stream));
+}
+
+unsigned int gdn_int8_lut_checksum(void) {
+    uint16_t lut[256];
+    int8_decay_lut(lut);
+    unsigned long long s = 0;
+    for (int f = 0; f < 256; ++f) s = (s * 31 + lut[f] + f) % 1000000007ull;
+    return static_cast<unsigned int>(s);
+}
+
 int gdn_device_status(gdn_stream_t stream) {
     if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) {
         cudaGetLastError();

@@ -37,6 +37,11 @@ def test_defaults_follow_the_paper(lib):
     assert [lib.gdn_default_residual_steps(c) for c in (16, 32, 64, 128)] == [3, 4, 8, 8]
 
 
+def test_int8_decay_table_matches_the_oracle(lib):
+    from oracle import gdn_oracle_int8 as orq
+    assert lib.gdn_int8_lut_checksum() == orq.lut_checksum()
+
+
 def test_status_strings(lib):
     for code in range(0, -8, -1):
         assert lib.gdn_status_string(code)
