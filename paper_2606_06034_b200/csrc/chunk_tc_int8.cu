@@ -9,7 +9,7 @@
 //
 //   rsr(x, r)  = sign(x) ((|x| + 2^(r-1)) >> r)
 //   Q8(acc, e) : r = max(0, bitlen(max |acc| on the support) - 7); q = clamp(rsr(acc, r), +-127); exponent e + r
-//   align(..)  : e_ref = max(min e, max e - 24); terms shifted to e_ref (left shift, or rsr) and summed in int64
+//   align(..)  : e_ref = max(min e, max e - 8); terms shifted to e_ref (left shift, or rsr) and summed (fits int32)
 //
 //   G = Kq Kq^T                                   MMA (K tile by TMA, 128-byte swizzle)
 //   Aq   = Q8(-(G o c), 2 k_exp - 15),  c = (beta_q_i Gam_ij + 2^14) >> 15, Gam from a 256-entry table of 2^(-f/256)
@@ -37,7 +37,15 @@ constexpr int kD = 128;
 constexpr int kC = 64;     // chunk size handled by this kernel
 constexpr int kHC = 32;    // chunk columns per thread
 constexpr int kSMax = 8;   // largest number of residual terms held in registers
+constexpr int kAlignWindow = 8;  // bits kept below the largest term of an aligned sum: every such sum fits 32 bits
 constexpr uint32_t kR0 = 0, kAS = 128, kTmemCols = 256;
+
+#ifdef GDN_TRACE
+__device__ long long g_trace8[4096];
+#define STAMP8(slot_) do { if (blockIdx.x == 0 && tid == 32 && trace_n < 200) { g_trace8[trace_n * 2] = (slot_); g_trace8[trace_n * 2 + 1] = clock64(); ++trace_n; } } while (0)
+#else
+#define STAMP8(slot_) do { } while (0)
+#endif
 
 struct ParamsI8 {
     const int16_t* beta_q;
@@ -89,11 +97,33 @@ __device__ __forceinline__ long long rsr64(long long x, int r) {
 }
 // x * 2^s for s >= 0, rounded right shift otherwise
 __device__ __forceinline__ long long shift64(long long x, int s) { return s >= 0 ? (x << s) : rsr64(x, -s); }
+// type-generic forms (T = int when every term provably fits 32 bits, long long otherwise)
+template <typename T>
+__device__ __forceinline__ T rsr_t(T x, int r) {  // r >= 0; (1 << r) >> 1 is the rounding half, 0 for r = 0
+    const T a = x < 0 ? -x : x;
+    const T q = (a + ((static_cast<T>(1) << r) >> 1)) >> r;
+    return x < 0 ? -q : q;
+}
+template <typename T>
+__device__ __forceinline__ T shift_t(T x, int s) { return s >= 0 ? (x << s) : rsr_t<T>(x, -s); }
+// One term of an aligned sum: x 2^s for s >= 0, rounded right shift otherwise. x fits 23 bits, so the right
+// shift is done in 32 bits (a shift of 31 or more gives 0, as the rounding rule demands for |x| < 2^30).
+template <typename T>
+__device__ __forceinline__ T term_t(int x, int s) {
+    if (s >= 0) return static_cast<T>(x) << s;
+    return static_cast<T>(rsr_t<int>(x, (-s) < 31 ? (-s) : 31));
+}
+__device__ __forceinline__ int term32(int x, int s) { return term_t<int>(x, s); }
+template <typename T>
+__device__ __forceinline__ unsigned long long abs_bits(T x) { return static_cast<unsigned long long>(x < 0 ? -x : x); }
+template <typename T>
+__device__ __forceinline__ int clamp127_t(T q) { return q > 127 ? 127 : (q < -127 ? -127 : static_cast<int>(q)); }
+
 __device__ __forceinline__ int clamp127(long long q) { return q > 127 ? 127 : (q < -127 ? -127 : static_cast<int>(q)); }
 __device__ __forceinline__ int q8_shift(int bitlen) { return bitlen > 7 ? bitlen - 7 : 0; }
 __device__ __forceinline__ int align_ref2(int e0, int e1) {
     const int lo = e0 < e1 ? e0 : e1, hi = e0 < e1 ? e1 : e0;
-    return lo > hi - 24 ? lo : hi - 24;
+    return lo > hi - kAlignWindow ? lo : hi - kAlignWindow;
 }
 __device__ __forceinline__ uint32_t pack4(int a, int b, int c, int d) {
     return (static_cast<uint32_t>(a) & 0xFFu) | ((static_cast<uint32_t>(b) & 0xFFu) << 8) | ((static_cast<uint32_t>(c) & 0xFFu) << 16) |
@@ -141,6 +171,9 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
     const int lane = tid & 31;
+#ifdef GDN_TRACE
+    int trace_n = 0;
+#endif
 
     if (tid == 0) {
         mbar_init(&bar_k, 1);
@@ -214,6 +247,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
         const int chunk_in_head = (tc.t0 + cb) / kC;
         const bool chunk_valid = (tc.t0 + cb) < p.T;
 
+        STAMP8(1);
         int bq = 0, dq = 0, kexp = 0, vexp = 0;
         if (row_valid) {
             bq = static_cast<int>(static_cast<uint16_t>(p.beta_q[grow]));
@@ -252,6 +286,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
         cta_barrier();
         int slot = 0;
 
+        STAMP8(2);
         // ---- I1-I3: Aq = Q8(-(G o c))
         if (!wait_bar(&bar_mma, par_mma)) { ok = false; break; }
         par_mma ^= 1;
@@ -262,24 +297,25 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             uint32_t g[kHC];
             tmem_ld32(lane_base + kR0 + cb + col0, g);
             tmem_wait_ld();
-            // the products are formed twice (once for the scale, once for the mantissas) instead of kept in registers
-            auto acc_a = [&](int jl) -> long long {
-                const int j = col0 + jl;
-                if (j >= il) return 0;
-                const int dlt = dq - sdecay[cb + j];
-                const int sh = dlt >> 8;
-                const int gam = (sh < 16) ? (static_cast<int>(slut[dlt & 255]) >> sh) : 0;
-                const int c = (bq * gam + (1 << 14)) >> 15;
-                return -static_cast<long long>(static_cast<int>(g[jl])) * c;
-            };
+            int cq[kHC];  // c_ij = (beta_q_i Gam_ij + 2^14) >> 15, 0 on and above the diagonal
             unsigned long long m = 0;
 #pragma unroll
-            for (int jl = 0; jl < kHC; ++jl) m |= absll(acc_a(jl));
+            for (int jl = 0; jl < kHC; ++jl) {
+                const int j = col0 + jl;
+                const int dlt = dq - sdecay[cb + j];
+                const int sh = dlt >> 8;
+                const int gam = (sh >= 0 && sh < 16) ? (static_cast<int>(slut[dlt & 255]) >> sh) : 0;
+                const int c = (j < il) ? ((bq * gam + (1 << 14)) >> 15) : 0;
+                cq[jl] = c;
+                m |= abs_bits<long long>(static_cast<long long>(static_cast<int>(g[jl])) * c);
+            }
             const int r = q8_shift(chunk_bitlen(m, slot++));
 #pragma unroll
-            for (int jl = 0; jl < kHC; ++jl) aq[jl] = clamp127(rsr64(acc_a(jl), r));
+            for (int jl = 0; jl < kHC; ++jl)
+                aq[jl] = clamp127_t<long long>(rsr_t<long long>(-static_cast<long long>(static_cast<int>(g[jl])) * cq[jl], r));
             eA = 2 * kexp - 15 + r;
         }
+        STAMP8(3);
         // Aq bytes to the private row; entries next to the diagonal and right of this half come back from there
         uint8_t* rowa = sRowA + t * 64;
         {
@@ -292,106 +328,111 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             *reinterpret_cast<uint4*>(rowa + col0 + 16) = v1;
         }
         cta_barrier();
-        int ab[4], anext[4];
-        ab[0] = 0;
-#pragma unroll
-        for (int e = 1; e <= 3; ++e) ab[e] = (il - e >= 0) ? static_cast<int>(static_cast<int8_t>(rowa[il - e])) : 0;
-#pragma unroll
-        for (int e = 0; e < 3; ++e) anext[e] = (h == 0) ? static_cast<int>(static_cast<int8_t>(rowa[kHC + e])) : 0;
-        anext[3] = 0;
-        // P_1 = band of Aq: zero beyond distance N
-        int p1[4];
-#pragma unroll
-        for (int e = 0; e <= 3; ++e) p1[e] = (e >= 1 && e <= N) ? ab[e] : 0;
+        int ab1 = 0, ab2 = 0, ab3 = 0;  // Aq[i][i-1..i-3]
+        if (il >= 1) ab1 = static_cast<int>(static_cast<int8_t>(rowa[il - 1]));
+        if (il >= 2) ab2 = static_cast<int>(static_cast<int8_t>(rowa[il - 2]));
+        if (il >= 3) ab3 = static_cast<int>(static_cast<int8_t>(rowa[il - 3]));
+        int an0 = 0, an1 = 0, an2 = 0;  // Aq[i][32..34] for the left half: the entries right of its columns
         if (h == 0) {
-            sAB[t * 8 + 1] = p1[1];
-            sAB[t * 8 + 2] = p1[2];
-            sAB[t * 8 + 3] = p1[3];
+            an0 = static_cast<int>(static_cast<int8_t>(rowa[kHC + 0]));
+            an1 = static_cast<int>(static_cast<int8_t>(rowa[kHC + 1]));
+            an2 = static_cast<int>(static_cast<int8_t>(rowa[kHC + 2]));
+        }
+        // P_1 = band of Aq: zero beyond distance N
+        const int p11 = ab1, p12 = (N >= 2) ? ab2 : 0, p13 = (N >= 3) ? ab3 : 0;
+        if (h == 0) {
+            sAB[t * 8 + 1] = p11;
+            sAB[t * 8 + 2] = p12;
+            sAB[t * 8 + 3] = p13;
         }
         cta_barrier();
 
+        STAMP8(4);
         // ---- I4: P_2, P_3 (band only), I5: T0q
-        int t0q[4] = {0, 0, 0, 0};
+        int t0q1 = 0, t0q2 = 0, t0q3 = 0;  // T0q[i][i-1..i-3]
         int eT0;
         {
             const int r1 = (t - 1) > 0 ? (t - 1) : 0, r2 = (t - 2) > 0 ? (t - 2) : 0;
-            // P_2 on distances 2..N
-            int acc2[4] = {0, 0, 0, 0};
-            acc2[2] = p1[1] * sAB[r1 * 8 + 1];
-            acc2[3] = p1[1] * sAB[r1 * 8 + 2] + p1[2] * sAB[r2 * 8 + 1];
-            if (N < 2) acc2[2] = 0;
-            if (N < 3) acc2[3] = 0;
-            int p2[4] = {0, 0, 0, 0}, p3 = 0;
+            // P_2 on distances 2..N: sum over the intermediate row
+            int acc22 = (N >= 2) ? p11 * sAB[r1 * 8 + 1] : 0;
+            int acc23 = (N >= 3) ? p11 * sAB[r1 * 8 + 2] + p12 * sAB[r2 * 8 + 1] : 0;
+            int p22 = 0, p23 = 0, p33 = 0;
             int e2 = 0, e3 = 0;
             if (N >= 2) {
-                unsigned long long m = (h == 0) ? (absll(acc2[2]) | absll(acc2[3])) : 0ull;
+                const unsigned long long m = (h == 0) ? (abs_bits<int>(acc22) | abs_bits<int>(acc23)) : 0ull;
                 const int r = q8_shift(chunk_bitlen(m, slot++));
-                p2[2] = clamp127(rsr64(acc2[2], r));
-                p2[3] = clamp127(rsr64(acc2[3], r));
+                p22 = clamp127_t<int>(rsr_t<int>(acc22, r));
+                p23 = clamp127_t<int>(rsr_t<int>(acc23, r));
                 e2 = eA + eA + r;
             }
             if (N >= 3) {
                 // P_3 at distance 3: P_2[i][i-2] * Aq[i-2][i-3]
-                const int acc3 = p2[2] * sAB[r2 * 8 + 1];
-                const int r = q8_shift(chunk_bitlen((h == 0) ? absll(acc3) : 0ull, slot++));
-                p3 = clamp127(rsr64(acc3, r));
+                const int acc3 = p22 * sAB[r2 * 8 + 1];
+                const int r = q8_shift(chunk_bitlen((h == 0) ? abs_bits<int>(acc3) : 0ull, slot++));
+                p33 = clamp127_t<int>(rsr_t<int>(acc3, r));
                 e3 = e2 + eA + r;
             }
-            // align(P_1..P_N)
+            // align(P_1..P_N): at most three small terms per band entry
             int emin = eA, emax = eA;
             if (N >= 2) { emin = min(emin, e2); emax = max(emax, e2); }
             if (N >= 3) { emin = min(emin, e3); emax = max(emax, e3); }
-            const int eref = max(emin, emax - 24);
-            long long accT[4] = {0, 0, 0, 0};
-#pragma unroll
-            for (int d = 1; d <= 3; ++d) {
-                long long s = shift64(p1[d], eA - eref);
-                if (N >= 2 && d >= 2) s += shift64(p2[d], e2 - eref);
-                if (N >= 3 && d >= 3) s += shift64(p3, e3 - eref);
-                accT[d] = (d <= N && il - d >= 0) ? s : 0;
-            }
-            unsigned long long m = (h == 0) ? (absll(accT[1]) | absll(accT[2]) | absll(accT[3])) : 0ull;
+            const int eref = max(emin, emax - kAlignWindow);
+            const int s1 = eA - eref, s2 = e2 - eref, s3 = e3 - eref;
+            int a1 = term32(p11, s1);
+            int a2 = term32(p12, s1) + ((N >= 2) ? term32(p22, s2) : 0);
+            int a3 = term32(p13, s1) + ((N >= 2) ? term32(p23, s2) : 0) + ((N >= 3) ? term32(p33, s3) : 0);
+            if (!(N >= 1 && il >= 1)) a1 = 0;
+            if (!(N >= 2 && il >= 2)) a2 = 0;
+            if (!(N >= 3 && il >= 3)) a3 = 0;
+            const unsigned long long m = (h == 0) ? (abs_bits<int>(a1) | abs_bits<int>(a2) | abs_bits<int>(a3)) : 0ull;
             const int r = q8_shift(chunk_bitlen(m, slot++));
-#pragma unroll
-            for (int d = 1; d <= 3; ++d) t0q[d] = clamp127(rsr64(accT[d], r));
+            t0q1 = clamp127_t<int>(rsr_t<int>(a1, r));
+            t0q2 = clamp127_t<int>(rsr_t<int>(a2, r));
+            t0q3 = clamp127_t<int>(rsr_t<int>(a3, r));
             eT0 = eref + r;
             if (h == 0) {
-#pragma unroll
-                for (int e = 1; e <= 3; ++e)
-                    if (il - e >= 0) sSH[(t - e) * 4 + (e - 1)] = t0q[e];
+                if (il >= 1) sSH[(t - 1) * 4 + 0] = t0q1;
+                if (il >= 2) sSH[(t - 2) * 4 + 1] = t0q2;
+                if (il >= 3) sSH[(t - 3) * 4 + 2] = t0q3;
             }
             cta_barrier();
         }
 
+        STAMP8(5);
         // ---- I6: Eq = Q8(align(Aq, Aq T0q)) on i-j > N
         int eq[kHC];
         int eE;
         {
             const int eref = align_ref2(eA, eA + eT0);
-            auto acc_e = [&](int jl) -> long long {
-                if (il - (col0 + jl) <= N) return 0;
-                const int4 c4 = *reinterpret_cast<const int4*>(sSH + (cb + col0 + jl) * 4);
-                const int cc[3] = {c4.x, c4.y, c4.z};
-                int prod = 0;
-#pragma unroll
-                for (int e = 1; e <= 3; ++e) {
-                    const int k = jl + e;
-                    const int ak = (k < kHC) ? aq[(k < kHC) ? k : 0] : anext[(k >= kHC) ? k - kHC : 0];
-                    prod += ak * cc[e - 1];
-                }
-                return shift64(aq[jl], eA - eref) + shift64(prod, eA + eT0 - eref);
-            };
+            const int sa = eA - eref, sp = eA + eT0 - eref;
+            int acc[kHC];  // |Aq| < 2^7 and |Aq T0q| <= 3 * 127^2 < 2^16, shifted left by at most 8
             unsigned long long m = 0;
 #pragma unroll
-            for (int jl = 0; jl < kHC; ++jl) m |= absll(acc_e(jl));
+            for (int jl = 0; jl < kHC; ++jl) {
+                const int4 c4 = *reinterpret_cast<const int4*>(sSH + (cb + col0 + jl) * 4);
+                const int a1 = (jl + 1 < kHC) ? aq[(jl + 1 < kHC) ? jl + 1 : 0] : ((jl + 1 == kHC) ? an0 : (jl + 1 == kHC + 1 ? an1 : an2));
+                const int a2 = (jl + 2 < kHC) ? aq[(jl + 2 < kHC) ? jl + 2 : 0] : ((jl + 2 == kHC) ? an0 : (jl + 2 == kHC + 1 ? an1 : an2));
+                const int a3 = (jl + 3 < kHC) ? aq[(jl + 3 < kHC) ? jl + 3 : 0] : ((jl + 3 == kHC) ? an0 : (jl + 3 == kHC + 1 ? an1 : an2));
+                const bool on = (il - (col0 + jl)) > N;
+                const int v = on ? (term32(aq[jl], sa) + term32(a1 * c4.x + a2 * c4.y + a3 * c4.z, sp)) : 0;
+                acc[jl] = v;
+                m |= abs_bits<int>(v);
+            }
             const int r = q8_shift(chunk_bitlen(m, slot++));
 #pragma unroll
-            for (int jl = 0; jl < kHC; ++jl) eq[jl] = clamp127(rsr64(acc_e(jl), r));
+            for (int jl = 0; jl < kHC; ++jl) eq[jl] = clamp127_t<int>(rsr_t<int>(acc[jl], r));
             eE = eref + r;
         }
+        STAMP8(6);
         // packed rows of the powers R_s (R_1 = Eq) and their exponents
         uint32_t rpk[kSMax][kHC / 4];
         int er[kSMax];
+#pragma unroll
+        for (int s = 0; s < kSMax; ++s) {
+            er[s] = 0;
+#pragma unroll
+            for (int w = 0; w < kHC / 4; ++w) rpk[s][w] = 0u;
+        }
         int n_terms = 0;
         if (S >= 1) {
 #pragma unroll
@@ -435,24 +476,28 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             tmem_ld32(lane_base + kR0 + cb + col0, dres);
             tmem_wait_ld();
             unsigned long long m = 0;
+            const int dmin = s * (N + 1);
 #pragma unroll
             for (int jl = 0; jl < kHC; ++jl) {
-                int v = static_cast<int>(dres[jl]);
-                if (il - (col0 + jl) < s * (N + 1)) v = 0;
+                const int v = (il - (col0 + jl) >= dmin) ? static_cast<int>(dres[jl]) : 0;
                 dres[jl] = static_cast<uint32_t>(v);
-                m |= absll(v);
+                m |= abs_bits<int>(v);
             }
             const int r = q8_shift(chunk_bitlen(m, slot++));
 #pragma unroll
             for (int w = 0; w < kHC / 4; ++w)
-                rpk[s - 1][w] = pack4(clamp127(rsr64(static_cast<int>(dres[4 * w]), r)), clamp127(rsr64(static_cast<int>(dres[4 * w + 1]), r)),
-                                      clamp127(rsr64(static_cast<int>(dres[4 * w + 2]), r)), clamp127(rsr64(static_cast<int>(dres[4 * w + 3]), r)));
+                rpk[s - 1][w] = pack4(clamp127_t<int>(rsr_t<int>(static_cast<int>(dres[4 * w]), r)),
+                                      clamp127_t<int>(rsr_t<int>(static_cast<int>(dres[4 * w + 1]), r)),
+                                      clamp127_t<int>(rsr_t<int>(static_cast<int>(dres[4 * w + 2]), r)),
+                                      clamp127_t<int>(rsr_t<int>(static_cast<int>(dres[4 * w + 3]), r)));
             er[s - 1] = er[s - 2] + eE + r;
             n_terms = s;
         }
         if (!ok) break;
 
-        // ---- Sq = Q8(align(R_1..))
+        STAMP8(7);
+        // ---- Sq = Q8(align(R_1..)): the exponents fall by several bits per power, so most terms are
+        // shifted far to the right; a term whose right shift exceeds 7 rounds to zero and is skipped
         int sq[kHC];
         int eS = 0;
         if (n_terms > 0) {
@@ -460,25 +505,30 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
 #pragma unroll
             for (int s = 1; s < kSMax; ++s)
                 if (s < n_terms) { emin = min(emin, er[s]); emax = max(emax, er[s]); }
-            const int eref = max(emin, emax - 24);
-            auto acc_s = [&](int jl) -> long long {
-                long long a = 0;
+            const int eref = max(emin, emax - kAlignWindow);
+            int sh[kSMax];
 #pragma unroll
-                for (int s = 0; s < kSMax; ++s)
-                    if (s < n_terms) a += shift64(byte_at(rpk[s][jl >> 2], jl & 3), er[s] - eref);
-                return a;
-            };
+            for (int s = 0; s < kSMax; ++s) sh[s] = (s < n_terms) ? er[s] - eref : -64;
+            int acc[kHC];
             unsigned long long m = 0;
 #pragma unroll
-            for (int jl = 0; jl < kHC; ++jl) m |= absll(acc_s(jl));
+            for (int jl = 0; jl < kHC; ++jl) {
+                int a = 0;
+#pragma unroll
+                for (int s = 0; s < kSMax; ++s)
+                    if (sh[s] >= -7) a += term32(byte_at(rpk[s][jl >> 2], jl & 3), sh[s]);
+                acc[jl] = a;
+                m |= abs_bits<int>(a);
+            }
             const int r = q8_shift(chunk_bitlen(m, slot++));
 #pragma unroll
-            for (int jl = 0; jl < kHC; ++jl) sq[jl] = clamp127(rsr64(acc_s(jl), r));
+            for (int jl = 0; jl < kHC; ++jl) sq[jl] = clamp127_t<int>(rsr_t<int>(acc[jl], r));
             eS = eref + r;
         } else {
 #pragma unroll
             for (int jl = 0; jl < kHC; ++jl) sq[jl] = 0;
         }
+        STAMP8(8);
         // Sq bytes to the private rows (the rows above are needed for T0q Sq)
         {
             uint4 v0, v1;
@@ -491,6 +541,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
         }
         cta_barrier();
 
+        STAMP8(9);
         // ---- I8: Toffq = Q8(align(T0q, Sq, T0q Sq)) on i > j
         int toff[kHC];
         int eT;
@@ -500,35 +551,40 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             for (int jl = 0; jl < kHC; ++jl) prod[jl] = 0;
 #pragma unroll
             for (int e = 1; e <= 3; ++e) {
-                const int r = (t - e) > 0 ? (t - e) : 0;
-                const int cf = (il - e >= 0) ? t0q[e] : 0;
-                const uint4 a0 = *reinterpret_cast<const uint4*>(sRowA + r * 64 + col0);
-                const uint4 a1 = *reinterpret_cast<const uint4*>(sRowA + r * 64 + col0 + 16);
+                const int rr = (t - e) > 0 ? (t - e) : 0;
+                const int cf = (il - e >= 0) ? (e == 1 ? t0q1 : (e == 2 ? t0q2 : t0q3)) : 0;
+                const uint4 a0 = *reinterpret_cast<const uint4*>(sRowA + rr * 64 + col0);
+                const uint4 a1 = *reinterpret_cast<const uint4*>(sRowA + rr * 64 + col0 + 16);
                 const uint32_t w[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
 #pragma unroll
                 for (int jl = 0; jl < kHC; ++jl) prod[jl] += cf * byte_at(w[jl >> 2], jl & 3);
             }
             const int e0 = eT0, e1 = eS, e2 = eT0 + eS;
             const int emin = min(e0, min(e1, e2)), emax = max(e0, max(e1, e2));
-            const int eref = max(emin, emax - 24);
-            auto acc_t = [&](int jl) -> long long {
-                const int d = il - (col0 + jl);
-                if (d <= 0) return 0;
-                int band = 0;
-#pragma unroll
-                for (int e = 1; e <= 3; ++e)
-                    if (d == e) band = t0q[e];
-                return shift64(band, e0 - eref) + shift64(sq[jl], e1 - eref) + shift64(prod[jl], e2 - eref);
-            };
+            const int eref = max(emin, emax - kAlignWindow);
+            const int s0 = e0 - eref, s1 = e1 - eref, s2 = e2 - eref;
+            // the band entry and Sq never share an element (band: distance <= N, Sq: distance > N): one value per
+            // element with its own shift; entries below 2^7, the product below 3 * 127^2 < 2^16
+            int acc[kHC];
             unsigned long long m = 0;
 #pragma unroll
-            for (int jl = 0; jl < kHC; ++jl) m |= absll(acc_t(jl));
+            for (int jl = 0; jl < kHC; ++jl) {
+                const int d = il - (col0 + jl);
+                int v = sq[jl];
+                if (d == 1 && N >= 1) v = t0q1;
+                if (d == 2 && N >= 2) v = t0q2;
+                if (d == 3 && N >= 3) v = t0q3;
+                const int a = (d > 0) ? (term32(v, (d <= N) ? s0 : s1) + term32(prod[jl], s2)) : 0;
+                acc[jl] = a;
+                m |= abs_bits<int>(a);
+            }
             const int r = q8_shift(chunk_bitlen(m, slot++));
 #pragma unroll
-            for (int jl = 0; jl < kHC; ++jl) toff[jl] = clamp127(rsr64(acc_t(jl), r));
+            for (int jl = 0; jl < kHC; ++jl) toff[jl] = clamp127_t<int>(rsr_t<int>(acc[jl], r));
             eT = eref + r;
         }
 
+        STAMP8(10);
         // ---- I9: Tbq = Q8(Toffq_ij beta_q_j); A operand of W/U (block diagonal, int8 in TMEM)
         int eTb;
         {
@@ -537,14 +593,14 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
 #pragma unroll
             for (int jl = 0; jl < kHC; ++jl) {
                 acc[jl] = toff[jl] * sbeta[cb + col0 + jl];
-                m |= absll(acc[jl]);
+                m |= abs_bits<int>(acc[jl]);
             }
             const int r = q8_shift(chunk_bitlen(m, slot++));
             uint32_t r8[8];
 #pragma unroll
             for (int w = 0; w < 8; ++w)
-                r8[w] = pack4(clamp127(rsr64(acc[4 * w], r)), clamp127(rsr64(acc[4 * w + 1], r)), clamp127(rsr64(acc[4 * w + 2], r)),
-                              clamp127(rsr64(acc[4 * w + 3], r)));
+                r8[w] = pack4(clamp127_t<int>(rsr_t<int>(acc[4 * w], r)), clamp127_t<int>(rsr_t<int>(acc[4 * w + 1], r)),
+                              clamp127_t<int>(rsr_t<int>(acc[4 * w + 2], r)), clamp127_t<int>(rsr_t<int>(acc[4 * w + 3], r)));
             eTb = eT - 15 + r;
             // row t's block occupies packed columns [cb/4, cb/4 + 16) of a 32-column operand; the other 16 are zero
             tmem_st8(lane_base + kAS + cb / 4 + h * 8, r8);
@@ -553,6 +609,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             tmem_st8(lane_base + kAS + (16 - cb / 4) + h * 8, r8);
             tmem_wait_st();
         }
+        STAMP8(11);
         // Toffq row -> staging (64-byte lines, 64-byte TMA swizzle) -> bulk tensor store of 32 rows per warp (h = 0 issues)
         uint8_t* stage = smem + kOffStage;
         if (p.Toff != nullptr) {
@@ -586,12 +643,13 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             mma_commit(&bar_mma);
         }
 
+        STAMP8(12);
         // ---- I10: W, then U
 #pragma unroll 1
         for (int half = 0; half < 2; ++half) {
             const int xexp = (half == 0) ? kexp : vexp;
             const uint8_t* xtile = (half == 0) ? sK : sV;
-            // own row of the int8 tile (64 columns of this thread): diagonal term beta_q_i * Xq_i
+            // diagonal term beta_q_i * Xq_i for this thread's 64 columns, from its own row of the int8 tile
             uint32_t xr[16];
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
@@ -603,10 +661,8 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             tc_fence_after_sync();
             const int ep = eTb + xexp, ed = xexp - 15;
             const int eref = align_ref2(ep, ed);
-            auto acc_w = [&](uint32_t raw, int col) -> long long {
-                return shift64(static_cast<int>(raw), ep - eref) +
-                       shift64(static_cast<long long>(bq) * byte_at(xr[col >> 2], col & 3), ed - eref);
-            };
+            const int sp = ep - eref, sd = ed - eref;
+            // |Tbq Xq| <= 128 * 127^2 < 2^21, |beta_q Xq| < 2^22; at most one of them is shifted left, by at most 8
             // pass 1: the scale (bit length of the largest magnitude over the chunk's C x d block)
             unsigned long long m = 0;
 #pragma unroll
@@ -615,7 +671,8 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 tmem_ld32(lane_base + kR0 + h * 64 + c0, r);
                 tmem_wait_ld();
 #pragma unroll
-                for (int i = 0; i < 32; ++i) m |= absll(acc_w(r[i], c0 + i));
+                for (int i = 0; i < 32; ++i)
+                    m |= abs_bits<int>(term32(static_cast<int>(r[i]), sp) + term32(bq * byte_at(xr[(c0 + i) >> 2], (c0 + i) & 3), sd));
             }
             const int rr = q8_shift(chunk_bitlen(m, slot++));
             // after that barrier every thread holds its own row of the K (V) tile in registers, and the products that
@@ -642,17 +699,19 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 uint32_t r[32];
                 tmem_ld32(lane_base + kR0 + h * 64 + c0, r);
                 tmem_wait_ld();
+                int qv[32];
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    qv[i] = clamp127_t<int>(rsr_t<int>(
+                        term32(static_cast<int>(r[i]), sp) + term32(bq * byte_at(xr[(c0 + i) >> 2], (c0 + i) & 3), sd), rr));
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
-                    uint32_t w4[4];
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const int i = c * 16 + q * 4;
-                        w4[q] = pack4(clamp127(rsr64(acc_w(r[i], c0 + i), rr)), clamp127(rsr64(acc_w(r[i + 1], c0 + i + 1), rr)),
-                                      clamp127(rsr64(acc_w(r[i + 2], c0 + i + 2), rr)), clamp127(rsr64(acc_w(r[i + 3], c0 + i + 3), rr)));
-                    }
                     const int cc = c0 / 16 + c;
-                    *reinterpret_cast<uint4*>(sub + lane * 64 + ((cc ^ ((lane >> 1) & 3)) << 4)) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+                    const uint4 v = make_uint4(pack4(qv[16 * c + 0], qv[16 * c + 1], qv[16 * c + 2], qv[16 * c + 3]),
+                                               pack4(qv[16 * c + 4], qv[16 * c + 5], qv[16 * c + 6], qv[16 * c + 7]),
+                                               pack4(qv[16 * c + 8], qv[16 * c + 9], qv[16 * c + 10], qv[16 * c + 11]),
+                                               pack4(qv[16 * c + 12], qv[16 * c + 13], qv[16 * c + 14], qv[16 * c + 15]));
+                    *reinterpret_cast<uint4*>(sub + lane * 64 + ((cc ^ ((lane >> 1) & 3)) << 4)) = v;
                 }
             }
             if (half == 0) {
@@ -678,6 +737,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 tma_store_commit();
             }
         }
+        STAMP8(13);
         par_kv ^= 1;
     }
     if (lane == 0) tma_store_wait_all<0>();
@@ -723,6 +783,12 @@ bool make_map(CUtensorMap* tm, const void* base, long long heads, int T, int col
 }
 
 }  // namespace
+
+#ifdef GDN_TRACE
+extern "C" int gdn_debug_read_trace8(long long* host_out) {
+    return cudaMemcpyFromSymbol(host_out, g_trace8, sizeof(long long) * 4096) == cudaSuccess ? 0 : -1;
+}
+#endif
 
 void int8_decay_lut(uint16_t* out) {
     for (int f = 0; f < 256; ++f) out[f] = static_cast<uint16_t>(floor(32768.0 * exp2(-static_cast<double>(f) / 256.0) + 0.5));
