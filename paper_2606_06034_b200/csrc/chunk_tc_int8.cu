@@ -114,6 +114,14 @@ __device__ __forceinline__ T term_t(int x, int s) {
     return static_cast<T>(rsr_t<int>(x, (-s) < 31 ? (-s) : 31));
 }
 __device__ __forceinline__ int term32(int x, int s) { return term_t<int>(x, s); }
+// clamp(rsr(x, r), +-127) for 32-bit x
+__device__ __forceinline__ int q8_32(int x, int r) {
+    const int sgn = x >> 31;
+    int a = (x ^ sgn) - sgn;
+    a = (a + ((1 << r) >> 1)) >> r;
+    a = a > 127 ? 127 : a;
+    return (a ^ sgn) - sgn;
+}
 template <typename T>
 __device__ __forceinline__ unsigned long long abs_bits(T x) { return static_cast<unsigned long long>(x < 0 ? -x : x); }
 template <typename T>
@@ -361,15 +369,15 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             if (N >= 2) {
                 const unsigned long long m = (h == 0) ? (abs_bits<int>(acc22) | abs_bits<int>(acc23)) : 0ull;
                 const int r = q8_shift(chunk_bitlen(m, slot++));
-                p22 = clamp127_t<int>(rsr_t<int>(acc22, r));
-                p23 = clamp127_t<int>(rsr_t<int>(acc23, r));
+                p22 = q8_32(acc22, r);
+                p23 = q8_32(acc23, r);
                 e2 = eA + eA + r;
             }
             if (N >= 3) {
                 // P_3 at distance 3: P_2[i][i-2] * Aq[i-2][i-3]
                 const int acc3 = p22 * sAB[r2 * 8 + 1];
                 const int r = q8_shift(chunk_bitlen((h == 0) ? abs_bits<int>(acc3) : 0ull, slot++));
-                p33 = clamp127_t<int>(rsr_t<int>(acc3, r));
+                p33 = q8_32(acc3, r);
                 e3 = e2 + eA + r;
             }
             // align(P_1..P_N): at most three small terms per band entry
@@ -386,9 +394,9 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             if (!(N >= 3 && il >= 3)) a3 = 0;
             const unsigned long long m = (h == 0) ? (abs_bits<int>(a1) | abs_bits<int>(a2) | abs_bits<int>(a3)) : 0ull;
             const int r = q8_shift(chunk_bitlen(m, slot++));
-            t0q1 = clamp127_t<int>(rsr_t<int>(a1, r));
-            t0q2 = clamp127_t<int>(rsr_t<int>(a2, r));
-            t0q3 = clamp127_t<int>(rsr_t<int>(a3, r));
+            t0q1 = q8_32(a1, r);
+            t0q2 = q8_32(a2, r);
+            t0q3 = q8_32(a3, r);
             eT0 = eref + r;
             if (h == 0) {
                 if (il >= 1) sSH[(t - 1) * 4 + 0] = t0q1;
@@ -406,6 +414,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             const int eref = align_ref2(eA, eA + eT0);
             const int sa = eA - eref, sp = eA + eT0 - eref;
             int acc[kHC];  // |Aq| < 2^7 and |Aq T0q| <= 3 * 127^2 < 2^16, shifted left by at most 8
+            const bool left = sa >= 0 && sp >= 0;
             unsigned long long m = 0;
 #pragma unroll
             for (int jl = 0; jl < kHC; ++jl) {
@@ -414,13 +423,14 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 const int a2 = (jl + 2 < kHC) ? aq[(jl + 2 < kHC) ? jl + 2 : 0] : ((jl + 2 == kHC) ? an0 : (jl + 2 == kHC + 1 ? an1 : an2));
                 const int a3 = (jl + 3 < kHC) ? aq[(jl + 3 < kHC) ? jl + 3 : 0] : ((jl + 3 == kHC) ? an0 : (jl + 3 == kHC + 1 ? an1 : an2));
                 const bool on = (il - (col0 + jl)) > N;
-                const int v = on ? (term32(aq[jl], sa) + term32(a1 * c4.x + a2 * c4.y + a3 * c4.z, sp)) : 0;
+                const int pr = a1 * c4.x + a2 * c4.y + a3 * c4.z;
+                const int v = on ? (left ? ((aq[jl] << sa) + (pr << sp)) : (term32(aq[jl], sa) + term32(pr, sp))) : 0;
                 acc[jl] = v;
                 m |= abs_bits<int>(v);
             }
             const int r = q8_shift(chunk_bitlen(m, slot++));
 #pragma unroll
-            for (int jl = 0; jl < kHC; ++jl) eq[jl] = clamp127_t<int>(rsr_t<int>(acc[jl], r));
+            for (int jl = 0; jl < kHC; ++jl) eq[jl] = q8_32(acc[jl], r);
             eE = eref + r;
         }
         STAMP8(6);
@@ -486,10 +496,10 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             const int r = q8_shift(chunk_bitlen(m, slot++));
 #pragma unroll
             for (int w = 0; w < kHC / 4; ++w)
-                rpk[s - 1][w] = pack4(clamp127_t<int>(rsr_t<int>(static_cast<int>(dres[4 * w]), r)),
-                                      clamp127_t<int>(rsr_t<int>(static_cast<int>(dres[4 * w + 1]), r)),
-                                      clamp127_t<int>(rsr_t<int>(static_cast<int>(dres[4 * w + 2]), r)),
-                                      clamp127_t<int>(rsr_t<int>(static_cast<int>(dres[4 * w + 3]), r)));
+                rpk[s - 1][w] = pack4(q8_32(static_cast<int>(dres[4 * w]), r),
+                                      q8_32(static_cast<int>(dres[4 * w + 1]), r),
+                                      q8_32(static_cast<int>(dres[4 * w + 2]), r),
+                                      q8_32(static_cast<int>(dres[4 * w + 3]), r));
             er[s - 1] = er[s - 2] + eE + r;
             n_terms = s;
         }
@@ -510,19 +520,24 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
 #pragma unroll
             for (int s = 0; s < kSMax; ++s) sh[s] = (s < n_terms) ? er[s] - eref : -64;
             int acc[kHC];
+#pragma unroll
+            for (int jl = 0; jl < kHC; ++jl) acc[jl] = 0;
+#pragma unroll
+            for (int s = 0; s < kSMax; ++s) {
+                if (sh[s] >= 0) {
+#pragma unroll
+                    for (int jl = 0; jl < kHC; ++jl) acc[jl] += byte_at(rpk[s][jl >> 2], jl & 3) << sh[s];
+                } else if (sh[s] >= -7) {
+#pragma unroll
+                    for (int jl = 0; jl < kHC; ++jl) acc[jl] += rsr_t<int>(byte_at(rpk[s][jl >> 2], jl & 3), -sh[s]);
+                }
+            }
             unsigned long long m = 0;
 #pragma unroll
-            for (int jl = 0; jl < kHC; ++jl) {
-                int a = 0;
-#pragma unroll
-                for (int s = 0; s < kSMax; ++s)
-                    if (sh[s] >= -7) a += term32(byte_at(rpk[s][jl >> 2], jl & 3), sh[s]);
-                acc[jl] = a;
-                m |= abs_bits<int>(a);
-            }
+            for (int jl = 0; jl < kHC; ++jl) m |= abs_bits<int>(acc[jl]);
             const int r = q8_shift(chunk_bitlen(m, slot++));
 #pragma unroll
-            for (int jl = 0; jl < kHC; ++jl) sq[jl] = clamp127_t<int>(rsr_t<int>(acc[jl], r));
+            for (int jl = 0; jl < kHC; ++jl) sq[jl] = q8_32(acc[jl], r);
             eS = eref + r;
         } else {
 #pragma unroll
@@ -565,6 +580,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             const int s0 = e0 - eref, s1 = e1 - eref, s2 = e2 - eref;
             // the band entry and Sq never share an element (band: distance <= N, Sq: distance > N): one value per
             // element with its own shift; entries below 2^7, the product below 3 * 127^2 < 2^16
+            const bool left = s0 >= 0 && s1 >= 0 && s2 >= 0;
             int acc[kHC];
             unsigned long long m = 0;
 #pragma unroll
@@ -574,13 +590,15 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 if (d == 1 && N >= 1) v = t0q1;
                 if (d == 2 && N >= 2) v = t0q2;
                 if (d == 3 && N >= 3) v = t0q3;
-                const int a = (d > 0) ? (term32(v, (d <= N) ? s0 : s1) + term32(prod[jl], s2)) : 0;
+                const int a = (d > 0) ? (left ? ((v << ((d <= N) ? s0 : s1)) + (prod[jl] << s2))
+                                              : (term32(v, (d <= N) ? s0 : s1) + term32(prod[jl], s2)))
+                                      : 0;
                 acc[jl] = a;
                 m |= abs_bits<int>(a);
             }
             const int r = q8_shift(chunk_bitlen(m, slot++));
 #pragma unroll
-            for (int jl = 0; jl < kHC; ++jl) toff[jl] = clamp127_t<int>(rsr_t<int>(acc[jl], r));
+            for (int jl = 0; jl < kHC; ++jl) toff[jl] = q8_32(acc[jl], r);
             eT = eref + r;
         }
 
@@ -599,8 +617,8 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             uint32_t r8[8];
 #pragma unroll
             for (int w = 0; w < 8; ++w)
-                r8[w] = pack4(clamp127_t<int>(rsr_t<int>(acc[4 * w], r)), clamp127_t<int>(rsr_t<int>(acc[4 * w + 1], r)),
-                              clamp127_t<int>(rsr_t<int>(acc[4 * w + 2], r)), clamp127_t<int>(rsr_t<int>(acc[4 * w + 3], r)));
+                r8[w] = pack4(q8_32(acc[4 * w], r), q8_32(acc[4 * w + 1], r),
+                              q8_32(acc[4 * w + 2], r), q8_32(acc[4 * w + 3], r));
             eTb = eT - 15 + r;
             // row t's block occupies packed columns [cb/4, cb/4 + 16) of a 32-column operand; the other 16 are zero
             tmem_st8(lane_base + kAS + cb / 4 + h * 8, r8);
@@ -664,15 +682,22 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             const int sp = ep - eref, sd = ed - eref;
             // |Tbq Xq| <= 128 * 127^2 < 2^21, |beta_q Xq| < 2^22; at most one of them is shifted left, by at most 8
             // pass 1: the scale (bit length of the largest magnitude over the chunk's C x d block)
+            const bool left = sp >= 0 && sd >= 0;  // the usual case: plain left shifts
             unsigned long long m = 0;
 #pragma unroll
             for (int c0 = 0; c0 < 64; c0 += 32) {
                 uint32_t r[32];
                 tmem_ld32(lane_base + kR0 + h * 64 + c0, r);
                 tmem_wait_ld();
+                if (left) {
 #pragma unroll
-                for (int i = 0; i < 32; ++i)
-                    m |= abs_bits<int>(term32(static_cast<int>(r[i]), sp) + term32(bq * byte_at(xr[(c0 + i) >> 2], (c0 + i) & 3), sd));
+                    for (int i = 0; i < 32; ++i)
+                        m |= abs_bits<int>((static_cast<int>(r[i]) << sp) + ((bq * byte_at(xr[(c0 + i) >> 2], (c0 + i) & 3)) << sd));
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        m |= abs_bits<int>(term32(static_cast<int>(r[i]), sp) + term32(bq * byte_at(xr[(c0 + i) >> 2], (c0 + i) & 3), sd));
+                }
             }
             const int rr = q8_shift(chunk_bitlen(m, slot++));
             // after that barrier every thread holds its own row of the K (V) tile in registers, and the products that
@@ -700,10 +725,15 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 tmem_ld32(lane_base + kR0 + h * 64 + c0, r);
                 tmem_wait_ld();
                 int qv[32];
+                if (left) {
 #pragma unroll
-                for (int i = 0; i < 32; ++i)
-                    qv[i] = clamp127_t<int>(rsr_t<int>(
-                        term32(static_cast<int>(r[i]), sp) + term32(bq * byte_at(xr[(c0 + i) >> 2], (c0 + i) & 3), sd), rr));
+                    for (int i = 0; i < 32; ++i)
+                        qv[i] = q8_32((static_cast<int>(r[i]) << sp) + ((bq * byte_at(xr[(c0 + i) >> 2], (c0 + i) & 3)) << sd), rr);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        qv[i] = q8_32(term32(static_cast<int>(r[i]), sp) + term32(bq * byte_at(xr[(c0 + i) >> 2], (c0 + i) & 3), sd), rr);
+                }
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
                     const int cc = c0 / 16 + c;
