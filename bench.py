@@ -287,6 +287,21 @@ def run_extras(gdn, gen, dev, args):
             del inp, outs
         except Exception as exc:  # an unsupported extra must not lose the headline
             out[f"{name}:{method}"] = {"error": repr(exc)}
+    # INT8 variant on the prefill shapes (integer inputs quantised once from the same tensors)
+    try:
+        inp = gen.make_workload("prefill_gqa", device=dev)
+        q = gen.make_int8_inputs(inp)
+        outs = gdn.chunk_prepare_int8(q)
+        fn = lambda: gdn.chunk_prepare_int8(q, outputs=outs)
+        total_ms, _ = device_time_steps(fn, 10, 3, None)
+        ms = total_ms / 10
+        group = inp.H_v // inp.H_k
+        by = inp.C * inp.d_k / group + inp.C * inp.d_v + inp.C * inp.d_k + inp.C * inp.d_v + inp.C * inp.C + 6 * inp.C
+        out["prefill_gqa:int8"] = {"chunks_per_s": q.n_chunks / (ms * 1e-3), "ms": ms,
+                                   "hbm_frac": q.n_chunks * by / (ms * 1e-3) / 1e9 / hbm_peak}
+        del inp, q, outs
+    except Exception as exc:
+        out["prefill_gqa:int8"] = {"error": repr(exc)}
     return out
 
 
