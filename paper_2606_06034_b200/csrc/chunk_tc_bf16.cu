@@ -302,11 +302,16 @@ __device__ __forceinline__ TileCoord decode_tile(uint32_t tile, const Params& p)
     return c;
 }
 
-template <int C, int NB, int MODE>
+// MERGE: the tile is ONE chunk of 128 tokens whose two 64 x 64 diagonal blocks are inverted by the scheme above
+// (C = 64 is then the block size) and whose lower-left block follows from App. E, Eq. 28:
+// T21 = -T22 A21 T11, evaluated as Y = A21 + A21 X11, T21 = -(Y + X22 Y) with X = T - I of the blocks, so that
+// the identity parts stay in fp32 and only the small products pass through bf16 operands.
+template <int C, int NB, int MODE, bool MERGE>
 __global__ void __launch_bounds__(kThreads, 2)
 chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                 const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmU,
                 const __grid_constant__ CUtensorMap tmT, const Params p) {
+    static_assert(!MERGE || (C == 64 && MODE == INV_NEUMANN), "the block merge is built for 64-blocks of the Neumann scheme");
     using L = Smem<C, NB>;
     using SP = Split<C>;
     constexpr int NBP = L::NBP;
@@ -449,6 +454,22 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         STAMP(3);
         tc_fence_after_sync();
         float a[HC];
+        if constexpr (MERGE) {
+            // rows of the second block keep their part of the lower-left Gram block (columns 0..63) in R2:
+            // R0..R1 is overwritten by the residual rounds
+            if (wq >= 2) {
+                uint32_t r[32], r16[16];
+                tmem_ld32(lane_base + kR0 + h * 32, r);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 16; ++i) r16[i] = r[i];
+                tmem_st16(lane_base + kR2 + h * 32, r16);
+#pragma unroll
+                for (int i = 0; i < 16; ++i) r16[i] = r[16 + i];
+                tmem_st16(lane_base + kR2 + h * 32 + 16, r16);
+                tmem_wait_st();
+            }
+        }
         if (active) {
             load_diag_block<C>(lane_base, kR0, t, h, a);
             const float gs = gi_ * kLog2e;
@@ -680,6 +701,92 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         }
         // a[] = this thread's part of the far row (T - I - L)
 
+        float y[HC];  // MERGE, rows of the second block: A21 part, then Y, then T21 (columns of the first block)
+#pragma unroll
+        for (int j = 0; j < HC; ++j) y[j] = 0.f;
+        if constexpr (MERGE) {
+            const uint32_t idesc_m = instr_desc(128, 64, 1, 1, 0, 1, 1);
+            // X = T - I of the row's diagonal block as packed bf16 (band without the unit diagonal + far part)
+            uint32_t xrow[PCH];
+            {
+                uint16_t vals[NB + 1];
+                vals[0] = 0;
+#pragma unroll
+                for (int e = 1; e <= NB; ++e) vals[e] = bf16_bits(lb[e]);
+                uint32_t bpL[PCH];
+                build_band_row<C, NB>(br_row, t, il, col0, n_band, vals, bpL);
+#pragma unroll
+                for (int i = 0; i < PCH; ++i) xrow[i] = (pack_bf16x2(a[2 * i], a[2 * i + 1]) & keep[i]) | bpL[i];
+            }
+            if (wq < 2) {
+                // first block: X11 rows as the B operand [64 x 64] (MN-major, no swizzle) of Y = A21 + A21 X11
+#pragma unroll
+                for (int c = 0; c < CPT; ++c)
+                    *reinterpret_cast<uint4*>(sEB + ((col0 >> 3) + c) * 1024 + t * 16) =
+                        make_uint4(xrow[4 * c], xrow[4 * c + 1], xrow[4 * c + 2], xrow[4 * c + 3]);
+            } else {
+                // second block: A21_ij = beta_i e^{g_i - g_j} G_ij, j in the first block (fp32), bf16 copy as A operand
+                uint32_t gq[32];
+                tmem_ld32(lane_base + kR2 + h * 32, gq);
+                tmem_wait_ld();
+                const float gs = gi_ * kLog2e;
+                const float4* sg4 = reinterpret_cast<const float4*>(sg + col0);
+#pragma unroll
+                for (int j4 = 0; j4 < HC / 4; ++j4) {
+                    const float4 gv = sg4[j4];
+                    const float gj[4] = {gv.x, gv.y, gv.z, gv.w};
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        y[j4 * 4 + q] = bi * fast_exp2(fmaf(-gj[q], kLog2e, gs)) * __uint_as_float(gq[j4 * 4 + q]);
+                }
+                uint32_t pk[PCH];
+#pragma unroll
+                for (int i = 0; i < PCH; ++i) pk[i] = pack_bf16x2(y[2 * i], y[2 * i + 1]);
+                store_stacked_operand<C>(lane_base + kAS, h, pk);
+                tmem_wait_st();
+            }
+#pragma unroll 1
+            for (int step = 0; step < 2; ++step) {
+                fence_proxy_async_smem();
+                tc_fence_before_sync();
+                compute_barrier();
+                if (tid == 0) {
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) {
+                        const uint64_t bd = smem_desc(sEB_a + ks * 256, 128, 1024, SWZ_NONE);
+                        mma_f16_ts(tmem + kR0, tmem + kAS + ks * 8, bd, idesc_m, ks > 0);
+                    }
+                    mma_commit(&bar_mma);
+                }
+                if (!wait_bar(&bar_mma, par_mma)) { ok = false; break; }
+                par_mma ^= 1;
+                tc_fence_after_sync();
+                if (wq >= 2) {
+                    uint32_t d[32];
+                    tmem_ld32(lane_base + kR0 + h * 32, d);
+                    tmem_wait_ld();
+                    if (step == 0) {
+                        // Y = A21 + A21 X11; then Y rows as B operand and X22 rows as A operand of X22 Y
+#pragma unroll
+                        for (int j = 0; j < HC; ++j) y[j] += __uint_as_float(d[j]);
+#pragma unroll
+                        for (int c = 0; c < CPT; ++c)
+                            *reinterpret_cast<uint4*>(sEB + ((col0 >> 3) + c) * 1024 + il * 16) =
+                                make_uint4(pack_bf16x2(y[8 * c + 0], y[8 * c + 1]), pack_bf16x2(y[8 * c + 2], y[8 * c + 3]),
+                                           pack_bf16x2(y[8 * c + 4], y[8 * c + 5]), pack_bf16x2(y[8 * c + 6], y[8 * c + 7]));
+                        store_stacked_operand<C>(lane_base + kAS, h, xrow);
+                        tmem_wait_st();
+                    } else {
+                        // T21 = -(Y + X22 Y)
+#pragma unroll
+                        for (int j = 0; j < HC; ++j) y[j] = -(y[j] + __uint_as_float(d[j]));
+                    }
+                }
+            }
+            if (!ok) break;
+        }
+
         STAMP(9);
         // ---- A operands for W/U: T diag(beta) = hi + lo, hi over the whole row, lo only on band + diagonal
         if (active) {
@@ -701,7 +808,20 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 const float2 bb = sb2[i];
                 pk[i] = (pack_bf16x2(a[2 * i] * bb.x, a[2 * i + 1] * bb.y) & keep[i]) | bp[i];
             }
-            store_a_operand<C, true>(lane_base + kAS, t, h, pk);
+            if (MERGE && wq >= 2) {
+                // second block of a 128-chunk: columns of the first block carry T21 diag(beta) instead of zeros
+                store_a_operand<C, false>(lane_base + kAS, t, h, pk);
+                const float2* sb1 = reinterpret_cast<const float2*>(sbeta + col0);
+                uint32_t po[PCH];
+#pragma unroll
+                for (int i = 0; i < PCH; ++i) {
+                    const float2 bb = sb1[i];
+                    po[i] = pack_bf16x2(y[2 * i] * bb.x, y[2 * i + 1] * bb.y);
+                }
+                store_stacked_operand<C>(lane_base + kAS, h, po);
+            } else {
+                store_a_operand<C, true>(lane_base + kAS, t, h, pk);
+            }
             build_band_row<C, NB>(br_row, t, il, col0, n_band, lo, bp);
             store_a_operand<C, true>(lane_base + kR2, t, h, bp);
             tmem_wait_st();
@@ -723,7 +843,31 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         STAMP(8);
         // ---- T row -> Tinv: each half-row goes to a staging line in the TMA swizzle layout (the band-row
         // region is free now); one bulk tensor store of 32 rows x HC columns per warp, overlapping the W products
-        if (p.Tinv != nullptr && active) {
+        if (MERGE && p.Tinv != nullptr) {
+            // rows of the 128 x 128 inverse in four column groups of 32 (64-byte lines, 64-byte TMA swizzle):
+            // the row's diagonal-block part, and its part of the other block column (T21, or zeros above it)
+            const int gd = (cb >> 5) + h;                  // group of the diagonal-block part
+            const int go = (wq >= 2) ? h : (2 + h);        // group of the off-diagonal part
+            const uint32_t rowd = scratch_a + gd * 8192 + t * 64;
+            const uint32_t rowo = scratch_a + go * 8192 + t * 64;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                sts128(rowd + (swz<4>(t, c) << 4),
+                       (pack_bf16x2(a[c * 8 + 0], a[c * 8 + 1]) & keep[c * 4 + 0]) | bpT[c * 4 + 0],
+                       (pack_bf16x2(a[c * 8 + 2], a[c * 8 + 3]) & keep[c * 4 + 1]) | bpT[c * 4 + 1],
+                       (pack_bf16x2(a[c * 8 + 4], a[c * 8 + 5]) & keep[c * 4 + 2]) | bpT[c * 4 + 2],
+                       (pack_bf16x2(a[c * 8 + 6], a[c * 8 + 7]) & keep[c * 4 + 3]) | bpT[c * 4 + 3]);
+                sts128(rowo + (swz<4>(t, c) << 4), pack_bf16x2(y[c * 8 + 0], y[c * 8 + 1]), pack_bf16x2(y[c * 8 + 2], y[c * 8 + 3]),
+                       pack_bf16x2(y[c * 8 + 4], y[c * 8 + 5]), pack_bf16x2(y[c * 8 + 6], y[c * 8 + 7]));
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                tma_store_3d(&tmT, smem + L::kEB + gd * 8192 + wrow0 * 64, gd * 32, tc.t0 + wrow0, tc.bhv);
+                tma_store_3d(&tmT, smem + L::kEB + go * 8192 + wrow0 * 64, go * 32, tc.t0 + wrow0, tc.bhv);
+                tma_store_commit();
+            }
+        } else if (p.Tinv != nullptr && active) {
             constexpr int RB = HC * 2;  // bytes per staged half-row
             const uint32_t stage = smem_u32(smem + L::kBR) + h * (kTile * RB);
             const uint32_t trow = stage + t * RB;
@@ -860,11 +1004,11 @@ struct Maps {
     CUtensorMap K, V, W, U, T;
 };
 
-template <int C, int NB, int MODE>
+template <int C, int NB, int MODE, bool MERGE>
 int launch_one(const Maps& m, const Params& prm, cudaStream_t stream) {
     using L = Smem<C, NB>;
     const int smem = L::kTotal + 1024;
-    auto kern = chunk_tc_kernel<C, NB, MODE>;
+    auto kern = chunk_tc_kernel<C, NB, MODE, MERGE>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return GDN_ERR_LAUNCH;
     long long grid = prm.n_tiles < 2 * 148 ? prm.n_tiles : 2 * 148;
     kern<<<static_cast<int>(grid), kThreads, smem, stream>>>(m.K, m.V, m.W, m.U, m.T, prm);
@@ -872,10 +1016,10 @@ int launch_one(const Maps& m, const Params& prm, cudaStream_t stream) {
     return cudaGetLastError() == cudaSuccess ? GDN_OK : GDN_ERR_LAUNCH;
 }
 
-template <int C, int MODE>
+template <int C, int MODE, bool MERGE = false>
 int launch_c(const Maps& m, const Params& prm, cudaStream_t stream) {
-    if (MODE != INV_NEUMANN || prm.N <= 3) return launch_one<C, 3, MODE>(m, prm, stream);
-    return launch_one<C, 7, MODE>(m, prm, stream);
+    if (MODE != INV_NEUMANN || prm.N <= 3) return launch_one<C, 3, MODE, MERGE>(m, prm, stream);
+    return launch_one<C, 7, MODE, MERGE>(m, prm, stream);
 }
 
 }  // namespace
@@ -888,7 +1032,7 @@ extern "C" int gdn_debug_read_trace(long long* host_out) {
 
 int launch_tc_bf16(const Problem& p, InverseMode mode, cudaStream_t stream) {
     if (p.d_k != kD || p.d_v != kD) return GDN_ERR_UNSUPPORTED;
-    if (!(p.C == 16 || p.C == 32 || p.C == 64)) return GDN_ERR_UNSUPPORTED;
+    if (!(p.C == 16 || p.C == 32 || p.C == 64 || (p.C == 128 && mode == INV_NEUMANN))) return GDN_ERR_UNSUPPORTED;
     if (mode == INV_NEUMANN && (p.order < 1 || p.order > 7)) return GDN_ERR_UNSUPPORTED;
     if (mode == INV_FWDSUBST_BLOCKED) return GDN_ERR_UNSUPPORTED;
     if ((long long)p.B * p.H_v * p.T == 0) return GDN_OK;
@@ -897,7 +1041,7 @@ int launch_tc_bf16(const Problem& p, InverseMode mode, cudaStream_t stream) {
     Maps m;
     const long long hk = (long long)p.B * p.H_k, hv = (long long)p.B * p.H_v;
     // Tinv leaves in boxes of 32 rows x (C/2 columns for C >= 32, else C columns): 64-, 32- and 32-byte lines
-    const int tbox = (p.C >= 32) ? p.C / 2 : p.C;
+    const int tbox = (p.C == 128) ? 32 : ((p.C >= 32) ? p.C / 2 : p.C);
     const CUtensorMapSwizzle tsw = (tbox * 2 == 64) ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
     if (!make_map(&m.K, p.K, hk, p.T, kD, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
     if (!make_map(&m.V, p.V, hv, p.T, kD, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
@@ -927,6 +1071,7 @@ int launch_tc_bf16(const Problem& p, InverseMode mode, cudaStream_t stream) {
         switch (p.C) {
             case 16: return launch_c<16, INV_NEUMANN>(m, prm, stream);
             case 32: return launch_c<32, INV_NEUMANN>(m, prm, stream);
+            case 128: return launch_c<64, INV_NEUMANN, true>(m, prm, stream);
             default: return launch_c<64, INV_NEUMANN>(m, prm, stream);
         }
     }

@@ -98,6 +98,15 @@ def test_bf16_other_orders_and_steps(C, N, S):
     _check(inp, TOL_BF16, N, S)
 
 
+@pytest.mark.parametrize("N,S", [(-1, -1), (3, 2), (2, 4)])
+def test_bf16_chunk_128_block_merge(N, S):
+    """C = 128: two 64-blocks by the scheme plus the block formula of App. E for the lower-left block."""
+    inp = gen.make_inputs(2, 2, 4, 512, 128, 128, 128, seed=45 + N + S)
+    _check(inp, TOL_BF16, N, S)
+    inp = gen.make_inputs(1, 1, 2, 128, 128, 128, 128, seed=46)
+    _check(inp, TOL_BF16, N, S)
+
+
 def test_bf16_truncation_is_honoured():
     """With few residual terms the truncated result differs visibly from the exact inverse;
     the kernel must reproduce the truncated one."""
