@@ -173,6 +173,19 @@ def device_time_steps(fn, steps: int, warmup: int, dist_ctx):
     return total_ms, per
 
 
+def max_over_ranks(total_ms: float, device, dist_ctx) -> float:
+    """The slowest rank's device time counts (all-reduce MAX; identity on one rank)."""
+    t = torch.tensor([total_ms], dtype=torch.float64, device=device)
+    if dist_ctx is not None:
+        dist_ctx.all_reduce(t, op=dist_ctx.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_throughput(chunks_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Every rank processes its own shard of `chunks_per_rank` chunks per step (weak scaling, no exchange)."""
+    return world * chunks_per_rank / (ms_per_step * 1e-3)
+
+
 def run_ours(args, rank, world, dist_ctx):
     from paper_2606_06034_b200 import binding as gdn
     from paper_2606_06034_b200 import inputs as gen
@@ -201,13 +214,9 @@ def run_ours(args, rank, world, dist_ctx):
     if status != gdn.GDN_OK:
         raise RuntimeError(f"kernel status {status}")
 
-    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-    if dist_ctx is not None:
-        import torch.distributed as dist
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, dev, dist_ctx)
     ms_per_step = total_ms / args.steps
-    value = world * n_chunks / (ms_per_step * 1e-3)
+    value = whole_job_throughput(n_chunks, world, ms_per_step)
 
     bytes_chunk = algorithmic_bytes_per_chunk(C, inp.d_k, inp.d_v, group)
     flops_chunk = nominal_flops_per_chunk(C, inp.d_k, inp.d_v)
@@ -272,7 +281,8 @@ def run_extras(gdn, gen, dev, args):
     """Other workloads and the forward-substitution comparison, timed the same way (not the headline)."""
     out = {}
     hbm_peak, _, _ = measured_peaks()
-    plan = [("sweep_c16", "neumann"), ("sweep_c32", "neumann"), ("sweep_c64", "neumann"), ("sweep_c64", "fwdsubst"),
+    plan = [("sweep_c16", "neumann"), ("sweep_c32", "neumann"), ("sweep_c64", "neumann"), ("sweep_c128", "neumann"),
+            ("sweep_c64", "fwdsubst"),
             ("sweep_c32", "fwdsubst"), ("sweep_c16", "fwdsubst"), ("prefill_gqa", "neumann")]
     for name, method in plan:
         try:
@@ -308,7 +318,7 @@ def run_extras(gdn, gen, dev, args):
 def run_reference(args):
     """The base contract's reference arm: the CPU oracle, as it stands, on the host cores."""
     steps, warm = args.steps, args.warmup
-    budget_per_step = max(0.2, min(10.0, 120.0 / max(1, steps + warm)))
+    budget_per_step = max(0.2, min(10.0, args.cpu_seconds, 120.0 / max(1, steps + warm)))
     vals = []
     info = None
     for i in range(warm + steps):
