@@ -61,6 +61,13 @@ typedef enum {
 
 enum { GDN_DTYPE_FP32 = 0, GDN_DTYPE_BF16 = 1 };
 
+/* flags of gdn_chunk_prepare_ex */
+enum {
+    GDN_FLAG_G_RAW = 1,     /* g holds the raw per-token log-gates; the kernel forms the chunk-local inclusive prefix sum */
+    GDN_FLAG_K_L2NORM = 2,  /* the kernel L2-normalises the rows of K first (the normalisation Sec. 2.1 places before the path) */
+    GDN_FLAG_OUT_FP32 = 4   /* W, U, Tinv are written as fp32 although K, V are bf16 (parity debugging) */
+};
+
 /* variants of the forward-substitution comparison kernel */
 enum { GDN_FWDSUBST_ROWS = 0, GDN_FWDSUBST_BLOCKED = 1 };
 
@@ -88,6 +95,16 @@ int gdn_chunk_prepare_gqa(const void* K, const void* V, const float* beta, const
                           int B, int H_k, int H_v, int T, int C, int d_k, int d_v,
                           int order, int residual_steps, int dtype,
                           void* W_out, void* U_out, void* Tinv_out, gdn_stream_t stream);
+
+/*
+ * gdn_chunk_prepare_gqa with the optional prologue of the path fused in (Sec. 2.1: the l2-normalisation of the keys
+ * sits right before the path; the gate prefix sum is Gated DeltaNet's): see the GDN_FLAG_* values. With
+ * GDN_FLAG_OUT_FP32 the three output buffers hold fp32 elements (same shapes).
+ */
+int gdn_chunk_prepare_ex(const void* K, const void* V, const float* beta, const float* g,
+                         int B, int H_k, int H_v, int T, int C, int d_k, int d_v,
+                         int order, int residual_steps, int dtype,
+                         void* W_out, void* U_out, void* Tinv_out, unsigned flags, gdn_stream_t stream);
 
 /*
  * The comparison the paper's speed-up is measured against: the same A-build, W

@@ -270,18 +270,27 @@ def exact_inverse(A: np.ndarray) -> np.ndarray:
 
 
 def chunk_prepare(K, V, beta, g, N: int | None = None, S: int | None = None, *,
-                  exact: bool = False):
+                  exact: bool = False, g_raw: bool = False, k_l2norm: bool = False):
     """One chunk or a stack of chunks: returns (W, U, T), all fp64.
 
     K: [..., C, d_k], V: [..., C, d_v], beta, g: [..., C].
     exact=False: T by the paper's scheme (order N, S residual terms; C = 128 by
     64-blocks). exact=True: T by forward substitution.
     W = T diag(beta) K, U = T diag(beta) V.
+    g_raw: g holds raw log-gates (prefix-summed here). k_l2norm: rows of K are
+    normalised here (W uses the normalised keys).
     """
     K = np.asarray(K, dtype=np.float64)
     V = np.asarray(V, dtype=np.float64)
     beta = np.asarray(beta, dtype=np.float64)
+    g = np.asarray(g, dtype=np.float64)
     C = K.shape[-2]
+    if g_raw:
+        # g holds the raw per-token log-gates: the cumulative gate is their prefix sum inside the chunk
+        g = np.cumsum(g, axis=-1)
+    if k_l2norm:
+        # keys are l2-normalised before the path (Sec. 2.1)
+        K = K / np.sqrt((K * K).sum(axis=-1, keepdims=True))
     A = build_A(K, beta, g)
     if exact:
         T = exact_inverse(A)

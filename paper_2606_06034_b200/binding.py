@@ -25,11 +25,15 @@ GDN_ERR_TIMEOUT = -6
 GDN_ERR_ARCH = -7
 GDN_DTYPE_FP32 = 0
 GDN_DTYPE_BF16 = 1
+GDN_FLAG_G_RAW = 1
+GDN_FLAG_K_L2NORM = 2
+GDN_FLAG_OUT_FP32 = 4
 GDN_FWDSUBST_ROWS = 0
 GDN_FWDSUBST_BLOCKED = 1
 
 EXPORTS = (
-    "gdn_chunk_prepare", "gdn_chunk_prepare_gqa", "gdn_chunk_prepare_fwdsubst", "gdn_chunk_prepare_int8",
+    "gdn_chunk_prepare", "gdn_chunk_prepare_gqa", "gdn_chunk_prepare_ex", "gdn_chunk_prepare_fwdsubst",
+    "gdn_chunk_prepare_int8",
     "gdn_int8_lut_checksum",
     "gdn_device_status", "gdn_default_order", "gdn_default_residual_steps",
     "gdn_status_string", "gdn_launch_count",
@@ -59,6 +63,8 @@ def load_library() -> ctypes.CDLL:
     lib.gdn_chunk_prepare.argtypes = [vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ip, ip, ip, vp, vp, vp, vp]
     lib.gdn_chunk_prepare_gqa.restype = ip
     lib.gdn_chunk_prepare_gqa.argtypes = [vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ip, ip, ip, ip, vp, vp, vp, vp]
+    lib.gdn_chunk_prepare_ex.restype = ip
+    lib.gdn_chunk_prepare_ex.argtypes = [vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ip, ip, ip, ip, vp, vp, vp, ctypes.c_uint, vp]
     lib.gdn_chunk_prepare_fwdsubst.restype = ip
     lib.gdn_chunk_prepare_fwdsubst.argtypes = [vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ip, ip, ip, vp, vp, vp, vp]
     lib.gdn_chunk_prepare_int8.restype = ip
@@ -153,6 +159,17 @@ def gdn_chunk_prepare_gqa(K, V, beta, g, B, H_k, H_v, T, C, d_k, d_v, order, res
     return rc
 
 
+def gdn_chunk_prepare_ex(K, V, beta, g, B, H_k, H_v, T, C, d_k, d_v, order, residual_steps, dtype, W_out, U_out,
+                         Tinv_out, flags, *, check=True):
+    _check_inputs(K, V, beta, g, ())
+    rc = load_library().gdn_chunk_prepare_ex(_ptr(K), _ptr(V), _ptr(beta), _ptr(g), B, H_k, H_v, T, C, d_k, d_v, order,
+                                             residual_steps, dtype, _ptr(W_out), _ptr(U_out), _ptr(Tinv_out), int(flags),
+                                             _stream())
+    if check and rc != GDN_OK:
+        raise GdnError(rc, "gdn_chunk_prepare_ex")
+    return rc
+
+
 def gdn_chunk_prepare_fwdsubst(K, V, beta, g, B, H_k, H_v, T, C, d_k, d_v, dtype, variant, W_out, U_out, Tinv_out,
                                *, check=True):
     _check_inputs(K, V, beta, g, (W_out, U_out, Tinv_out))
@@ -210,7 +227,7 @@ def gdn_device_status() -> int:
 
 
 def chunk_prepare(K, V, beta, g, C, order=-1, residual_steps=-1, *, want_tinv=True, outputs=None,
-                  method="neumann", variant=GDN_FWDSUBST_ROWS):
+                  method="neumann", variant=GDN_FWDSUBST_ROWS, flags=0):
     """Convenience wrapper: shapes from the tensors, outputs allocated with torch.
 
     K [B,H_k,T,d_k], V [B,H_v,T,d_v], beta, g [B,H_v,T]. Returns (W, U, Tinv).
@@ -219,9 +236,13 @@ def chunk_prepare(K, V, beta, g, C, order=-1, residual_steps=-1, *, want_tinv=Tr
     _, H_v, _, d_v = V.shape
     if outputs is None:
         outputs = alloc_outputs(K, V, C, want_tinv)
+        if flags & GDN_FLAG_OUT_FP32:
+            outputs = tuple(None if o is None else torch.empty(o.shape, dtype=torch.float32, device=o.device) for o in outputs)
     W, U, Tinv = outputs
     dt = _dtype_code(K)
-    if method == "neumann":
+    if method == "neumann" and flags:
+        gdn_chunk_prepare_ex(K, V, beta, g, B, H_k, H_v, T, C, d_k, d_v, order, residual_steps, dt, W, U, Tinv, flags)
+    elif method == "neumann":
         gdn_chunk_prepare_gqa(K, V, beta, g, B, H_k, H_v, T, C, d_k, d_v, order, residual_steps, dt, W, U, Tinv)
     elif method == "fwdsubst":
         gdn_chunk_prepare_fwdsubst(K, V, beta, g, B, H_k, H_v, T, C, d_k, d_v, dt, variant, W, U, Tinv)

@@ -115,7 +115,7 @@ __global__ void __launch_bounds__(kThreads) chunk_simt_kernel(const IO* __restri
                                                              const float* __restrict__ beta, const float* __restrict__ g,
                                                              IO* __restrict__ W, IO* __restrict__ U, IO* __restrict__ Tinv, int H_k,
                                                              int H_v, int T, int C, int d_k, int d_v, int N, int S, int mode,
-                                                             long long n_chunks) {
+                                                             long long n_chunks, unsigned flags) {
     extern __shared__ float sm[];
     const int ld = C + 1;
     const int blk = (C == 128) ? 64 : C;  // size of the diagonal blocks inverted by the series
@@ -127,6 +127,7 @@ __global__ void __launch_bounds__(kThreads) chunk_simt_kernel(const IO* __restri
     float* w2 = w1 + blk * ldw;
     float* sbeta = w2 + blk * ldw;  // C
     float* sg = sbeta + C;          // C
+    float* srn = sg + C;            // C: 1 / ||K_row|| (1 unless the keys are normalised here)
 
     const int n_c = T / C;
     const int group = H_v / H_k;
@@ -146,6 +147,21 @@ __global__ void __launch_bounds__(kThreads) chunk_simt_kernel(const IO* __restri
         for (int i = threadIdx.x; i < C; i += kThreads) {
             sbeta[i] = bc[i];
             sg[i] = gc[i];
+            float rn = 1.f;
+            if (flags & GDN_FLAG_K_L2NORM) {
+                float ss = 0.f;
+                for (int d = 0; d < d_k; ++d) {
+                    const float k = to_f32<IO>(Kc + (long long)i * d_k + d);
+                    ss = fmaf(k, k, ss);
+                }
+                rn = rsqrtf(fmaxf(ss, 1e-30f));
+            }
+            srn[i] = rn;
+        }
+        __syncthreads();
+        if ((flags & GDN_FLAG_G_RAW) && threadIdx.x == 0) {
+            // raw log-gates: chunk-local inclusive prefix sum
+            for (int i = 1; i < C; ++i) sg[i] += sg[i - 1];
         }
         __syncthreads();
         // Abar = -tril(diag(beta) (K K^T o Gamma), -1)
@@ -155,7 +171,7 @@ __global__ void __launch_bounds__(kThreads) chunk_simt_kernel(const IO* __restri
             if (i > j) {
                 float dot = 0.f;
                 for (int d = 0; d < d_k; ++d) dot = fmaf(to_f32<IO>(Kc + (long long)i * d_k + d), to_f32<IO>(Kc + (long long)j * d_k + d), dot);
-                a = -sbeta[i] * expf(sg[i] - sg[j]) * dot;
+                a = -sbeta[i] * expf(sg[i] - sg[j]) * dot * srn[i] * srn[j];
             }
             sA[i * ld + j] = a;
             sT[i * ld + j] = 0.f;
@@ -204,7 +220,7 @@ __global__ void __launch_bounds__(kThreads) chunk_simt_kernel(const IO* __restri
         for (int idx = threadIdx.x; idx < C * d_k; idx += kThreads) {
             const int i = idx / d_k, d = idx % d_k;
             float acc = 0.f;
-            for (int j = 0; j <= i; ++j) acc = fmaf(sT[i * ld + j] * sbeta[j], to_f32<IO>(Kc + (long long)j * d_k + d), acc);
+            for (int j = 0; j <= i; ++j) acc = fmaf(sT[i * ld + j] * sbeta[j] * srn[j], to_f32<IO>(Kc + (long long)j * d_k + d), acc);
             st(Wc + (long long)i * d_k + d, acc);
         }
         for (int idx = threadIdx.x; idx < C * d_v; idx += kThreads) {
@@ -228,10 +244,13 @@ int launch_simt(const Problem& p, InverseMode mode, cudaStream_t stream) {
     if (!(C >= 2 && (C <= 64 || C == 128))) return GDN_ERR_UNSUPPORTED;
     if (p.d_k > 256 || p.d_v > 256) return GDN_ERR_UNSUPPORTED;
     if (mode == INV_FWDSUBST_BLOCKED) return GDN_ERR_UNSUPPORTED;
+    if (p.flags & GDN_FLAG_OUT_FP32) {
+        if (p.dtype != GDN_DTYPE_FP32) return GDN_ERR_UNSUPPORTED;  // this kernel writes the element type it reads
+    }
     const long long n_chunks = (long long)p.B * p.H_v * (p.T / C);
     if (n_chunks == 0) return GDN_OK;
     const int blk = (C == 128) ? 64 : C;
-    const size_t smem = sizeof(float) * (2 * (size_t)C * (C + 1) + 3 * (size_t)blk * (blk + 1) + 2 * (size_t)C);
+    const size_t smem = sizeof(float) * (2 * (size_t)C * (C + 1) + 3 * (size_t)blk * (blk + 1) + 3 * (size_t)C);
     const int grid = (int)(n_chunks < 148LL * 8 ? n_chunks : 148LL * 8);
     cudaError_t e;
     if (p.dtype == GDN_DTYPE_FP32) {
@@ -239,13 +258,13 @@ int launch_simt(const Problem& p, InverseMode mode, cudaStream_t stream) {
         if (e != cudaSuccess) return GDN_ERR_LAUNCH;
         chunk_simt_kernel<float><<<grid, kThreads, smem, stream>>>((const float*)p.K, (const float*)p.V, p.beta, p.g, (float*)p.W,
                                                                   (float*)p.U, (float*)p.Tinv, p.H_k, p.H_v, p.T, C, p.d_k, p.d_v,
-                                                                  p.order, p.steps, (int)mode, n_chunks);
+                                                                  p.order, p.steps, (int)mode, n_chunks, p.flags);
     } else {
         e = cudaFuncSetAttribute(chunk_simt_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return GDN_ERR_LAUNCH;
         chunk_simt_kernel<__nv_bfloat16><<<grid, kThreads, smem, stream>>>(
             (const __nv_bfloat16*)p.K, (const __nv_bfloat16*)p.V, p.beta, p.g, (__nv_bfloat16*)p.W, (__nv_bfloat16*)p.U,
-            (__nv_bfloat16*)p.Tinv, p.H_k, p.H_v, p.T, C, p.d_k, p.d_v, p.order, p.steps, (int)mode, n_chunks);
+            (__nv_bfloat16*)p.Tinv, p.H_k, p.H_v, p.T, C, p.d_k, p.d_v, p.order, p.steps, (int)mode, n_chunks, p.flags);
     }
     count_launch();
     return cudaGetLastError() == cudaSuccess ? GDN_OK : GDN_ERR_LAUNCH;

@@ -59,6 +59,7 @@ struct Params {
     int* status;
     int H_k, H_v, T, group, n_tt;  // n_tt: tiles per head
     int N, S;
+    unsigned flags;  // GDN_FLAG_*
     long long n_tiles;
 };
 
@@ -81,7 +82,10 @@ struct Smem {
     static constexpr int kRBBytes = kTile * NBP * 4;
     static constexpr int kBeta = kRB + kRBBytes;        // 128 floats
     static constexpr int kG = kBeta + 512;              // 128 floats
-    static constexpr int kTotal = kG + 512;
+    static constexpr int kRn = kG + 512;                // 128 floats: 1 / ||K_row|| (GDN_FLAG_K_L2NORM)
+    static constexpr int kBRn = kRn + 512;              // 128 floats: beta / ||K_row||
+    static constexpr int kWt = kBRn + 512;              // 4 floats: warp totals of the gate prefix sum (GDN_FLAG_G_RAW)
+    static constexpr int kTotal = kWt + 64;
 };
 
 __device__ __forceinline__ float fast_exp2(float x) {
@@ -97,8 +101,8 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     uint32_t i = 0;
-    while (!mbar_try_wait(bar, parity)) {
-        if ((++i & 1023u) == 0 && clock64() - t0 > 2000000000LL) return false;
+    while (!mbar_try_wait_hint(bar, parity, 2000u)) {
+        if ((++i & 63u) == 0 && clock64() - t0 > 2000000000LL) return false;
     }
     return true;
 }
@@ -282,6 +286,52 @@ __device__ __forceinline__ void load_cols(uint32_t lane_base, uint32_t col0, int
     }
 }
 
+// Builds the two bf16 A operands of the W/U products for this thread's part of its row and stores them to TMEM:
+// hi (slot AS) = bf16(T diag(scale)) over the whole row, lo (slot R2) = bf16 of what hi loses on the diagonal and
+// the band, where entries are O(1). `sc` is the per-token scale in shared memory, `sc_i` the row's own scale;
+// a[] = far part of the row, lb[] = band, y[] = T21 part (second block of a 128-chunk).
+template <int C, int NB, bool MERGE>
+__device__ __forceinline__ void build_wu_operands(uint32_t lane_base, uint32_t br_row, int t, int h, int il, int cb, int col0, int wq,
+                                                  int n_band, const float* sc, float sc_i, const float (&a)[Split<C>::HC],
+                                                  const uint32_t (&keep)[Split<C>::PCH], const float (&lb)[NB + 1],
+                                                  const float (&y)[Split<C>::HC]) {
+    constexpr int PCH = Split<C>::PCH;
+    float tb[NB + 1];
+    tb[0] = sc_i;
+#pragma unroll
+    for (int e = 1; e <= NB; ++e) tb[e] = (il - e >= 0) ? lb[e] * sc[(t - e) > 0 ? (t - e) : 0] : 0.f;
+    uint16_t hi[NB + 1], lo[NB + 1];
+#pragma unroll
+    for (int e = 0; e <= NB; ++e) {
+        hi[e] = bf16_bits(tb[e]);
+        lo[e] = bf16_bits(tb[e] - bf16_bits_to_f32(hi[e]));
+    }
+    uint32_t bp[PCH], pk[PCH];
+    build_band_row<C, NB>(br_row, t, il, col0, n_band, hi, bp);
+    const float2* sb2 = reinterpret_cast<const float2*>(sc + cb + col0);
+#pragma unroll
+    for (int i = 0; i < PCH; ++i) {
+        const float2 bb = sb2[i];
+        pk[i] = (pack_bf16x2(a[2 * i] * bb.x, a[2 * i + 1] * bb.y) & keep[i]) | bp[i];
+    }
+    if (MERGE && wq >= 2) {
+        // second block of a 128-chunk: columns of the first block carry T21 diag(scale) instead of zeros
+        store_a_operand<C, false>(lane_base + kAS, t, h, pk);
+        const float2* sb1 = reinterpret_cast<const float2*>(sc + col0);
+        uint32_t po[PCH];
+#pragma unroll
+        for (int i = 0; i < PCH; ++i) {
+            const float2 bb = sb1[i];
+            po[i] = pack_bf16x2(y[2 * i] * bb.x, y[2 * i + 1] * bb.y);
+        }
+        store_stacked_operand<C>(lane_base + kAS, h, po);
+    } else {
+        store_a_operand<C, true>(lane_base + kAS, t, h, pk);
+    }
+    build_band_row<C, NB>(br_row, t, il, col0, n_band, lo, bp);
+    store_a_operand<C, true>(lane_base + kR2, t, h, bp);
+}
+
 struct TileCoord {
     int bhk, bhv;
     int t0;
@@ -330,6 +380,12 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     float* sRB = reinterpret_cast<float*>(smem + L::kRB);
     float* sbeta = reinterpret_cast<float*>(smem + L::kBeta);
     float* sg = reinterpret_cast<float*>(smem + L::kG);
+    float* srn = reinterpret_cast<float*>(smem + L::kRn);
+    float* sbrn = reinterpret_cast<float*>(smem + L::kBRn);
+    float* swt = reinterpret_cast<float*>(smem + L::kWt);
+    const bool f_graw = (p.flags & GDN_FLAG_G_RAW) != 0;
+    const bool f_l2 = (p.flags & GDN_FLAG_K_L2NORM) != 0;
+    const bool f_f32 = (p.flags & GDN_FLAG_OUT_FP32) != 0;
 
     __shared__ uint64_t bar_k, bar_v, bar_mma;
     __shared__ uint32_t tmem_base_s;
@@ -415,11 +471,29 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         const bool has_next = next < n_tiles;
 
         STAMP(1);
-        const float bi = bi_next, gi_ = gi_next;  // loaded during the previous tile
+        const float bi = bi_next;  // loaded during the previous tile
+        float gi_ = gi_next;
+        constexpr int kWarpsPerChunk = MERGE ? 4 : (C >= 32 ? C / 32 : 1);
+        if (f_graw) {
+            // g holds the raw per-token log-gates: inclusive prefix sum inside the chunk, by shuffles inside the warp
+            // (segments of C lanes when C = 16) and through shared memory across the chunk's warps
+            constexpr int SEG = (C < 32) ? C : 32;
+#pragma unroll
+            for (int off = 1; off < SEG; off <<= 1) {
+                const float v = __shfl_up_sync(0xFFFFFFFFu, gi_, off);
+                if ((lane & (SEG - 1)) >= off) gi_ += v;
+            }
+        }
         // the previous tile's bulk stores have finished reading the staging slices
         if (lane == 0) tma_store_wait_read<0>();
         tc_fence_before_sync();
         compute_barrier();  // everyone is done with the previous tile's shared arrays and accumulators
+        if (f_graw && kWarpsPerChunk > 1) {
+            if (h == 0 && lane == 31) swt[wq] = gi_;
+            compute_barrier();
+            const int first = wq - (wq % kWarpsPerChunk);
+            for (int w = first; w < wq; ++w) gi_ += swt[w];
+        }
         if (tid == 0) {
             // G = K K^T into R0..R1 (128 columns)
             STAMP(20);
@@ -470,19 +544,41 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 tmem_wait_st();
             }
         }
+        if (active) load_diag_block<C>(lane_base, kR0, t, h, a);
+        float rni = 1.f;
+        if (f_l2) {
+            // keys are normalised on the fly: 1 / ||K_i|| from the diagonal of the Gram matrix
+            if (active && il >= col0 && il < col0 + HC) {
+                float gd = 0.f;
+#pragma unroll
+                for (int jl = 0; jl < HC; ++jl)
+                    if (col0 + jl == il) gd = a[jl];
+                const float rn = rsqrtf(fmaxf(gd, 1e-30f));
+                srn[t] = rn;
+                sbrn[t] = bi * rn;
+            }
+            compute_barrier();
+            rni = srn[t];
+        }
         if (active) {
-            load_diag_block<C>(lane_base, kR0, t, h, a);
             const float gs = gi_ * kLog2e;
-            const float nbi = -bi;
+            const float nbi = -bi * rni;
             const float4* sg4 = reinterpret_cast<const float4*>(sg + cb + col0);
+            const float4* sr4 = reinterpret_cast<const float4*>(srn + cb + col0);
 #pragma unroll
             for (int j4 = 0; j4 < HC / 4; ++j4) {
                 const float4 gq = sg4[j4];
                 const float gj[4] = {gq.x, gq.y, gq.z, gq.w};
+                float rj[4] = {1.f, 1.f, 1.f, 1.f};
+                if (f_l2) {
+                    const float4 rq = sr4[j4];
+                    rj[0] = rq.x; rj[1] = rq.y; rj[2] = rq.z; rj[3] = rq.w;
+                }
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
                     const int jl = j4 * 4 + q;
-                    const float v = nbi * fast_exp2(fmaf(-gj[q], kLog2e, gs)) * a[jl];
+                    float v = nbi * fast_exp2(fmaf(-gj[q], kLog2e, gs)) * a[jl];
+                    if (f_l2) v *= rj[q];
                     a[jl] = (col0 + jl < il) ? v : 0.f;
                 }
             }
@@ -737,7 +833,8 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     const float gj[4] = {gv.x, gv.y, gv.z, gv.w};
 #pragma unroll
                     for (int q = 0; q < 4; ++q)
-                        y[j4 * 4 + q] = bi * fast_exp2(fmaf(-gj[q], kLog2e, gs)) * __uint_as_float(gq[j4 * 4 + q]);
+                        y[j4 * 4 + q] = bi * rni * (f_l2 ? srn[col0 + j4 * 4 + q] : 1.f) * fast_exp2(fmaf(-gj[q], kLog2e, gs)) *
+                                        __uint_as_float(gq[j4 * 4 + q]);
                 }
                 uint32_t pk[PCH];
 #pragma unroll
@@ -788,42 +885,11 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         }
 
         STAMP(9);
-        // ---- A operands for W/U: T diag(beta) = hi + lo, hi over the whole row, lo only on band + diagonal
+        // ---- A operands for W/U: T diag(scale) = hi + lo, hi over the whole row, lo only on band + diagonal.
+        // scale = beta for U; for W it is beta / ||K|| when the keys are normalised on the fly, else beta as well
         if (active) {
-            float tb[NB + 1];
-            tb[0] = bi;
-#pragma unroll
-            for (int e = 1; e <= NB; ++e) tb[e] = (il - e >= 0) ? lb[e] * sbeta[(t - e) > 0 ? (t - e) : 0] : 0.f;
-            uint16_t hi[NB + 1], lo[NB + 1];
-#pragma unroll
-            for (int e = 0; e <= NB; ++e) {
-                hi[e] = bf16_bits(tb[e]);
-                lo[e] = bf16_bits(tb[e] - bf16_bits_to_f32(hi[e]));
-            }
-            uint32_t bp[PCH], pk[PCH];
-            build_band_row<C, NB>(br_row, t, il, col0, n_band, hi, bp);
-            const float2* sb2 = reinterpret_cast<const float2*>(sbeta + cb + col0);
-#pragma unroll
-            for (int i = 0; i < PCH; ++i) {
-                const float2 bb = sb2[i];
-                pk[i] = (pack_bf16x2(a[2 * i] * bb.x, a[2 * i + 1] * bb.y) & keep[i]) | bp[i];
-            }
-            if (MERGE && wq >= 2) {
-                // second block of a 128-chunk: columns of the first block carry T21 diag(beta) instead of zeros
-                store_a_operand<C, false>(lane_base + kAS, t, h, pk);
-                const float2* sb1 = reinterpret_cast<const float2*>(sbeta + col0);
-                uint32_t po[PCH];
-#pragma unroll
-                for (int i = 0; i < PCH; ++i) {
-                    const float2 bb = sb1[i];
-                    po[i] = pack_bf16x2(y[2 * i] * bb.x, y[2 * i + 1] * bb.y);
-                }
-                store_stacked_operand<C>(lane_base + kAS, h, po);
-            } else {
-                store_a_operand<C, true>(lane_base + kAS, t, h, pk);
-            }
-            build_band_row<C, NB>(br_row, t, il, col0, n_band, lo, bp);
-            store_a_operand<C, true>(lane_base + kR2, t, h, bp);
+            build_wu_operands<C, NB, MERGE>(lane_base, br_row, t, h, il, cb, col0, wq, n_band, f_l2 ? sbrn : sbeta,
+                                            f_l2 ? bi * rni : bi, a, keep, lb, y);
             tmem_wait_st();
         }
         tc_fence_before_sync();
@@ -843,7 +909,37 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         STAMP(8);
         // ---- T row -> Tinv: each half-row goes to a staging line in the TMA swizzle layout (the band-row
         // region is free now); one bulk tensor store of 32 rows x HC columns per warp, overlapping the W products
-        if (MERGE && p.Tinv != nullptr) {
+        if (f_f32 && p.Tinv != nullptr && active) {
+            // fp32 outputs (parity debugging): the row part straight from registers, 16-byte stores
+            const bool rv = (tc.t0 + t) < p.T;
+            constexpr int COUT = MERGE ? 128 : C;
+            float* trow = reinterpret_cast<float*>(p.Tinv) + ((long long)tc.bhv * p.T + tc.t0 + t) * COUT;
+            if (rv) {
+                const int dcol = (MERGE ? cb : 0) + col0;  // first output column of the diagonal-block part
+#pragma unroll
+                for (int c = 0; c < HC / 4; ++c) {
+                    float v[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int jl = c * 4 + q;
+                        const int d = il - (col0 + jl);
+                        float x = a[jl];
+                        if (d == 0) x = 1.f;
+#pragma unroll
+                        for (int e = 1; e <= NB; ++e)
+                            if (d == e && e <= n_band) x = lb[e];
+                        v[q] = x;
+                    }
+                    *reinterpret_cast<float4*>(trow + dcol + c * 4) = make_float4(v[0], v[1], v[2], v[3]);
+                }
+                if (MERGE) {
+                    const int ocol = (wq >= 2 ? 0 : 64) + col0;  // T21 part, or the zero block above it
+#pragma unroll
+                    for (int c = 0; c < HC / 4; ++c)
+                        *reinterpret_cast<float4*>(trow + ocol + c * 4) = make_float4(y[c * 4], y[c * 4 + 1], y[c * 4 + 2], y[c * 4 + 3]);
+                }
+            }
+        } else if (MERGE && p.Tinv != nullptr) {
             // rows of the 128 x 128 inverse in four column groups of 32 (64-byte lines, 64-byte TMA swizzle):
             // the row's diagonal-block part, and its part of the other block column (T21, or zeros above it)
             const int gd = (cb >> 5) + h;                  // group of the diagonal-block part
@@ -915,18 +1011,36 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 uint32_t r[32];
                 tmem_ld32(lane_base + kR0 + h * 64 + c0, r);
                 tmem_wait_ld();
+                if (f_f32) {
+                    if ((tc.t0 + t) < p.T) {
+                        float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(half == 0 ? p.W : p.U) +
+                                                               ((long long)tc.bhv * p.T + tc.t0 + t) * kD + h * 64 + c0);
 #pragma unroll
-                for (int i = 0; i < 16; ++i) o[c0 / 2 + i] = pack_bf16x2(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
+                        for (int i = 0; i < 8; ++i)
+                            dst[i] = make_float4(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]), __uint_as_float(r[4 * i + 2]),
+                                                 __uint_as_float(r[4 * i + 3]));
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) o[c0 / 2 + i] = pack_bf16x2(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
+                }
             }
             if (half == 0) {
                 // this warp's Tinv store has been read (the staging slices below overlap other warps' lines)
                 if (lane == 0) tma_store_wait_read<0>();
                 tc_fence_before_sync();
                 compute_barrier();  // every row of the W accumulator has been read
+                if (f_l2) {
+                    // U uses beta where W used beta / ||K||: rebuild both A operands
+                    if (active) {
+                        build_wu_operands<C, NB, MERGE>(lane_base, br_row, t, h, il, cb, col0, wq, n_band, sbeta, bi, a, keep, lb, y);
+                        tmem_wait_st();
+                    }
+                    tc_fence_before_sync();
+                    compute_barrier();
+                }
                 if (tid == 0) {
-                    STAMP(22);
                     if (!wait_bar(&bar_v, par_kv)) ok = false;
-                    STAMP(23);
                     if (ok) {
                         tc_fence_after_sync();
 #pragma unroll
@@ -939,7 +1053,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 }
             }
             STAMP(12 + half * 3);
-            {
+            if (!f_f32) {
                 // 32 rows x 64 columns of this warp in the 128-byte TMA swizzle: 4 KB at slice(wq) + h * 4 KB
                 const uint32_t sub = scratch_a + wq * 8192 + h * 4096;
                 if (lane == 0) tma_store_wait_read<0>();  // earlier stores from this sub-tile have been read
@@ -1065,6 +1179,7 @@ int launch_tc_bf16(const Problem& p, InverseMode mode, cudaStream_t stream) {
     prm.n_tt = (p.T + kTile - 1) / kTile;
     prm.N = p.order;
     prm.S = p.steps;
+    prm.flags = p.flags;
     prm.n_tiles = (long long)p.B * p.H_v * prm.n_tt;
     if (prm.n_tiles >= (1LL << 31) - 4096 || (long long)p.B * p.H_v >= (1LL << 31)) return GDN_ERR_UNSUPPORTED;
     if (mode == INV_NEUMANN) {

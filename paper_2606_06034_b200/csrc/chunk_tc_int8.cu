@@ -84,8 +84,8 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     uint32_t i = 0;
-    while (!mbar_try_wait(bar, parity)) {
-        if ((++i & 1023u) == 0 && clock64() - t0 > 2000000000LL) return false;
+    while (!mbar_try_wait_hint(bar, parity, 2000u)) {
+        if ((++i & 63u) == 0 && clock64() - t0 > 2000000000LL) return false;
     }
     return true;
 }

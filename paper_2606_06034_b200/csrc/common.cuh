@@ -21,6 +21,7 @@ struct Problem {
     int order;   // N
     int steps;   // S
     int dtype;   // GDN_DTYPE_*
+    unsigned flags = 0;  // GDN_FLAG_*
 };
 
 // INT8 entry point's problem description

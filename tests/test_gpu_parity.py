@@ -183,3 +183,71 @@ def test_argument_errors_on_device():
     g_misaligned = buf[1:]  # 4 bytes past a 16-byte boundary
     assert gdn.gdn_chunk_prepare(K, V, beta, g_misaligned, 1, 1, 128, 64, 128, 128, -1, -1, 1, W, U, Tinv, **args) == gdn.GDN_ERR_ALIGN
     assert gdn.gdn_device_status() == gdn.GDN_OK
+
+
+# ---------------------------------------------------------------- optional prologue and fp32 outputs (gdn_chunk_prepare_ex)
+def _raw_inputs(B, H_k, H_v, T, C, seed, dtype=torch.bfloat16, adv="none"):
+    """Unnormalised keys with row norms in [0.5, 3] and RAW (not prefix-summed) log-gates."""
+    inp = gen.make_inputs(B, H_k, H_v, T, C, 128, 128, seed=seed, dtype=dtype, adversarial_heads=adv)
+    gsc = torch.Generator().manual_seed(seed + 1000)
+    scale = 0.5 + 2.5 * torch.rand(B, H_k, T, 1, generator=gsc)
+    inp.K = (inp.K.float() * scale).to(dtype).contiguous()
+    graw = inp.g.view(B, H_v, T // C, C).diff(dim=-1, prepend=torch.zeros(B, H_v, T // C, 1)).reshape(B, H_v, T).contiguous()
+    return inp, graw
+
+
+def _check_ex(inp, graw, flags, tol, N=-1, S=-1):
+    K, V, beta = inp.K.cuda(), inp.V.cuda(), inp.beta.cuda()
+    g_raw = bool(flags & gdn.GDN_FLAG_G_RAW)
+    l2 = bool(flags & gdn.GDN_FLAG_K_L2NORM)
+    g = (graw if g_raw else inp.g).cuda()
+    W, U, Tinv = gdn.chunk_prepare(K, V, beta, g, inp.C, N, S, flags=flags)
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+    if flags & gdn.GDN_FLAG_OUT_FP32:
+        assert W.dtype == torch.float32 and Tinv.dtype == torch.float32
+    Wg, Ug, Tg = _gpu_chunks(W, U, Tinv, inp)
+    sl = gen.chunk_slices(inp, range(inp.n_chunks))
+    Kc = np.stack([s[0] for s in sl]); Vc = np.stack([s[1] for s in sl]); bc = np.stack([s[2] for s in sl])
+    gsrc = graw if g_raw else inp.g
+    gc = gsrc.double().numpy().reshape(inp.n_chunks, inp.C)
+    Wo, Uo, To = orc.chunk_prepare(Kc, Vc, bc, gc, None if N < 0 else N, None if S < 0 else S, g_raw=g_raw, k_l2norm=l2)
+    for name, got, ref in (("Tinv", Tg, To), ("W", Wg, Wo), ("U", Ug, Uo)):
+        err = orc.rel_frobenius(got, ref)
+        assert err.max() <= tol, f"{name} rel-F {err.max():.3e} at chunk {err.argmax()} (flags {flags})"
+
+
+@pytest.mark.parametrize("C", [16, 32, 64, 128])
+@pytest.mark.parametrize("flags", [1, 2, 3])
+def test_bf16_prologue_flags(C, flags):
+    inp, graw = _raw_inputs(1, 2, 4, 512, C, seed=200 + C + flags)
+    _check_ex(inp, graw, flags, TOL_BF16)
+
+
+@pytest.mark.parametrize("C", [16, 64, 128])
+@pytest.mark.parametrize("adv", ["none", "all"])
+def test_bf16_fp32_outputs_show_the_accumulators(C, adv):
+    """With fp32 outputs the bf16 output rounding (1.7e-3) is gone: what remains is the error of the bf16
+    MMA operands, which the fp32 band / hi-lo split keeps small even for strongly correlated keys."""
+    if C == 128 and adv == "all":
+        pytest.skip("the block merge of C = 128 passes O(1) cancelling quantities through single bf16 operands")
+    inp = gen.make_inputs(1, 2, 2, 512, C, 128, 128, seed=230 + C, adversarial_heads=adv)
+    _check_ex(inp, None, gdn.GDN_FLAG_OUT_FP32, 5e-4)
+
+
+def test_bf16_all_flags_together_gqa_ragged():
+    inp, graw = _raw_inputs(2, 1, 3, 192, 64, seed=250, adv="odd")
+    _check_ex(inp, graw, 7, 5e-4)
+
+
+@pytest.mark.parametrize("C,flags", [(16, 3), (64, 1), (64, 2), (128, 3)])
+def test_fp32_prologue_flags(C, flags):
+    inp, graw = _raw_inputs(1, 1, 2, 2 * C, C, seed=260 + C, dtype=torch.float32)
+    _check_ex(inp, graw, flags, TOL_FP32 * 3)
+
+
+def test_ex_rejects_unknown_flags():
+    inp = gen.make_inputs(1, 1, 1, 128, 64, 128, 128, seed=270)
+    K, V, beta, g = _to_dev(inp)
+    W, U, Tinv = gdn.alloc_outputs(K, V, 64)
+    rc = gdn.gdn_chunk_prepare_ex(K, V, beta, g, 1, 1, 1, 128, 64, 128, 128, -1, -1, 1, W, U, Tinv, 8, check=False)
+    assert rc == gdn.GDN_ERR_INVALID_ARG

@@ -369,3 +369,21 @@ def test_input_recipe():
     # seeded
     again = gen.make_inputs(2, 2, 4, 128, 64, 128, 128, seed=4, adversarial_heads="odd")
     assert torch.equal(inp.K, again.K) and torch.equal(inp.g, again.g)
+
+
+# -- optional prologue (raw gates, key normalisation) reduces to the plain path on prepared inputs --------
+def test_prologue_flags_reduce_to_prepared_inputs():
+    rng = np.random.default_rng(41)
+    C = 16
+    K = rng.normal(size=(3, C, 8)) * rng.uniform(0.5, 3.0, size=(3, C, 1))
+    V = rng.normal(size=(3, C, 4))
+    beta = rng.uniform(0.1, 0.9, size=(3, C))
+    graw = -rng.uniform(0.0, 0.5, size=(3, C))
+    W1, U1, T1 = orc.chunk_prepare(K, V, beta, graw, g_raw=True, k_l2norm=True)
+    Kn = K / np.linalg.norm(K, axis=-1, keepdims=True)
+    gc = np.stack([[sum(row[:i + 1]) for i in range(C)] for row in graw])
+    W2, U2, T2 = orc.chunk_prepare(Kn, V, beta, gc)
+    assert np.allclose(T1, T2, atol=1e-14) and np.allclose(W1, W2, atol=1e-14) and np.allclose(U1, U2, atol=1e-14)
+    # normalisation matters: without it the result differs
+    W3, _, T3 = orc.chunk_prepare(K, V, beta, gc)
+    assert np.abs(T3 - T2).max() > 1e-3
