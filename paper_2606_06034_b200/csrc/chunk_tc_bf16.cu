@@ -294,7 +294,7 @@ template <int C, int NB, bool MERGE>
 __device__ __forceinline__ void build_wu_operands(uint32_t lane_base, uint32_t br_row, int t, int h, int il, int cb, int col0, int wq,
                                                   int n_band, const float* sc, float sc_i, const float (&a)[Split<C>::HC],
                                                   const uint32_t (&keep)[Split<C>::PCH], const float (&lb)[NB + 1],
-                                                  const float (&y)[Split<C>::HC]) {
+                                                  const float (&y)[MERGE ? Split<C>::HC : 1]) {
     constexpr int PCH = Split<C>::PCH;
     float tb[NB + 1];
     tb[0] = sc_i;
@@ -314,20 +314,23 @@ __device__ __forceinline__ void build_wu_operands(uint32_t lane_base, uint32_t b
         const float2 bb = sb2[i];
         pk[i] = (pack_bf16x2(a[2 * i] * bb.x, a[2 * i + 1] * bb.y) & keep[i]) | bp[i];
     }
-    if (MERGE && wq >= 2) {
-        // second block of a 128-chunk: columns of the first block carry T21 diag(scale) instead of zeros
-        store_a_operand<C, false>(lane_base + kAS, t, h, pk);
-        const float2* sb1 = reinterpret_cast<const float2*>(sc + col0);
-        uint32_t po[PCH];
+    bool plain = true;
+    if constexpr (MERGE) {
+        if (wq >= 2) {
+            // second block of a 128-chunk: columns of the first block carry T21 diag(scale) instead of zeros
+            plain = false;
+            store_a_operand<C, false>(lane_base + kAS, t, h, pk);
+            const float2* sb1 = reinterpret_cast<const float2*>(sc + col0);
+            uint32_t po[PCH];
 #pragma unroll
-        for (int i = 0; i < PCH; ++i) {
-            const float2 bb = sb1[i];
-            po[i] = pack_bf16x2(y[2 * i] * bb.x, y[2 * i + 1] * bb.y);
+            for (int i = 0; i < PCH; ++i) {
+                const float2 bb = sb1[i];
+                po[i] = pack_bf16x2(y[2 * i] * bb.x, y[2 * i + 1] * bb.y);
+            }
+            store_stacked_operand<C>(lane_base + kAS, h, po);
         }
-        store_stacked_operand<C>(lane_base + kAS, h, po);
-    } else {
-        store_a_operand<C, true>(lane_base + kAS, t, h, pk);
     }
+    if (plain) store_a_operand<C, true>(lane_base + kAS, t, h, pk);
     build_band_row<C, NB>(br_row, t, il, col0, n_band, lo, bp);
     store_a_operand<C, true>(lane_base + kR2, t, h, bp);
 }
@@ -356,7 +359,8 @@ __device__ __forceinline__ TileCoord decode_tile(uint32_t tile, const Params& p)
 // (C = 64 is then the block size) and whose lower-left block follows from App. E, Eq. 28:
 // T21 = -T22 A21 T11, evaluated as Y = A21 + A21 X11, T21 = -(Y + X22 Y) with X = T - I of the blocks, so that
 // the identity parts stay in fp32 and only the small products pass through bf16 operands.
-template <int C, int NB, int MODE, bool MERGE>
+// EX: the optional prologue / fp32 outputs of gdn_chunk_prepare_ex are compiled in (flags read at run time).
+template <int C, int NB, int MODE, bool MERGE, bool EX>
 __global__ void __launch_bounds__(kThreads, 2)
 chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                 const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmU,
@@ -383,9 +387,9 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     float* srn = reinterpret_cast<float*>(smem + L::kRn);
     float* sbrn = reinterpret_cast<float*>(smem + L::kBRn);
     float* swt = reinterpret_cast<float*>(smem + L::kWt);
-    const bool f_graw = (p.flags & GDN_FLAG_G_RAW) != 0;
-    const bool f_l2 = (p.flags & GDN_FLAG_K_L2NORM) != 0;
-    const bool f_f32 = (p.flags & GDN_FLAG_OUT_FP32) != 0;
+    const bool f_graw = EX && (p.flags & GDN_FLAG_G_RAW) != 0;
+    const bool f_l2 = EX && (p.flags & GDN_FLAG_K_L2NORM) != 0;
+    const bool f_f32 = EX && (p.flags & GDN_FLAG_OUT_FP32) != 0;
 
     __shared__ uint64_t bar_k, bar_v, bar_mma;
     __shared__ uint32_t tmem_base_s;
@@ -797,9 +801,10 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         }
         // a[] = this thread's part of the far row (T - I - L)
 
-        float y[HC];  // MERGE, rows of the second block: A21 part, then Y, then T21 (columns of the first block)
+        constexpr int YN = MERGE ? HC : 1;
+        float y[YN];  // MERGE, rows of the second block: A21 part, then Y, then T21 (columns of the first block)
 #pragma unroll
-        for (int j = 0; j < HC; ++j) y[j] = 0.f;
+        for (int j = 0; j < YN; ++j) y[j] = 0.f;
         if constexpr (MERGE) {
             const uint32_t idesc_m = instr_desc(128, 64, 1, 1, 0, 1, 1);
             // X = T - I of the row's diagonal block as packed bf16 (band without the unit diagonal + far part)
@@ -932,7 +937,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     }
                     *reinterpret_cast<float4*>(trow + dcol + c * 4) = make_float4(v[0], v[1], v[2], v[3]);
                 }
-                if (MERGE) {
+                if constexpr (MERGE) {
                     const int ocol = (wq >= 2 ? 0 : 64) + col0;  // T21 part, or the zero block above it
 #pragma unroll
                     for (int c = 0; c < HC / 4; ++c)
@@ -940,6 +945,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 }
             }
         } else if (MERGE && p.Tinv != nullptr) {
+          if constexpr (MERGE) {
             // rows of the 128 x 128 inverse in four column groups of 32 (64-byte lines, 64-byte TMA swizzle):
             // the row's diagonal-block part, and its part of the other block column (T21, or zeros above it)
             const int gd = (cb >> 5) + h;                  // group of the diagonal-block part
@@ -963,6 +969,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 tma_store_3d(&tmT, smem + L::kEB + go * 8192 + wrow0 * 64, go * 32, tc.t0 + wrow0, tc.bhv);
                 tma_store_commit();
             }
+          }
         } else if (p.Tinv != nullptr && active) {
             constexpr int RB = HC * 2;  // bytes per staged half-row
             const uint32_t stage = smem_u32(smem + L::kBR) + h * (kTile * RB);
@@ -1118,16 +1125,22 @@ struct Maps {
     CUtensorMap K, V, W, U, T;
 };
 
-template <int C, int NB, int MODE, bool MERGE>
-int launch_one(const Maps& m, const Params& prm, cudaStream_t stream) {
+template <int C, int NB, int MODE, bool MERGE, bool EX>
+int launch_ex(const Maps& m, const Params& prm, cudaStream_t stream) {
     using L = Smem<C, NB>;
     const int smem = L::kTotal + 1024;
-    auto kern = chunk_tc_kernel<C, NB, MODE, MERGE>;
+    auto kern = chunk_tc_kernel<C, NB, MODE, MERGE, EX>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return GDN_ERR_LAUNCH;
     long long grid = prm.n_tiles < 2 * 148 ? prm.n_tiles : 2 * 148;
     kern<<<static_cast<int>(grid), kThreads, smem, stream>>>(m.K, m.V, m.W, m.U, m.T, prm);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? GDN_OK : GDN_ERR_LAUNCH;
+}
+
+template <int C, int NB, int MODE, bool MERGE>
+int launch_one(const Maps& m, const Params& prm, cudaStream_t stream) {
+    if (MODE == INV_NEUMANN && prm.flags != 0) return launch_ex<C, NB, MODE, MERGE, (MODE == INV_NEUMANN)>(m, prm, stream);
+    return launch_ex<C, NB, MODE, MERGE, false>(m, prm, stream);
 }
 
 template <int C, int MODE, bool MERGE = false>
