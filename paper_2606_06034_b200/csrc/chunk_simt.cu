@@ -203,6 +203,35 @@ __global__ void __launch_bounds__(kThreads) chunk_simt_kernel(const IO* __restri
                 }
                 __syncthreads();
             }
+        } else if (mode == INV_FWDSUBST_BLOCKED) {
+            // Blocked form (App. E): 16 x 16 diagonal blocks by substitution (Eq. 25), then block rows from
+            // S_ij = S_ii sum_{k<i} Abar_ik S_kj (Eq. 27 with T_ik = -Abar_ik); thread j owns column j.
+            for (int j = threadIdx.x; j < C; j += kThreads) {
+                const int bend = (j / 16 + 1) * 16;
+                for (int i = j + 1; i < bend; ++i) {
+                    float acc = sA[i * ld + j];
+                    for (int k = j + 1; k < i; ++k) acc = fmaf(sA[i * ld + k], sT[k * ld + j], acc);
+                    sT[i * ld + j] = acc;
+                }
+                sT[j * ld + j] = 1.f;
+            }
+            __syncthreads();
+            for (int j = threadIdx.x; j < C; j += kThreads) {
+                for (int bi = j / 16 + 1; bi < C / 16; ++bi) {
+                    float tmp[16];
+                    for (int r = 0; r < 16; ++r) {
+                        float acc = 0.f;
+                        for (int k = j; k < bi * 16; ++k) acc = fmaf(sA[(bi * 16 + r) * ld + k], sT[k * ld + j], acc);
+                        tmp[r] = acc;
+                    }
+                    for (int r = 0; r < 16; ++r) {
+                        float acc = 0.f;
+                        for (int q = 0; q <= r; ++q) acc = fmaf(sT[(bi * 16 + r) * ld + bi * 16 + q], tmp[q], acc);
+                        sT[(bi * 16 + r) * ld + j] = acc;
+                    }
+                }
+            }
+            __syncthreads();
         } else {
             // Forward substitution (Eq. 2-3): row i of X = Abar_i + Abar_{i,0:i} X_{0:i,:}; thread j owns column j.
             for (int j = threadIdx.x; j < C; j += kThreads) {
@@ -243,7 +272,7 @@ int launch_simt(const Problem& p, InverseMode mode, cudaStream_t stream) {
     const int C = p.C;
     if (!(C >= 2 && (C <= 64 || C == 128))) return GDN_ERR_UNSUPPORTED;
     if (p.d_k > 256 || p.d_v > 256) return GDN_ERR_UNSUPPORTED;
-    if (mode == INV_FWDSUBST_BLOCKED) return GDN_ERR_UNSUPPORTED;
+    if (mode == INV_FWDSUBST_BLOCKED && C % 16 != 0) return GDN_ERR_UNSUPPORTED;
     if (p.flags & GDN_FLAG_OUT_FP32) {
         if (p.dtype != GDN_DTYPE_FP32) return GDN_ERR_UNSUPPORTED;  // this kernel writes the element type it reads
     }

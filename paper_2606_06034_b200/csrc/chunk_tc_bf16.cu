@@ -694,19 +694,72 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             // column il of its chunk, which has no dependence on other columns.
             if (h == 0) {
                 float xcol[C];  // xcol[k] = T[k][il]
+                if constexpr (MODE == INV_FWDSUBST_BLOCKED) {
+                    // Blocked form (App. E): the 16 x 16 diagonal blocks are inverted by substitution independently
+                    // (Eq. 25), then block row bi follows from S_ij = S_ii sum_{k<i} Abar_ik S_kj (Eq. 27 with
+                    // T_ik = -Abar_ik). The inverted diagonal blocks go through shared memory (strictly lower
+                    // parts, 120 floats per block) because a column's thread needs the blocks of other columns.
+                    float* sDi = sSH;  // [8 blocks of the tile][120]; the band arrays are unused in this mode
+                    const int b0 = il >> 4, c16 = il & 15;
 #pragma unroll
-                for (int i = 0; i < C; ++i) {
-                    float acc = 0.f;
-                    const uint32_t ri = scratch_a + (cb + i) * (4 * C);
+                    for (int i = 0; i < C; ++i) {
+                        float acc = 0.f;
+                        const uint32_t ri = scratch_a + (cb + i) * (4 * C);
 #pragma unroll
-                    for (int k4 = 0; k4 < (i + 3) / 4; ++k4) {
-                        const uint4 q = lds128(ri + (swz<CPRF>(i, k4) << 4));  // (cb + i) and i agree in the swizzle bits
-                        if (k4 * 4 + 0 < i) acc = fmaf(__uint_as_float(q.x), xcol[k4 * 4 + 0], acc);
-                        if (k4 * 4 + 1 < i) acc = fmaf(__uint_as_float(q.y), xcol[(k4 * 4 + 1 < C) ? k4 * 4 + 1 : 0], acc);
-                        if (k4 * 4 + 2 < i) acc = fmaf(__uint_as_float(q.z), xcol[(k4 * 4 + 2 < C) ? k4 * 4 + 2 : 0], acc);
-                        if (k4 * 4 + 3 < i) acc = fmaf(__uint_as_float(q.w), xcol[(k4 * 4 + 3 < C) ? k4 * 4 + 3 : 0], acc);
+                        for (int k4 = (i & ~15) / 4; k4 < (i + 3) / 4; ++k4) {
+                            const uint4 q = lds128(ri + (swz<CPRF>(i, k4) << 4));
+                            if (k4 * 4 + 0 < i) acc = fmaf(__uint_as_float(q.x), xcol[k4 * 4 + 0], acc);
+                            if (k4 * 4 + 1 < i) acc = fmaf(__uint_as_float(q.y), xcol[(k4 * 4 + 1 < C) ? k4 * 4 + 1 : 0], acc);
+                            if (k4 * 4 + 2 < i) acc = fmaf(__uint_as_float(q.z), xcol[(k4 * 4 + 2 < C) ? k4 * 4 + 2 : 0], acc);
+                            if (k4 * 4 + 3 < i) acc = fmaf(__uint_as_float(q.w), xcol[(k4 * 4 + 3 < C) ? k4 * 4 + 3 : 0], acc);
+                        }
+                        xcol[i] = ((i >> 4) == b0 && i > il) ? acc : ((i == il) ? 1.f : 0.f);
+                        if ((i >> 4) == b0 && (i & 15) > c16)
+                            sDi[((cb >> 4) + (i >> 4)) * 120 + ((i & 15) * ((i & 15) - 1)) / 2 + c16] = xcol[i];
                     }
-                    xcol[i] = (i > il) ? acc : ((i == il) ? 1.f : 0.f);
+                    compute_barrier();  // the inverted diagonal blocks are published
+#pragma unroll
+                    for (int bi = 1; bi < C / 16; ++bi) {
+                        float tmp[16];
+#pragma unroll
+                        for (int r = 0; r < 16; ++r) {
+                            float acc = 0.f;
+                            const int i = bi * 16 + r;
+                            const uint32_t ri = scratch_a + (cb + i) * (4 * C);
+#pragma unroll
+                            for (int k4 = 0; k4 < bi * 4; ++k4) {
+                                const uint4 q = lds128(ri + (swz<CPRF>(i, k4) << 4));
+                                acc = fmaf(__uint_as_float(q.x), xcol[k4 * 4 + 0], acc);
+                                acc = fmaf(__uint_as_float(q.y), xcol[k4 * 4 + 1], acc);
+                                acc = fmaf(__uint_as_float(q.z), xcol[k4 * 4 + 2], acc);
+                                acc = fmaf(__uint_as_float(q.w), xcol[k4 * 4 + 3], acc);
+                            }
+                            tmp[r] = acc;
+                        }
+                        const float* Sd = sDi + ((cb >> 4) + bi) * 120;
+#pragma unroll
+                        for (int r = 0; r < 16; ++r) {
+                            float acc = tmp[r];
+#pragma unroll
+                            for (int q = 0; q < r; ++q) acc = fmaf(Sd[(r * (r - 1)) / 2 + q], tmp[q], acc);
+                            if (bi > b0) xcol[bi * 16 + r] = acc;
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < C; ++i) {
+                        float acc = 0.f;
+                        const uint32_t ri = scratch_a + (cb + i) * (4 * C);
+#pragma unroll
+                        for (int k4 = 0; k4 < (i + 3) / 4; ++k4) {
+                            const uint4 q = lds128(ri + (swz<CPRF>(i, k4) << 4));  // (cb + i) and i agree in the swizzle bits
+                            if (k4 * 4 + 0 < i) acc = fmaf(__uint_as_float(q.x), xcol[k4 * 4 + 0], acc);
+                            if (k4 * 4 + 1 < i) acc = fmaf(__uint_as_float(q.y), xcol[(k4 * 4 + 1 < C) ? k4 * 4 + 1 : 0], acc);
+                            if (k4 * 4 + 2 < i) acc = fmaf(__uint_as_float(q.z), xcol[(k4 * 4 + 2 < C) ? k4 * 4 + 2 : 0], acc);
+                            if (k4 * 4 + 3 < i) acc = fmaf(__uint_as_float(q.w), xcol[(k4 * 4 + 3 < C) ? k4 * 4 + 3 : 0], acc);
+                        }
+                        xcol[i] = (i > il) ? acc : ((i == il) ? 1.f : 0.f);
+                    }
                 }
                 compute_barrier();  // everyone has read Abar
 #pragma unroll
@@ -715,6 +768,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(xcol[i]) : "memory");
                 }
             } else {
+                if constexpr (MODE == INV_FWDSUBST_BLOCKED) compute_barrier();
                 compute_barrier();
             }
             compute_barrier();
@@ -1161,7 +1215,6 @@ int launch_tc_bf16(const Problem& p, InverseMode mode, cudaStream_t stream) {
     if (p.d_k != kD || p.d_v != kD) return GDN_ERR_UNSUPPORTED;
     if (!(p.C == 16 || p.C == 32 || p.C == 64 || (p.C == 128 && mode == INV_NEUMANN))) return GDN_ERR_UNSUPPORTED;
     if (mode == INV_NEUMANN && (p.order < 1 || p.order > 7)) return GDN_ERR_UNSUPPORTED;
-    if (mode == INV_FWDSUBST_BLOCKED) return GDN_ERR_UNSUPPORTED;
     if ((long long)p.B * p.H_v * p.T == 0) return GDN_OK;
     int* status = device_status_word();
     if (status == nullptr) return GDN_ERR_LAUNCH;
@@ -1201,6 +1254,13 @@ int launch_tc_bf16(const Problem& p, InverseMode mode, cudaStream_t stream) {
             case 32: return launch_c<32, INV_NEUMANN>(m, prm, stream);
             case 128: return launch_c<64, INV_NEUMANN, true>(m, prm, stream);
             default: return launch_c<64, INV_NEUMANN>(m, prm, stream);
+        }
+    }
+    if (mode == INV_FWDSUBST_BLOCKED) {
+        switch (p.C) {
+            case 16: return launch_c<16, INV_FWDSUBST_BLOCKED>(m, prm, stream);
+            case 32: return launch_c<32, INV_FWDSUBST_BLOCKED>(m, prm, stream);
+            default: return launch_c<64, INV_FWDSUBST_BLOCKED>(m, prm, stream);
         }
     }
     switch (p.C) {

@@ -156,6 +156,34 @@ def test_bf16_forward_substitution_kernel(C):
     _check(inp, TOL_BF16, method="fwdsubst", exact=True)
 
 
+@pytest.mark.parametrize("C", [16, 32, 64])
+def test_bf16_blocked_forward_substitution_kernel(C):
+    inp = gen.make_inputs(1, 2, 4, 512, C, 128, 128, seed=85 + C, adversarial_heads="odd")
+    K, V, beta, g = _to_dev(inp)
+    W, U, Tinv = gdn.chunk_prepare(K, V, beta, g, C, method="fwdsubst", variant=gdn.GDN_FWDSUBST_BLOCKED)
+    W2, U2, Tinv2 = gdn.chunk_prepare(K, V, beta, g, C, method="fwdsubst", variant=gdn.GDN_FWDSUBST_ROWS)
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+    Wg, Ug, Tg = _gpu_chunks(W, U, Tinv, inp)
+    Wo, Uo, To = _oracle(inp, exact=True)
+    for got, ref in ((Tg, To), (Wg, Wo), (Ug, Uo)):
+        floor = orc.rel_frobenius(_bf16_round(ref), ref)
+        assert np.all(orc.rel_frobenius(got, ref) <= np.maximum(TOL_BF16, floor + 2e-4))
+    # the two orders of the same substitution agree to bf16 output rounding
+    assert (Tinv.float() - Tinv2.float()).abs().max() <= 1e-2
+
+
+@pytest.mark.parametrize("C", [16, 32, 64, 128])
+def test_fp32_blocked_forward_substitution(C):
+    inp = gen.make_inputs(1, 1, 2, 2 * C, C, 64, 64, seed=95 + C, dtype=torch.float32)
+    K, V, beta, g = _to_dev(inp)
+    W, U, Tinv = gdn.chunk_prepare(K, V, beta, g, C, method="fwdsubst", variant=gdn.GDN_FWDSUBST_BLOCKED)
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+    Wg, Ug, Tg = _gpu_chunks(W, U, Tinv, inp)
+    Wo, Uo, To = _oracle(inp, exact=True)
+    assert orc.rel_frobenius(Tg, To).max() <= TOL_FP32 and orc.rel_frobenius(Wg, Wo).max() <= TOL_FP32
+    assert orc.rel_frobenius(Ug, Uo).max() <= TOL_FP32
+
+
 def test_empty_batch_is_a_no_op():
     K = torch.empty(0, 2, 128, 128, dtype=torch.bfloat16, device="cuda")
     V = torch.empty(0, 2, 128, 128, dtype=torch.bfloat16, device="cuda")
