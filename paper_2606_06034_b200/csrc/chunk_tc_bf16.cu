@@ -61,6 +61,7 @@ struct Params {
     int N, S;
     unsigned flags;  // GDN_FLAG_*
     long long n_tiles;
+    int s_gi, s_tt, s_bhk;  // the grid size as a step in (value head of the group, token tile, key-head row) digits
 };
 
 template <int C, int NB>
@@ -85,7 +86,8 @@ struct Smem {
     static constexpr int kRn = kG + 512;                // 128 floats: 1 / ||K_row|| (GDN_FLAG_K_L2NORM)
     static constexpr int kBRn = kRn + 512;              // 128 floats: beta / ||K_row||
     static constexpr int kWt = kBRn + 512;              // 4 floats: warp totals of the gate prefix sum (GDN_FLAG_G_RAW)
-    static constexpr int kTotal = kWt + 64;
+    static constexpr int kDummy = kWt + 64;             // one word per thread: target of band entries a thread does not own
+    static constexpr int kTotal = kDummy + kThreads * 4;
 };
 
 __device__ __forceinline__ float fast_exp2(float x) {
@@ -142,27 +144,34 @@ struct Split {
     static constexpr int PCH = HC / 2;             // packed bf16x2 words per thread
 };
 
-// Builds the thread's part of a packed bf16 row that is zero except vals[e] at column il - e
-// (e = 0..n_valid, skipped where the column is negative or outside [col0, col0 + HC)), through the row's
-// private shared-memory line: registers cannot be indexed by a per-thread position, shared memory can.
-// The two halves of a row own disjoint 16-byte chunks of the line, so they never race.
+// Packed bf16 rows that are zero except for the band (vals[e] at column il - e) are assembled through a private
+// shared-memory line per thread: registers cannot be indexed by a per-thread position, shared memory can.
+// The line of tile row t is stored chunk-major (16-byte chunk c of row t at c * 2048 + t * 16), so a warp's
+// accesses fall on consecutive addresses; the two halves of a row own disjoint chunks. Where column il - e lies
+// does not change from tile to tile: band_slots() computes the byte address of each band entry once per thread
+// (entries outside the thread's columns or beyond the band width point at a per-thread dummy word).
 template <int C, int NB>
-__device__ __forceinline__ void build_band_row(uint32_t row_addr, int t, int il, int col0, int n_valid,
-                                               const uint16_t (&vals)[NB + 1], uint32_t (&out)[Split<C>::PCH]) {
-    constexpr int CPR = C / 8;                 // chunks of the full row
-    constexpr int CPT = Split<C>::HC / 8;      // chunks owned by this thread
-    const int c0 = col0 >> 3;
-#pragma unroll
-    for (int c = 0; c < CPT; ++c) sts128(row_addr + (swz<CPR>(t, c0 + c) << 4), 0u, 0u, 0u, 0u);
+__device__ __forceinline__ void band_slots(uint32_t br_base, uint32_t dummy, int t, int il, int col0, int n_valid,
+                                           uint32_t (&slot)[NB + 1]) {
 #pragma unroll
     for (int e = 0; e <= NB; ++e) {
         const int j = il - e;
-        if (j >= col0 && j < col0 + Split<C>::HC && e <= n_valid)
-            sts16(row_addr + (swz<CPR>(t, j >> 3) << 4) + (j & 7) * 2, vals[e]);
+        const bool in = (j >= col0 && j < col0 + Split<C>::HC && e <= n_valid);
+        slot[e] = in ? br_base + (j >> 3) * (kTile * 16) + t * 16 + (j & 7) * 2 : dummy;
     }
+}
+// line = address of the thread's first chunk (br_base + (col0 / 8) * 2048 + t * 16)
+template <int C, int NB>
+__device__ __forceinline__ void build_band_row(uint32_t line, const uint32_t (&slot)[NB + 1], const uint16_t (&vals)[NB + 1],
+                                               uint32_t (&out)[Split<C>::PCH]) {
+    constexpr int CPT = Split<C>::HC / 8;  // chunks owned by this thread
+#pragma unroll
+    for (int c = 0; c < CPT; ++c) sts128(line + c * (kTile * 16), 0u, 0u, 0u, 0u);
+#pragma unroll
+    for (int e = 0; e <= NB; ++e) sts16(slot[e], vals[e]);
 #pragma unroll
     for (int c = 0; c < CPT; ++c) {
-        const uint4 v = lds128(row_addr + (swz<CPR>(t, c0 + c) << 4));
+        const uint4 v = lds128(line + c * (kTile * 16));
         out[c * 4 + 0] = v.x;
         out[c * 4 + 1] = v.y;
         out[c * 4 + 2] = v.z;
@@ -291,8 +300,9 @@ __device__ __forceinline__ void load_cols(uint32_t lane_base, uint32_t col0, int
 // the band, where entries are O(1). `sc` is the per-token scale in shared memory, `sc_i` the row's own scale;
 // a[] = far part of the row, lb[] = band, y[] = T21 part (second block of a 128-chunk).
 template <int C, int NB, bool MERGE>
-__device__ __forceinline__ void build_wu_operands(uint32_t lane_base, uint32_t br_row, int t, int h, int il, int cb, int col0, int wq,
-                                                  int n_band, const float* sc, float sc_i, const float (&a)[Split<C>::HC],
+__device__ __forceinline__ void build_wu_operands(uint32_t lane_base, uint32_t br_line, const uint32_t (&slot)[NB + 1], int t, int h,
+                                                  int il, int cb, int col0, int wq, const float* sc, float sc_i,
+                                                  const float (&a)[Split<C>::HC],
                                                   const uint32_t (&keep)[Split<C>::PCH], const float (&lb)[NB + 1],
                                                   const float (&y)[MERGE ? Split<C>::HC : 1]) {
     constexpr int PCH = Split<C>::PCH;
@@ -307,7 +317,7 @@ __device__ __forceinline__ void build_wu_operands(uint32_t lane_base, uint32_t b
         lo[e] = bf16_bits(tb[e] - bf16_bits_to_f32(hi[e]));
     }
     uint32_t bp[PCH], pk[PCH];
-    build_band_row<C, NB>(br_row, t, il, col0, n_band, hi, bp);
+    build_band_row<C, NB>(br_line, slot, hi, bp);
     const float2* sb2 = reinterpret_cast<const float2*>(sc + cb + col0);
 #pragma unroll
     for (int i = 0; i < PCH; ++i) {
@@ -331,7 +341,7 @@ __device__ __forceinline__ void build_wu_operands(uint32_t lane_base, uint32_t b
         }
     }
     if (plain) store_a_operand<C, true>(lane_base + kAS, t, h, pk);
-    build_band_row<C, NB>(br_row, t, il, col0, n_band, lo, bp);
+    build_band_row<C, NB>(br_line, slot, lo, bp);
     store_a_operand<C, true>(lane_base + kR2, t, h, bp);
 }
 
@@ -339,20 +349,37 @@ struct TileCoord {
     int bhk, bhv;
     int t0;
 };
-// tile index -> (key head row, value head row, first token); tiles that share a key tile are adjacent.
+// A tile index in mixed-radix digits: tile = (bhk * n_tt + tt) * group + gi, so that tiles sharing a key tile are
+// adjacent. A CTA walks its tiles by adding the grid size digit by digit (one carry per digit is enough because
+// every digit of the step is below its radix), which avoids integer divisions inside the tile loop.
 // All counts fit 32 bits (checked by the launcher).
-__device__ __forceinline__ TileCoord decode_tile(uint32_t tile, const Params& p) {
-    TileCoord c;
+struct TilePos {
+    int gi, tt, bhk;
+};
+__device__ __forceinline__ TilePos tile_pos(uint32_t tile, const Params& p) {
+    TilePos c;
     const uint32_t y = tile / static_cast<uint32_t>(p.group);
-    const uint32_t gi = tile - y * p.group;
-    const uint32_t bhk = y / static_cast<uint32_t>(p.n_tt);
-    const uint32_t tt = y - bhk * p.n_tt;
-    const uint32_t b = bhk / static_cast<uint32_t>(p.H_k);
-    const uint32_t hk = bhk - b * p.H_k;
-    c.bhk = static_cast<int>(bhk);
-    c.bhv = static_cast<int>(b * p.H_v + hk * p.group + gi);
-    c.t0 = static_cast<int>(tt) * kTile;
+    c.gi = static_cast<int>(tile - y * p.group);
+    c.bhk = static_cast<int>(y / static_cast<uint32_t>(p.n_tt));
+    c.tt = static_cast<int>(y - static_cast<uint32_t>(c.bhk) * p.n_tt);
     return c;
+}
+__device__ __forceinline__ void tile_advance(TilePos& c, const Params& p) {
+    c.gi += p.s_gi;
+    const int c1 = (c.gi >= p.group) ? 1 : 0;
+    c.gi -= c1 ? p.group : 0;
+    c.tt += p.s_tt + c1;
+    const int c2 = (c.tt >= p.n_tt) ? 1 : 0;
+    c.tt -= c2 ? p.n_tt : 0;
+    c.bhk += p.s_bhk + c2;
+}
+// (key head row, value head row, first token): value head row = bhk * group + gi because H_v = H_k * group
+__device__ __forceinline__ TileCoord tile_coord(const TilePos& c, const Params& p) {
+    TileCoord r;
+    r.bhk = c.bhk;
+    r.bhv = c.bhk * p.group + c.gi;
+    r.t0 = c.tt * kTile;
+    return r;
 }
 
 // MERGE: the tile is ONE chunk of 128 tokens whose two 64 x 64 diagonal blocks are inverted by the scheme above
@@ -360,12 +387,14 @@ __device__ __forceinline__ TileCoord decode_tile(uint32_t tile, const Params& p)
 // T21 = -T22 A21 T11, evaluated as Y = A21 + A21 X11, T21 = -(Y + X22 Y) with X = T - I of the blocks, so that
 // the identity parts stay in fp32 and only the small products pass through bf16 operands.
 // EX: the optional prologue / fp32 outputs of gdn_chunk_prepare_ex are compiled in (flags read at run time).
-template <int C, int NB, int MODE, bool MERGE, bool EX>
+// DBL: the residual sum is evaluated for S = 8 by the four-level doubling scheme (C = 64 only).
+template <int C, int NB, int MODE, bool MERGE, bool EX, bool DBL>
 __global__ void __launch_bounds__(kThreads, 2)
 chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                 const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmU,
                 const __grid_constant__ CUtensorMap tmT, const Params p) {
     static_assert(!MERGE || (C == 64 && MODE == INV_NEUMANN), "the block merge is built for 64-blocks of the Neumann scheme");
+    static_assert(!DBL || (C == 64 && MODE == INV_NEUMANN), "the doubling scheme is built for 64-blocks");
     using L = Smem<C, NB>;
     using SP = Split<C>;
     constexpr int NBP = L::NBP;
@@ -393,6 +422,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 
     __shared__ uint64_t bar_k, bar_v, bar_mma;
     __shared__ uint32_t tmem_base_s;
+    __shared__ int s_fail;  // set by warp 0 when one of its bounded waits ran out
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
@@ -405,6 +435,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         mbar_init(&bar_k, 1);
         mbar_init(&bar_v, 1);
         mbar_init(&bar_mma, 1);
+        s_fail = 0;
         mbar_fence_init();
         tma_prefetch_desc(&tmK);
         tma_prefetch_desc(&tmV);
@@ -428,8 +459,8 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 
     // Threads t and t + 128 share tile row t (TMEM lane t): half h owns the chunk-local columns
     // [h * HC, (h + 1) * HC) when C >= 32; for C = 16 only h = 0 works on the row (h = 1 joins for W/U).
-    // Thread 0 also issues every TMA load and every tcgen05.mma, right after the CTA barrier that says
-    // all rows of the operand are in place.
+    // One elected lane of warp 0 also issues every TMA load and every tcgen05.mma, right after the CTA barrier
+    // that says all rows of the operand are in place.
     const int t = tid & 127;
     const int h = tid >> 7;
     const bool active = SP::kSplit || (h == 0);
@@ -440,7 +471,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     const int wrow0 = wq * 32;                 // first tile row of the warp
     const uint32_t lane_base = tmem + (static_cast<uint32_t>(wq * 32) << 16);
     const uint32_t scratch_a = smem_u32(smem + L::kEB);
-    const uint32_t br_row = smem_u32(smem + L::kBR) + t * (2 * C);
+    const uint32_t br_line = smem_u32(smem + L::kBR) + (col0 >> 3) * (kTile * 16) + t * 16;
     const uint32_t rowf = scratch_a + t * (4 * C);  // private fp32 row (shared by the two halves)
     const uint32_t sK_a = smem_u32(sK), sV_a = smem_u32(sV), sEB_a = smem_u32(sEB);
     const uint32_t idesc_g = instr_desc(128, 128, 1, 1, 0, 0, 1);
@@ -448,9 +479,35 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     const uint32_t idesc_w = instr_desc(128, 128, 1, 1, 0, 1, 1);
     uint32_t par_mma = 0, par_kv = 0;
     bool ok = true;
+    // Completion of the MMAs committed to bar_mma: warp 0 polls the mbarrier, the other warps sleep on a hardware
+    // barrier that warp 0 joins afterwards (no polling instructions from 7 of the 8 warps). A timeout is published
+    // in s_fail, so that every thread leaves the tile loop at the same point.
+    auto wait_mma = [&]() -> bool {
+        if (warp == 0 && !wait_bar(&bar_mma, par_mma)) *reinterpret_cast<volatile int*>(&s_fail) = 1;
+        asm volatile("bar.sync 2, 256;" ::: "memory");
+        par_mma ^= 1;
+        return *reinterpret_cast<volatile int*>(&s_fail) == 0;
+    };
 
+    // tile-invariant per-thread band positions and keep-mask (0 on the band and the diagonal, ones elsewhere)
+    uint32_t slot[NB + 1];
+    uint32_t keep[PCH];
+    band_slots<C, NB>(smem_u32(smem + L::kBR), smem_u32(smem + L::kDummy) + tid * 4, t, il, col0, n_band, slot);
+    if (active) {
+        uint16_t vals[NB + 1];
+#pragma unroll
+        for (int e = 0; e <= NB; ++e) vals[e] = 0xFFFFu;
+        build_band_row<C, NB>(br_line, slot, vals, keep);
+#pragma unroll
+        for (int i = 0; i < PCH; ++i) keep[i] = ~keep[i];
+    } else {
+#pragma unroll
+        for (int i = 0; i < PCH; ++i) keep[i] = 0u;
+    }
+
+    TilePos pos_next = tile_pos(blockIdx.x, p);  // position of the tile after the one being worked on
     if (tid == 0 && blockIdx.x < n_tiles) {
-        const TileCoord c = decode_tile(blockIdx.x, p);
+        const TileCoord c = tile_coord(pos_next, p);
         mbar_arrive_expect_tx(&bar_k, 32768);
         tma_load_3d(sK, &tmK, &bar_k, 0, c.t0, c.bhk);
         tma_load_3d(sK + 16384, &tmK, &bar_k, 64, c.t0, c.bhk);
@@ -461,7 +518,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     // beta and g of the row are fetched one tile ahead
     float bi_next = 0.f, gi_next = 0.f;
     if (blockIdx.x < n_tiles) {
-        const TileCoord c = decode_tile(blockIdx.x, p);
+        const TileCoord c = tile_coord(pos_next, p);
         if (c.t0 + t < p.T) {
             const long long r = (long long)c.bhv * p.T + c.t0 + t;
             bi_next = __ldg(p.beta + r);
@@ -470,7 +527,8 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     }
 
     for (uint32_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-        const TileCoord tc = decode_tile(tile, p);
+        const TileCoord tc = tile_coord(pos_next, p);
+        tile_advance(pos_next, p);
         const uint32_t next = tile + gridDim.x;
         const bool has_next = next < n_tiles;
 
@@ -498,19 +556,21 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             const int first = wq - (wq % kWarpsPerChunk);
             for (int w = first; w < wq; ++w) gi_ += swt[w];
         }
-        if (tid == 0) {
+        if (warp == 0) {
             // G = K K^T into R0..R1 (128 columns)
             STAMP(20);
             if (!wait_bar(&bar_k, par_kv)) ok = false;
             STAMP(21);
             if (ok) {
                 tc_fence_after_sync();
+                if (elect_one()) {
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const uint64_t d = smem_desc(sK_a + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024, SWZ_128B);
-                    mma_f16_ss(tmem + kR0, d, d, idesc_g, ks > 0);
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const uint64_t d = smem_desc(sK_a + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024, SWZ_128B);
+                        mma_f16_ss(tmem + kR0, d, d, idesc_g, ks > 0);
+                    }
+                    mma_commit(&bar_mma);
                 }
-                mma_commit(&bar_mma);
             }
         }
         if (h == 0) {
@@ -527,8 +587,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 
         STAMP(2);
         // ---- A-build: this thread's part of the row of Abar, from the Gram block in TMEM
-        if (!wait_bar(&bar_mma, par_mma)) { ok = false; break; }
-        par_mma ^= 1;
+        if (!wait_mma()) { ok = false; break; }
         STAMP(3);
         tc_fence_after_sync();
         float a[HC];
@@ -599,7 +658,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         bi_next = 0.f;
         gi_next = 0.f;
         if (has_next) {
-            const TileCoord nc = decode_tile(next, p);
+            const TileCoord nc = tile_coord(pos_next, p);
             if (nc.t0 + t < p.T) {
                 const long long r = (long long)nc.bhv * p.T + nc.t0 + t;
                 bi_next = __ldg(p.beta + r);
@@ -794,27 +853,122 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         }
 
         STAMP(6);
-        // ---- packed bf16 forms of the band: keep-mask (0 on the band and diagonal) and I + L
-        uint32_t keep[PCH], bpT[PCH];
+        // ---- packed bf16 form of the band: I + L (the keep-mask, 0 on the band and diagonal, was built before the loop)
+        uint32_t bpT[PCH];
         if (active) {
             uint16_t vals[NB + 1];
-#pragma unroll
-            for (int e = 0; e <= NB; ++e) vals[e] = 0xFFFFu;
-            build_band_row<C, NB>(br_row, t, il, col0, n_band, vals, keep);
-#pragma unroll
-            for (int i = 0; i < PCH; ++i) keep[i] = ~keep[i];
             vals[0] = 0x3F80u;  // 1.0
 #pragma unroll
             for (int e = 1; e <= NB; ++e) vals[e] = bf16_bits(lb[e]);
-            build_band_row<C, NB>(br_row, t, il, col0, n_band, vals, bpT);
+            build_band_row<C, NB>(br_line, slot, vals, bpT);
         } else {
 #pragma unroll
-            for (int i = 0; i < PCH; ++i) { keep[i] = 0u; bpT[i] = 0u; }
+            for (int i = 0; i < PCH; ++i) bpT[i] = 0u;
         }
 
         STAMP(7);
         if constexpr (MODE == INV_NEUMANN) {
-            // ---- residual rounds: A_k = T0 + Z_k (bf16, TMEM), Z_{k+1} = A_k E, so that T = T0 + Z_S
+            // ---- residual correction T = T0 sum_{s<=S} E^s (Eq. 13). With X_m = T0 sum_{s<=m} E^s:
+            //   X_{m+1} = T0 + X_m E   and   X_{2m+1} = X_m + X_m E^{m+1}.
+            if constexpr (DBL) {
+                {
+                    // Four dependent products instead of eight: X_1 = T0 + T0 E and E^2; X_3 = X_1 + X_1 E^2 and E^4;
+                    // X_4 = T0 + X_3 E; X_8 = X_3 + X_4 E^4. Each level is one MMA per chunk m (M = 128, N = 64,
+                    // K = 64) whose A operand holds the X rows of chunk m on the chunk's own 64 lanes and the rows of
+                    // the power of E_m on the other 64 lanes, so the product of both with the level's B operand
+                    // (E_m, E_m^2 or E_m^4) comes out of the same instruction. A thread therefore owns, besides its
+                    // part of row il of X of its chunk, the same part of row il of the powers of the OTHER chunk's E.
+                    const int co = cb ^ 64;  // first tile row of the other chunk
+                    const uint32_t a_own = lane_base + kAS + (cb >> 1) + h * 16;
+                    const uint32_t a_oth = lane_base + kAS + (co >> 1) + h * 16;
+                    const uint32_t d_own = lane_base + kR0 + cb + h * 32;
+                    const uint32_t d_oth = lane_base + kR0 + co + h * 32;
+                    uint8_t* sQB = sEB + 16384;  // powers of E as B operand, same layout as E
+                    const uint32_t b_oth = ((co + col0) >> 3) * 1024 + il * 16;
+                    const uint32_t idesc_h = instr_desc(128, 64, 1, 1, 0, 1, 1);
+                    tmem_st16(a_own, bpT);
+                    compute_barrier();  // E of every row is in shared memory
+                    {
+                        uint32_t r16[16];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const uint4 v = *reinterpret_cast<const uint4*>(sEB + b_oth + j * 1024);
+                            r16[4 * j + 0] = v.x; r16[4 * j + 1] = v.y; r16[4 * j + 2] = v.z; r16[4 * j + 3] = v.w;
+                        }
+                        tmem_st16(a_oth, r16);
+                    }
+                    fence_proxy_async_smem();
+                    tmem_wait_st();
+#pragma unroll
+                    for (int lv = 0; lv < 4; ++lv) {
+                        STAMP(30 + lv);
+                        tc_fence_before_sync();
+                        compute_barrier();
+                        STAMP(40 + lv);
+                        if (warp == 0) {
+                            tc_fence_after_sync();
+                            const uint32_t bb = (lv == 0 || lv == 2) ? sEB_a : sEB_a + 16384;
+                            if (elect_one()) {
+#pragma unroll
+                            for (int m = 0; m < 2; ++m) {
+#pragma unroll
+                                for (int ks = 0; ks < 4; ++ks) {
+                                    const uint64_t bd = smem_desc(bb + m * 8192 + ks * 256, 128, 1024, SWZ_NONE);
+                                    mma_f16_ts(tmem + kR0 + 64 * m, tmem + kAS + 32 * m + ks * 8, bd, idesc_h, ks > 0);
+                                }
+                            }
+                            mma_commit(&bar_mma);
+                            }
+                        }
+                        if (!wait_mma()) { ok = false; break; }
+                        tc_fence_after_sync();
+                        STAMP(50 + lv);
+                        // in two halves of 16 columns, to keep the live registers down
+#pragma unroll
+                        for (int hh = 0; hh < 2; ++hh) {
+                            uint32_t d[16];
+                            tmem_ld16(d_own + hh * 16, d);
+                            tmem_wait_ld();
+                            if (lv == 0) {
+#pragma unroll
+                                for (int j = 0; j < 16; ++j) a[hh * 16 + j] = __uint_as_float(d[j]);
+                            } else if (lv != 2) {
+#pragma unroll
+                                for (int j = 0; j < 16; ++j) a[hh * 16 + j] += __uint_as_float(d[j]);
+                            }
+                            if (lv < 3) {
+                                uint32_t pk[8];
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) {
+                                    const uint32_t w = (lv == 2) ? pack_bf16x2(__uint_as_float(d[2 * i]), __uint_as_float(d[2 * i + 1]))
+                                                                 : pack_bf16x2(a[hh * 16 + 2 * i], a[hh * 16 + 2 * i + 1]);
+                                    pk[i] = (w & keep[hh * 8 + i]) | bpT[hh * 8 + i];
+                                }
+                                tmem_st8(a_own + hh * 8, pk);
+                            }
+                        }
+                        if (lv < 2) {
+#pragma unroll
+                            for (int hh = 0; hh < 2; ++hh) {
+                                uint32_t q[16], pq[8];
+                                tmem_ld16(d_oth + hh * 16, q);
+                                tmem_wait_ld();
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) pq[i] = pack_bf16x2(__uint_as_float(q[2 * i]), __uint_as_float(q[2 * i + 1]));
+                                if (lv == 0) tmem_st8(a_oth + hh * 8, pq);
+#pragma unroll
+                                for (int j2 = 0; j2 < 2; ++j2)
+                                    *reinterpret_cast<uint4*>(sQB + b_oth + (hh * 2 + j2) * 1024) =
+                                        make_uint4(pq[4 * j2], pq[4 * j2 + 1], pq[4 * j2 + 2], pq[4 * j2 + 3]);
+                            }
+                            fence_proxy_async_smem();
+                        }
+                        if (lv < 3) tmem_wait_st();
+                    }
+                    if (!ok) break;
+                }
+            } else {
+            // one product per term: A_k = T0 + Z_k (bf16, TMEM), Z_{k+1} = A_k E, T = T0 + Z_S
             for (int k = 0; k < S; ++k) {
                 if (active) {
                     uint32_t pk[PCH];
@@ -829,23 +983,29 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     fence_proxy_async_smem();
                     tmem_wait_st();
                 }
+                STAMP(60);
                 tc_fence_before_sync();
                 compute_barrier();
-                if (tid == 0) {
+                STAMP(61);
+                if (warp == 0) {
                     // [Z_1; Z_2; ...] <- [A_1; A_2; ...] [E_1 | E_2 | ...]: M = 128, N = 128, K = C; row t keeps
                     // the C columns of its own chunk
                     tc_fence_after_sync();
+                    if (elect_one()) {
 #pragma unroll
-                    for (int ks = 0; ks < C / 16; ++ks) {
-                        const uint64_t bd = smem_desc(sEB_a + ks * 256, 128, 16 * C, SWZ_NONE);
-                        mma_f16_ts(tmem + kR0, tmem + kAS + ks * 8, bd, idesc_c, ks > 0);
+                        for (int ks = 0; ks < C / 16; ++ks) {
+                            const uint64_t bd = smem_desc(sEB_a + ks * 256, 128, 16 * C, SWZ_NONE);
+                            mma_f16_ts(tmem + kR0, tmem + kAS + ks * 8, bd, idesc_c, ks > 0);
+                        }
+                        mma_commit(&bar_mma);
                     }
-                    mma_commit(&bar_mma);
                 }
-                if (!wait_bar(&bar_mma, par_mma)) { ok = false; break; }
-                par_mma ^= 1;
+                STAMP(62);
+                if (!wait_mma()) { ok = false; break; }
                 tc_fence_after_sync();
+                STAMP(63);
                 if (active) load_diag_block<C>(lane_base, kR0, t, h, a);
+            }
             }
             if (!ok) break;
             if (S == 0) {
@@ -869,7 +1029,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 #pragma unroll
                 for (int e = 1; e <= NB; ++e) vals[e] = bf16_bits(lb[e]);
                 uint32_t bpL[PCH];
-                build_band_row<C, NB>(br_row, t, il, col0, n_band, vals, bpL);
+                build_band_row<C, NB>(br_line, slot, vals, bpL);
 #pragma unroll
                 for (int i = 0; i < PCH; ++i) xrow[i] = (pack_bf16x2(a[2 * i], a[2 * i + 1]) & keep[i]) | bpL[i];
             }
@@ -906,17 +1066,18 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 fence_proxy_async_smem();
                 tc_fence_before_sync();
                 compute_barrier();
-                if (tid == 0) {
+                if (warp == 0) {
                     tc_fence_after_sync();
+                    if (elect_one()) {
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks) {
-                        const uint64_t bd = smem_desc(sEB_a + ks * 256, 128, 1024, SWZ_NONE);
-                        mma_f16_ts(tmem + kR0, tmem + kAS + ks * 8, bd, idesc_m, ks > 0);
+                        for (int ks = 0; ks < 4; ++ks) {
+                            const uint64_t bd = smem_desc(sEB_a + ks * 256, 128, 1024, SWZ_NONE);
+                            mma_f16_ts(tmem + kR0, tmem + kAS + ks * 8, bd, idesc_m, ks > 0);
+                        }
+                        mma_commit(&bar_mma);
                     }
-                    mma_commit(&bar_mma);
                 }
-                if (!wait_bar(&bar_mma, par_mma)) { ok = false; break; }
-                par_mma ^= 1;
+                if (!wait_mma()) { ok = false; break; }
                 tc_fence_after_sync();
                 if (wq >= 2) {
                     uint32_t d[32];
@@ -947,22 +1108,24 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         // ---- A operands for W/U: T diag(scale) = hi + lo, hi over the whole row, lo only on band + diagonal.
         // scale = beta for U; for W it is beta / ||K|| when the keys are normalised on the fly, else beta as well
         if (active) {
-            build_wu_operands<C, NB, MERGE>(lane_base, br_row, t, h, il, cb, col0, wq, n_band, f_l2 ? sbrn : sbeta,
+            build_wu_operands<C, NB, MERGE>(lane_base, br_line, slot, t, h, il, cb, col0, wq, f_l2 ? sbrn : sbeta,
                                             f_l2 ? bi * rni : bi, a, keep, lb, y);
             tmem_wait_st();
         }
         tc_fence_before_sync();
         compute_barrier();
-        if (tid == 0) {
+        if (warp == 0) {
             // W = (hi + lo) K: A operands in TMEM (AS: high bf16 half, R2: low half of the band),
             // B = the K tile read as an MN-major operand (both 64-column sub-tiles, N = 128)
             tc_fence_after_sync();
+            if (elect_one()) {
 #pragma unroll
-            for (int ks = 0; ks < 16; ++ks) {
-                const uint64_t bd = smem_desc(sK_a + (ks & 7) * 2048, 16384, 1024, SWZ_128B);
-                mma_f16_ts(tmem + kR0, tmem + ((ks < 8) ? kAS : kR2) + (ks & 7) * 8, bd, idesc_w, ks > 0);
+                for (int ks = 0; ks < 16; ++ks) {
+                    const uint64_t bd = smem_desc(sK_a + (ks & 7) * 2048, 16384, 1024, SWZ_128B);
+                    mma_f16_ts(tmem + kR0, tmem + ((ks < 8) ? kAS : kR2) + (ks & 7) * 8, bd, idesc_w, ks > 0);
+                }
+                mma_commit(&bar_mma);
             }
-            mma_commit(&bar_mma);
         }
 
         STAMP(8);
@@ -1049,13 +1212,12 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         // sub-tile of its warp -> one bulk tensor store (32 rows x 64 columns) per warp
 #pragma unroll 1
         for (int half = 0; half < 2; ++half) {
-            if (!wait_bar(&bar_mma, par_mma)) { ok = false; break; }
-            par_mma ^= 1;
+            if (!wait_mma()) { ok = false; break; }
             tc_fence_after_sync();
             STAMP(11 + half * 3);
-            if (tid == 0 && has_next) {
+            if (warp == 0 && has_next && elect_one()) {
                 // the products that read this tile's K (half 0) or V (half 1) are complete: prefetch the next tile's
-                const TileCoord nc = decode_tile(next, p);
+                const TileCoord nc = tile_coord(pos_next, p);
                 if (half == 0) {
                     mbar_arrive_expect_tx(&bar_k, 32768);
                     tma_load_3d(sK, &tmK, &bar_k, 0, nc.t0, nc.bhk);
@@ -1094,22 +1256,24 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 if (f_l2) {
                     // U uses beta where W used beta / ||K||: rebuild both A operands
                     if (active) {
-                        build_wu_operands<C, NB, MERGE>(lane_base, br_row, t, h, il, cb, col0, wq, n_band, sbeta, bi, a, keep, lb, y);
+                        build_wu_operands<C, NB, MERGE>(lane_base, br_line, slot, t, h, il, cb, col0, wq, sbeta, bi, a, keep, lb, y);
                         tmem_wait_st();
                     }
                     tc_fence_before_sync();
                     compute_barrier();
                 }
-                if (tid == 0) {
+                if (warp == 0) {
                     if (!wait_bar(&bar_v, par_kv)) ok = false;
                     if (ok) {
                         tc_fence_after_sync();
+                        if (elect_one()) {
 #pragma unroll
-                        for (int ks = 0; ks < 16; ++ks) {
-                            const uint64_t bd = smem_desc(sV_a + (ks & 7) * 2048, 16384, 1024, SWZ_128B);
-                            mma_f16_ts(tmem + kR0, tmem + ((ks < 8) ? kAS : kR2) + (ks & 7) * 8, bd, idesc_w, ks > 0);
+                            for (int ks = 0; ks < 16; ++ks) {
+                                const uint64_t bd = smem_desc(sV_a + (ks & 7) * 2048, 16384, 1024, SWZ_128B);
+                                mma_f16_ts(tmem + kR0, tmem + ((ks < 8) ? kAS : kR2) + (ks & 7) * 8, bd, idesc_w, ks > 0);
+                            }
+                            mma_commit(&bar_mma);
                         }
-                        mma_commit(&bar_mma);
                     }
                 }
             }
@@ -1179,22 +1343,34 @@ struct Maps {
     CUtensorMap K, V, W, U, T;
 };
 
-template <int C, int NB, int MODE, bool MERGE, bool EX>
+template <int C, int NB, int MODE, bool MERGE, bool EX, bool DBL>
 int launch_ex(const Maps& m, const Params& prm, cudaStream_t stream) {
     using L = Smem<C, NB>;
     const int smem = L::kTotal + 1024;
-    auto kern = chunk_tc_kernel<C, NB, MODE, MERGE, EX>;
+    auto kern = chunk_tc_kernel<C, NB, MODE, MERGE, EX, DBL>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return GDN_ERR_LAUNCH;
     long long grid = prm.n_tiles < 2 * 148 ? prm.n_tiles : 2 * 148;
-    kern<<<static_cast<int>(grid), kThreads, smem, stream>>>(m.K, m.V, m.W, m.U, m.T, prm);
+    Params q = prm;
+    const long long y = grid / prm.group;
+    q.s_gi = static_cast<int>(grid - y * prm.group);
+    q.s_bhk = static_cast<int>(y / prm.n_tt);
+    q.s_tt = static_cast<int>(y - static_cast<long long>(q.s_bhk) * prm.n_tt);
+    kern<<<static_cast<int>(grid), kThreads, smem, stream>>>(m.K, m.V, m.W, m.U, m.T, q);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? GDN_OK : GDN_ERR_LAUNCH;
 }
 
 template <int C, int NB, int MODE, bool MERGE>
 int launch_one(const Maps& m, const Params& prm, cudaStream_t stream) {
-    if (MODE == INV_NEUMANN && prm.flags != 0) return launch_ex<C, NB, MODE, MERGE, (MODE == INV_NEUMANN)>(m, prm, stream);
-    return launch_ex<C, NB, MODE, MERGE, false>(m, prm, stream);
+    constexpr bool kNeu = (MODE == INV_NEUMANN);
+    constexpr bool kDbl = kNeu && C == 64;
+    const bool dbl = kDbl && prm.S == 8;
+    if (kNeu && prm.flags != 0) {
+        if (dbl) return launch_ex<C, NB, MODE, MERGE, kNeu, kDbl>(m, prm, stream);
+        return launch_ex<C, NB, MODE, MERGE, kNeu, false>(m, prm, stream);
+    }
+    if (dbl) return launch_ex<C, NB, MODE, MERGE, false, kDbl>(m, prm, stream);
+    return launch_ex<C, NB, MODE, MERGE, false, false>(m, prm, stream);
 }
 
 template <int C, int MODE, bool MERGE = false>
