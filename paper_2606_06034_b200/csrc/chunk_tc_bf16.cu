@@ -121,6 +121,11 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
     return v;
 }
+__device__ __forceinline__ float4 lds128f(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+    return v;
+}
 __device__ __forceinline__ float lds32f(uint32_t addr) {
     float v;
     asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
@@ -318,11 +323,12 @@ __device__ __forceinline__ void build_wu_operands(uint32_t lane_base, uint32_t b
     }
     uint32_t bp[PCH], pk[PCH];
     build_band_row<C, NB>(br_line, slot, hi, bp);
-    const float2* sb2 = reinterpret_cast<const float2*>(sc + cb + col0);
+    const uint32_t sb_a = smem_u32(sc + cb + col0);
 #pragma unroll
-    for (int i = 0; i < PCH; ++i) {
-        const float2 bb = sb2[i];
-        pk[i] = (pack_bf16x2(a[2 * i] * bb.x, a[2 * i + 1] * bb.y) & keep[i]) | bp[i];
+    for (int i = 0; i < PCH / 2; ++i) {
+        const float4 bb = lds128f(sb_a + i * 16);
+        pk[2 * i] = (pack_bf16x2(a[4 * i] * bb.x, a[4 * i + 1] * bb.y) & keep[2 * i]) | bp[2 * i];
+        pk[2 * i + 1] = (pack_bf16x2(a[4 * i + 2] * bb.z, a[4 * i + 3] * bb.w) & keep[2 * i + 1]) | bp[2 * i + 1];
     }
     bool plain = true;
     if constexpr (MERGE) {
@@ -474,6 +480,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     const uint32_t br_line = smem_u32(smem + L::kBR) + (col0 >> 3) * (kTile * 16) + t * 16;
     const uint32_t rowf = scratch_a + t * (4 * C);  // private fp32 row (shared by the two halves)
     const uint32_t sK_a = smem_u32(sK), sV_a = smem_u32(sV), sEB_a = smem_u32(sEB);
+    const uint32_t sSH_a = smem_u32(smem + L::kSH), sg_a = smem_u32(smem + L::kG);
     const uint32_t idesc_g = instr_desc(128, 128, 1, 1, 0, 0, 1);
     const uint32_t idesc_c = instr_desc(128, 128, 1, 1, 0, 1, 1);
     const uint32_t idesc_w = instr_desc(128, 128, 1, 1, 0, 1, 1);
@@ -626,11 +633,10 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         if (active) {
             const float gs = gi_ * kLog2e;
             const float nbi = -bi * rni;
-            const float4* sg4 = reinterpret_cast<const float4*>(sg + cb + col0);
             const float4* sr4 = reinterpret_cast<const float4*>(srn + cb + col0);
 #pragma unroll
             for (int j4 = 0; j4 < HC / 4; ++j4) {
-                const float4 gq = sg4[j4];
+                const float4 gq = lds128f(sg_a + (cb + col0 + j4 * 4) * 4);
                 const float gj[4] = {gq.x, gq.y, gq.z, gq.w};
                 float rj[4] = {1.f, 1.f, 1.f, 1.f};
                 if (f_l2) {
@@ -718,11 +724,11 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     float v = a[jl];
                     float cc[NBP];
                     if constexpr (NBP == 4) {
-                        const float4 c4 = *reinterpret_cast<const float4*>(sSH + (cb + col0 + jl) * 4);
+                        const float4 c4 = lds128f(sSH_a + (cb + col0 + jl) * 16);
                         cc[0] = c4.x; cc[1] = c4.y; cc[2] = c4.z; cc[3] = c4.w;
                     } else {
-                        const float4 c4 = *reinterpret_cast<const float4*>(sSH + (cb + col0 + jl) * 8);
-                        const float4 d4 = *reinterpret_cast<const float4*>(sSH + (cb + col0 + jl) * 8 + 4);
+                        const float4 c4 = lds128f(sSH_a + (cb + col0 + jl) * 32);
+                        const float4 d4 = lds128f(sSH_a + (cb + col0 + jl) * 32 + 16);
                         cc[0] = c4.x; cc[1] = c4.y; cc[2] = c4.z; cc[3] = c4.w;
                         cc[4] = d4.x; cc[5] = d4.y; cc[6] = d4.z; cc[7] = d4.w;
                     }
