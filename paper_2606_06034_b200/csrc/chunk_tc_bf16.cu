@@ -646,9 +646,12 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
                     const int jl = j4 * 4 + q;
-                    float v = nbi * fast_exp2(fmaf(-gj[q], kLog2e, gs)) * a[jl];
+                    // Entries on and above the diagonal are NOT zeroed here: every later use either reads strictly
+                    // lower entries only or multiplies them by a band entry that is zero, so they only have to be
+                    // finite, which the clamp of the exponent (<= 0 for every lower entry) guarantees.
+                    float v = nbi * fast_exp2(fminf(fmaf(-gj[q], kLog2e, gs), 64.f)) * a[jl];
                     if (f_l2) v *= rj[q];
-                    a[jl] = (col0 + jl < il) ? v : 0.f;
+                    a[jl] = (C < 64 && !(col0 + jl < il)) ? 0.f : v;  // (for C < 64 the mask is kept: it costs less there than it saves)
                 }
             }
             // the row of Abar goes to its private fp32 line: entries next to the diagonal (and, for the
