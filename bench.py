@@ -253,8 +253,8 @@ def run_ours(args, rank, world, dist_ctx):
 
 # per-launch DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under profiles/
 TRAFFIC_PER_LAUNCH: dict = {
-    "sweep_c64": 248.6e6,     # profiles/chunk_tc_kernel_bf16_c64_sweep_c64.md
-    "prefill_gqa": 1027.9e6,  # profiles/chunk_tc_kernel_bf16_c64_prefill_gqa.md
+    "sweep_c64": 248.9e6,     # profiles/chunk_tc_kernel_bf16_c64_sweep_c64.md
+    "prefill_gqa": 1029.0e6,  # profiles/chunk_tc_kernel_bf16_c64_prefill_gqa.md
 }
 
 
