@@ -304,12 +304,12 @@ __device__ __forceinline__ void load_cols(uint32_t lane_base, uint32_t col0, int
 // hi (slot AS) = bf16(T diag(scale)) over the whole row, lo (slot R2) = bf16 of what hi loses on the diagonal and
 // the band, where entries are O(1). `sc` is the per-token scale in shared memory, `sc_i` the row's own scale;
 // a[] = far part of the row, lb[] = band, y[] = T21 part (second block of a 128-chunk).
-template <int C, int NB, bool MERGE>
+template <int C, int NB, bool MERGE, bool YPART = MERGE>
 __device__ __forceinline__ void build_wu_operands(uint32_t lane_base, uint32_t br_line, const uint32_t (&slot)[NB + 1], int t, int h,
                                                   int il, int cb, int col0, int wq, const float* sc, float sc_i,
                                                   const float (&a)[Split<C>::HC],
                                                   const uint32_t (&keep)[Split<C>::PCH], const float (&lb)[NB + 1],
-                                                  const float (&y)[MERGE ? Split<C>::HC : 1]) {
+                                                  const float (&y)[YPART ? Split<C>::HC : 1]) {
     constexpr int PCH = Split<C>::PCH;
     float tb[NB + 1];
     tb[0] = sc_i;
@@ -336,14 +336,16 @@ __device__ __forceinline__ void build_wu_operands(uint32_t lane_base, uint32_t b
             // second block of a 128-chunk: columns of the first block carry T21 diag(scale) instead of zeros
             plain = false;
             store_a_operand<C, false>(lane_base + kAS, t, h, pk);
-            const float2* sb1 = reinterpret_cast<const float2*>(sc + col0);
-            uint32_t po[PCH];
+            if constexpr (YPART) {
+                const float2* sb1 = reinterpret_cast<const float2*>(sc + col0);
+                uint32_t po[PCH];
 #pragma unroll
-            for (int i = 0; i < PCH; ++i) {
-                const float2 bb = sb1[i];
-                po[i] = pack_bf16x2(y[2 * i] * bb.x, y[2 * i + 1] * bb.y);
+                for (int i = 0; i < PCH; ++i) {
+                    const float2 bb = sb1[i];
+                    po[i] = pack_bf16x2(y[2 * i] * bb.x, y[2 * i + 1] * bb.y);
+                }
+                store_stacked_operand<C>(lane_base + kAS, h, po);
             }
-            store_stacked_operand<C>(lane_base + kAS, h, po);
         }
     }
     if (plain) store_a_operand<C, true>(lane_base + kAS, t, h, pk);
@@ -1024,11 +1026,26 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         }
         // a[] = this thread's part of the far row (T - I - L)
 
-        constexpr int YN = MERGE ? HC : 1;
-        float y[YN];  // MERGE, rows of the second block: A21 part, then Y, then T21 (columns of the first block)
+        // MERGE, rows of the second block: A21 part, then Y, then T21 (columns of the first block). Without the optional
+        // prologue the T21 part is consumed (Tinv staging, W/U operand) at the end of the merge, which ends its live
+        // range there; with it the operand is rebuilt for U, so the values stay in registers (y[]).
+        constexpr bool Y_EARLY = MERGE && !EX;
+        constexpr int YN = (MERGE && !Y_EARLY) ? HC : 1;
+        float y[YN];
 #pragma unroll
         for (int j = 0; j < YN; ++j) y[j] = 0.f;
+        uint32_t yp[Y_EARLY ? PCH : 1];  // Y_EARLY: the T21 part as packed bf16, for the Tinv staging line
+        yp[0] = 0u;
         if constexpr (MERGE) {
+            float yl[Y_EARLY ? HC : 1];
+            float* ym;
+            if constexpr (Y_EARLY) {
+                ym = yl;
+#pragma unroll
+                for (int j = 0; j < HC; ++j) yl[j] = 0.f;
+            } else {
+                ym = y;
+            }
             const uint32_t idesc_m = instr_desc(128, 64, 1, 1, 0, 1, 1);
             // X = T - I of the row's diagonal block as packed bf16 (band without the unit diagonal + far part)
             uint32_t xrow[PCH];
@@ -1049,25 +1066,31 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     *reinterpret_cast<uint4*>(sEB + ((col0 >> 3) + c) * 1024 + t * 16) =
                         make_uint4(xrow[4 * c], xrow[4 * c + 1], xrow[4 * c + 2], xrow[4 * c + 3]);
             } else {
-                // second block: A21_ij = beta_i e^{g_i - g_j} G_ij, j in the first block (fp32), bf16 copy as A operand
-                uint32_t gq[32];
-                tmem_ld32(lane_base + kR2 + h * 32, gq);
-                tmem_wait_ld();
+                // second block: A21_ij = beta_i e^{g_i - g_j} G_ij, j in the first block (fp32), bf16 copy as A operand.
+                // In two halves of 16 columns to keep the live registers down.
                 const float gs = gi_ * kLog2e;
-                const float4* sg4 = reinterpret_cast<const float4*>(sg + col0);
 #pragma unroll
-                for (int j4 = 0; j4 < HC / 4; ++j4) {
-                    const float4 gv = sg4[j4];
-                    const float gj[4] = {gv.x, gv.y, gv.z, gv.w};
+                for (int hh = 0; hh < 2; ++hh) {
+                    uint32_t gq[16];
+                    tmem_ld16(lane_base + kR2 + h * 32 + hh * 16, gq);
+                    tmem_wait_ld();
 #pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        y[j4 * 4 + q] = bi * rni * (f_l2 ? srn[col0 + j4 * 4 + q] : 1.f) * fast_exp2(fmaf(-gj[q], kLog2e, gs)) *
+                    for (int j4 = 0; j4 < 4; ++j4) {
+                        const int j0 = hh * 16 + j4 * 4;
+                        const float4 gv = lds128f(sg_a + (col0 + j0) * 4);
+                        const float gj[4] = {gv.x, gv.y, gv.z, gv.w};
+#pragma unroll
+                        for (int q = 0; q < 4; ++q)
+                            ym[j0 + q] = bi * rni * (f_l2 ? srn[col0 + j0 + q] : 1.f) * fast_exp2(fmaf(-gj[q], kLog2e, gs)) *
                                         __uint_as_float(gq[j4 * 4 + q]);
+                    }
                 }
                 uint32_t pk[PCH];
 #pragma unroll
-                for (int i = 0; i < PCH; ++i) pk[i] = pack_bf16x2(y[2 * i], y[2 * i + 1]);
+                for (int i = 0; i < PCH; ++i) pk[i] = pack_bf16x2(ym[2 * i], ym[2 * i + 1]);
                 store_stacked_operand<C>(lane_base + kAS, h, pk);
+                // the parked Gram block has been read: R2 takes the X22 rows, the A operand of the second product
+                store_stacked_operand<C>(lane_base + kR2, h, xrow);
                 tmem_wait_st();
             }
 #pragma unroll 1
@@ -1081,7 +1104,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 #pragma unroll
                         for (int ks = 0; ks < 4; ++ks) {
                             const uint64_t bd = smem_desc(sEB_a + ks * 256, 128, 1024, SWZ_NONE);
-                            mma_f16_ts(tmem + kR0, tmem + kAS + ks * 8, bd, idesc_m, ks > 0);
+                            mma_f16_ts(tmem + kR0, tmem + (step == 0 ? kAS : kR2) + ks * 8, bd, idesc_m, ks > 0);
                         }
                         mma_commit(&bar_mma);
                     }
@@ -1089,35 +1112,56 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 if (!wait_mma()) { ok = false; break; }
                 tc_fence_after_sync();
                 if (wq >= 2) {
-                    uint32_t d[32];
-                    tmem_ld32(lane_base + kR0 + h * 32, d);
-                    tmem_wait_ld();
-                    if (step == 0) {
-                        // Y = A21 + A21 X11; then Y rows as B operand and X22 rows as A operand of X22 Y
 #pragma unroll
-                        for (int j = 0; j < HC; ++j) y[j] += __uint_as_float(d[j]);
+                    for (int hh = 0; hh < 2; ++hh) {
+                        uint32_t d[16];
+                        tmem_ld16(lane_base + kR0 + h * 32 + hh * 16, d);
+                        tmem_wait_ld();
+                        if (step == 0) {
+                            // Y = A21 + A21 X11; Y rows become the B operand of X22 Y
 #pragma unroll
-                        for (int c = 0; c < CPT; ++c)
-                            *reinterpret_cast<uint4*>(sEB + ((col0 >> 3) + c) * 1024 + il * 16) =
-                                make_uint4(pack_bf16x2(y[8 * c + 0], y[8 * c + 1]), pack_bf16x2(y[8 * c + 2], y[8 * c + 3]),
-                                           pack_bf16x2(y[8 * c + 4], y[8 * c + 5]), pack_bf16x2(y[8 * c + 6], y[8 * c + 7]));
-                        store_stacked_operand<C>(lane_base + kAS, h, xrow);
-                        tmem_wait_st();
-                    } else {
-                        // T21 = -(Y + X22 Y)
+                            for (int j = 0; j < 16; ++j) ym[hh * 16 + j] += __uint_as_float(d[j]);
 #pragma unroll
-                        for (int j = 0; j < HC; ++j) y[j] = -(y[j] + __uint_as_float(d[j]));
+                            for (int c = 0; c < 2; ++c) {
+                                const int j0 = hh * 16 + c * 8;
+                                *reinterpret_cast<uint4*>(sEB + ((col0 >> 3) + hh * 2 + c) * 1024 + il * 16) =
+                                    make_uint4(pack_bf16x2(ym[j0 + 0], ym[j0 + 1]), pack_bf16x2(ym[j0 + 2], ym[j0 + 3]),
+                                               pack_bf16x2(ym[j0 + 4], ym[j0 + 5]), pack_bf16x2(ym[j0 + 6], ym[j0 + 7]));
+                            }
+                        } else {
+                            // T21 = -(Y + X22 Y)
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) ym[hh * 16 + j] = -(ym[hh * 16 + j] + __uint_as_float(d[j]));
+                        }
                     }
                 }
             }
             if (!ok) break;
+            if constexpr (Y_EARLY) {
+                // the row's part of the other block column of Tinv (T21, or the zeros above it), packed for the
+                // staging line (which overlaps the band-row lines that the W/U operands still need)
+#pragma unroll
+                for (int i = 0; i < PCH; ++i) yp[i] = pack_bf16x2(ym[2 * i], ym[2 * i + 1]);
+                // T21 diag(beta): the first-block columns of the W/U operand of the second block's rows
+                if (wq >= 2) {
+                    const uint32_t sb_a = smem_u32(sbeta + col0);
+                    uint32_t po[PCH];
+#pragma unroll
+                    for (int i = 0; i < PCH / 2; ++i) {
+                        const float4 bb = lds128f(sb_a + i * 16);
+                        po[2 * i] = pack_bf16x2(ym[4 * i] * bb.x, ym[4 * i + 1] * bb.y);
+                        po[2 * i + 1] = pack_bf16x2(ym[4 * i + 2] * bb.z, ym[4 * i + 3] * bb.w);
+                    }
+                    store_stacked_operand<C>(lane_base + kAS, h, po);
+                }
+            }
         }
 
         STAMP(9);
         // ---- A operands for W/U: T diag(scale) = hi + lo, hi over the whole row, lo only on band + diagonal.
         // scale = beta for U; for W it is beta / ||K|| when the keys are normalised on the fly, else beta as well
         if (active) {
-            build_wu_operands<C, NB, MERGE>(lane_base, br_line, slot, t, h, il, cb, col0, wq, f_l2 ? sbrn : sbeta,
+            build_wu_operands<C, NB, MERGE, MERGE && !Y_EARLY>(lane_base, br_line, slot, t, h, il, cb, col0, wq, f_l2 ? sbrn : sbeta,
                                             f_l2 ? bi * rni : bi, a, keep, lb, y);
             tmem_wait_st();
         }
@@ -1163,7 +1207,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     }
                     *reinterpret_cast<float4*>(trow + dcol + c * 4) = make_float4(v[0], v[1], v[2], v[3]);
                 }
-                if constexpr (MERGE) {
+                if constexpr (MERGE && !Y_EARLY) {
                     const int ocol = (wq >= 2 ? 0 : 64) + col0;  // T21 part, or the zero block above it
 #pragma unroll
                     for (int c = 0; c < HC / 4; ++c)
@@ -1185,8 +1229,11 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                        (pack_bf16x2(a[c * 8 + 2], a[c * 8 + 3]) & keep[c * 4 + 1]) | bpT[c * 4 + 1],
                        (pack_bf16x2(a[c * 8 + 4], a[c * 8 + 5]) & keep[c * 4 + 2]) | bpT[c * 4 + 2],
                        (pack_bf16x2(a[c * 8 + 6], a[c * 8 + 7]) & keep[c * 4 + 3]) | bpT[c * 4 + 3]);
-                sts128(rowo + (swz<4>(t, c) << 4), pack_bf16x2(y[c * 8 + 0], y[c * 8 + 1]), pack_bf16x2(y[c * 8 + 2], y[c * 8 + 3]),
-                       pack_bf16x2(y[c * 8 + 4], y[c * 8 + 5]), pack_bf16x2(y[c * 8 + 6], y[c * 8 + 7]));
+                if constexpr (Y_EARLY)
+                    sts128(rowo + (swz<4>(t, c) << 4), yp[c * 4 + 0], yp[c * 4 + 1], yp[c * 4 + 2], yp[c * 4 + 3]);
+                else
+                    sts128(rowo + (swz<4>(t, c) << 4), pack_bf16x2(y[c * 8 + 0], y[c * 8 + 1]), pack_bf16x2(y[c * 8 + 2], y[c * 8 + 3]),
+                           pack_bf16x2(y[c * 8 + 4], y[c * 8 + 5]), pack_bf16x2(y[c * 8 + 6], y[c * 8 + 7]));
             }
             fence_proxy_async_smem();
             __syncwarp();
@@ -1265,7 +1312,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 if (f_l2) {
                     // U uses beta where W used beta / ||K||: rebuild both A operands
                     if (active) {
-                        build_wu_operands<C, NB, MERGE>(lane_base, br_line, slot, t, h, il, cb, col0, wq, sbeta, bi, a, keep, lb, y);
+                        build_wu_operands<C, NB, MERGE, MERGE && !Y_EARLY>(lane_base, br_line, slot, t, h, il, cb, col0, wq, sbeta, bi, a, keep, lb, y);
                         tmem_wait_st();
                     }
                     tc_fence_before_sync();
