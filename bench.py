@@ -311,7 +311,7 @@ def run_extras(gdn, gen, dev, args):
     out = {}
     hbm_peak, _, _ = measured_peaks()
     plan = [("sweep_c16", "neumann"), ("sweep_c32", "neumann"), ("sweep_c64", "neumann"), ("sweep_c128", "neumann"),
-            ("sweep_c64", "fwdsubst"), ("sweep_c64", "fwdsubst-blocked"),
+            ("sweep_c64", "neumann-s15"), ("sweep_c64", "fwdsubst"), ("sweep_c64", "fwdsubst-blocked"),
             ("sweep_c32", "fwdsubst"), ("sweep_c16", "fwdsubst"), ("prefill_gqa", "neumann")]
     for name, method in plan:
         try:
@@ -319,7 +319,10 @@ def run_extras(gdn, gen, dev, args):
             outs = gdn.alloc_outputs(inp.K, inp.V, inp.C)
             meth, var = (method.split("-") + ["rows"])[:2]
             variant = gdn.GDN_FWDSUBST_BLOCKED if var == "blocked" else gdn.GDN_FWDSUBST_ROWS
-            fn = lambda: gdn.chunk_prepare(inp.K, inp.V, inp.beta, inp.g, inp.C, outputs=outs, method=meth, variant=variant)
+            # "neumann-s15": all 15 residual terms (the exact inverse at N = 3, C = 64) by the doubling scheme
+            n_ord, n_res = (3, 15) if var == "s15" else (-1, -1)
+            fn = lambda: gdn.chunk_prepare(inp.K, inp.V, inp.beta, inp.g, inp.C, n_ord, n_res, outputs=outs, method=meth,
+                                           variant=variant)
             total_ms, _ = device_time_steps(fn, 20, 3, None)
             ms = total_ms / 20
             by = algorithmic_bytes_per_chunk(inp.C, inp.d_k, inp.d_v, inp.H_v // inp.H_k)

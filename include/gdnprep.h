@@ -33,6 +33,8 @@
  *   - Value head h reads key head h / (H_v / H_k); H_v must be a multiple of H_k.
  *   - order = N >= 1 and residual_steps = S >= 0; -1 selects the paper's value
  *     for the chunk size (gdn_default_order, gdn_default_residual_steps).
+ *     S >= ceil(C / (N + 1)) - 1 keeps every non-zero term (E^s = 0 beyond), i.e. the
+ *     exact inverse: S = 15 at C = 64, N = 3.
  *   - Return value: GDN_OK or a negative gdn_status. On any error nothing is
  *     launched. No exception crosses this boundary.
  *   - Pointers must be 16-byte aligned; T must be a multiple of C.

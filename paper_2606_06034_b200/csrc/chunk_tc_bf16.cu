@@ -395,14 +395,15 @@ __device__ __forceinline__ TileCoord tile_coord(const TilePos& c, const Params& 
 // T21 = -T22 A21 T11, evaluated as Y = A21 + A21 X11, T21 = -(Y + X22 Y) with X = T - I of the blocks, so that
 // the identity parts stay in fp32 and only the small products pass through bf16 operands.
 // EX: the optional prologue / fp32 outputs of gdn_chunk_prepare_ex are compiled in (flags read at run time).
-// DBL: the residual sum is evaluated for S = 8 by the four-level doubling scheme (C = 64 only).
-template <int C, int NB, int MODE, bool MERGE, bool EX, bool DBL>
+// DBL: 8 or 15 = the residual sum for that S is evaluated by the four-level doubling scheme (C = 64 only); 0 = one
+// product per term.
+template <int C, int NB, int MODE, bool MERGE, bool EX, int DBL>
 __global__ void __launch_bounds__(kThreads, 2)
 chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                 const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmU,
                 const __grid_constant__ CUtensorMap tmT, const Params p) {
     static_assert(!MERGE || (C == 64 && MODE == INV_NEUMANN), "the block merge is built for 64-blocks of the Neumann scheme");
-    static_assert(!DBL || (C == 64 && MODE == INV_NEUMANN), "the doubling scheme is built for 64-blocks");
+    static_assert(DBL == 0 || ((DBL == 8 || DBL == 15) && C == 64 && MODE == INV_NEUMANN), "the doubling scheme is built for 64-blocks");
     using L = Smem<C, NB>;
     using SP = Split<C>;
     constexpr int NBP = L::NBP;
@@ -881,10 +882,14 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         if constexpr (MODE == INV_NEUMANN) {
             // ---- residual correction T = T0 sum_{s<=S} E^s (Eq. 13). With X_m = T0 sum_{s<=m} E^s:
             //   X_{m+1} = T0 + X_m E   and   X_{2m+1} = X_m + X_m E^{m+1}.
-            if constexpr (DBL) {
+            if constexpr (DBL != 0) {
                 {
+                    constexpr bool kFull = (DBL == 15);
                     // Four dependent products instead of eight: X_1 = T0 + T0 E and E^2; X_3 = X_1 + X_1 E^2 and E^4;
-                    // X_4 = T0 + X_3 E; X_8 = X_3 + X_4 E^4. Each level is one MMA per chunk m (M = 128, N = 64,
+                    // X_4 = T0 + X_3 E; X_8 = X_3 + X_4 E^4. With S = 15 (kFull) the last two levels are
+                    // X_7 = X_3 + X_3 E^4 and E^8; X_15 = X_7 + X_7 E^8, which is the exact inverse at N = 3
+                    // because E^16 = 0 (the Newton-Schulz / factorised form of Eq. 12-13 with the same four levels).
+                    // Each level is one MMA per chunk m (M = 128, N = 64,
                     // K = 64) whose A operand holds the X rows of chunk m on the chunk's own 64 lanes and the rows of
                     // the power of E_m on the other 64 lanes, so the product of both with the level's B operand
                     // (E_m, E_m^2 or E_m^4) comes out of the same instruction. A thread therefore owns, besides its
@@ -918,7 +923,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                         STAMP(40 + lv);
                         if (warp == 0) {
                             tc_fence_after_sync();
-                            const uint32_t bb = (lv == 0 || lv == 2) ? sEB_a : sEB_a + 16384;
+                            const uint32_t bb = (lv == 0 || (lv == 2 && !kFull)) ? sEB_a : sEB_a + 16384;
                             if (elect_one()) {
 #pragma unroll
                             for (int m = 0; m < 2; ++m) {
@@ -943,7 +948,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                             if (lv == 0) {
 #pragma unroll
                                 for (int j = 0; j < 16; ++j) a[hh * 16 + j] = __uint_as_float(d[j]);
-                            } else if (lv != 2) {
+                            } else if (lv != 2 || kFull) {
 #pragma unroll
                                 for (int j = 0; j < 16; ++j) a[hh * 16 + j] += __uint_as_float(d[j]);
                             }
@@ -951,14 +956,14 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                                 uint32_t pk[8];
 #pragma unroll
                                 for (int i = 0; i < 8; ++i) {
-                                    const uint32_t w = (lv == 2) ? pack_bf16x2(__uint_as_float(d[2 * i]), __uint_as_float(d[2 * i + 1]))
+                                    const uint32_t w = (lv == 2 && !kFull) ? pack_bf16x2(__uint_as_float(d[2 * i]), __uint_as_float(d[2 * i + 1]))
                                                                  : pack_bf16x2(a[hh * 16 + 2 * i], a[hh * 16 + 2 * i + 1]);
                                     pk[i] = (w & keep[hh * 8 + i]) | bpT[hh * 8 + i];
                                 }
                                 tmem_st8(a_own + hh * 8, pk);
                             }
                         }
-                        if (lv < 2) {
+                        if (lv < (kFull ? 3 : 2)) {
 #pragma unroll
                             for (int hh = 0; hh < 2; ++hh) {
                                 uint32_t q[16], pq[8];
@@ -966,7 +971,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                                 tmem_wait_ld();
 #pragma unroll
                                 for (int i = 0; i < 8; ++i) pq[i] = pack_bf16x2(__uint_as_float(q[2 * i]), __uint_as_float(q[2 * i + 1]));
-                                if (lv == 0) tmem_st8(a_oth + hh * 8, pq);
+                                if (lv < (kFull ? 2 : 1)) tmem_st8(a_oth + hh * 8, pq);
 #pragma unroll
                                 for (int j2 = 0; j2 < 2; ++j2)
                                     *reinterpret_cast<uint4*>(sQB + b_oth + (hh * 2 + j2) * 1024) =
@@ -1399,7 +1404,7 @@ struct Maps {
     CUtensorMap K, V, W, U, T;
 };
 
-template <int C, int NB, int MODE, bool MERGE, bool EX, bool DBL>
+template <int C, int NB, int MODE, bool MERGE, bool EX, int DBL>
 int launch_ex(const Maps& m, const Params& prm, cudaStream_t stream) {
     using L = Smem<C, NB>;
     const int smem = L::kTotal + 1024;
@@ -1420,13 +1425,15 @@ template <int C, int NB, int MODE, bool MERGE>
 int launch_one(const Maps& m, const Params& prm, cudaStream_t stream) {
     constexpr bool kNeu = (MODE == INV_NEUMANN);
     constexpr bool kDbl = kNeu && C == 64;
-    const bool dbl = kDbl && prm.S == 8;
+    const int dbl = !kDbl ? 0 : (prm.S == 8 ? 8 : (prm.S == 15 ? 15 : 0));
     if (kNeu && prm.flags != 0) {
-        if (dbl) return launch_ex<C, NB, MODE, MERGE, kNeu, kDbl>(m, prm, stream);
-        return launch_ex<C, NB, MODE, MERGE, kNeu, false>(m, prm, stream);
+        if (dbl == 8) return launch_ex<C, NB, MODE, MERGE, kNeu, kDbl ? 8 : 0>(m, prm, stream);
+        if (dbl == 15) return launch_ex<C, NB, MODE, MERGE, kNeu, kDbl ? 15 : 0>(m, prm, stream);
+        return launch_ex<C, NB, MODE, MERGE, kNeu, 0>(m, prm, stream);
     }
-    if (dbl) return launch_ex<C, NB, MODE, MERGE, false, kDbl>(m, prm, stream);
-    return launch_ex<C, NB, MODE, MERGE, false, false>(m, prm, stream);
+    if (dbl == 8) return launch_ex<C, NB, MODE, MERGE, false, kDbl ? 8 : 0>(m, prm, stream);
+    if (dbl == 15) return launch_ex<C, NB, MODE, MERGE, false, kDbl ? 15 : 0>(m, prm, stream);
+    return launch_ex<C, NB, MODE, MERGE, false, 0>(m, prm, stream);
 }
 
 template <int C, int MODE, bool MERGE = false>

@@ -98,7 +98,16 @@ def test_bf16_other_orders_and_steps(C, N, S):
     _check(inp, TOL_BF16, N, S)
 
 
-@pytest.mark.parametrize("N,S", [(-1, -1), (3, 2), (2, 4)])
+@pytest.mark.parametrize("adv", ["none", "all"])
+def test_bf16_full_residual_sum_is_the_exact_inverse(adv):
+    """S = 15 at N = 3, C = 64 keeps every term (E^16 = 0): the kernel's four-level doubling form of the sum must
+    match both the oracle's truncated evaluation with S = 15 and the exact inverse by forward substitution."""
+    inp = gen.make_inputs(2, 2, 2, 1024, 64, 128, 128, seed=47, adversarial_heads=adv)
+    _check(inp, TOL_BF16, 3, 15)
+    _check(inp, TOL_BF16, 3, 15, exact=True)
+
+
+@pytest.mark.parametrize("N,S", [(-1, -1), (3, 2), (2, 4), (3, 15)])
 def test_bf16_chunk_128_block_merge(N, S):
     """C = 128: two 64-blocks by the scheme plus the block formula of App. E for the lower-left block."""
     inp = gen.make_inputs(2, 2, 4, 512, 128, 128, 128, seed=45 + N + S)
