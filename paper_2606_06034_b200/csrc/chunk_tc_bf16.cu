@@ -338,19 +338,24 @@ __device__ __forceinline__ void build_wu_operands(uint32_t lane_base, uint32_t b
             store_a_operand<C, false>(lane_base + kAS, t, h, pk);
             if constexpr (YPART) {
                 const float2* sb1 = reinterpret_cast<const float2*>(sc + col0);
-                uint32_t po[PCH];
+                uint32_t po[PCH], pl[PCH];
 #pragma unroll
                 for (int i = 0; i < PCH; ++i) {
                     const float2 bb = sb1[i];
-                    po[i] = pack_bf16x2(y[2 * i] * bb.x, y[2 * i + 1] * bb.y);
+                    const float v0 = y[2 * i] * bb.x, v1 = y[2 * i + 1] * bb.y;
+                    po[i] = pack_bf16x2(v0, v1);
+                    pl[i] = pack_bf16x2(v0 - bf16_lo(po[i]), v1 - bf16_hi(po[i]));
                 }
                 store_stacked_operand<C>(lane_base + kAS, h, po);
+                store_stacked_operand<C>(lane_base + kR2, h, pl);
             }
         }
     }
     if (plain) store_a_operand<C, true>(lane_base + kAS, t, h, pk);
     build_band_row<C, NB>(br_line, slot, lo, bp);
-    store_a_operand<C, true>(lane_base + kR2, t, h, bp);
+    // rows of the second block of a 128-chunk keep the lo half of T21 diag(scale) in the first block's columns
+    if (plain) store_a_operand<C, true>(lane_base + kR2, t, h, bp);
+    else store_a_operand<C, false>(lane_base + kR2, t, h, bp);
 }
 
 struct TileCoord {
@@ -1052,27 +1057,13 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 ym = y;
             }
             const uint32_t idesc_m = instr_desc(128, 64, 1, 1, 0, 1, 1);
-            // X = T - I of the row's diagonal block as packed bf16 (band without the unit diagonal + far part)
-            uint32_t xrow[PCH];
-            {
-                uint16_t vals[NB + 1];
-                vals[0] = 0;
-#pragma unroll
-                for (int e = 1; e <= NB; ++e) vals[e] = bf16_bits(lb[e]);
-                uint32_t bpL[PCH];
-                build_band_row<C, NB>(br_line, slot, vals, bpL);
-#pragma unroll
-                for (int i = 0; i < PCH; ++i) xrow[i] = (pack_bf16x2(a[2 * i], a[2 * i + 1]) & keep[i]) | bpL[i];
-            }
-            if (wq < 2) {
-                // first block: X11 rows as the B operand [64 x 64] (MN-major, no swizzle) of Y = A21 + A21 X11
-#pragma unroll
-                for (int c = 0; c < CPT; ++c)
-                    *reinterpret_cast<uint4*>(sEB + ((col0 >> 3) + c) * 1024 + t * 16) =
-                        make_uint4(xrow[4 * c], xrow[4 * c + 1], xrow[4 * c + 2], xrow[4 * c + 3]);
-            } else {
-                // second block: A21_ij = beta_i e^{g_i - g_j} G_ij, j in the first block (fp32), bf16 copy as A operand.
-                // In two halves of 16 columns to keep the live registers down.
+            // Both products of the merge cancel strongly when the keys of a chunk are correlated (A21 has entries
+            // near 1, Y = A21 T11 is small), so every operand goes in as hi + lo (two bf16 halves) and each product
+            // is hi*hi + lo*hi + hi*lo; the identity parts stay in fp32.
+            if (wq >= 2) {
+                // second block: A21_ij = beta_i e^{g_i - g_j} G_ij, j in the first block (fp32); its hi and lo halves
+                // are the A operands (AS columns 0..31 and 32..63). In two halves of 16 columns to keep the live
+                // registers down.
                 const float gs = gi_ * kLog2e;
 #pragma unroll
                 for (int hh = 0; hh < 2; ++hh) {
@@ -1087,17 +1078,58 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 #pragma unroll
                         for (int q = 0; q < 4; ++q)
                             ym[j0 + q] = bi * rni * (f_l2 ? srn[col0 + j0 + q] : 1.f) * fast_exp2(fmaf(-gj[q], kLog2e, gs)) *
-                                        __uint_as_float(gq[j4 * 4 + q]);
+                                         __uint_as_float(gq[j4 * 4 + q]);
+                    }
+                    uint32_t ph[8], pl[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const float v0 = ym[hh * 16 + 2 * i], v1 = ym[hh * 16 + 2 * i + 1];
+                        ph[i] = pack_bf16x2(v0, v1);
+                        pl[i] = pack_bf16x2(v0 - bf16_lo(ph[i]), v1 - bf16_hi(ph[i]));
+                    }
+                    tmem_st8(lane_base + kAS + h * 16 + hh * 8, ph);
+                    tmem_st8(lane_base + kAS + 32 + h * 16 + hh * 8, pl);
+                }
+            }
+            // X = T - I of the row's diagonal block (band without the unit diagonal + far part) as hi and lo halves:
+            // X11 rows are the B operands of the first product ([64 x 64], MN-major, no swizzle; hi at 0, lo at 8 KB),
+            // X22 rows the A operands of the second (R2 columns 0..31 and 32..63; the parked Gram block has been read).
+            // One half (hi, then lo) and 16 columns at a time, stored at once, to keep the live registers down.
+            {
+                uint16_t vals[NB + 1];
+                vals[0] = 0;
+#pragma unroll
+                for (int e = 1; e <= NB; ++e) vals[e] = bf16_bits(lb[e]);
+#pragma unroll
+                for (int part = 0; part < 2; ++part) {
+                    uint32_t bp[PCH];
+                    if (part == 1) {
+#pragma unroll
+                        for (int e = 1; e <= NB; ++e) vals[e] = bf16_bits(lb[e] - bf16_bits_to_f32(vals[e]));
+                    }
+                    build_band_row<C, NB>(br_line, slot, vals, bp);
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh) {
+                        uint32_t x[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const int k = hh * 8 + i;
+                            uint32_t w = pack_bf16x2(a[2 * k], a[2 * k + 1]);
+                            if (part == 1) w = pack_bf16x2(a[2 * k] - bf16_lo(w), a[2 * k + 1] - bf16_hi(w));
+                            x[i] = (w & keep[k]) | bp[k];
+                        }
+                        if (wq < 2) {
+#pragma unroll
+                            for (int c = 0; c < 2; ++c)
+                                *reinterpret_cast<uint4*>(sEB + part * 8192 + ((col0 >> 3) + hh * 2 + c) * 1024 + t * 16) =
+                                    make_uint4(x[4 * c], x[4 * c + 1], x[4 * c + 2], x[4 * c + 3]);
+                        } else {
+                            tmem_st8(lane_base + kR2 + part * 32 + h * 16 + hh * 8, x);
+                        }
                     }
                 }
-                uint32_t pk[PCH];
-#pragma unroll
-                for (int i = 0; i < PCH; ++i) pk[i] = pack_bf16x2(ym[2 * i], ym[2 * i + 1]);
-                store_stacked_operand<C>(lane_base + kAS, h, pk);
-                // the parked Gram block has been read: R2 takes the X22 rows, the A operand of the second product
-                store_stacked_operand<C>(lane_base + kR2, h, xrow);
-                tmem_wait_st();
             }
+            tmem_wait_st();
 #pragma unroll 1
             for (int step = 0; step < 2; ++step) {
                 fence_proxy_async_smem();
@@ -1106,10 +1138,15 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 if (warp == 0) {
                     tc_fence_after_sync();
                     if (elect_one()) {
+                        const uint32_t a_hi = tmem + (step == 0 ? kAS : kR2), a_lo = a_hi + 32;
 #pragma unroll
-                        for (int ks = 0; ks < 4; ++ks) {
-                            const uint64_t bd = smem_desc(sEB_a + ks * 256, 128, 1024, SWZ_NONE);
-                            mma_f16_ts(tmem + kR0, tmem + (step == 0 ? kAS : kR2) + ks * 8, bd, idesc_m, ks > 0);
+                        for (int part = 0; part < 3; ++part) {
+                            // hi*hi, lo*hi, hi*lo
+#pragma unroll
+                            for (int ks = 0; ks < 4; ++ks) {
+                                const uint64_t bd = smem_desc(sEB_a + (part == 2 ? 8192 : 0) + ks * 256, 128, 1024, SWZ_NONE);
+                                mma_f16_ts(tmem + kR0, (part == 1 ? a_lo : a_hi) + ks * 8, bd, idesc_m, part > 0 || ks > 0);
+                            }
                         }
                         mma_commit(&bar_mma);
                     }
@@ -1123,15 +1160,22 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                         tmem_ld16(lane_base + kR0 + h * 32 + hh * 16, d);
                         tmem_wait_ld();
                         if (step == 0) {
-                            // Y = A21 + A21 X11; Y rows become the B operand of X22 Y
+                            // Y = A21 + A21 X11; Y rows (hi, lo) become the B operands of X22 Y
 #pragma unroll
                             for (int j = 0; j < 16; ++j) ym[hh * 16 + j] += __uint_as_float(d[j]);
 #pragma unroll
                             for (int c = 0; c < 2; ++c) {
                                 const int j0 = hh * 16 + c * 8;
-                                *reinterpret_cast<uint4*>(sEB + ((col0 >> 3) + hh * 2 + c) * 1024 + il * 16) =
-                                    make_uint4(pack_bf16x2(ym[j0 + 0], ym[j0 + 1]), pack_bf16x2(ym[j0 + 2], ym[j0 + 3]),
-                                               pack_bf16x2(ym[j0 + 4], ym[j0 + 5]), pack_bf16x2(ym[j0 + 6], ym[j0 + 7]));
+                                uint32_t wh[4], wl[4];
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) {
+                                    const float v0 = ym[j0 + 2 * i], v1 = ym[j0 + 2 * i + 1];
+                                    wh[i] = pack_bf16x2(v0, v1);
+                                    wl[i] = pack_bf16x2(v0 - bf16_lo(wh[i]), v1 - bf16_hi(wh[i]));
+                                }
+                                const uint32_t off = ((col0 >> 3) + hh * 2 + c) * 1024 + il * 16;
+                                *reinterpret_cast<uint4*>(sEB + off) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
+                                *reinterpret_cast<uint4*>(sEB + 8192 + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
                             }
                         } else {
                             // T21 = -(Y + X22 Y)
@@ -1150,14 +1194,18 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 // T21 diag(beta): the first-block columns of the W/U operand of the second block's rows
                 if (wq >= 2) {
                     const uint32_t sb_a = smem_u32(sbeta + col0);
-                    uint32_t po[PCH];
+                    uint32_t po[PCH], pl[PCH];
 #pragma unroll
                     for (int i = 0; i < PCH / 2; ++i) {
                         const float4 bb = lds128f(sb_a + i * 16);
-                        po[2 * i] = pack_bf16x2(ym[4 * i] * bb.x, ym[4 * i + 1] * bb.y);
-                        po[2 * i + 1] = pack_bf16x2(ym[4 * i + 2] * bb.z, ym[4 * i + 3] * bb.w);
+                        const float v0 = ym[4 * i] * bb.x, v1 = ym[4 * i + 1] * bb.y, v2 = ym[4 * i + 2] * bb.z, v3 = ym[4 * i + 3] * bb.w;
+                        po[2 * i] = pack_bf16x2(v0, v1);
+                        po[2 * i + 1] = pack_bf16x2(v2, v3);
+                        pl[2 * i] = pack_bf16x2(v0 - bf16_lo(po[2 * i]), v1 - bf16_hi(po[2 * i]));
+                        pl[2 * i + 1] = pack_bf16x2(v2 - bf16_lo(po[2 * i + 1]), v3 - bf16_hi(po[2 * i + 1]));
                     }
                     store_stacked_operand<C>(lane_base + kAS, h, po);
+                    store_stacked_operand<C>(lane_base + kR2, h, pl);  // the lo operand keeps these columns (see build_wu_operands)
                 }
             }
         }
@@ -1168,6 +1216,16 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         if (active) {
             build_wu_operands<C, NB, MERGE, MERGE && !Y_EARLY>(lane_base, br_line, slot, t, h, il, cb, col0, wq, f_l2 ? sbrn : sbeta,
                                             f_l2 ? bi * rni : bi, a, keep, lb, y);
+            if constexpr (MERGE) {
+                // I + L again for the Tinv rows: rebuilt here instead of being carried across the merge, where
+                // registers are scarce (it must be built before the barrier below: the Tinv staging lines of other
+                // rows overlap this row's private line)
+                uint16_t vals[NB + 1];
+                vals[0] = 0x3F80u;
+#pragma unroll
+                for (int e = 1; e <= NB; ++e) vals[e] = bf16_bits(lb[e]);
+                build_band_row<C, NB>(br_line, slot, vals, bpT);
+            }
             tmem_wait_st();
         }
         tc_fence_before_sync();

@@ -108,9 +108,14 @@ def test_bf16_full_residual_sum_is_the_exact_inverse(adv):
 
 
 @pytest.mark.parametrize("N,S", [(-1, -1), (3, 2), (2, 4), (3, 15)])
-def test_bf16_chunk_128_block_merge(N, S):
-    """C = 128: two 64-blocks by the scheme plus the block formula of App. E for the lower-left block."""
-    inp = gen.make_inputs(2, 2, 4, 512, 128, 128, 128, seed=45 + N + S)
+@pytest.mark.parametrize("adv", ["none", "odd"])
+def test_bf16_chunk_128_block_merge(N, S, adv):
+    """C = 128: two 64-blocks by the scheme plus the block formula of App. E for the lower-left block. On strongly
+    correlated keys both products of the merge cancel (A21 has entries near 1, A21 T11 is small): the kernel's
+    hi + lo operands must keep the result at the bf16 rounding floor there too."""
+    if adv == "odd" and S in (2, 4):
+        pytest.skip("few residual terms on adversarial blocks: the truncated series itself has not converged")
+    inp = gen.make_inputs(2, 2, 4, 512, 128, 128, 128, seed=45 + N + S, adversarial_heads=adv)
     _check(inp, TOL_BF16, N, S)
     inp = gen.make_inputs(1, 1, 2, 128, 128, 128, 128, seed=46)
     _check(inp, TOL_BF16, N, S)
@@ -265,8 +270,6 @@ def test_bf16_prologue_flags(C, flags):
 def test_bf16_fp32_outputs_show_the_accumulators(C, adv):
     """With fp32 outputs the bf16 output rounding (1.7e-3) is gone: what remains is the error of the bf16
     MMA operands, which the fp32 band / hi-lo split keeps small even for strongly correlated keys."""
-    if C == 128 and adv == "all":
-        pytest.skip("the block merge of C = 128 passes O(1) cancelling quantities through single bf16 operands")
     inp = gen.make_inputs(1, 2, 2, 512, C, 128, 128, seed=230 + C, adversarial_heads=adv)
     _check_ex(inp, None, gdn.GDN_FLAG_OUT_FP32, 5e-4)
 
