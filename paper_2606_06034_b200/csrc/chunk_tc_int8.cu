@@ -104,6 +104,12 @@ __device__ __forceinline__ T rsr_t(T x, int r) {  // r >= 0; (1 << r) >> 1 is th
     const T q = (a + ((static_cast<T>(1) << r) >> 1)) >> r;
     return x < 0 ? -q : q;
 }
+// 32-bit form without branches (see q8_32)
+__device__ __forceinline__ int rsr32(int x, int r) {
+    const int half = static_cast<int>((1u << r) >> 1);
+    const int neg1 = (r > 0) ? (x >> 31) : 0;
+    return (x + half + neg1) >> r;
+}
 template <typename T>
 __device__ __forceinline__ T shift_t(T x, int s) { return s >= 0 ? (x << s) : rsr_t<T>(x, -s); }
 // One term of an aligned sum: x 2^s for s >= 0, rounded right shift otherwise. x fits 23 bits, so the right
@@ -111,16 +117,16 @@ __device__ __forceinline__ T shift_t(T x, int s) { return s >= 0 ? (x << s) : rs
 template <typename T>
 __device__ __forceinline__ T term_t(int x, int s) {
     if (s >= 0) return static_cast<T>(x) << s;
-    return static_cast<T>(rsr_t<int>(x, (-s) < 31 ? (-s) : 31));
+    return static_cast<T>(rsr32(x, (-s) < 31 ? (-s) : 31));
 }
 __device__ __forceinline__ int term32(int x, int s) { return term_t<int>(x, s); }
-// clamp(rsr(x, r), +-127) for 32-bit x
+// clamp(rsr(x, r), +-127) for 32-bit x, branch-free: for x < 0 the rounded magnitude shift equals the arithmetic
+// shift of x + half - 1 (floor((x + h - 1) / 2^r) = -floor((|x| + h) / 2^r) because 2^r - h = h); r = 0 gives x.
 __device__ __forceinline__ int q8_32(int x, int r) {
-    const int sgn = x >> 31;
-    int a = (x ^ sgn) - sgn;
-    a = (a + ((1 << r) >> 1)) >> r;
-    a = a > 127 ? 127 : a;
-    return (a ^ sgn) - sgn;
+    const int half = static_cast<int>((1u << r) >> 1);
+    const int neg1 = (r > 0) ? (x >> 31) : 0;  // -1 for negative x when something is shifted out
+    const int y = (x + half + neg1) >> r;
+    return max(min(y, 127), -127);
 }
 template <typename T>
 __device__ __forceinline__ unsigned long long abs_bits(T x) { return static_cast<unsigned long long>(x < 0 ? -x : x); }
@@ -133,11 +139,24 @@ __device__ __forceinline__ int align_ref2(int e0, int e1) {
     const int lo = e0 < e1 ? e0 : e1, hi = e0 < e1 ? e1 : e0;
     return lo > hi - kAlignWindow ? lo : hi - kAlignWindow;
 }
-__device__ __forceinline__ uint32_t pack4(int a, int b, int c, int d) {
-    return (static_cast<uint32_t>(a) & 0xFFu) | ((static_cast<uint32_t>(b) & 0xFFu) << 8) | ((static_cast<uint32_t>(c) & 0xFFu) << 16) |
-           ((static_cast<uint32_t>(d) & 0xFFu) << 24);
+// prmt.b32 in its default mode: nibble n of `sel` picks the source byte of result byte n (0-3 from a, 4-7 from b);
+// bit 3 of the nibble replicates that byte's sign bit instead of copying the byte
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
 }
-__device__ __forceinline__ int byte_at(uint32_t w, int i) { return static_cast<int>(static_cast<int8_t>((w >> (8 * i)) & 0xFFu)); }
+// low bytes of four ints -> one word (three byte permutes)
+__device__ __forceinline__ uint32_t pack4(int a, int b, int c, int d) {
+    const uint32_t ab = prmt(static_cast<uint32_t>(a), static_cast<uint32_t>(b), 0x0040u);
+    const uint32_t cd = prmt(static_cast<uint32_t>(c), static_cast<uint32_t>(d), 0x0040u);
+    return prmt(ab, cd, 0x5410u);
+}
+// byte i of w, sign-extended (one byte permute: selector 8|i replicates the sign of byte i)
+__device__ __forceinline__ int byte_at(uint32_t w, int i) {
+    const uint32_t sx = 8u | static_cast<uint32_t>(i);
+    return static_cast<int>(prmt(w, 0u, (sx << 12) | (sx << 8) | (sx << 4) | static_cast<uint32_t>(i)));
+}
 
 struct TileCoord {
     int bhk, bhv, t0;
@@ -305,8 +324,12 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             uint32_t g[kHC];
             tmem_ld32(lane_base + kR0 + cb + col0, g);
             tmem_wait_ld();
-            int cq[kHC];  // c_ij = (beta_q_i Gam_ij + 2^14) >> 15, 0 on and above the diagonal
-            unsigned long long m = 0;
+            // c_ij = (beta_q_i Gam_ij + 2^14) >> 15 (< 2^15), 0 on and above the diagonal. |G| < 2^21, so |G| c needs
+            // 36 bits: it is kept as a (hi, lo) pair of 32-bit words; the shift r = bitlen - 7 stays below 32, so the
+            // rounded shift is one funnel shift of the pair. Aq = -G c: the sign is restored at the end (the rounding
+            // rule is symmetric).
+            int cq[kHC];
+            uint32_t mlo = 0, mhi = 0;
 #pragma unroll
             for (int jl = 0; jl < kHC; ++jl) {
                 const int j = col0 + jl;
@@ -315,12 +338,21 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 const int gam = (sh >= 0 && sh < 16) ? (static_cast<int>(slut[dlt & 255]) >> sh) : 0;
                 const int c = (j < il) ? ((bq * gam + (1 << 14)) >> 15) : 0;
                 cq[jl] = c;
-                m |= abs_bits<long long>(static_cast<long long>(static_cast<int>(g[jl])) * c);
+                const uint32_t ag = static_cast<uint32_t>(abs(static_cast<int>(g[jl])));
+                mlo |= ag * static_cast<uint32_t>(c);
+                mhi |= __umulhi(ag, static_cast<uint32_t>(c));
             }
-            const int r = q8_shift(chunk_bitlen(m, slot++));
+            const int r = q8_shift(chunk_bitlen((static_cast<unsigned long long>(mhi) << 32) | mlo, slot++));
+            const uint32_t half = (1u << r) >> 1;
 #pragma unroll
-            for (int jl = 0; jl < kHC; ++jl)
-                aq[jl] = clamp127_t<long long>(rsr_t<long long>(-static_cast<long long>(static_cast<int>(g[jl])) * cq[jl], r));
+            for (int jl = 0; jl < kHC; ++jl) {
+                const int gv = static_cast<int>(g[jl]);
+                const uint32_t ag = static_cast<uint32_t>(abs(gv)), c = static_cast<uint32_t>(cq[jl]);
+                const uint32_t lo = ag * c, lo2 = lo + half;
+                const uint32_t hi2 = __umulhi(ag, c) + (lo2 < lo ? 1u : 0u);
+                const int q = static_cast<int>(min(__funnelshift_r(lo2, hi2, r), 127u));
+                aq[jl] = (gv < 0) ? q : -q;
+            }
             eA = 2 * kexp - 15 + r;
         }
         STAMP8(3);
@@ -486,13 +518,10 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             tmem_ld32(lane_base + kR0 + cb + col0, dres);
             tmem_wait_ld();
             unsigned long long m = 0;
-            const int dmin = s * (N + 1);
+            // R_{s-1} is zero for i - j < (s - 1)(N + 1) and Eq for i - j <= N: the integer product is exactly zero
+            // for i - j < s (N + 1), no mask needed
 #pragma unroll
-            for (int jl = 0; jl < kHC; ++jl) {
-                const int v = (il - (col0 + jl) >= dmin) ? static_cast<int>(dres[jl]) : 0;
-                dres[jl] = static_cast<uint32_t>(v);
-                m |= abs_bits<int>(v);
-            }
+            for (int jl = 0; jl < kHC; ++jl) m |= abs_bits<int>(static_cast<int>(dres[jl]));
             const int r = q8_shift(chunk_bitlen(m, slot++));
 #pragma unroll
             for (int w = 0; w < kHC / 4; ++w)
@@ -529,7 +558,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                     for (int jl = 0; jl < kHC; ++jl) acc[jl] += byte_at(rpk[s][jl >> 2], jl & 3) << sh[s];
                 } else if (sh[s] >= -7) {
 #pragma unroll
-                    for (int jl = 0; jl < kHC; ++jl) acc[jl] += rsr_t<int>(byte_at(rpk[s][jl >> 2], jl & 3), -sh[s]);
+                    for (int jl = 0; jl < kHC; ++jl) acc[jl] += rsr32(byte_at(rpk[s][jl >> 2], jl & 3), -sh[s]);
                 }
             }
             unsigned long long m = 0;
