@@ -128,6 +128,7 @@ __device__ __forceinline__ int q8_32(int x, int r) {
     const int y = (x + half + neg1) >> r;
     return max(min(y, 127), -127);
 }
+__device__ __forceinline__ uint32_t abs32(int x) { return static_cast<uint32_t>(abs(x)); }
 template <typename T>
 __device__ __forceinline__ unsigned long long abs_bits(T x) { return static_cast<unsigned long long>(x < 0 ? -x : x); }
 template <typename T>
@@ -255,7 +256,14 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             (static_cast<unsigned long long>(sred[(slot * 2 + ci) * 2 + 1]) << 32) | sred[(slot * 2 + ci) * 2 + 0];
         return all ? 64 - __clzll(static_cast<long long>(all)) : 0;
     };
-    auto absll = [](long long x) -> unsigned long long { return static_cast<unsigned long long>(x < 0 ? -x : x); };
+    // the same for values known to fit 32 bits (one warp reduction, one shared-memory atomic)
+    auto chunk_bitlen32 = [&](uint32_t m, int slot) -> int {
+        const uint32_t lo = __reduce_or_sync(0xFFFFFFFFu, m);
+        if (lane == 0 && lo) atomicOr(&sred[(slot * 2 + ci) * 2 + 0], lo);
+        cta_barrier();
+        const uint32_t all = sred[(slot * 2 + ci) * 2 + 0];
+        return 32 - __clz(static_cast<int>(all));
+    };
 
     if (tid == 0 && blockIdx.x < n_tiles) {
         const TileCoord c = decode_tile(blockIdx.x, p);
@@ -399,8 +407,8 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             int p22 = 0, p23 = 0, p33 = 0;
             int e2 = 0, e3 = 0;
             if (N >= 2) {
-                const unsigned long long m = (h == 0) ? (abs_bits<int>(acc22) | abs_bits<int>(acc23)) : 0ull;
-                const int r = q8_shift(chunk_bitlen(m, slot++));
+                const uint32_t m = (h == 0) ? (abs32(acc22) | abs32(acc23)) : 0u;
+                const int r = q8_shift(chunk_bitlen32(m, slot++));
                 p22 = q8_32(acc22, r);
                 p23 = q8_32(acc23, r);
                 e2 = eA + eA + r;
@@ -408,7 +416,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             if (N >= 3) {
                 // P_3 at distance 3: P_2[i][i-2] * Aq[i-2][i-3]
                 const int acc3 = p22 * sAB[r2 * 8 + 1];
-                const int r = q8_shift(chunk_bitlen((h == 0) ? abs_bits<int>(acc3) : 0ull, slot++));
+                const int r = q8_shift(chunk_bitlen32((h == 0) ? abs32(acc3) : 0u, slot++));
                 p33 = q8_32(acc3, r);
                 e3 = e2 + eA + r;
             }
@@ -424,8 +432,8 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             if (!(N >= 1 && il >= 1)) a1 = 0;
             if (!(N >= 2 && il >= 2)) a2 = 0;
             if (!(N >= 3 && il >= 3)) a3 = 0;
-            const unsigned long long m = (h == 0) ? (abs_bits<int>(a1) | abs_bits<int>(a2) | abs_bits<int>(a3)) : 0ull;
-            const int r = q8_shift(chunk_bitlen(m, slot++));
+            const uint32_t m = (h == 0) ? (abs32(a1) | abs32(a2) | abs32(a3)) : 0u;
+            const int r = q8_shift(chunk_bitlen32(m, slot++));
             t0q1 = q8_32(a1, r);
             t0q2 = q8_32(a2, r);
             t0q3 = q8_32(a3, r);
@@ -447,7 +455,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             const int sa = eA - eref, sp = eA + eT0 - eref;
             int acc[kHC];  // |Aq| < 2^7 and |Aq T0q| <= 3 * 127^2 < 2^16, shifted left by at most 8
             const bool left = sa >= 0 && sp >= 0;
-            unsigned long long m = 0;
+            uint32_t m = 0;
 #pragma unroll
             for (int jl = 0; jl < kHC; ++jl) {
                 const int4 c4 = *reinterpret_cast<const int4*>(sSH + (cb + col0 + jl) * 4);
@@ -458,9 +466,9 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 const int pr = a1 * c4.x + a2 * c4.y + a3 * c4.z;
                 const int v = on ? (left ? ((aq[jl] << sa) + (pr << sp)) : (term32(aq[jl], sa) + term32(pr, sp))) : 0;
                 acc[jl] = v;
-                m |= abs_bits<int>(v);
+                m |= abs32(v);
             }
-            const int r = q8_shift(chunk_bitlen(m, slot++));
+            const int r = q8_shift(chunk_bitlen32(m, slot++));
 #pragma unroll
             for (int jl = 0; jl < kHC; ++jl) eq[jl] = q8_32(acc[jl], r);
             eE = eref + r;
@@ -517,12 +525,12 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             uint32_t dres[kHC];
             tmem_ld32(lane_base + kR0 + cb + col0, dres);
             tmem_wait_ld();
-            unsigned long long m = 0;
+            uint32_t m = 0;
             // R_{s-1} is zero for i - j < (s - 1)(N + 1) and Eq for i - j <= N: the integer product is exactly zero
             // for i - j < s (N + 1), no mask needed
 #pragma unroll
-            for (int jl = 0; jl < kHC; ++jl) m |= abs_bits<int>(static_cast<int>(dres[jl]));
-            const int r = q8_shift(chunk_bitlen(m, slot++));
+            for (int jl = 0; jl < kHC; ++jl) m |= abs32(static_cast<int>(dres[jl]));
+            const int r = q8_shift(chunk_bitlen32(m, slot++));
 #pragma unroll
             for (int w = 0; w < kHC / 4; ++w)
                 rpk[s - 1][w] = pack4(q8_32(static_cast<int>(dres[4 * w]), r),
@@ -561,10 +569,10 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                     for (int jl = 0; jl < kHC; ++jl) acc[jl] += rsr32(byte_at(rpk[s][jl >> 2], jl & 3), -sh[s]);
                 }
             }
-            unsigned long long m = 0;
+            uint32_t m = 0;
 #pragma unroll
-            for (int jl = 0; jl < kHC; ++jl) m |= abs_bits<int>(acc[jl]);
-            const int r = q8_shift(chunk_bitlen(m, slot++));
+            for (int jl = 0; jl < kHC; ++jl) m |= abs32(acc[jl]);
+            const int r = q8_shift(chunk_bitlen32(m, slot++));
 #pragma unroll
             for (int jl = 0; jl < kHC; ++jl) sq[jl] = q8_32(acc[jl], r);
             eS = eref + r;
@@ -611,7 +619,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             // element with its own shift; entries below 2^7, the product below 3 * 127^2 < 2^16
             const bool left = s0 >= 0 && s1 >= 0 && s2 >= 0;
             int acc[kHC];
-            unsigned long long m = 0;
+            uint32_t m = 0;
 #pragma unroll
             for (int jl = 0; jl < kHC; ++jl) {
                 const int d = il - (col0 + jl);
@@ -623,9 +631,9 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                                               : (term32(v, (d <= N) ? s0 : s1) + term32(prod[jl], s2)))
                                       : 0;
                 acc[jl] = a;
-                m |= abs_bits<int>(a);
+                m |= abs32(a);
             }
-            const int r = q8_shift(chunk_bitlen(m, slot++));
+            const int r = q8_shift(chunk_bitlen32(m, slot++));
 #pragma unroll
             for (int jl = 0; jl < kHC; ++jl) toff[jl] = q8_32(acc[jl], r);
             eT = eref + r;
@@ -636,13 +644,13 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
         int eTb;
         {
             int acc[kHC];
-            unsigned long long m = 0;
+            uint32_t m = 0;
 #pragma unroll
             for (int jl = 0; jl < kHC; ++jl) {
                 acc[jl] = toff[jl] * sbeta[cb + col0 + jl];
-                m |= abs_bits<int>(acc[jl]);
+                m |= abs32(acc[jl]);
             }
-            const int r = q8_shift(chunk_bitlen(m, slot++));
+            const int r = q8_shift(chunk_bitlen32(m, slot++));
             uint32_t r8[8];
 #pragma unroll
             for (int w = 0; w < 8; ++w)
@@ -712,23 +720,25 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             // |Tbq Xq| <= 128 * 127^2 < 2^21, |beta_q Xq| < 2^22; at most one of them is shifted left, by at most 8
             // pass 1: the scale (bit length of the largest magnitude over the chunk's C x d block)
             const bool left = sp >= 0 && sd >= 0;  // the usual case: plain left shifts
-            unsigned long long m = 0;
+            const int psc = left ? (1 << sp) : 0, bqs = left ? (bq << sd) : 0;
+            uint32_t m = 0;
 #pragma unroll
             for (int c0 = 0; c0 < 64; c0 += 32) {
                 uint32_t r[32];
                 tmem_ld32(lane_base + kR0 + h * 64 + c0, r);
                 tmem_wait_ld();
                 if (left) {
+                    // shifts folded into the multipliers: two multiply-adds per element
 #pragma unroll
                     for (int i = 0; i < 32; ++i)
-                        m |= abs_bits<int>((static_cast<int>(r[i]) << sp) + ((bq * byte_at(xr[(c0 + i) >> 2], (c0 + i) & 3)) << sd));
+                        m |= abs32(static_cast<int>(r[i]) * psc + byte_at(xr[(c0 + i) >> 2], (c0 + i) & 3) * bqs);
                 } else {
 #pragma unroll
                     for (int i = 0; i < 32; ++i)
-                        m |= abs_bits<int>(term32(static_cast<int>(r[i]), sp) + term32(bq * byte_at(xr[(c0 + i) >> 2], (c0 + i) & 3), sd));
+                        m |= abs32(term32(static_cast<int>(r[i]), sp) + term32(bq * byte_at(xr[(c0 + i) >> 2], (c0 + i) & 3), sd));
                 }
             }
-            const int rr = q8_shift(chunk_bitlen(m, slot++));
+            const int rr = q8_shift(chunk_bitlen32(m, slot++));
             // after that barrier every thread holds its own row of the K (V) tile in registers, and the products that
             // read the tile are complete: the next tile's K (V) may land
             if (tid == 0 && has_next) {
@@ -757,7 +767,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 if (left) {
 #pragma unroll
                     for (int i = 0; i < 32; ++i)
-                        qv[i] = q8_32((static_cast<int>(r[i]) << sp) + ((bq * byte_at(xr[(c0 + i) >> 2], (c0 + i) & 3)) << sd), rr);
+                        qv[i] = q8_32(static_cast<int>(r[i]) * psc + byte_at(xr[(c0 + i) >> 2], (c0 + i) & 3) * bqs, rr);
                 } else {
 #pragma unroll
                     for (int i = 0; i < 32; ++i)
