@@ -120,13 +120,36 @@ __device__ __forceinline__ T term_t(int x, int s) {
     return static_cast<T>(rsr32(x, (-s) < 31 ? (-s) : 31));
 }
 __device__ __forceinline__ int term32(int x, int s) { return term_t<int>(x, s); }
-// clamp(rsr(x, r), +-127) for 32-bit x, branch-free: for x < 0 the rounded magnitude shift equals the arithmetic
-// shift of x + half - 1 (floor((x + h - 1) / 2^r) = -floor((|x| + h) / 2^r) because 2^r - h = h); r = 0 gives x.
-__device__ __forceinline__ int q8_32(int x, int r) {
-    const int half = static_cast<int>((1u << r) >> 1);
-    const int neg1 = (r > 0) ? (x >> 31) : 0;  // -1 for negative x when something is shifted out
-    const int y = (x + half + neg1) >> r;
-    return max(min(y, 127), -127);
+// Rounding constants of one requantisation (uniform over a chunk): shift, rounding half, and an all-ones mask when
+// something is shifted out.
+struct Rnd {
+    int r, half, mask;
+};
+__device__ __forceinline__ Rnd make_rnd(int r) {
+    Rnd q;
+    q.r = r;
+    q.half = static_cast<int>((1u << r) >> 1);
+    q.mask = (r > 0) ? -1 : 0;
+    return q;
+}
+// rsr(x, r), branch-free: for x < 0 the rounded magnitude shift equals the arithmetic shift of x + half - 1
+// (floor((x + h - 1) / 2^r) = -floor((|x| + h) / 2^r) because 2^r - h = h); r = 0 gives x.
+__device__ __forceinline__ int rsr_rnd(int x, const Rnd& q) { return (x + q.half + ((x >> 31) & q.mask)) >> q.r; }
+// clamp(rsr(x, r), +-127)
+__device__ __forceinline__ int q8_32(int x, const Rnd& q) { return max(min(rsr_rnd(x, q), 127), -127); }
+__device__ __forceinline__ int q8_32(int x, int r) { return q8_32(x, make_rnd(r)); }
+// cvt.pack.sat.s8.s32.b32: d[7:0] = sat8(b), d[15:8] = sat8(a), d[31:16] = c[15:0]
+__device__ __forceinline__ uint32_t pack_sat_s8(int a, int b, uint32_t c) {
+    uint32_t d;
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+// four requantised values as one word of int8: the lower clamp (-127) is explicit, the upper one (127) is the
+// saturation of the pack (rsr never exceeds 128 in magnitude here)
+__device__ __forceinline__ uint32_t q8_pack4(int x0, int x1, int x2, int x3, const Rnd& q) {
+    const int y0 = max(rsr_rnd(x0, q), -127), y1 = max(rsr_rnd(x1, q), -127);
+    const int y2 = max(rsr_rnd(x2, q), -127), y3 = max(rsr_rnd(x3, q), -127);
+    return pack_sat_s8(y1, y0, pack_sat_s8(y3, y2, 0u));
 }
 __device__ __forceinline__ uint32_t abs32(int x) { return static_cast<uint32_t>(abs(x)); }
 template <typename T>
@@ -469,8 +492,9 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 m |= abs32(v);
             }
             const int r = q8_shift(chunk_bitlen32(m, slot++));
+            const Rnd rq = make_rnd(r);
 #pragma unroll
-            for (int jl = 0; jl < kHC; ++jl) eq[jl] = q8_32(acc[jl], r);
+            for (int jl = 0; jl < kHC; ++jl) eq[jl] = q8_32(acc[jl], rq);
             eE = eref + r;
         }
         STAMP8(6);
@@ -531,12 +555,11 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
 #pragma unroll
             for (int jl = 0; jl < kHC; ++jl) m |= abs32(static_cast<int>(dres[jl]));
             const int r = q8_shift(chunk_bitlen32(m, slot++));
+            const Rnd rq = make_rnd(r);
 #pragma unroll
             for (int w = 0; w < kHC / 4; ++w)
-                rpk[s - 1][w] = pack4(q8_32(static_cast<int>(dres[4 * w]), r),
-                                      q8_32(static_cast<int>(dres[4 * w + 1]), r),
-                                      q8_32(static_cast<int>(dres[4 * w + 2]), r),
-                                      q8_32(static_cast<int>(dres[4 * w + 3]), r));
+                rpk[s - 1][w] = q8_pack4(static_cast<int>(dres[4 * w]), static_cast<int>(dres[4 * w + 1]),
+                                         static_cast<int>(dres[4 * w + 2]), static_cast<int>(dres[4 * w + 3]), rq);
             er[s - 1] = er[s - 2] + eE + r;
             n_terms = s;
         }
@@ -573,8 +596,9 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
 #pragma unroll
             for (int jl = 0; jl < kHC; ++jl) m |= abs32(acc[jl]);
             const int r = q8_shift(chunk_bitlen32(m, slot++));
+            const Rnd rq = make_rnd(r);
 #pragma unroll
-            for (int jl = 0; jl < kHC; ++jl) sq[jl] = q8_32(acc[jl], r);
+            for (int jl = 0; jl < kHC; ++jl) sq[jl] = q8_32(acc[jl], rq);
             eS = eref + r;
         } else {
 #pragma unroll
@@ -634,8 +658,9 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 m |= abs32(a);
             }
             const int r = q8_shift(chunk_bitlen32(m, slot++));
+            const Rnd rq = make_rnd(r);
 #pragma unroll
-            for (int jl = 0; jl < kHC; ++jl) toff[jl] = q8_32(acc[jl], r);
+            for (int jl = 0; jl < kHC; ++jl) toff[jl] = q8_32(acc[jl], rq);
             eT = eref + r;
         }
 
@@ -651,11 +676,11 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 m |= abs32(acc[jl]);
             }
             const int r = q8_shift(chunk_bitlen32(m, slot++));
+            const Rnd rq9 = make_rnd(r);
             uint32_t r8[8];
 #pragma unroll
             for (int w = 0; w < 8; ++w)
-                r8[w] = pack4(q8_32(acc[4 * w], r), q8_32(acc[4 * w + 1], r),
-                              q8_32(acc[4 * w + 2], r), q8_32(acc[4 * w + 3], r));
+                r8[w] = q8_pack4(acc[4 * w], acc[4 * w + 1], acc[4 * w + 2], acc[4 * w + 3], rq9);
             eTb = eT - 15 + r;
             // row t's block occupies packed columns [cb/4, cb/4 + 16) of a 32-column operand; the other 16 are zero
             tmem_st8(lane_base + kAS + cb / 4 + h * 8, r8);
@@ -739,6 +764,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 }
             }
             const int rr = q8_shift(chunk_bitlen32(m, slot++));
+            const Rnd rqw = make_rnd(rr);
             // after that barrier every thread holds its own row of the K (V) tile in registers, and the products that
             // read the tile are complete: the next tile's K (V) may land
             if (tid == 0 && has_next) {
@@ -763,23 +789,23 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 uint32_t r[32];
                 tmem_ld32(lane_base + kR0 + h * 64 + c0, r);
                 tmem_wait_ld();
-                int qv[32];
+                int qv[32];  // the sums before requantisation
                 if (left) {
 #pragma unroll
                     for (int i = 0; i < 32; ++i)
-                        qv[i] = q8_32(static_cast<int>(r[i]) * psc + byte_at(xr[(c0 + i) >> 2], (c0 + i) & 3) * bqs, rr);
+                        qv[i] = static_cast<int>(r[i]) * psc + byte_at(xr[(c0 + i) >> 2], (c0 + i) & 3) * bqs;
                 } else {
 #pragma unroll
                     for (int i = 0; i < 32; ++i)
-                        qv[i] = q8_32(term32(static_cast<int>(r[i]), sp) + term32(bq * byte_at(xr[(c0 + i) >> 2], (c0 + i) & 3), sd), rr);
+                        qv[i] = term32(static_cast<int>(r[i]), sp) + term32(bq * byte_at(xr[(c0 + i) >> 2], (c0 + i) & 3), sd);
                 }
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
                     const int cc = c0 / 16 + c;
-                    const uint4 v = make_uint4(pack4(qv[16 * c + 0], qv[16 * c + 1], qv[16 * c + 2], qv[16 * c + 3]),
-                                               pack4(qv[16 * c + 4], qv[16 * c + 5], qv[16 * c + 6], qv[16 * c + 7]),
-                                               pack4(qv[16 * c + 8], qv[16 * c + 9], qv[16 * c + 10], qv[16 * c + 11]),
-                                               pack4(qv[16 * c + 12], qv[16 * c + 13], qv[16 * c + 14], qv[16 * c + 15]));
+                    const uint4 v = make_uint4(q8_pack4(qv[16 * c + 0], qv[16 * c + 1], qv[16 * c + 2], qv[16 * c + 3], rqw),
+                                               q8_pack4(qv[16 * c + 4], qv[16 * c + 5], qv[16 * c + 6], qv[16 * c + 7], rqw),
+                                               q8_pack4(qv[16 * c + 8], qv[16 * c + 9], qv[16 * c + 10], qv[16 * c + 11], rqw),
+                                               q8_pack4(qv[16 * c + 12], qv[16 * c + 13], qv[16 * c + 14], qv[16 * c + 15], rqw));
                     *reinterpret_cast<uint4*>(sub + lane * 64 + ((cc ^ ((lane >> 1) & 3)) << 4)) = v;
                 }
             }
