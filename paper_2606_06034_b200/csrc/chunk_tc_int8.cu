@@ -747,6 +747,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             const bool left = sp >= 0 && sd >= 0;  // the usual case: plain left shifts
             const int psc = left ? (1 << sp) : 0, bqs = left ? (bq << sd) : 0;
             uint32_t m = 0;
+            int sums[64];  // the aligned sums of this thread's 64 columns stay in registers between the two passes
 #pragma unroll
             for (int c0 = 0; c0 < 64; c0 += 32) {
                 uint32_t r[32];
@@ -756,12 +757,14 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                     // shifts folded into the multipliers: two multiply-adds per element
 #pragma unroll
                     for (int i = 0; i < 32; ++i)
-                        m |= abs32(static_cast<int>(r[i]) * psc + byte_at(xr[(c0 + i) >> 2], (c0 + i) & 3) * bqs);
+                        sums[c0 + i] = static_cast<int>(r[i]) * psc + byte_at(xr[(c0 + i) >> 2], (c0 + i) & 3) * bqs;
                 } else {
 #pragma unroll
                     for (int i = 0; i < 32; ++i)
-                        m |= abs32(term32(static_cast<int>(r[i]), sp) + term32(bq * byte_at(xr[(c0 + i) >> 2], (c0 + i) & 3), sd));
+                        sums[c0 + i] = term32(static_cast<int>(r[i]), sp) + term32(bq * byte_at(xr[(c0 + i) >> 2], (c0 + i) & 3), sd);
                 }
+#pragma unroll
+                for (int i = 0; i < 32; ++i) m |= abs32(sums[c0 + i]);
             }
             const int rr = q8_shift(chunk_bitlen32(m, slot++));
             const Rnd rqw = make_rnd(rr);
@@ -786,19 +789,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             __syncwarp();
 #pragma unroll
             for (int c0 = 0; c0 < 64; c0 += 32) {
-                uint32_t r[32];
-                tmem_ld32(lane_base + kR0 + h * 64 + c0, r);
-                tmem_wait_ld();
-                int qv[32];  // the sums before requantisation
-                if (left) {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        qv[i] = static_cast<int>(r[i]) * psc + byte_at(xr[(c0 + i) >> 2], (c0 + i) & 3) * bqs;
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        qv[i] = term32(static_cast<int>(r[i]), sp) + term32(bq * byte_at(xr[(c0 + i) >> 2], (c0 + i) & 3), sd);
-                }
+                const int* qv = sums + c0;
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
                     const int cc = c0 / 16 + c;
@@ -811,7 +802,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             }
             if (half == 0) {
                 tc_fence_before_sync();
-                cta_barrier();  // every row of the W accumulator has been read twice
+                cta_barrier();  // every row of the W accumulator has been read
                 if (tid == 0) {
                     if (!wait_bar(&bar_v, par_kv)) ok = false;
                     if (ok) {
