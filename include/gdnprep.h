@@ -129,13 +129,17 @@ int gdn_chunk_prepare_fwdsubst(const void* K, const void* V, const float* beta, 
  *   non-decreasing inside every chunk (not checked).
  *   Wq_out [B,H_v,T,d_k], Uq_out [B,H_v,T,d_v] int8 with w_exp_out, u_exp_out [B,H_v,T/C];
  *   Toff_q_out [B,H_v,T/C,C,C] int8 (may be NULL) with t_exp_out [B,H_v,T/C]: T = I + Toff_q * 2^t_exp.
+ *   dbg_acc_out (may be NULL; meant for small cases): every int32 tensor-core accumulator of the chain,
+ *   [B,H_v,T/C, C, 8*C + d_k + d_v] int32. Row i of a chunk holds: columns [0, C) the Gram row Kq Kq^T;
+ *   columns [(s-1)*C, s*C) for s = 2..8 the row of the power product R_{s-1} Eq (left untouched for powers
+ *   that the parameters skip: the caller zeroes the buffer); then d_k columns of Tbq Kq and d_v of Tbq Vq.
  * Supported: C = 64, d_k = d_v = 128, 1 <= order <= 3 (the paper's low-bit limit), residual_steps <= 8.
  */
 int gdn_chunk_prepare_int8(const int8_t* Kq, const int8_t* Vq, const int32_t* k_exp, const int32_t* v_exp,
                            const uint16_t* beta_q, const int32_t* decay_q,
                            int B, int H_k, int H_v, int T, int C, int d_k, int d_v, int order, int residual_steps,
                            int8_t* Wq_out, int8_t* Uq_out, int32_t* w_exp_out, int32_t* u_exp_out,
-                           int8_t* Toff_q_out, int32_t* t_exp_out, gdn_stream_t stream);
+                           int8_t* Toff_q_out, int32_t* t_exp_out, int32_t* dbg_acc_out, gdn_stream_t stream);
 
 /* Checksum of the 256-entry gate-decay table round(2^15 * 2^(-f/256)) the INT8 kernel uses
  * (sum_f: s = (31 s + table[f] + f) mod 1000000007), so that a CPU evaluation can confirm it holds the same table. */

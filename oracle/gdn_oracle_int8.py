@@ -297,6 +297,7 @@ def chunk_prepare_int8(Kq, Vq, k_exp, v_exp, beta_q, decay_q, N: int, S: int):
     Eq, eE = _q8_np(accE, eref, far)
     # I7
     R = []
+    acc_R = {}  # s -> the int32 product R_{s-1} Eq before requantisation
     if S >= 1:
         R.append((Eq, eE))
         for s in range(2, S + 1):
@@ -304,7 +305,8 @@ def chunk_prepare_int8(Kq, Vq, k_exp, v_exp, beta_q, decay_q, N: int, S: int):
                 break
             sup = d >= s * (N + 1)
             prev, eprev = R[-1]
-            Rs, es = _q8_np(_mm_i32(prev, Eq), eprev + eE, sup)
+            acc_R[s] = _mm_i32(prev, Eq)
+            Rs, es = _q8_np(acc_R[s], eprev + eE, sup)
             R.append((Rs, es))
     if R:
         accS, eref = _align_np(R, far)
@@ -323,11 +325,21 @@ def chunk_prepare_int8(Kq, Vq, k_exp, v_exp, beta_q, decay_q, N: int, S: int):
         prod = _mm_i32(Tbq, Xq)
         diag = beta_q[:, :, None] * Xq
         acc, er = _align_np([(prod, eTb + x_exp), (diag, x_exp - 15)], full)
-        return _q8_np(acc, er, full)
+        return _q8_np(acc, er, full) + (prod,)
 
-    Wq, eW = out_rows(Kq, k_exp)
-    Uq, eU = out_rows(Vq, v_exp)
-    return {"Wq": Wq.astype(np.int8), "w_exp": eW, "Uq": Uq.astype(np.int8), "u_exp": eU,
+    Wq, eW, acc_W = out_rows(Kq, k_exp)
+    Uq, eU, acc_U = out_rows(Vq, v_exp)
+    # the matrix products an implementation is expected to run on integer matrix units, before any rounding:
+    # Gram rows, the power products R_{s-1} Eq (s = 2..8, zeros where skipped), Tbq Kq and Tbq Vq
+    acc_all = np.zeros((n, C, 8 * C + dk + Vq.shape[-1]), dtype=np.int64)
+    acc_all[:, :, :C] = G
+    for s_, prod_ in acc_R.items():
+        if s_ <= 8:
+            acc_all[:, :, (s_ - 1) * C:s_ * C] = prod_
+    acc_all[:, :, 8 * C:8 * C + dk] = acc_W
+    acc_all[:, :, 8 * C + dk:] = acc_U
+    return {"acc": acc_all,
+            "Wq": Wq.astype(np.int8), "w_exp": eW, "Uq": Uq.astype(np.int8), "u_exp": eU,
             "Toffq": Toffq.astype(np.int8), "t_exp": eT, "Aq": Aq.astype(np.int8), "a_exp": eA,
             "Eq": Eq.astype(np.int8), "e_exp": eE, "T0q": T0q.astype(np.int8), "t0_exp": eT0}
 

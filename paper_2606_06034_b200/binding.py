@@ -68,7 +68,7 @@ def load_library() -> ctypes.CDLL:
     lib.gdn_chunk_prepare_fwdsubst.restype = ip
     lib.gdn_chunk_prepare_fwdsubst.argtypes = [vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ip, ip, ip, vp, vp, vp, vp]
     lib.gdn_chunk_prepare_int8.restype = ip
-    lib.gdn_chunk_prepare_int8.argtypes = [vp, vp, vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ip, ip, ip, vp, vp, vp, vp, vp, vp, vp]
+    lib.gdn_chunk_prepare_int8.argtypes = [vp, vp, vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ip, ip, ip, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.gdn_int8_lut_checksum.restype = ctypes.c_uint
     lib.gdn_int8_lut_checksum.argtypes = []
     lib.gdn_device_status.restype = ip
@@ -186,7 +186,7 @@ def gdn_int8_lut_checksum() -> int:
 
 
 def gdn_chunk_prepare_int8(Kq, Vq, k_exp, v_exp, beta_q, decay_q, B, H_k, H_v, T, C, d_k, d_v, order, residual_steps,
-                           Wq_out, Uq_out, w_exp_out, u_exp_out, Toff_q_out, t_exp_out, *, check=True):
+                           Wq_out, Uq_out, w_exp_out, u_exp_out, Toff_q_out, t_exp_out, dbg_acc_out=None, *, check=True):
     """Raw call of the INT8 entry point (tensors instead of pointers, torch's current stream)."""
     for t in (Kq, Vq, k_exp, v_exp, beta_q, decay_q, Wq_out, Uq_out, w_exp_out, u_exp_out, t_exp_out):
         if not t.is_cuda or not t.is_contiguous():
@@ -194,16 +194,17 @@ def gdn_chunk_prepare_int8(Kq, Vq, k_exp, v_exp, beta_q, decay_q, B, H_k, H_v, T
     rc = load_library().gdn_chunk_prepare_int8(_ptr(Kq), _ptr(Vq), _ptr(k_exp), _ptr(v_exp), _ptr(beta_q), _ptr(decay_q),
                                                B, H_k, H_v, T, C, d_k, d_v, order, residual_steps, _ptr(Wq_out),
                                                _ptr(Uq_out), _ptr(w_exp_out), _ptr(u_exp_out), _ptr(Toff_q_out),
-                                               _ptr(t_exp_out), _stream())
+                                               _ptr(t_exp_out), _ptr(dbg_acc_out), _stream())
     if check and rc != GDN_OK:
         raise GdnError(rc, "gdn_chunk_prepare_int8")
     return rc
 
 
-def chunk_prepare_int8(q, order=-1, residual_steps=-1, *, want_toff=True, outputs=None):
+def chunk_prepare_int8(q, order=-1, residual_steps=-1, *, want_toff=True, outputs=None, dbg_acc=None):
     """Convenience wrapper over integer inputs (an `inputs.Int8Inputs` whose tensors live on the GPU).
 
-    Returns (Wq, Uq, w_exp, u_exp, Toff_q, t_exp).
+    Returns (Wq, Uq, w_exp, u_exp, Toff_q, t_exp). `dbg_acc`: optional zeroed int32 tensor
+    [B, H_v, T/C, C, 8*C + d_k + d_v] that receives the tensor-core accumulators (small cases).
     """
     dev = q.Kq.device
     n_c = q.T // q.C
@@ -217,7 +218,7 @@ def chunk_prepare_int8(q, order=-1, residual_steps=-1, *, want_toff=True, output
         outputs = (Wq, Uq, w_exp, u_exp, Toff, t_exp)
     Wq, Uq, w_exp, u_exp, Toff, t_exp = outputs
     gdn_chunk_prepare_int8(q.Kq, q.Vq, q.k_exp, q.v_exp, q.beta_q, q.decay_q, q.B, q.H_k, q.H_v, q.T, q.C, q.d_k, q.d_v,
-                           order, residual_steps, Wq, Uq, w_exp, u_exp, Toff, t_exp)
+                           order, residual_steps, Wq, Uq, w_exp, u_exp, Toff, t_exp, dbg_acc)
     return outputs
 
 

@@ -56,6 +56,7 @@ struct ParamsI8 {
     int32_t* u_exp;
     int32_t* t_exp;
     int8_t* Toff;  // may be null
+    int32_t* dbg;  // may be null: [heads * chunks][64][8 * 64 + 128 + 128] accumulators
     int* status;
     int H_k, H_v, T, group, n_tt;
     int N, S;
@@ -305,6 +306,11 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
         const int chunk_in_head = (tc.t0 + cb) / kC;
         const bool chunk_valid = (tc.t0 + cb) < p.T;
 
+        // row of the accumulator dump (debugging aid of small cases; null in normal use)
+        constexpr int kDbgRow = 8 * kC + 2 * kD;
+        int32_t* dbg_row = (p.dbg != nullptr && row_valid)
+                               ? p.dbg + (((long long)tc.bhv * n_c + chunk_in_head) * kC + il) * kDbgRow
+                               : nullptr;
         STAMP8(1);
         int bq = 0, dq = 0, kexp = 0, vexp = 0;
         if (row_valid) {
@@ -355,6 +361,10 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             uint32_t g[kHC];
             tmem_ld32(lane_base + kR0 + cb + col0, g);
             tmem_wait_ld();
+            if (dbg_row != nullptr) {
+#pragma unroll
+                for (int jl = 0; jl < kHC; ++jl) dbg_row[col0 + jl] = static_cast<int>(g[jl]);
+            }
             // c_ij = (beta_q_i Gam_ij + 2^14) >> 15 (< 2^15), 0 on and above the diagonal. |G| < 2^21, so |G| c needs
             // 36 bits: it is kept as a (hi, lo) pair of 32-bit words; the shift r = bitlen - 7 stays below 32, so the
             // rounded shift is one funnel shift of the pair. Aq = -G c: the sign is restored at the end (the rounding
@@ -549,6 +559,10 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             uint32_t dres[kHC];
             tmem_ld32(lane_base + kR0 + cb + col0, dres);
             tmem_wait_ld();
+            if (dbg_row != nullptr) {
+#pragma unroll
+                for (int jl = 0; jl < kHC; ++jl) dbg_row[(s - 1) * kC + col0 + jl] = static_cast<int>(dres[jl]);
+            }
             uint32_t m = 0;
             // R_{s-1} is zero for i - j < (s - 1)(N + 1) and Eq for i - j <= N: the integer product is exactly zero
             // for i - j < s (N + 1), no mask needed
@@ -753,6 +767,10 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 uint32_t r[32];
                 tmem_ld32(lane_base + kR0 + h * 64 + c0, r);
                 tmem_wait_ld();
+                if (dbg_row != nullptr) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) dbg_row[8 * kC + half * kD + h * 64 + c0 + i] = static_cast<int>(r[i]);
+                }
                 if (left) {
                     // shifts folded into the multipliers: two multiply-adds per element
 #pragma unroll
@@ -905,6 +923,7 @@ int launch_tc_int8(const ProblemI8& q, cudaStream_t stream) {
     prm.u_exp = q.u_exp;
     prm.t_exp = q.t_exp;
     prm.Toff = q.Toff;
+    prm.dbg = q.dbg;
     prm.status = status;
     prm.H_k = q.H_k;
     prm.H_v = q.H_v;

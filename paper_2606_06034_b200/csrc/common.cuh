@@ -38,6 +38,7 @@ struct ProblemI8 {
     int32_t* u_exp;
     int8_t* Toff;  // may be null
     int32_t* t_exp;
+    int32_t* dbg;  // may be null: tensor-core accumulators of the chain
     int B, H_k, H_v, T, C, d_k, d_v;
     int order, steps;
 };

@@ -126,7 +126,7 @@ int gdn_chunk_prepare_fwdsubst(const void* K, const void* V, const float* beta, 
 int gdn_chunk_prepare_int8(const int8_t* Kq, const int8_t* Vq, const int32_t* k_exp, const int32_t* v_exp, const uint16_t* beta_q,
                            const int32_t* decay_q, int B, int H_k, int H_v, int T, int C, int d_k, int d_v, int order,
                            int residual_steps, int8_t* Wq_out, int8_t* Uq_out, int32_t* w_exp_out, int32_t* u_exp_out,
-                           int8_t* Toff_q_out, int32_t* t_exp_out, gdn_stream_t stream) {
+                           int8_t* Toff_q_out, int32_t* t_exp_out, int32_t* dbg_acc_out, gdn_stream_t stream) {
     if (order == -1) order = gdn_default_order(C);
     if (residual_steps == -1) residual_steps = gdn_default_residual_steps(C);
     if (Kq == nullptr || Vq == nullptr || k_exp == nullptr || v_exp == nullptr || beta_q == nullptr || decay_q == nullptr ||
@@ -135,12 +135,12 @@ int gdn_chunk_prepare_int8(const int8_t* Kq, const int8_t* Vq, const int32_t* k_
     if (B < 0 || H_k <= 0 || H_v <= 0 || T < 0 || C < 2 || d_k <= 0 || d_v <= 0) return GDN_ERR_INVALID_ARG;
     if (H_v % H_k != 0 || T % C != 0) return GDN_ERR_INVALID_ARG;
     if (order < 1 || order >= C || residual_steps < 0) return GDN_ERR_INVALID_ARG;
-    if (!aligned16(Kq) || !aligned16(Vq) || !aligned16(Wq_out) || !aligned16(Uq_out) || !aligned16(Toff_q_out))
+    if (!aligned16(Kq) || !aligned16(Vq) || !aligned16(Wq_out) || !aligned16(Uq_out) || !aligned16(Toff_q_out) || !aligned16(dbg_acc_out))
         return GDN_ERR_ALIGN;
     const int rc = check_arch();
     if (rc != GDN_OK) return rc;
     ProblemI8 q{Kq, Vq, k_exp, v_exp, reinterpret_cast<const int16_t*>(beta_q), decay_q, Wq_out, Uq_out, w_exp_out, u_exp_out,
-                Toff_q_out, t_exp_out, B, H_k, H_v, T, C, d_k, d_v, order, residual_steps};
+                Toff_q_out, t_exp_out, dbg_acc_out, B, H_k, H_v, T, C, d_k, d_v, order, residual_steps};
     return launch_tc_int8(q, static_cast<cudaStream_t>(stream));
 }
 

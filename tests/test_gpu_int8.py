@@ -73,3 +73,21 @@ def test_int8_unsupported_configurations():
     with pytest.raises(gdn.GdnError) as e:
         gdn.chunk_prepare_int8(qd, 4, 3)
     assert e.value.status == gdn.GDN_ERR_UNSUPPORTED
+
+
+def test_int8_tensor_core_accumulators_match():
+    """dbg_acc_out: every int32 accumulator of the products that run on the tensor cores (Gram rows, the power
+    products, Tbq Kq, Tbq Vq) equals the oracle's exact integer product."""
+    inp = gen.make_inputs(1, 1, 2, 192, 64, 128, 128, seed=140, adversarial_heads="odd")
+    q = gen.make_int8_inputs(inp)
+    qd = _to_dev(q)
+    n, C = q.n_chunks, q.C
+    dbg = torch.zeros(q.B, q.H_v, q.T // C, C, 8 * C + q.d_k + q.d_v, dtype=torch.int32, device="cuda")
+    gdn.chunk_prepare_int8(qd, dbg_acc=dbg)
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+    Kq, Vq, ke, ve, bq, dq = gen.int8_chunk_slices(q, range(n))
+    ref = orq.chunk_prepare_int8(Kq, Vq, ke, ve, bq, dq, gdn.gdn_default_order(C), gdn.gdn_default_residual_steps(C))
+    got = dbg.reshape(n, C, -1).cpu().numpy().astype(np.int64)
+    bad = np.argwhere(got != ref["acc"])
+    assert bad.size == 0, f"{len(bad)} accumulator mismatches, first at {bad[0]}"
+    assert np.abs(ref["acc"]).max() < 2 ** 31
