@@ -28,6 +28,7 @@ GDN_DTYPE_BF16 = 1
 GDN_FLAG_G_RAW = 1
 GDN_FLAG_K_L2NORM = 2
 GDN_FLAG_OUT_FP32 = 4
+GDN_FLAG_LAYOUT_BTHD = 8
 GDN_FWDSUBST_ROWS = 0
 GDN_FWDSUBST_BLOCKED = 1
 
@@ -127,12 +128,16 @@ def _check_inputs(K, V, beta, g, outs):
         raise TypeError("K and V share a dtype; beta and g are fp32")
 
 
-def alloc_outputs(K, V, C, want_tinv=True):
-    """Allocates W [B,H_v,T,d_k], U [B,H_v,T,d_v], Tinv [B,H_v,T/C,C,C] with torch."""
-    B, H_v, T, d_v = V.shape
+def alloc_outputs(K, V, C, want_tinv=True, token_major=False):
+    """Allocates W [B,H_v,T,d_k], U [B,H_v,T,d_v], Tinv [B,H_v,T/C,C,C] with torch
+    (token_major: K, V are [B,T,H,d] and so are W, U; Tinv keeps its layout)."""
+    if token_major:
+        B, T, H_v, d_v = V.shape
+    else:
+        B, H_v, T, d_v = V.shape
     d_k = K.shape[-1]
-    W = torch.empty(B, H_v, T, d_k, dtype=K.dtype, device=K.device)
-    U = torch.empty(B, H_v, T, d_v, dtype=K.dtype, device=K.device)
+    W = torch.empty((B, T, H_v, d_k) if token_major else (B, H_v, T, d_k), dtype=K.dtype, device=K.device)
+    U = torch.empty((B, T, H_v, d_v) if token_major else (B, H_v, T, d_v), dtype=K.dtype, device=K.device)
     Tinv = torch.empty(B, H_v, T // C, C, C, dtype=K.dtype, device=K.device) if want_tinv else None
     return W, U, Tinv
 
@@ -232,11 +237,18 @@ def chunk_prepare(K, V, beta, g, C, order=-1, residual_steps=-1, *, want_tinv=Tr
     """Convenience wrapper: shapes from the tensors, outputs allocated with torch.
 
     K [B,H_k,T,d_k], V [B,H_v,T,d_v], beta, g [B,H_v,T]. Returns (W, U, Tinv).
+    With GDN_FLAG_LAYOUT_BTHD in `flags` the tensors are token-major: K [B,T,H_k,d_k], V [B,T,H_v,d_v],
+    beta, g [B,T,H_v], W [B,T,H_v,d_k], U [B,T,H_v,d_v] (Tinv keeps [B,H_v,T/C,C,C]).
     """
-    B, H_k, T, d_k = K.shape
-    _, H_v, _, d_v = V.shape
+    token_major = bool(flags & GDN_FLAG_LAYOUT_BTHD)
+    if token_major:
+        B, T, H_k, d_k = K.shape
+        _, _, H_v, d_v = V.shape
+    else:
+        B, H_k, T, d_k = K.shape
+        _, H_v, _, d_v = V.shape
     if outputs is None:
-        outputs = alloc_outputs(K, V, C, want_tinv)
+        outputs = alloc_outputs(K, V, C, want_tinv, token_major)
         if flags & GDN_FLAG_OUT_FP32:
             outputs = tuple(None if o is None else torch.empty(o.shape, dtype=torch.float32, device=o.device) for o in outputs)
     W, U, Tinv = outputs

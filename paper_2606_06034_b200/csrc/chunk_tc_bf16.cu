@@ -361,6 +361,11 @@ __device__ __forceinline__ void build_wu_operands(uint32_t lane_base, uint32_t b
 struct TileCoord {
     int bhk, bhv;
     int t0;
+    // where the tile sits in memory: first TMA coordinates of the K tile (feature column, outermost index) and of the
+    // V / W / U tiles, index of the tile's first token in beta / g, and the stride between tokens there
+    int kx, kz, vx, vz;
+    long long r0;
+    int rs;
 };
 // A tile index in mixed-radix digits: tile = (bhk * n_tt + tt) * group + gi, so that tiles sharing a key tile are
 // adjacent. A CTA walks its tiles by adding the grid size digit by digit (one carry per digit is enough because
@@ -386,12 +391,33 @@ __device__ __forceinline__ void tile_advance(TilePos& c, const Params& p) {
     c.tt -= c2 ? p.n_tt : 0;
     c.bhk += p.s_bhk + c2;
 }
-// (key head row, value head row, first token): value head row = bhk * group + gi because H_v = H_k * group
+// (key head row, value head row, first token): value head row = bhk * group + gi because H_v = H_k * group.
+// Head-major tensors [B, H, T, d] are seen by TMA as (d, T, B * H); token-major ones [B, T, H, d]
+// (GDN_FLAG_LAYOUT_BTHD, only in the EX instantiations) as (H * d, T, B), the head selecting a column range.
+template <bool EX>
 __device__ __forceinline__ TileCoord tile_coord(const TilePos& c, const Params& p) {
     TileCoord r;
     r.bhk = c.bhk;
     r.bhv = c.bhk * p.group + c.gi;
     r.t0 = c.tt * kTile;
+    if (EX && (p.flags & GDN_FLAG_LAYOUT_BTHD)) {
+        const int b = c.bhk / p.H_k;
+        const int hk = c.bhk - b * p.H_k;
+        const int hv = hk * p.group + c.gi;
+        r.kx = hk * kD;
+        r.kz = b;
+        r.vx = hv * kD;
+        r.vz = b;
+        r.r0 = ((long long)b * p.T + r.t0) * p.H_v + hv;
+        r.rs = p.H_v;
+    } else {
+        r.kx = 0;
+        r.kz = r.bhk;
+        r.vx = 0;
+        r.vz = r.bhv;
+        r.r0 = (long long)r.bhv * p.T + r.t0;
+        r.rs = 1;
+    }
     return r;
 }
 
@@ -522,27 +548,27 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 
     TilePos pos_next = tile_pos(blockIdx.x, p);  // position of the tile after the one being worked on
     if (tid == 0 && blockIdx.x < n_tiles) {
-        const TileCoord c = tile_coord(pos_next, p);
+        const TileCoord c = tile_coord<EX>(pos_next, p);
         mbar_arrive_expect_tx(&bar_k, 32768);
-        tma_load_3d(sK, &tmK, &bar_k, 0, c.t0, c.bhk);
-        tma_load_3d(sK + 16384, &tmK, &bar_k, 64, c.t0, c.bhk);
+        tma_load_3d(sK, &tmK, &bar_k, c.kx, c.t0, c.kz);
+        tma_load_3d(sK + 16384, &tmK, &bar_k, c.kx + 64, c.t0, c.kz);
         mbar_arrive_expect_tx(&bar_v, 32768);
-        tma_load_3d(sV, &tmV, &bar_v, 0, c.t0, c.bhv);
-        tma_load_3d(sV + 16384, &tmV, &bar_v, 64, c.t0, c.bhv);
+        tma_load_3d(sV, &tmV, &bar_v, c.vx, c.t0, c.vz);
+        tma_load_3d(sV + 16384, &tmV, &bar_v, c.vx + 64, c.t0, c.vz);
     }
     // beta and g of the row are fetched one tile ahead
     float bi_next = 0.f, gi_next = 0.f;
     if (blockIdx.x < n_tiles) {
-        const TileCoord c = tile_coord(pos_next, p);
+        const TileCoord c = tile_coord<EX>(pos_next, p);
         if (c.t0 + t < p.T) {
-            const long long r = (long long)c.bhv * p.T + c.t0 + t;
+            const long long r = c.r0 + (long long)t * c.rs;
             bi_next = __ldg(p.beta + r);
             gi_next = __ldg(p.g + r);
         }
     }
 
     for (uint32_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-        const TileCoord tc = tile_coord(pos_next, p);
+        const TileCoord tc = tile_coord<EX>(pos_next, p);
         tile_advance(pos_next, p);
         const uint32_t next = tile + gridDim.x;
         const bool has_next = next < n_tiles;
@@ -675,9 +701,9 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         bi_next = 0.f;
         gi_next = 0.f;
         if (has_next) {
-            const TileCoord nc = tile_coord(pos_next, p);
+            const TileCoord nc = tile_coord<EX>(pos_next, p);
             if (nc.t0 + t < p.T) {
-                const long long r = (long long)nc.bhv * p.T + nc.t0 + t;
+                const long long r = nc.r0 + (long long)t * nc.rs;
                 bi_next = __ldg(p.beta + r);
                 gi_next = __ldg(p.g + r);
             }
@@ -1336,15 +1362,15 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             STAMP(11 + half * 3);
             if (warp == 0 && has_next && elect_one()) {
                 // the products that read this tile's K (half 0) or V (half 1) are complete: prefetch the next tile's
-                const TileCoord nc = tile_coord(pos_next, p);
+                const TileCoord nc = tile_coord<EX>(pos_next, p);
                 if (half == 0) {
                     mbar_arrive_expect_tx(&bar_k, 32768);
-                    tma_load_3d(sK, &tmK, &bar_k, 0, nc.t0, nc.bhk);
-                    tma_load_3d(sK + 16384, &tmK, &bar_k, 64, nc.t0, nc.bhk);
+                    tma_load_3d(sK, &tmK, &bar_k, nc.kx, nc.t0, nc.kz);
+                    tma_load_3d(sK + 16384, &tmK, &bar_k, nc.kx + 64, nc.t0, nc.kz);
                 } else {
                     mbar_arrive_expect_tx(&bar_v, 32768);
-                    tma_load_3d(sV, &tmV, &bar_v, 0, nc.t0, nc.bhv);
-                    tma_load_3d(sV + 16384, &tmV, &bar_v, 64, nc.t0, nc.bhv);
+                    tma_load_3d(sV, &tmV, &bar_v, nc.vx, nc.t0, nc.vz);
+                    tma_load_3d(sV + 16384, &tmV, &bar_v, nc.vx + 64, nc.t0, nc.vz);
                 }
             }
             uint32_t o[32];
@@ -1356,7 +1382,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 if (f_f32) {
                     if ((tc.t0 + t) < p.T) {
                         float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(half == 0 ? p.W : p.U) +
-                                                               ((long long)tc.bhv * p.T + tc.t0 + t) * kD + h * 64 + c0);
+                                                               (tc.r0 + (long long)t * tc.rs) * kD + h * 64 + c0);
 #pragma unroll
                         for (int i = 0; i < 8; ++i)
                             dst[i] = make_float4(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]), __uint_as_float(r[4 * i + 2]),
@@ -1408,7 +1434,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) {
-                    tma_store_3d((half == 0) ? &tmW : &tmU, smem + L::kEB + wq * 8192 + h * 4096, h * 64, tc.t0 + wrow0, tc.bhv);
+                    tma_store_3d((half == 0) ? &tmW : &tmU, smem + L::kEB + wq * 8192 + h * 4096, tc.vx + h * 64, tc.t0 + wrow0, tc.vz);
                     tma_store_commit();
                 }
             }
@@ -1520,10 +1546,15 @@ int launch_tc_bf16(const Problem& p, InverseMode mode, cudaStream_t stream) {
     // Tinv leaves in boxes of 32 rows x (C/2 columns for C >= 32, else C columns): 64-, 32- and 32-byte lines
     const int tbox = (p.C == 128) ? 32 : ((p.C >= 32) ? p.C / 2 : p.C);
     const CUtensorMapSwizzle tsw = (tbox * 2 == 64) ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
-    if (!make_map(&m.K, p.K, hk, p.T, kD, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
-    if (!make_map(&m.V, p.V, hv, p.T, kD, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
-    if (!make_map(&m.W, p.W, hv, p.T, kD, 64, 32, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
-    if (!make_map(&m.U, p.U, hv, p.T, kD, 64, 32, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
+    // head-major [B, H, T, d]: (d, T, B * H); token-major [B, T, H, d]: (H * d, T, B), the head picks the columns
+    const bool bthd = (p.flags & GDN_FLAG_LAYOUT_BTHD) != 0;
+    if (bthd && mode != INV_NEUMANN) return GDN_ERR_UNSUPPORTED;
+    const long long zk = bthd ? p.B : hk, zv = bthd ? p.B : hv;
+    const int ck = bthd ? p.H_k * kD : kD, cv = bthd ? p.H_v * kD : kD;
+    if (!make_map(&m.K, p.K, zk, p.T, ck, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
+    if (!make_map(&m.V, p.V, zv, p.T, cv, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
+    if (!make_map(&m.W, p.W, zv, p.T, cv, 64, 32, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
+    if (!make_map(&m.U, p.U, zv, p.T, cv, 64, 32, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
     // Tinv rows are C wide; without a Tinv output the map points at W (never used by the kernel then)
     if (!make_map(&m.T, p.Tinv != nullptr ? p.Tinv : p.W, hv, p.T, p.Tinv != nullptr ? p.C : kD, p.Tinv != nullptr ? tbox : 64, 32,
                   p.Tinv != nullptr ? tsw : CU_TENSOR_MAP_SWIZZLE_128B))

@@ -285,9 +285,53 @@ def test_fp32_prologue_flags(C, flags):
     _check_ex(inp, graw, flags, TOL_FP32 * 3)
 
 
+@pytest.mark.parametrize("C", [16, 32, 64, 128])
+@pytest.mark.parametrize("extra", [0, 3, 7])
+def test_bf16_token_major_layout(C, extra):
+    """GDN_FLAG_LAYOUT_BTHD: K, V, beta, g, W, U in [B, T, H, d] order (grouped heads, a ragged last tile); the
+    result must equal the head-major one element for element after transposing back, and meet the oracle bars."""
+    inp, graw = _raw_inputs(2, 2, 4, 3 * C if C == 128 else 320 if C != 32 else 352, C, seed=280 + C, adv="odd")
+    if not (extra & gdn.GDN_FLAG_K_L2NORM):
+        inp = gen.make_inputs(2, 2, 4, inp.T, C, 128, 128, seed=280 + C, adversarial_heads="odd")
+    g_src = graw if (extra & gdn.GDN_FLAG_G_RAW) else inp.g
+    K, V, beta, g = inp.K.cuda(), inp.V.cuda(), inp.beta.cuda(), g_src.cuda()
+    tm = lambda x: x.transpose(1, 2).contiguous()
+    flags = extra | gdn.GDN_FLAG_LAYOUT_BTHD
+    W, U, Tinv = gdn.chunk_prepare(tm(K), tm(V), tm(beta), tm(g), C, flags=flags)
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+    assert W.shape == (inp.B, inp.T, inp.H_v, inp.d_k) and Tinv.shape == (inp.B, inp.H_v, inp.T // C, C, C)
+    # reference: the same call in the head-major layout (the extra flags go through the same instantiation)
+    if extra:
+        W0, U0, T0 = gdn.chunk_prepare(K, V, beta, g, C, flags=extra)
+    else:
+        W0, U0, T0 = gdn.chunk_prepare(K, V, beta, g, C)
+    assert torch.equal(tm(W0) if W0.dtype == W.dtype else tm(W0), W)
+    assert torch.equal(tm(U0), U)
+    assert torch.equal(T0, Tinv)
+    # and against the oracle
+    Wg, Ug, Tg = _gpu_chunks(W.transpose(1, 2).contiguous(), U.transpose(1, 2).contiguous(), Tinv, inp)
+    sl = gen.chunk_slices(inp, range(inp.n_chunks))
+    Kc = np.stack([s[0] for s in sl]); Vc = np.stack([s[1] for s in sl]); bc = np.stack([s[2] for s in sl])
+    gc = g_src.double().numpy().reshape(inp.n_chunks, C)
+    Wo, Uo, To = orc.chunk_prepare(Kc, Vc, bc, gc, None, None, g_raw=bool(extra & 1), k_l2norm=bool(extra & 2))
+    tol = 5e-4 if (extra & gdn.GDN_FLAG_OUT_FP32) else TOL_BF16 + 3e-4
+    for name, got, ref in (("Tinv", Tg, To), ("W", Wg, Wo), ("U", Ug, Uo)):
+        err = orc.rel_frobenius(got, ref)
+        assert err.max() <= tol, f"{name} rel-F {err.max():.3e} at chunk {err.argmax()}"
+
+
+def test_token_major_layout_is_bf16_only():
+    inp = gen.make_inputs(1, 1, 1, 128, 64, 128, 128, seed=281, dtype=torch.float32)
+    K, V, beta, g = _to_dev(inp)
+    W, U, Tinv = gdn.alloc_outputs(K, V, 64)
+    rc = gdn.gdn_chunk_prepare_ex(K, V, beta, g, 1, 1, 1, 128, 64, 128, 128, -1, -1, 0, W, U, Tinv,
+                                  gdn.GDN_FLAG_LAYOUT_BTHD, check=False)
+    assert rc == gdn.GDN_ERR_UNSUPPORTED
+
+
 def test_ex_rejects_unknown_flags():
     inp = gen.make_inputs(1, 1, 1, 128, 64, 128, 128, seed=270)
     K, V, beta, g = _to_dev(inp)
     W, U, Tinv = gdn.alloc_outputs(K, V, 64)
-    rc = gdn.gdn_chunk_prepare_ex(K, V, beta, g, 1, 1, 1, 128, 64, 128, 128, -1, -1, 1, W, U, Tinv, 8, check=False)
+    rc = gdn.gdn_chunk_prepare_ex(K, V, beta, g, 1, 1, 1, 128, 64, 128, 128, -1, -1, 1, W, U, Tinv, 16, check=False)
     assert rc == gdn.GDN_ERR_INVALID_ARG
