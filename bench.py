@@ -195,9 +195,22 @@ def run_ours(args, rank, world, dist_ctx):
     C, group = inp.C, inp.H_v // inp.H_k
     outs = gdn.alloc_outputs(inp.K, inp.V, C)
     n_chunks = inp.n_chunks
+    # --method other than the default times one of the other kernels as the step (used for the ncu summaries of the
+    # forward-substitution comparison and of the INT8 variant); the headline is always --method neumann
+    method = args.method
+    q8 = q8_outs = None
+    if method == "int8":
+        q8 = gen.make_int8_inputs(inp)
+        q8_outs = gdn.chunk_prepare_int8(q8)
 
     def step():
-        gdn.chunk_prepare(inp.K, inp.V, inp.beta, inp.g, C, outputs=outs)
+        if method == "neumann":
+            gdn.chunk_prepare(inp.K, inp.V, inp.beta, inp.g, C, outputs=outs)
+        elif method == "int8":
+            gdn.chunk_prepare_int8(q8, outputs=q8_outs)
+        else:
+            gdn.chunk_prepare(inp.K, inp.V, inp.beta, inp.g, C, outputs=outs, method="fwdsubst",
+                              variant=gdn.GDN_FWDSUBST_BLOCKED if method == "fwdsubst-blocked" else gdn.GDN_FWDSUBST_ROWS)
 
     sampler = ClockSampler(torch.cuda.current_device())
     launches0 = gdn.gdn_launch_count()
@@ -219,22 +232,25 @@ def run_ours(args, rank, world, dist_ctx):
     value = whole_job_throughput(n_chunks, world, ms_per_step)
 
     bytes_chunk = algorithmic_bytes_per_chunk(C, inp.d_k, inp.d_v, group)
+    if method == "int8":  # one byte per element, u16 beta + i32 decay per token
+        bytes_chunk = C * inp.d_k / group + C * inp.d_v + C * inp.d_k + C * inp.d_v + C * C + 6 * C
     flops_chunk = nominal_flops_per_chunk(C, inp.d_k, inp.d_v)
     hbm_peak, bf16_peak, peak_kind = measured_peaks()
     launch_ms = float(np.mean(per))
     achieved = n_chunks * bytes_chunk / (launch_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak,
-                "traffic": TRAFFIC_PER_LAUNCH.get(args.workload), "peak_kind": peak_kind,
+                "traffic": TRAFFIC_PER_LAUNCH.get(args.workload) if method == "neumann" else None, "peak_kind": peak_kind,
                 "algorithmic_bytes_per_launch": n_chunks * bytes_chunk,
-                "kernel": "chunk_tc_kernel<C=%d>" % C,
+                "kernel": ("chunk_tc_int8_kernel" if method == "int8" else "chunk_tc_kernel<C=%d>" % C),
                 "effective_tflops": n_chunks * flops_chunk / (launch_ms * 1e-3) / 1e12,
                 "tensor_time_frac_of_bf16_peak": (n_chunks * flops_chunk / (launch_ms * 1e-3) / 1e12) / bf16_peak}
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "s8" if method == "int8" else "bf16",
         "data": "synthetic", "impl": "ours",
-        "config": {"workload": args.workload, "B": inp.B, "H_k": inp.H_k, "H_v": inp.H_v, "T": inp.T, "C": C, "d_k": inp.d_k,
+        "config": {"workload": args.workload, "method": method, "B": inp.B, "H_k": inp.H_k, "H_v": inp.H_v, "T": inp.T, "C": C, "d_k": inp.d_k,
                    "d_v": inp.d_v, "order": gdn.gdn_default_order(C), "residual_steps": gdn.gdn_default_residual_steps(C),
                    "chunks_per_gpu": n_chunks, "parallelism": f"independent shards x{world}, no collective",
                    "l2_policy": "inputs+outputs %.0f MB per step, larger than the 126 MB L2" % (n_chunks * bytes_chunk / 1e6)},
@@ -242,7 +258,7 @@ def run_ours(args, rank, world, dist_ctx):
         "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline,
     }
 
-    if rank == 0 and not args.no_e2e:
+    if rank == 0 and not args.no_e2e and method == "neumann":
         line["e2e"] = run_e2e(inp, outs, gdn, args, world, n_chunks)
     if rank == 0 and not args.no_extras:
         line["extras"] = run_extras(gdn, gen, dev, args)
@@ -382,6 +398,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--method", default="neumann", choices=["neumann", "fwdsubst", "fwdsubst-blocked", "int8"])
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extras", action="store_true")
