@@ -74,9 +74,8 @@ struct Smem {
     static constexpr int kEB = 65536;
     static constexpr int kEBBytes = kTile * C * 2;
     static constexpr int kBR = kEB + kEBBytes;
-    static constexpr int kBRBytes = kTile * C * 2;
     static constexpr int NBP = (NB <= 3) ? 4 : 8;
-    static constexpr int kScratchBytes = 32768;         // >= kEBBytes + kBRBytes; also the 4 x 8 KB store staging slices
+    static constexpr int kScratchBytes = 32768;         // >= kEBBytes + kTile * C * 2 (BR); also the 4 x 8 KB store staging slices
     static constexpr int kSH = kEB + kScratchBytes;     // column form of the band: [128 + 8][NBP] floats
     static constexpr int kSHBytes = (kTile + 8) * NBP * 4;
     static constexpr int kRB = kSH + kSHBytes;          // row form of the band: [128][NBP] floats
@@ -282,24 +281,6 @@ __device__ __forceinline__ void load_diag_block(uint32_t lane_base, uint32_t col
     }
 }
 
-// Reads the thread's columns of a 128 x C accumulator (same address for the whole warp).
-template <int C>
-__device__ __forceinline__ void load_cols(uint32_t lane_base, uint32_t col0, int h, float (&r)[Split<C>::HC]) {
-    if constexpr (C == 64) {
-        uint32_t q[32];
-        tmem_ld32(lane_base + col0 + h * 32, q);
-        tmem_wait_ld();
-#pragma unroll
-        for (int i = 0; i < 32; ++i) r[i] = __uint_as_float(q[i]);
-    } else {
-        uint32_t q[16];
-        tmem_ld16(lane_base + col0 + ((C == 32) ? h * 16 : 0), q);
-        tmem_wait_ld();
-#pragma unroll
-        for (int i = 0; i < 16; ++i) r[i] = __uint_as_float(q[i]);
-    }
-}
-
 // Builds the two bf16 A operands of the W/U products for this thread's part of its row and stores them to TMEM:
 // hi (slot AS) = bf16(T diag(scale)) over the whole row, lo (slot R2) = bf16 of what hi loses on the diagonal and
 // the band, where entries are O(1). `sc` is the per-token scale in shared memory, `sc_i` the row's own scale;
@@ -440,7 +421,6 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     constexpr int NBP = L::NBP;
     constexpr int HC = SP::HC;     // columns of the chunk handled by this thread
     constexpr int PCH = SP::PCH;   // packed words handled by this thread
-    constexpr int CPR = C / 8;     // 16-byte chunks of a packed bf16 row
     constexpr int CPRF = C / 4;    // 16-byte chunks of an fp32 row
     constexpr int CPT = HC / 8;    // packed chunks owned by this thread
     constexpr int CPTF = HC / 4;   // fp32 chunks owned by this thread

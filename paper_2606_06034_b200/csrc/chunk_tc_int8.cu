@@ -91,36 +91,18 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity) {
     return true;
 }
 
-__device__ __forceinline__ long long rsr64(long long x, int r) {
-    if (r <= 0) return x;
-    const long long a = ((x < 0 ? -x : x) + (1LL << (r - 1))) >> r;
-    return x < 0 ? -a : a;
-}
-// x * 2^s for s >= 0, rounded right shift otherwise
-__device__ __forceinline__ long long shift64(long long x, int s) { return s >= 0 ? (x << s) : rsr64(x, -s); }
-// type-generic forms (T = int when every term provably fits 32 bits, long long otherwise)
-template <typename T>
-__device__ __forceinline__ T rsr_t(T x, int r) {  // r >= 0; (1 << r) >> 1 is the rounding half, 0 for r = 0
-    const T a = x < 0 ? -x : x;
-    const T q = (a + ((static_cast<T>(1) << r) >> 1)) >> r;
-    return x < 0 ? -q : q;
-}
-// 32-bit form without branches (see q8_32)
+// rsr(x, r): rounded right shift, half away from zero; 32-bit form without branches (see rsr_rnd)
 __device__ __forceinline__ int rsr32(int x, int r) {
     const int half = static_cast<int>((1u << r) >> 1);
     const int neg1 = (r > 0) ? (x >> 31) : 0;
     return (x + half + neg1) >> r;
 }
-template <typename T>
-__device__ __forceinline__ T shift_t(T x, int s) { return s >= 0 ? (x << s) : rsr_t<T>(x, -s); }
 // One term of an aligned sum: x 2^s for s >= 0, rounded right shift otherwise. x fits 23 bits, so the right
 // shift is done in 32 bits (a shift of 31 or more gives 0, as the rounding rule demands for |x| < 2^30).
-template <typename T>
-__device__ __forceinline__ T term_t(int x, int s) {
-    if (s >= 0) return static_cast<T>(x) << s;
-    return static_cast<T>(rsr32(x, (-s) < 31 ? (-s) : 31));
+__device__ __forceinline__ int term32(int x, int s) {
+    if (s >= 0) return x << s;
+    return rsr32(x, (-s) < 31 ? (-s) : 31);
 }
-__device__ __forceinline__ int term32(int x, int s) { return term_t<int>(x, s); }
 // Rounding constants of one requantisation (uniform over a chunk): shift, rounding half, and an all-ones mask when
 // something is shifted out.
 struct Rnd {
@@ -153,12 +135,7 @@ __device__ __forceinline__ uint32_t q8_pack4(int x0, int x1, int x2, int x3, con
     return pack_sat_s8(y1, y0, pack_sat_s8(y3, y2, 0u));
 }
 __device__ __forceinline__ uint32_t abs32(int x) { return static_cast<uint32_t>(abs(x)); }
-template <typename T>
-__device__ __forceinline__ unsigned long long abs_bits(T x) { return static_cast<unsigned long long>(x < 0 ? -x : x); }
-template <typename T>
-__device__ __forceinline__ int clamp127_t(T q) { return q > 127 ? 127 : (q < -127 ? -127 : static_cast<int>(q)); }
 
-__device__ __forceinline__ int clamp127(long long q) { return q > 127 ? 127 : (q < -127 ? -127 : static_cast<int>(q)); }
 __device__ __forceinline__ int q8_shift(int bitlen) { return bitlen > 7 ? bitlen - 7 : 0; }
 __device__ __forceinline__ int align_ref2(int e0, int e1) {
     const int lo = e0 < e1 ? e0 : e1, hi = e0 < e1 ? e1 : e0;
