@@ -156,6 +156,15 @@ unsigned int gdn_int8_lut_checksum(void);
  */
 int gdn_device_status(gdn_stream_t stream);
 
+/*
+ * Self-test of the bounded waits (no counterpart in the paper): launches one small kernel that waits, with the
+ * same wait routine and budget (about a second) as the compute kernels, on an mbarrier that nothing ever
+ * completes. The wait gives up, the kernel records GDN_ERR_TIMEOUT and returns normally: the next
+ * gdn_device_status(stream) reports GDN_ERR_TIMEOUT once, and the context stays usable. Returns GDN_OK when
+ * the kernel was enqueued.
+ */
+int gdn_selftest_bounded_wait(gdn_stream_t stream);
+
 /* Paper's parameters per chunk size: N = 3; S = 8 for C = 64 (Sec. 4.1) and for the
  * 64-blocks of C = 128 (App. H), S = 4 for C = 32 (Sec. 4.3); C = 16 is not in the
  * paper: S = 3, which makes the result exact. Other C: S = ceil(C/4) - 1. */

@@ -34,7 +34,7 @@ GDN_FWDSUBST_BLOCKED = 1
 
 EXPORTS = (
     "gdn_chunk_prepare", "gdn_chunk_prepare_gqa", "gdn_chunk_prepare_ex", "gdn_chunk_prepare_fwdsubst",
-    "gdn_chunk_prepare_int8",
+    "gdn_chunk_prepare_int8", "gdn_selftest_bounded_wait",
     "gdn_int8_lut_checksum",
     "gdn_device_status", "gdn_default_order", "gdn_default_residual_steps",
     "gdn_status_string", "gdn_launch_count",
@@ -71,6 +71,8 @@ def load_library() -> ctypes.CDLL:
     lib.gdn_chunk_prepare_int8.restype = ip
     lib.gdn_chunk_prepare_int8.argtypes = [vp, vp, vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ip, ip, ip, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.gdn_int8_lut_checksum.restype = ctypes.c_uint
+    lib.gdn_selftest_bounded_wait.argtypes = [vp]
+    lib.gdn_selftest_bounded_wait.restype = ip
     lib.gdn_int8_lut_checksum.argtypes = []
     lib.gdn_device_status.restype = ip
     lib.gdn_device_status.argtypes = [vp]
@@ -225,6 +227,11 @@ def chunk_prepare_int8(q, order=-1, residual_steps=-1, *, want_toff=True, output
     gdn_chunk_prepare_int8(q.Kq, q.Vq, q.k_exp, q.v_exp, q.beta_q, q.decay_q, q.B, q.H_k, q.H_v, q.T, q.C, q.d_k, q.d_v,
                            order, residual_steps, Wq, Uq, w_exp, u_exp, Toff, t_exp, dbg_acc)
     return outputs
+
+
+def gdn_selftest_bounded_wait() -> int:
+    """Enqueues the bounded-wait self-test on torch's current stream (see the header)."""
+    return load_library().gdn_selftest_bounded_wait(_stream())
 
 
 def gdn_device_status() -> int:

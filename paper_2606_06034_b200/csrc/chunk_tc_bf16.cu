@@ -1514,6 +1514,27 @@ extern "C" int gdn_debug_read_trace(long long* host_out) {
 }
 #endif
 
+namespace {
+// waits on an mbarrier that never completes: wait_bar must give up after its budget and report it
+__global__ void wait_selftest_kernel(int* status) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        mbar_fence_init();
+    }
+    __syncthreads();
+    if (!wait_bar(&bar, 0) && threadIdx.x == 0) atomicExch(status, GDN_ERR_TIMEOUT);
+}
+}  // namespace
+
+int launch_wait_selftest(cudaStream_t stream) {
+    int* status = device_status_word();
+    if (status == nullptr) return GDN_ERR_LAUNCH;
+    wait_selftest_kernel<<<1, 32, 0, stream>>>(status);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? GDN_OK : GDN_ERR_LAUNCH;
+}
+
 int launch_tc_bf16(const Problem& p, InverseMode mode, cudaStream_t stream) {
     if (p.d_k != kD || p.d_v != kD) return GDN_ERR_UNSUPPORTED;
     if (!(p.C == 16 || p.C == 32 || p.C == 64 || (p.C == 128 && mode == INV_NEUMANN))) return GDN_ERR_UNSUPPORTED;

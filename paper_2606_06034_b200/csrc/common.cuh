@@ -52,6 +52,7 @@ void count_launch();
 // Kernel launchers. Each returns a gdn_status and launches on `stream`.
 int launch_simt(const Problem& p, InverseMode mode, cudaStream_t stream);
 int launch_tc_bf16(const Problem& p, InverseMode mode, cudaStream_t stream);
+int launch_wait_selftest(cudaStream_t stream);
 int launch_tc_int8(const ProblemI8& p, cudaStream_t stream);
 void int8_decay_lut(uint16_t* out256);  // table of round(2^15 * 2^(-f/256))
 

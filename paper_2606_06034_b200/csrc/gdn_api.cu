@@ -148,6 +148,12 @@ int gdn_chunk_prepare_int8(const int8_t* Kq, const int8_t* Vq, const int32_t* k_
     return launch_tc_int8(q, static_cast<cudaStream_t>(stream));
 }
 
+int gdn_selftest_bounded_wait(gdn_stream_t stream) {
+    const int rc = check_arch();
+    if (rc != GDN_OK) return rc;
+    return launch_wait_selftest(static_cast<cudaStream_t>(stream));
+}
+
 unsigned int gdn_int8_lut_checksum(void) {
     uint16_t lut[256];
     int8_decay_lut(lut);

@@ -335,3 +335,14 @@ def test_ex_rejects_unknown_flags():
     W, U, Tinv = gdn.alloc_outputs(K, V, 64)
     rc = gdn.gdn_chunk_prepare_ex(K, V, beta, g, 1, 1, 1, 128, 64, 128, 128, -1, -1, 1, W, U, Tinv, 16, check=False)
     assert rc == gdn.GDN_ERR_INVALID_ARG
+
+
+def test_bounded_wait_gives_up_and_reports():
+    """A wait on an mbarrier that nothing completes runs out after about a second: the status word reports
+    GDN_ERR_TIMEOUT once, and the context stays usable (a normal call afterwards is correct)."""
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+    assert gdn.gdn_selftest_bounded_wait() == gdn.GDN_OK
+    assert gdn.gdn_device_status() == gdn.GDN_ERR_TIMEOUT
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+    inp = gen.make_inputs(1, 1, 1, 256, 64, 128, 128, seed=290)
+    _check(inp, TOL_BF16)
