@@ -68,6 +68,8 @@ enum {
     GDN_FLAG_G_RAW = 1,     /* g holds the raw per-token log-gates; the kernel forms the chunk-local inclusive prefix sum */
     GDN_FLAG_K_L2NORM = 2,  /* the kernel L2-normalises the rows of K first (the normalisation Sec. 2.1 places before the path) */
     GDN_FLAG_OUT_FP32 = 4,  /* W, U, Tinv are written as fp32 although K, V are bf16 (parity debugging) */
+    GDN_FLAG_W_GATED = 16,  /* W = T diag(beta * exp(g)) K: the gated form the state update of the layer consumes
+                               (g as given, or the chunk-local prefix sum with GDN_FLAG_G_RAW); U is unchanged */
     GDN_FLAG_LAYOUT_BTHD = 8 /* token-major tensors as model code keeps them: K [B,T,H_k,d_k], V [B,T,H_v,d_v],
                                 beta, g [B,T,H_v], W [B,T,H_v,d_k], U [B,T,H_v,d_v]; Tinv stays [B,H_v,T/C,C,C].
                                 bf16 only (GDN_ERR_UNSUPPORTED with GDN_DTYPE_FP32) */

@@ -270,7 +270,7 @@ def exact_inverse(A: np.ndarray) -> np.ndarray:
 
 
 def chunk_prepare(K, V, beta, g, N: int | None = None, S: int | None = None, *,
-                  exact: bool = False, g_raw: bool = False, k_l2norm: bool = False):
+                  exact: bool = False, g_raw: bool = False, k_l2norm: bool = False, w_gated: bool = False):
     """One chunk or a stack of chunks: returns (W, U, T), all fp64.
 
     K: [..., C, d_k], V: [..., C, d_v], beta, g: [..., C].
@@ -278,7 +278,9 @@ def chunk_prepare(K, V, beta, g, N: int | None = None, S: int | None = None, *,
     64-blocks). exact=True: T by forward substitution.
     W = T diag(beta) K, U = T diag(beta) V.
     g_raw: g holds raw log-gates (prefix-summed here). k_l2norm: rows of K are
-    normalised here (W uses the normalised keys).
+    normalised here (W uses the normalised keys). w_gated: W = T diag(beta * exp(g)) K,
+    the form in which the chunk-wise state update consumes W (U_new = U - W S_0^T for a
+    state S_0 carried into the chunk); U is unchanged.
     """
     K = np.asarray(K, dtype=np.float64)
     V = np.asarray(V, dtype=np.float64)
@@ -298,7 +300,8 @@ def chunk_prepare(K, V, beta, g, N: int | None = None, S: int | None = None, *,
         N = default_order(C) if N is None or N < 0 else N
         S = default_residual_steps(C) if S is None or S < 0 else S
         T = chunk_inverse(A, N, S, block=64 if C == 128 else None)
-    W = np.matmul(T, beta[..., :, None] * K)
+    wscale = beta * np.exp(g) if w_gated else beta
+    W = np.matmul(T, wscale[..., :, None] * K)
     U = np.matmul(T, beta[..., :, None] * V)
     return W, U, T
 

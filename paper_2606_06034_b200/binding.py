@@ -29,6 +29,7 @@ GDN_FLAG_G_RAW = 1
 GDN_FLAG_K_L2NORM = 2
 GDN_FLAG_OUT_FP32 = 4
 GDN_FLAG_LAYOUT_BTHD = 8
+GDN_FLAG_W_GATED = 16
 GDN_FWDSUBST_ROWS = 0
 GDN_FWDSUBST_BLOCKED = 1
 

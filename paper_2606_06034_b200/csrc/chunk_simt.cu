@@ -249,7 +249,9 @@ __global__ void __launch_bounds__(kThreads) chunk_simt_kernel(const IO* __restri
         for (int idx = threadIdx.x; idx < C * d_k; idx += kThreads) {
             const int i = idx / d_k, d = idx % d_k;
             float acc = 0.f;
-            for (int j = 0; j <= i; ++j) acc = fmaf(sT[i * ld + j] * sbeta[j] * srn[j], to_f32<IO>(Kc + (long long)j * d_k + d), acc);
+            for (int j = 0; j <= i; ++j)
+                acc = fmaf(sT[i * ld + j] * sbeta[j] * srn[j] * ((flags & GDN_FLAG_W_GATED) ? expf(sg[j]) : 1.f),
+                           to_f32<IO>(Kc + (long long)j * d_k + d), acc);
             st(Wc + (long long)i * d_k + d, acc);
         }
         for (int idx = threadIdx.x; idx < C * d_v; idx += kThreads) {

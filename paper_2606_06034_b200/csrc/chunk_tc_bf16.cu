@@ -438,6 +438,8 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     float* swt = reinterpret_cast<float*>(smem + L::kWt);
     const bool f_graw = EX && (p.flags & GDN_FLAG_G_RAW) != 0;
     const bool f_l2 = EX && (p.flags & GDN_FLAG_K_L2NORM) != 0;
+    const bool f_wg = EX && (p.flags & GDN_FLAG_W_GATED) != 0;
+    const bool two_scales = f_l2 || f_wg;  // the W operand is scaled by something other than beta
     const bool f_f32 = EX && (p.flags & GDN_FLAG_OUT_FP32) != 0;
 
     __shared__ uint64_t bar_k, bar_v, bar_mma;
@@ -639,10 +641,14 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     if (col0 + jl == il) gd = a[jl];
                 const float rn = rsqrtf(fmaxf(gd, 1e-30f));
                 srn[t] = rn;
-                sbrn[t] = bi * rn;
+                sbrn[t] = bi * rn * (f_wg ? fast_exp2(gi_ * kLog2e) : 1.f);
             }
             compute_barrier();
             rni = srn[t];
+        } else if (f_wg) {
+            // gated W: the column scale of the W operand is beta_j exp(g_j)
+            if (h == 0) sbrn[t] = bi * fast_exp2(gi_ * kLog2e);
+            compute_barrier();
         }
         if (active) {
             const float gs = gi_ * kLog2e;
@@ -1220,8 +1226,8 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         // ---- A operands for W/U: T diag(scale) = hi + lo, hi over the whole row, lo only on band + diagonal.
         // scale = beta for U; for W it is beta / ||K|| when the keys are normalised on the fly, else beta as well
         if (active) {
-            build_wu_operands<C, NB, MERGE, MERGE && !Y_EARLY>(lane_base, br_line, slot, t, h, il, cb, col0, wq, f_l2 ? sbrn : sbeta,
-                                            f_l2 ? bi * rni : bi, a, keep, lb, y);
+            build_wu_operands<C, NB, MERGE, MERGE && !Y_EARLY>(lane_base, br_line, slot, t, h, il, cb, col0, wq, two_scales ? sbrn : sbeta,
+                                            two_scales ? sbrn[t] : bi, a, keep, lb, y);
             if constexpr (MERGE) {
                 // I + L again for the Tinv rows: rebuilt here instead of being carried across the merge, where
                 // registers are scarce (it must be built before the barrier below: the Tinv staging lines of other
@@ -1378,8 +1384,8 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 if (lane == 0) tma_store_wait_read<0>();
                 tc_fence_before_sync();
                 compute_barrier();  // every row of the W accumulator has been read
-                if (f_l2) {
-                    // U uses beta where W used beta / ||K||: rebuild both A operands
+                if (two_scales) {
+                    // U uses beta where W used beta / ||K|| (or beta exp(g)): rebuild both A operands
                     if (active) {
                         build_wu_operands<C, NB, MERGE, MERGE && !Y_EARLY>(lane_base, br_line, slot, t, h, il, cb, col0, wq, sbeta, bi, a, keep, lb, y);
                         tmem_wait_st();

@@ -112,7 +112,8 @@ int gdn_chunk_prepare_gqa(const void* K, const void* V, const float* beta, const
 int gdn_chunk_prepare_ex(const void* K, const void* V, const float* beta, const float* g, int B, int H_k, int H_v, int T, int C,
                          int d_k, int d_v, int order, int residual_steps, int dtype, void* W_out, void* U_out, void* Tinv_out,
                          unsigned flags, gdn_stream_t stream) {
-    if (flags & ~static_cast<unsigned>(GDN_FLAG_G_RAW | GDN_FLAG_K_L2NORM | GDN_FLAG_OUT_FP32 | GDN_FLAG_LAYOUT_BTHD))
+    if (flags & ~static_cast<unsigned>(GDN_FLAG_G_RAW | GDN_FLAG_K_L2NORM | GDN_FLAG_OUT_FP32 | GDN_FLAG_LAYOUT_BTHD |
+                                       GDN_FLAG_W_GATED))
         return GDN_ERR_INVALID_ARG;
     Problem p{K, V, beta, g, W_out, U_out, Tinv_out, B, H_k, H_v, T, C, d_k, d_v, order, residual_steps, dtype};
     p.flags = flags;

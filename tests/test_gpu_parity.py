@@ -252,7 +252,8 @@ def _check_ex(inp, graw, flags, tol, N=-1, S=-1):
     Kc = np.stack([s[0] for s in sl]); Vc = np.stack([s[1] for s in sl]); bc = np.stack([s[2] for s in sl])
     gsrc = graw if g_raw else inp.g
     gc = gsrc.double().numpy().reshape(inp.n_chunks, inp.C)
-    Wo, Uo, To = orc.chunk_prepare(Kc, Vc, bc, gc, None if N < 0 else N, None if S < 0 else S, g_raw=g_raw, k_l2norm=l2)
+    Wo, Uo, To = orc.chunk_prepare(Kc, Vc, bc, gc, None if N < 0 else N, None if S < 0 else S, g_raw=g_raw, k_l2norm=l2,
+                                   w_gated=bool(flags & gdn.GDN_FLAG_W_GATED))
     for name, got, ref in (("Tinv", Tg, To), ("W", Wg, Wo), ("U", Ug, Uo)):
         err = orc.rel_frobenius(got, ref)
         assert err.max() <= tol, f"{name} rel-F {err.max():.3e} at chunk {err.argmax()} (flags {flags})"
@@ -272,6 +273,22 @@ def test_bf16_fp32_outputs_show_the_accumulators(C, adv):
     MMA operands, which the fp32 band / hi-lo split keeps small even for strongly correlated keys."""
     inp = gen.make_inputs(1, 2, 2, 512, C, 128, 128, seed=230 + C, adversarial_heads=adv)
     _check_ex(inp, None, gdn.GDN_FLAG_OUT_FP32, 5e-4)
+
+
+@pytest.mark.parametrize("C", [16, 32, 64, 128])
+@pytest.mark.parametrize("flags", [16, 17, 19, 23])
+def test_bf16_gated_w(C, flags):
+    """GDN_FLAG_W_GATED: W = T diag(beta exp(g)) K, alone and with the raw-gate / key-normalisation / fp32 flags."""
+    inp, graw = _raw_inputs(1, 2, 2, 4 * C, C, seed=300 + C + flags, adv="odd" if C <= 64 else "none")
+    if not (flags & gdn.GDN_FLAG_K_L2NORM):
+        inp = gen.make_inputs(1, 2, 2, 4 * C, C, 128, 128, seed=300 + C + flags, adversarial_heads="odd" if C <= 64 else "none")
+    _check_ex(inp, graw, flags, 5e-4 if (flags & gdn.GDN_FLAG_OUT_FP32) else TOL_BF16 + 3e-4)
+
+
+@pytest.mark.parametrize("C", [16, 64, 128])
+def test_fp32_gated_w(C):
+    inp, graw = _raw_inputs(1, 1, 2, 2 * C, C, seed=310 + C, dtype=torch.float32)
+    _check_ex(inp, graw, 16 + 3, TOL_FP32 * 3)
 
 
 def test_bf16_all_flags_together_gqa_ragged():
@@ -333,7 +350,7 @@ def test_ex_rejects_unknown_flags():
     inp = gen.make_inputs(1, 1, 1, 128, 64, 128, 128, seed=270)
     K, V, beta, g = _to_dev(inp)
     W, U, Tinv = gdn.alloc_outputs(K, V, 64)
-    rc = gdn.gdn_chunk_prepare_ex(K, V, beta, g, 1, 1, 1, 128, 64, 128, 128, -1, -1, 1, W, U, Tinv, 16, check=False)
+    rc = gdn.gdn_chunk_prepare_ex(K, V, beta, g, 1, 1, 1, 128, 64, 128, 128, -1, -1, 1, W, U, Tinv, 32, check=False)
     assert rc == gdn.GDN_ERR_INVALID_ARG
 
 

@@ -88,6 +88,18 @@ def test_chunk_quantities_reproduce_gated_delta_rule_recurrence():
     S_chunk = S0 + sum(np.outer(Unew[i], K[i]) for i in range(C))
     assert np.allclose(S_end, S_chunk, atol=1e-12)
 
+    # gated AND a non-zero initial state: needs the gated W = T diag(beta exp(g)) K
+    Wg, Ug, _ = orc.chunk_prepare(K, V, beta, g, exact=True, w_gated=True)
+    assert np.array_equal(Ug, U)
+    S_end = recurrence(S0, graw)
+    Unew = Ug - Wg @ S0.T
+    S_chunk = math.exp(g[-1]) * S0 + sum(math.exp(g[-1] - g[i]) * np.outer(Unew[i], K[i]) for i in range(C))
+    assert np.allclose(S_end, S_chunk, atol=1e-12)
+    # and the ungated W would be wrong here
+    Unew_bad = U - W @ S0.T
+    S_bad = math.exp(g[-1]) * S0 + sum(math.exp(g[-1] - g[i]) * np.outer(Unew_bad[i], K[i]) for i in range(C))
+    assert not np.allclose(S_end, S_bad, atol=1e-6)
+
 
 # -- P2 / P12: exact inverse -----------------------------------------------------
 def test_forward_substitution_closed_forms_c2_c3():
