@@ -245,6 +245,8 @@ def run_ours(args, rank, world, dist_ctx):
                 "effective_tflops": n_chunks * flops_chunk / (launch_ms * 1e-3) / 1e12,
                 "tensor_time_frac_of_bf16_peak": (n_chunks * flops_chunk / (launch_ms * 1e-3) / 1e12) / bf16_peak}
 
+    per_sorted = sorted(per)
+    roofline["launch_us"] = {"mean": launch_ms * 1e3, "median": per_sorted[len(per_sorted) // 2] * 1e3, "best": per_sorted[0] * 1e3}
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
