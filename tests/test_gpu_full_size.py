@@ -87,3 +87,36 @@ def test_int8_prefill_shapes_at_full_size():
     for key in ("t_exp", "Toffq", "w_exp", "Wq", "u_exp", "Uq"):
         bad = np.argwhere(got[key] != ref[key])
         assert bad.size == 0, f"{key}: {len(bad)} mismatches, first at {bad[0]}"
+
+
+@pytest.mark.parametrize("name", ["sweep_c16", "sweep_c64", "sweep_c128", "prefill_gqa"])
+def test_repeated_launches_are_bit_identical(name):
+    """The kernels have no atomics on data and a fixed evaluation order per chunk, so repeated launches must agree
+    bit for bit, also while another stream keeps the memory system busy (a cheap probe for shared-memory or TMEM
+    races, which show up as run-to-run differences)."""
+    inp = gen.make_workload(name, device="cuda")
+    ref = gdn.chunk_prepare(inp.K, inp.V, inp.beta, inp.g, inp.C)
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+    side = torch.cuda.Stream()
+    junk = torch.empty(64 << 20, dtype=torch.uint8, device="cuda")
+    for rep in range(6):
+        if rep % 2 == 1:
+            with torch.cuda.stream(side):
+                for _ in range(8):
+                    junk.add_(1)
+        out = gdn.chunk_prepare(inp.K, inp.V, inp.beta, inp.g, inp.C)
+        for a, b in zip(out, ref):
+            assert torch.equal(a, b), f"{name}: launch {rep} differs from the first"
+    torch.cuda.synchronize()
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+
+
+def test_repeated_int8_launches_are_bit_identical():
+    inp = gen.make_workload("sweep_c64", device="cuda")
+    q = gen.make_int8_inputs(inp)
+    ref = gdn.chunk_prepare_int8(q)
+    for rep in range(4):
+        out = gdn.chunk_prepare_int8(q)
+        for a, b in zip(out, ref):
+            assert torch.equal(a, b), f"launch {rep} differs from the first"
+    assert gdn.gdn_device_status() == gdn.GDN_OK
