@@ -307,6 +307,62 @@ def chunk_prepare(K, V, beta, g, N: int | None = None, S: int | None = None, *,
 
 
 # ----------------------------------------------------------------------------
+# The rest of the chunk-wise layer: state passing and output, given W and U
+# ----------------------------------------------------------------------------
+def gated_delta_rule(Q, K, V, beta, g_raw, scale: float = 1.0, S0=None):
+    """Token-by-token gated delta rule, the definition the chunk-wise form stands for.
+
+    Q, K: [T, d_k]; V: [T, d_v]; beta, g_raw (raw per-token log-gates): [T].
+    State S is [d_v, d_k]:  S_t = a_t S_{t-1} (I - beta_t k_t k_t^T) + beta_t v_t k_t^T,  a_t = exp(g_raw_t),
+    output o_t = scale * S_t q_t. Returns (O [T, d_v], S_T).
+    """
+    Q = np.asarray(Q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64)
+    beta = np.asarray(beta, dtype=np.float64)
+    g_raw = np.asarray(g_raw, dtype=np.float64)
+    T, dv = V.shape
+    S = np.zeros((dv, K.shape[1])) if S0 is None else np.array(S0, dtype=np.float64)
+    O = np.zeros((T, dv))
+    for t in range(T):
+        S = math.exp(g_raw[t]) * S
+        S = S - beta[t] * np.outer(S @ K[t], K[t]) + beta[t] * np.outer(V[t], K[t])
+        O[t] = scale * (S @ Q[t])
+    return O, S
+
+
+def chunk_state_output(Q, K, W_gated, U, g, C: int, scale: float = 1.0, S0=None):
+    """Chunk-wise state passing and output of one (batch, head) sequence, given W and U of every chunk.
+
+    Q, K, W_gated: [T, d_k]; U: [T, d_v]; g: [T] cumulative log-gate, CHUNK-LOCAL (inclusive prefix sum that
+    restarts in every chunk of C tokens). W_gated = T diag(beta exp(g)) K, U = T diag(beta) V.
+    Per chunk, with S0 the state [d_v, d_k] carried in:
+        U_new = U - W_gated S0^T
+        o_i   = scale * ( exp(g_i) S0 q_i + sum_{j <= i} exp(g_i - g_j) <k_j, q_i> U_new_j )
+        S_end = exp(g_C) S0 + sum_j exp(g_C - g_j) U_new_j k_j^T        (g_C: the chunk's last g)
+    Returns (O [T, d_v], S after the last chunk).
+    """
+    Q = np.asarray(Q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    W_gated = np.asarray(W_gated, dtype=np.float64)
+    U = np.asarray(U, dtype=np.float64)
+    g = np.asarray(g, dtype=np.float64)
+    T, dv = U.shape
+    assert T % C == 0
+    S = np.zeros((dv, K.shape[1])) if S0 is None else np.array(S0, dtype=np.float64)
+    O = np.zeros((T, dv))
+    causal = np.tril(np.ones((C, C)))
+    for c in range(T // C):
+        sl = slice(c * C, (c + 1) * C)
+        q, k, w, u, gc = Q[sl], K[sl], W_gated[sl], U[sl], g[sl]
+        u_new = u - w @ S.T
+        P = (q @ k.T) * np.exp(gc[:, None] - gc[None, :]) * causal
+        O[sl] = scale * (np.exp(gc)[:, None] * (q @ S.T) + P @ u_new)
+        S = math.exp(gc[-1]) * S + (u_new * np.exp(gc[-1] - gc)[:, None]).T @ k
+    return O, S
+
+
+# ----------------------------------------------------------------------------
 # Error measures used by the tests and reports
 # ----------------------------------------------------------------------------
 def rel_frobenius(x: np.ndarray, ref: np.ndarray) -> np.ndarray:

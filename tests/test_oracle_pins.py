@@ -101,6 +101,40 @@ def test_chunk_quantities_reproduce_gated_delta_rule_recurrence():
     assert not np.allclose(S_end, S_bad, atol=1e-6)
 
 
+def test_chunkwise_state_passing_and_output_equal_the_token_recurrence():
+    """chunk_state_output (W, U given per chunk) against the token-by-token gated delta rule over several chunks,
+    from a non-zero initial state, with grouped scaling; also that an ungated W or a global (not chunk-local)
+    cumulative gate would be wrong, so the conventions are pinned and not just the code path."""
+    rng = np.random.default_rng(11)
+    C, n_chunks, dk, dv = 8, 4, 5, 6
+    T = C * n_chunks
+    K = rng.normal(size=(T, dk))
+    K /= np.linalg.norm(K, axis=1, keepdims=True)
+    Q = rng.normal(size=(T, dk))
+    V = rng.normal(size=(T, dv))
+    beta = 1 / (1 + np.exp(-rng.normal(size=T)))
+    graw = -np.log1p(np.exp(rng.normal(size=T)))
+    S0 = rng.normal(size=(dv, dk))
+    O_ref, S_ref = orc.gated_delta_rule(Q, K, V, beta, graw, scale=0.7, S0=S0)
+    g_local = np.cumsum(graw.reshape(n_chunks, C), axis=1).reshape(T)
+    W = np.zeros((T, dk)); U = np.zeros((T, dv)); Wplain = np.zeros((T, dk))
+    for c in range(n_chunks):
+        sl = slice(c * C, (c + 1) * C)
+        W[sl], U[sl], _ = orc.chunk_prepare(K[sl], V[sl], beta[sl], g_local[sl], exact=True, w_gated=True)
+        Wplain[sl], _, _ = orc.chunk_prepare(K[sl], V[sl], beta[sl], g_local[sl], exact=True)
+    O, S = orc.chunk_state_output(Q, K, W, U, g_local, C, scale=0.7, S0=S0)
+    assert np.allclose(O, O_ref, atol=1e-12) and np.allclose(S, S_ref, atol=1e-12)
+    # zero initial state as the default
+    O0_ref, S0_ref = orc.gated_delta_rule(Q, K, V, beta, graw)
+    O0, S0_end = orc.chunk_state_output(Q, K, W, U, g_local, C)
+    assert np.allclose(O0, O0_ref, atol=1e-12) and np.allclose(S0_end, S0_ref, atol=1e-12)
+    # conventions: the ungated W, or a cumulative gate that does not restart per chunk, give something else
+    O_bad, _ = orc.chunk_state_output(Q, K, Wplain, U, g_local, C, scale=0.7, S0=S0)
+    assert not np.allclose(O_bad, O_ref, atol=1e-6)
+    O_bad2, _ = orc.chunk_state_output(Q, K, W, U, np.cumsum(graw), C, scale=0.7, S0=S0)
+    assert not np.allclose(O_bad2, O_ref, atol=1e-6)
+
+
 # -- P2 / P12: exact inverse -----------------------------------------------------
 def test_forward_substitution_closed_forms_c2_c3():
     a = 0.37
