@@ -146,6 +146,25 @@ int gdn_chunk_prepare_int8(const int8_t* Kq, const int8_t* Vq, const int32_t* k_
                            int8_t* Wq_out, int8_t* Uq_out, int32_t* w_exp_out, int32_t* u_exp_out,
                            int8_t* Toff_q_out, int32_t* t_exp_out, int32_t* dbg_acc_out, gdn_stream_t stream);
 
+/*
+ * The rest of the chunk-wise layer (Sec. 2.1: the quantities W and U exist for this), given W and U of every chunk:
+ * state passing between chunks and the output. Per (batch, value head), chunk after chunk, with S the state
+ * [d_v x d_k] carried from chunk to chunk:
+ *     U_new = U - W S^T
+ *     o_i   = scale * ( exp(g_i) S q_i + sum_{j <= i} exp(g_i - g_j) <k_j, q_i> U_new_j )
+ *     S    <- exp(g_C) S + sum_j exp(g_C - g_j) U_new_j k_j^T          (g_C: g of the chunk's last token)
+ * which equals the token-by-token gated delta rule S_t = a_t S_{t-1} (I - beta_t k_t k_t^T) + beta_t v_t k_t^T,
+ * o_t = scale * S_t q_t when W = T diag(beta exp(g)) K (gdn_chunk_prepare_ex with GDN_FLAG_W_GATED) and
+ * U = T diag(beta) V.
+ *   Q, K [B,H_k,T,d_k], W_gated [B,H_v,T,d_k], U [B,H_v,T,d_v] bf16; g [B,H_v,T] fp32, the cumulative log-gate
+ *   that RESTARTS in every chunk (chunk-local inclusive prefix sum); S_in [B,H_v,d_v,d_k] fp32 or NULL (zero state);
+ *   O_out [B,H_v,T,d_v] bf16; S_out [B,H_v,d_v,d_k] fp32 or NULL.
+ * Supported: C = 64, d_k = d_v = 128, T a multiple of C. fp32 state, bf16 tensor-core operands.
+ */
+int gdn_chunk_state_output(const void* Q, const void* K, const void* W_gated, const void* U, const float* g,
+                           int B, int H_k, int H_v, int T, int C, int d_k, int d_v, float scale,
+                           const float* S_in, void* O_out, float* S_out, gdn_stream_t stream);
+
 /* Checksum of the 256-entry gate-decay table round(2^15 * 2^(-f/256)) the INT8 kernel uses
  * (sum_f: s = (31 s + table[f] + f) mod 1000000007), so that a CPU evaluation can confirm it holds the same table. */
 unsigned int gdn_int8_lut_checksum(void);

@@ -35,7 +35,7 @@ GDN_FWDSUBST_BLOCKED = 1
 
 EXPORTS = (
     "gdn_chunk_prepare", "gdn_chunk_prepare_gqa", "gdn_chunk_prepare_ex", "gdn_chunk_prepare_fwdsubst",
-    "gdn_chunk_prepare_int8", "gdn_selftest_bounded_wait",
+    "gdn_chunk_prepare_int8", "gdn_chunk_state_output", "gdn_selftest_bounded_wait",
     "gdn_int8_lut_checksum",
     "gdn_device_status", "gdn_default_order", "gdn_default_residual_steps",
     "gdn_status_string", "gdn_launch_count",
@@ -72,6 +72,8 @@ def load_library() -> ctypes.CDLL:
     lib.gdn_chunk_prepare_int8.restype = ip
     lib.gdn_chunk_prepare_int8.argtypes = [vp, vp, vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ip, ip, ip, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.gdn_int8_lut_checksum.restype = ctypes.c_uint
+    lib.gdn_chunk_state_output.argtypes = [vp, vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ip, ctypes.c_float, vp, vp, vp, vp]
+    lib.gdn_chunk_state_output.restype = ip
     lib.gdn_selftest_bounded_wait.argtypes = [vp]
     lib.gdn_selftest_bounded_wait.restype = ip
     lib.gdn_int8_lut_checksum.argtypes = []
@@ -228,6 +230,32 @@ def chunk_prepare_int8(q, order=-1, residual_steps=-1, *, want_toff=True, output
     gdn_chunk_prepare_int8(q.Kq, q.Vq, q.k_exp, q.v_exp, q.beta_q, q.decay_q, q.B, q.H_k, q.H_v, q.T, q.C, q.d_k, q.d_v,
                            order, residual_steps, Wq, Uq, w_exp, u_exp, Toff, t_exp, dbg_acc)
     return outputs
+
+
+def gdn_chunk_state_output(Q, K, W_gated, U, g, B, H_k, H_v, T, C, d_k, d_v, scale, S_in, O_out, S_out, *, check=True):
+    """Raw call of the state-passing / output entry point (tensors instead of pointers, torch's current stream)."""
+    for t in (Q, K, W_gated, U, g, S_in, O_out, S_out):
+        if t is not None and (not t.is_cuda or not t.is_contiguous()):
+            raise ValueError("all tensors must be contiguous CUDA tensors (there is no CPU path)")
+    rc = load_library().gdn_chunk_state_output(_ptr(Q), _ptr(K), _ptr(W_gated), _ptr(U), _ptr(g), B, H_k, H_v, T, C, d_k, d_v,
+                                               ctypes.c_float(scale), _ptr(S_in), _ptr(O_out), _ptr(S_out), _stream())
+    if check and rc != GDN_OK:
+        raise GdnError(rc, "gdn_chunk_state_output")
+    return rc
+
+
+def chunk_state_output(Q, K, W_gated, U, g, C, scale=1.0, S_in=None, *, want_state=True, outputs=None):
+    """Convenience wrapper: Q, K [B,H_k,T,d_k], W_gated [B,H_v,T,d_k], U [B,H_v,T,d_v], g [B,H_v,T] (chunk-local
+    cumulative log-gate). Returns (O [B,H_v,T,d_v], S_out [B,H_v,d_v,d_k] fp32 or None)."""
+    B, H_k, T, d_k = K.shape
+    _, H_v, _, d_v = U.shape
+    if outputs is None:
+        O = torch.empty(B, H_v, T, d_v, dtype=U.dtype, device=U.device)
+        S_out = torch.empty(B, H_v, d_v, d_k, dtype=torch.float32, device=U.device) if want_state else None
+    else:
+        O, S_out = outputs
+    gdn_chunk_state_output(Q, K, W_gated, U, g, B, H_k, H_v, T, C, d_k, d_v, scale, S_in, O, S_out)
+    return O, S_out
 
 
 def gdn_selftest_bounded_wait() -> int:

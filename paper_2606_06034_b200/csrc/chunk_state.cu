@@ -1,0 +1,470 @@
+// State passing and output of chunk-wise Gated DeltaNet, given W (gated) and U of every chunk (tcgen05 + TMEM + TMA).
+//
+// What it computes, per (batch, value head), chunk after chunk (C = 64 tokens, S0 = state [d_v x d_k] carried in,
+// g = chunk-local cumulative log-gate, W = T diag(beta exp(g)) K, U = T diag(beta) V from the chunk-prepare path):
+//     U_new = U - W S0^T
+//     o_i   = scale (exp(g_i) S0 q_i + sum_{j <= i} exp(g_i - g_j) <k_j, q_i> U_new_j)
+//     S_end = exp(g_C) S0 + sum_j exp(g_C - g_j) U_new_j k_j^T
+// This is the WY form of the gated delta rule that the chunk-prepare quantities exist for (Sec. 2.1); the chunks of
+// one head are a serial chain, heads are independent.
+//
+// Everything is evaluated with the value dimension on the 128 TMEM lanes ("transposed"): one CTA per (batch, head)
+// keeps the state S [d_v x d_k] as an fp32 accumulator in TMEM for the whole sequence, lane t = value feature t.
+//     D1  = S0 W^T - U^T      A = bf16(S0) in TMEM, B = W tile; the transpose of U comes from the tensor core as
+//                             (-I) U^T with a constant A operand, so no thread ever transposes anything
+//     PT  = K Q^T             lanes 0..63 = token j, columns = token i
+//     O1  = S0 Q^T
+//     O2  = U_new^T P^T       A = bf16(U_new^T) (written over D1's columns), B = P_ij = exp(g_i-g_j) PT_ji [j <= i]
+//     S  += (U_new^T exp(g_C - g_j)) K     accumulated onto exp(g_C) S0 (the decay is a pass over the TMEM columns)
+//     O^T = scale (exp(g_i) O1 + O2)  -> transposed through shared memory -> bulk tensor store
+// Two MMA groups per chunk; Q, K, W, U tiles of the next chunk are in flight (two stages) while a chunk is worked on.
+// All operand layouts are the ones the chunk-prepare kernel uses.
+#include <cuda.h>
+
+#include "common.cuh"
+#include "sm100_ptx.cuh"
+
+namespace gdn {
+namespace {
+
+using namespace sm100;
+
+constexpr int kC = 64;         // chunk size
+constexpr int kD = 128;        // d_k = d_v
+constexpr int kThreads = 256;  // two threads per TMEM lane
+constexpr float kLog2e = 1.4426950408889634f;
+
+// TMEM column map (512 columns: one CTA per SM)
+constexpr uint32_t kSD = 0;    // 128: state S, fp32 accumulator
+constexpr uint32_t kSA = 128;  // 64: bf16(S0) as A operand (K = d_k)
+constexpr uint32_t kIA = 192;  // 64: -I as A operand (K = d_v), constant
+constexpr uint32_t kD1 = 256;  // 64: S0 W^T - U^T, then the two bf16 forms of U_new^T as A operands
+constexpr uint32_t kPT = 320;  // 64: K Q^T (lanes 0..63)
+constexpr uint32_t kO1 = 384;  // 64: S0 Q^T
+constexpr uint32_t kO2 = 448;  // 64: U_new^T P^T
+constexpr uint32_t kTmemCols = 512;
+
+// shared memory map (bytes; 1 KB aligned). A [64 x 128] bf16 tile is two [64 x 64] sub-tiles of 8 KB (128B swizzle).
+constexpr int kTileBytes = 16384;
+constexpr int kStageBytes = 4 * kTileBytes;  // Q, K, W, U
+constexpr int kOffQ = 0, kOffK = kTileBytes, kOffW = 2 * kTileBytes, kOffU = 3 * kTileBytes;
+constexpr int kOffP = 2 * kStageBytes;       // 8 KB: P as B operand [64 x 64] (MN-major, no swizzle)
+constexpr int kOffO = kOffP + 8192;          // 16 KB: O tile staged for the bulk store (128B swizzle)
+constexpr int kOffG = kOffO + kTileBytes;    // 3 x 64 floats: exp(g_i), exp(g_C - g_j), g
+constexpr int kSmemTotal = kOffG + 3 * 64 * 4;
+
+struct ParamsS {
+    const float* g;
+    const float* S_in;  // may be null
+    float* S_out;       // may be null
+    int* status;
+    int H_k, H_v, T, group;
+    float scale;
+};
+
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// bounded mbarrier wait (about a second), as in the chunk-prepare kernels
+__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    uint32_t i = 0;
+    while (!mbar_try_wait_hint(bar, parity, 2000u)) {
+        if ((++i & 63u) == 0 && clock64() - t0 > 2000000000LL) return false;
+    }
+    return true;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                   const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmU,
+                   const __grid_constant__ CUtensorMap tmO, const ParamsS p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    float* se = reinterpret_cast<float*>(smem + kOffG);  // exp(g_i)
+    float* sf = se + 64;                                  // exp(g_C - g_j)
+    float* sg = sf + 64;                                  // g_i
+
+    __shared__ uint64_t bar_full[2], bar_mma;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int s_fail;
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    const int lane = tid & 31;
+    const int t = tid & 127;  // TMEM lane: value feature (state rows, output columns); token j for PT
+    const int h = tid >> 7;   // column half
+    const int wq = warp & 3;
+
+    if (tid == 0) {
+        mbar_init(&bar_full[0], 1);
+        mbar_init(&bar_full[1], 1);
+        mbar_init(&bar_mma, 1);
+        s_fail = 0;
+        mbar_fence_init();
+        tma_prefetch_desc(&tmQ);
+        tma_prefetch_desc(&tmK);
+        tma_prefetch_desc(&tmW);
+        tma_prefetch_desc(&tmU);
+        tma_prefetch_desc(&tmO);
+    }
+    if (warp == 0) {
+        tmem_alloc(&tmem_base_s, kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = tmem_base_s;
+    const uint32_t lane_base = tmem + (static_cast<uint32_t>(wq * 32) << 16);
+
+    const int bhv = blockIdx.x;
+    const int b = bhv / p.H_v, hv = bhv - b * p.H_v;
+    const int bhk = b * p.H_k + hv / p.group;
+    const int n_c = p.T / kC;
+    const float* gseq = p.g + (long long)bhv * p.T;
+    const uint32_t smem_a = smem_u32(smem);
+    // M = 128, N = 64 / 128; A from TMEM (or K-major shared memory), B K-major or MN-major
+    const uint32_t idesc_kk64 = instr_desc(128, 64, 1, 1, 0, 0, 1);
+    const uint32_t idesc_mn64 = instr_desc(128, 64, 1, 1, 0, 1, 1);
+    const uint32_t idesc_mn128 = instr_desc(128, 128, 1, 1, 0, 1, 1);
+
+    uint32_t par_mma = 0;
+    bool ok = true;
+    auto wait_mma = [&]() -> bool {
+        if (warp == 0 && !wait_bar(&bar_mma, par_mma)) *reinterpret_cast<volatile int*>(&s_fail) = 1;
+        asm volatile("bar.sync 2, 256;" ::: "memory");
+        par_mma ^= 1;
+        return *reinterpret_cast<volatile int*>(&s_fail) == 0;
+    };
+    auto load_stage = [&](int c) {  // one elected thread: the four tiles of chunk c into stage c & 1
+        uint8_t* st = smem + (c & 1) * kStageBytes;
+        uint64_t* bar = &bar_full[c & 1];
+        mbar_arrive_expect_tx(bar, kStageBytes);
+        const int t0 = c * kC;
+        tma_load_3d(st + kOffQ, &tmQ, bar, 0, t0, bhk);
+        tma_load_3d(st + kOffQ + 8192, &tmQ, bar, 64, t0, bhk);
+        tma_load_3d(st + kOffK, &tmK, bar, 0, t0, bhk);
+        tma_load_3d(st + kOffK + 8192, &tmK, bar, 64, t0, bhk);
+        tma_load_3d(st + kOffW, &tmW, bar, 0, t0, bhv);
+        tma_load_3d(st + kOffW + 8192, &tmW, bar, 64, t0, bhv);
+        tma_load_3d(st + kOffU, &tmU, bar, 0, t0, bhv);
+        tma_load_3d(st + kOffU + 8192, &tmU, bar, 64, t0, bhv);
+    };
+
+    if (warp == 0 && n_c > 0 && elect_one()) {
+        load_stage(0);
+        if (n_c > 1) load_stage(1);
+    }
+
+    // ---- constant A operand -I, initial state, and its bf16 copy
+    {
+        uint32_t r[16];
+#pragma unroll
+        for (int part = 0; part < 2; ++part) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const int col = h * 32 + part * 16 + i;  // packed column: features 2 col, 2 col + 1
+                r[i] = (col == (t >> 1)) ? ((t & 1) ? 0xBF800000u : 0x0000BF80u) : 0u;
+            }
+            tmem_st16(lane_base + kIA + h * 32 + part * 16, r);
+        }
+        // this thread's half of state row t: columns [64 h, 64 h + 64)
+        const float* s0 = (p.S_in != nullptr) ? p.S_in + ((long long)bhv * kD + t) * kD + h * 64 : nullptr;
+#pragma unroll
+        for (int part = 0; part < 4; ++part) {
+            uint32_t v[16], pk[8];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) v[i] = (s0 != nullptr) ? __float_as_uint(__ldg(s0 + part * 16 + i)) : 0u;
+            tmem_st16(lane_base + kSD + h * 64 + part * 16, v);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) pk[i] = pack_bf16x2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
+            tmem_st8(lane_base + kSA + h * 32 + part * 8, pk);
+        }
+        tmem_wait_st();
+    }
+    // gates of the first chunk
+    float g_reg = 0.f, gC_reg = 0.f;
+    if (n_c > 0) {
+        if (tid < 64) g_reg = __ldg(gseq + tid);
+        gC_reg = __ldg(gseq + kC - 1);
+    }
+
+    for (int c = 0; c < n_c; ++c) {
+        uint8_t* st = smem + (c & 1) * kStageBytes;
+        const uint32_t st_a = smem_a + (c & 1) * kStageBytes;
+        const float gC = gC_reg;
+        if (tid < 64) {
+            sg[tid] = g_reg;
+            se[tid] = fast_exp2(g_reg * kLog2e);
+            sf[tid] = fast_exp2((gC - g_reg) * kLog2e);
+        }
+        if (c + 1 < n_c) {
+            if (tid < 64) g_reg = __ldg(gseq + (c + 1) * kC + tid);
+            gC_reg = __ldg(gseq + (c + 2) * kC - 1);
+        }
+        // the previous chunk's output store has finished reading the staging tile
+        if (tid == 0) tma_store_wait_read<0>();
+        tc_fence_before_sync();
+        __syncthreads();  // bf16(S0) and the gate tables are in place
+
+        if (warp == 0) {
+            if (!wait_bar(&bar_full[c & 1], (c >> 1) & 1)) *reinterpret_cast<volatile int*>(&s_fail) = 1;
+            tc_fence_after_sync();
+            if (*reinterpret_cast<volatile int*>(&s_fail) == 0 && elect_one()) {
+                // D1 = (-I) U^T + S0 W^T
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint64_t bd = smem_desc(st_a + kOffU + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024, SWZ_128B);
+                    mma_f16_ts(tmem + kD1, tmem + kIA + ks * 8, bd, idesc_kk64, ks > 0);
+                }
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint64_t bd = smem_desc(st_a + kOffW + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024, SWZ_128B);
+                    mma_f16_ts(tmem + kD1, tmem + kSA + ks * 8, bd, idesc_kk64, true);
+                }
+                // PT = K Q^T (rows 64..127 of the A operand read past the 64-row tile: unused lanes)
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint64_t ad = smem_desc(st_a + kOffK + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024, SWZ_128B);
+                    const uint64_t bd = smem_desc(st_a + kOffQ + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024, SWZ_128B);
+                    mma_f16_ss(tmem + kPT, ad, bd, idesc_kk64, ks > 0);
+                }
+                // O1 = S0 Q^T
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint64_t bd = smem_desc(st_a + kOffQ + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024, SWZ_128B);
+                    mma_f16_ts(tmem + kO1, tmem + kSA + ks * 8, bd, idesc_kk64, ks > 0);
+                }
+                mma_commit(&bar_mma);
+            }
+        }
+        // ---- while those run: decay of the accumulator, S <- exp(g_C) S0 (the products above read the bf16 copy)
+        {
+            const float dec = fast_exp2(gC * kLog2e);
+#pragma unroll
+            for (int part = 0; part < 2; ++part) {
+                uint32_t v[32];
+                tmem_ld32(lane_base + kSD + h * 64 + part * 32, v);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * dec);
+                uint32_t w16[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) w16[i] = v[i];
+                tmem_st16(lane_base + kSD + h * 64 + part * 32, w16);
+#pragma unroll
+                for (int i = 0; i < 16; ++i) w16[i] = v[16 + i];
+                tmem_st16(lane_base + kSD + h * 64 + part * 32 + 16, w16);
+            }
+            tmem_wait_st();
+        }
+        if (!wait_mma()) { ok = false; break; }
+        tc_fence_after_sync();
+
+        // ---- U_new^T = -D1: plain and gate-scaled bf16 copies, written over this thread's own D1 columns
+        // (h = 0: plain -> columns 0..15, scaled -> 16..31; h = 1: 32..47 and 48..63)
+        {
+            uint32_t d[32];
+            tmem_ld32(lane_base + kD1 + h * 32, d);
+            tmem_wait_ld();
+            uint32_t pp[16], ps[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const float u0 = -__uint_as_float(d[2 * i]), u1 = -__uint_as_float(d[2 * i + 1]);
+                const float2 f = *reinterpret_cast<const float2*>(sf + h * 32 + 2 * i);
+                pp[i] = pack_bf16x2(u0, u1);
+                ps[i] = pack_bf16x2(u0 * f.x, u1 * f.y);
+            }
+            tmem_st16(lane_base + kD1 + h * 32, pp);
+            tmem_st16(lane_base + kD1 + h * 32 + 16, ps);
+        }
+        // ---- P_ij = exp(g_i - g_j) PT_ji for j <= i: token j = lane (rows 0..63 only), this thread's 32 columns i
+        if (wq < 2) {
+            uint32_t d[32];
+            tmem_ld32(lane_base + kPT + h * 32, d);
+            tmem_wait_ld();
+            const float gj = sg[t] * kLog2e;
+#pragma unroll
+            for (int c4 = 0; c4 < 4; ++c4) {
+                uint32_t w[4];
+#pragma unroll
+                for (int i2 = 0; i2 < 4; ++i2) {
+                    float v[2];
+#pragma unroll
+                    for (int q = 0; q < 2; ++q) {
+                        const int i = h * 32 + c4 * 8 + i2 * 2 + q;
+                        const float x = __uint_as_float(d[c4 * 8 + i2 * 2 + q]) * fast_exp2(fminf(fmaf(sg[i], kLog2e, -gj), 0.f));
+                        v[q] = (t <= i) ? x : 0.f;
+                    }
+                    w[i2] = pack_bf16x2(v[0], v[1]);
+                }
+                // B operand [K-dim = j][N = i], MN-major, no swizzle: the 16-byte piece of row j for column group n8
+                *reinterpret_cast<uint4*>(smem + kOffP + (h * 4 + c4) * 1024 + t * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+        }
+        fence_proxy_async_smem();
+        tmem_wait_st();
+        tc_fence_before_sync();
+        __syncthreads();
+
+        if (warp == 0) {
+            tc_fence_after_sync();
+            if (elect_one()) {
+                // O2 = U_new^T P^T (K-dim = 64 tokens; the plain copy sits at columns 0..15 and 32..47)
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) {
+                    const uint64_t bd = smem_desc(smem_a + kOffP + ks * 256, 128, 1024, SWZ_NONE);
+                    mma_f16_ts(tmem + kO2, tmem + kD1 + (ks < 2 ? ks * 8 : 32 + (ks - 2) * 8), bd, idesc_mn64, ks > 0);
+                }
+                // S += (U_new^T exp(g_C - g_j)) K (the K tile as MN-major operand, N = 128)
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) {
+                    const uint64_t bd = smem_desc(st_a + kOffK + ks * 2048, 8192, 1024, SWZ_128B);
+                    mma_f16_ts(tmem + kSD, tmem + kD1 + 16 + (ks < 2 ? ks * 8 : 32 + (ks - 2) * 8), bd, idesc_mn128, true);
+                }
+                mma_commit(&bar_mma);
+            }
+        }
+        // ---- meanwhile: exp(g_i) O1
+        float o[32];
+        {
+            uint32_t d[32];
+            tmem_ld32(lane_base + kO1 + h * 32, d);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) o[i] = __uint_as_float(d[i]) * se[h * 32 + i];
+        }
+        if (!wait_mma()) { ok = false; break; }
+        tc_fence_after_sync();
+        // the tiles of this stage are free: the chunk after the next one may land there
+        if (warp == 0 && c + 2 < n_c && elect_one()) load_stage(c + 2);
+
+        // ---- O^T = scale (exp(g_i) O1 + O2): element (token i, feature t) of the staged tile
+        {
+            uint32_t d[32];
+            tmem_ld32(lane_base + kO2 + h * 32, d);
+            tmem_wait_ld();
+            uint8_t* sub = smem + kOffO + (t >> 6) * 8192;
+            const int cch = (t & 63) >> 3;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const int tok = h * 32 + i;
+                const __nv_bfloat16 v = __float2bfloat16_rn(p.scale * (o[i] + __uint_as_float(d[i])));
+                *reinterpret_cast<__nv_bfloat16*>(sub + tok * 128 + ((cch ^ (tok & 7)) << 4) + (t & 7) * 2) = v;
+            }
+        }
+        // ---- bf16 copy of the new state for the next chunk's products
+        {
+#pragma unroll
+            for (int part = 0; part < 2; ++part) {
+                uint32_t v[32], pk[16];
+                tmem_ld32(lane_base + kSD + h * 64 + part * 32, v);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 16; ++i) pk[i] = pack_bf16x2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
+                tmem_st16(lane_base + kSA + h * 32 + part * 16, pk);
+            }
+            tmem_wait_st();
+        }
+        fence_proxy_async_smem();
+        tc_fence_before_sync();
+        __syncthreads();
+        if (tid == 0) {  // the same thread waits for these stores (bulk groups are per thread)
+            tma_store_3d(&tmO, smem + kOffO, 0, c * kC, bhv);
+            tma_store_3d(&tmO, smem + kOffO + 8192, 64, c * kC, bhv);
+            tma_store_commit();
+        }
+    }
+
+    // ---- final state
+    if (ok && p.S_out != nullptr) {
+        float* so = p.S_out + ((long long)bhv * kD + t) * kD + h * 64;
+#pragma unroll
+        for (int part = 0; part < 2; ++part) {
+            uint32_t v[32];
+            tmem_ld32(lane_base + kSD + h * 64 + part * 32, v);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                *reinterpret_cast<float4*>(so + part * 32 + i * 4) =
+                    make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]), __uint_as_float(v[4 * i + 2]),
+                                __uint_as_float(v[4 * i + 3]));
+        }
+    }
+    if (tid == 0) tma_store_wait_all<0>();
+    if (!ok) atomicExch(p.status, GDN_ERR_TIMEOUT);
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem, kTmemCols);
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (fn == nullptr) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess)
+            return nullptr;
+        fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+// [heads][T][128] bf16 tensor, boxes of 64 rows x 64 columns, 128-byte swizzle
+bool make_map(CUtensorMap* tm, const void* base, long long heads, int T) {
+    EncodeTiledFn enc = get_encode_fn();
+    if (enc == nullptr) return false;
+    cuuint64_t dims[3] = {static_cast<cuuint64_t>(kD), static_cast<cuuint64_t>(T), static_cast<cuuint64_t>(heads)};
+    cuuint64_t strides[2] = {static_cast<cuuint64_t>(kD) * 2, static_cast<cuuint64_t>(T) * kD * 2};
+    cuuint32_t box[3] = {64, static_cast<cuuint32_t>(kC), 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+int launch_chunk_state(const ProblemS& q, cudaStream_t stream) {
+    if (q.d_k != kD || q.d_v != kD || q.C != kC) return GDN_ERR_UNSUPPORTED;
+    const long long hk = (long long)q.B * q.H_k, hv = (long long)q.B * q.H_v;
+    if (hv == 0 || q.T == 0) return GDN_OK;
+    if (hv >= (1LL << 31)) return GDN_ERR_UNSUPPORTED;
+    int* status = device_status_word();
+    if (status == nullptr) return GDN_ERR_LAUNCH;
+    CUtensorMap mQ, mK, mW, mU, mO;
+    if (!make_map(&mQ, q.Q, hk, q.T) || !make_map(&mK, q.K, hk, q.T) || !make_map(&mW, q.W, hv, q.T) ||
+        !make_map(&mU, q.U, hv, q.T) || !make_map(&mO, q.O, hv, q.T))
+        return GDN_ERR_LAUNCH;
+    ParamsS prm;
+    prm.g = q.g;
+    prm.S_in = q.S_in;
+    prm.S_out = q.S_out;
+    prm.status = status;
+    prm.H_k = q.H_k;
+    prm.H_v = q.H_v;
+    prm.T = q.T;
+    prm.group = q.H_v / q.H_k;
+    prm.scale = q.scale;
+    const int smem = kSmemTotal + 1024;
+    if (cudaFuncSetAttribute(chunk_state_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+        return GDN_ERR_LAUNCH;
+    chunk_state_kernel<<<static_cast<int>(hv), kThreads, smem, stream>>>(mQ, mK, mW, mU, mO, prm);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? GDN_OK : GDN_ERR_LAUNCH;
+}
+
+}  // namespace gdn

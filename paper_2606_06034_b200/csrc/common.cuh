@@ -43,6 +43,20 @@ struct ProblemI8 {
     int order, steps;
 };
 
+// State passing + output of the layer, given W (gated) and U of every chunk
+struct ProblemS {
+    const void* Q;
+    const void* K;
+    const void* W;
+    const void* U;
+    const float* g;
+    const float* S_in;  // may be null (zero state)
+    void* O;
+    float* S_out;       // may be null
+    int B, H_k, H_v, T, C, d_k, d_v;
+    float scale;
+};
+
 enum InverseMode { INV_NEUMANN = 0, INV_FWDSUBST_ROWS = 1, INV_FWDSUBST_BLOCKED = 2 };
 
 // Status word written by kernels (one per device, static device memory).
@@ -53,6 +67,7 @@ void count_launch();
 int launch_simt(const Problem& p, InverseMode mode, cudaStream_t stream);
 int launch_tc_bf16(const Problem& p, InverseMode mode, cudaStream_t stream);
 int launch_wait_selftest(cudaStream_t stream);
+int launch_chunk_state(const ProblemS& p, cudaStream_t stream);
 int launch_tc_int8(const ProblemI8& p, cudaStream_t stream);
 void int8_decay_lut(uint16_t* out256);  // table of round(2^15 * 2^(-f/256))
 

@@ -149,6 +149,21 @@ int gdn_chunk_prepare_int8(const int8_t* Kq, const int8_t* Vq, const int32_t* k_
     return launch_tc_int8(q, static_cast<cudaStream_t>(stream));
 }
 
+int gdn_chunk_state_output(const void* Q, const void* K, const void* W_gated, const void* U, const float* g, int B, int H_k,
+                           int H_v, int T, int C, int d_k, int d_v, float scale, const float* S_in, void* O_out, float* S_out,
+                           gdn_stream_t stream) {
+    if (Q == nullptr || K == nullptr || W_gated == nullptr || U == nullptr || g == nullptr || O_out == nullptr) return GDN_ERR_NULL;
+    if (B < 0 || H_k <= 0 || H_v <= 0 || T < 0 || C < 2 || d_k <= 0 || d_v <= 0) return GDN_ERR_INVALID_ARG;
+    if (H_v % H_k != 0 || T % C != 0) return GDN_ERR_INVALID_ARG;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(W_gated) || !aligned16(U) || !aligned16(g) || !aligned16(S_in) ||
+        !aligned16(O_out) || !aligned16(S_out))
+        return GDN_ERR_ALIGN;
+    const int rc = check_arch();
+    if (rc != GDN_OK) return rc;
+    ProblemS q{Q, K, W_gated, U, g, S_in, O_out, S_out, B, H_k, H_v, T, C, d_k, d_v, scale};
+    return launch_chunk_state(q, static_cast<cudaStream_t>(stream));
+}
+
 int gdn_selftest_bounded_wait(gdn_stream_t stream) {
     const int rc = check_arch();
     if (rc != GDN_OK) return rc;

@@ -1,0 +1,90 @@
+"""State passing + output of the chunk-wise layer (gdn_chunk_state_output) against the fp64 oracle.
+
+The CUDA call consumes the bf16 W (gated) and U that the chunk-prepare kernel produced; the oracle is given exactly the
+same values (upcast), so what is compared is this step alone. A second test runs the two CUDA calls back to back
+against the token-by-token gated delta rule on the original inputs (the whole layer)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import gdn_oracle as orc
+from paper_2606_06034_b200 import binding as gdn
+from paper_2606_06034_b200 import inputs as gen
+
+pytestmark = pytest.mark.gpu
+
+# relative Frobenius error per chunk of O and of the final state: bf16 operands (state, U_new, P) with fp32
+# accumulation and a bf16 output
+TOL_O = 4e-3
+TOL_S = 2e-3
+
+
+def _queries(inp, seed):
+    gq = torch.Generator().manual_seed(seed)
+    Q = torch.randn(inp.B, inp.H_k, inp.T, inp.d_k, generator=gq)
+    Q = Q / Q.norm(dim=-1, keepdim=True)
+    return Q.to(inp.K.dtype).contiguous()
+
+
+def _run(inp, Q, scale, S0):
+    K, V, beta, g = inp.K.cuda(), inp.V.cuda(), inp.beta.cuda(), inp.g.cuda()
+    W, U, _ = gdn.chunk_prepare(K, V, beta, g, inp.C, flags=gdn.GDN_FLAG_W_GATED)
+    O, S = gdn.chunk_state_output(Q.cuda(), K, W, U, g, inp.C, scale, None if S0 is None else S0.cuda())
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+    return W, U, O, S
+
+
+@pytest.mark.parametrize("B,H_k,H_v,T", [(1, 1, 1, 64), (1, 1, 1, 256), (2, 2, 4, 512), (1, 2, 2, 1024)])
+@pytest.mark.parametrize("with_state", [False, True])
+def test_state_output_matches_oracle(B, H_k, H_v, T, with_state):
+    C = 64
+    inp = gen.make_inputs(B, H_k, H_v, T, C, 128, 128, seed=400 + T + H_v)
+    Q = _queries(inp, 401 + T)
+    scale = 128 ** -0.5
+    S0 = None
+    if with_state:
+        S0 = 0.1 * torch.randn(B, H_v, 128, 128, generator=torch.Generator().manual_seed(402))
+    W, U, O, S = _run(inp, Q, scale, S0)
+    group = H_v // H_k
+    for b in range(B):
+        for hv in range(H_v):
+            hk = hv // group
+            Oo, So = orc.chunk_state_output(Q[b, hk].double().numpy(), inp.K[b, hk].double().numpy(),
+                                            W[b, hv].double().cpu().numpy(), U[b, hv].double().cpu().numpy(),
+                                            inp.g[b, hv].double().numpy(), C, scale,
+                                            None if S0 is None else S0[b, hv].double().numpy())
+            Og = O[b, hv].double().cpu().numpy().reshape(T // C, C, 128)
+            eO = orc.rel_frobenius(Og, Oo.reshape(T // C, C, 128))
+            assert eO.max() <= TOL_O, f"O rel-F {eO.max():.3e} at chunk {eO.argmax()} of head ({b},{hv})"
+            eS = orc.rel_frobenius(S[b, hv].double().cpu().numpy()[None], So[None])
+            assert eS.max() <= TOL_S, f"S rel-F {eS.max():.3e} of head ({b},{hv})"
+
+
+def test_whole_layer_matches_the_token_recurrence():
+    """chunk-prepare (gated W, U) + state passing/output on the GPU against the token-by-token gated delta rule."""
+    C, T = 64, 512
+    inp = gen.make_inputs(1, 1, 2, T, C, 128, 128, seed=410)
+    Q = _queries(inp, 411)
+    scale = 128 ** -0.5
+    _, _, O, S = _run(inp, Q, scale, None)
+    graw = inp.g.view(1, 2, T // C, C).diff(dim=-1, prepend=torch.zeros(1, 2, T // C, 1)).reshape(1, 2, T)
+    for hv in range(2):
+        Oo, So = orc.gated_delta_rule(Q[0, 0].double().numpy(), inp.K[0, 0].double().numpy(), inp.V[0, hv].double().numpy(),
+                                      inp.beta[0, hv].double().numpy(), graw[0, hv].double().numpy(), scale)
+        Og = O[0, hv].double().cpu().numpy().reshape(T // C, C, 128)
+        eO = orc.rel_frobenius(Og, Oo.reshape(T // C, C, 128))
+        assert eO.max() <= 1e-2, f"O rel-F {eO.max():.3e} at chunk {eO.argmax()}"
+        eS = orc.rel_frobenius(S[0, hv].double().cpu().numpy()[None], So[None])
+        assert eS.max() <= 1e-2, f"S rel-F {eS.max():.3e}"
+
+
+def test_state_output_argument_errors():
+    inp = gen.make_inputs(1, 1, 1, 128, 64, 128, 128, seed=420)
+    K = inp.K.cuda()
+    g = inp.g.cuda()
+    O = torch.empty(1, 1, 128, 128, dtype=torch.bfloat16, device="cuda")
+    args = dict(check=False)
+    assert gdn.gdn_chunk_state_output(K, K, K, K, g, 1, 1, 1, 128, 32, 128, 128, 1.0, None, O, None, **args) == gdn.GDN_ERR_UNSUPPORTED
+    assert gdn.gdn_chunk_state_output(K, K, K, K, g, 1, 1, 1, 100, 64, 128, 128, 1.0, None, O, None, **args) == gdn.GDN_ERR_INVALID_ARG
+    assert gdn.gdn_chunk_state_output(None, K, K, K, g, 1, 1, 1, 128, 64, 128, 128, 1.0, None, O, None, **args) == gdn.GDN_ERR_NULL
+    assert gdn.gdn_device_status() == gdn.GDN_OK
