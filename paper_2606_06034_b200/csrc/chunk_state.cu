@@ -10,7 +10,9 @@
 //
 // Everything is evaluated with the value dimension on the 128 TMEM lanes ("transposed"): one CTA per (batch, head)
 // keeps the state S [d_v x d_k] as an fp32 accumulator in TMEM for the whole sequence, lane t = value feature t.
-//     D1  = S0 W^T - U^T      A = bf16(S0) in TMEM, B = W tile; the transpose of U comes from the tensor core as
+//     D1  = S0 W^T - U^T      A = S0 as hi + lo bf16 halves in TMEM (the state is O(1) while U_new can be small:
+//                             a single bf16 copy costs 1e-2 on strongly correlated keys), B = W tile; the
+//                             transpose of U comes from the tensor core as
 //                             (-I) U^T with a constant A operand, so no thread ever transposes anything
 //     PT  = K Q^T             lanes 0..63 = token j, columns = token i
 //     O1  = S0 Q^T
@@ -39,17 +41,17 @@ constexpr uint32_t kSD = 0;    // 128: state S, fp32 accumulator
 constexpr uint32_t kSA = 128;  // 64: bf16(S0) as A operand (K = d_k)
 constexpr uint32_t kIA = 192;  // 64: -I as A operand (K = d_v), constant
 constexpr uint32_t kD1 = 256;  // 64: S0 W^T - U^T, then the two bf16 forms of U_new^T as A operands
-constexpr uint32_t kPT = 320;  // 64: K Q^T (lanes 0..63)
+constexpr uint32_t kPT = 320;  // 64: K Q^T (lanes 0..63); once read, the lo bf16 halves of the two forms of U_new^T
 constexpr uint32_t kO1 = 384;  // 64: S0 Q^T
-constexpr uint32_t kO2 = 448;  // 64: U_new^T P^T
+constexpr uint32_t kO2 = 448;  // 64: U_new^T P^T; between chunks it holds the lo bf16 half of S0 (A operand)
 constexpr uint32_t kTmemCols = 512;
 
 // shared memory map (bytes; 1 KB aligned). A [64 x 128] bf16 tile is two [64 x 64] sub-tiles of 8 KB (128B swizzle).
 constexpr int kTileBytes = 16384;
 constexpr int kStageBytes = 4 * kTileBytes;  // Q, K, W, U
 constexpr int kOffQ = 0, kOffK = kTileBytes, kOffW = 2 * kTileBytes, kOffU = 3 * kTileBytes;
-constexpr int kOffP = 2 * kStageBytes;       // 8 KB: P as B operand [64 x 64] (MN-major, no swizzle)
-constexpr int kOffO = kOffP + 8192;          // 16 KB: O tile staged for the bulk store (128B swizzle)
+constexpr int kOffP = 2 * kStageBytes;       // 2 x 8 KB: P as B operand [64 x 64] (MN-major, no swizzle), hi and lo halves
+constexpr int kOffO = kOffP + 16384;          // 16 KB: O tile staged for the bulk store (128B swizzle)
 constexpr int kOffG = kOffO + kTileBytes;    // 3 x 64 floats: exp(g_i), exp(g_C - g_j), g
 constexpr int kSmemTotal = kOffG + 3 * 64 * 4;
 
@@ -89,7 +91,7 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     float* sf = se + 64;                                  // exp(g_C - g_j)
     float* sg = sf + 64;                                  // g_i
 
-    __shared__ uint64_t bar_full[2], bar_mma;
+    __shared__ uint64_t bar_full[2], bar_mma, bar_d1;
     __shared__ uint32_t tmem_base_s;
     __shared__ int s_fail;
 
@@ -104,6 +106,7 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         mbar_init(&bar_full[0], 1);
         mbar_init(&bar_full[1], 1);
         mbar_init(&bar_mma, 1);
+        mbar_init(&bar_d1, 1);
         s_fail = 0;
         mbar_fence_init();
         tma_prefetch_desc(&tmQ);
@@ -139,6 +142,13 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         if (warp == 0 && !wait_bar(&bar_mma, par_mma)) *reinterpret_cast<volatile int*>(&s_fail) = 1;
         asm volatile("bar.sync 2, 256;" ::: "memory");
         par_mma ^= 1;
+        return *reinterpret_cast<volatile int*>(&s_fail) == 0;
+    };
+    uint32_t par_d1 = 0;
+    auto wait_d1 = [&]() -> bool {
+        if (warp == 0 && !wait_bar(&bar_d1, par_d1)) *reinterpret_cast<volatile int*>(&s_fail) = 1;
+        asm volatile("bar.sync 3, 256;" ::: "memory");
+        par_d1 ^= 1;
         return *reinterpret_cast<volatile int*>(&s_fail) == 0;
     };
     auto load_stage = [&](int c) {  // one elected thread: the four tiles of chunk c into stage c & 1
@@ -184,6 +194,10 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 #pragma unroll
             for (int i = 0; i < 8; ++i) pk[i] = pack_bf16x2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
             tmem_st8(lane_base + kSA + h * 32 + part * 8, pk);
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                pk[i] = pack_bf16x2(__uint_as_float(v[2 * i]) - bf16_lo(pk[i]), __uint_as_float(v[2 * i + 1]) - bf16_hi(pk[i]));
+            tmem_st8(lane_base + kO2 + h * 32 + part * 8, pk);
         }
         tmem_wait_st();
     }
@@ -216,17 +230,22 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             if (!wait_bar(&bar_full[c & 1], (c >> 1) & 1)) *reinterpret_cast<volatile int*>(&s_fail) = 1;
             tc_fence_after_sync();
             if (*reinterpret_cast<volatile int*>(&s_fail) == 0 && elect_one()) {
-                // D1 = (-I) U^T + S0 W^T
+                // D1 = (-I) U^T + (S0_hi + S0_lo) W^T, with its own completion barrier: the threads start on it while
+                // the other products of the group still run
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
                     const uint64_t bd = smem_desc(st_a + kOffU + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024, SWZ_128B);
                     mma_f16_ts(tmem + kD1, tmem + kIA + ks * 8, bd, idesc_kk64, ks > 0);
                 }
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const uint64_t bd = smem_desc(st_a + kOffW + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024, SWZ_128B);
-                    mma_f16_ts(tmem + kD1, tmem + kSA + ks * 8, bd, idesc_kk64, true);
+                for (int part = 0; part < 2; ++part) {
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const uint64_t bd = smem_desc(st_a + kOffW + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024, SWZ_128B);
+                        mma_f16_ts(tmem + kD1, tmem + (part == 0 ? kSA : kO2) + ks * 8, bd, idesc_kk64, true);
+                    }
                 }
+                mma_commit(&bar_d1);
                 // PT = K Q^T (rows 64..127 of the A operand read past the 64-row tile: unused lanes)
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
@@ -234,11 +253,14 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                     const uint64_t bd = smem_desc(st_a + kOffQ + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024, SWZ_128B);
                     mma_f16_ss(tmem + kPT, ad, bd, idesc_kk64, ks > 0);
                 }
-                // O1 = S0 Q^T
+                // O1 = (S0_hi + S0_lo) Q^T
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const uint64_t bd = smem_desc(st_a + kOffQ + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024, SWZ_128B);
-                    mma_f16_ts(tmem + kO1, tmem + kSA + ks * 8, bd, idesc_kk64, ks > 0);
+                for (int part = 0; part < 2; ++part) {
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const uint64_t bd = smem_desc(st_a + kOffQ + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024, SWZ_128B);
+                        mma_f16_ts(tmem + kO1, tmem + (part == 0 ? kSA : kO2) + ks * 8, bd, idesc_kk64, part > 0 || ks > 0);
+                    }
                 }
                 mma_commit(&bar_mma);
             }
@@ -263,11 +285,14 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             }
             tmem_wait_st();
         }
-        if (!wait_mma()) { ok = false; break; }
+        if (!wait_d1()) { ok = false; break; }
         tc_fence_after_sync();
 
-        // ---- U_new^T = -D1: plain and gate-scaled bf16 copies, written over this thread's own D1 columns
-        // (h = 0: plain -> columns 0..15, scaled -> 16..31; h = 1: 32..47 and 48..63)
+        // ---- U_new^T = -D1 as bf16 hi + lo, plain and gate-scaled (the sums over the tokens of a chunk telescope
+        // on correlated keys, so single bf16 copies cost 1e-2 there). The hi halves are written over this thread's own
+        // D1 columns (h = 0: plain -> columns 0..15, scaled -> 16..31; h = 1: 32..47 and 48..63), the lo halves at
+        // the same offsets of the PT region once PT has been read.
+        uint32_t lp[16], ls[16];
         {
             uint32_t d[32];
             tmem_ld32(lane_base + kD1 + h * 32, d);
@@ -277,13 +302,18 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             for (int i = 0; i < 16; ++i) {
                 const float u0 = -__uint_as_float(d[2 * i]), u1 = -__uint_as_float(d[2 * i + 1]);
                 const float2 f = *reinterpret_cast<const float2*>(sf + h * 32 + 2 * i);
+                const float s0 = u0 * f.x, s1 = u1 * f.y;
                 pp[i] = pack_bf16x2(u0, u1);
-                ps[i] = pack_bf16x2(u0 * f.x, u1 * f.y);
+                ps[i] = pack_bf16x2(s0, s1);
+                lp[i] = pack_bf16x2(u0 - bf16_lo(pp[i]), u1 - bf16_hi(pp[i]));
+                ls[i] = pack_bf16x2(s0 - bf16_lo(ps[i]), s1 - bf16_hi(ps[i]));
             }
             tmem_st16(lane_base + kD1 + h * 32, pp);
             tmem_st16(lane_base + kD1 + h * 32 + 16, ps);
         }
-        // ---- P_ij = exp(g_i - g_j) PT_ji for j <= i: token j = lane (rows 0..63 only), this thread's 32 columns i
+        if (!wait_mma()) { ok = false; break; }
+        tc_fence_after_sync();
+        // ---- P_ij = exp(g_i - g_j) PT_ji for j <= i (hi + lo): token j = lane (rows 0..63 only), this thread's 32 columns i
         if (wq < 2) {
             uint32_t d[32];
             tmem_ld32(lane_base + kPT + h * 32, d);
@@ -291,7 +321,7 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             const float gj = sg[t] * kLog2e;
 #pragma unroll
             for (int c4 = 0; c4 < 4; ++c4) {
-                uint32_t w[4];
+                uint32_t w[4], wl[4];
 #pragma unroll
                 for (int i2 = 0; i2 < 4; ++i2) {
                     float v[2];
@@ -302,11 +332,15 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                         v[q] = (t <= i) ? x : 0.f;
                     }
                     w[i2] = pack_bf16x2(v[0], v[1]);
+                    wl[i2] = pack_bf16x2(v[0] - bf16_lo(w[i2]), v[1] - bf16_hi(w[i2]));
                 }
                 // B operand [K-dim = j][N = i], MN-major, no swizzle: the 16-byte piece of row j for column group n8
                 *reinterpret_cast<uint4*>(smem + kOffP + (h * 4 + c4) * 1024 + t * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+                *reinterpret_cast<uint4*>(smem + kOffP + 8192 + (h * 4 + c4) * 1024 + t * 16) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
             }
         }
+        tmem_st16(lane_base + kPT + h * 32, lp);
+        tmem_st16(lane_base + kPT + h * 32 + 16, ls);
         fence_proxy_async_smem();
         tmem_wait_st();
         tc_fence_before_sync();
@@ -315,17 +349,26 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         if (warp == 0) {
             tc_fence_after_sync();
             if (elect_one()) {
-                // O2 = U_new^T P^T (K-dim = 64 tokens; the plain copy sits at columns 0..15 and 32..47)
+                // O2 = U_new^T P^T = Uh Ph + Ul Ph + Uh Pl (K-dim = 64 tokens; the plain copies sit at columns 0..15 and
+                // 32..47 of their regions)
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks) {
-                    const uint64_t bd = smem_desc(smem_a + kOffP + ks * 256, 128, 1024, SWZ_NONE);
-                    mma_f16_ts(tmem + kO2, tmem + kD1 + (ks < 2 ? ks * 8 : 32 + (ks - 2) * 8), bd, idesc_mn64, ks > 0);
+                for (int part = 0; part < 3; ++part) {
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) {
+                        const uint64_t bd = smem_desc(smem_a + kOffP + (part == 2 ? 8192 : 0) + ks * 256, 128, 1024, SWZ_NONE);
+                        mma_f16_ts(tmem + kO2, tmem + (part == 1 ? kPT : kD1) + (ks < 2 ? ks * 8 : 32 + (ks - 2) * 8), bd,
+                                   idesc_mn64, part > 0 || ks > 0);
+                    }
                 }
-                // S += (U_new^T exp(g_C - g_j)) K (the K tile as MN-major operand, N = 128)
+                // S += (U_new^T exp(g_C - g_j)) K, hi + lo (the K tile as MN-major operand, N = 128)
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks) {
-                    const uint64_t bd = smem_desc(st_a + kOffK + ks * 2048, 8192, 1024, SWZ_128B);
-                    mma_f16_ts(tmem + kSD, tmem + kD1 + 16 + (ks < 2 ? ks * 8 : 32 + (ks - 2) * 8), bd, idesc_mn128, true);
+                for (int part = 0; part < 2; ++part) {
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) {
+                        const uint64_t bd = smem_desc(st_a + kOffK + ks * 2048, 8192, 1024, SWZ_128B);
+                        mma_f16_ts(tmem + kSD, tmem + (part == 0 ? kD1 : kPT) + 16 + (ks < 2 ? ks * 8 : 32 + (ks - 2) * 8), bd,
+                                   idesc_mn128, true);
+                    }
                 }
                 mma_commit(&bar_mma);
             }
@@ -358,7 +401,7 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 *reinterpret_cast<__nv_bfloat16*>(sub + tok * 128 + ((cch ^ (tok & 7)) << 4) + (t & 7) * 2) = v;
             }
         }
-        // ---- bf16 copy of the new state for the next chunk's products
+        // ---- bf16 copies (hi, lo) of the new state for the next chunk's products
         {
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
@@ -368,6 +411,11 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 #pragma unroll
                 for (int i = 0; i < 16; ++i) pk[i] = pack_bf16x2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
                 tmem_st16(lane_base + kSA + h * 32 + part * 16, pk);
+                // the lo half goes where O2 was (this thread has read its O2 columns above)
+#pragma unroll
+                for (int i = 0; i < 16; ++i)
+                    pk[i] = pack_bf16x2(__uint_as_float(v[2 * i]) - bf16_lo(pk[i]), __uint_as_float(v[2 * i + 1]) - bf16_hi(pk[i]));
+                tmem_st16(lane_base + kO2 + h * 32 + part * 16, pk);
             }
             tmem_wait_st();
         }

@@ -13,10 +13,11 @@ from paper_2606_06034_b200 import inputs as gen
 
 pytestmark = pytest.mark.gpu
 
-# relative Frobenius error per chunk of O and of the final state: bf16 operands (state, U_new, P) with fp32
-# accumulation and a bf16 output
-TOL_O = 4e-3
-TOL_S = 2e-3
+# Relative Frobenius error per chunk of O and of the final state. Every operand that can cancel (state, U_new, P) goes
+# through the tensor cores as hi + lo bf16 halves with fp32 accumulation, so what remains is the bf16 rounding of the
+# output itself (1.7e-3, the same floor as W and U of the chunk-prepare path) and ~1e-6 on the fp32 state.
+TOL_O = 2.2e-3
+TOL_S = 1e-4
 
 
 def _queries(inp, seed):
@@ -88,3 +89,33 @@ def test_state_output_argument_errors():
     assert gdn.gdn_chunk_state_output(K, K, K, K, g, 1, 1, 1, 100, 64, 128, 128, 1.0, None, O, None, **args) == gdn.GDN_ERR_INVALID_ARG
     assert gdn.gdn_chunk_state_output(None, K, K, K, g, 1, 1, 1, 128, 64, 128, 128, 1.0, None, O, None, **args) == gdn.GDN_ERR_NULL
     assert gdn.gdn_device_status() == gdn.GDN_OK
+
+
+@pytest.mark.parametrize("name", ["sweep_c64", "prefill_gqa", "stress"])
+def test_state_output_at_full_size(name):
+    """The benchmark workloads in one launch each (chunk-prepare with the gated W, then state passing + output):
+    sampled heads are compared with the oracle over their whole sequence (the chain of up to 1024 chunks is where
+    an error in the carried state would accumulate), every output must be finite, and a second launch must agree
+    bit for bit."""
+    inp = gen.make_workload(name, device="cuda")
+    C, T = inp.C, inp.T
+    Q = torch.randn(inp.B, inp.H_k, T, inp.d_k, device="cuda", generator=torch.Generator(device="cuda").manual_seed(430))
+    Q = (Q / Q.norm(dim=-1, keepdim=True)).to(torch.bfloat16)
+    scale = 128 ** -0.5
+    W, U, _ = gdn.chunk_prepare(inp.K, inp.V, inp.beta, inp.g, C, flags=gdn.GDN_FLAG_W_GATED)
+    O, S = gdn.chunk_state_output(Q, inp.K, W, U, inp.g, C, scale)
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+    assert bool(torch.isfinite(O).all()) and bool(torch.isfinite(S).all())
+    O2, S2 = gdn.chunk_state_output(Q, inp.K, W, U, inp.g, C, scale)
+    assert torch.equal(O, O2) and torch.equal(S, S2)
+    group = inp.H_v // inp.H_k
+    heads = [(0, 0), (inp.B - 1, inp.H_v - 1), (0, 1 % inp.H_v)]  # head 1 is adversarial in the stress workload
+    for b, hv in dict.fromkeys(heads):
+        hk = hv // group
+        Oo, So = orc.chunk_state_output(Q[b, hk].double().cpu().numpy(), inp.K[b, hk].double().cpu().numpy(),
+                                        W[b, hv].double().cpu().numpy(), U[b, hv].double().cpu().numpy(),
+                                        inp.g[b, hv].double().cpu().numpy(), C, scale)
+        eO = orc.rel_frobenius(O[b, hv].double().cpu().numpy().reshape(T // C, C, 128), Oo.reshape(T // C, C, 128))
+        assert eO.max() <= TOL_O, f"{name}: O rel-F {eO.max():.3e} at chunk {eO.argmax()} of head ({b},{hv})"
+        eS = orc.rel_frobenius(S[b, hv].double().cpu().numpy()[None], So[None])
+        assert eS.max() <= TOL_S, f"{name}: S rel-F {eS.max():.3e} of head ({b},{hv})"
