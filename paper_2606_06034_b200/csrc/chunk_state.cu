@@ -33,7 +33,7 @@ using namespace sm100;
 
 constexpr int kC = 64;         // chunk size
 constexpr int kD = 128;        // d_k = d_v
-constexpr int kThreads = 256;  // two threads per TMEM lane
+constexpr int kThreads = 256;  // compute threads, two per TMEM lane; one more warp issues the TMA loads and the MMAs
 constexpr float kLog2e = 1.4426950408889634f;
 
 // TMEM column map (512 columns: one CTA per SM)
@@ -81,7 +81,7 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity) {
     return true;
 }
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads + 32, 1)
 chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                    const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmU,
                    const __grid_constant__ CUtensorMap tmO, const ParamsS p) {
@@ -91,22 +91,28 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     float* sf = se + 64;                                  // exp(g_C - g_j)
     float* sg = sf + 64;                                  // g_i
 
-    __shared__ uint64_t bar_full[2], bar_mma, bar_d1;
+    // One mbarrier per MMA group (never two pending phases on one barrier), two per-stage TMA barriers, and two
+    // barriers on which the 256 compute threads tell the issuing warp that operands are in place.
+    __shared__ uint64_t bar_full[2], bar_pre, bar_d1, bar_o1, bar_g2, bar_rdy_a, bar_rdy_2;
     __shared__ uint32_t tmem_base_s;
     __shared__ int s_fail;
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
-    const int lane = tid & 31;
     const int t = tid & 127;  // TMEM lane: value feature (state rows, output columns); token j for PT
-    const int h = tid >> 7;   // column half
+    const int h = (tid >> 7) & 1;  // column half
     const int wq = warp & 3;
+    const bool issuer = warp == kThreads / 32;  // warp 8: every TMA load and every tcgen05.mma
 
     if (tid == 0) {
         mbar_init(&bar_full[0], 1);
         mbar_init(&bar_full[1], 1);
-        mbar_init(&bar_mma, 1);
+        mbar_init(&bar_pre, 1);
         mbar_init(&bar_d1, 1);
+        mbar_init(&bar_o1, 1);
+        mbar_init(&bar_g2, 1);
+        mbar_init(&bar_rdy_a, kThreads);
+        mbar_init(&bar_rdy_2, kThreads);
         s_fail = 0;
         mbar_fence_init();
         tma_prefetch_desc(&tmQ);
@@ -131,112 +137,66 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     const int n_c = p.T / kC;
     const float* gseq = p.g + (long long)bhv * p.T;
     const uint32_t smem_a = smem_u32(smem);
-    // M = 128, N = 64 / 128; A from TMEM (or K-major shared memory), B K-major or MN-major
-    const uint32_t idesc_kk64 = instr_desc(128, 64, 1, 1, 0, 0, 1);
-    const uint32_t idesc_mn64 = instr_desc(128, 64, 1, 1, 0, 1, 1);
-    const uint32_t idesc_mn128 = instr_desc(128, 128, 1, 1, 0, 1, 1);
+    volatile int* fail = reinterpret_cast<volatile int*>(&s_fail);
 
-    uint32_t par_mma = 0;
-    bool ok = true;
-    auto wait_mma = [&]() -> bool {
-        if (warp == 0 && !wait_bar(&bar_mma, par_mma)) *reinterpret_cast<volatile int*>(&s_fail) = 1;
-        asm volatile("bar.sync 2, 256;" ::: "memory");
-        par_mma ^= 1;
-        return *reinterpret_cast<volatile int*>(&s_fail) == 0;
-    };
-    uint32_t par_d1 = 0;
-    auto wait_d1 = [&]() -> bool {
-        if (warp == 0 && !wait_bar(&bar_d1, par_d1)) *reinterpret_cast<volatile int*>(&s_fail) = 1;
-        asm volatile("bar.sync 3, 256;" ::: "memory");
-        par_d1 ^= 1;
-        return *reinterpret_cast<volatile int*>(&s_fail) == 0;
-    };
-    auto load_stage = [&](int c) {  // one elected thread: the four tiles of chunk c into stage c & 1
-        uint8_t* st = smem + (c & 1) * kStageBytes;
-        uint64_t* bar = &bar_full[c & 1];
-        mbar_arrive_expect_tx(bar, kStageBytes);
-        const int t0 = c * kC;
-        tma_load_3d(st + kOffQ, &tmQ, bar, 0, t0, bhk);
-        tma_load_3d(st + kOffQ + 8192, &tmQ, bar, 64, t0, bhk);
-        tma_load_3d(st + kOffK, &tmK, bar, 0, t0, bhk);
-        tma_load_3d(st + kOffK + 8192, &tmK, bar, 64, t0, bhk);
-        tma_load_3d(st + kOffW, &tmW, bar, 0, t0, bhv);
-        tma_load_3d(st + kOffW + 8192, &tmW, bar, 64, t0, bhv);
-        tma_load_3d(st + kOffU, &tmU, bar, 0, t0, bhv);
-        tma_load_3d(st + kOffU + 8192, &tmU, bar, 64, t0, bhv);
-    };
-
-    if (warp == 0 && n_c > 0 && elect_one()) {
-        load_stage(0);
-        if (n_c > 1) load_stage(1);
-    }
-
-    // ---- constant A operand -I, initial state, and its bf16 copy
-    {
-        uint32_t r[16];
-#pragma unroll
-        for (int part = 0; part < 2; ++part) {
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const int col = h * 32 + part * 16 + i;  // packed column: features 2 col, 2 col + 1
-                r[i] = (col == (t >> 1)) ? ((t & 1) ? 0xBF800000u : 0x0000BF80u) : 0u;
-            }
-            tmem_st16(lane_base + kIA + h * 32 + part * 16, r);
-        }
-        // this thread's half of state row t: columns [64 h, 64 h + 64)
-        const float* s0 = (p.S_in != nullptr) ? p.S_in + ((long long)bhv * kD + t) * kD + h * 64 : nullptr;
-#pragma unroll
-        for (int part = 0; part < 4; ++part) {
-            uint32_t v[16], pk[8];
-#pragma unroll
-            for (int i = 0; i < 16; ++i) v[i] = (s0 != nullptr) ? __float_as_uint(__ldg(s0 + part * 16 + i)) : 0u;
-            tmem_st16(lane_base + kSD + h * 64 + part * 16, v);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) pk[i] = pack_bf16x2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
-            tmem_st8(lane_base + kSA + h * 32 + part * 8, pk);
-#pragma unroll
-            for (int i = 0; i < 8; ++i)
-                pk[i] = pack_bf16x2(__uint_as_float(v[2 * i]) - bf16_lo(pk[i]), __uint_as_float(v[2 * i + 1]) - bf16_hi(pk[i]));
-            tmem_st8(lane_base + kO2 + h * 32 + part * 8, pk);
-        }
-        tmem_wait_st();
-    }
-    // gates of the first chunk
-    float g_reg = 0.f, gC_reg = 0.f;
-    if (n_c > 0) {
-        if (tid < 64) g_reg = __ldg(gseq + tid);
-        gC_reg = __ldg(gseq + kC - 1);
-    }
-
-    for (int c = 0; c < n_c; ++c) {
-        uint8_t* st = smem + (c & 1) * kStageBytes;
-        const uint32_t st_a = smem_a + (c & 1) * kStageBytes;
-        const float gC = gC_reg;
-        if (tid < 64) {
-            sg[tid] = g_reg;
-            se[tid] = fast_exp2(g_reg * kLog2e);
-            sf[tid] = fast_exp2((gC - g_reg) * kLog2e);
-        }
-        if (c + 1 < n_c) {
-            if (tid < 64) g_reg = __ldg(gseq + (c + 1) * kC + tid);
-            gC_reg = __ldg(gseq + (c + 2) * kC - 1);
-        }
-        // the previous chunk's output store has finished reading the staging tile
-        if (tid == 0) tma_store_wait_read<0>();
-        tc_fence_before_sync();
-        __syncthreads();  // bf16(S0) and the gate tables are in place
-
-        if (warp == 0) {
-            if (!wait_bar(&bar_full[c & 1], (c >> 1) & 1)) *reinterpret_cast<volatile int*>(&s_fail) = 1;
+    if (issuer) {
+        // ================= issuing warp: TMA loads and every tcgen05.mma, in the order the tensor pipe runs them
+        const uint32_t idesc_kk64 = instr_desc(128, 64, 1, 1, 0, 0, 1);   // B K-major (a TMA tile as [N x K])
+        const uint32_t idesc_mn64 = instr_desc(128, 64, 1, 1, 0, 1, 1);   // B MN-major
+        const uint32_t idesc_mn128 = instr_desc(128, 128, 1, 1, 0, 1, 1);
+        auto load_stage = [&](int c) {  // the four tiles of chunk c into stage c & 1
+            uint8_t* st = smem + (c & 1) * kStageBytes;
+            uint64_t* bar = &bar_full[c & 1];
+            mbar_arrive_expect_tx(bar, kStageBytes);
+            const int t0 = c * kC;
+            tma_load_3d(st + kOffQ, &tmQ, bar, 0, t0, bhk);
+            tma_load_3d(st + kOffQ + 8192, &tmQ, bar, 64, t0, bhk);
+            tma_load_3d(st + kOffK, &tmK, bar, 0, t0, bhk);
+            tma_load_3d(st + kOffK + 8192, &tmK, bar, 64, t0, bhk);
+            tma_load_3d(st + kOffW, &tmW, bar, 0, t0, bhv);
+            tma_load_3d(st + kOffW + 8192, &tmW, bar, 64, t0, bhv);
+            tma_load_3d(st + kOffU, &tmU, bar, 0, t0, bhv);
+            tma_load_3d(st + kOffU + 8192, &tmU, bar, 64, t0, bhv);
+        };
+        // the products of chunk c that do not depend on the state: D1 <- (-I) U^T and PT = K Q^T
+        auto issue_pre = [&](int c) {
+            const uint32_t sa = smem_a + (c & 1) * kStageBytes;
+            if (!wait_bar(&bar_full[c & 1], (c >> 1) & 1)) *fail = 1;
             tc_fence_after_sync();
-            if (*reinterpret_cast<volatile int*>(&s_fail) == 0 && elect_one()) {
-                // D1 = (-I) U^T + (S0_hi + S0_lo) W^T, with its own completion barrier: the threads start on it while
-                // the other products of the group still run
+            if (*fail == 0 && elect_one()) {
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
-                    const uint64_t bd = smem_desc(st_a + kOffU + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024, SWZ_128B);
+                    const uint64_t bd = smem_desc(sa + kOffU + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024, SWZ_128B);
                     mma_f16_ts(tmem + kD1, tmem + kIA + ks * 8, bd, idesc_kk64, ks > 0);
                 }
+                // rows 64..127 of the A operand read past the 64-row K tile: unused lanes
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint64_t ad = smem_desc(sa + kOffK + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024, SWZ_128B);
+                    const uint64_t bd = smem_desc(sa + kOffQ + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024, SWZ_128B);
+                    mma_f16_ss(tmem + kPT, ad, bd, idesc_kk64, ks > 0);
+                }
+                mma_commit(&bar_pre);
+            }
+            __syncwarp();
+        };
+        if (n_c > 0) {
+            if (elect_one()) {
+                load_stage(0);
+                if (n_c > 1) load_stage(1);
+            }
+            __syncwarp();
+        }
+        uint32_t par_a = 0, par_2 = 0, par_g2 = 0;
+        for (int c = 0; c < n_c && *fail == 0; ++c) {
+            const uint32_t st_a = smem_a + (c & 1) * kStageBytes;
+            // the state copies (and, for the first chunk, the constant operand) are in place
+            if (!wait_bar(&bar_rdy_a, par_a)) *fail = 1;
+            par_a ^= 1;
+            tc_fence_after_sync();
+            if (c == 0) issue_pre(0);
+            if (*fail == 0 && elect_one()) {
+                // D1 += (S0_hi + S0_lo) W^T onto -U^T, with its own completion barrier
 #pragma unroll
                 for (int part = 0; part < 2; ++part) {
 #pragma unroll
@@ -246,13 +206,6 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                     }
                 }
                 mma_commit(&bar_d1);
-                // PT = K Q^T (rows 64..127 of the A operand read past the 64-row tile: unused lanes)
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const uint64_t ad = smem_desc(st_a + kOffK + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024, SWZ_128B);
-                    const uint64_t bd = smem_desc(st_a + kOffQ + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024, SWZ_128B);
-                    mma_f16_ss(tmem + kPT, ad, bd, idesc_kk64, ks > 0);
-                }
                 // O1 = (S0_hi + S0_lo) Q^T
 #pragma unroll
                 for (int part = 0; part < 2; ++part) {
@@ -262,93 +215,14 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                         mma_f16_ts(tmem + kO1, tmem + (part == 0 ? kSA : kO2) + ks * 8, bd, idesc_kk64, part > 0 || ks > 0);
                     }
                 }
-                mma_commit(&bar_mma);
+                mma_commit(&bar_o1);
             }
-        }
-        // ---- while those run: decay of the accumulator, S <- exp(g_C) S0 (the products above read the bf16 copy)
-        {
-            const float dec = fast_exp2(gC * kLog2e);
-#pragma unroll
-            for (int part = 0; part < 2; ++part) {
-                uint32_t v[32];
-                tmem_ld32(lane_base + kSD + h * 64 + part * 32, v);
-                tmem_wait_ld();
-#pragma unroll
-                for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * dec);
-                uint32_t w16[16];
-#pragma unroll
-                for (int i = 0; i < 16; ++i) w16[i] = v[i];
-                tmem_st16(lane_base + kSD + h * 64 + part * 32, w16);
-#pragma unroll
-                for (int i = 0; i < 16; ++i) w16[i] = v[16 + i];
-                tmem_st16(lane_base + kSD + h * 64 + part * 32 + 16, w16);
-            }
-            tmem_wait_st();
-        }
-        if (!wait_d1()) { ok = false; break; }
-        tc_fence_after_sync();
-
-        // ---- U_new^T = -D1 as bf16 hi + lo, plain and gate-scaled (the sums over the tokens of a chunk telescope
-        // on correlated keys, so single bf16 copies cost 1e-2 there). The hi halves are written over this thread's own
-        // D1 columns (h = 0: plain -> columns 0..15, scaled -> 16..31; h = 1: 32..47 and 48..63), the lo halves at
-        // the same offsets of the PT region once PT has been read.
-        uint32_t lp[16], ls[16];
-        {
-            uint32_t d[32];
-            tmem_ld32(lane_base + kD1 + h * 32, d);
-            tmem_wait_ld();
-            uint32_t pp[16], ps[16];
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const float u0 = -__uint_as_float(d[2 * i]), u1 = -__uint_as_float(d[2 * i + 1]);
-                const float2 f = *reinterpret_cast<const float2*>(sf + h * 32 + 2 * i);
-                const float s0 = u0 * f.x, s1 = u1 * f.y;
-                pp[i] = pack_bf16x2(u0, u1);
-                ps[i] = pack_bf16x2(s0, s1);
-                lp[i] = pack_bf16x2(u0 - bf16_lo(pp[i]), u1 - bf16_hi(pp[i]));
-                ls[i] = pack_bf16x2(s0 - bf16_lo(ps[i]), s1 - bf16_hi(ps[i]));
-            }
-            tmem_st16(lane_base + kD1 + h * 32, pp);
-            tmem_st16(lane_base + kD1 + h * 32 + 16, ps);
-        }
-        if (!wait_mma()) { ok = false; break; }
-        tc_fence_after_sync();
-        // ---- P_ij = exp(g_i - g_j) PT_ji for j <= i (hi + lo): token j = lane (rows 0..63 only), this thread's 32 columns i
-        if (wq < 2) {
-            uint32_t d[32];
-            tmem_ld32(lane_base + kPT + h * 32, d);
-            tmem_wait_ld();
-            const float gj = sg[t] * kLog2e;
-#pragma unroll
-            for (int c4 = 0; c4 < 4; ++c4) {
-                uint32_t w[4], wl[4];
-#pragma unroll
-                for (int i2 = 0; i2 < 4; ++i2) {
-                    float v[2];
-#pragma unroll
-                    for (int q = 0; q < 2; ++q) {
-                        const int i = h * 32 + c4 * 8 + i2 * 2 + q;
-                        const float x = __uint_as_float(d[c4 * 8 + i2 * 2 + q]) * fast_exp2(fminf(fmaf(sg[i], kLog2e, -gj), 0.f));
-                        v[q] = (t <= i) ? x : 0.f;
-                    }
-                    w[i2] = pack_bf16x2(v[0], v[1]);
-                    wl[i2] = pack_bf16x2(v[0] - bf16_lo(w[i2]), v[1] - bf16_hi(w[i2]));
-                }
-                // B operand [K-dim = j][N = i], MN-major, no swizzle: the 16-byte piece of row j for column group n8
-                *reinterpret_cast<uint4*>(smem + kOffP + (h * 4 + c4) * 1024 + t * 16) = make_uint4(w[0], w[1], w[2], w[3]);
-                *reinterpret_cast<uint4*>(smem + kOffP + 8192 + (h * 4 + c4) * 1024 + t * 16) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
-            }
-        }
-        tmem_st16(lane_base + kPT + h * 32, lp);
-        tmem_st16(lane_base + kPT + h * 32 + 16, ls);
-        fence_proxy_async_smem();
-        tmem_wait_st();
-        tc_fence_before_sync();
-        __syncthreads();
-
-        if (warp == 0) {
+            __syncwarp();
+            // U_new^T (hi, lo; plain, scaled), P (hi, lo) and the decayed accumulator are in place
+            if (!wait_bar(&bar_rdy_2, par_2)) *fail = 1;
+            par_2 ^= 1;
             tc_fence_after_sync();
-            if (elect_one()) {
+            if (*fail == 0 && elect_one()) {
                 // O2 = U_new^T P^T = Uh Ph + Ul Ph + Uh Pl (K-dim = 64 tokens; the plain copies sit at columns 0..15 and
                 // 32..47 of their regions)
 #pragma unroll
@@ -370,84 +244,232 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                                    idesc_mn128, true);
                     }
                 }
-                mma_commit(&bar_mma);
+                mma_commit(&bar_g2);
             }
+            __syncwarp();
+            // D1 and PT are only read by the products just issued, which the tensor pipe runs first: the
+            // state-independent products of the next chunk follow them directly
+            if (c + 1 < n_c) issue_pre(c + 1);
+            // once those products are complete the tiles of this stage are free for the chunk after the next one
+            if (!wait_bar(&bar_g2, par_g2)) *fail = 1;
+            par_g2 ^= 1;
+            if (*fail == 0 && c + 2 < n_c && elect_one()) load_stage(c + 2);
+            __syncwarp();
         }
-        // ---- meanwhile: exp(g_i) O1
-        float o[32];
+    } else {
+        // ================= compute threads (256): two per TMEM lane
+        uint32_t par_pre = 0, par_d1 = 0, par_o1 = 0, par_g2 = 0;
+        // completion of an MMA group: warp 0 polls the mbarrier, the other warps sleep on a hardware barrier
+        auto wait_group = [&](uint64_t* bar, uint32_t& par) -> bool {
+            if (warp == 0 && !wait_bar(bar, par)) *fail = 1;
+            asm volatile("bar.sync 2, 256;" ::: "memory");
+            par ^= 1;
+            tc_fence_after_sync();
+            return *fail == 0;
+        };
+        // ---- constant A operand -I, initial state, and its bf16 copies (hi in kSA, lo in kO2)
         {
-            uint32_t d[32];
-            tmem_ld32(lane_base + kO1 + h * 32, d);
-            tmem_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) o[i] = __uint_as_float(d[i]) * se[h * 32 + i];
-        }
-        if (!wait_mma()) { ok = false; break; }
-        tc_fence_after_sync();
-        // the tiles of this stage are free: the chunk after the next one may land there
-        if (warp == 0 && c + 2 < n_c && elect_one()) load_stage(c + 2);
-
-        // ---- O^T = scale (exp(g_i) O1 + O2): element (token i, feature t) of the staged tile
-        {
-            uint32_t d[32];
-            tmem_ld32(lane_base + kO2 + h * 32, d);
-            tmem_wait_ld();
-            uint8_t* sub = smem + kOffO + (t >> 6) * 8192;
-            const int cch = (t & 63) >> 3;
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                const int tok = h * 32 + i;
-                const __nv_bfloat16 v = __float2bfloat16_rn(p.scale * (o[i] + __uint_as_float(d[i])));
-                *reinterpret_cast<__nv_bfloat16*>(sub + tok * 128 + ((cch ^ (tok & 7)) << 4) + (t & 7) * 2) = v;
-            }
-        }
-        // ---- bf16 copies (hi, lo) of the new state for the next chunk's products
-        {
+            uint32_t r[16];
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
-                uint32_t v[32], pk[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const int col = h * 32 + part * 16 + i;  // packed column: features 2 col, 2 col + 1
+                    r[i] = (col == (t >> 1)) ? ((t & 1) ? 0xBF800000u : 0x0000BF80u) : 0u;
+                }
+                tmem_st16(lane_base + kIA + h * 32 + part * 16, r);
+            }
+            // this thread's half of state row t: columns [64 h, 64 h + 64)
+            const float* s0 = (p.S_in != nullptr) ? p.S_in + ((long long)bhv * kD + t) * kD + h * 64 : nullptr;
+#pragma unroll
+            for (int part = 0; part < 4; ++part) {
+                uint32_t v[16], pk[8];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) v[i] = (s0 != nullptr) ? __float_as_uint(__ldg(s0 + part * 16 + i)) : 0u;
+                tmem_st16(lane_base + kSD + h * 64 + part * 16, v);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) pk[i] = pack_bf16x2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
+                tmem_st8(lane_base + kSA + h * 32 + part * 8, pk);
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    pk[i] = pack_bf16x2(__uint_as_float(v[2 * i]) - bf16_lo(pk[i]), __uint_as_float(v[2 * i + 1]) - bf16_hi(pk[i]));
+                tmem_st8(lane_base + kO2 + h * 32 + part * 8, pk);
+            }
+            tmem_wait_st();
+            tc_fence_before_sync();
+            mbar_arrive(&bar_rdy_a);
+        }
+        // gates of the first chunk
+        float g_reg = 0.f, gC_reg = 0.f;
+        if (n_c > 0) {
+            if (tid < 64) g_reg = __ldg(gseq + tid);
+            gC_reg = __ldg(gseq + kC - 1);
+        }
+        bool ok = true;
+        for (int c = 0; c < n_c; ++c) {
+            const float gC = gC_reg;
+            if (tid < 64) {
+                sg[tid] = g_reg;
+                se[tid] = fast_exp2(g_reg * kLog2e);
+                sf[tid] = fast_exp2((gC - g_reg) * kLog2e);
+            }
+            if (c + 1 < n_c) {
+                if (tid < 64) g_reg = __ldg(gseq + (c + 1) * kC + tid);
+                gC_reg = __ldg(gseq + (c + 2) * kC - 1);
+            }
+            // the previous chunk's output store has finished reading the staging tile
+            if (tid == 0) tma_store_wait_read<0>();
+            asm volatile("bar.sync 1, 256;" ::: "memory");  // gate tables visible, staging tile free
+
+            // ---- decay of the accumulator, S <- exp(g_C) S0 (the products of this chunk read the bf16 copies)
+            {
+                const float dec = fast_exp2(gC * kLog2e);
+#pragma unroll
+                for (int part = 0; part < 2; ++part) {
+                    uint32_t v[32];
+                    tmem_ld32(lane_base + kSD + h * 64 + part * 32, v);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * dec);
+                    uint32_t w16[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) w16[i] = v[i];
+                    tmem_st16(lane_base + kSD + h * 64 + part * 32, w16);
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) w16[i] = v[16 + i];
+                    tmem_st16(lane_base + kSD + h * 64 + part * 32 + 16, w16);
+                }
+            }
+            // ---- P_ij = exp(g_i - g_j) PT_ji for j <= i (hi + lo): token j = lane (rows 0..63 only), this thread's 32 columns i
+            if (!wait_group(&bar_pre, par_pre)) { ok = false; break; }
+            if (wq < 2) {
+                uint32_t d[32];
+                tmem_ld32(lane_base + kPT + h * 32, d);
+                tmem_wait_ld();
+                const float gj = sg[t] * kLog2e;
+#pragma unroll
+                for (int c4 = 0; c4 < 4; ++c4) {
+                    uint32_t w[4], wl[4];
+#pragma unroll
+                    for (int i2 = 0; i2 < 4; ++i2) {
+                        float v[2];
+#pragma unroll
+                        for (int q = 0; q < 2; ++q) {
+                            const int i = h * 32 + c4 * 8 + i2 * 2 + q;
+                            const float x = __uint_as_float(d[c4 * 8 + i2 * 2 + q]) * fast_exp2(fminf(fmaf(sg[i], kLog2e, -gj), 0.f));
+                            v[q] = (t <= i) ? x : 0.f;
+                        }
+                        w[i2] = pack_bf16x2(v[0], v[1]);
+                        wl[i2] = pack_bf16x2(v[0] - bf16_lo(w[i2]), v[1] - bf16_hi(w[i2]));
+                    }
+                    // B operand [K-dim = j][N = i], MN-major, no swizzle: the 16-byte piece of row j for column group n8
+                    *reinterpret_cast<uint4*>(smem + kOffP + (h * 4 + c4) * 1024 + t * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+                    *reinterpret_cast<uint4*>(smem + kOffP + 8192 + (h * 4 + c4) * 1024 + t * 16) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
+                }
+            }
+            // ---- U_new^T = -D1 as bf16 hi + lo, plain and gate-scaled (the sums over the tokens of a chunk telescope
+            // on correlated keys, so single bf16 copies cost 1e-2 there). The hi halves are written over this thread's
+            // own D1 columns (h = 0: plain -> columns 0..15, scaled -> 16..31; h = 1: 32..47 and 48..63), the lo halves
+            // at the same offsets of the PT region (this thread's PT columns have been read above).
+            if (!wait_group(&bar_d1, par_d1)) { ok = false; break; }
+            {
+                uint32_t d[32];
+                tmem_ld32(lane_base + kD1 + h * 32, d);
+                tmem_wait_ld();
+                uint32_t pp[16], ps[16], lp[16], ls[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const float u0 = -__uint_as_float(d[2 * i]), u1 = -__uint_as_float(d[2 * i + 1]);
+                    const float2 f = *reinterpret_cast<const float2*>(sf + h * 32 + 2 * i);
+                    const float s0 = u0 * f.x, s1 = u1 * f.y;
+                    pp[i] = pack_bf16x2(u0, u1);
+                    ps[i] = pack_bf16x2(s0, s1);
+                    lp[i] = pack_bf16x2(u0 - bf16_lo(pp[i]), u1 - bf16_hi(pp[i]));
+                    ls[i] = pack_bf16x2(s0 - bf16_lo(ps[i]), s1 - bf16_hi(ps[i]));
+                }
+                tmem_st16(lane_base + kD1 + h * 32, pp);
+                tmem_st16(lane_base + kD1 + h * 32 + 16, ps);
+                tmem_st16(lane_base + kPT + h * 32, lp);
+                tmem_st16(lane_base + kPT + h * 32 + 16, ls);
+            }
+            fence_proxy_async_smem();
+            tmem_wait_st();
+            tc_fence_before_sync();
+            mbar_arrive(&bar_rdy_2);
+
+            // ---- exp(g_i) O1
+            if (!wait_group(&bar_o1, par_o1)) { ok = false; break; }
+            float o[32];
+            {
+                uint32_t d[32];
+                tmem_ld32(lane_base + kO1 + h * 32, d);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) o[i] = __uint_as_float(d[i]) * se[h * 32 + i];
+            }
+            if (!wait_group(&bar_g2, par_g2)) { ok = false; break; }
+            // ---- O^T = scale (exp(g_i) O1 + O2): element (token i, feature t) of the staged tile
+            {
+                uint32_t d[32];
+                tmem_ld32(lane_base + kO2 + h * 32, d);
+                tmem_wait_ld();
+                uint8_t* sub = smem + kOffO + (t >> 6) * 8192;
+                const int cch = (t & 63) >> 3;
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const int tok = h * 32 + i;
+                    const __nv_bfloat16 v = __float2bfloat16_rn(p.scale * (o[i] + __uint_as_float(d[i])));
+                    *reinterpret_cast<__nv_bfloat16*>(sub + tok * 128 + ((cch ^ (tok & 7)) << 4) + (t & 7) * 2) = v;
+                }
+            }
+            // ---- bf16 copies (hi, lo) of the new state for the next chunk's products; the lo half goes where O2 was
+            // (this thread has read its O2 columns above)
+            {
+#pragma unroll
+                for (int part = 0; part < 2; ++part) {
+                    uint32_t v[32], pk[16];
+                    tmem_ld32(lane_base + kSD + h * 64 + part * 32, v);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) pk[i] = pack_bf16x2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
+                    tmem_st16(lane_base + kSA + h * 32 + part * 16, pk);
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        pk[i] = pack_bf16x2(__uint_as_float(v[2 * i]) - bf16_lo(pk[i]), __uint_as_float(v[2 * i + 1]) - bf16_hi(pk[i]));
+                    tmem_st16(lane_base + kO2 + h * 32 + part * 16, pk);
+                }
+                tmem_wait_st();
+                tc_fence_before_sync();
+                mbar_arrive(&bar_rdy_a);
+            }
+            fence_proxy_async_smem();
+            asm volatile("bar.sync 1, 256;" ::: "memory");  // the staged output tile is complete
+            if (tid == 0) {  // the same thread waits for these stores (bulk groups are per thread)
+                tma_store_3d(&tmO, smem + kOffO, 0, c * kC, bhv);
+                tma_store_3d(&tmO, smem + kOffO + 8192, 64, c * kC, bhv);
+                tma_store_commit();
+            }
+        }
+        // ---- final state
+        if (ok && p.S_out != nullptr) {
+            float* so = p.S_out + ((long long)bhv * kD + t) * kD + h * 64;
+#pragma unroll
+            for (int part = 0; part < 2; ++part) {
+                uint32_t v[32];
                 tmem_ld32(lane_base + kSD + h * 64 + part * 32, v);
                 tmem_wait_ld();
 #pragma unroll
-                for (int i = 0; i < 16; ++i) pk[i] = pack_bf16x2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
-                tmem_st16(lane_base + kSA + h * 32 + part * 16, pk);
-                // the lo half goes where O2 was (this thread has read its O2 columns above)
-#pragma unroll
-                for (int i = 0; i < 16; ++i)
-                    pk[i] = pack_bf16x2(__uint_as_float(v[2 * i]) - bf16_lo(pk[i]), __uint_as_float(v[2 * i + 1]) - bf16_hi(pk[i]));
-                tmem_st16(lane_base + kO2 + h * 32 + part * 16, pk);
+                for (int i = 0; i < 8; ++i)
+                    *reinterpret_cast<float4*>(so + part * 32 + i * 4) =
+                        make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]), __uint_as_float(v[4 * i + 2]),
+                                    __uint_as_float(v[4 * i + 3]));
             }
-            tmem_wait_st();
         }
-        fence_proxy_async_smem();
-        tc_fence_before_sync();
-        __syncthreads();
-        if (tid == 0) {  // the same thread waits for these stores (bulk groups are per thread)
-            tma_store_3d(&tmO, smem + kOffO, 0, c * kC, bhv);
-            tma_store_3d(&tmO, smem + kOffO + 8192, 64, c * kC, bhv);
-            tma_store_commit();
-        }
+        if (tid == 0) tma_store_wait_all<0>();
     }
-
-    // ---- final state
-    if (ok && p.S_out != nullptr) {
-        float* so = p.S_out + ((long long)bhv * kD + t) * kD + h * 64;
-#pragma unroll
-        for (int part = 0; part < 2; ++part) {
-            uint32_t v[32];
-            tmem_ld32(lane_base + kSD + h * 64 + part * 32, v);
-            tmem_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 8; ++i)
-                *reinterpret_cast<float4*>(so + part * 32 + i * 4) =
-                    make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]), __uint_as_float(v[4 * i + 2]),
-                                __uint_as_float(v[4 * i + 3]));
-        }
-    }
-    if (tid == 0) tma_store_wait_all<0>();
-    if (!ok) atomicExch(p.status, GDN_ERR_TIMEOUT);
     tc_fence_before_sync();
     __syncthreads();
+    if (tid == 0 && *fail != 0) atomicExch(p.status, GDN_ERR_TIMEOUT);
     if (warp == 0) {
         tc_fence_after_sync();
         tmem_dealloc(tmem, kTmemCols);
@@ -510,7 +532,7 @@ int launch_chunk_state(const ProblemS& q, cudaStream_t stream) {
     const int smem = kSmemTotal + 1024;
     if (cudaFuncSetAttribute(chunk_state_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
         return GDN_ERR_LAUNCH;
-    chunk_state_kernel<<<static_cast<int>(hv), kThreads, smem, stream>>>(mQ, mK, mW, mU, mO, prm);
+    chunk_state_kernel<<<static_cast<int>(hv), kThreads + 32, smem, stream>>>(mQ, mK, mW, mU, mO, prm);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? GDN_OK : GDN_ERR_LAUNCH;
 }
