@@ -33,7 +33,7 @@ using namespace sm100;
 
 constexpr int kC = 64;         // chunk size
 constexpr int kD = 128;        // d_k = d_v
-constexpr int kThreads = 256;  // compute threads, two per TMEM lane; one more warp issues the TMA loads and the MMAs
+constexpr int kThreads = 512;  // compute threads, four per TMEM lane; one more warp issues the TMA loads and the MMAs
 constexpr float kLog2e = 1.4426950408889634f;
 
 // TMEM column map (512 columns: one CTA per SM)
@@ -100,7 +100,7 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
     const int t = tid & 127;  // TMEM lane: value feature (state rows, output columns); token j for PT
-    const int h = (tid >> 7) & 1;  // column half
+    const int h = (tid >> 7) & 3;  // column quarter: 16 of the 64 columns of a product, 32 of the 128 state columns
     const int wq = warp & 3;
     const bool issuer = warp == kThreads / 32;  // warp 8: every TMA load and every tcgen05.mma
 
@@ -223,14 +223,14 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             par_2 ^= 1;
             tc_fence_after_sync();
             if (*fail == 0 && elect_one()) {
-                // O2 = U_new^T P^T = Uh Ph + Ul Ph + Uh Pl (K-dim = 64 tokens; the plain copies sit at columns 0..15 and
-                // 32..47 of their regions)
+                // O2 = U_new^T P^T = Uh Ph + Ul Ph + Uh Pl (K-dim = 64 tokens; the plain copy of tokens 16 ks.. sits at
+                // columns 16 ks .. 16 ks + 7 of its region, the gate-scaled one at 16 ks + 8 ..)
 #pragma unroll
                 for (int part = 0; part < 3; ++part) {
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks) {
                         const uint64_t bd = smem_desc(smem_a + kOffP + (part == 2 ? 8192 : 0) + ks * 256, 128, 1024, SWZ_NONE);
-                        mma_f16_ts(tmem + kO2, tmem + (part == 1 ? kPT : kD1) + (ks < 2 ? ks * 8 : 32 + (ks - 2) * 8), bd,
+                        mma_f16_ts(tmem + kO2, tmem + (part == 1 ? kPT : kD1) + ks * 16, bd,
                                    idesc_mn64, part > 0 || ks > 0);
                     }
                 }
@@ -240,7 +240,7 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks) {
                         const uint64_t bd = smem_desc(st_a + kOffK + ks * 2048, 8192, 1024, SWZ_128B);
-                        mma_f16_ts(tmem + kSD, tmem + (part == 0 ? kD1 : kPT) + 16 + (ks < 2 ? ks * 8 : 32 + (ks - 2) * 8), bd,
+                        mma_f16_ts(tmem + kSD, tmem + (part == 0 ? kD1 : kPT) + ks * 16 + 8, bd,
                                    idesc_mn128, true);
                     }
                 }
@@ -257,12 +257,12 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             __syncwarp();
         }
     } else {
-        // ================= compute threads (256): two per TMEM lane
+        // ================= compute threads (512): four per TMEM lane
         uint32_t par_pre = 0, par_d1 = 0, par_o1 = 0, par_g2 = 0;
         // completion of an MMA group: warp 0 polls the mbarrier, the other warps sleep on a hardware barrier
         auto wait_group = [&](uint64_t* bar, uint32_t& par) -> bool {
             if (warp == 0 && !wait_bar(bar, par)) *fail = 1;
-            asm volatile("bar.sync 2, 256;" ::: "memory");
+            asm volatile("bar.sync 2, 512;" ::: "memory");
             par ^= 1;
             tc_fence_after_sync();
             return *fail == 0;
@@ -271,29 +271,26 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         {
             uint32_t r[16];
 #pragma unroll
-            for (int part = 0; part < 2; ++part) {
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const int col = h * 32 + part * 16 + i;  // packed column: features 2 col, 2 col + 1
-                    r[i] = (col == (t >> 1)) ? ((t & 1) ? 0xBF800000u : 0x0000BF80u) : 0u;
-                }
-                tmem_st16(lane_base + kIA + h * 32 + part * 16, r);
+            for (int i = 0; i < 16; ++i) {
+                const int col = h * 16 + i;  // packed column: features 2 col, 2 col + 1
+                r[i] = (col == (t >> 1)) ? ((t & 1) ? 0xBF800000u : 0x0000BF80u) : 0u;
             }
-            // this thread's half of state row t: columns [64 h, 64 h + 64)
-            const float* s0 = (p.S_in != nullptr) ? p.S_in + ((long long)bhv * kD + t) * kD + h * 64 : nullptr;
+            tmem_st16(lane_base + kIA + h * 16, r);
+            // this thread's quarter of state row t: columns [32 h, 32 h + 32)
+            const float* s0 = (p.S_in != nullptr) ? p.S_in + ((long long)bhv * kD + t) * kD + h * 32 : nullptr;
 #pragma unroll
-            for (int part = 0; part < 4; ++part) {
+            for (int part = 0; part < 2; ++part) {
                 uint32_t v[16], pk[8];
 #pragma unroll
                 for (int i = 0; i < 16; ++i) v[i] = (s0 != nullptr) ? __float_as_uint(__ldg(s0 + part * 16 + i)) : 0u;
-                tmem_st16(lane_base + kSD + h * 64 + part * 16, v);
+                tmem_st16(lane_base + kSD + h * 32 + part * 16, v);
 #pragma unroll
                 for (int i = 0; i < 8; ++i) pk[i] = pack_bf16x2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
-                tmem_st8(lane_base + kSA + h * 32 + part * 8, pk);
+                tmem_st8(lane_base + kSA + h * 16 + part * 8, pk);
 #pragma unroll
                 for (int i = 0; i < 8; ++i)
                     pk[i] = pack_bf16x2(__uint_as_float(v[2 * i]) - bf16_lo(pk[i]), __uint_as_float(v[2 * i + 1]) - bf16_hi(pk[i]));
-                tmem_st8(lane_base + kO2 + h * 32 + part * 8, pk);
+                tmem_st8(lane_base + kO2 + h * 16 + part * 8, pk);
             }
             tmem_wait_st();
             tc_fence_before_sync();
@@ -319,78 +316,73 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             }
             // the previous chunk's output store has finished reading the staging tile
             if (tid == 0) tma_store_wait_read<0>();
-            asm volatile("bar.sync 1, 256;" ::: "memory");  // gate tables visible, staging tile free
+            asm volatile("bar.sync 1, 512;" ::: "memory");  // gate tables visible, staging tile free
 
             // ---- decay of the accumulator, S <- exp(g_C) S0 (the products of this chunk read the bf16 copies)
             {
                 const float dec = fast_exp2(gC * kLog2e);
+                uint32_t v[32];
+                tmem_ld32(lane_base + kSD + h * 32, v);
+                tmem_wait_ld();
 #pragma unroll
-                for (int part = 0; part < 2; ++part) {
-                    uint32_t v[32];
-                    tmem_ld32(lane_base + kSD + h * 64 + part * 32, v);
-                    tmem_wait_ld();
+                for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * dec);
+                uint32_t w16[16];
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * dec);
-                    uint32_t w16[16];
+                for (int i = 0; i < 16; ++i) w16[i] = v[i];
+                tmem_st16(lane_base + kSD + h * 32, w16);
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) w16[i] = v[i];
-                    tmem_st16(lane_base + kSD + h * 64 + part * 32, w16);
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) w16[i] = v[16 + i];
-                    tmem_st16(lane_base + kSD + h * 64 + part * 32 + 16, w16);
-                }
+                for (int i = 0; i < 16; ++i) w16[i] = v[16 + i];
+                tmem_st16(lane_base + kSD + h * 32 + 16, w16);
             }
-            // ---- P_ij = exp(g_i - g_j) PT_ji for j <= i (hi + lo): token j = lane (rows 0..63 only), this thread's 32 columns i
+            // ---- P_ij = exp(g_i - g_j) PT_ji for j <= i (hi + lo): token j = lane (rows 0..63 only), this thread's 16 columns i
             if (!wait_group(&bar_pre, par_pre)) { ok = false; break; }
             if (wq < 2) {
-                uint32_t d[32];
-                tmem_ld32(lane_base + kPT + h * 32, d);
+                uint32_t d[16];
+                tmem_ld16(lane_base + kPT + h * 16, d);
                 tmem_wait_ld();
                 const float gj = sg[t] * kLog2e;
 #pragma unroll
-                for (int c4 = 0; c4 < 4; ++c4) {
+                for (int c2 = 0; c2 < 2; ++c2) {
                     uint32_t w[4], wl[4];
 #pragma unroll
                     for (int i2 = 0; i2 < 4; ++i2) {
                         float v[2];
 #pragma unroll
                         for (int q = 0; q < 2; ++q) {
-                            const int i = h * 32 + c4 * 8 + i2 * 2 + q;
-                            const float x = __uint_as_float(d[c4 * 8 + i2 * 2 + q]) * fast_exp2(fminf(fmaf(sg[i], kLog2e, -gj), 0.f));
+                            const int i = h * 16 + c2 * 8 + i2 * 2 + q;
+                            const float x = __uint_as_float(d[c2 * 8 + i2 * 2 + q]) * fast_exp2(fminf(fmaf(sg[i], kLog2e, -gj), 0.f));
                             v[q] = (t <= i) ? x : 0.f;
                         }
                         w[i2] = pack_bf16x2(v[0], v[1]);
                         wl[i2] = pack_bf16x2(v[0] - bf16_lo(w[i2]), v[1] - bf16_hi(w[i2]));
                     }
                     // B operand [K-dim = j][N = i], MN-major, no swizzle: the 16-byte piece of row j for column group n8
-                    *reinterpret_cast<uint4*>(smem + kOffP + (h * 4 + c4) * 1024 + t * 16) = make_uint4(w[0], w[1], w[2], w[3]);
-                    *reinterpret_cast<uint4*>(smem + kOffP + 8192 + (h * 4 + c4) * 1024 + t * 16) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
+                    *reinterpret_cast<uint4*>(smem + kOffP + (h * 2 + c2) * 1024 + t * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+                    *reinterpret_cast<uint4*>(smem + kOffP + 8192 + (h * 2 + c2) * 1024 + t * 16) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
                 }
             }
             // ---- U_new^T = -D1 as bf16 hi + lo, plain and gate-scaled (the sums over the tokens of a chunk telescope
-            // on correlated keys, so single bf16 copies cost 1e-2 there). The hi halves are written over this thread's
-            // own D1 columns (h = 0: plain -> columns 0..15, scaled -> 16..31; h = 1: 32..47 and 48..63), the lo halves
-            // at the same offsets of the PT region (this thread's PT columns have been read above).
+            // on correlated keys, so single bf16 copies cost 1e-2 there). This thread's 16 tokens are one k-step of the
+            // products that consume them: the hi halves are written over its own D1 columns (plain -> 16 h .. 16 h + 7,
+            // scaled -> 16 h + 8 ..), the lo halves at the same offsets of the PT region (read above by this thread).
             if (!wait_group(&bar_d1, par_d1)) { ok = false; break; }
             {
-                uint32_t d[32];
-                tmem_ld32(lane_base + kD1 + h * 32, d);
+                uint32_t d[16];
+                tmem_ld16(lane_base + kD1 + h * 16, d);
                 tmem_wait_ld();
-                uint32_t pp[16], ps[16], lp[16], ls[16];
+                uint32_t hi[16], lo[16];
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
+                for (int i = 0; i < 8; ++i) {
                     const float u0 = -__uint_as_float(d[2 * i]), u1 = -__uint_as_float(d[2 * i + 1]);
-                    const float2 f = *reinterpret_cast<const float2*>(sf + h * 32 + 2 * i);
+                    const float2 f = *reinterpret_cast<const float2*>(sf + h * 16 + 2 * i);
                     const float s0 = u0 * f.x, s1 = u1 * f.y;
-                    pp[i] = pack_bf16x2(u0, u1);
-                    ps[i] = pack_bf16x2(s0, s1);
-                    lp[i] = pack_bf16x2(u0 - bf16_lo(pp[i]), u1 - bf16_hi(pp[i]));
-                    ls[i] = pack_bf16x2(s0 - bf16_lo(ps[i]), s1 - bf16_hi(ps[i]));
+                    hi[i] = pack_bf16x2(u0, u1);
+                    hi[8 + i] = pack_bf16x2(s0, s1);
+                    lo[i] = pack_bf16x2(u0 - bf16_lo(hi[i]), u1 - bf16_hi(hi[i]));
+                    lo[8 + i] = pack_bf16x2(s0 - bf16_lo(hi[8 + i]), s1 - bf16_hi(hi[8 + i]));
                 }
-                tmem_st16(lane_base + kD1 + h * 32, pp);
-                tmem_st16(lane_base + kD1 + h * 32 + 16, ps);
-                tmem_st16(lane_base + kPT + h * 32, lp);
-                tmem_st16(lane_base + kPT + h * 32 + 16, ls);
+                tmem_st16(lane_base + kD1 + h * 16, hi);
+                tmem_st16(lane_base + kPT + h * 16, lo);
             }
             fence_proxy_async_smem();
             tmem_wait_st();
@@ -399,25 +391,25 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 
             // ---- exp(g_i) O1
             if (!wait_group(&bar_o1, par_o1)) { ok = false; break; }
-            float o[32];
+            float o[16];
             {
-                uint32_t d[32];
-                tmem_ld32(lane_base + kO1 + h * 32, d);
+                uint32_t d[16];
+                tmem_ld16(lane_base + kO1 + h * 16, d);
                 tmem_wait_ld();
 #pragma unroll
-                for (int i = 0; i < 32; ++i) o[i] = __uint_as_float(d[i]) * se[h * 32 + i];
+                for (int i = 0; i < 16; ++i) o[i] = __uint_as_float(d[i]) * se[h * 16 + i];
             }
             if (!wait_group(&bar_g2, par_g2)) { ok = false; break; }
             // ---- O^T = scale (exp(g_i) O1 + O2): element (token i, feature t) of the staged tile
             {
-                uint32_t d[32];
-                tmem_ld32(lane_base + kO2 + h * 32, d);
+                uint32_t d[16];
+                tmem_ld16(lane_base + kO2 + h * 16, d);
                 tmem_wait_ld();
                 uint8_t* sub = smem + kOffO + (t >> 6) * 8192;
                 const int cch = (t & 63) >> 3;
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const int tok = h * 32 + i;
+                for (int i = 0; i < 16; ++i) {
+                    const int tok = h * 16 + i;
                     const __nv_bfloat16 v = __float2bfloat16_rn(p.scale * (o[i] + __uint_as_float(d[i])));
                     *reinterpret_cast<__nv_bfloat16*>(sub + tok * 128 + ((cch ^ (tok & 7)) << 4) + (t & 7) * 2) = v;
                 }
@@ -425,25 +417,22 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             // ---- bf16 copies (hi, lo) of the new state for the next chunk's products; the lo half goes where O2 was
             // (this thread has read its O2 columns above)
             {
+                uint32_t v[32], pk[16];
+                tmem_ld32(lane_base + kSD + h * 32, v);
+                tmem_wait_ld();
 #pragma unroll
-                for (int part = 0; part < 2; ++part) {
-                    uint32_t v[32], pk[16];
-                    tmem_ld32(lane_base + kSD + h * 64 + part * 32, v);
-                    tmem_wait_ld();
+                for (int i = 0; i < 16; ++i) pk[i] = pack_bf16x2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
+                tmem_st16(lane_base + kSA + h * 16, pk);
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) pk[i] = pack_bf16x2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
-                    tmem_st16(lane_base + kSA + h * 32 + part * 16, pk);
-#pragma unroll
-                    for (int i = 0; i < 16; ++i)
-                        pk[i] = pack_bf16x2(__uint_as_float(v[2 * i]) - bf16_lo(pk[i]), __uint_as_float(v[2 * i + 1]) - bf16_hi(pk[i]));
-                    tmem_st16(lane_base + kO2 + h * 32 + part * 16, pk);
-                }
+                for (int i = 0; i < 16; ++i)
+                    pk[i] = pack_bf16x2(__uint_as_float(v[2 * i]) - bf16_lo(pk[i]), __uint_as_float(v[2 * i + 1]) - bf16_hi(pk[i]));
+                tmem_st16(lane_base + kO2 + h * 16, pk);
                 tmem_wait_st();
                 tc_fence_before_sync();
                 mbar_arrive(&bar_rdy_a);
             }
             fence_proxy_async_smem();
-            asm volatile("bar.sync 1, 256;" ::: "memory");  // the staged output tile is complete
+            asm volatile("bar.sync 1, 512;" ::: "memory");  // the staged output tile is complete
             if (tid == 0) {  // the same thread waits for these stores (bulk groups are per thread)
                 tma_store_3d(&tmO, smem + kOffO, 0, c * kC, bhv);
                 tma_store_3d(&tmO, smem + kOffO + 8192, 64, c * kC, bhv);
@@ -452,18 +441,15 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         }
         // ---- final state
         if (ok && p.S_out != nullptr) {
-            float* so = p.S_out + ((long long)bhv * kD + t) * kD + h * 64;
+            float* so = p.S_out + ((long long)bhv * kD + t) * kD + h * 32;
+            uint32_t v[32];
+            tmem_ld32(lane_base + kSD + h * 32, v);
+            tmem_wait_ld();
 #pragma unroll
-            for (int part = 0; part < 2; ++part) {
-                uint32_t v[32];
-                tmem_ld32(lane_base + kSD + h * 64 + part * 32, v);
-                tmem_wait_ld();
-#pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    *reinterpret_cast<float4*>(so + part * 32 + i * 4) =
-                        make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]), __uint_as_float(v[4 * i + 2]),
-                                    __uint_as_float(v[4 * i + 3]));
-            }
+            for (int i = 0; i < 8; ++i)
+                *reinterpret_cast<float4*>(so + i * 4) =
+                    make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]), __uint_as_float(v[4 * i + 2]),
+                                __uint_as_float(v[4 * i + 3]));
         }
         if (tid == 0) tma_store_wait_all<0>();
     }
