@@ -202,12 +202,22 @@ def run_ours(args, rank, world, dist_ctx):
     if method == "int8":
         q8 = gen.make_int8_inputs(inp)
         q8_outs = gdn.chunk_prepare_int8(q8)
+    st_args = None
+    if method == "state":  # state passing + output of the layer, given the gated W and U
+        gq = torch.Generator(device=dev).manual_seed(99)
+        Qs = torch.randn(inp.B, inp.H_k, inp.T, inp.d_k, device=dev, generator=gq)
+        Qs = (Qs / Qs.norm(dim=-1, keepdim=True)).to(inp.K.dtype)
+        Wg, Ug, _ = gdn.chunk_prepare(inp.K, inp.V, inp.beta, inp.g, C, flags=gdn.GDN_FLAG_W_GATED, want_tinv=False)
+        st_outs = gdn.chunk_state_output(Qs, inp.K, Wg, Ug, inp.g, C, inp.d_k ** -0.5)
+        st_args = (Qs, Wg, Ug, st_outs)
 
     def step():
         if method == "neumann":
             gdn.chunk_prepare(inp.K, inp.V, inp.beta, inp.g, C, outputs=outs)
         elif method == "int8":
             gdn.chunk_prepare_int8(q8, outputs=q8_outs)
+        elif method == "state":
+            gdn.chunk_state_output(st_args[0], inp.K, st_args[1], st_args[2], inp.g, C, inp.d_k ** -0.5, outputs=st_args[3])
         else:
             gdn.chunk_prepare(inp.K, inp.V, inp.beta, inp.g, C, outputs=outs, method="fwdsubst",
                               variant=gdn.GDN_FWDSUBST_BLOCKED if method == "fwdsubst-blocked" else gdn.GDN_FWDSUBST_ROWS)
@@ -232,6 +242,8 @@ def run_ours(args, rank, world, dist_ctx):
     value = whole_job_throughput(n_chunks, world, ms_per_step)
 
     bytes_chunk = algorithmic_bytes_per_chunk(C, inp.d_k, inp.d_v, group)
+    if method == "state":  # Q, K (shared by a group), W, U read, O written, g
+        bytes_chunk = C * inp.d_k * 2 * (2.0 / group + 1) + 2 * C * inp.d_v * 2 + 4 * C
     if method == "int8":  # one byte per element, u16 beta + i32 decay per token
         bytes_chunk = C * inp.d_k / group + C * inp.d_v + C * inp.d_k + C * inp.d_v + C * C + 6 * C
     flops_chunk = nominal_flops_per_chunk(C, inp.d_k, inp.d_v)
@@ -241,7 +253,7 @@ def run_ours(args, rank, world, dist_ctx):
     roofline = {"bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak,
                 "traffic": TRAFFIC_PER_LAUNCH.get(args.workload) if method == "neumann" else None, "peak_kind": peak_kind,
                 "algorithmic_bytes_per_launch": n_chunks * bytes_chunk,
-                "kernel": ("chunk_tc_int8_kernel" if method == "int8" else "chunk_tc_kernel<C=%d>" % C),
+                "kernel": {"int8": "chunk_tc_int8_kernel", "state": "chunk_state_kernel"}.get(method, "chunk_tc_kernel<C=%d>" % C),
                 "effective_tflops": n_chunks * flops_chunk / (launch_ms * 1e-3) / 1e12,
                 "tensor_time_frac_of_bf16_peak": (n_chunks * flops_chunk / (launch_ms * 1e-3) / 1e12) / bf16_peak}
 
@@ -349,6 +361,27 @@ def run_extras(gdn, gen, dev, args):
             del inp, outs
         except Exception as exc:  # an unsupported extra must not lose the headline
             out[f"{name}:{method}"] = {"error": repr(exc)}
+    # the rest of the layer (state passing + output, given the gated W and U) on the prefill and stress shapes
+    for name in ("prefill_gqa", "stress"):
+        try:
+            inp = gen.make_workload(name, device=dev)
+            gq = torch.Generator(device=dev).manual_seed(99)
+            Q = torch.randn(inp.B, inp.H_k, inp.T, inp.d_k, device=dev, generator=gq)
+            Q = (Q / Q.norm(dim=-1, keepdim=True)).to(inp.K.dtype)
+            W, U, _ = gdn.chunk_prepare(inp.K, inp.V, inp.beta, inp.g, inp.C, flags=gdn.GDN_FLAG_W_GATED, want_tinv=False)
+            outs = gdn.chunk_state_output(Q, inp.K, W, U, inp.g, inp.C, inp.d_k ** -0.5)
+            fn = lambda: gdn.chunk_state_output(Q, inp.K, W, U, inp.g, inp.C, inp.d_k ** -0.5, outputs=outs)
+            total_ms, _ = device_time_steps(fn, 5, 2, None)
+            ms = total_ms / 5
+            group = inp.H_v // inp.H_k
+            # Q, K tiles (shared by a group), W, U read, O written, g
+            by = inp.C * inp.d_k * 2 * (2.0 / group + 1) + 2 * inp.C * inp.d_v * 2 + 4 * inp.C
+            out[f"{name}:state_output"] = {"chunks_per_s": inp.n_chunks / (ms * 1e-3), "ms": ms,
+                                           "hbm_frac": inp.n_chunks * by / (ms * 1e-3) / 1e9 / hbm_peak,
+                                           "us_per_chunk_of_a_sequence": ms * 1e3 / (inp.T // inp.C)}
+            del inp, Q, W, U, outs
+        except Exception as exc:
+            out[f"{name}:state_output"] = {"error": repr(exc)}
     # INT8 variant on the prefill shapes (integer inputs quantised once from the same tensors)
     try:
         inp = gen.make_workload("prefill_gqa", device=dev)
@@ -400,7 +433,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--method", default="neumann", choices=["neumann", "fwdsubst", "fwdsubst-blocked", "int8"])
+    ap.add_argument("--method", default="neumann", choices=["neumann", "fwdsubst", "fwdsubst-blocked", "int8", "state"])
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extras", action="store_true")
