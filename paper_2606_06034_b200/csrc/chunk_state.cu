@@ -33,7 +33,7 @@ using namespace sm100;
 
 constexpr int kC = 64;         // chunk size
 constexpr int kD = 128;        // d_k = d_v
-constexpr int kThreads = 512;  // compute threads, four per TMEM lane; one more warp issues the TMA loads and the MMAs
+constexpr int kThreads = 512;  // compute threads, four per TMEM lane; two more warps issue the MMAs and the TMA loads
 constexpr float kLog2e = 1.4426950408889634f;
 
 // TMEM column map (512 columns: one CTA per SM)
@@ -51,9 +51,18 @@ constexpr int kTileBytes = 16384;
 constexpr int kStageBytes = 4 * kTileBytes;  // Q, K, W, U
 constexpr int kOffQ = 0, kOffK = kTileBytes, kOffW = 2 * kTileBytes, kOffU = 3 * kTileBytes;
 constexpr int kOffP = 2 * kStageBytes;       // 2 x 8 KB: P as B operand [64 x 64] (MN-major, no swizzle), hi and lo halves
-constexpr int kOffO = kOffP + 16384;          // 16 KB: O tile staged for the bulk store (128B swizzle)
-constexpr int kOffG = kOffO + kTileBytes;    // 3 x 64 floats: exp(g_i), exp(g_C - g_j), g
-constexpr int kSmemTotal = kOffG + 3 * 64 * 4;
+constexpr int kOffO = kOffP + 16384;          // 2 x 16 KB: O tile staged for the bulk store (128B swizzle), two buffers
+constexpr int kOffG = kOffO + 2 * kTileBytes;  // 2 x 3 x 64 floats: exp(g_i), exp(g_C - g_j), g; two buffers
+constexpr int kSmemTotal = kOffG + 2 * 3 * 64 * 4;
+
+#ifdef GDN_TRACE
+__device__ long long g_trace_s[4096];
+// slot, clock pairs of block 0: compute thread 0 at [0, 2048), the issuing warp's lane 0 at [2048, 4096)
+#define STAMPS(slot_) do { if (blockIdx.x == 0 && (tid == 0 || tid == kThreads) && trace_n < 500) { \
+    g_trace_s[(tid == 0 ? 0 : 2048) + trace_n * 2] = (slot_); g_trace_s[(tid == 0 ? 0 : 2048) + trace_n * 2 + 1] = clock64(); ++trace_n; } } while (0)
+#else
+#define STAMPS(slot_) do { } while (0)
+#endif
 
 struct ParamsS {
     const float* g;
@@ -81,28 +90,31 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity) {
     return true;
 }
 
-__global__ void __launch_bounds__(kThreads + 32, 1)
+__global__ void __launch_bounds__(kThreads + 64, 1)
 chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                    const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmU,
                    const __grid_constant__ CUtensorMap tmO, const ParamsS p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    float* se = reinterpret_cast<float*>(smem + kOffG);  // exp(g_i)
-    float* sf = se + 64;                                  // exp(g_C - g_j)
-    float* sg = sf + 64;                                  // g_i
+    float* gtab = reinterpret_cast<float*>(smem + kOffG);  // per buffer: exp(g_i), exp(g_C - g_j), g_i (64 each)
 
     // One mbarrier per MMA group (never two pending phases on one barrier), two per-stage TMA barriers, and two
     // barriers on which the 256 compute threads tell the issuing warp that operands are in place.
-    __shared__ uint64_t bar_full[2], bar_pre, bar_d1, bar_o1, bar_g2, bar_rdy_a, bar_rdy_2;
+    __shared__ uint64_t bar_full[2], bar_pre, bar_d1, bar_o1, bar_o2, bar_g2, bar_rdy_a, bar_rdy_2;
     __shared__ uint32_t tmem_base_s;
     __shared__ int s_fail;
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
+#ifdef GDN_TRACE
+    int trace_n = 0;
+#endif
     const int t = tid & 127;  // TMEM lane: value feature (state rows, output columns); token j for PT
     const int h = (tid >> 7) & 3;  // column quarter: 16 of the 64 columns of a product, 32 of the 128 state columns
     const int wq = warp & 3;
-    const bool issuer = warp == kThreads / 32;  // warp 8: every TMA load and every tcgen05.mma
+    const int lane = tid & 31;
+    const bool issuer = warp == kThreads / 32;        // every tcgen05.mma
+    const bool producer = warp == kThreads / 32 + 1;  // every TMA load
 
     if (tid == 0) {
         mbar_init(&bar_full[0], 1);
@@ -110,6 +122,7 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         mbar_init(&bar_pre, 1);
         mbar_init(&bar_d1, 1);
         mbar_init(&bar_o1, 1);
+        mbar_init(&bar_o2, 1);
         mbar_init(&bar_g2, 1);
         mbar_init(&bar_rdy_a, kThreads);
         mbar_init(&bar_rdy_2, kThreads);
@@ -139,25 +152,39 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     const uint32_t smem_a = smem_u32(smem);
     volatile int* fail = reinterpret_cast<volatile int*>(&s_fail);
 
-    if (issuer) {
-        // ================= issuing warp: TMA loads and every tcgen05.mma, in the order the tensor pipe runs them
+    if (producer) {
+        // ================= loading warp: the four tiles of chunk c into stage c & 1, as soon as the products that
+        // read the stage's previous tiles are complete
+        if (elect_one()) {
+            auto load_stage = [&](int c) {
+                uint8_t* st = smem + (c & 1) * kStageBytes;
+                uint64_t* bar = &bar_full[c & 1];
+                mbar_arrive_expect_tx(bar, kStageBytes);
+                const int t0 = c * kC;
+                tma_load_3d(st + kOffQ, &tmQ, bar, 0, t0, bhk);
+                tma_load_3d(st + kOffQ + 8192, &tmQ, bar, 64, t0, bhk);
+                tma_load_3d(st + kOffK, &tmK, bar, 0, t0, bhk);
+                tma_load_3d(st + kOffK + 8192, &tmK, bar, 64, t0, bhk);
+                tma_load_3d(st + kOffW, &tmW, bar, 0, t0, bhv);
+                tma_load_3d(st + kOffW + 8192, &tmW, bar, 64, t0, bhv);
+                tma_load_3d(st + kOffU, &tmU, bar, 0, t0, bhv);
+                tma_load_3d(st + kOffU + 8192, &tmU, bar, 64, t0, bhv);
+            };
+            if (n_c > 0) load_stage(0);
+            if (n_c > 1) load_stage(1);
+            uint32_t par = 0;
+            for (int c = 0; c + 2 < n_c && *fail == 0; ++c) {
+                if (!wait_bar(&bar_g2, par)) *fail = 1;
+                par ^= 1;
+                if (*fail == 0) load_stage(c + 2);
+            }
+        }
+        __syncwarp();
+    } else if (issuer) {
+        // ================= issuing warp: every tcgen05.mma, in the order the tensor pipe runs them
         const uint32_t idesc_kk64 = instr_desc(128, 64, 1, 1, 0, 0, 1);   // B K-major (a TMA tile as [N x K])
         const uint32_t idesc_mn64 = instr_desc(128, 64, 1, 1, 0, 1, 1);   // B MN-major
         const uint32_t idesc_mn128 = instr_desc(128, 128, 1, 1, 0, 1, 1);
-        auto load_stage = [&](int c) {  // the four tiles of chunk c into stage c & 1
-            uint8_t* st = smem + (c & 1) * kStageBytes;
-            uint64_t* bar = &bar_full[c & 1];
-            mbar_arrive_expect_tx(bar, kStageBytes);
-            const int t0 = c * kC;
-            tma_load_3d(st + kOffQ, &tmQ, bar, 0, t0, bhk);
-            tma_load_3d(st + kOffQ + 8192, &tmQ, bar, 64, t0, bhk);
-            tma_load_3d(st + kOffK, &tmK, bar, 0, t0, bhk);
-            tma_load_3d(st + kOffK + 8192, &tmK, bar, 64, t0, bhk);
-            tma_load_3d(st + kOffW, &tmW, bar, 0, t0, bhv);
-            tma_load_3d(st + kOffW + 8192, &tmW, bar, 64, t0, bhv);
-            tma_load_3d(st + kOffU, &tmU, bar, 0, t0, bhv);
-            tma_load_3d(st + kOffU + 8192, &tmU, bar, 64, t0, bhv);
-        };
         // the products of chunk c that do not depend on the state: D1 <- (-I) U^T and PT = K Q^T
         auto issue_pre = [&](int c) {
             const uint32_t sa = smem_a + (c & 1) * kStageBytes;
@@ -180,19 +207,14 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             }
             __syncwarp();
         };
-        if (n_c > 0) {
-            if (elect_one()) {
-                load_stage(0);
-                if (n_c > 1) load_stage(1);
-            }
-            __syncwarp();
-        }
-        uint32_t par_a = 0, par_2 = 0, par_g2 = 0;
+        uint32_t par_a = 0, par_2 = 0;
         for (int c = 0; c < n_c && *fail == 0; ++c) {
             const uint32_t st_a = smem_a + (c & 1) * kStageBytes;
             // the state copies (and, for the first chunk, the constant operand) are in place
+            STAMPS(100);
             if (!wait_bar(&bar_rdy_a, par_a)) *fail = 1;
             par_a ^= 1;
+            STAMPS(101);
             tc_fence_after_sync();
             if (c == 0) issue_pre(0);
             if (*fail == 0 && elect_one()) {
@@ -218,9 +240,11 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 mma_commit(&bar_o1);
             }
             __syncwarp();
+            STAMPS(102);
             // U_new^T (hi, lo; plain, scaled), P (hi, lo) and the decayed accumulator are in place
             if (!wait_bar(&bar_rdy_2, par_2)) *fail = 1;
             par_2 ^= 1;
+            STAMPS(103);
             tc_fence_after_sync();
             if (*fail == 0 && elect_one()) {
                 // O2 = U_new^T P^T = Uh Ph + Ul Ph + Uh Pl (K-dim = 64 tokens; the plain copy of tokens 16 ks.. sits at
@@ -234,6 +258,7 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                                    idesc_mn64, part > 0 || ks > 0);
                     }
                 }
+                mma_commit(&bar_o2);  // the output is finished while the state update still runs
                 // S += (U_new^T exp(g_C - g_j)) K, hi + lo (the K tile as MN-major operand, N = 128)
 #pragma unroll
                 for (int part = 0; part < 2; ++part) {
@@ -249,23 +274,22 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             __syncwarp();
             // D1 and PT are only read by the products just issued, which the tensor pipe runs first: the
             // state-independent products of the next chunk follow them directly
+            STAMPS(104);
             if (c + 1 < n_c) issue_pre(c + 1);
-            // once those products are complete the tiles of this stage are free for the chunk after the next one
-            if (!wait_bar(&bar_g2, par_g2)) *fail = 1;
-            par_g2 ^= 1;
-            if (*fail == 0 && c + 2 < n_c && elect_one()) load_stage(c + 2);
-            __syncwarp();
+            STAMPS(105);
         }
     } else {
         // ================= compute threads (512): four per TMEM lane
-        uint32_t par_pre = 0, par_d1 = 0, par_o1 = 0, par_g2 = 0;
+        uint32_t par_pre = 0, par_d1 = 0, par_o1 = 0, par_o2 = 0, par_g2 = 0;
         // completion of an MMA group: warp 0 polls the mbarrier, the other warps sleep on a hardware barrier
+        // completion of an MMA group: lane 0 of every warp polls the mbarrier (no CTA-wide barrier on this path)
         auto wait_group = [&](uint64_t* bar, uint32_t& par) -> bool {
-            if (warp == 0 && !wait_bar(bar, par)) *fail = 1;
-            asm volatile("bar.sync 2, 512;" ::: "memory");
+            int good = 1;
+            if (lane == 0 && !wait_bar(bar, par)) { *fail = 1; good = 0; }
+            good = __shfl_sync(0xFFFFFFFFu, good, 0);
             par ^= 1;
             tc_fence_after_sync();
-            return *fail == 0;
+            return good != 0;
         };
         // ---- constant A operand -I, initial state, and its bf16 copies (hi in kSA, lo in kO2)
         {
@@ -303,21 +327,29 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             gC_reg = __ldg(gseq + kC - 1);
         }
         bool ok = true;
+        // gate tables of a chunk: written by 64 threads into the buffer of that chunk one barrier before they are read
+        auto fill_tables = [&](int c) {
+            if (tid < 64) {
+                float* tb = gtab + (c & 1) * 192;
+                tb[tid] = fast_exp2(g_reg * kLog2e);
+                tb[64 + tid] = fast_exp2((gC_reg - g_reg) * kLog2e);
+                tb[128 + tid] = g_reg;
+            }
+        };
+        if (n_c > 0) fill_tables(0);
+        asm volatile("bar.sync 1, 512;" ::: "memory");
         for (int c = 0; c < n_c; ++c) {
             const float gC = gC_reg;
-            if (tid < 64) {
-                sg[tid] = g_reg;
-                se[tid] = fast_exp2(g_reg * kLog2e);
-                sf[tid] = fast_exp2((gC - g_reg) * kLog2e);
-            }
+            const float* se = gtab + (c & 1) * 192;  // exp(g_i)
+            const float* sf = se + 64;               // exp(g_C - g_j)
+            const float* sg = se + 128;              // g_i
             if (c + 1 < n_c) {
                 if (tid < 64) g_reg = __ldg(gseq + (c + 1) * kC + tid);
                 gC_reg = __ldg(gseq + (c + 2) * kC - 1);
             }
-            // the previous chunk's output store has finished reading the staging tile
-            if (tid == 0) tma_store_wait_read<0>();
-            asm volatile("bar.sync 1, 512;" ::: "memory");  // gate tables visible, staging tile free
+            STAMPS(1);
 
+            STAMPS(2);
             // ---- decay of the accumulator, S <- exp(g_C) S0 (the products of this chunk read the bf16 copies)
             {
                 const float dec = fast_exp2(gC * kLog2e);
@@ -335,7 +367,9 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 tmem_st16(lane_base + kSD + h * 32 + 16, w16);
             }
             // ---- P_ij = exp(g_i - g_j) PT_ji for j <= i (hi + lo): token j = lane (rows 0..63 only), this thread's 16 columns i
+            STAMPS(3);
             if (!wait_group(&bar_pre, par_pre)) { ok = false; break; }
+            STAMPS(4);
             if (wq < 2) {
                 uint32_t d[16];
                 tmem_ld16(lane_base + kPT + h * 16, d);
@@ -366,6 +400,7 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             // products that consume them: the hi halves are written over its own D1 columns (plain -> 16 h .. 16 h + 7,
             // scaled -> 16 h + 8 ..), the lo halves at the same offsets of the PT region (read above by this thread).
             if (!wait_group(&bar_d1, par_d1)) { ok = false; break; }
+            STAMPS(6);
             {
                 uint32_t d[16];
                 tmem_ld16(lane_base + kD1 + h * 16, d);
@@ -388,9 +423,11 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             tmem_wait_st();
             tc_fence_before_sync();
             mbar_arrive(&bar_rdy_2);
+            STAMPS(7);
 
             // ---- exp(g_i) O1
             if (!wait_group(&bar_o1, par_o1)) { ok = false; break; }
+            STAMPS(8);
             float o[16];
             {
                 uint32_t d[16];
@@ -399,13 +436,15 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 #pragma unroll
                 for (int i = 0; i < 16; ++i) o[i] = __uint_as_float(d[i]) * se[h * 16 + i];
             }
-            if (!wait_group(&bar_g2, par_g2)) { ok = false; break; }
+            STAMPS(9);
+            if (!wait_group(&bar_o2, par_o2)) { ok = false; break; }
+            STAMPS(10);
             // ---- O^T = scale (exp(g_i) O1 + O2): element (token i, feature t) of the staged tile
             {
                 uint32_t d[16];
                 tmem_ld16(lane_base + kO2 + h * 16, d);
                 tmem_wait_ld();
-                uint8_t* sub = smem + kOffO + (t >> 6) * 8192;
+                uint8_t* sub = smem + kOffO + (c & 1) * kTileBytes + (t >> 6) * 8192;
                 const int cch = (t & 63) >> 3;
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
@@ -416,6 +455,8 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             }
             // ---- bf16 copies (hi, lo) of the new state for the next chunk's products; the lo half goes where O2 was
             // (this thread has read its O2 columns above)
+            if (!wait_group(&bar_g2, par_g2)) { ok = false; break; }
+            STAMPS(12);
             {
                 uint32_t v[32], pk[16];
                 tmem_ld32(lane_base + kSD + h * 32, v);
@@ -431,11 +472,16 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 tc_fence_before_sync();
                 mbar_arrive(&bar_rdy_a);
             }
+            STAMPS(11);
+            if (c + 1 < n_c) fill_tables(c + 1);
             fence_proxy_async_smem();
-            asm volatile("bar.sync 1, 512;" ::: "memory");  // the staged output tile is complete
+            // the store of the previous chunk has finished reading its staging buffer, which the next chunk writes
+            // (issued a whole chunk ago: this never waits in practice; the barrier below publishes it)
+            if (tid == 0) tma_store_wait_read<0>();
+            asm volatile("bar.sync 1, 512;" ::: "memory");  // the staged output tile and the next gate tables are complete
             if (tid == 0) {  // the same thread waits for these stores (bulk groups are per thread)
-                tma_store_3d(&tmO, smem + kOffO, 0, c * kC, bhv);
-                tma_store_3d(&tmO, smem + kOffO + 8192, 64, c * kC, bhv);
+                tma_store_3d(&tmO, smem + kOffO + (c & 1) * kTileBytes, 0, c * kC, bhv);
+                tma_store_3d(&tmO, smem + kOffO + (c & 1) * kTileBytes + 8192, 64, c * kC, bhv);
                 tma_store_commit();
             }
         }
@@ -494,6 +540,12 @@ bool make_map(CUtensorMap* tm, const void* base, long long heads, int T) {
 
 }  // namespace
 
+#ifdef GDN_TRACE
+extern "C" int gdn_debug_read_trace_state(long long* host_out) {
+    return cudaMemcpyFromSymbol(host_out, g_trace_s, sizeof(long long) * 4096) == cudaSuccess ? 0 : -1;
+}
+#endif
+
 int launch_chunk_state(const ProblemS& q, cudaStream_t stream) {
     if (q.d_k != kD || q.d_v != kD || q.C != kC) return GDN_ERR_UNSUPPORTED;
     const long long hk = (long long)q.B * q.H_k, hv = (long long)q.B * q.H_v;
@@ -518,7 +570,7 @@ int launch_chunk_state(const ProblemS& q, cudaStream_t stream) {
     const int smem = kSmemTotal + 1024;
     if (cudaFuncSetAttribute(chunk_state_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
         return GDN_ERR_LAUNCH;
-    chunk_state_kernel<<<static_cast<int>(hv), kThreads + 32, smem, stream>>>(mQ, mK, mW, mU, mO, prm);
+    chunk_state_kernel<<<static_cast<int>(hv), kThreads + 64, smem, stream>>>(mQ, mK, mW, mU, mO, prm);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? GDN_OK : GDN_ERR_LAUNCH;
 }
