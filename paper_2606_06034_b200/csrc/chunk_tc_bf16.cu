@@ -1,9 +1,9 @@
 // Tensor-core kernel (tcgen05 + TMEM + TMA) for the bf16 chunk-prepare path.
 //
-// Work item = one tile of 128 consecutive tokens of one (batch, value head): 128 / C chunks, which
-// sit as diagonal blocks of every 128 x 128 operand (chunks are independent, so the tile's matrices
-// are block diagonal). Thread t of the four compute warps owns row t of the tile (TMEM lane t); a
-// fifth warp's lane 0 issues the TMA loads and every tcgen05.mma.
+// Work item = one tile of 128 consecutive tokens of one (batch, value head): 128 / C chunks, which sit as diagonal
+// blocks of every 128 x 128 operand (chunks are independent, so the tile's matrices are block diagonal). Threads t and
+// t + 128 share row t of the tile (TMEM lane t) and split its chunk columns; one elected lane of warp 0 issues the TMA
+// loads and every tcgen05.mma. Two CTAs per SM, persistent over the tiles.
 //
 // Per tile (paper's notation, Abar = -A, Sec. 3 / Alg. 1):
 //   G = K K^T                         tcgen05.mma, K tile staged by TMA (128B swizzle)      -> TMEM
@@ -11,16 +11,18 @@
 //   L = T0 - I = band_{1<=i-j<=N}(sum_n Abar^n)  (Eq. 7, 10, 11), by the distance recursion
 //       L_d[i] = Abar[i,i-d] + sum_{e<d} Abar[i,i-e] L_{d-e}[i-e], which equals the masked sum exactly
 //   E = Abar + Abar L  on i-j > N, exactly 0 inside the band (Eq. 13)               registers, fp32
-//   X_1 = E, X_{k+1} = E + X_k E  (S-1 dependent MMAs; X as bf16 A operand in TMEM, E as B in smem)
-//   far = X_S + L X_S = T - I - L                                                     (one MMA)
-//   T = I + L + far  -> Tinv
-//   W = (I + L) diag(beta) K  [fp32 FMAs on the band]  +  (far diag(beta)) K  [MMA], same for U with V
-// Only small quantities (E, X, far) pass through bf16 MMA operands; the identity and the O(1) band
-// stay in fp32, which keeps the result within bf16 output rounding of the fp64 definition even for
-// strongly correlated keys.
+//   residual sum (Eq. 13): Z_0 = 0, Z_{k+1} = (T0 + Z_k) E, k < S, so that T = T0 + Z_S; chunks stacked along M,
+//       A operand = bf16(T0 + Z_k) in TMEM, B operand = E in shared memory. For S = 8 and S = 15 at C = 64 the same
+//       sum by four doubling levels (X_{2m+1} = X_m + X_m E^{m+1}), see the kernel body.
+//   T = I + L + Z_S  -> Tinv
+//   W = (T diag(beta)) K, U = (T diag(beta)) V: T diag(beta) as hi + lo bf16 A operands (lo on band and diagonal),
+//       the K / V tile itself as MN-major B operand
+//   C = 128: the two 64-blocks as above, then the block formula of App. E for the lower-left block (hi + lo operands).
+// The identity and the O(1) band never pass through a single bf16 operand, which keeps the result within bf16 output
+// rounding of the fp64 definition even for strongly correlated keys.
 //
-// The forward-substitution comparison (Eq. 2-3) replaces the L/E/X/far steps by a column-parallel
-// substitution in shared memory and reuses everything else.
+// The forward-substitution comparisons (Eq. 2-3; App. E for the blocked form) replace the L / E / residual steps by a
+// column-parallel substitution in shared memory and reuse everything else.
 #include <cuda.h>
 
 #include "common.cuh"
