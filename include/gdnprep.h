@@ -157,13 +157,14 @@ int gdn_chunk_prepare_int8(const int8_t* Kq, const int8_t* Vq, const int32_t* k_
  * o_t = scale * S_t q_t when W = T diag(beta exp(g)) K (gdn_chunk_prepare_ex with GDN_FLAG_W_GATED) and
  * U = T diag(beta) V.
  *   Q, K [B,H_k,T,d_k], W_gated [B,H_v,T,d_k], U [B,H_v,T,d_v] bf16; g [B,H_v,T] fp32, the cumulative log-gate
- *   that RESTARTS in every chunk (chunk-local inclusive prefix sum); S_in [B,H_v,d_v,d_k] fp32 or NULL (zero state);
+ *   that RESTARTS in every chunk (chunk-local inclusive prefix sum), or with flags = GDN_FLAG_G_RAW the raw per-token
+ *   log-gates (the prefix sum is then formed here, as gdn_chunk_prepare_ex does); no other flag is accepted; S_in [B,H_v,d_v,d_k] fp32 or NULL (zero state);
  *   O_out [B,H_v,T,d_v] bf16; S_out [B,H_v,d_v,d_k] fp32 or NULL.
  * Supported: C = 64, d_k = d_v = 128, T a multiple of C. fp32 state, bf16 tensor-core operands.
  */
 int gdn_chunk_state_output(const void* Q, const void* K, const void* W_gated, const void* U, const float* g,
                            int B, int H_k, int H_v, int T, int C, int d_k, int d_v, float scale,
-                           const float* S_in, void* O_out, float* S_out, gdn_stream_t stream);
+                           const float* S_in, void* O_out, float* S_out, unsigned flags, gdn_stream_t stream);
 
 /* Checksum of the 256-entry gate-decay table round(2^15 * 2^(-f/256)) the INT8 kernel uses
  * (sum_f: s = (31 s + table[f] + f) mod 1000000007), so that a CPU evaluation can confirm it holds the same table. */

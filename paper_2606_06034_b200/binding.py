@@ -72,7 +72,8 @@ def load_library() -> ctypes.CDLL:
     lib.gdn_chunk_prepare_int8.restype = ip
     lib.gdn_chunk_prepare_int8.argtypes = [vp, vp, vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ip, ip, ip, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.gdn_int8_lut_checksum.restype = ctypes.c_uint
-    lib.gdn_chunk_state_output.argtypes = [vp, vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ip, ctypes.c_float, vp, vp, vp, vp]
+    lib.gdn_chunk_state_output.argtypes = [vp, vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ip, ctypes.c_float, vp, vp, vp,
+                                           ctypes.c_uint, vp]
     lib.gdn_chunk_state_output.restype = ip
     lib.gdn_selftest_bounded_wait.argtypes = [vp]
     lib.gdn_selftest_bounded_wait.restype = ip
@@ -232,19 +233,21 @@ def chunk_prepare_int8(q, order=-1, residual_steps=-1, *, want_toff=True, output
     return outputs
 
 
-def gdn_chunk_state_output(Q, K, W_gated, U, g, B, H_k, H_v, T, C, d_k, d_v, scale, S_in, O_out, S_out, *, check=True):
+def gdn_chunk_state_output(Q, K, W_gated, U, g, B, H_k, H_v, T, C, d_k, d_v, scale, S_in, O_out, S_out, flags=0, *,
+                           check=True):
     """Raw call of the state-passing / output entry point (tensors instead of pointers, torch's current stream)."""
     for t in (Q, K, W_gated, U, g, S_in, O_out, S_out):
         if t is not None and (not t.is_cuda or not t.is_contiguous()):
             raise ValueError("all tensors must be contiguous CUDA tensors (there is no CPU path)")
     rc = load_library().gdn_chunk_state_output(_ptr(Q), _ptr(K), _ptr(W_gated), _ptr(U), _ptr(g), B, H_k, H_v, T, C, d_k, d_v,
-                                               ctypes.c_float(scale), _ptr(S_in), _ptr(O_out), _ptr(S_out), _stream())
+                                               ctypes.c_float(scale), _ptr(S_in), _ptr(O_out), _ptr(S_out), flags,
+                                               _stream())
     if check and rc != GDN_OK:
         raise GdnError(rc, "gdn_chunk_state_output")
     return rc
 
 
-def chunk_state_output(Q, K, W_gated, U, g, C, scale=1.0, S_in=None, *, want_state=True, outputs=None):
+def chunk_state_output(Q, K, W_gated, U, g, C, scale=1.0, S_in=None, *, want_state=True, outputs=None, flags=0):
     """Convenience wrapper: Q, K [B,H_k,T,d_k], W_gated [B,H_v,T,d_k], U [B,H_v,T,d_v], g [B,H_v,T] (chunk-local
     cumulative log-gate). Returns (O [B,H_v,T,d_v], S_out [B,H_v,d_v,d_k] fp32 or None)."""
     B, H_k, T, d_k = K.shape
@@ -254,7 +257,7 @@ def chunk_state_output(Q, K, W_gated, U, g, C, scale=1.0, S_in=None, *, want_sta
         S_out = torch.empty(B, H_v, d_v, d_k, dtype=torch.float32, device=U.device) if want_state else None
     else:
         O, S_out = outputs
-    gdn_chunk_state_output(Q, K, W_gated, U, g, B, H_k, H_v, T, C, d_k, d_v, scale, S_in, O, S_out)
+    gdn_chunk_state_output(Q, K, W_gated, U, g, B, H_k, H_v, T, C, d_k, d_v, scale, S_in, O, S_out, flags)
     return O, S_out
 
 

@@ -71,6 +71,7 @@ struct ParamsS {
     int* status;
     int H_k, H_v, T, group;
     float scale;
+    unsigned flags;  // GDN_FLAG_G_RAW: g holds raw log-gates, prefix-summed inside every chunk here
 };
 
 __device__ __forceinline__ float fast_exp2(float x) {
@@ -321,32 +322,42 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             mbar_arrive(&bar_rdy_a);
         }
         // gates of the first chunk
-        float g_reg = 0.f, gC_reg = 0.f;
-        if (n_c > 0) {
-            if (tid < 64) g_reg = __ldg(gseq + tid);
-            gC_reg = __ldg(gseq + kC - 1);
-        }
+        float g_reg = 0.f;
+        if (n_c > 0 && tid < 64) g_reg = __ldg(gseq + tid);
         bool ok = true;
         // gate tables of a chunk: written by 64 threads into the buffer of that chunk one barrier before they are read
+        const bool g_raw = (p.flags & GDN_FLAG_G_RAW) != 0;
         auto fill_tables = [&](int c) {
             if (tid < 64) {
                 float* tb = gtab + (c & 1) * 192;
-                tb[tid] = fast_exp2(g_reg * kLog2e);
-                tb[64 + tid] = fast_exp2((gC_reg - g_reg) * kLog2e);
-                tb[128 + tid] = g_reg;
+                float gc = g_reg;
+                if (g_raw) {
+                    // inclusive prefix sum over the chunk's 64 tokens: inside each of the two warps by shuffles ...
+#pragma unroll
+                    for (int off = 1; off < 32; off <<= 1) {
+                        const float v = __shfl_up_sync(0xFFFFFFFFu, gc, off);
+                        if (lane >= off) gc += v;
+                    }
+                    if (tid == 31) tb[128 + 63] = gc;  // ... and the first warp's total through the table itself
+                    asm volatile("bar.sync 3, 64;" ::: "memory");
+                    if (tid >= 32) gc += tb[128 + 63];
+                    asm volatile("bar.sync 3, 64;" ::: "memory");
+                }
+                tb[128 + tid] = gc;
+                asm volatile("bar.sync 3, 64;" ::: "memory");
+                const float gC = tb[128 + 63];  // cumulative gate of the chunk's last token
+                tb[tid] = fast_exp2(gc * kLog2e);
+                tb[64 + tid] = fast_exp2((gC - gc) * kLog2e);
             }
         };
         if (n_c > 0) fill_tables(0);
         asm volatile("bar.sync 1, 512;" ::: "memory");
         for (int c = 0; c < n_c; ++c) {
-            const float gC = gC_reg;
             const float* se = gtab + (c & 1) * 192;  // exp(g_i)
             const float* sf = se + 64;               // exp(g_C - g_j)
-            const float* sg = se + 128;              // g_i
-            if (c + 1 < n_c) {
-                if (tid < 64) g_reg = __ldg(gseq + (c + 1) * kC + tid);
-                gC_reg = __ldg(gseq + (c + 2) * kC - 1);
-            }
+            const float* sg = se + 128;              // g_i (cumulative inside the chunk)
+            const float gC = sg[63];
+            if (c + 1 < n_c && tid < 64) g_reg = __ldg(gseq + (c + 1) * kC + tid);
             STAMPS(1);
 
             STAMPS(2);
@@ -567,6 +578,7 @@ int launch_chunk_state(const ProblemS& q, cudaStream_t stream) {
     prm.T = q.T;
     prm.group = q.H_v / q.H_k;
     prm.scale = q.scale;
+    prm.flags = q.flags;
     const int smem = kSmemTotal + 1024;
     if (cudaFuncSetAttribute(chunk_state_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
         return GDN_ERR_LAUNCH;

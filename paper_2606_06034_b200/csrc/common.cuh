@@ -55,6 +55,7 @@ struct ProblemS {
     float* S_out;       // may be null
     int B, H_k, H_v, T, C, d_k, d_v;
     float scale;
+    unsigned flags;
 };
 
 enum InverseMode { INV_NEUMANN = 0, INV_FWDSUBST_ROWS = 1, INV_FWDSUBST_BLOCKED = 2 };

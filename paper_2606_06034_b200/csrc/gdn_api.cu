@@ -151,7 +151,8 @@ int gdn_chunk_prepare_int8(const int8_t* Kq, const int8_t* Vq, const int32_t* k_
 
 int gdn_chunk_state_output(const void* Q, const void* K, const void* W_gated, const void* U, const float* g, int B, int H_k,
                            int H_v, int T, int C, int d_k, int d_v, float scale, const float* S_in, void* O_out, float* S_out,
-                           gdn_stream_t stream) {
+                           unsigned flags, gdn_stream_t stream) {
+    if (flags & ~static_cast<unsigned>(GDN_FLAG_G_RAW)) return GDN_ERR_INVALID_ARG;
     if (Q == nullptr || K == nullptr || W_gated == nullptr || U == nullptr || g == nullptr || O_out == nullptr) return GDN_ERR_NULL;
     if (B < 0 || H_k <= 0 || H_v <= 0 || T < 0 || C < 2 || d_k <= 0 || d_v <= 0) return GDN_ERR_INVALID_ARG;
     if (H_v % H_k != 0 || T % C != 0) return GDN_ERR_INVALID_ARG;
@@ -160,7 +161,7 @@ int gdn_chunk_state_output(const void* Q, const void* K, const void* W_gated, co
         return GDN_ERR_ALIGN;
     const int rc = check_arch();
     if (rc != GDN_OK) return rc;
-    ProblemS q{Q, K, W_gated, U, g, S_in, O_out, S_out, B, H_k, H_v, T, C, d_k, d_v, scale};
+    ProblemS q{Q, K, W_gated, U, g, S_in, O_out, S_out, B, H_k, H_v, T, C, d_k, d_v, scale, flags};
     return launch_chunk_state(q, static_cast<cudaStream_t>(stream));
 }
 

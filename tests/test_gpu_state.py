@@ -79,15 +79,41 @@ def test_whole_layer_matches_the_token_recurrence():
         assert eS.max() <= 1e-2, f"S rel-F {eS.max():.3e}"
 
 
+def test_whole_layer_from_raw_gates_and_unnormalised_keys():
+    """Both calls with the raw per-token log-gates (prefix sums formed inside the kernels) and the key normalisation
+    fused into the first call, against the token-by-token rule on the normalised keys."""
+    C, T = 64, 384
+    inp = gen.make_inputs(1, 1, 2, T, C, 128, 128, seed=412)
+    Q = _queries(inp, 413)
+    scale = 128 ** -0.5
+    graw = inp.g.view(1, 2, T // C, C).diff(dim=-1, prepend=torch.zeros(1, 2, T // C, 1)).reshape(1, 2, T).contiguous()
+    Kun = (inp.K.float() * 1.7).to(torch.bfloat16)  # unnormalised keys; the kernel normalises them for A, W
+    flags = gdn.GDN_FLAG_W_GATED | gdn.GDN_FLAG_G_RAW | gdn.GDN_FLAG_K_L2NORM
+    W, U, _ = gdn.chunk_prepare(Kun.cuda(), inp.V.cuda(), inp.beta.cuda(), graw.cuda(), C, flags=flags)
+    Kn = Kun.double() / Kun.double().norm(dim=-1, keepdim=True)
+    # the state kernel multiplies by the keys it is given: the normalised ones, rounded to bf16 as a model would
+    Kn16 = Kn.to(torch.bfloat16)
+    O, S = gdn.chunk_state_output(Q.cuda(), Kn16.cuda(), W, U, graw.cuda(), C, scale, flags=gdn.GDN_FLAG_G_RAW)
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+    for hv in range(2):
+        Oo, So = orc.gated_delta_rule(Q[0, 0].double().numpy(), Kn[0, 0].numpy(), inp.V[0, hv].double().numpy(),
+                                      inp.beta[0, hv].double().numpy(), graw[0, hv].double().numpy(), scale)
+        eO = orc.rel_frobenius(O[0, hv].double().cpu().numpy().reshape(T // C, C, 128), Oo.reshape(T // C, C, 128))
+        assert eO.max() <= 1e-2, f"O rel-F {eO.max():.3e} at chunk {eO.argmax()}"
+        eS = orc.rel_frobenius(S[0, hv].double().cpu().numpy()[None], So[None])
+        assert eS.max() <= 1e-2, f"S rel-F {eS.max():.3e}"
+
+
 def test_state_output_argument_errors():
     inp = gen.make_inputs(1, 1, 1, 128, 64, 128, 128, seed=420)
     K = inp.K.cuda()
     g = inp.g.cuda()
     O = torch.empty(1, 1, 128, 128, dtype=torch.bfloat16, device="cuda")
     args = dict(check=False)
-    assert gdn.gdn_chunk_state_output(K, K, K, K, g, 1, 1, 1, 128, 32, 128, 128, 1.0, None, O, None, **args) == gdn.GDN_ERR_UNSUPPORTED
-    assert gdn.gdn_chunk_state_output(K, K, K, K, g, 1, 1, 1, 100, 64, 128, 128, 1.0, None, O, None, **args) == gdn.GDN_ERR_INVALID_ARG
-    assert gdn.gdn_chunk_state_output(None, K, K, K, g, 1, 1, 1, 128, 64, 128, 128, 1.0, None, O, None, **args) == gdn.GDN_ERR_NULL
+    assert gdn.gdn_chunk_state_output(K, K, K, K, g, 1, 1, 1, 128, 32, 128, 128, 1.0, None, O, None, 0, **args) == gdn.GDN_ERR_UNSUPPORTED
+    assert gdn.gdn_chunk_state_output(K, K, K, K, g, 1, 1, 1, 100, 64, 128, 128, 1.0, None, O, None, 0, **args) == gdn.GDN_ERR_INVALID_ARG
+    assert gdn.gdn_chunk_state_output(None, K, K, K, g, 1, 1, 1, 128, 64, 128, 128, 1.0, None, O, None, 0, **args) == gdn.GDN_ERR_NULL
+    assert gdn.gdn_chunk_state_output(K, K, K, K, g, 1, 1, 1, 128, 64, 128, 128, 1.0, None, O, None, 2, **args) == gdn.GDN_ERR_INVALID_ARG
     assert gdn.gdn_device_status() == gdn.GDN_OK
 
 
