@@ -50,6 +50,41 @@ def algorithmic_bytes_per_chunk(C: int, d_k: int, d_v: int, group: int, esize: i
     return (C * d_k * esize) / group + C * d_v * esize + C * d_k * esize + C * d_v * esize + C * C * esize + 8 * C
 
 
+def int8_integer_ops_per_chunk(C: int, d_k: int, d_v: int, N: int, S: int) -> float:
+    """32-bit integer ALU operations the INT8 variant needs per chunk outside the tensor-core products, counted from
+    its definition (one op = one add, shift, logic op, min/max, compare/select or multiply on one element):
+    a requantisation costs 7 per element of its support (magnitude, running maximum, rounding add, sign fix,
+    shift, two clamps), an aligned sum 2 per term and element (shift, add), the gate factor 11 per strictly lower
+    entry (difference, table index, shift count, look-up, shift, range test, beta product, rounding add, shift,
+    and the two-word product with the Gram entry), the band products and A T0, T0 S (banded operand) one
+    multiply-add per term."""
+    lower = C * (C - 1) // 2
+    band = sum(C - d for d in range(1, N + 1))
+    far = lower - band
+    sup = lambda m: (C - m) * (C - m + 1) // 2 if m < C else 0  # entries with i - j >= m
+    ops = 11 * lower + 7 * lower                                    # gate factor, A
+    for n in range(2, N + 1):                                       # band powers
+        ops += sum((d - 1) * (C - d) for d in range(n, N + 1)) + 7 * sum(C - d for d in range(n, N + 1))
+    ops += 2 * N * band + 7 * band                                  # T0
+    ops += N * far + 2 * 2 * far + 7 * far                          # E
+    terms = far
+    for s_ in range(2, S + 1):                                      # powers of E (products on the tensor cores)
+        if s_ * (N + 1) >= C:
+            break
+        ops += 7 * sup(s_ * (N + 1))
+        terms += sup(s_ * (N + 1))
+    ops += 2 * terms + 7 * far                                      # sum of the powers
+    ops += N * far + 2 * (band + 2 * far) + 7 * lower               # T - I
+    ops += 8 * lower                                                # T diag(beta)
+    ops += (1 + 4 + 7) * C * (d_k + d_v)                            # W, U: diagonal term, aligned sum, requantisation
+    return float(ops)
+
+
+# integer ALU peak: 148 SMs x 4 sub-partitions x one 16-lane integer pipe each x the maximum SM clock
+INT_ALU_LANES = 148 * 4 * 16
+SM_MAX_GHZ = 1.965
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -257,6 +292,15 @@ def run_ours(args, rank, world, dist_ctx):
                 "effective_tflops": n_chunks * flops_chunk / (launch_ms * 1e-3) / 1e12,
                 "tensor_time_frac_of_bf16_peak": (n_chunks * flops_chunk / (launch_ms * 1e-3) / 1e12) / bf16_peak}
 
+    if method == "int8":
+        # DRAM runs at a few per cent and the tensor pipe at 5 %: the variant is bound by the integer arithmetic between
+        # the products (ncu: integer pipe 65 % busy), so that is the roofline it is reported against
+        ops = int8_integer_ops_per_chunk(C, inp.d_k, inp.d_v, gdn.gdn_default_order(C), gdn.gdn_default_residual_steps(C))
+        alu_peak = INT_ALU_LANES * SM_MAX_GHZ / 1e3  # Tiop/s
+        alu = n_chunks * ops / (launch_ms * 1e-3) / 1e12
+        roofline.update({"bound": "alu", "achieved": alu, "peak": alu_peak, "unit": "Tiop/s", "frac": alu / alu_peak,
+                         "peak_kind": "derived: 148 SMs x 64 integer lanes x 1.965 GHz",
+                         "algorithmic_int_ops_per_chunk": ops, "hbm_frac": achieved / hbm_peak, "hbm_gbs": achieved})
     per_sorted = sorted(per)
     roofline["launch_us"] = {"mean": launch_ms * 1e3, "median": per_sorted[len(per_sorted) // 2] * 1e3, "best": per_sorted[0] * 1e3}
     line = {
@@ -392,8 +436,10 @@ def run_extras(gdn, gen, dev, args):
         ms = total_ms / 10
         group = inp.H_v // inp.H_k
         by = inp.C * inp.d_k / group + inp.C * inp.d_v + inp.C * inp.d_k + inp.C * inp.d_v + inp.C * inp.C + 6 * inp.C
+        ops = int8_integer_ops_per_chunk(q.C, q.d_k, q.d_v, gdn.gdn_default_order(q.C), gdn.gdn_default_residual_steps(q.C))
         out["prefill_gqa:int8"] = {"chunks_per_s": q.n_chunks / (ms * 1e-3), "ms": ms,
-                                   "hbm_frac": q.n_chunks * by / (ms * 1e-3) / 1e9 / hbm_peak}
+                                   "hbm_frac": q.n_chunks * by / (ms * 1e-3) / 1e9 / hbm_peak,
+                                   "int_alu_frac": q.n_chunks * ops / (ms * 1e-3) / (INT_ALU_LANES * SM_MAX_GHZ * 1e9)}
         del inp, q, outs
     except Exception as exc:
         out["prefill_gqa:int8"] = {"error": repr(exc)}
