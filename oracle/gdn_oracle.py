@@ -306,6 +306,51 @@ def chunk_prepare(K, V, beta, g, N: int | None = None, S: int | None = None, *,
     return W, U, T
 
 
+def chunk_table(cu_seqlens, C: int):
+    """Chunks of packed variable-length sequences: sequence s holds tokens [cu_seqlens[s], cu_seqlens[s+1]) and is cut
+    into chunks of C tokens from its own first token; its last chunk may be shorter. Returns (start, length) lists."""
+    start, length = [], []
+    for s in range(len(cu_seqlens) - 1):
+        a, b = int(cu_seqlens[s]), int(cu_seqlens[s + 1])
+        assert b >= a
+        for t0 in range(a, b, C):
+            start.append(t0)
+            length.append(min(C, b - t0))
+    return start, length
+
+
+def chunk_prepare_varlen(K, V, beta, g, cu_seqlens, C: int, N: int | None = None, S: int | None = None, *,
+                         exact: bool = False, g_raw: bool = False, k_l2norm: bool = False, w_gated: bool = False):
+    """One head of packed variable-length sequences: K [T, d_k], V [T, d_v], beta, g [T] (g: cumulative log-gate
+    restarting in every chunk, chunks counted from each sequence's first token; or raw with g_raw).
+
+    A chunk shorter than C is the chunk of C tokens whose missing tokens write nothing: beta = 0, zero key and
+    value, no further decay (raw log-gate 0, i.e. the cumulative gate of the last real token). The scheme of
+    `chunk_prepare` is applied to that padded chunk and the rows of the real tokens are kept.
+    Returns (W [T, d_k], U [T, d_v], Tinv [n_chunks, C, C], start, length).
+    """
+    K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64)
+    beta = np.asarray(beta, dtype=np.float64)
+    g = np.asarray(g, dtype=np.float64)
+    if k_l2norm:
+        K = K / np.sqrt((K * K).sum(axis=-1, keepdims=True))
+    start, length = chunk_table(cu_seqlens, C)
+    W = np.zeros_like(K)
+    U = np.zeros_like(V)
+    Tinv = np.zeros((len(start), C, C))
+    for c, (a, L) in enumerate(zip(start, length)):
+        Kc = np.zeros((C, K.shape[1])); Vc = np.zeros((C, V.shape[1])); bc = np.zeros(C); gc = np.zeros(C)
+        Kc[:L] = K[a:a + L]; Vc[:L] = V[a:a + L]; bc[:L] = beta[a:a + L]; gc[:L] = g[a:a + L]
+        if not g_raw:
+            gc[L:] = gc[L - 1]
+        Wc, Uc, Tc = chunk_prepare(Kc, Vc, bc, gc, N, S, exact=exact, g_raw=g_raw, w_gated=w_gated)
+        W[a:a + L] = Wc[:L]
+        U[a:a + L] = Uc[:L]
+        Tinv[c] = Tc
+    return W, U, Tinv, start, length
+
+
 # ----------------------------------------------------------------------------
 # The rest of the chunk-wise layer: state passing and output, given W and U
 # ----------------------------------------------------------------------------

@@ -135,6 +135,62 @@ def test_chunkwise_state_passing_and_output_equal_the_token_recurrence():
     assert not np.allclose(O_bad2, O_ref, atol=1e-6)
 
 
+def test_variable_length_sequences_equal_the_token_recurrence_per_sequence():
+    """Packed sequences of ragged lengths: the chunk quantities of `chunk_prepare_varlen` (chunks counted from each
+    sequence's first token, the last one short) carried through the chunk-wise state passing reproduce the
+    token-by-token gated delta rule run on every sequence by itself; the padding tokens of a short chunk leave the
+    state alone. Also pinned: the chunk table, and that the rows of real tokens do not depend on what a padded
+    chunk holds beyond its length."""
+    rng = np.random.default_rng(21)
+    C, dk, dv = 8, 5, 6
+    lens = [13, 8, 3, 17]
+    cu = np.concatenate([[0], np.cumsum(lens)])
+    T = int(cu[-1])
+    start, length = orc.chunk_table(cu, C)
+    assert start == [0, 8, 13, 21, 24, 32, 40] and length == [8, 5, 8, 3, 8, 8, 1]
+    K = rng.normal(size=(T, dk))
+    K /= np.linalg.norm(K, axis=1, keepdims=True)
+    Q = rng.normal(size=(T, dk))
+    V = rng.normal(size=(T, dv))
+    beta = 1 / (1 + np.exp(-rng.normal(size=T)))
+    graw = -np.log1p(np.exp(rng.normal(size=T)))
+    g_local = np.zeros(T)
+    for a, L in zip(start, length):
+        g_local[a:a + L] = np.cumsum(graw[a:a + L])
+    W, U, Tinv, st2, ln2 = orc.chunk_prepare_varlen(K, V, beta, g_local, cu, C, exact=True, w_gated=True)
+    assert st2 == start and ln2 == length
+    Wr, Ur, Tr, _, _ = orc.chunk_prepare_varlen(K, V, beta, graw, cu, C, exact=True, w_gated=True, g_raw=True)
+    assert np.allclose(Wr, W, atol=1e-13) and np.allclose(Ur, U, atol=1e-13) and np.allclose(Tr, Tinv, atol=1e-13)
+    ci = 0
+    for s_, L in enumerate(lens):
+        a = int(cu[s_])
+        O_ref, S_ref = orc.gated_delta_rule(Q[a:a + L], K[a:a + L], V[a:a + L], beta[a:a + L], graw[a:a + L], scale=0.9)
+        # the sequence padded to whole chunks: padding rows carry zero W, U, K and the gate of the last real token
+        n_c = -(-L // C)
+        Lp = n_c * C
+        pad = lambda x: np.concatenate([x[a:a + L], np.zeros((Lp - L,) + x.shape[1:])])
+        gp = pad(g_local)
+        if Lp > L:
+            gp[L:] = g_local[a + L - 1]
+        O, S = orc.chunk_state_output(pad(Q), pad(K), pad(W), pad(U), gp, C, scale=0.9)
+        assert np.allclose(O[:L], O_ref, atol=1e-12) and np.allclose(S, S_ref, atol=1e-12)
+        for c in range(n_c):
+            Lc = length[ci]
+            # rows of padding tokens are rows of the identity, real rows never look at padding columns
+            assert np.array_equal(Tinv[ci][Lc:], np.eye(C)[Lc:])
+            assert np.count_nonzero(Tinv[ci][:Lc, Lc:]) == 0
+            # the leading block is the exact inverse of the short chunk itself
+            A = orc.build_A(K[start[ci]:start[ci] + Lc], beta[start[ci]:start[ci] + Lc], g_local[start[ci]:start[ci] + Lc])
+            assert np.allclose(Tinv[ci][:Lc, :Lc], np.linalg.inv(np.eye(Lc) + A), atol=1e-12)
+            ci += 1
+    # lengths that are multiples of C: the packed form is the dense one
+    cu2 = [0, 16, 24]
+    Wd, Ud, Td, _, _ = orc.chunk_prepare_varlen(K[:24], V[:24], beta[:24], graw[:24], cu2, C, 3, 2, g_raw=True)
+    Wc, Uc, Tc = orc.chunk_prepare(K[:24].reshape(3, C, dk), V[:24].reshape(3, C, dv), beta[:24].reshape(3, C),
+                                   graw[:24].reshape(3, C), 3, 2, g_raw=True)
+    assert np.array_equal(Wd, Wc.reshape(24, dk)) and np.array_equal(Ud, Uc.reshape(24, dv)) and np.array_equal(Td, Tc)
+
+
 # -- P2 / P12: exact inverse -----------------------------------------------------
 def test_forward_substitution_closed_forms_c2_c3():
     a = 0.37
