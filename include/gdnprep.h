@@ -147,6 +147,27 @@ int gdn_chunk_prepare_int8(const int8_t* Kq, const int8_t* Vq, const int32_t* k_
                            int8_t* Toff_q_out, int32_t* t_exp_out, int32_t* dbg_acc_out, gdn_stream_t stream);
 
 /*
+ * gdn_chunk_prepare_ex for packed variable-length sequences (one batch of sequences laid end to end along the token
+ * axis, as model code passes them with cumulative sequence lengths). Every sequence is cut into chunks of C tokens from
+ * its own first token; its last chunk may be shorter. A short chunk is the chunk of C tokens whose missing tokens
+ * write nothing (beta = 0, no further decay): the scheme of Sec. 3 runs on it unchanged and only the rows of real
+ * tokens are stored.
+ *   K [H_k,T_total,d_k], V [H_v,T_total,d_v], beta, g [H_v,T_total], W_out [H_v,T_total,d_k], U_out [H_v,T_total,d_v]
+ *   (bf16; or token-major [T_total,H,d] and [T_total,H_v] with GDN_FLAG_LAYOUT_BTHD); g restarts in every chunk (or raw
+ *   log-gates with GDN_FLAG_G_RAW).
+ *   chunk_start, chunk_len: DEVICE arrays of n_chunks int32: first token and length (1..C) of every chunk, in any
+ *   order; chunks must not overlap.
+ *   Tinv_out (optional) [H_v, P, C, C] bf16 with P = n_chunks rounded up to a multiple of 128 / C: block c belongs to
+ *   chunk c of the table; rows of missing tokens are rows of the identity, blocks c >= n_chunks are identities.
+ * flags: GDN_FLAG_G_RAW, GDN_FLAG_K_L2NORM, GDN_FLAG_W_GATED, GDN_FLAG_LAYOUT_BTHD. bf16 only, C in {16, 32, 64, 128},
+ * d_k = d_v = 128. Rows of W_out / U_out that no chunk covers are left untouched.
+ */
+int gdn_chunk_prepare_varlen(const void* K, const void* V, const float* beta, const float* g,
+                             const int32_t* chunk_start, const int32_t* chunk_len, int n_chunks, int T_total,
+                             int H_k, int H_v, int C, int d_k, int d_v, int order, int residual_steps,
+                             void* W_out, void* U_out, void* Tinv_out, unsigned flags, gdn_stream_t stream);
+
+/*
  * The rest of the chunk-wise layer (Sec. 2.1: the quantities W and U exist for this), given W and U of every chunk:
  * state passing between chunks and the output. Per (batch, value head), chunk after chunk, with S the state
  * [d_v x d_k] carried from chunk to chunk:

@@ -34,7 +34,8 @@ GDN_FWDSUBST_ROWS = 0
 GDN_FWDSUBST_BLOCKED = 1
 
 EXPORTS = (
-    "gdn_chunk_prepare", "gdn_chunk_prepare_gqa", "gdn_chunk_prepare_ex", "gdn_chunk_prepare_fwdsubst",
+    "gdn_chunk_prepare", "gdn_chunk_prepare_gqa", "gdn_chunk_prepare_ex", "gdn_chunk_prepare_varlen",
+    "gdn_chunk_prepare_fwdsubst",
     "gdn_chunk_prepare_int8", "gdn_chunk_state_output", "gdn_selftest_bounded_wait",
     "gdn_int8_lut_checksum",
     "gdn_device_status", "gdn_default_order", "gdn_default_residual_steps",
@@ -67,6 +68,8 @@ def load_library() -> ctypes.CDLL:
     lib.gdn_chunk_prepare_gqa.argtypes = [vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ip, ip, ip, ip, vp, vp, vp, vp]
     lib.gdn_chunk_prepare_ex.restype = ip
     lib.gdn_chunk_prepare_ex.argtypes = [vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ip, ip, ip, ip, vp, vp, vp, ctypes.c_uint, vp]
+    lib.gdn_chunk_prepare_varlen.restype = ip
+    lib.gdn_chunk_prepare_varlen.argtypes = [vp, vp, vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ip, ip, ip, vp, vp, vp, ctypes.c_uint, vp]
     lib.gdn_chunk_prepare_fwdsubst.restype = ip
     lib.gdn_chunk_prepare_fwdsubst.argtypes = [vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ip, ip, ip, vp, vp, vp, vp]
     lib.gdn_chunk_prepare_int8.restype = ip
@@ -179,6 +182,58 @@ def gdn_chunk_prepare_ex(K, V, beta, g, B, H_k, H_v, T, C, d_k, d_v, order, resi
     if check and rc != GDN_OK:
         raise GdnError(rc, "gdn_chunk_prepare_ex")
     return rc
+
+
+def gdn_chunk_prepare_varlen(K, V, beta, g, chunk_start, chunk_len, n_chunks, T_total, H_k, H_v, C, d_k, d_v, order,
+                             residual_steps, W_out, U_out, Tinv_out, flags, *, check=True):
+    _check_inputs(K, V, beta, g, (W_out, U_out, Tinv_out))
+    for t in (chunk_start, chunk_len):
+        if t is not None and (not t.is_cuda or not t.is_contiguous() or t.dtype != torch.int32):
+            raise TypeError("chunk_start and chunk_len are contiguous int32 CUDA tensors")
+    rc = load_library().gdn_chunk_prepare_varlen(_ptr(K), _ptr(V), _ptr(beta), _ptr(g), _ptr(chunk_start), _ptr(chunk_len),
+                                                 n_chunks, T_total, H_k, H_v, C, d_k, d_v, order, residual_steps,
+                                                 _ptr(W_out), _ptr(U_out), _ptr(Tinv_out), int(flags), _stream())
+    if check and rc != GDN_OK:
+        raise GdnError(rc, "gdn_chunk_prepare_varlen")
+    return rc
+
+
+def chunk_table(cu_seqlens, C):
+    """First token and length of every chunk of packed sequences (host lists): sequence s holds the tokens
+    [cu_seqlens[s], cu_seqlens[s + 1]) and is cut into chunks of C tokens from its own start."""
+    bounds = [int(x) for x in cu_seqlens]
+    start, length = [], []
+    for a, b in zip(bounds[:-1], bounds[1:]):
+        if b < a:
+            raise ValueError("cu_seqlens must be non-decreasing")
+        n_full, rest = divmod(b - a, C)
+        start += [a + i * C for i in range(n_full + (1 if rest else 0))]
+        length += [C] * n_full + ([rest] if rest else [])
+    return start, length
+
+
+def chunk_prepare_varlen(K, V, beta, g, cu_seqlens, C, order=-1, residual_steps=-1, *, want_tinv=True, flags=0):
+    """Packed variable-length sequences: K [H_k,T,d_k], V [H_v,T,d_v], beta, g [H_v,T] (with GDN_FLAG_LAYOUT_BTHD:
+    [T,H,d] and [T,H_v]), cu_seqlens = the sequence boundaries on the host. Returns (W, U, Tinv [H_v,n_chunks,C,C] or
+    None, chunk_start, chunk_len) with the chunk table as int32 CUDA tensors."""
+    token_major = bool(flags & GDN_FLAG_LAYOUT_BTHD)
+    if token_major:
+        T, H_k, d_k = K.shape
+        _, H_v, d_v = V.shape
+    else:
+        H_k, T, d_k = K.shape
+        H_v, _, d_v = V.shape
+    start, length = chunk_table(cu_seqlens, C)
+    n = len(start)
+    cs = torch.tensor(start, dtype=torch.int32, device=K.device)
+    cl = torch.tensor(length, dtype=torch.int32, device=K.device)
+    per_tile = max(1, 128 // C)
+    padded = -(-n // per_tile) * per_tile
+    W = torch.zeros((T, H_v, d_k) if token_major else (H_v, T, d_k), dtype=K.dtype, device=K.device)
+    U = torch.zeros_like(V)
+    Tinv = torch.empty(H_v, padded, C, C, dtype=K.dtype, device=K.device) if want_tinv else None
+    gdn_chunk_prepare_varlen(K, V, beta, g, cs, cl, n, T, H_k, H_v, C, d_k, d_v, order, residual_steps, W, U, Tinv, flags)
+    return W, U, (Tinv[:, :n] if want_tinv else None), cs, cl
 
 
 def gdn_chunk_prepare_fwdsubst(K, V, beta, g, B, H_k, H_v, T, C, d_k, d_v, dtype, variant, W_out, U_out, Tinv_out,

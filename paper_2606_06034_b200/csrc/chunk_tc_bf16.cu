@@ -52,6 +52,8 @@ __device__ long long g_trace[4096];
 #define STAMP(slot) do { } while (0)
 #endif
 
+// (New fields go at the END: the struct's layout decides which parameters ptxas fetches with one wide load, and a
+// field inserted in the middle moved the default instantiation from 36 to 96 bytes of spill, 10 % of its speed.)
 struct Params {
     const float* beta;
     const float* g;
@@ -63,7 +65,13 @@ struct Params {
     int N, S;
     unsigned flags;  // GDN_FLAG_*
     long long n_tiles;
+    // packed variable-length sequences (EX instantiations only, B = 1): first token and length of every chunk; T is
+    // then the padded token count n_tt * 128 and T_total the real one
+    const int* chunk_start;
+    const int* chunk_len;
+    int n_chunks, T_total;
     int s_gi, s_tt, s_bhk;  // the grid size as a step in (value head of the group, token tile, key-head row) digits
+    int n_mid;  // EX instantiations: range of the middle digit of the tile walk, n_tt (head-major tensors) or H_k (token-major)
 };
 
 template <int C, int NB>
@@ -357,36 +365,45 @@ struct TileCoord {
 struct TilePos {
     int gi, tt, bhk;
 };
+template <int EX>
 __device__ __forceinline__ TilePos tile_pos(uint32_t tile, const Params& p) {
     TilePos c;
+    const int n_mid = EX ? p.n_mid : p.n_tt;
     const uint32_t y = tile / static_cast<uint32_t>(p.group);
     c.gi = static_cast<int>(tile - y * p.group);
-    c.bhk = static_cast<int>(y / static_cast<uint32_t>(p.n_tt));
-    c.tt = static_cast<int>(y - static_cast<uint32_t>(c.bhk) * p.n_tt);
+    c.bhk = static_cast<int>(y / static_cast<uint32_t>(n_mid));
+    c.tt = static_cast<int>(y - static_cast<uint32_t>(c.bhk) * n_mid);
     return c;
 }
+template <int EX>
 __device__ __forceinline__ void tile_advance(TilePos& c, const Params& p) {
+    const int n_mid = EX ? p.n_mid : p.n_tt;
     c.gi += p.s_gi;
     const int c1 = (c.gi >= p.group) ? 1 : 0;
     c.gi -= c1 ? p.group : 0;
     c.tt += p.s_tt + c1;
-    const int c2 = (c.tt >= p.n_tt) ? 1 : 0;
-    c.tt -= c2 ? p.n_tt : 0;
+    const int c2 = (c.tt >= n_mid) ? 1 : 0;
+    c.tt -= c2 ? n_mid : 0;
     c.bhk += p.s_bhk + c2;
 }
 // (key head row, value head row, first token): value head row = bhk * group + gi because H_v = H_k * group.
 // Head-major tensors [B, H, T, d] are seen by TMA as (d, T, B * H); token-major ones [B, T, H, d]
 // (GDN_FLAG_LAYOUT_BTHD, only in the EX instantiations) as (H * d, T, B), the head selecting a column range.
-template <bool EX>
+// There the walk is (value head of the group, key head, batch * n_tt + token tile) instead, so that the CTAs running
+// at one time read all heads of the same tokens: a token's heads are contiguous in memory.
+template <int EX>
 __device__ __forceinline__ TileCoord tile_coord(const TilePos& c, const Params& p) {
     TileCoord r;
     r.bhk = c.bhk;
     r.bhv = c.bhk * p.group + c.gi;
     r.t0 = c.tt * kTile;
     if (EX && (p.flags & GDN_FLAG_LAYOUT_BTHD)) {
-        const int b = c.bhk / p.H_k;
-        const int hk = c.bhk - b * p.H_k;
+        const int hk = c.tt;
+        const int b = c.bhk / p.n_tt;
         const int hv = hk * p.group + c.gi;
+        r.bhk = b * p.H_k + hk;
+        r.bhv = b * p.H_v + hv;
+        r.t0 = (c.bhk - b * p.n_tt) * kTile;
         r.kx = hk * kD;
         r.kz = b;
         r.vx = hv * kD;
@@ -408,10 +425,11 @@ __device__ __forceinline__ TileCoord tile_coord(const TilePos& c, const Params& 
 // (C = 64 is then the block size) and whose lower-left block follows from App. E, Eq. 28:
 // T21 = -T22 A21 T11, evaluated as Y = A21 + A21 X11, T21 = -(Y + X22 Y) with X = T - I of the blocks, so that
 // the identity parts stay in fp32 and only the small products pass through bf16 operands.
-// EX: the optional prologue / fp32 outputs of gdn_chunk_prepare_ex are compiled in (flags read at run time).
+// EX: 1 = the optional prologue, layouts and packed sequences of gdn_chunk_prepare_ex / _varlen are compiled in (flags
+// read at run time); 2 = also the fp32 outputs (parity debugging; they cost registers, so they have their own code).
 // DBL: 8 or 15 = the residual sum for that S is evaluated by the four-level doubling scheme (C = 64 only); 0 = one
 // product per term.
-template <int C, int NB, int MODE, bool MERGE, bool EX, int DBL>
+template <int C, int NB, int MODE, bool MERGE, int EX, int DBL>
 __global__ void __launch_bounds__(kThreads, 2)
 chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                 const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmU,
@@ -442,7 +460,9 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     const bool f_l2 = EX && (p.flags & GDN_FLAG_K_L2NORM) != 0;
     const bool f_wg = EX && (p.flags & GDN_FLAG_W_GATED) != 0;
     const bool two_scales = f_l2 || f_wg;  // the W operand is scaled by something other than beta
-    const bool f_f32 = EX && (p.flags & GDN_FLAG_OUT_FP32) != 0;
+    const bool f_f32 = EX == 2 && (p.flags & GDN_FLAG_OUT_FP32) != 0;
+    const bool f_var = EX && p.chunk_start != nullptr;
+    constexpr int CR = MERGE ? kTile : C;  // tokens of a chunk
 
     __shared__ uint64_t bar_k, bar_v, bar_mma;
     __shared__ uint32_t tmem_base_s;
@@ -530,36 +550,77 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         for (int i = 0; i < PCH; ++i) keep[i] = 0u;
     }
 
-    TilePos pos_next = tile_pos(blockIdx.x, p);  // position of the tile after the one being worked on
+    // K (or V) rows of a tile: one box of 128 tokens per 64-column half, or, with variable-length sequences, one box
+    // per chunk from the chunk's own first token (rows past its length belong to the next sequence or are filled
+    // with zeros past the end of the tensor: beta = 0 below keeps them out of every result)
+    auto load_tile = [&](uint8_t* dst, const CUtensorMap* tm, uint64_t* bar, int x, int t0, int z) {
+        mbar_arrive_expect_tx(bar, 32768);
+        if (EX && f_var) {
+            const int cid0 = (t0 / kTile) * (kTile / CR);
+#pragma unroll 1
+            for (int m = 0; m < kTile / CR; ++m) {
+                const int st = (cid0 + m < p.n_chunks) ? __ldg(p.chunk_start + cid0 + m) : 0;
+                tma_load_3d(dst + m * (CR * 128), tm, bar, x, st, z);
+                tma_load_3d(dst + 16384 + m * (CR * 128), tm, bar, x + 64, st, z);
+            }
+        } else {
+            tma_load_3d(dst, tm, bar, x, t0, z);
+            tma_load_3d(dst + 16384, tm, bar, x + 64, t0, z);
+        }
+    };
+    // beta and g of this thread's row of a tile, and (variable-length sequences) the row's token in the packed
+    // tensors, -1 for a row past its chunk's length: such a row has beta = 0 and the gate of the chunk's last token
+    auto fetch_row = [&](const TilePos& pos, float& b_out, float& g_out, int& tok_out) {
+        const TileCoord c = tile_coord<EX>(pos, p);
+        b_out = 0.f;
+        g_out = 0.f;
+        tok_out = -1;
+        if (EX && f_var) {
+            const int cid = (c.t0 / kTile) * (kTile / CR) + t / CR;
+            const int r = t % CR;
+            int st = 0, len = 0;
+            if (cid < p.n_chunks) {
+                st = __ldg(p.chunk_start + cid);
+                len = __ldg(p.chunk_len + cid);
+            }
+            const bool bthd = (p.flags & GDN_FLAG_LAYOUT_BTHD) != 0;
+            const long long base = bthd ? c.bhv : (long long)c.bhv * p.T_total;
+            const long long stride = bthd ? p.H_v : 1;
+            if (r < len) {
+                tok_out = st + r;
+                const long long row = base + (long long)tok_out * stride;
+                b_out = __ldg(p.beta + row);
+                g_out = __ldg(p.g + row);
+            } else if (len > 0 && !f_graw) {
+                g_out = __ldg(p.g + base + (long long)(st + len - 1) * stride);
+            }
+        } else if (c.t0 + t < p.T) {
+            const long long r = c.r0 + (long long)t * c.rs;
+            b_out = __ldg(p.beta + r);
+            g_out = __ldg(p.g + r);
+        }
+    };
+    TilePos pos_next = tile_pos<EX>(blockIdx.x, p);  // position of the tile after the one being worked on
     if (tid == 0 && blockIdx.x < n_tiles) {
         const TileCoord c = tile_coord<EX>(pos_next, p);
-        mbar_arrive_expect_tx(&bar_k, 32768);
-        tma_load_3d(sK, &tmK, &bar_k, c.kx, c.t0, c.kz);
-        tma_load_3d(sK + 16384, &tmK, &bar_k, c.kx + 64, c.t0, c.kz);
-        mbar_arrive_expect_tx(&bar_v, 32768);
-        tma_load_3d(sV, &tmV, &bar_v, c.vx, c.t0, c.vz);
-        tma_load_3d(sV + 16384, &tmV, &bar_v, c.vx + 64, c.t0, c.vz);
+        load_tile(sK, &tmK, &bar_k, c.kx, c.t0, c.kz);
+        load_tile(sV, &tmV, &bar_v, c.vx, c.t0, c.vz);
     }
     // beta and g of the row are fetched one tile ahead
     float bi_next = 0.f, gi_next = 0.f;
-    if (blockIdx.x < n_tiles) {
-        const TileCoord c = tile_coord<EX>(pos_next, p);
-        if (c.t0 + t < p.T) {
-            const long long r = c.r0 + (long long)t * c.rs;
-            bi_next = __ldg(p.beta + r);
-            gi_next = __ldg(p.g + r);
-        }
-    }
+    int gtok_next = -1;
+    if (blockIdx.x < n_tiles) fetch_row(pos_next, bi_next, gi_next, gtok_next);
 
     for (uint32_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
         const TileCoord tc = tile_coord<EX>(pos_next, p);
-        tile_advance(pos_next, p);
+        tile_advance<EX>(pos_next, p);
         const uint32_t next = tile + gridDim.x;
         const bool has_next = next < n_tiles;
 
         STAMP(1);
         const float bi = bi_next;  // loaded during the previous tile
         float gi_ = gi_next;
+        const int gtok = gtok_next;
         constexpr int kWarpsPerChunk = MERGE ? 4 : (C >= 32 ? C / 32 : 1);
         if (f_graw) {
             // g holds the raw per-token log-gates: inclusive prefix sum inside the chunk, by shuffles inside the warp
@@ -641,7 +702,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 #pragma unroll
                 for (int jl = 0; jl < HC; ++jl)
                     if (col0 + jl == il) gd = a[jl];
-                const float rn = rsqrtf(fmaxf(gd, 1e-30f));
+                const float rn = (f_var && gtok < 0) ? 0.f : rsqrtf(fmaxf(gd, 1e-30f));
                 srn[t] = rn;
                 sbrn[t] = bi * rn * (f_wg ? fast_exp2(gi_ * kLog2e) : 1.f);
             }
@@ -688,14 +749,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         }
         bi_next = 0.f;
         gi_next = 0.f;
-        if (has_next) {
-            const TileCoord nc = tile_coord<EX>(pos_next, p);
-            if (nc.t0 + t < p.T) {
-                const long long r = nc.r0 + (long long)t * nc.rs;
-                bi_next = __ldg(p.beta + r);
-                gi_next = __ldg(p.g + r);
-            }
-        }
+        if (has_next) fetch_row(pos_next, bi_next, gi_next, gtok_next);
         compute_barrier();  // both halves of every fp32 row are written
 
         STAMP(4);
@@ -1351,15 +1405,10 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             if (warp == 0 && has_next && elect_one()) {
                 // the products that read this tile's K (half 0) or V (half 1) are complete: prefetch the next tile's
                 const TileCoord nc = tile_coord<EX>(pos_next, p);
-                if (half == 0) {
-                    mbar_arrive_expect_tx(&bar_k, 32768);
-                    tma_load_3d(sK, &tmK, &bar_k, nc.kx, nc.t0, nc.kz);
-                    tma_load_3d(sK + 16384, &tmK, &bar_k, nc.kx + 64, nc.t0, nc.kz);
-                } else {
-                    mbar_arrive_expect_tx(&bar_v, 32768);
-                    tma_load_3d(sV, &tmV, &bar_v, nc.vx, nc.t0, nc.vz);
-                    tma_load_3d(sV + 16384, &tmV, &bar_v, nc.vx + 64, nc.t0, nc.vz);
-                }
+                if (half == 0)
+                    load_tile(sK, &tmK, &bar_k, nc.kx, nc.t0, nc.kz);
+                else
+                    load_tile(sV, &tmV, &bar_v, nc.vx, nc.t0, nc.vz);
             }
             uint32_t o[32];
 #pragma unroll
@@ -1411,7 +1460,24 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 }
             }
             STAMP(12 + half * 3);
-            if (!f_f32) {
+            // variable-length sequences: a warp whose 32 rows are 32 consecutive real tokens stores them like the dense
+            // path (token coordinate of its first row); otherwise (a short chunk, or two chunks that are not adjacent in
+            // memory) every row of a real token goes out by itself, so that nothing reaches a neighbouring sequence
+            bool bulk = true;
+            int tok0 = tc.t0 + wrow0;
+            if (f_var) {
+                tok0 = __shfl_sync(0xFFFFFFFFu, gtok, 0);
+                bulk = __all_sync(0xFFFFFFFFu, gtok >= 0 && gtok == tok0 + lane);
+            }
+            if (!f_f32 && !bulk) {
+                if (gtok >= 0) {
+                    const bool bthd = (p.flags & GDN_FLAG_LAYOUT_BTHD) != 0;
+                    const long long row = bthd ? (long long)gtok * p.H_v + tc.bhv : (long long)tc.bhv * p.T_total + gtok;
+                    uint4* dst = reinterpret_cast<uint4*>((half == 0 ? p.W : p.U) + row * kD + h * 64);
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) dst[c] = make_uint4(o[c * 4 + 0], o[c * 4 + 1], o[c * 4 + 2], o[c * 4 + 3]);
+                }
+            } else if (!f_f32) {
                 // 32 rows x 64 columns of this warp in the 128-byte TMA swizzle: 4 KB at slice(wq) + h * 4 KB
                 const uint32_t sub = scratch_a + wq * 8192 + h * 4096;
                 if (lane == 0) tma_store_wait_read<0>();  // earlier stores from this sub-tile have been read
@@ -1422,7 +1488,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) {
-                    tma_store_3d((half == 0) ? &tmW : &tmU, smem + L::kEB + wq * 8192 + h * 4096, tc.vx + h * 64, tc.t0 + wrow0, tc.vz);
+                    tma_store_3d((half == 0) ? &tmW : &tmU, smem + L::kEB + wq * 8192 + h * 4096, tc.vx + h * 64, tok0, tc.vz);
                     tma_store_commit();
                 }
             }
@@ -1476,7 +1542,7 @@ struct Maps {
     CUtensorMap K, V, W, U, T;
 };
 
-template <int C, int NB, int MODE, bool MERGE, bool EX, int DBL>
+template <int C, int NB, int MODE, bool MERGE, int EX, int DBL>
 int launch_ex(const Maps& m, const Params& prm, cudaStream_t stream) {
     using L = Smem<C, NB>;
     const int smem = L::kTotal + 1024;
@@ -1486,8 +1552,8 @@ int launch_ex(const Maps& m, const Params& prm, cudaStream_t stream) {
     Params q = prm;
     const long long y = grid / prm.group;
     q.s_gi = static_cast<int>(grid - y * prm.group);
-    q.s_bhk = static_cast<int>(y / prm.n_tt);
-    q.s_tt = static_cast<int>(y - static_cast<long long>(q.s_bhk) * prm.n_tt);
+    q.s_bhk = static_cast<int>(y / prm.n_mid);
+    q.s_tt = static_cast<int>(y - static_cast<long long>(q.s_bhk) * prm.n_mid);
     kern<<<static_cast<int>(grid), kThreads, smem, stream>>>(m.K, m.V, m.W, m.U, m.T, q);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? GDN_OK : GDN_ERR_LAUNCH;
@@ -1498,14 +1564,19 @@ int launch_one(const Maps& m, const Params& prm, cudaStream_t stream) {
     constexpr bool kNeu = (MODE == INV_NEUMANN);
     constexpr bool kDbl = kNeu && C == 64;
     const int dbl = !kDbl ? 0 : (prm.S == 8 ? 8 : (prm.S == 15 ? 15 : 0));
-    if (kNeu && prm.flags != 0) {
-        if (dbl == 8) return launch_ex<C, NB, MODE, MERGE, kNeu, kDbl ? 8 : 0>(m, prm, stream);
-        if (dbl == 15) return launch_ex<C, NB, MODE, MERGE, kNeu, kDbl ? 15 : 0>(m, prm, stream);
-        return launch_ex<C, NB, MODE, MERGE, kNeu, 0>(m, prm, stream);
+    if (kNeu && (prm.flags & GDN_FLAG_OUT_FP32) != 0) {
+        if (dbl == 8) return launch_ex<C, NB, MODE, MERGE, kNeu ? 2 : 0, kDbl ? 8 : 0>(m, prm, stream);
+        if (dbl == 15) return launch_ex<C, NB, MODE, MERGE, kNeu ? 2 : 0, kDbl ? 15 : 0>(m, prm, stream);
+        return launch_ex<C, NB, MODE, MERGE, kNeu ? 2 : 0, 0>(m, prm, stream);
     }
-    if (dbl == 8) return launch_ex<C, NB, MODE, MERGE, false, kDbl ? 8 : 0>(m, prm, stream);
-    if (dbl == 15) return launch_ex<C, NB, MODE, MERGE, false, kDbl ? 15 : 0>(m, prm, stream);
-    return launch_ex<C, NB, MODE, MERGE, false, 0>(m, prm, stream);
+    if (kNeu && (prm.flags != 0 || prm.chunk_start != nullptr)) {
+        if (dbl == 8) return launch_ex<C, NB, MODE, MERGE, kNeu ? 1 : 0, kDbl ? 8 : 0>(m, prm, stream);
+        if (dbl == 15) return launch_ex<C, NB, MODE, MERGE, kNeu ? 1 : 0, kDbl ? 15 : 0>(m, prm, stream);
+        return launch_ex<C, NB, MODE, MERGE, kNeu ? 1 : 0, 0>(m, prm, stream);
+    }
+    if (dbl == 8) return launch_ex<C, NB, MODE, MERGE, 0, kDbl ? 8 : 0>(m, prm, stream);
+    if (dbl == 15) return launch_ex<C, NB, MODE, MERGE, 0, kDbl ? 15 : 0>(m, prm, stream);
+    return launch_ex<C, NB, MODE, MERGE, 0, 0>(m, prm, stream);
 }
 
 template <int C, int MODE, bool MERGE = false>
@@ -1548,6 +1619,8 @@ int launch_tc_bf16(const Problem& p, InverseMode mode, cudaStream_t stream) {
     if (!(p.C == 16 || p.C == 32 || p.C == 64 || (p.C == 128 && mode == INV_NEUMANN))) return GDN_ERR_UNSUPPORTED;
     if (mode == INV_NEUMANN && (p.order < 1 || p.order > 7)) return GDN_ERR_UNSUPPORTED;
     if ((long long)p.B * p.H_v * p.T == 0) return GDN_OK;
+    const bool varlen = p.chunk_start != nullptr;
+    if (varlen && (mode != INV_NEUMANN || p.B != 1 || p.T % kTile != 0)) return GDN_ERR_UNSUPPORTED;
     int* status = device_status_word();
     if (status == nullptr) return GDN_ERR_LAUNCH;
     Maps m;
@@ -1560,10 +1633,14 @@ int launch_tc_bf16(const Problem& p, InverseMode mode, cudaStream_t stream) {
     if (bthd && mode != INV_NEUMANN) return GDN_ERR_UNSUPPORTED;
     const long long zk = bthd ? p.B : hk, zv = bthd ? p.B : hv;
     const int ck = bthd ? p.H_k * kD : kD, cv = bthd ? p.H_v * kD : kD;
-    if (!make_map(&m.K, p.K, zk, p.T, ck, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
-    if (!make_map(&m.V, p.V, zv, p.T, cv, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
-    if (!make_map(&m.W, p.W, zv, p.T, cv, 64, 32, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
-    if (!make_map(&m.U, p.U, zv, p.T, cv, 64, 32, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
+    // variable-length sequences: the inputs hold T_total tokens and are loaded one chunk per box (W and U leave
+    // by plain stores there, their maps are not used)
+    const int t_in = varlen ? p.T_total : p.T;
+    const int in_rows = varlen ? p.C : 128;
+    if (!make_map(&m.K, p.K, zk, t_in, ck, 64, in_rows, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
+    if (!make_map(&m.V, p.V, zv, t_in, cv, 64, in_rows, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
+    if (!make_map(&m.W, p.W, zv, t_in, cv, 64, 32, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
+    if (!make_map(&m.U, p.U, zv, t_in, cv, 64, 32, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
     // Tinv rows are C wide; without a Tinv output the map points at W (never used by the kernel then)
     if (!make_map(&m.T, p.Tinv != nullptr ? p.Tinv : p.W, hv, p.T, p.Tinv != nullptr ? p.C : kD, p.Tinv != nullptr ? tbox : 64, 32,
                   p.Tinv != nullptr ? tsw : CU_TENSOR_MAP_SWIZZLE_128B))
@@ -1580,9 +1657,14 @@ int launch_tc_bf16(const Problem& p, InverseMode mode, cudaStream_t stream) {
     prm.T = p.T;
     prm.group = p.H_v / p.H_k;
     prm.n_tt = (p.T + kTile - 1) / kTile;
+    prm.n_mid = bthd ? p.H_k : prm.n_tt;
     prm.N = p.order;
     prm.S = p.steps;
     prm.flags = p.flags;
+    prm.chunk_start = p.chunk_start;
+    prm.chunk_len = p.chunk_len;
+    prm.n_chunks = p.n_chunks;
+    prm.T_total = p.T_total;
     prm.n_tiles = (long long)p.B * p.H_v * prm.n_tt;
     if (prm.n_tiles >= (1LL << 31) - 4096 || (long long)p.B * p.H_v >= (1LL << 31)) return GDN_ERR_UNSUPPORTED;
     if (mode == INV_NEUMANN) {

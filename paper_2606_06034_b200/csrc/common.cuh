@@ -22,6 +22,12 @@ struct Problem {
     int steps;   // S
     int dtype;   // GDN_DTYPE_*
     unsigned flags = 0;  // GDN_FLAG_*
+    // packed variable-length sequences (B = 1): device arrays with the first token and the length of every chunk;
+    // T is then the padded token count (a multiple of 128), T_total the number of tokens the tensors hold
+    const int* chunk_start = nullptr;
+    const int* chunk_len = nullptr;
+    int n_chunks = 0;
+    int T_total = 0;
 };
 
 // INT8 entry point's problem description

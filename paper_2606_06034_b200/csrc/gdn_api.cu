@@ -120,6 +120,34 @@ int gdn_chunk_prepare_ex(const void* K, const void* V, const float* beta, const 
     return run(p, INV_NEUMANN, static_cast<cudaStream_t>(stream));
 }
 
+int gdn_chunk_prepare_varlen(const void* K, const void* V, const float* beta, const float* g, const int32_t* chunk_start,
+                             const int32_t* chunk_len, int n_chunks, int T_total, int H_k, int H_v, int C, int d_k, int d_v,
+                             int order, int residual_steps, void* W_out, void* U_out, void* Tinv_out, unsigned flags,
+                             gdn_stream_t stream) {
+    if (flags & ~static_cast<unsigned>(GDN_FLAG_G_RAW | GDN_FLAG_K_L2NORM | GDN_FLAG_LAYOUT_BTHD | GDN_FLAG_W_GATED))
+        return GDN_ERR_INVALID_ARG;
+    if (chunk_start == nullptr || chunk_len == nullptr) return GDN_ERR_NULL;
+    if (n_chunks < 0 || T_total < 0) return GDN_ERR_INVALID_ARG;
+    if (!(C == 16 || C == 32 || C == 64 || C == 128)) return C >= 2 ? GDN_ERR_UNSUPPORTED : GDN_ERR_INVALID_ARG;
+    // the chunks are walked in tiles of 128 token rows: T is the padded row count
+    const long long rows = ((long long)n_chunks * C + 127) / 128 * 128;
+    if (rows >= (1LL << 31)) return GDN_ERR_UNSUPPORTED;
+    Problem p{K, V, beta, g, W_out, U_out, Tinv_out, 1, H_k, H_v, static_cast<int>(rows), C, d_k, d_v, order, residual_steps,
+              GDN_DTYPE_BF16};
+    p.flags = flags;
+    p.chunk_start = chunk_start;
+    p.chunk_len = chunk_len;
+    p.n_chunks = n_chunks;
+    p.T_total = T_total;
+    if (n_chunks == 0 || T_total == 0) {
+        if (p.order == -1) p.order = gdn_default_order(C);
+        if (p.steps == -1) p.steps = gdn_default_residual_steps(C);
+        const int rc = validate(p, true);
+        return rc != GDN_OK ? rc : check_arch();
+    }
+    return run(p, INV_NEUMANN, static_cast<cudaStream_t>(stream));
+}
+
 int gdn_chunk_prepare_fwdsubst(const void* K, const void* V, const float* beta, const float* g, int B, int H_k, int H_v, int T,
                                int C, int d_k, int d_v, int dtype, int variant, void* W_out, void* U_out, void* Tinv_out,
                                gdn_stream_t stream) {

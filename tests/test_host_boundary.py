@@ -71,6 +71,15 @@ def test_bad_arguments_are_rejected_without_a_device(lib):
     assert call(Ti=mis) == gdn.GDN_ERR_ALIGN
     assert lib.gdn_chunk_prepare_gqa(p, p, p, p, 1, 2, 3, 128, 64, 128, 128, -1, -1, 1, p, p, p, None) == gdn.GDN_ERR_INVALID_ARG
     assert lib.gdn_chunk_prepare_fwdsubst(p, p, p, p, 1, 1, 1, 128, 64, 128, 128, 1, 5, p, p, p, None) == gdn.GDN_ERR_INVALID_ARG
+    vl = lambda **kw: lib.gdn_chunk_prepare_varlen(*[kw.get(k, d) for k, d in (
+        ("K", p), ("V", p), ("beta", p), ("g", p), ("cs", p), ("cl", p), ("n", 2), ("T", 128), ("Hk", 1), ("Hv", 1), ("C", 64),
+        ("dk", 128), ("dv", 128), ("N", -1), ("S", -1), ("W", p), ("U", p), ("Ti", p), ("flags", 0), ("stream", None))])
+    assert vl(cs=None) == gdn.GDN_ERR_NULL
+    assert vl(n=-1) == gdn.GDN_ERR_INVALID_ARG
+    assert vl(C=48) == gdn.GDN_ERR_UNSUPPORTED
+    assert vl(flags=gdn.GDN_FLAG_OUT_FP32) == gdn.GDN_ERR_INVALID_ARG
+    assert vl(Hk=2, Hv=3) == gdn.GDN_ERR_INVALID_ARG
+    assert vl(W=mis) == gdn.GDN_ERR_ALIGN
     # valid arguments but no sm_100 device in this process: refused, nothing launched
     import torch
     if not torch.cuda.is_available():
@@ -84,3 +93,18 @@ def test_binding_refuses_host_tensors():
     b = torch.zeros(1, 1, 64)
     with pytest.raises(ValueError):
         gdn.chunk_prepare(K, K, b, b, 64)
+
+
+def test_chunk_table_of_packed_sequences():
+    """Host-side chunking of packed sequences (each sequence chunked from its own first token, last chunk short),
+    against the oracle's own table."""
+    from oracle import gdn_oracle as orc
+    for C in (16, 64, 128):
+        for cu in ([0, 5, 5, 70, 198, 199, 327], [0, C], [0, C - 1, 2 * C], [0]):
+            start, length = gdn.chunk_table(cu, C)
+            o_start, o_length = orc.chunk_table(cu, C)
+            assert list(start) == list(o_start) and list(length) == list(o_length)
+            assert sum(length) == cu[-1] and all(1 <= n <= C for n in length)
+    with pytest.raises(ValueError):
+        gdn.chunk_table([0, 10, 5], 64)
+
