@@ -426,7 +426,8 @@ __device__ __forceinline__ TileCoord tile_coord(const TilePos& c, const Params& 
 // T21 = -T22 A21 T11, evaluated as Y = A21 + A21 X11, T21 = -(Y + X22 Y) with X = T - I of the blocks, so that
 // the identity parts stay in fp32 and only the small products pass through bf16 operands.
 // EX: 1 = the optional prologue, layouts and packed sequences of gdn_chunk_prepare_ex / _varlen are compiled in (flags
-// read at run time); 2 = also the fp32 outputs (parity debugging; they cost registers, so they have their own code).
+// read at run time); 2 = also the fp32 outputs (parity debugging); 3 = 1 for packed variable-length sequences. The
+// last two cost registers, so each has its own code.
 // DBL: 8 or 15 = the residual sum for that S is evaluated by the four-level doubling scheme (C = 64 only); 0 = one
 // product per term.
 template <int C, int NB, int MODE, bool MERGE, int EX, int DBL>
@@ -461,7 +462,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     const bool f_wg = EX && (p.flags & GDN_FLAG_W_GATED) != 0;
     const bool two_scales = f_l2 || f_wg;  // the W operand is scaled by something other than beta
     const bool f_f32 = EX == 2 && (p.flags & GDN_FLAG_OUT_FP32) != 0;
-    const bool f_var = EX && p.chunk_start != nullptr;
+    constexpr bool f_var = EX == 3;
     constexpr int CR = MERGE ? kTile : C;  // tokens of a chunk
 
     __shared__ uint64_t bar_k, bar_v, bar_mma;
@@ -632,13 +633,13 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 if ((lane & (SEG - 1)) >= off) gi_ += v;
             }
         }
+        // (the warp totals of the previous tile were read right after that tile's first barrier: free to overwrite)
+        if (f_graw && kWarpsPerChunk > 1 && h == 0 && lane == 31) swt[wq] = gi_;
         // the previous tile's bulk stores have finished reading the staging slices
         if (lane == 0) tma_store_wait_read<0>();
         tc_fence_before_sync();
         compute_barrier();  // everyone is done with the previous tile's shared arrays and accumulators
         if (f_graw && kWarpsPerChunk > 1) {
-            if (h == 0 && lane == 31) swt[wq] = gi_;
-            compute_barrier();
             const int first = wq - (wq % kWarpsPerChunk);
             for (int w = first; w < wq; ++w) gi_ += swt[w];
         }
@@ -709,9 +710,9 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             compute_barrier();
             rni = srn[t];
         } else if (f_wg) {
-            // gated W: the column scale of the W operand is beta_j exp(g_j)
+            // gated W: the column scale of the W operand is beta_j exp(g_j) (read after the barriers of the stages
+            // below)
             if (h == 0) sbrn[t] = bi * fast_exp2(gi_ * kLog2e);
-            compute_barrier();
         }
         if (active) {
             const float gs = gi_ * kLog2e;
@@ -1569,7 +1570,12 @@ int launch_one(const Maps& m, const Params& prm, cudaStream_t stream) {
         if (dbl == 15) return launch_ex<C, NB, MODE, MERGE, kNeu ? 2 : 0, kDbl ? 15 : 0>(m, prm, stream);
         return launch_ex<C, NB, MODE, MERGE, kNeu ? 2 : 0, 0>(m, prm, stream);
     }
-    if (kNeu && (prm.flags != 0 || prm.chunk_start != nullptr)) {
+    if (kNeu && prm.chunk_start != nullptr) {
+        if (dbl == 8) return launch_ex<C, NB, MODE, MERGE, kNeu ? 3 : 0, kDbl ? 8 : 0>(m, prm, stream);
+        if (dbl == 15) return launch_ex<C, NB, MODE, MERGE, kNeu ? 3 : 0, kDbl ? 15 : 0>(m, prm, stream);
+        return launch_ex<C, NB, MODE, MERGE, kNeu ? 3 : 0, 0>(m, prm, stream);
+    }
+    if (kNeu && prm.flags != 0) {
         if (dbl == 8) return launch_ex<C, NB, MODE, MERGE, kNeu ? 1 : 0, kDbl ? 8 : 0>(m, prm, stream);
         if (dbl == 15) return launch_ex<C, NB, MODE, MERGE, kNeu ? 1 : 0, kDbl ? 15 : 0>(m, prm, stream);
         return launch_ex<C, NB, MODE, MERGE, kNeu ? 1 : 0, 0>(m, prm, stream);
