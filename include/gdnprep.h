@@ -187,6 +187,21 @@ int gdn_chunk_state_output(const void* Q, const void* K, const void* W_gated, co
                            int B, int H_k, int H_v, int T, int C, int d_k, int d_v, float scale,
                            const float* S_in, void* O_out, float* S_out, unsigned flags, gdn_stream_t stream);
 
+/*
+ * gdn_chunk_state_output for packed variable-length sequences (the tensors gdn_chunk_prepare_varlen works on): sequence s
+ * holds the tokens [cu_seqlens[s], cu_seqlens[s + 1]) and has its own state. One CTA per (sequence, value head) walks
+ * the sequence's chunks from its first token; in a short last chunk the tokens past the end write nothing and the rows
+ * of the output past the end are not stored.
+ *   Q, K [H_k,T_total,d_k], W_gated [H_v,T_total,d_k], U [H_v,T_total,d_v] bf16; g [H_v,T_total] (restarting in every
+ *   chunk of every sequence, or raw with GDN_FLAG_G_RAW); cu_seqlens: DEVICE array of n_seq + 1 int32, non-decreasing,
+ *   cu_seqlens[n_seq] <= T_total; S_in, S_out [n_seq,H_v,d_v,d_k] fp32 (either may be NULL); O_out [H_v,T_total,d_v].
+ * Supported: C = 64, d_k = d_v = 128, head-major tensors.
+ */
+int gdn_chunk_state_output_varlen(const void* Q, const void* K, const void* W_gated, const void* U, const float* g,
+                                  const int32_t* cu_seqlens, int n_seq, int T_total, int H_k, int H_v, int C,
+                                  int d_k, int d_v, float scale, const float* S_in, void* O_out, float* S_out,
+                                  unsigned flags, gdn_stream_t stream);
+
 /* Checksum of the 256-entry gate-decay table round(2^15 * 2^(-f/256)) the INT8 kernel uses
  * (sum_f: s = (31 s + table[f] + f) mod 1000000007), so that a CPU evaluation can confirm it holds the same table. */
 unsigned int gdn_int8_lut_checksum(void);

@@ -36,7 +36,7 @@ GDN_FWDSUBST_BLOCKED = 1
 EXPORTS = (
     "gdn_chunk_prepare", "gdn_chunk_prepare_gqa", "gdn_chunk_prepare_ex", "gdn_chunk_prepare_varlen",
     "gdn_chunk_prepare_fwdsubst",
-    "gdn_chunk_prepare_int8", "gdn_chunk_state_output", "gdn_selftest_bounded_wait",
+    "gdn_chunk_prepare_int8", "gdn_chunk_state_output", "gdn_chunk_state_output_varlen", "gdn_selftest_bounded_wait",
     "gdn_int8_lut_checksum",
     "gdn_device_status", "gdn_default_order", "gdn_default_residual_steps",
     "gdn_status_string", "gdn_launch_count",
@@ -78,6 +78,9 @@ def load_library() -> ctypes.CDLL:
     lib.gdn_chunk_state_output.argtypes = [vp, vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ip, ctypes.c_float, vp, vp, vp,
                                            ctypes.c_uint, vp]
     lib.gdn_chunk_state_output.restype = ip
+    lib.gdn_chunk_state_output_varlen.argtypes = [vp, vp, vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ip, ctypes.c_float, vp, vp, vp,
+                                                  ctypes.c_uint, vp]
+    lib.gdn_chunk_state_output_varlen.restype = ip
     lib.gdn_selftest_bounded_wait.argtypes = [vp]
     lib.gdn_selftest_bounded_wait.restype = ip
     lib.gdn_int8_lut_checksum.argtypes = []
@@ -300,6 +303,35 @@ def gdn_chunk_state_output(Q, K, W_gated, U, g, B, H_k, H_v, T, C, d_k, d_v, sca
     if check and rc != GDN_OK:
         raise GdnError(rc, "gdn_chunk_state_output")
     return rc
+
+
+def gdn_chunk_state_output_varlen(Q, K, W_gated, U, g, cu_seqlens, n_seq, T_total, H_k, H_v, C, d_k, d_v, scale, S_in, O_out,
+                                  S_out, flags=0, *, check=True):
+    """Raw call of the packed-sequence form (cu_seqlens: int32 CUDA tensor of n_seq + 1 boundaries)."""
+    for t in (Q, K, W_gated, U, g, cu_seqlens, S_in, O_out, S_out):
+        if t is not None and (not t.is_cuda or not t.is_contiguous()):
+            raise ValueError("all tensors must be contiguous CUDA tensors (there is no CPU path)")
+    if cu_seqlens is not None and cu_seqlens.dtype != torch.int32:
+        raise TypeError("cu_seqlens is an int32 tensor")
+    rc = load_library().gdn_chunk_state_output_varlen(_ptr(Q), _ptr(K), _ptr(W_gated), _ptr(U), _ptr(g), _ptr(cu_seqlens), n_seq,
+                                                      T_total, H_k, H_v, C, d_k, d_v, ctypes.c_float(scale), _ptr(S_in),
+                                                      _ptr(O_out), _ptr(S_out), flags, _stream())
+    if check and rc != GDN_OK:
+        raise GdnError(rc, "gdn_chunk_state_output_varlen")
+    return rc
+
+
+def chunk_state_output_varlen(Q, K, W_gated, U, g, cu_seqlens, C, scale=1.0, S_in=None, *, want_state=True, flags=0):
+    """Packed sequences: Q, K [H_k,T,d_k], W_gated [H_v,T,d_k], U [H_v,T,d_v], g [H_v,T]; cu_seqlens on the host.
+    Returns (O [H_v,T,d_v], S_out [n_seq,H_v,d_v,d_k] fp32 or None); rows of O that no sequence covers stay zero."""
+    H_k, T, d_k = K.shape
+    H_v, _, d_v = U.shape
+    cu = torch.tensor([int(x) for x in cu_seqlens], dtype=torch.int32, device=U.device)
+    n_seq = cu.numel() - 1
+    O = torch.zeros(H_v, T, d_v, dtype=U.dtype, device=U.device)
+    S_out = torch.empty(n_seq, H_v, d_v, d_k, dtype=torch.float32, device=U.device) if want_state else None
+    gdn_chunk_state_output_varlen(Q, K, W_gated, U, g, cu, n_seq, T, H_k, H_v, C, d_k, d_v, scale, S_in, O, S_out, flags)
+    return O, S_out
 
 
 def chunk_state_output(Q, K, W_gated, U, g, C, scale=1.0, S_in=None, *, want_state=True, outputs=None, flags=0):

@@ -72,6 +72,10 @@ struct ParamsS {
     int H_k, H_v, T, group;
     float scale;
     unsigned flags;  // GDN_FLAG_G_RAW: g holds raw log-gates, prefix-summed inside every chunk here
+    // packed variable-length sequences (B = 1): sequence s holds the tokens [cu_seqlens[s], cu_seqlens[s + 1]) of tensors
+    // with T tokens per head and is chunked from its own first token; null for dense tensors
+    const int* cu_seqlens;
+    __nv_bfloat16* O;  // output tensor (rows of a short last chunk are stored one by one)
 };
 
 __device__ __forceinline__ float fast_exp2(float x) {
@@ -91,6 +95,8 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity) {
     return true;
 }
 
+// VAR: packed variable-length sequences (own instantiation: its masks sit on the chain the dense case is bound by)
+template <bool VAR>
 __global__ void __launch_bounds__(kThreads + 64, 1)
 chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                    const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmU,
@@ -145,11 +151,15 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     const uint32_t tmem = tmem_base_s;
     const uint32_t lane_base = tmem + (static_cast<uint32_t>(wq * 32) << 16);
 
-    const int bhv = blockIdx.x;
-    const int b = bhv / p.H_v, hv = bhv - b * p.H_v;
-    const int bhk = b * p.H_k + hv / p.group;
-    const int n_c = p.T / kC;
-    const float* gseq = p.g + (long long)bhv * p.T;
+    // dense: one CTA per (batch, value head), bhv = row of the [B * H_v, T] tensors. Packed sequences: one CTA per
+    // (sequence, value head); the tensors have one batch row per head and the sequence starts at token tok0
+    const int b = blockIdx.x / p.H_v, hv = blockIdx.x - b * p.H_v;
+    const int tok0 = VAR ? __ldg(p.cu_seqlens + b) : 0;
+    const int len = VAR ? __ldg(p.cu_seqlens + b + 1) - tok0 : p.T;
+    const int bhv = VAR ? hv : blockIdx.x;
+    const int bhk = VAR ? hv / p.group : b * p.H_k + hv / p.group;
+    const int n_c = (len + kC - 1) / kC;
+    const float* gseq = p.g + (long long)bhv * p.T + tok0;
     const uint32_t smem_a = smem_u32(smem);
     volatile int* fail = reinterpret_cast<volatile int*>(&s_fail);
 
@@ -161,7 +171,7 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 uint8_t* st = smem + (c & 1) * kStageBytes;
                 uint64_t* bar = &bar_full[c & 1];
                 mbar_arrive_expect_tx(bar, kStageBytes);
-                const int t0 = c * kC;
+                const int t0 = tok0 + c * kC;
                 tma_load_3d(st + kOffQ, &tmQ, bar, 0, t0, bhk);
                 tma_load_3d(st + kOffQ + 8192, &tmQ, bar, 64, t0, bhk);
                 tma_load_3d(st + kOffK, &tmK, bar, 0, t0, bhk);
@@ -302,7 +312,7 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             }
             tmem_st16(lane_base + kIA + h * 16, r);
             // this thread's quarter of state row t: columns [32 h, 32 h + 32)
-            const float* s0 = (p.S_in != nullptr) ? p.S_in + ((long long)bhv * kD + t) * kD + h * 32 : nullptr;
+            const float* s0 = (p.S_in != nullptr) ? p.S_in + ((long long)blockIdx.x * kD + t) * kD + h * 32 : nullptr;
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
                 uint32_t v[16], pk[8];
@@ -323,7 +333,8 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         }
         // gates of the first chunk
         float g_reg = 0.f;
-        if (n_c > 0 && tid < 64) g_reg = __ldg(gseq + tid);
+        // (a short last chunk: tokens past the sequence's end decay nothing and write nothing)
+        if (n_c > 0 && tid < 64) g_reg = (!VAR || tid < len) ? __ldg(gseq + tid) : 0.f;
         bool ok = true;
         // gate tables of a chunk: written by 64 threads into the buffer of that chunk one barrier before they are read
         const bool g_raw = (p.flags & GDN_FLAG_G_RAW) != 0;
@@ -331,6 +342,7 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             if (tid < 64) {
                 float* tb = gtab + (c & 1) * 192;
                 float gc = g_reg;
+                const int left = len - c * kC;  // tokens of this chunk (>= 64 except for a short last chunk)
                 if (g_raw) {
                     // inclusive prefix sum over the chunk's 64 tokens: inside each of the two warps by shuffles ...
 #pragma unroll
@@ -345,6 +357,13 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 }
                 tb[128 + tid] = gc;
                 asm volatile("bar.sync 3, 64;" ::: "memory");
+                if (VAR && !g_raw && left < kC) {
+                    // cumulative gates: tokens past the end keep the gate of the last real token
+                    gc = tb[128 + (tid < left ? tid : left - 1)];
+                    asm volatile("bar.sync 3, 64;" ::: "memory");
+                    tb[128 + tid] = gc;
+                    asm volatile("bar.sync 3, 64;" ::: "memory");
+                }
                 const float gC = tb[128 + 63];  // cumulative gate of the chunk's last token
                 tb[tid] = fast_exp2(gc * kLog2e);
                 tb[64 + tid] = fast_exp2((gC - gc) * kLog2e);
@@ -357,7 +376,9 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             const float* sf = se + 64;               // exp(g_C - g_j)
             const float* sg = se + 128;              // g_i (cumulative inside the chunk)
             const float gC = sg[63];
-            if (c + 1 < n_c && tid < 64) g_reg = __ldg(gseq + (c + 1) * kC + tid);
+            const int left = len - c * kC;
+            const bool short_chunk = VAR && left < kC;
+            if (c + 1 < n_c && tid < 64) g_reg = (!VAR || (c + 1) * kC + tid < len) ? __ldg(gseq + (c + 1) * kC + tid) : 0.f;
             STAMPS(1);
 
             STAMPS(2);
@@ -419,7 +440,11 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 uint32_t hi[16], lo[16];
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
-                    const float u0 = -__uint_as_float(d[2 * i]), u1 = -__uint_as_float(d[2 * i + 1]);
+                    float u0 = -__uint_as_float(d[2 * i]), u1 = -__uint_as_float(d[2 * i + 1]);
+                    if (short_chunk) {  // rows past the sequence's end hold another sequence's W, U
+                        if (h * 16 + 2 * i >= left) u0 = 0.f;
+                        if (h * 16 + 2 * i + 1 >= left) u1 = 0.f;
+                    }
                     const float2 f = *reinterpret_cast<const float2*>(sf + h * 16 + 2 * i);
                     const float s0 = u0 * f.x, s1 = u1 * f.y;
                     hi[i] = pack_bf16x2(u0, u1);
@@ -490,15 +515,23 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             // (issued a whole chunk ago: this never waits in practice; the barrier below publishes it)
             if (tid == 0) tma_store_wait_read<0>();
             asm volatile("bar.sync 1, 512;" ::: "memory");  // the staged output tile and the next gate tables are complete
-            if (tid == 0) {  // the same thread waits for these stores (bulk groups are per thread)
-                tma_store_3d(&tmO, smem + kOffO + (c & 1) * kTileBytes, 0, c * kC, bhv);
-                tma_store_3d(&tmO, smem + kOffO + (c & 1) * kTileBytes + 8192, 64, c * kC, bhv);
+            if (short_chunk) {
+                // only the rows of real tokens leave, 16 bytes per thread and step, from the staged (swizzled) tile
+                for (int q = tid; q < left * 16; q += kThreads) {
+                    const int tok = q >> 4, ch = q & 15;  // 16-byte piece ch of the token's 256-byte row
+                    const uint4 v = *reinterpret_cast<const uint4*>(smem + kOffO + (c & 1) * kTileBytes + (ch >> 3) * 8192 +
+                                                                    tok * 128 + (((ch & 7) ^ (tok & 7)) << 4));
+                    *reinterpret_cast<uint4*>(p.O + ((long long)bhv * p.T + tok0 + c * kC + tok) * kD + ch * 8) = v;
+                }
+            } else if (tid == 0) {  // the same thread waits for these stores (bulk groups are per thread)
+                tma_store_3d(&tmO, smem + kOffO + (c & 1) * kTileBytes, 0, tok0 + c * kC, bhv);
+                tma_store_3d(&tmO, smem + kOffO + (c & 1) * kTileBytes + 8192, 64, tok0 + c * kC, bhv);
                 tma_store_commit();
             }
         }
         // ---- final state
         if (ok && p.S_out != nullptr) {
-            float* so = p.S_out + ((long long)bhv * kD + t) * kD + h * 32;
+            float* so = p.S_out + ((long long)blockIdx.x * kD + t) * kD + h * 32;
             uint32_t v[32];
             tmem_ld32(lane_base + kSD + h * 32, v);
             tmem_wait_ld();
@@ -559,8 +592,12 @@ extern "C" int gdn_debug_read_trace_state(long long* host_out) {
 
 int launch_chunk_state(const ProblemS& q, cudaStream_t stream) {
     if (q.d_k != kD || q.d_v != kD || q.C != kC) return GDN_ERR_UNSUPPORTED;
-    const long long hk = (long long)q.B * q.H_k, hv = (long long)q.B * q.H_v;
-    if (hv == 0 || q.T == 0) return GDN_OK;
+    // packed sequences: B counts the sequences, the tensors have one row of T tokens per head
+    const bool var = q.cu_seqlens != nullptr;
+    const long long hk = var ? q.H_k : (long long)q.B * q.H_k, hv = var ? q.H_v : (long long)q.B * q.H_v;
+    const long long n_cta = (long long)q.B * q.H_v;
+    if (n_cta == 0 || q.T == 0) return GDN_OK;
+    if (n_cta >= (1LL << 31)) return GDN_ERR_UNSUPPORTED;
     if (hv >= (1LL << 31)) return GDN_ERR_UNSUPPORTED;
     int* status = device_status_word();
     if (status == nullptr) return GDN_ERR_LAUNCH;
@@ -579,10 +616,12 @@ int launch_chunk_state(const ProblemS& q, cudaStream_t stream) {
     prm.group = q.H_v / q.H_k;
     prm.scale = q.scale;
     prm.flags = q.flags;
+    prm.cu_seqlens = q.cu_seqlens;
+    prm.O = static_cast<__nv_bfloat16*>(q.O);
     const int smem = kSmemTotal + 1024;
-    if (cudaFuncSetAttribute(chunk_state_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
-        return GDN_ERR_LAUNCH;
-    chunk_state_kernel<<<static_cast<int>(hv), kThreads + 64, smem, stream>>>(mQ, mK, mW, mU, mO, prm);
+    auto kern = var ? chunk_state_kernel<true> : chunk_state_kernel<false>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return GDN_ERR_LAUNCH;
+    kern<<<static_cast<int>(n_cta), kThreads + 64, smem, stream>>>(mQ, mK, mW, mU, mO, prm);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? GDN_OK : GDN_ERR_LAUNCH;
 }

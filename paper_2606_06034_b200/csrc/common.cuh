@@ -62,6 +62,9 @@ struct ProblemS {
     int B, H_k, H_v, T, C, d_k, d_v;
     float scale;
     unsigned flags;
+    // packed variable-length sequences: B sequences, sequence s = tokens [cu_seqlens[s], cu_seqlens[s + 1]) of tensors
+    // with T tokens per head (device array of B + 1 int32); null for dense tensors
+    const int* cu_seqlens = nullptr;
 };
 
 enum InverseMode { INV_NEUMANN = 0, INV_FWDSUBST_ROWS = 1, INV_FWDSUBST_BLOCKED = 2 };

@@ -193,6 +193,26 @@ int gdn_chunk_state_output(const void* Q, const void* K, const void* W_gated, co
     return launch_chunk_state(q, static_cast<cudaStream_t>(stream));
 }
 
+int gdn_chunk_state_output_varlen(const void* Q, const void* K, const void* W_gated, const void* U, const float* g,
+                                  const int32_t* cu_seqlens, int n_seq, int T_total, int H_k, int H_v, int C, int d_k, int d_v,
+                                  float scale, const float* S_in, void* O_out, float* S_out, unsigned flags,
+                                  gdn_stream_t stream) {
+    if (flags & ~static_cast<unsigned>(GDN_FLAG_G_RAW)) return GDN_ERR_INVALID_ARG;
+    if (Q == nullptr || K == nullptr || W_gated == nullptr || U == nullptr || g == nullptr || O_out == nullptr ||
+        cu_seqlens == nullptr)
+        return GDN_ERR_NULL;
+    if (n_seq < 0 || H_k <= 0 || H_v <= 0 || T_total < 0 || C < 2 || d_k <= 0 || d_v <= 0) return GDN_ERR_INVALID_ARG;
+    if (H_v % H_k != 0) return GDN_ERR_INVALID_ARG;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(W_gated) || !aligned16(U) || !aligned16(g) || !aligned16(S_in) ||
+        !aligned16(O_out) || !aligned16(S_out))
+        return GDN_ERR_ALIGN;
+    const int rc = check_arch();
+    if (rc != GDN_OK) return rc;
+    ProblemS q{Q, K, W_gated, U, g, S_in, O_out, S_out, n_seq, H_k, H_v, T_total, C, d_k, d_v, scale, flags};
+    q.cu_seqlens = cu_seqlens;
+    return launch_chunk_state(q, static_cast<cudaStream_t>(stream));
+}
+
 int gdn_selftest_bounded_wait(gdn_stream_t stream) {
     const int rc = check_arch();
     if (rc != GDN_OK) return rc;

@@ -139,3 +139,73 @@ def test_varlen_argument_errors():
     assert call(K, K, b, b, cs, cs, 2, 128, 1, 1, 64, 128, 128, -1, -1, K, K, None, gdn.GDN_FLAG_OUT_FP32) == gdn.GDN_ERR_INVALID_ARG
     assert call(K, K, b, b, cs, cs, 0, 128, 1, 1, 64, 128, 128, -1, -1, K, K, None, 0) == gdn.GDN_OK
     assert gdn.gdn_device_status() == gdn.GDN_OK
+
+
+def _queries(H_k, T, seed):
+    gq = torch.Generator().manual_seed(seed)
+    Q = torch.randn(H_k, T, 128, generator=gq)
+    return (Q / Q.norm(dim=-1, keepdim=True)).to(torch.bfloat16)
+
+
+@pytest.mark.parametrize("with_state,raw", [(False, False), (True, False), (True, True)])
+def test_packed_layer_matches_the_token_recurrence_per_sequence(with_state, raw):
+    """Both packed calls back to back (gated W, U per chunk; then state passing and output per sequence) against the
+    token-by-token gated delta rule run on every sequence by itself, each with its own initial and final state."""
+    C = 64
+    lens = [130, 64, 5, 1, 200, 63, 65, 128]
+    H_k, H_v = 2, 4
+    K, V, beta, g, graw, cu = _packed_inputs(lens, H_k, H_v, C, seed=600)
+    T = int(cu[-1])
+    Q = _queries(H_k, T, 601)
+    scale = 128 ** -0.5
+    S0 = 0.1 * torch.randn(len(lens), H_v, 128, 128, generator=torch.Generator().manual_seed(602)) if with_state else None
+    gates = graw if raw else g
+    flags = gdn.GDN_FLAG_W_GATED | (gdn.GDN_FLAG_G_RAW if raw else 0)
+    W, U, _, _, _ = gdn.chunk_prepare_varlen(K.cuda(), V.cuda(), beta.cuda(), gates.cuda(), cu, C, flags=flags, want_tinv=False)
+    O, S = gdn.chunk_state_output_varlen(Q.cuda(), K.cuda(), W, U, gates.cuda(), cu, C, scale,
+                                         None if S0 is None else S0.cuda(), flags=gdn.GDN_FLAG_G_RAW if raw else 0)
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+    assert bool(torch.isfinite(O).all()) and bool(torch.isfinite(S).all())
+    for s_, L in enumerate(lens):
+        a = int(cu[s_])
+        for hv in range(H_v):
+            hk = hv // (H_v // H_k)
+            Oo, So = orc.gated_delta_rule(Q[hk, a:a + L].double().numpy(), K[hk, a:a + L].double().numpy(),
+                                          V[hv, a:a + L].double().numpy(), beta[hv, a:a + L].double().numpy(),
+                                          graw[hv, a:a + L].double().numpy(), scale,
+                                          None if S0 is None else S0[s_, hv].double().numpy())
+            eO = orc.rel_frobenius(O[hv, a:a + L].double().cpu().numpy()[None], Oo[None])
+            assert eO.max() <= 1e-2, f"sequence {s_} (len {L}) head {hv}: O rel-F {eO.max():.3e}"
+            eS = orc.rel_frobenius(S[s_, hv].double().cpu().numpy()[None], So[None])
+            assert eS.max() <= 1e-2, f"sequence {s_} (len {L}) head {hv}: S rel-F {eS.max():.3e}"
+
+
+def test_packed_state_output_matches_oracle_on_the_same_w_u():
+    """The state / output step alone: the oracle gets the bf16 W, U the first call produced (padded per sequence)."""
+    C = 64
+    lens = [100, 64, 7, 191]
+    K, V, beta, g, graw, cu = _packed_inputs(lens, 1, 2, C, seed=610)
+    T = int(cu[-1])
+    Q = _queries(1, T, 611)
+    scale = 128 ** -0.5
+    W, U, _, _, _ = gdn.chunk_prepare_varlen(K.cuda(), V.cuda(), beta.cuda(), g.cuda(), cu, C, flags=gdn.GDN_FLAG_W_GATED,
+                                             want_tinv=False)
+    O, S = gdn.chunk_state_output_varlen(Q.cuda(), K.cuda(), W, U, g.cuda(), cu, C, scale)
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+    for s_, L in enumerate(lens):
+        a = int(cu[s_])
+        Lp = -(-L // C) * C
+        for hv in range(2):
+            def pad(x):
+                out = np.zeros((Lp,) + tuple(x.shape[1:]))
+                out[:L] = x[a:a + L].double().cpu().numpy()
+                return out
+            gp = pad(g[hv])
+            gp[L:] = gp[L - 1]
+            Oo, So = orc.chunk_state_output(pad(Q[0]), pad(K[0]), pad(W[hv]), pad(U[hv]), gp, C, scale)
+            eO = orc.rel_frobenius(O[hv, a:a + L].double().cpu().numpy()[None], Oo[None, :L])
+            assert eO.max() <= 2.2e-3, f"sequence {s_} head {hv}: O rel-F {eO.max():.3e}"
+            eS = orc.rel_frobenius(S[s_, hv].double().cpu().numpy()[None], So[None])
+            assert eS.max() <= 1e-4, f"sequence {s_} head {hv}: S rel-F {eS.max():.3e}"
+    # rows of O past the last sequence stay untouched (none here), and nothing wrote outside [0, T)
+    assert O.shape == (2, T, 128)
