@@ -21,6 +21,8 @@
 //     O^T = scale (exp(g_i) O1 + O2)  -> transposed through shared memory -> bulk tensor store
 // Two MMA groups per chunk; Q, K, W, U tiles of the next chunk are in flight (two stages) while a chunk is worked on.
 // All operand layouts are the ones the chunk-prepare kernel uses.
+// Packed variable-length sequences (second instantiation): one CTA per (sequence, value head), starting at the
+// sequence's first token; the tokens a short last chunk lacks decay nothing and write nothing.
 #include <cuda.h>
 
 #include "common.cuh"
