@@ -109,7 +109,7 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 
     // One mbarrier per MMA group (never two pending phases on one barrier), two per-stage TMA barriers, and two
     // barriers on which the 256 compute threads tell the issuing warp that operands are in place.
-    __shared__ uint64_t bar_full[2], bar_pre, bar_d1, bar_o1, bar_o2, bar_g2, bar_rdy_a, bar_rdy_2;
+    __shared__ uint64_t bar_full[2], bar_pre, bar_d1, bar_o2, bar_g2, bar_rdy_a, bar_rdy_2;
     __shared__ uint32_t tmem_base_s;
     __shared__ int s_fail;
 
@@ -130,7 +130,6 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         mbar_init(&bar_full[1], 1);
         mbar_init(&bar_pre, 1);
         mbar_init(&bar_d1, 1);
-        mbar_init(&bar_o1, 1);
         mbar_init(&bar_o2, 1);
         mbar_init(&bar_g2, 1);
         mbar_init(&bar_rdy_a, kThreads);
@@ -250,7 +249,8 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                         mma_f16_ts(tmem + kO1, tmem + (part == 0 ? kSA : kO2) + ks * 8, bd, idesc_kk64, part > 0 || ks > 0);
                     }
                 }
-                mma_commit(&bar_o1);
+                // (no completion barrier of its own: the commit behind the output product below covers it, and a wait
+                // costs the threads ~200 cycles even on a completed phase)
             }
             __syncwarp();
             STAMPS(102);
@@ -293,16 +293,16 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         }
     } else {
         // ================= compute threads (512): four per TMEM lane
-        uint32_t par_pre = 0, par_d1 = 0, par_o1 = 0, par_o2 = 0, par_g2 = 0;
-        // completion of an MMA group: warp 0 polls the mbarrier, the other warps sleep on a hardware barrier
-        // completion of an MMA group: lane 0 of every warp polls the mbarrier (no CTA-wide barrier on this path)
+        uint32_t par_pre = 0, par_d1 = 0, par_o2 = 0, par_g2 = 0;
+        // completion of an MMA group: every lane polls the mbarrier (no CTA-wide barrier on this path). A poll of a
+        // completed phase costs ~200 cycles whoever issues it; polling from lane 0 alone added a divergent branch and a
+        // shuffle, ~150 cycles more per wait.
         auto wait_group = [&](uint64_t* bar, uint32_t& par) -> bool {
-            int good = 1;
-            if (lane == 0 && !wait_bar(bar, par)) { *fail = 1; good = 0; }
-            good = __shfl_sync(0xFFFFFFFFu, good, 0);
+            const bool good = wait_bar(bar, par);
+            if (!good) *fail = 1;
             par ^= 1;
             tc_fence_after_sync();
-            return good != 0;
+            return good;
         };
         // ---- constant A operand -I, initial state, and its bf16 copies (hi in kSA, lo in kO2)
         {
@@ -336,12 +336,16 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         // gates of the first chunk
         float g_reg = 0.f;
         // (a short last chunk: tokens past the sequence's end decay nothing and write nothing)
-        if (n_c > 0 && tid < 64) g_reg = (!VAR || tid < len) ? __ldg(gseq + tid) : 0.f;
+        // The gate tables are the job of threads 64..127: their lanes hold no row of P, so they are idle while the other
+        // half of the CTA forms P.
+        const int tt = tid - 64;  // token of a table thread
+        const bool tabler = tt >= 0 && tt < 64;
+        if (n_c > 0 && tabler) g_reg = (!VAR || tt < len) ? __ldg(gseq + tt) : 0.f;
         bool ok = true;
         // gate tables of a chunk: written by 64 threads into the buffer of that chunk one barrier before they are read
         const bool g_raw = (p.flags & GDN_FLAG_G_RAW) != 0;
         auto fill_tables = [&](int c) {
-            if (tid < 64) {
+            if (tabler) {
                 float* tb = gtab + (c & 1) * 192;
                 float gc = g_reg;
                 const int left = len - c * kC;  // tokens of this chunk (>= 64 except for a short last chunk)
@@ -352,23 +356,23 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                         const float v = __shfl_up_sync(0xFFFFFFFFu, gc, off);
                         if (lane >= off) gc += v;
                     }
-                    if (tid == 31) tb[128 + 63] = gc;  // ... and the first warp's total through the table itself
+                    if (tt == 31) tb[128 + 63] = gc;  // ... and the first warp's total through the table itself
                     asm volatile("bar.sync 3, 64;" ::: "memory");
-                    if (tid >= 32) gc += tb[128 + 63];
+                    if (tt >= 32) gc += tb[128 + 63];
                     asm volatile("bar.sync 3, 64;" ::: "memory");
                 }
-                tb[128 + tid] = gc;
+                tb[128 + tt] = gc;
                 asm volatile("bar.sync 3, 64;" ::: "memory");
                 if (VAR && !g_raw && left < kC) {
                     // cumulative gates: tokens past the end keep the gate of the last real token
-                    gc = tb[128 + (tid < left ? tid : left - 1)];
+                    gc = tb[128 + (tt < left ? tt : left - 1)];
                     asm volatile("bar.sync 3, 64;" ::: "memory");
-                    tb[128 + tid] = gc;
+                    tb[128 + tt] = gc;
                     asm volatile("bar.sync 3, 64;" ::: "memory");
                 }
                 const float gC = tb[128 + 63];  // cumulative gate of the chunk's last token
-                tb[tid] = fast_exp2(gc * kLog2e);
-                tb[64 + tid] = fast_exp2((gC - gc) * kLog2e);
+                tb[tt] = fast_exp2(gc * kLog2e);
+                tb[64 + tt] = fast_exp2((gC - gc) * kLog2e);
             }
         };
         if (n_c > 0) fill_tables(0);
@@ -380,7 +384,7 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             const float gC = sg[63];
             const int left = len - c * kC;
             const bool short_chunk = VAR && left < kC;
-            if (c + 1 < n_c && tid < 64) g_reg = (!VAR || (c + 1) * kC + tid < len) ? __ldg(gseq + (c + 1) * kC + tid) : 0.f;
+            if (c + 1 < n_c && tabler) g_reg = (!VAR || (c + 1) * kC + tt < len) ? __ldg(gseq + (c + 1) * kC + tt) : 0.f;
             STAMPS(1);
 
             STAMPS(2);
@@ -429,6 +433,8 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                     *reinterpret_cast<uint4*>(smem + kOffP + 8192 + (h * 2 + c2) * 1024 + t * 16) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
                 }
             }
+            // the next chunk's gate tables, by threads that had no part in P (published by the barrier at the chunk's end)
+            if (c + 1 < n_c) fill_tables(c + 1);
             // ---- U_new^T = -D1 as bf16 hi + lo, plain and gate-scaled (the sums over the tokens of a chunk telescope
             // on correlated keys, so single bf16 copies cost 1e-2 there). This thread's 16 tokens are one k-step of the
             // products that consume them: the hi halves are written over its own D1 columns (plain -> 16 h .. 16 h + 7,
@@ -463,8 +469,8 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             mbar_arrive(&bar_rdy_2);
             STAMPS(7);
 
-            // ---- exp(g_i) O1
-            if (!wait_group(&bar_o1, par_o1)) { ok = false; break; }
+            // ---- exp(g_i) O1 (complete with O2: products finish in the order they were issued)
+            if (!wait_group(&bar_o2, par_o2)) { ok = false; break; }
             STAMPS(8);
             float o[16];
             {
@@ -474,8 +480,6 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 #pragma unroll
                 for (int i = 0; i < 16; ++i) o[i] = __uint_as_float(d[i]) * se[h * 16 + i];
             }
-            STAMPS(9);
-            if (!wait_group(&bar_o2, par_o2)) { ok = false; break; }
             STAMPS(10);
             // ---- O^T = scale (exp(g_i) O1 + O2): element (token i, feature t) of the staged tile
             {
@@ -511,7 +515,6 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 mbar_arrive(&bar_rdy_a);
             }
             STAMPS(11);
-            if (c + 1 < n_c) fill_tables(c + 1);
             fence_proxy_async_smem();
             // the store of the previous chunk has finished reading its staging buffer, which the next chunk writes
             // (issued a whole chunk ago: this never waits in practice; the barrier below publishes it)
