@@ -97,6 +97,18 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity) {
     return true;
 }
 
+// Hand-off from the 512 compute threads to the issuing warp over a hardware barrier: the threads arrive and go on, the
+// issuing warp waits. (An mbarrier poll costs the waiting warp ~200-300 cycles per hand-off on the chain of the
+// sequence; this is a few tens.) The wait has no bound of its own: threads whose own bounded waits run out arrive on both hand-offs before they leave.
+template <int ID>
+__device__ __forceinline__ void handoff_arrive() {
+    asm volatile("bar.arrive %0, %1;" ::"n"(ID), "n"(kThreads + 32) : "memory");
+}
+template <int ID>
+__device__ __forceinline__ void handoff_wait() {
+    asm volatile("bar.sync %0, %1;" ::"n"(ID), "n"(kThreads + 32) : "memory");
+}
+
 // VAR: packed variable-length sequences (own instantiation: its masks sit on the chain the dense case is bound by)
 template <bool VAR>
 __global__ void __launch_bounds__(kThreads + 64, 1)
@@ -109,7 +121,7 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 
     // One mbarrier per MMA group (never two pending phases on one barrier), two per-stage TMA barriers, and two
     // barriers on which the 256 compute threads tell the issuing warp that operands are in place.
-    __shared__ uint64_t bar_full[2], bar_pre, bar_d1, bar_o2, bar_g2, bar_rdy_a, bar_rdy_2;
+    __shared__ uint64_t bar_full[2], bar_pre, bar_d1, bar_o2, bar_g2;
     __shared__ uint32_t tmem_base_s;
     __shared__ int s_fail;
 
@@ -132,8 +144,6 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         mbar_init(&bar_d1, 1);
         mbar_init(&bar_o2, 1);
         mbar_init(&bar_g2, 1);
-        mbar_init(&bar_rdy_a, kThreads);
-        mbar_init(&bar_rdy_2, kThreads);
         s_fail = 0;
         mbar_fence_init();
         tma_prefetch_desc(&tmQ);
@@ -219,13 +229,11 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             }
             __syncwarp();
         };
-        uint32_t par_a = 0, par_2 = 0;
         for (int c = 0; c < n_c && *fail == 0; ++c) {
             const uint32_t st_a = smem_a + (c & 1) * kStageBytes;
             // the state copies (and, for the first chunk, the constant operand) are in place
             STAMPS(100);
-            if (!wait_bar(&bar_rdy_a, par_a)) *fail = 1;
-            par_a ^= 1;
+            handoff_wait<4>();
             STAMPS(101);
             tc_fence_after_sync();
             if (c == 0) issue_pre(0);
@@ -255,8 +263,7 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             __syncwarp();
             STAMPS(102);
             // U_new^T (hi, lo; plain, scaled), P (hi, lo) and the decayed accumulator are in place
-            if (!wait_bar(&bar_rdy_2, par_2)) *fail = 1;
-            par_2 ^= 1;
+            handoff_wait<5>();
             STAMPS(103);
             tc_fence_after_sync();
             if (*fail == 0 && elect_one()) {
@@ -331,7 +338,7 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             }
             tmem_wait_st();
             tc_fence_before_sync();
-            mbar_arrive(&bar_rdy_a);
+            handoff_arrive<4>();
         }
         // gates of the first chunk
         float g_reg = 0.f;
@@ -413,6 +420,12 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 tmem_ld16(lane_base + kPT + h * 16, d);
                 tmem_wait_ld();
                 const float gj = sg[t] * kLog2e;
+                float gi16[16];  // g of this thread's 16 columns (four 16-byte loads instead of sixteen scalar ones)
+#pragma unroll
+                for (int i4 = 0; i4 < 4; ++i4) {
+                    const float4 q4 = *reinterpret_cast<const float4*>(sg + h * 16 + i4 * 4);
+                    gi16[i4 * 4 + 0] = q4.x; gi16[i4 * 4 + 1] = q4.y; gi16[i4 * 4 + 2] = q4.z; gi16[i4 * 4 + 3] = q4.w;
+                }
 #pragma unroll
                 for (int c2 = 0; c2 < 2; ++c2) {
                     uint32_t w[4], wl[4];
@@ -422,7 +435,8 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 #pragma unroll
                         for (int q = 0; q < 2; ++q) {
                             const int i = h * 16 + c2 * 8 + i2 * 2 + q;
-                            const float x = __uint_as_float(d[c2 * 8 + i2 * 2 + q]) * fast_exp2(fminf(fmaf(sg[i], kLog2e, -gj), 0.f));
+                            const float x = __uint_as_float(d[c2 * 8 + i2 * 2 + q]) *
+                                            fast_exp2(fminf(fmaf(gi16[c2 * 8 + i2 * 2 + q], kLog2e, -gj), 0.f));
                             v[q] = (t <= i) ? x : 0.f;
                         }
                         w[i2] = pack_bf16x2(v[0], v[1]);
@@ -447,14 +461,20 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 tmem_wait_ld();
                 uint32_t hi[16], lo[16];
 #pragma unroll
+                float f16[16];
+#pragma unroll
+                for (int i4 = 0; i4 < 4; ++i4) {
+                    const float4 q4 = *reinterpret_cast<const float4*>(sf + h * 16 + i4 * 4);
+                    f16[i4 * 4 + 0] = q4.x; f16[i4 * 4 + 1] = q4.y; f16[i4 * 4 + 2] = q4.z; f16[i4 * 4 + 3] = q4.w;
+                }
+#pragma unroll
                 for (int i = 0; i < 8; ++i) {
                     float u0 = -__uint_as_float(d[2 * i]), u1 = -__uint_as_float(d[2 * i + 1]);
                     if (short_chunk) {  // rows past the sequence's end hold another sequence's W, U
                         if (h * 16 + 2 * i >= left) u0 = 0.f;
                         if (h * 16 + 2 * i + 1 >= left) u1 = 0.f;
                     }
-                    const float2 f = *reinterpret_cast<const float2*>(sf + h * 16 + 2 * i);
-                    const float s0 = u0 * f.x, s1 = u1 * f.y;
+                    const float s0 = u0 * f16[2 * i], s1 = u1 * f16[2 * i + 1];
                     hi[i] = pack_bf16x2(u0, u1);
                     hi[8 + i] = pack_bf16x2(s0, s1);
                     lo[i] = pack_bf16x2(u0 - bf16_lo(hi[i]), u1 - bf16_hi(hi[i]));
@@ -466,7 +486,7 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             fence_proxy_async_smem();
             tmem_wait_st();
             tc_fence_before_sync();
-            mbar_arrive(&bar_rdy_2);
+            handoff_arrive<5>();
             STAMPS(7);
 
             // ---- exp(g_i) O1 (complete with O2: products finish in the order they were issued)
@@ -478,7 +498,13 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 tmem_ld16(lane_base + kO1 + h * 16, d);
                 tmem_wait_ld();
 #pragma unroll
-                for (int i = 0; i < 16; ++i) o[i] = __uint_as_float(d[i]) * se[h * 16 + i];
+                for (int i4 = 0; i4 < 4; ++i4) {
+                    const float4 e4 = *reinterpret_cast<const float4*>(se + h * 16 + i4 * 4);
+                    o[i4 * 4 + 0] = __uint_as_float(d[i4 * 4 + 0]) * e4.x;
+                    o[i4 * 4 + 1] = __uint_as_float(d[i4 * 4 + 1]) * e4.y;
+                    o[i4 * 4 + 2] = __uint_as_float(d[i4 * 4 + 2]) * e4.z;
+                    o[i4 * 4 + 3] = __uint_as_float(d[i4 * 4 + 3]) * e4.w;
+                }
             }
             STAMPS(10);
             // ---- O^T = scale (exp(g_i) O1 + O2): element (token i, feature t) of the staged tile
@@ -512,7 +538,7 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 tmem_st16(lane_base + kO2 + h * 16, pk);
                 tmem_wait_st();
                 tc_fence_before_sync();
-                mbar_arrive(&bar_rdy_a);
+                handoff_arrive<4>();
             }
             STAMPS(11);
             fence_proxy_async_smem();
@@ -533,6 +559,11 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 tma_store_3d(&tmO, smem + kOffO + (c & 1) * kTileBytes + 8192, 64, tok0 + c * kC, bhv);
                 tma_store_commit();
             }
+        }
+        if (!ok) {
+            // a bounded wait ran out (s_fail is set): release the issuing warp from whichever hand-off it waits on
+            handoff_arrive<4>();
+            handoff_arrive<5>();
         }
         // ---- final state
         if (ok && p.S_out != nullptr) {
