@@ -54,8 +54,8 @@ constexpr int kStageBytes = 4 * kTileBytes;  // Q, K, W, U
 constexpr int kOffQ = 0, kOffK = kTileBytes, kOffW = 2 * kTileBytes, kOffU = 3 * kTileBytes;
 constexpr int kOffP = 2 * kStageBytes;       // 2 x 8 KB: P as B operand [64 x 64] (MN-major, no swizzle), hi and lo halves
 constexpr int kOffO = kOffP + 16384;          // 2 x 16 KB: O tile staged for the bulk store (128B swizzle), two buffers
-constexpr int kOffG = kOffO + 2 * kTileBytes;  // 2 x 3 x 64 floats: exp(g_i), exp(g_C - g_j), g; two buffers
-constexpr int kSmemTotal = kOffG + 2 * 3 * 64 * 4;
+constexpr int kOffG = kOffO + 2 * kTileBytes;  // 3 x 3 x 64 floats: exp(g_i), exp(g_C - g_j), g; three buffers
+constexpr int kSmemTotal = kOffG + 3 * 3 * 64 * 4;
 
 #ifdef GDN_TRACE
 __device__ long long g_trace_s[4096];
@@ -121,7 +121,7 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 
     // One mbarrier per MMA group (never two pending phases on one barrier), two per-stage TMA barriers, and two
     // barriers on which the 256 compute threads tell the issuing warp that operands are in place.
-    __shared__ uint64_t bar_full[2], bar_pre, bar_d1, bar_o2, bar_g2;
+    __shared__ uint64_t bar_full[2], bar_pre, bar_d1, bar_o2, bar_g2, bar_stg[2];
     __shared__ uint32_t tmem_base_s;
     __shared__ int s_fail;
 
@@ -144,6 +144,8 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         mbar_init(&bar_d1, 1);
         mbar_init(&bar_o2, 1);
         mbar_init(&bar_g2, 1);
+        mbar_init(&bar_stg[0], 1);
+        mbar_init(&bar_stg[1], 1);
         s_fail = 0;
         mbar_fence_init();
         tma_prefetch_desc(&tmQ);
@@ -175,32 +177,49 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     volatile int* fail = reinterpret_cast<volatile int*>(&s_fail);
 
     if (producer) {
-        // ================= loading warp: the four tiles of chunk c into stage c & 1, as soon as the products that
-        // read the stage's previous tiles are complete
-        if (elect_one()) {
-            auto load_stage = [&](int c) {
-                uint8_t* st = smem + (c & 1) * kStageBytes;
-                uint64_t* bar = &bar_full[c & 1];
-                mbar_arrive_expect_tx(bar, kStageBytes);
-                const int t0 = tok0 + c * kC;
-                tma_load_3d(st + kOffQ, &tmQ, bar, 0, t0, bhk);
-                tma_load_3d(st + kOffQ + 8192, &tmQ, bar, 64, t0, bhk);
-                tma_load_3d(st + kOffK, &tmK, bar, 0, t0, bhk);
-                tma_load_3d(st + kOffK + 8192, &tmK, bar, 64, t0, bhk);
-                tma_load_3d(st + kOffW, &tmW, bar, 0, t0, bhv);
-                tma_load_3d(st + kOffW + 8192, &tmW, bar, 64, t0, bhv);
-                tma_load_3d(st + kOffU, &tmU, bar, 0, t0, bhv);
-                tma_load_3d(st + kOffU + 8192, &tmU, bar, 64, t0, bhv);
-            };
+        // ================= loading / storing warp: the four tiles of chunk c into stage c & 1, as soon as the products
+        // that read the stage's previous tiles are complete; and the bulk stores of the staged output tiles, so that
+        // no compute thread waits for the others at the end of a chunk
+        const bool lead = elect_one();
+        auto load_stage = [&](int c) {
+            uint8_t* st = smem + (c & 1) * kStageBytes;
+            uint64_t* bar = &bar_full[c & 1];
+            mbar_arrive_expect_tx(bar, kStageBytes);
+            const int t0 = tok0 + c * kC;
+            tma_load_3d(st + kOffQ, &tmQ, bar, 0, t0, bhk);
+            tma_load_3d(st + kOffQ + 8192, &tmQ, bar, 64, t0, bhk);
+            tma_load_3d(st + kOffK, &tmK, bar, 0, t0, bhk);
+            tma_load_3d(st + kOffK + 8192, &tmK, bar, 64, t0, bhk);
+            tma_load_3d(st + kOffW, &tmW, bar, 0, t0, bhv);
+            tma_load_3d(st + kOffW + 8192, &tmW, bar, 64, t0, bhv);
+            tma_load_3d(st + kOffU, &tmU, bar, 0, t0, bhv);
+            tma_load_3d(st + kOffU + 8192, &tmU, bar, 64, t0, bhv);
+        };
+        if (lead) {
             if (n_c > 0) load_stage(0);
             if (n_c > 1) load_stage(1);
-            uint32_t par = 0;
-            for (int c = 0; c + 2 < n_c && *fail == 0; ++c) {
-                if (!wait_bar(&bar_g2, par)) *fail = 1;
-                par ^= 1;
-                if (*fail == 0) load_stage(c + 2);
-            }
         }
+        uint32_t par = 0;
+        for (int c = 0; c < n_c && *fail == 0; ++c) {
+            // the staged output tile of chunk c is complete (every compute thread has arrived)
+            handoff_wait<6>();
+            if (lead && *fail == 0) {
+                if (!(VAR && len - c * kC < kC)) {  // (a short last chunk is stored row by row by the compute threads)
+                    tma_store_3d(&tmO, smem + kOffO + (c & 1) * kTileBytes, 0, tok0 + c * kC, bhv);
+                    tma_store_3d(&tmO, smem + kOffO + (c & 1) * kTileBytes + 8192, 64, tok0 + c * kC, bhv);
+                    tma_store_commit();
+                    tma_store_wait_read<0>();
+                }
+                mbar_arrive(&bar_stg[c & 1]);  // the staging buffer may be written again (chunk c + 2)
+                if (c + 2 < n_c) {
+                    if (!wait_bar(&bar_g2, par)) *fail = 1;
+                    if (*fail == 0) load_stage(c + 2);
+                }
+            }
+            par ^= 1;
+            __syncwarp();
+        }
+        if (lead) tma_store_wait_all<0>();
         __syncwarp();
     } else if (issuer) {
         // ================= issuing warp: every tcgen05.mma, in the order the tensor pipe runs them
@@ -353,7 +372,7 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         const bool g_raw = (p.flags & GDN_FLAG_G_RAW) != 0;
         auto fill_tables = [&](int c) {
             if (tabler) {
-                float* tb = gtab + (c & 1) * 192;
+                float* tb = gtab + (c % 3) * 192;
                 float gc = g_reg;
                 const int left = len - c * kC;  // tokens of this chunk (>= 64 except for a short last chunk)
                 if (g_raw) {
@@ -385,7 +404,7 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         if (n_c > 0) fill_tables(0);
         asm volatile("bar.sync 1, 512;" ::: "memory");
         for (int c = 0; c < n_c; ++c) {
-            const float* se = gtab + (c & 1) * 192;  // exp(g_i)
+            const float* se = gtab + (c % 3) * 192;  // exp(g_i)
             const float* sf = se + 64;               // exp(g_C - g_j)
             const float* sg = se + 128;              // g_i (cumulative inside the chunk)
             const float gC = sg[63];
@@ -489,6 +508,9 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             handoff_arrive<5>();
             STAMPS(7);
 
+            // the bulk store of chunk c - 2 has finished reading this chunk's staging buffer (polled here, in the shadow of
+            // the output product)
+            if (c >= 2 && !wait_bar(&bar_stg[c & 1], ((c - 2) >> 1) & 1)) { *fail = 1; ok = false; break; }
             // ---- exp(g_i) O1 (complete with O2: products finish in the order they were issued)
             if (!wait_group(&bar_o2, par_o2)) { ok = false; break; }
             STAMPS(8);
@@ -521,6 +543,9 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                     *reinterpret_cast<__nv_bfloat16*>(sub + tok * 128 + ((cch ^ (tok & 7)) << 4) + (t & 7) * 2) = v;
                 }
             }
+            // the tile goes to the storing warp: no compute thread waits for the others here
+            fence_proxy_async_smem();
+            handoff_arrive<6>();
             // ---- bf16 copies (hi, lo) of the new state for the next chunk's products; the lo half goes where O2 was
             // (this thread has read its O2 columns above)
             if (!wait_group(&bar_g2, par_g2)) { ok = false; break; }
@@ -541,29 +566,23 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 handoff_arrive<4>();
             }
             STAMPS(11);
-            fence_proxy_async_smem();
-            // the store of the previous chunk has finished reading its staging buffer, which the next chunk writes
-            // (issued a whole chunk ago: this never waits in practice; the barrier below publishes it)
-            if (tid == 0) tma_store_wait_read<0>();
-            asm volatile("bar.sync 1, 512;" ::: "memory");  // the staged output tile and the next gate tables are complete
             if (short_chunk) {
                 // only the rows of real tokens leave, 16 bytes per thread and step, from the staged (swizzled) tile
+                asm volatile("bar.sync 1, 512;" ::: "memory");  // (last chunk of a packed sequence only)
                 for (int q = tid; q < left * 16; q += kThreads) {
                     const int tok = q >> 4, ch = q & 15;  // 16-byte piece ch of the token's 256-byte row
                     const uint4 v = *reinterpret_cast<const uint4*>(smem + kOffO + (c & 1) * kTileBytes + (ch >> 3) * 8192 +
                                                                     tok * 128 + (((ch & 7) ^ (tok & 7)) << 4));
                     *reinterpret_cast<uint4*>(p.O + ((long long)bhv * p.T + tok0 + c * kC + tok) * kD + ch * 8) = v;
                 }
-            } else if (tid == 0) {  // the same thread waits for these stores (bulk groups are per thread)
-                tma_store_3d(&tmO, smem + kOffO + (c & 1) * kTileBytes, 0, tok0 + c * kC, bhv);
-                tma_store_3d(&tmO, smem + kOffO + (c & 1) * kTileBytes + 8192, 64, tok0 + c * kC, bhv);
-                tma_store_commit();
             }
         }
         if (!ok) {
-            // a bounded wait ran out (s_fail is set): release the issuing warp from whichever hand-off it waits on
+            // a bounded wait ran out (s_fail is set): release the issuing and the storing warp from whichever hand-off
+            // they wait on (both leave their loops when they see s_fail)
             handoff_arrive<4>();
             handoff_arrive<5>();
+            handoff_arrive<6>();
         }
         // ---- final state
         if (ok && p.S_out != nullptr) {
@@ -577,7 +596,6 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                     make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]), __uint_as_float(v[4 * i + 2]),
                                 __uint_as_float(v[4 * i + 3]));
         }
-        if (tid == 0) tma_store_wait_all<0>();
     }
     tc_fence_before_sync();
     __syncthreads();
