@@ -179,7 +179,9 @@ int gdn_chunk_prepare_varlen(const void* K, const void* V, const float* beta, co
  * U = T diag(beta) V.
  *   Q, K [B,H_k,T,d_k], W_gated [B,H_v,T,d_k], U [B,H_v,T,d_v] bf16; g [B,H_v,T] fp32, the cumulative log-gate
  *   that RESTARTS in every chunk (chunk-local inclusive prefix sum), or with flags = GDN_FLAG_G_RAW the raw per-token
- *   log-gates (the prefix sum is then formed here, as gdn_chunk_prepare_ex does); no other flag is accepted; S_in [B,H_v,d_v,d_k] fp32 or NULL (zero state);
+ *   log-gates (the prefix sum is then formed here, as gdn_chunk_prepare_ex does); with GDN_FLAG_LAYOUT_BTHD the
+ *   tensors are token-major: Q, K [B,T,H_k,d_k], W_gated, U, O_out [B,T,H_v,d], g [B,T,H_v] (the state keeps its
+ *   layout); no other flag is accepted; S_in [B,H_v,d_v,d_k] fp32 or NULL (zero state);
  *   O_out [B,H_v,T,d_v] bf16; S_out [B,H_v,d_v,d_k] fp32 or NULL.
  * Supported: C = 64, d_k = d_v = 128, T a multiple of C. fp32 state, bf16 tensor-core operands.
  */
@@ -195,7 +197,8 @@ int gdn_chunk_state_output(const void* Q, const void* K, const void* W_gated, co
  *   Q, K [H_k,T_total,d_k], W_gated [H_v,T_total,d_k], U [H_v,T_total,d_v] bf16; g [H_v,T_total] (restarting in every
  *   chunk of every sequence, or raw with GDN_FLAG_G_RAW); cu_seqlens: DEVICE array of n_seq + 1 int32, non-decreasing,
  *   cu_seqlens[n_seq] <= T_total; S_in, S_out [n_seq,H_v,d_v,d_k] fp32 (either may be NULL); O_out [H_v,T_total,d_v].
- * Supported: C = 64, d_k = d_v = 128, head-major tensors.
+ *   With GDN_FLAG_LAYOUT_BTHD: Q, K [T_total,H_k,d_k], W_gated, U, O_out [T_total,H_v,d], g [T_total,H_v].
+ * Supported: C = 64, d_k = d_v = 128.
  */
 int gdn_chunk_state_output_varlen(const void* Q, const void* K, const void* W_gated, const void* U, const float* g,
                                   const int32_t* cu_seqlens, int n_seq, int T_total, int H_k, int H_v, int C,

@@ -324,11 +324,15 @@ def gdn_chunk_state_output_varlen(Q, K, W_gated, U, g, cu_seqlens, n_seq, T_tota
 def chunk_state_output_varlen(Q, K, W_gated, U, g, cu_seqlens, C, scale=1.0, S_in=None, *, want_state=True, flags=0):
     """Packed sequences: Q, K [H_k,T,d_k], W_gated [H_v,T,d_k], U [H_v,T,d_v], g [H_v,T]; cu_seqlens on the host.
     Returns (O [H_v,T,d_v], S_out [n_seq,H_v,d_v,d_k] fp32 or None); rows of O that no sequence covers stay zero."""
-    H_k, T, d_k = K.shape
-    H_v, _, d_v = U.shape
+    if flags & GDN_FLAG_LAYOUT_BTHD:  # token-major: [T, H, d]
+        T, H_k, d_k = K.shape
+        _, H_v, d_v = U.shape
+    else:
+        H_k, T, d_k = K.shape
+        H_v, _, d_v = U.shape
     cu = torch.tensor([int(x) for x in cu_seqlens], dtype=torch.int32, device=U.device)
     n_seq = cu.numel() - 1
-    O = torch.zeros(H_v, T, d_v, dtype=U.dtype, device=U.device)
+    O = torch.zeros_like(U)
     S_out = torch.empty(n_seq, H_v, d_v, d_k, dtype=torch.float32, device=U.device) if want_state else None
     gdn_chunk_state_output_varlen(Q, K, W_gated, U, g, cu, n_seq, T, H_k, H_v, C, d_k, d_v, scale, S_in, O, S_out, flags)
     return O, S_out
@@ -337,10 +341,14 @@ def chunk_state_output_varlen(Q, K, W_gated, U, g, cu_seqlens, C, scale=1.0, S_i
 def chunk_state_output(Q, K, W_gated, U, g, C, scale=1.0, S_in=None, *, want_state=True, outputs=None, flags=0):
     """Convenience wrapper: Q, K [B,H_k,T,d_k], W_gated [B,H_v,T,d_k], U [B,H_v,T,d_v], g [B,H_v,T] (chunk-local
     cumulative log-gate). Returns (O [B,H_v,T,d_v], S_out [B,H_v,d_v,d_k] fp32 or None)."""
-    B, H_k, T, d_k = K.shape
-    _, H_v, _, d_v = U.shape
+    if flags & GDN_FLAG_LAYOUT_BTHD:  # token-major: [B, T, H, d]
+        B, T, H_k, d_k = K.shape
+        _, _, H_v, d_v = U.shape
+    else:
+        B, H_k, T, d_k = K.shape
+        _, H_v, _, d_v = U.shape
     if outputs is None:
-        O = torch.empty(B, H_v, T, d_v, dtype=U.dtype, device=U.device)
+        O = torch.empty_like(U)
         S_out = torch.empty(B, H_v, d_v, d_k, dtype=torch.float32, device=U.device) if want_state else None
     else:
         O, S_out = outputs

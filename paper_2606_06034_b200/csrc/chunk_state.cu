@@ -171,8 +171,16 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     const int len = VAR ? __ldg(p.cu_seqlens + b + 1) - tok0 : p.T;
     const int bhv = VAR ? hv : blockIdx.x;
     const int bhk = VAR ? hv / p.group : b * p.H_k + hv / p.group;
+    // Token-major tensors [B, T, H, d] (GDN_FLAG_LAYOUT_BTHD) are seen by TMA as (H * d, T, B): the head picks the first
+    // column of a box, the batch its outermost index; consecutive tokens of g are H_v apart.
+    const bool bthd = (p.flags & GDN_FLAG_LAYOUT_BTHD) != 0;
+    const int bz = VAR ? 0 : b;
+    const int kx = bthd ? (hv / p.group) * kD : 0, kz = bthd ? bz : bhk;  // Q, K boxes
+    const int vx = bthd ? hv * kD : 0, vz = bthd ? bz : bhv;              // W, U, O boxes
+    const long long grow0 = bthd ? ((long long)bz * p.T + tok0) * p.H_v + hv : (long long)bhv * p.T + tok0;  // first token's row
+    const int gstep = bthd ? p.H_v : 1;
     const int n_c = (len + kC - 1) / kC;
-    const float* gseq = p.g + (long long)bhv * p.T + tok0;
+    const float* gseq = p.g + grow0;
     const uint32_t smem_a = smem_u32(smem);
     volatile int* fail = reinterpret_cast<volatile int*>(&s_fail);
 
@@ -186,14 +194,14 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             uint64_t* bar = &bar_full[c & 1];
             mbar_arrive_expect_tx(bar, kStageBytes);
             const int t0 = tok0 + c * kC;
-            tma_load_3d(st + kOffQ, &tmQ, bar, 0, t0, bhk);
-            tma_load_3d(st + kOffQ + 8192, &tmQ, bar, 64, t0, bhk);
-            tma_load_3d(st + kOffK, &tmK, bar, 0, t0, bhk);
-            tma_load_3d(st + kOffK + 8192, &tmK, bar, 64, t0, bhk);
-            tma_load_3d(st + kOffW, &tmW, bar, 0, t0, bhv);
-            tma_load_3d(st + kOffW + 8192, &tmW, bar, 64, t0, bhv);
-            tma_load_3d(st + kOffU, &tmU, bar, 0, t0, bhv);
-            tma_load_3d(st + kOffU + 8192, &tmU, bar, 64, t0, bhv);
+            tma_load_3d(st + kOffQ, &tmQ, bar, kx, t0, kz);
+            tma_load_3d(st + kOffQ + 8192, &tmQ, bar, kx + 64, t0, kz);
+            tma_load_3d(st + kOffK, &tmK, bar, kx, t0, kz);
+            tma_load_3d(st + kOffK + 8192, &tmK, bar, kx + 64, t0, kz);
+            tma_load_3d(st + kOffW, &tmW, bar, vx, t0, vz);
+            tma_load_3d(st + kOffW + 8192, &tmW, bar, vx + 64, t0, vz);
+            tma_load_3d(st + kOffU, &tmU, bar, vx, t0, vz);
+            tma_load_3d(st + kOffU + 8192, &tmU, bar, vx + 64, t0, vz);
         };
         if (lead) {
             if (n_c > 0) load_stage(0);
@@ -205,8 +213,8 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             handoff_wait<6>();
             if (lead && *fail == 0) {
                 if (!(VAR && len - c * kC < kC)) {  // (a short last chunk is stored row by row by the compute threads)
-                    tma_store_3d(&tmO, smem + kOffO + (c & 1) * kTileBytes, 0, tok0 + c * kC, bhv);
-                    tma_store_3d(&tmO, smem + kOffO + (c & 1) * kTileBytes + 8192, 64, tok0 + c * kC, bhv);
+                    tma_store_3d(&tmO, smem + kOffO + (c & 1) * kTileBytes, vx, tok0 + c * kC, vz);
+                    tma_store_3d(&tmO, smem + kOffO + (c & 1) * kTileBytes + 8192, vx + 64, tok0 + c * kC, vz);
                     tma_store_commit();
                     tma_store_wait_read<0>();
                 }
@@ -366,7 +374,7 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         // half of the CTA forms P.
         const int tt = tid - 64;  // token of a table thread
         const bool tabler = tt >= 0 && tt < 64;
-        if (n_c > 0 && tabler) g_reg = (!VAR || tt < len) ? __ldg(gseq + tt) : 0.f;
+        if (n_c > 0 && tabler) g_reg = (!VAR || tt < len) ? __ldg(gseq + tt * gstep) : 0.f;
         bool ok = true;
         // gate tables of a chunk: written by 64 threads into the buffer of that chunk one barrier before they are read
         const bool g_raw = (p.flags & GDN_FLAG_G_RAW) != 0;
@@ -410,7 +418,7 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             const float gC = sg[63];
             const int left = len - c * kC;
             const bool short_chunk = VAR && left < kC;
-            if (c + 1 < n_c && tabler) g_reg = (!VAR || (c + 1) * kC + tt < len) ? __ldg(gseq + (c + 1) * kC + tt) : 0.f;
+            if (c + 1 < n_c && tabler) g_reg = (!VAR || (c + 1) * kC + tt < len) ? __ldg(gseq + ((c + 1) * kC + tt) * gstep) : 0.f;
             STAMPS(1);
 
             STAMPS(2);
@@ -573,7 +581,7 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                     const int tok = q >> 4, ch = q & 15;  // 16-byte piece ch of the token's 256-byte row
                     const uint4 v = *reinterpret_cast<const uint4*>(smem + kOffO + (c & 1) * kTileBytes + (ch >> 3) * 8192 +
                                                                     tok * 128 + (((ch & 7) ^ (tok & 7)) << 4));
-                    *reinterpret_cast<uint4*>(p.O + ((long long)bhv * p.T + tok0 + c * kC + tok) * kD + ch * 8) = v;
+                    *reinterpret_cast<uint4*>(p.O + (grow0 + (long long)(c * kC + tok) * gstep) * kD + ch * 8) = v;
                 }
             }
         }
@@ -623,12 +631,13 @@ EncodeTiledFn get_encode_fn() {
     return fn;
 }
 
-// [heads][T][128] bf16 tensor, boxes of 64 rows x 64 columns, 128-byte swizzle
-bool make_map(CUtensorMap* tm, const void* base, long long heads, int T) {
+// [heads][T][cols] bf16 tensor (cols = 128, or H * 128 for token-major tensors with heads = B), boxes of 64 rows x 64
+// columns, 128-byte swizzle
+bool make_map(CUtensorMap* tm, const void* base, long long heads, int T, int cols) {
     EncodeTiledFn enc = get_encode_fn();
     if (enc == nullptr) return false;
-    cuuint64_t dims[3] = {static_cast<cuuint64_t>(kD), static_cast<cuuint64_t>(T), static_cast<cuuint64_t>(heads)};
-    cuuint64_t strides[2] = {static_cast<cuuint64_t>(kD) * 2, static_cast<cuuint64_t>(T) * kD * 2};
+    cuuint64_t dims[3] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(T), static_cast<cuuint64_t>(heads)};
+    cuuint64_t strides[2] = {static_cast<cuuint64_t>(cols) * 2, static_cast<cuuint64_t>(T) * cols * 2};
     cuuint32_t box[3] = {64, static_cast<cuuint32_t>(kC), 1};
     cuuint32_t estr[3] = {1, 1, 1};
     return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
@@ -656,8 +665,12 @@ int launch_chunk_state(const ProblemS& q, cudaStream_t stream) {
     int* status = device_status_word();
     if (status == nullptr) return GDN_ERR_LAUNCH;
     CUtensorMap mQ, mK, mW, mU, mO;
-    if (!make_map(&mQ, q.Q, hk, q.T) || !make_map(&mK, q.K, hk, q.T) || !make_map(&mW, q.W, hv, q.T) ||
-        !make_map(&mU, q.U, hv, q.T) || !make_map(&mO, q.O, hv, q.T))
+    const bool bthd = (q.flags & GDN_FLAG_LAYOUT_BTHD) != 0;
+    const long long nb = var ? 1 : q.B;
+    const long long zk = bthd ? nb : hk, zv = bthd ? nb : hv;
+    const int ck = bthd ? q.H_k * kD : kD, cv = bthd ? q.H_v * kD : kD;
+    if (!make_map(&mQ, q.Q, zk, q.T, ck) || !make_map(&mK, q.K, zk, q.T, ck) || !make_map(&mW, q.W, zv, q.T, cv) ||
+        !make_map(&mU, q.U, zv, q.T, cv) || !make_map(&mO, q.O, zv, q.T, cv))
         return GDN_ERR_LAUNCH;
     ParamsS prm;
     prm.g = q.g;

@@ -145,3 +145,20 @@ def test_state_output_at_full_size(name):
         assert eO.max() <= TOL_O, f"{name}: O rel-F {eO.max():.3e} at chunk {eO.argmax()} of head ({b},{hv})"
         eS = orc.rel_frobenius(S[b, hv].double().cpu().numpy()[None], So[None])
         assert eS.max() <= TOL_S, f"{name}: S rel-F {eS.max():.3e} of head ({b},{hv})"
+
+
+def test_token_major_layout_gives_the_same_bits():
+    """GDN_FLAG_LAYOUT_BTHD: the tensors as model code keeps them, [B,T,H,d]; only addresses change."""
+    C, T = 64, 384
+    inp = gen.make_inputs(2, 2, 4, T, C, 128, 128, seed=450)
+    Q = _queries(inp, 451).cuda()
+    scale = 128 ** -0.5
+    S0 = (0.1 * torch.randn(2, 4, 128, 128, generator=torch.Generator().manual_seed(452))).cuda()
+    K, g = inp.K.cuda(), inp.g.cuda()
+    W, U, _ = gdn.chunk_prepare(K, inp.V.cuda(), inp.beta.cuda(), g, C, flags=gdn.GDN_FLAG_W_GATED)
+    O, S = gdn.chunk_state_output(Q, K, W, U, g, C, scale, S0)
+    tm = lambda x: x.transpose(1, 2).contiguous()
+    Ot, St = gdn.chunk_state_output(tm(Q), tm(K), tm(W), tm(U), g.transpose(1, 2).contiguous(), C, scale, S0,
+                                    flags=gdn.GDN_FLAG_LAYOUT_BTHD)
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+    assert torch.equal(Ot.transpose(1, 2), O) and torch.equal(St, S)

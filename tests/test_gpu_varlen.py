@@ -209,3 +209,23 @@ def test_packed_state_output_matches_oracle_on_the_same_w_u():
             assert eS.max() <= 1e-4, f"sequence {s_} head {hv}: S rel-F {eS.max():.3e}"
     # rows of O past the last sequence stay untouched (none here), and nothing wrote outside [0, T)
     assert O.shape == (2, T, 128)
+
+
+def test_packed_layer_token_major_gives_the_same_bits():
+    """Both packed calls on token-major tensors [T,H,d] reproduce the head-major results bit for bit."""
+    C = 64
+    lens = [100, 64, 7, 191, 1]
+    K, V, beta, g, graw, cu = _packed_inputs(lens, 2, 4, C, seed=620)
+    T = int(cu[-1])
+    Q = _queries(2, T, 621)
+    scale = 128 ** -0.5
+    f = gdn.GDN_FLAG_W_GATED | gdn.GDN_FLAG_G_RAW
+    W, U, _, _, _ = gdn.chunk_prepare_varlen(K.cuda(), V.cuda(), beta.cuda(), graw.cuda(), cu, C, flags=f, want_tinv=False)
+    O, S = gdn.chunk_state_output_varlen(Q.cuda(), K.cuda(), W, U, graw.cuda(), cu, C, scale, flags=gdn.GDN_FLAG_G_RAW)
+    tm = lambda x: x.transpose(0, 1).contiguous().cuda()
+    b = gdn.GDN_FLAG_LAYOUT_BTHD
+    Wt, Ut, _, _, _ = gdn.chunk_prepare_varlen(tm(K), tm(V), tm(beta), tm(graw), cu, C, flags=f | b, want_tinv=False)
+    Ot, St = gdn.chunk_state_output_varlen(tm(Q), tm(K), Wt, Ut, tm(graw), cu, C, scale, flags=gdn.GDN_FLAG_G_RAW | b)
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+    assert torch.equal(Wt.transpose(0, 1), W) and torch.equal(Ut.transpose(0, 1), U)
+    assert torch.equal(Ot.transpose(0, 1), O) and torch.equal(St, S)
