@@ -205,6 +205,27 @@ int gdn_chunk_state_output_varlen(const void* Q, const void* K, const void* W_ga
                                   int d_k, int d_v, float scale, const float* S_in, void* O_out, float* S_out,
                                   unsigned flags, gdn_stream_t stream);
 
+/*
+ * gdn_chunk_state_output for FEW LONG sequences (one per value head, B = 1): the chunks of a sequence are a serial
+ * chain, so with fewer sequences than SMs most of the GPU idles. Here every sequence is cut into `segments` runs of
+ * whole chunks. The state at the end of a segment is an affine map of the state at its start, S_end = S_start M + N
+ * (M: d_k x d_k, N: d_v x d_k): a first pass forms N (the segment from a zero state) and M (the segment from the
+ * identity with U = 0) of every segment in parallel, without queries or output; a short recurrence gives every
+ * segment's initial state; a second pass runs all segments in parallel with their output. Three passes' worth of
+ * state work instead of one, on `segments` times as many SMs.
+ *   Tensors as gdn_chunk_state_output with B = 1 (head-major [H,T,d], or [T,H,d] with GDN_FLAG_LAYOUT_BTHD).
+ *   segments: 1 = the plain call; gdn_chunk_state_segments(H_v) proposes the count that fills the SMs in one wave.
+ *   workspace: DEVICE memory of gdn_chunk_state_segmented_workspace(H_v, segments) bytes, 16-byte aligned, owned by
+ *   the caller and free to reuse when the stream has passed the call.
+ * The result differs from the plain call by fp32 rounding of the state recurrence only.
+ */
+int gdn_chunk_state_segments(int H_v);
+size_t gdn_chunk_state_segmented_workspace(int H_v, int segments);
+int gdn_chunk_state_output_segmented(const void* Q, const void* K, const void* W_gated, const void* U, const float* g,
+                                     int H_k, int H_v, int T, int C, int d_k, int d_v, float scale,
+                                     const float* S_in, void* O_out, float* S_out, int segments,
+                                     void* workspace, size_t workspace_bytes, unsigned flags, gdn_stream_t stream);
+
 /* Checksum of the 256-entry gate-decay table round(2^15 * 2^(-f/256)) the INT8 kernel uses
  * (sum_f: s = (31 s + table[f] + f) mod 1000000007), so that a CPU evaluation can confirm it holds the same table. */
 unsigned int gdn_int8_lut_checksum(void);

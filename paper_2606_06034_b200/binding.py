@@ -36,7 +36,8 @@ GDN_FWDSUBST_BLOCKED = 1
 EXPORTS = (
     "gdn_chunk_prepare", "gdn_chunk_prepare_gqa", "gdn_chunk_prepare_ex", "gdn_chunk_prepare_varlen",
     "gdn_chunk_prepare_fwdsubst",
-    "gdn_chunk_prepare_int8", "gdn_chunk_state_output", "gdn_chunk_state_output_varlen", "gdn_selftest_bounded_wait",
+    "gdn_chunk_prepare_int8", "gdn_chunk_state_output", "gdn_chunk_state_output_varlen", "gdn_chunk_state_output_segmented",
+    "gdn_chunk_state_segments", "gdn_chunk_state_segmented_workspace", "gdn_selftest_bounded_wait",
     "gdn_int8_lut_checksum",
     "gdn_device_status", "gdn_default_order", "gdn_default_residual_steps",
     "gdn_status_string", "gdn_launch_count",
@@ -81,6 +82,13 @@ def load_library() -> ctypes.CDLL:
     lib.gdn_chunk_state_output_varlen.argtypes = [vp, vp, vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ip, ctypes.c_float, vp, vp, vp,
                                                   ctypes.c_uint, vp]
     lib.gdn_chunk_state_output_varlen.restype = ip
+    lib.gdn_chunk_state_segments.argtypes = [ip]
+    lib.gdn_chunk_state_segments.restype = ip
+    lib.gdn_chunk_state_segmented_workspace.argtypes = [ip, ip]
+    lib.gdn_chunk_state_segmented_workspace.restype = ctypes.c_size_t
+    lib.gdn_chunk_state_output_segmented.argtypes = [vp, vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ctypes.c_float, vp, vp, vp, ip,
+                                                     vp, ctypes.c_size_t, ctypes.c_uint, vp]
+    lib.gdn_chunk_state_output_segmented.restype = ip
     lib.gdn_selftest_bounded_wait.argtypes = [vp]
     lib.gdn_selftest_bounded_wait.restype = ip
     lib.gdn_int8_lut_checksum.argtypes = []
@@ -319,6 +327,36 @@ def gdn_chunk_state_output_varlen(Q, K, W_gated, U, g, cu_seqlens, n_seq, T_tota
     if check and rc != GDN_OK:
         raise GdnError(rc, "gdn_chunk_state_output_varlen")
     return rc
+
+
+def chunk_state_output_segmented(Q, K, W_gated, U, g, C, scale=1.0, S_in=None, *, segments=0, want_state=True, flags=0,
+                                 workspace=None):
+    """Few long sequences (B = 1; Q, K [H_k,T,d_k], W_gated, U [H_v,T,d], g [H_v,T], or token-major with
+    GDN_FLAG_LAYOUT_BTHD): the segmented form of the state passing. segments = 0: the library's proposal.
+    Returns (O, S_out [H_v,d_v,d_k] or None)."""
+    if flags & GDN_FLAG_LAYOUT_BTHD:
+        T, H_k, d_k = K.shape
+        _, H_v, d_v = U.shape
+    else:
+        H_k, T, d_k = K.shape
+        H_v, _, d_v = U.shape
+    lib = load_library()
+    if segments <= 0:
+        segments = int(lib.gdn_chunk_state_segments(H_v))
+    need = int(lib.gdn_chunk_state_segmented_workspace(H_v, segments))
+    if workspace is None and need > 0:
+        workspace = torch.empty(need, dtype=torch.uint8, device=U.device)
+    for t in (Q, K, W_gated, U, g, S_in):
+        if t is not None and (not t.is_cuda or not t.is_contiguous()):
+            raise ValueError("all tensors must be contiguous CUDA tensors (there is no CPU path)")
+    O = torch.empty_like(U)
+    S_out = torch.empty(H_v, d_v, d_k, dtype=torch.float32, device=U.device) if want_state else None
+    rc = lib.gdn_chunk_state_output_segmented(_ptr(Q), _ptr(K), _ptr(W_gated), _ptr(U), _ptr(g), H_k, H_v, T, C, d_k, d_v,
+                                              ctypes.c_float(scale), _ptr(S_in), _ptr(O), _ptr(S_out), segments,
+                                              _ptr(workspace), need, flags, _stream())
+    if rc != GDN_OK:
+        raise GdnError(rc, "gdn_chunk_state_output_segmented")
+    return O, S_out
 
 
 def chunk_state_output_varlen(Q, K, W_gated, U, g, cu_seqlens, C, scale=1.0, S_in=None, *, want_state=True, flags=0):

@@ -74,9 +74,11 @@ struct ParamsS {
     int H_k, H_v, T, group;
     float scale;
     unsigned flags;  // GDN_FLAG_G_RAW: g holds raw log-gates, prefix-summed inside every chunk here
-    // packed variable-length sequences (B = 1): sequence s holds the tokens [cu_seqlens[s], cu_seqlens[s + 1]) of tensors
+    // packed variable-length sequences (B = 1): sequence s holds the tokens [seq_start[s], seq_end[s]) of tensors
     // with T tokens per head and is chunked from its own first token; null for dense tensors
-    const int* cu_seqlens;
+    const int* seq_start;  // first token of sequence s
+    const int* seq_end;    // one past its last token (the public call passes cu_seqlens and cu_seqlens + 1)
+    const int* seq_no_u;   // optional: sequence s runs with U = 0 (the state map of a segment, see the segmented call)
     __nv_bfloat16* O;  // output tensor (rows of a short last chunk are stored one by one)
 };
 
@@ -110,7 +112,8 @@ __device__ __forceinline__ void handoff_wait() {
 }
 
 // VAR: packed variable-length sequences (own instantiation: its masks sit on the chain the dense case is bound by)
-template <bool VAR>
+// SO: state only: no queries, no output (the first pass of the segmented call); U may be absent per sequence.
+template <bool VAR, bool SO>
 __global__ void __launch_bounds__(kThreads + 64, 1)
 chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                    const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmU,
@@ -167,8 +170,9 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     // dense: one CTA per (batch, value head), bhv = row of the [B * H_v, T] tensors. Packed sequences: one CTA per
     // (sequence, value head); the tensors have one batch row per head and the sequence starts at token tok0
     const int b = blockIdx.x / p.H_v, hv = blockIdx.x - b * p.H_v;
-    const int tok0 = VAR ? __ldg(p.cu_seqlens + b) : 0;
-    const int len = VAR ? __ldg(p.cu_seqlens + b + 1) - tok0 : p.T;
+    const int tok0 = VAR ? __ldg(p.seq_start + b) : 0;
+    const int len = VAR ? __ldg(p.seq_end + b) - tok0 : p.T;
+    const bool no_u = SO && p.seq_no_u != nullptr && __ldg(p.seq_no_u + b) != 0;
     const int bhv = VAR ? hv : blockIdx.x;
     const int bhk = VAR ? hv / p.group : b * p.H_k + hv / p.group;
     // Token-major tensors [B, T, H, d] (GDN_FLAG_LAYOUT_BTHD) are seen by TMA as (H * d, T, B): the head picks the first
@@ -192,10 +196,12 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         auto load_stage = [&](int c) {
             uint8_t* st = smem + (c & 1) * kStageBytes;
             uint64_t* bar = &bar_full[c & 1];
-            mbar_arrive_expect_tx(bar, kStageBytes);
+            mbar_arrive_expect_tx(bar, SO ? 3 * kTileBytes : kStageBytes);
             const int t0 = tok0 + c * kC;
-            tma_load_3d(st + kOffQ, &tmQ, bar, kx, t0, kz);
-            tma_load_3d(st + kOffQ + 8192, &tmQ, bar, kx + 64, t0, kz);
+            if (!SO) {
+                tma_load_3d(st + kOffQ, &tmQ, bar, kx, t0, kz);
+                tma_load_3d(st + kOffQ + 8192, &tmQ, bar, kx + 64, t0, kz);
+            }
             tma_load_3d(st + kOffK, &tmK, bar, kx, t0, kz);
             tma_load_3d(st + kOffK + 8192, &tmK, bar, kx + 64, t0, kz);
             tma_load_3d(st + kOffW, &tmW, bar, vx, t0, vz);
@@ -210,15 +216,15 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         uint32_t par = 0;
         for (int c = 0; c < n_c && *fail == 0; ++c) {
             // the staged output tile of chunk c is complete (every compute thread has arrived)
-            handoff_wait<6>();
+            if (!SO) handoff_wait<6>();
             if (lead && *fail == 0) {
-                if (!(VAR && len - c * kC < kC)) {  // (a short last chunk is stored row by row by the compute threads)
+                if (!SO && !(VAR && len - c * kC < kC)) {  // (a short last chunk is stored row by row by the compute threads)
                     tma_store_3d(&tmO, smem + kOffO + (c & 1) * kTileBytes, vx, tok0 + c * kC, vz);
                     tma_store_3d(&tmO, smem + kOffO + (c & 1) * kTileBytes + 8192, vx + 64, tok0 + c * kC, vz);
                     tma_store_commit();
                     tma_store_wait_read<0>();
                 }
-                mbar_arrive(&bar_stg[c & 1]);  // the staging buffer may be written again (chunk c + 2)
+                if (!SO) mbar_arrive(&bar_stg[c & 1]);  // the staging buffer may be written again (chunk c + 2)
                 if (c + 2 < n_c) {
                     if (!wait_bar(&bar_g2, par)) *fail = 1;
                     if (*fail == 0) load_stage(c + 2);
@@ -240,19 +246,23 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             if (!wait_bar(&bar_full[c & 1], (c >> 1) & 1)) *fail = 1;
             tc_fence_after_sync();
             if (*fail == 0 && elect_one()) {
+                if (!no_u) {
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const uint64_t bd = smem_desc(sa + kOffU + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024, SWZ_128B);
-                    mma_f16_ts(tmem + kD1, tmem + kIA + ks * 8, bd, idesc_kk64, ks > 0);
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const uint64_t bd = smem_desc(sa + kOffU + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024, SWZ_128B);
+                        mma_f16_ts(tmem + kD1, tmem + kIA + ks * 8, bd, idesc_kk64, ks > 0);
+                    }
                 }
-                // rows 64..127 of the A operand read past the 64-row K tile: unused lanes
+                if (!SO) {
+                    // rows 64..127 of the A operand read past the 64-row K tile: unused lanes
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const uint64_t ad = smem_desc(sa + kOffK + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024, SWZ_128B);
-                    const uint64_t bd = smem_desc(sa + kOffQ + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024, SWZ_128B);
-                    mma_f16_ss(tmem + kPT, ad, bd, idesc_kk64, ks > 0);
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const uint64_t ad = smem_desc(sa + kOffK + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024, SWZ_128B);
+                        const uint64_t bd = smem_desc(sa + kOffQ + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024, SWZ_128B);
+                        mma_f16_ss(tmem + kPT, ad, bd, idesc_kk64, ks > 0);
+                    }
+                    mma_commit(&bar_pre);  // (state only: nothing of this group is waited for by itself)
                 }
-                mma_commit(&bar_pre);
             }
             __syncwarp();
         };
@@ -271,17 +281,20 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks) {
                         const uint64_t bd = smem_desc(st_a + kOffW + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024, SWZ_128B);
-                        mma_f16_ts(tmem + kD1, tmem + (part == 0 ? kSA : kO2) + ks * 8, bd, idesc_kk64, true);
+                        mma_f16_ts(tmem + kD1, tmem + (part == 0 ? kSA : kO2) + ks * 8, bd, idesc_kk64,
+                                   !no_u || part > 0 || ks > 0);
                     }
                 }
                 mma_commit(&bar_d1);
-                // O1 = (S0_hi + S0_lo) Q^T
+                if (!SO) {
+                    // O1 = (S0_hi + S0_lo) Q^T
 #pragma unroll
-                for (int part = 0; part < 2; ++part) {
+                    for (int part = 0; part < 2; ++part) {
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {
-                        const uint64_t bd = smem_desc(st_a + kOffQ + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024, SWZ_128B);
-                        mma_f16_ts(tmem + kO1, tmem + (part == 0 ? kSA : kO2) + ks * 8, bd, idesc_kk64, part > 0 || ks > 0);
+                        for (int ks = 0; ks < 8; ++ks) {
+                            const uint64_t bd = smem_desc(st_a + kOffQ + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024, SWZ_128B);
+                            mma_f16_ts(tmem + kO1, tmem + (part == 0 ? kSA : kO2) + ks * 8, bd, idesc_kk64, part > 0 || ks > 0);
+                        }
                     }
                 }
                 // (no completion barrier of its own: the commit behind the output product below covers it, and a wait
@@ -294,18 +307,20 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             STAMPS(103);
             tc_fence_after_sync();
             if (*fail == 0 && elect_one()) {
-                // O2 = U_new^T P^T = Uh Ph + Ul Ph + Uh Pl (K-dim = 64 tokens; the plain copy of tokens 16 ks.. sits at
-                // columns 16 ks .. 16 ks + 7 of its region, the gate-scaled one at 16 ks + 8 ..)
+                if (!SO) {
+                    // O2 = U_new^T P^T = Uh Ph + Ul Ph + Uh Pl (K-dim = 64 tokens; the plain copy of tokens 16 ks.. sits
+                    // at columns 16 ks .. 16 ks + 7 of its region, the gate-scaled one at 16 ks + 8 ..)
 #pragma unroll
-                for (int part = 0; part < 3; ++part) {
+                    for (int part = 0; part < 3; ++part) {
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks) {
-                        const uint64_t bd = smem_desc(smem_a + kOffP + (part == 2 ? 8192 : 0) + ks * 256, 128, 1024, SWZ_NONE);
-                        mma_f16_ts(tmem + kO2, tmem + (part == 1 ? kPT : kD1) + ks * 16, bd,
-                                   idesc_mn64, part > 0 || ks > 0);
+                        for (int ks = 0; ks < 4; ++ks) {
+                            const uint64_t bd = smem_desc(smem_a + kOffP + (part == 2 ? 8192 : 0) + ks * 256, 128, 1024, SWZ_NONE);
+                            mma_f16_ts(tmem + kO2, tmem + (part == 1 ? kPT : kD1) + ks * 16, bd,
+                                       idesc_mn64, part > 0 || ks > 0);
+                        }
                     }
+                    mma_commit(&bar_o2);  // the output is finished while the state update still runs
                 }
-                mma_commit(&bar_o2);  // the output is finished while the state update still runs
                 // S += (U_new^T exp(g_C - g_j)) K, hi + lo (the K tile as MN-major operand, N = 128)
 #pragma unroll
                 for (int part = 0; part < 2; ++part) {
@@ -440,9 +455,9 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             }
             // ---- P_ij = exp(g_i - g_j) PT_ji for j <= i (hi + lo): token j = lane (rows 0..63 only), this thread's 16 columns i
             STAMPS(3);
-            if (!wait_group(&bar_pre, par_pre)) { ok = false; break; }
+            if (!SO && !wait_group(&bar_pre, par_pre)) { ok = false; break; }
             STAMPS(4);
-            if (wq < 2) {
+            if (!SO && wq < 2) {
                 uint32_t d[16];
                 tmem_ld16(lane_base + kPT + h * 16, d);
                 tmem_wait_ld();
@@ -516,44 +531,46 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             handoff_arrive<5>();
             STAMPS(7);
 
-            // the bulk store of chunk c - 2 has finished reading this chunk's staging buffer (polled here, in the shadow of
-            // the output product)
-            if (c >= 2 && !wait_bar(&bar_stg[c & 1], ((c - 2) >> 1) & 1)) { *fail = 1; ok = false; break; }
-            // ---- exp(g_i) O1 (complete with O2: products finish in the order they were issued)
-            if (!wait_group(&bar_o2, par_o2)) { ok = false; break; }
-            STAMPS(8);
-            float o[16];
-            {
-                uint32_t d[16];
-                tmem_ld16(lane_base + kO1 + h * 16, d);
-                tmem_wait_ld();
-#pragma unroll
-                for (int i4 = 0; i4 < 4; ++i4) {
-                    const float4 e4 = *reinterpret_cast<const float4*>(se + h * 16 + i4 * 4);
-                    o[i4 * 4 + 0] = __uint_as_float(d[i4 * 4 + 0]) * e4.x;
-                    o[i4 * 4 + 1] = __uint_as_float(d[i4 * 4 + 1]) * e4.y;
-                    o[i4 * 4 + 2] = __uint_as_float(d[i4 * 4 + 2]) * e4.z;
-                    o[i4 * 4 + 3] = __uint_as_float(d[i4 * 4 + 3]) * e4.w;
+            if (!SO) {
+                // the bulk store of chunk c - 2 has finished reading this chunk's staging buffer (polled here, in the shadow of
+                // the output product)
+                if (c >= 2 && !wait_bar(&bar_stg[c & 1], ((c - 2) >> 1) & 1)) { *fail = 1; ok = false; break; }
+                // ---- exp(g_i) O1 (complete with O2: products finish in the order they were issued)
+                if (!wait_group(&bar_o2, par_o2)) { ok = false; break; }
+                STAMPS(8);
+                float o[16];
+                {
+                    uint32_t d[16];
+                    tmem_ld16(lane_base + kO1 + h * 16, d);
+                    tmem_wait_ld();
+    #pragma unroll
+                    for (int i4 = 0; i4 < 4; ++i4) {
+                        const float4 e4 = *reinterpret_cast<const float4*>(se + h * 16 + i4 * 4);
+                        o[i4 * 4 + 0] = __uint_as_float(d[i4 * 4 + 0]) * e4.x;
+                        o[i4 * 4 + 1] = __uint_as_float(d[i4 * 4 + 1]) * e4.y;
+                        o[i4 * 4 + 2] = __uint_as_float(d[i4 * 4 + 2]) * e4.z;
+                        o[i4 * 4 + 3] = __uint_as_float(d[i4 * 4 + 3]) * e4.w;
+                    }
                 }
-            }
-            STAMPS(10);
-            // ---- O^T = scale (exp(g_i) O1 + O2): element (token i, feature t) of the staged tile
-            {
-                uint32_t d[16];
-                tmem_ld16(lane_base + kO2 + h * 16, d);
-                tmem_wait_ld();
-                uint8_t* sub = smem + kOffO + (c & 1) * kTileBytes + (t >> 6) * 8192;
-                const int cch = (t & 63) >> 3;
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const int tok = h * 16 + i;
-                    const __nv_bfloat16 v = __float2bfloat16_rn(p.scale * (o[i] + __uint_as_float(d[i])));
-                    *reinterpret_cast<__nv_bfloat16*>(sub + tok * 128 + ((cch ^ (tok & 7)) << 4) + (t & 7) * 2) = v;
+                STAMPS(10);
+                // ---- O^T = scale (exp(g_i) O1 + O2): element (token i, feature t) of the staged tile
+                {
+                    uint32_t d[16];
+                    tmem_ld16(lane_base + kO2 + h * 16, d);
+                    tmem_wait_ld();
+                    uint8_t* sub = smem + kOffO + (c & 1) * kTileBytes + (t >> 6) * 8192;
+                    const int cch = (t & 63) >> 3;
+    #pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const int tok = h * 16 + i;
+                        const __nv_bfloat16 v = __float2bfloat16_rn(p.scale * (o[i] + __uint_as_float(d[i])));
+                        *reinterpret_cast<__nv_bfloat16*>(sub + tok * 128 + ((cch ^ (tok & 7)) << 4) + (t & 7) * 2) = v;
+                    }
                 }
+                // the tile goes to the storing warp: no compute thread waits for the others here
+                fence_proxy_async_smem();
+                handoff_arrive<6>();
             }
-            // the tile goes to the storing warp: no compute thread waits for the others here
-            fence_proxy_async_smem();
-            handoff_arrive<6>();
             // ---- bf16 copies (hi, lo) of the new state for the next chunk's products; the lo half goes where O2 was
             // (this thread has read its O2 columns above)
             if (!wait_group(&bar_g2, par_g2)) { ok = false; break; }
@@ -574,7 +591,7 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 handoff_arrive<4>();
             }
             STAMPS(11);
-            if (short_chunk) {
+            if (!SO && short_chunk) {
                 // only the rows of real tokens leave, 16 bytes per thread and step, from the staged (swizzled) tile
                 asm volatile("bar.sync 1, 512;" ::: "memory");  // (last chunk of a packed sequence only)
                 for (int q = tid; q < left * 16; q += kThreads) {
@@ -645,7 +662,143 @@ bool make_map(CUtensorMap* tm, const void* base, long long heads, int T, int col
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// ---- the segmented call: a long sequence cut into P segments whose state maps are formed in parallel
+// Set-up of the first pass: the token ranges of its 2P - 3 runs (runs 0 .. P-2: segment s from a zero state, segment 0
+// from the caller's; runs P-1 .. 2P-4: segments 1 .. P-2 from the identity with U = 0, which gives the matrix M of
+// S_end = S_start M + N), their initial states, the token ranges of the second pass and its first initial state.
+__global__ void segmented_setup_kernel(int P, int H_v, int n_chunks, const float* S_user, float* S_in1, float* S_start,
+                                       int* start1, int* end1, int* no_u1, int* start3, int* end3) {
+    const int n1 = 2 * P - 3;
+    if (blockIdx.x == 0 && threadIdx.x < 32) {
+        for (int s_ = threadIdx.x; s_ < n1; s_ += 32) {
+            const int seg = (s_ <= P - 2) ? s_ : s_ - (P - 2);
+            start1[s_] = (int)((long long)n_chunks * seg / P) * kC;
+            end1[s_] = (int)((long long)n_chunks * (seg + 1) / P) * kC;
+            no_u1[s_] = (s_ <= P - 2) ? 0 : 1;
+        }
+        for (int s_ = threadIdx.x; s_ < P; s_ += 32) {
+            start3[s_] = (int)((long long)n_chunks * s_ / P) * kC;
+            end3[s_] = (int)((long long)n_chunks * (s_ + 1) / P) * kC;
+        }
+    }
+    const long long per = (long long)H_v * kD * kD;
+    const long long total = (long long)n1 * per;
+    for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total + per; e += (long long)gridDim.x * blockDim.x) {
+        if (e < total) {
+            const int s_ = (int)(e / per);
+            const long long r = e - (long long)s_ * per;
+            const int idx = (int)(r % (kD * kD));
+            float v = 0.f;
+            if (s_ == 0) v = (S_user != nullptr) ? S_user[r] : 0.f;
+            else if (s_ > P - 2) v = (idx / kD == idx % kD) ? 1.f : 0.f;
+            S_in1[e] = v;
+        } else {
+            const long long r = e - total;
+            S_start[r] = (S_user != nullptr) ? S_user[r] : 0.f;
+        }
+    }
+}
+
+// S_start[k] = S_start[k-1] M_{k-1} + N_{k-1} for k = 2 .. P-1, S_start[1] = N_0 (the first segment ran from the caller's
+// state). One CTA per (value head, block of 16 state rows): the rows of the state are independent. fp32 FMAs.
+__global__ void __launch_bounds__(256) segmented_combine_kernel(int P, int H_v, const float* S_out1, float* S_start) {
+    __shared__ float cur[16][kD];
+    const int hv = blockIdx.x, r0 = blockIdx.y * 16;
+    const long long per = (long long)H_v * kD * kD;
+    const int col = threadIdx.x & 127, rh = threadIdx.x >> 7;  // this thread: column col, rows r0 + rh, r0 + rh + 2, ...
+    const float* N0 = S_out1 + (long long)hv * kD * kD;
+    for (int i = 0; i < 8; ++i) {
+        const int r = rh + 2 * i;
+        const float v = N0[(r0 + r) * kD + col];
+        cur[r][col] = v;
+        S_start[per + (long long)hv * kD * kD + (r0 + r) * kD + col] = v;
+    }
+    __syncthreads();
+    for (int k = 2; k < P; ++k) {
+        const float* M = S_out1 + (long long)(P - 1 + (k - 2)) * per + (long long)hv * kD * kD;  // M of segment k - 1
+        const float* N = S_out1 + (long long)(k - 1) * per + (long long)hv * kD * kD;            // N of segment k - 1
+        float acc[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[i] = N[(r0 + rh + 2 * i) * kD + col];
+        for (int d = 0; d < kD; ++d) {
+            const float m = M[d * kD + col];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) acc[i] = fmaf(cur[rh + 2 * i][d], m, acc[i]);
+        }
+        __syncthreads();
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            cur[rh + 2 * i][col] = acc[i];
+            S_start[(long long)k * per + (long long)hv * kD * kD + (r0 + rh + 2 * i) * kD + col] = acc[i];
+        }
+        __syncthreads();
+    }
+}
+
 }  // namespace
+
+size_t chunk_state_segmented_workspace(int H_v, int P) {
+    if (P < 2) return 0;
+    const size_t per = (size_t)H_v * kD * kD * sizeof(float);
+    const size_t n1 = (size_t)(2 * P - 3);
+    return (2 * n1 + 2 * (size_t)P) * per + (3 * n1 + 2 * (size_t)P) * sizeof(int) + 256;
+}
+
+int chunk_state_auto_segments(long long H_v) {
+    int n_sm = 0, dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        return 1;
+    int P = 1;
+    while (P < 8 && H_v * (2 * (P + 1) - 3) <= n_sm) ++P;
+    return P;
+}
+
+// One sequence per value head (B = 1), cut into P segments: first pass = every segment's state map in parallel (state
+// only), then the segments' initial states by a short recurrence, then every segment in parallel with its output.
+int launch_chunk_state_segmented(const ProblemS& q, int P, void* workspace, cudaStream_t stream) {
+    if (q.B != 1 || q.seq_start != nullptr) return GDN_ERR_UNSUPPORTED;
+    const int n_chunks = q.T / kC;
+    if (P > n_chunks) P = n_chunks;
+    if (P < 2) return launch_chunk_state(q, stream);
+    const size_t per = (size_t)q.H_v * kD * kD;
+    const size_t n1 = (size_t)(2 * P - 3);
+    float* S_in1 = static_cast<float*>(workspace);
+    float* S_out1 = S_in1 + n1 * per;
+    float* S_start = S_out1 + n1 * per;
+    float* S_out3 = S_start + (size_t)P * per;
+    int* start1 = reinterpret_cast<int*>(S_out3 + (size_t)P * per);
+    int* end1 = start1 + n1;
+    int* no_u1 = end1 + n1;
+    int* start3 = no_u1 + n1;
+    int* end3 = start3 + P;
+    segmented_setup_kernel<<<256, 256, 0, stream>>>(P, q.H_v, n_chunks, q.S_in, S_in1, S_start, start1, end1, no_u1, start3, end3);
+    count_launch();
+    ProblemS a = q;
+    a.B = static_cast<int>(n1);
+    a.S_in = S_in1;
+    a.S_out = S_out1;
+    a.O = q.O;  // not written
+    a.seq_start = start1;
+    a.seq_end = end1;
+    a.seq_no_u = no_u1;
+    a.state_only = true;
+    int rc = launch_chunk_state(a, stream);
+    if (rc != GDN_OK) return rc;
+    segmented_combine_kernel<<<dim3(q.H_v, kD / 16), 256, 0, stream>>>(P, q.H_v, S_out1, S_start);
+    count_launch();
+    ProblemS b = q;
+    b.B = P;
+    b.S_in = S_start;
+    b.S_out = (q.S_out != nullptr) ? S_out3 : nullptr;
+    b.seq_start = start3;
+    b.seq_end = end3;
+    rc = launch_chunk_state(b, stream);
+    if (rc != GDN_OK) return rc;
+    if (q.S_out != nullptr &&
+        cudaMemcpyAsync(q.S_out, S_out3 + (size_t)(P - 1) * per, per * sizeof(float), cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
+        return GDN_ERR_LAUNCH;
+    return cudaGetLastError() == cudaSuccess ? GDN_OK : GDN_ERR_LAUNCH;
+}
 
 #ifdef GDN_TRACE
 extern "C" int gdn_debug_read_trace_state(long long* host_out) {
@@ -656,7 +809,8 @@ extern "C" int gdn_debug_read_trace_state(long long* host_out) {
 int launch_chunk_state(const ProblemS& q, cudaStream_t stream) {
     if (q.d_k != kD || q.d_v != kD || q.C != kC) return GDN_ERR_UNSUPPORTED;
     // packed sequences: B counts the sequences, the tensors have one row of T tokens per head
-    const bool var = q.cu_seqlens != nullptr;
+    const bool var = q.seq_start != nullptr;
+    if (q.state_only && !var) return GDN_ERR_UNSUPPORTED;
     const long long hk = var ? q.H_k : (long long)q.B * q.H_k, hv = var ? q.H_v : (long long)q.B * q.H_v;
     const long long n_cta = (long long)q.B * q.H_v;
     if (n_cta == 0 || q.T == 0) return GDN_OK;
@@ -683,10 +837,12 @@ int launch_chunk_state(const ProblemS& q, cudaStream_t stream) {
     prm.group = q.H_v / q.H_k;
     prm.scale = q.scale;
     prm.flags = q.flags;
-    prm.cu_seqlens = q.cu_seqlens;
+    prm.seq_start = q.seq_start;
+    prm.seq_end = q.seq_end;
+    prm.seq_no_u = q.seq_no_u;
     prm.O = static_cast<__nv_bfloat16*>(q.O);
     const int smem = kSmemTotal + 1024;
-    auto kern = var ? chunk_state_kernel<true> : chunk_state_kernel<false>;
+    auto kern = q.state_only ? chunk_state_kernel<true, true> : (var ? chunk_state_kernel<true, false> : chunk_state_kernel<false, false>);
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return GDN_ERR_LAUNCH;
     kern<<<static_cast<int>(n_cta), kThreads + 64, smem, stream>>>(mQ, mK, mW, mU, mO, prm);
     count_launch();

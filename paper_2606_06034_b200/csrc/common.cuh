@@ -62,9 +62,13 @@ struct ProblemS {
     int B, H_k, H_v, T, C, d_k, d_v;
     float scale;
     unsigned flags;
-    // packed variable-length sequences: B sequences, sequence s = tokens [cu_seqlens[s], cu_seqlens[s + 1]) of tensors
-    // with T tokens per head (device array of B + 1 int32); null for dense tensors
-    const int* cu_seqlens = nullptr;
+    // packed variable-length sequences: B sequences, sequence s = tokens [seq_start[s], seq_end[s]) of tensors with T
+    // tokens per head (device arrays of B int32; the public call passes cu_seqlens and cu_seqlens + 1); null for dense
+    const int* seq_start = nullptr;
+    const int* seq_end = nullptr;
+    // state only (packed form): no queries, no output, only S_out; seq_no_u[s] != 0: sequence s runs with U = 0
+    bool state_only = false;
+    const int* seq_no_u = nullptr;
 };
 
 enum InverseMode { INV_NEUMANN = 0, INV_FWDSUBST_ROWS = 1, INV_FWDSUBST_BLOCKED = 2 };
@@ -78,6 +82,10 @@ int launch_simt(const Problem& p, InverseMode mode, cudaStream_t stream);
 int launch_tc_bf16(const Problem& p, InverseMode mode, cudaStream_t stream);
 int launch_wait_selftest(cudaStream_t stream);
 int launch_chunk_state(const ProblemS& p, cudaStream_t stream);
+// the segmented form for few long sequences (B = 1): P segments per sequence, workspace of chunk_state_segmented_workspace bytes
+int launch_chunk_state_segmented(const ProblemS& q, int P, void* workspace, cudaStream_t stream);
+size_t chunk_state_segmented_workspace(int H_v, int P);
+int chunk_state_auto_segments(long long H_v);
 int launch_tc_int8(const ProblemI8& p, cudaStream_t stream);
 void int8_decay_lut(uint16_t* out256);  // table of round(2^15 * 2^(-f/256))
 

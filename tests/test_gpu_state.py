@@ -162,3 +162,57 @@ def test_token_major_layout_gives_the_same_bits():
                                     flags=gdn.GDN_FLAG_LAYOUT_BTHD)
     assert gdn.gdn_device_status() == gdn.GDN_OK
     assert torch.equal(Ot.transpose(1, 2), O) and torch.equal(St, S)
+
+
+@pytest.mark.parametrize("segments", [2, 3, 5])
+@pytest.mark.parametrize("with_state", [False, True])
+def test_segmented_call_matches_the_plain_call_and_the_oracle(segments, with_state):
+    """Few long sequences: segments' state maps in parallel, a short recurrence for their initial states, then all
+    segments with their output. Against the plain call (the state recurrence is re-associated: fp32 rounding only) and
+    against the oracle on the same W, U."""
+    C, T = 64, 1024
+    inp = gen.make_inputs(1, 1, 2, T, C, 128, 128, seed=460)
+    Q = _queries(inp, 461)
+    scale = 128 ** -0.5
+    S0 = 0.1 * torch.randn(1, 2, 128, 128, generator=torch.Generator().manual_seed(462)) if with_state else None
+    K, g = inp.K.cuda(), inp.g.cuda()
+    W, U, _ = gdn.chunk_prepare(K, inp.V.cuda(), inp.beta.cuda(), g, C, flags=gdn.GDN_FLAG_W_GATED)
+    O_ref, S_ref = gdn.chunk_state_output(Q.cuda(), K, W, U, g, C, scale, None if S0 is None else S0.cuda())
+    O, S = gdn.chunk_state_output_segmented(Q[0].cuda(), K[0], W[0], U[0], g[0], C, scale,
+                                            None if S0 is None else S0[0].cuda(), segments=segments)
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+    for hv in range(2):
+        Oo, So = orc.chunk_state_output(Q[0, 0].double().numpy(), inp.K[0, 0].double().numpy(), W[0, hv].double().cpu().numpy(),
+                                        U[0, hv].double().cpu().numpy(), inp.g[0, hv].double().numpy(), C, scale,
+                                        None if S0 is None else S0[0, hv].double().numpy())
+        eO = orc.rel_frobenius(O[hv].double().cpu().numpy().reshape(T // C, C, 128), Oo.reshape(T // C, C, 128))
+        assert eO.max() <= TOL_O, f"O rel-F {eO.max():.3e} at chunk {eO.argmax()} of head {hv}"
+        eS = orc.rel_frobenius(S[hv].double().cpu().numpy()[None], So[None])
+        assert eS.max() <= TOL_S, f"S rel-F {eS.max():.3e} of head {hv}"
+    dO = orc.rel_frobenius(O.double().cpu().numpy().reshape(2, -1, 128), O_ref[0].double().cpu().numpy().reshape(2, -1, 128))
+    assert dO.max() <= 2e-3
+
+
+def test_segmented_call_on_the_prefill_shapes():
+    """The library's own segment count on the prefill workload (32 sequences of 512 chunks): finite, deterministic, and
+    sampled heads against the oracle over the whole sequence."""
+    inp = gen.make_workload("prefill_gqa", device="cuda")
+    C, T = inp.C, inp.T
+    Q = torch.randn(inp.H_k, T, inp.d_k, device="cuda", generator=torch.Generator(device="cuda").manual_seed(470))
+    Q = (Q / Q.norm(dim=-1, keepdim=True)).to(torch.bfloat16)
+    scale = 128 ** -0.5
+    W, U, _ = gdn.chunk_prepare(inp.K, inp.V, inp.beta, inp.g, C, flags=gdn.GDN_FLAG_W_GATED)
+    O, S = gdn.chunk_state_output_segmented(Q, inp.K[0], W[0], U[0], inp.g[0], C, scale)
+    O2, S2 = gdn.chunk_state_output_segmented(Q, inp.K[0], W[0], U[0], inp.g[0], C, scale)
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+    assert bool(torch.isfinite(O).all()) and bool(torch.isfinite(S).all())
+    assert torch.equal(O, O2) and torch.equal(S, S2)
+    group = inp.H_v // inp.H_k
+    for hv in (0, inp.H_v - 1):
+        Oo, So = orc.chunk_state_output(Q[hv // group].double().cpu().numpy(), inp.K[0, hv // group].double().cpu().numpy(),
+                                        W[0, hv].double().cpu().numpy(), U[0, hv].double().cpu().numpy(),
+                                        inp.g[0, hv].double().cpu().numpy(), C, scale)
+        eO = orc.rel_frobenius(O[hv].double().cpu().numpy().reshape(T // C, C, 128), Oo.reshape(T // C, C, 128))
+        assert eO.max() <= TOL_O, f"O rel-F {eO.max():.3e} at chunk {eO.argmax()} of head {hv}"
+        eS = orc.rel_frobenius(S[hv].double().cpu().numpy()[None], So[None])
+        assert eS.max() <= TOL_S, f"S rel-F {eS.max():.3e} of head {hv}"
