@@ -431,6 +431,15 @@ def run_extras(gdn, gen, dev, args):
             out[f"{name}:state_output"] = {"chunks_per_s": inp.n_chunks / (ms * 1e-3), "ms": ms,
                                            "hbm_frac": inp.n_chunks * by / (ms * 1e-3) / 1e9 / hbm_peak,
                                            "us_per_chunk_of_a_sequence": ms * 1e3 / (inp.T // inp.C)}
+            if inp.B == 1:
+                # few long sequences: the segmented form (state maps of the segments in parallel)
+                fn = lambda: gdn.chunk_state_output_segmented(Q[0], inp.K[0], W[0], U[0], inp.g[0], inp.C, inp.d_k ** -0.5)
+                total_ms, _ = device_time_steps(fn, 5, 2, None)
+                ms = total_ms / 5
+                out[f"{name}:state_output_segmented"] = {
+                    "segments": int(gdn.load_library().gdn_chunk_state_segments(inp.H_v)),
+                    "chunks_per_s": inp.n_chunks / (ms * 1e-3), "ms": ms,
+                    "hbm_frac": inp.n_chunks * by / (ms * 1e-3) / 1e9 / hbm_peak}
             del inp, Q, W, U, outs
         except Exception as exc:
             out[f"{name}:state_output"] = {"error": repr(exc)}
