@@ -413,36 +413,6 @@ def run_extras(gdn, gen, dev, args):
             del inp, outs
         except Exception as exc:  # an unsupported extra must not lose the headline
             out[f"{name}:{method}"] = {"error": repr(exc)}
-    # the rest of the layer (state passing + output, given the gated W and U) on the prefill and stress shapes
-    for name in ("prefill_gqa", "stress"):
-        try:
-            inp = gen.make_workload(name, device=dev)
-            gq = torch.Generator(device=dev).manual_seed(99)
-            Q = torch.randn(inp.B, inp.H_k, inp.T, inp.d_k, device=dev, generator=gq)
-            Q = (Q / Q.norm(dim=-1, keepdim=True)).to(inp.K.dtype)
-            W, U, _ = gdn.chunk_prepare(inp.K, inp.V, inp.beta, inp.g, inp.C, flags=gdn.GDN_FLAG_W_GATED, want_tinv=False)
-            outs = gdn.chunk_state_output(Q, inp.K, W, U, inp.g, inp.C, inp.d_k ** -0.5)
-            fn = lambda: gdn.chunk_state_output(Q, inp.K, W, U, inp.g, inp.C, inp.d_k ** -0.5, outputs=outs)
-            total_ms, _ = device_time_steps(fn, 5, 2, None)
-            ms = total_ms / 5
-            group = inp.H_v // inp.H_k
-            # Q, K tiles (shared by a group), W, U read, O written, g
-            by = inp.C * inp.d_k * 2 * (2.0 / group + 1) + 2 * inp.C * inp.d_v * 2 + 4 * inp.C
-            out[f"{name}:state_output"] = {"chunks_per_s": inp.n_chunks / (ms * 1e-3), "ms": ms,
-                                           "hbm_frac": inp.n_chunks * by / (ms * 1e-3) / 1e9 / hbm_peak,
-                                           "us_per_chunk_of_a_sequence": ms * 1e3 / (inp.T // inp.C)}
-            if inp.B == 1:
-                # few long sequences: the segmented form (state maps of the segments in parallel)
-                fn = lambda: gdn.chunk_state_output_segmented(Q[0], inp.K[0], W[0], U[0], inp.g[0], inp.C, inp.d_k ** -0.5)
-                total_ms, _ = device_time_steps(fn, 5, 2, None)
-                ms = total_ms / 5
-                out[f"{name}:state_output_segmented"] = {
-                    "segments": int(gdn.load_library().gdn_chunk_state_segments(inp.H_v)),
-                    "chunks_per_s": inp.n_chunks / (ms * 1e-3), "ms": ms,
-                    "hbm_frac": inp.n_chunks * by / (ms * 1e-3) / 1e9 / hbm_peak}
-            del inp, Q, W, U, outs
-        except Exception as exc:
-            out[f"{name}:state_output"] = {"error": repr(exc)}
     # the model-native call on the prefill shapes: token-major tensors, raw gates, fused key normalisation, gated W;
     # and the same tokens as 201 packed sequences of ragged lengths (seeded cuts)
     try:
@@ -493,6 +463,37 @@ def run_extras(gdn, gen, dev, args):
         del inp, q, outs
     except Exception as exc:
         out["prefill_gqa:int8"] = {"error": repr(exc)}
+    # the rest of the layer (state passing + output, given the gated W and U) on the prefill and stress shapes; last,
+    # because the stress shapes (20 GB, milliseconds per launch) push the GPU into its power cap
+    for name in ("prefill_gqa", "stress"):
+        try:
+            inp = gen.make_workload(name, device=dev)
+            gq = torch.Generator(device=dev).manual_seed(99)
+            Q = torch.randn(inp.B, inp.H_k, inp.T, inp.d_k, device=dev, generator=gq)
+            Q = (Q / Q.norm(dim=-1, keepdim=True)).to(inp.K.dtype)
+            W, U, _ = gdn.chunk_prepare(inp.K, inp.V, inp.beta, inp.g, inp.C, flags=gdn.GDN_FLAG_W_GATED, want_tinv=False)
+            outs = gdn.chunk_state_output(Q, inp.K, W, U, inp.g, inp.C, inp.d_k ** -0.5)
+            fn = lambda: gdn.chunk_state_output(Q, inp.K, W, U, inp.g, inp.C, inp.d_k ** -0.5, outputs=outs)
+            total_ms, _ = device_time_steps(fn, 5, 2, None)
+            ms = total_ms / 5
+            group = inp.H_v // inp.H_k
+            # Q, K tiles (shared by a group), W, U read, O written, g
+            by = inp.C * inp.d_k * 2 * (2.0 / group + 1) + 2 * inp.C * inp.d_v * 2 + 4 * inp.C
+            out[f"{name}:state_output"] = {"chunks_per_s": inp.n_chunks / (ms * 1e-3), "ms": ms,
+                                           "hbm_frac": inp.n_chunks * by / (ms * 1e-3) / 1e9 / hbm_peak,
+                                           "us_per_chunk_of_a_sequence": ms * 1e3 / (inp.T // inp.C)}
+            if inp.B == 1:
+                # few long sequences: the segmented form (state maps of the segments in parallel)
+                fn = lambda: gdn.chunk_state_output_segmented(Q[0], inp.K[0], W[0], U[0], inp.g[0], inp.C, inp.d_k ** -0.5)
+                total_ms, _ = device_time_steps(fn, 5, 2, None)
+                ms = total_ms / 5
+                out[f"{name}:state_output_segmented"] = {
+                    "segments": int(gdn.load_library().gdn_chunk_state_segments(inp.H_v)),
+                    "chunks_per_s": inp.n_chunks / (ms * 1e-3), "ms": ms,
+                    "hbm_frac": inp.n_chunks * by / (ms * 1e-3) / 1e9 / hbm_peak}
+            del inp, Q, W, U, outs
+        except Exception as exc:
+            out[f"{name}:state_output"] = {"error": repr(exc)}
     return out
 
 
