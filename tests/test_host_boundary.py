@@ -80,6 +80,20 @@ def test_bad_arguments_are_rejected_without_a_device(lib):
     assert vl(flags=gdn.GDN_FLAG_OUT_FP32) == gdn.GDN_ERR_INVALID_ARG
     assert vl(Hk=2, Hv=3) == gdn.GDN_ERR_INVALID_ARG
     assert vl(W=mis) == gdn.GDN_ERR_ALIGN
+    lib.gdn_chunk_state_segmented_workspace.restype = ctypes.c_size_t
+    assert lib.gdn_chunk_state_segmented_workspace(32, 1) == 0
+    assert lib.gdn_chunk_state_segmented_workspace(32, 3) >= (2 * 3 + 2 * 3) * 32 * 128 * 128 * 4
+    seg = lambda **kw: lib.gdn_chunk_state_output_segmented(*[kw.get(k, d) for k, d in (
+        ("Q", p), ("K", p), ("W", p), ("U", p), ("g", p), ("Hk", 1), ("Hv", 1), ("T", 256), ("C", 64), ("dk", 128), ("dv", 128),
+        ("scale", ctypes.c_float(1.0)), ("S_in", None), ("O", p), ("S_out", None), ("segments", 2), ("ws", p),
+        ("ws_bytes", ctypes.c_size_t(1 << 30)), ("flags", 0), ("stream", None))])
+    assert seg(Q=None) == gdn.GDN_ERR_NULL
+    assert seg(ws=None) == gdn.GDN_ERR_NULL
+    assert seg(segments=0) == gdn.GDN_ERR_INVALID_ARG
+    assert seg(ws_bytes=ctypes.c_size_t(16)) == gdn.GDN_ERR_INVALID_ARG
+    assert seg(T=100) == gdn.GDN_ERR_INVALID_ARG
+    assert seg(flags=gdn.GDN_FLAG_W_GATED) == gdn.GDN_ERR_INVALID_ARG
+    assert seg(ws=mis) == gdn.GDN_ERR_ALIGN
     # valid arguments but no sm_100 device in this process: refused, nothing launched
     import torch
     if not torch.cuda.is_available():
