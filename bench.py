@@ -187,9 +187,13 @@ def time_oracle(workload: str, budget_s: float, seed_offset: int = 0):
 
 
 # ----------------------------------------------------------------------------- GPU legs
-def device_time_steps(fn, steps: int, warmup: int, dist_ctx):
+def device_time_steps(fn, steps: int, warmup: int, dist_ctx, finalize=None):
+    """Device time of `steps` calls of fn on the current stream. finalize (optional) joins work that fn left running on
+    other streams; it is called after the last step, inside the timed region."""
     for _ in range(warmup):
         fn()
+    if finalize is not None:
+        finalize()
     torch.cuda.synchronize()
     if dist_ctx is not None:
         dist_ctx.barrier()
@@ -200,9 +204,13 @@ def device_time_steps(fn, steps: int, warmup: int, dist_ctx):
     # interval would otherwise hold the host's launch latency instead of device time
     fn()
     fn()
+    if finalize is not None:
+        finalize()  # work on side streams must not leak into the timed region
     evs[0].record(stream)
     for i in range(steps):
         fn()
+        if finalize is not None and i == steps - 1:
+            finalize()
         evs[i + 1].record(stream)
     torch.cuda.synchronize()
     if dist_ctx is not None:
@@ -351,7 +359,7 @@ def run_e2e(inp, outs, gdn, args, world, n_chunks):
     steps = max(3, min(args.steps, 10))
 
     B = inp.K.shape[0]
-    streams = [torch.cuda.Stream(), torch.cuda.Stream()] if B >= 2 else []
+    streams = [torch.cuda.Stream() for _ in range(min(B, 4))] if B >= 2 else []
 
     def step_serial():
         for h, d in zip(host_in, dev_in):
@@ -362,30 +370,35 @@ def run_e2e(inp, outs, gdn, args, world, n_chunks):
 
     def step_pipelined():
         # one batch entry per slice, slices alternate between two streams: the device -> host copy of a slice
-        # overlaps the host -> device copy of the next one (PCIe is full duplex) and both overlap the kernels
-        cur = torch.cuda.current_stream()
-        start = torch.cuda.Event()
-        start.record(cur)
-        for st in streams:
-            st.wait_event(start)
+        # overlaps the host -> device copy of the next one (PCIe is full duplex) and both overlap the kernels.
+        # Consecutive steps are not joined (a slice always runs on the same stream, so its buffers are reused in
+        # order): the copies of step k + 1 start while step k drains, as in a serving loop; `join` closes the region.
         for b in range(B):
-            with torch.cuda.stream(streams[b % 2]):
+            with torch.cuda.stream(streams[b % len(streams)]):
                 for h, d in zip(host_in, dev_in):
                     d[b:b + 1].copy_(h[b:b + 1], non_blocking=True)
                 gdn.chunk_prepare(dev_in[0][b:b + 1], dev_in[1][b:b + 1], dev_in[2][b:b + 1], dev_in[3][b:b + 1], inp.C,
                                   outputs=tuple(o[b:b + 1] for o in outs))
                 for h, d in zip(host_out, outs):
                     h[b:b + 1].copy_(d[b:b + 1], non_blocking=True)
+
+    def join():
+        cur = torch.cuda.current_stream()
         for st in streams:
             done = torch.cuda.Event()
             done.record(st)
             cur.wait_event(done)
 
+    # the side streams start behind everything already queued on the current stream
+    start = torch.cuda.Event()
+    start.record(torch.cuda.current_stream())
+    for st in streams:
+        st.wait_event(start)
     step = step_pipelined if streams else step_serial
-    total_ms, _ = device_time_steps(step, steps, 2, None)
+    total_ms, _ = device_time_steps(step, steps, 2, None, finalize=join if streams else None)
     return {"value": world * n_chunks / (total_ms / steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
             "d2h_bytes_per_step": d2h, "steps": steps, "ms_per_step": total_ms / steps,
-            "pipeline": ("%d slices over 2 streams" % B) if streams else "one slice"}
+            "pipeline": ("%d slices over %d streams, steps back to back" % (B, len(streams))) if streams else "one slice"}
 
 
 def run_extras(gdn, gen, dev, args):
