@@ -229,3 +229,39 @@ def test_packed_layer_token_major_gives_the_same_bits():
     assert gdn.gdn_device_status() == gdn.GDN_OK
     assert torch.equal(Wt.transpose(0, 1), W) and torch.equal(Ut.transpose(0, 1), U)
     assert torch.equal(Ot.transpose(0, 1), O) and torch.equal(St, S)
+
+
+def test_empty_sequences_and_empty_batches():
+    """Degenerate inputs: a sequence of length zero among others (its state passes through unchanged, it has no chunk),
+    no sequences at all, and a dense call with no tokens."""
+    C = 64
+    lens = [70, 0, 5]
+    K, V, beta, g, graw, cu = _packed_inputs(lens, 1, 2, C, seed=630)
+    T = int(cu[-1])
+    Q = _queries(1, T, 631)
+    scale = 128 ** -0.5
+    S0 = (0.1 * torch.randn(3, 2, 128, 128, generator=torch.Generator().manual_seed(632))).cuda()
+    W, U, Tinv, cs, cl = gdn.chunk_prepare_varlen(K.cuda(), V.cuda(), beta.cuda(), g.cuda(), cu, C, flags=gdn.GDN_FLAG_W_GATED)
+    assert cs.cpu().tolist() == [0, 64, 70] and cl.cpu().tolist() == [64, 6, 5]
+    O, S = gdn.chunk_state_output_varlen(Q.cuda(), K.cuda(), W, U, g.cuda(), cu, C, scale, S0)
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+    assert torch.equal(S[1], S0[1])  # the empty sequence
+    for s_, L in ((0, 70), (2, 5)):
+        a = int(cu[s_])
+        for hv in range(2):
+            Oo, So = orc.gated_delta_rule(Q[0, a:a + L].double().numpy(), K[0, a:a + L].double().numpy(),
+                                          V[hv, a:a + L].double().numpy(), beta[hv, a:a + L].double().numpy(),
+                                          graw[hv, a:a + L].double().numpy(), scale, S0[s_, hv].double().cpu().numpy())
+            eO = orc.rel_frobenius(O[hv, a:a + L].double().cpu().numpy()[None], Oo[None])
+            eS = orc.rel_frobenius(S[s_, hv].double().cpu().numpy()[None], So[None])
+            assert eO.max() <= 1e-2 and eS.max() <= 1e-2
+    # no sequences, no chunks: nothing is launched, nothing is written
+    before = gdn.gdn_launch_count()
+    e32 = torch.zeros(1, dtype=torch.int32, device="cuda")
+    Wz = torch.full((2, T, 128), 3.0, dtype=torch.bfloat16, device="cuda")
+    assert gdn.gdn_chunk_prepare_varlen(K.cuda(), V.cuda(), beta.cuda(), g.cuda(), e32, e32, 0, T, 1, 2, C, 128, 128, -1, -1,
+                                        Wz, Wz.clone(), None, 0) == gdn.GDN_OK
+    assert gdn.gdn_chunk_state_output_varlen(Q.cuda(), K.cuda(), W, U, g.cuda(), e32, 0, T, 1, 2, C, 128, 128, scale, None,
+                                             Wz, None) == gdn.GDN_OK
+    assert gdn.gdn_launch_count() == before and bool((Wz == 3.0).all())
+    assert gdn.gdn_device_status() == gdn.GDN_OK
