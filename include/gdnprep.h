@@ -181,7 +181,10 @@ int gdn_chunk_prepare_varlen(const void* K, const void* V, const float* beta, co
  *   that RESTARTS in every chunk (chunk-local inclusive prefix sum), or with flags = GDN_FLAG_G_RAW the raw per-token
  *   log-gates (the prefix sum is then formed here, as gdn_chunk_prepare_ex does); with GDN_FLAG_LAYOUT_BTHD the
  *   tensors are token-major: Q, K [B,T,H_k,d_k], W_gated, U, O_out [B,T,H_v,d], g [B,T,H_v] (the state keeps its
- *   layout); no other flag is accepted; S_in [B,H_v,d_v,d_k] fp32 or NULL (zero state);
+ *   layout); with GDN_FLAG_K_L2NORM the rows of K AND of Q are L2-normalised here (1 / ||k_j|| and 1 / ||q_i|| from the
+ *   tiles in shared memory, applied to the products, so a model passes its raw projections to both calls: W_gated then
+ *   comes from gdn_chunk_prepare_ex with the same flag); no other flag is accepted; S_in [B,H_v,d_v,d_k] fp32 or NULL
+ *   (zero state);
  *   O_out [B,H_v,T,d_v] bf16; S_out [B,H_v,d_v,d_k] fp32 or NULL.
  * Supported: C = 64, d_k = d_v = 128, T a multiple of C. fp32 state, bf16 tensor-core operands.
  */

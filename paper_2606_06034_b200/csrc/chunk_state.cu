@@ -54,8 +54,9 @@ constexpr int kStageBytes = 4 * kTileBytes;  // Q, K, W, U
 constexpr int kOffQ = 0, kOffK = kTileBytes, kOffW = 2 * kTileBytes, kOffU = 3 * kTileBytes;
 constexpr int kOffP = 2 * kStageBytes;       // 2 x 8 KB: P as B operand [64 x 64] (MN-major, no swizzle), hi and lo halves
 constexpr int kOffO = kOffP + 16384;          // 2 x 16 KB: O tile staged for the bulk store (128B swizzle), two buffers
-constexpr int kOffG = kOffO + 2 * kTileBytes;  // 3 x 3 x 64 floats: exp(g_i), exp(g_C - g_j), g; three buffers
-constexpr int kSmemTotal = kOffG + 3 * 3 * 64 * 4;
+constexpr int kTab = 5 * 64;  // floats per table buffer: exp(g_i), exp(g_C - g_j), g, 1 / ||k_j||, 1 / ||q_i||
+constexpr int kOffG = kOffO + 2 * kTileBytes;  // three table buffers
+constexpr int kSmemTotal = kOffG + 3 * kTab * 4;
 
 #ifdef GDN_TRACE
 __device__ long long g_trace_s[4096];
@@ -113,14 +114,15 @@ __device__ __forceinline__ void handoff_wait() {
 
 // VAR: packed variable-length sequences (own instantiation: its masks sit on the chain the dense case is bound by)
 // SO: state only: no queries, no output (the first pass of the segmented call); U may be absent per sequence.
-template <bool VAR, bool SO>
+// NRM: GDN_FLAG_K_L2NORM (keys and queries normalised here): own instantiations, the plain chain pays nothing for it.
+template <bool VAR, bool SO, bool NRM>
 __global__ void __launch_bounds__(kThreads + 64, 1)
 chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                    const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmU,
                    const __grid_constant__ CUtensorMap tmO, const ParamsS p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    float* gtab = reinterpret_cast<float*>(smem + kOffG);  // per buffer: exp(g_i), exp(g_C - g_j), g_i (64 each)
+    float* gtab = reinterpret_cast<float*>(smem + kOffG);  // per buffer: exp(g_i), exp(g_C - g_j), g_i, 1/||k||, 1/||q|| (64 each)
 
     // One mbarrier per MMA group (never two pending phases on one barrier), two per-stage TMA barriers, and two
     // barriers on which the 256 compute threads tell the issuing warp that operands are in place.
@@ -222,12 +224,14 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                     tma_store_3d(&tmO, smem + kOffO + (c & 1) * kTileBytes, vx, tok0 + c * kC, vz);
                     tma_store_3d(&tmO, smem + kOffO + (c & 1) * kTileBytes + 8192, vx + 64, tok0 + c * kC, vz);
                     tma_store_commit();
-                    tma_store_wait_read<0>();
                 }
-                if (!SO) mbar_arrive(&bar_stg[c & 1]);  // the staging buffer may be written again (chunk c + 2)
                 if (c + 2 < n_c) {
                     if (!wait_bar(&bar_g2, par)) *fail = 1;
                     if (*fail == 0) load_stage(c + 2);
+                }
+                if (!SO) {
+                    tma_store_wait_read<0>();
+                    mbar_arrive(&bar_stg[c & 1]);  // the staging buffer may be written again (chunk c + 2)
                 }
             }
             par ^= 1;
@@ -393,9 +397,10 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         bool ok = true;
         // gate tables of a chunk: written by 64 threads into the buffer of that chunk one barrier before they are read
         const bool g_raw = (p.flags & GDN_FLAG_G_RAW) != 0;
+        constexpr bool f_nrm = NRM;
         auto fill_tables = [&](int c) {
             if (tabler) {
-                float* tb = gtab + (c % 3) * 192;
+                float* tb = gtab + (c % 3) * kTab;
                 float gc = g_reg;
                 const int left = len - c * kC;  // tokens of this chunk (>= 64 except for a short last chunk)
                 if (g_raw) {
@@ -420,14 +425,56 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                     asm volatile("bar.sync 3, 64;" ::: "memory");
                 }
                 const float gC = tb[128 + 63];  // cumulative gate of the chunk's last token
-                tb[tt] = fast_exp2(gc * kLog2e);
-                tb[64 + tt] = fast_exp2((gC - gc) * kLog2e);
+                // (with the keys and queries normalised here, their factors ride on the two gate factors: exp(g_i) only
+                // ever multiplies a product with q_i, exp(g_C - g_j) one with k_j)
+                tb[tt] = fast_exp2(gc * kLog2e) * (f_nrm ? tb[256 + tt] : 1.f);
+                tb[64 + tt] = fast_exp2((gC - gc) * kLog2e) * (f_nrm ? tb[192 + tt] : 1.f);
             }
         };
-        if (n_c > 0) fill_tables(0);
+        // GDN_FLAG_K_L2NORM: 1 / ||k_j|| and 1 / ||q_i|| of chunk c from its tiles in shared memory, by the 256 threads
+        // whose lanes hold no row of P (the sum of squares of a row does not care about the swizzle inside the row)
+        auto fill_norms = [&](int c) {
+            if (wq >= 2) {
+                // (the issuing warp has waited for these tiles, or will; observing the phase here orders the reads below)
+                if (!wait_bar(&bar_full[c & 1], (c >> 1) & 1)) *fail = 1;
+                const int u = (tid >> 7) * 64 + (tid & 63);  // 0 .. 255
+                float* tb = gtab + (c % 3) * kTab;
+                // A warp reads 512 contiguous bytes per step (four rows of a 64-column sub-tile): conflict-free. Thread u
+                // sees rows u >> 3 and 32 + (u >> 3) of both sub-tiles; the eight lanes of a row add up by shuffles.
+#pragma unroll
+                for (int which = 0; which < (SO ? 1 : 2); ++which) {
+                    const uint8_t* tile = smem + (c & 1) * kStageBytes + (which == 0 ? kOffK : kOffQ) + u * 16;
+                    float acc[2] = {0.f, 0.f};
+#pragma unroll
+                    for (int it = 0; it < 4; ++it) {
+                        const uint4 w4 = *reinterpret_cast<const uint4*>(tile + (it >> 1) * 8192 + (it & 1) * 4096);
+                        const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const float a = __uint_as_float(w[i] << 16), b = __uint_as_float(w[i] & 0xFFFF0000u);
+                            acc[it & 1] = fmaf(a, a, fmaf(b, b, acc[it & 1]));
+                        }
+                    }
+#pragma unroll
+                    for (int off = 1; off < 8; off <<= 1) {
+                        acc[0] += __shfl_xor_sync(0xFFFFFFFFu, acc[0], off);
+                        acc[1] += __shfl_xor_sync(0xFFFFFFFFu, acc[1], off);
+                    }
+                    if ((u & 7) == 0) {
+                        tb[(which == 0 ? 192 : 256) + (u >> 3)] = rsqrtf(fmaxf(acc[0], 1e-30f));
+                        tb[(which == 0 ? 192 : 256) + 32 + (u >> 3)] = rsqrtf(fmaxf(acc[1], 1e-30f));
+                    }
+                }
+                asm volatile("bar.sync 7, 256;" ::: "memory");
+            }
+        };
+        if (n_c > 0) {
+            if (f_nrm) fill_norms(0);
+            fill_tables(0);
+        }
         asm volatile("bar.sync 1, 512;" ::: "memory");
         for (int c = 0; c < n_c; ++c) {
-            const float* se = gtab + (c % 3) * 192;  // exp(g_i)
+            const float* se = gtab + (c % 3) * kTab;  // exp(g_i)
             const float* sf = se + 64;               // exp(g_C - g_j)
             const float* sg = se + 128;              // g_i (cumulative inside the chunk)
             const float gC = sg[63];
@@ -462,6 +509,7 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 tmem_ld16(lane_base + kPT + h * 16, d);
                 tmem_wait_ld();
                 const float gj = sg[t] * kLog2e;
+                const float rkj = f_nrm ? sg[64 + t] : 1.f;
                 float gi16[16];  // g of this thread's 16 columns (four 16-byte loads instead of sixteen scalar ones)
 #pragma unroll
                 for (int i4 = 0; i4 < 4; ++i4) {
@@ -477,8 +525,9 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 #pragma unroll
                         for (int q = 0; q < 2; ++q) {
                             const int i = h * 16 + c2 * 8 + i2 * 2 + q;
-                            const float x = __uint_as_float(d[c2 * 8 + i2 * 2 + q]) *
-                                            fast_exp2(fminf(fmaf(gi16[c2 * 8 + i2 * 2 + q], kLog2e, -gj), 0.f));
+                            float x = __uint_as_float(d[c2 * 8 + i2 * 2 + q]) *
+                                      fast_exp2(fminf(fmaf(gi16[c2 * 8 + i2 * 2 + q], kLog2e, -gj), 0.f));
+                            if (f_nrm) x *= rkj * sg[128 + i];  // 1 / (||k_j|| ||q_i||)
                             v[q] = (t <= i) ? x : 0.f;
                         }
                         w[i2] = pack_bf16x2(v[0], v[1]);
@@ -490,7 +539,7 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 }
             }
             // the next chunk's gate tables, by threads that had no part in P (published by the barrier at the chunk's end)
-            if (c + 1 < n_c) fill_tables(c + 1);
+            if (c + 1 < n_c && !f_nrm) fill_tables(c + 1);
             // ---- U_new^T = -D1 as bf16 hi + lo, plain and gate-scaled (the sums over the tokens of a chunk telescope
             // on correlated keys, so single bf16 copies cost 1e-2 there). This thread's 16 tokens are one k-step of the
             // products that consume them: the hi halves are written over its own D1 columns (plain -> 16 h .. 16 h + 7,
@@ -530,6 +579,12 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             tc_fence_before_sync();
             handoff_arrive<5>();
             STAMPS(7);
+            // with the norms of the next chunk's keys and queries in the tables, both are formed here instead: the next
+            // chunk's tiles are still on their way while P is formed, and the threads idle now anyway
+            if (c + 1 < n_c && f_nrm) {
+                fill_norms(c + 1);
+                fill_tables(c + 1);
+            }
 
             if (!SO) {
                 // the bulk store of chunk c - 2 has finished reading this chunk's staging buffer (polled here, in the shadow of
@@ -842,7 +897,10 @@ int launch_chunk_state(const ProblemS& q, cudaStream_t stream) {
     prm.seq_no_u = q.seq_no_u;
     prm.O = static_cast<__nv_bfloat16*>(q.O);
     const int smem = kSmemTotal + 1024;
-    auto kern = q.state_only ? chunk_state_kernel<true, true> : (var ? chunk_state_kernel<true, false> : chunk_state_kernel<false, false>);
+    const bool nrm = (q.flags & GDN_FLAG_K_L2NORM) != 0;
+    auto kern = q.state_only ? (nrm ? chunk_state_kernel<true, true, true> : chunk_state_kernel<true, true, false>)
+                : var        ? (nrm ? chunk_state_kernel<true, false, true> : chunk_state_kernel<true, false, false>)
+                             : (nrm ? chunk_state_kernel<false, false, true> : chunk_state_kernel<false, false, false>);
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return GDN_ERR_LAUNCH;
     kern<<<static_cast<int>(n_cta), kThreads + 64, smem, stream>>>(mQ, mK, mW, mU, mO, prm);
     count_launch();

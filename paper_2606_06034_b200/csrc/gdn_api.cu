@@ -180,7 +180,7 @@ int gdn_chunk_prepare_int8(const int8_t* Kq, const int8_t* Vq, const int32_t* k_
 int gdn_chunk_state_output(const void* Q, const void* K, const void* W_gated, const void* U, const float* g, int B, int H_k,
                            int H_v, int T, int C, int d_k, int d_v, float scale, const float* S_in, void* O_out, float* S_out,
                            unsigned flags, gdn_stream_t stream) {
-    if (flags & ~static_cast<unsigned>(GDN_FLAG_G_RAW | GDN_FLAG_LAYOUT_BTHD)) return GDN_ERR_INVALID_ARG;
+    if (flags & ~static_cast<unsigned>(GDN_FLAG_G_RAW | GDN_FLAG_LAYOUT_BTHD | GDN_FLAG_K_L2NORM)) return GDN_ERR_INVALID_ARG;
     if (Q == nullptr || K == nullptr || W_gated == nullptr || U == nullptr || g == nullptr || O_out == nullptr) return GDN_ERR_NULL;
     if (B < 0 || H_k <= 0 || H_v <= 0 || T < 0 || C < 2 || d_k <= 0 || d_v <= 0) return GDN_ERR_INVALID_ARG;
     if (H_v % H_k != 0 || T % C != 0) return GDN_ERR_INVALID_ARG;
@@ -203,7 +203,7 @@ int gdn_chunk_state_output_segmented(const void* Q, const void* K, const void* W
                                      int H_v, int T, int C, int d_k, int d_v, float scale, const float* S_in, void* O_out,
                                      float* S_out, int segments, void* workspace, size_t workspace_bytes, unsigned flags,
                                      gdn_stream_t stream) {
-    if (flags & ~static_cast<unsigned>(GDN_FLAG_G_RAW | GDN_FLAG_LAYOUT_BTHD)) return GDN_ERR_INVALID_ARG;
+    if (flags & ~static_cast<unsigned>(GDN_FLAG_G_RAW | GDN_FLAG_LAYOUT_BTHD | GDN_FLAG_K_L2NORM)) return GDN_ERR_INVALID_ARG;
     if (Q == nullptr || K == nullptr || W_gated == nullptr || U == nullptr || g == nullptr || O_out == nullptr) return GDN_ERR_NULL;
     if (H_k <= 0 || H_v <= 0 || T < 0 || C < 2 || d_k <= 0 || d_v <= 0 || segments < 1 || segments > 64) return GDN_ERR_INVALID_ARG;
     if (H_v % H_k != 0 || T % C != 0) return GDN_ERR_INVALID_ARG;
@@ -222,7 +222,7 @@ int gdn_chunk_state_output_varlen(const void* Q, const void* K, const void* W_ga
                                   const int32_t* cu_seqlens, int n_seq, int T_total, int H_k, int H_v, int C, int d_k, int d_v,
                                   float scale, const float* S_in, void* O_out, float* S_out, unsigned flags,
                                   gdn_stream_t stream) {
-    if (flags & ~static_cast<unsigned>(GDN_FLAG_G_RAW | GDN_FLAG_LAYOUT_BTHD)) return GDN_ERR_INVALID_ARG;
+    if (flags & ~static_cast<unsigned>(GDN_FLAG_G_RAW | GDN_FLAG_LAYOUT_BTHD | GDN_FLAG_K_L2NORM)) return GDN_ERR_INVALID_ARG;
     if (Q == nullptr || K == nullptr || W_gated == nullptr || U == nullptr || g == nullptr || O_out == nullptr ||
         cu_seqlens == nullptr)
         return GDN_ERR_NULL;

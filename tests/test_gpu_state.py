@@ -113,7 +113,7 @@ def test_state_output_argument_errors():
     assert gdn.gdn_chunk_state_output(K, K, K, K, g, 1, 1, 1, 128, 32, 128, 128, 1.0, None, O, None, 0, **args) == gdn.GDN_ERR_UNSUPPORTED
     assert gdn.gdn_chunk_state_output(K, K, K, K, g, 1, 1, 1, 100, 64, 128, 128, 1.0, None, O, None, 0, **args) == gdn.GDN_ERR_INVALID_ARG
     assert gdn.gdn_chunk_state_output(None, K, K, K, g, 1, 1, 1, 128, 64, 128, 128, 1.0, None, O, None, 0, **args) == gdn.GDN_ERR_NULL
-    assert gdn.gdn_chunk_state_output(K, K, K, K, g, 1, 1, 1, 128, 64, 128, 128, 1.0, None, O, None, 2, **args) == gdn.GDN_ERR_INVALID_ARG
+    assert gdn.gdn_chunk_state_output(K, K, K, K, g, 1, 1, 1, 128, 64, 128, 128, 1.0, None, O, None, gdn.GDN_FLAG_OUT_FP32, **args) == gdn.GDN_ERR_INVALID_ARG
     assert gdn.gdn_device_status() == gdn.GDN_OK
 
 
@@ -216,3 +216,37 @@ def test_segmented_call_on_the_prefill_shapes():
         assert eO.max() <= TOL_O, f"O rel-F {eO.max():.3e} at chunk {eO.argmax()} of head {hv}"
         eS = orc.rel_frobenius(S[hv].double().cpu().numpy()[None], So[None])
         assert eS.max() <= TOL_S, f"S rel-F {eS.max():.3e} of head {hv}"
+
+
+@pytest.mark.parametrize("token_major", [False, True])
+def test_model_native_layer_from_raw_projections(token_major):
+    """The call sequence of a model: raw key / query projections (normalised inside both kernels), raw log-gates,
+    optionally token-major tensors; against the token-by-token rule on the normalised keys and queries."""
+    C, T = 64, 448
+    inp = gen.make_inputs(1, 2, 4, T, C, 128, 128, seed=480)
+    gq = torch.Generator().manual_seed(481)
+    Qun = (1.3 * torch.randn(1, 2, T, 128, generator=gq)).to(torch.bfloat16)
+    Kun = (inp.K.float() * (0.5 + torch.rand(1, 2, T, 1, generator=gq))).to(torch.bfloat16)
+    scale = 128 ** -0.5
+    graw = inp.g.view(1, 4, T // C, C).diff(dim=-1, prepend=torch.zeros(1, 4, T // C, 1)).reshape(1, 4, T).contiguous()
+    f1 = gdn.GDN_FLAG_W_GATED | gdn.GDN_FLAG_G_RAW | gdn.GDN_FLAG_K_L2NORM
+    f2 = gdn.GDN_FLAG_G_RAW | gdn.GDN_FLAG_K_L2NORM
+    if token_major:
+        tm = lambda x: x.transpose(1, 2).contiguous().cuda()
+        b = gdn.GDN_FLAG_LAYOUT_BTHD
+        W, U, _ = gdn.chunk_prepare(tm(Kun), tm(inp.V), tm(inp.beta), tm(graw), C, flags=f1 | b, want_tinv=False)
+        O, S = gdn.chunk_state_output(tm(Qun), tm(Kun), W, U, tm(graw), C, scale, flags=f2 | b)
+        O = O.transpose(1, 2)
+    else:
+        W, U, _ = gdn.chunk_prepare(Kun.cuda(), inp.V.cuda(), inp.beta.cuda(), graw.cuda(), C, flags=f1, want_tinv=False)
+        O, S = gdn.chunk_state_output(Qun.cuda(), Kun.cuda(), W, U, graw.cuda(), C, scale, flags=f2)
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+    Kn = Kun.double() / Kun.double().norm(dim=-1, keepdim=True)
+    Qn = Qun.double() / Qun.double().norm(dim=-1, keepdim=True)
+    for hv in range(4):
+        Oo, So = orc.gated_delta_rule(Qn[0, hv // 2].numpy(), Kn[0, hv // 2].numpy(), inp.V[0, hv].double().numpy(),
+                                      inp.beta[0, hv].double().numpy(), graw[0, hv].double().numpy(), scale)
+        eO = orc.rel_frobenius(O[0, hv].double().cpu().numpy().reshape(T // C, C, 128), Oo.reshape(T // C, C, 128))
+        assert eO.max() <= 1e-2, f"O rel-F {eO.max():.3e} at chunk {eO.argmax()} of head {hv}"
+        eS = orc.rel_frobenius(S[0, hv].double().cpu().numpy()[None], So[None])
+        assert eS.max() <= 1e-2, f"S rel-F {eS.max():.3e} of head {hv}"
