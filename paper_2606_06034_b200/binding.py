@@ -394,6 +394,22 @@ def chunk_state_output(Q, K, W_gated, U, g, C, scale=1.0, S_in=None, *, want_sta
     return O, S_out
 
 
+def gated_delta_layer(Q, K, V, beta, g_raw, C=64, scale=None, S_in=None, *, cu_seqlens=None, token_major=True,
+                      qk_l2norm=True, want_state=True):
+    """The chunk-wise layer as model code calls it: the two library calls back to back (chunk-prepare with the gated W,
+    then state passing and output) on raw per-token log-gates and, with qk_l2norm, raw key / query projections.
+    Dense: Q, K [B,T,H_k,d], V [B,T,H_v,d], beta, g_raw [B,T,H_v] (token_major) or the head-major forms. Packed
+    sequences (cu_seqlens on the host): the same tensors without the batch axis. Returns (O, S_out or None)."""
+    flags = GDN_FLAG_G_RAW | (GDN_FLAG_LAYOUT_BTHD if token_major else 0) | (GDN_FLAG_K_L2NORM if qk_l2norm else 0)
+    if scale is None:
+        scale = float(K.shape[-1]) ** -0.5
+    if cu_seqlens is not None:
+        W, U, _, _, _ = chunk_prepare_varlen(K, V, beta, g_raw, cu_seqlens, C, flags=flags | GDN_FLAG_W_GATED, want_tinv=False)
+        return chunk_state_output_varlen(Q, K, W, U, g_raw, cu_seqlens, C, scale, S_in, want_state=want_state, flags=flags)
+    W, U, _ = chunk_prepare(K, V, beta, g_raw, C, flags=flags | GDN_FLAG_W_GATED, want_tinv=False)
+    return chunk_state_output(Q, K, W, U, g_raw, C, scale, S_in, want_state=want_state, flags=flags)
+
+
 def gdn_selftest_bounded_wait() -> int:
     """Enqueues the bounded-wait self-test on torch's current stream (see the header)."""
     return load_library().gdn_selftest_bounded_wait(_stream())

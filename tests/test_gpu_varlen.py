@@ -265,3 +265,28 @@ def test_empty_sequences_and_empty_batches():
                                              Wz, None) == gdn.GDN_OK
     assert gdn.gdn_launch_count() == before and bool((Wz == 3.0).all())
     assert gdn.gdn_device_status() == gdn.GDN_OK
+
+
+def test_layer_wrapper_on_packed_token_major_raw_projections():
+    """`gated_delta_layer`: packed sequences, token-major tensors, raw gates, raw key / query projections, one call."""
+    C = 64
+    lens = [150, 64, 9, 200]
+    K, V, beta, g, graw, cu = _packed_inputs(lens, 2, 4, C, seed=640)
+    T = int(cu[-1])
+    gq = torch.Generator().manual_seed(641)
+    Qun = (1.7 * torch.randn(2, T, 128, generator=gq)).to(torch.bfloat16)
+    Kun = (K.float() * (0.5 + torch.rand(2, T, 1, generator=gq))).to(torch.bfloat16)
+    tm = lambda x: x.transpose(0, 1).contiguous().cuda()
+    O, S = gdn.gated_delta_layer(tm(Qun), tm(Kun), tm(V), tm(beta), tm(graw), C, cu_seqlens=cu)
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+    O = O.transpose(0, 1)
+    Kn = Kun.double() / Kun.double().norm(dim=-1, keepdim=True)
+    Qn = Qun.double() / Qun.double().norm(dim=-1, keepdim=True)
+    for s_, L in enumerate(lens):
+        a = int(cu[s_])
+        for hv in range(4):
+            Oo, So = orc.gated_delta_rule(Qn[hv // 2, a:a + L].numpy(), Kn[hv // 2, a:a + L].numpy(), V[hv, a:a + L].double().numpy(),
+                                          beta[hv, a:a + L].double().numpy(), graw[hv, a:a + L].double().numpy(), 128 ** -0.5)
+            eO = orc.rel_frobenius(O[hv, a:a + L].double().cpu().numpy()[None], Oo[None])
+            eS = orc.rel_frobenius(S[s_, hv].double().cpu().numpy()[None], So[None])
+            assert eO.max() <= 1e-2 and eS.max() <= 1e-2, f"sequence {s_} head {hv}: O {eO.max():.3e} S {eS.max():.3e}"
