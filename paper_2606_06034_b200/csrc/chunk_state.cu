@@ -646,6 +646,9 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 handoff_arrive<4>();
             }
             STAMPS(11);
+            // With the norms in the tables, the next chunk's tables are written after this chunk's hand-off (see above),
+            // so the hand-off -> product -> completion chain does not order them before their readers: one barrier.
+            if (NRM && c + 1 < n_c) asm volatile("bar.sync 1, 512;" ::: "memory");
             if (!SO && short_chunk) {
                 // only the rows of real tokens leave, 16 bytes per thread and step, from the staged (swizzled) tile
                 asm volatile("bar.sync 1, 512;" ::: "memory");  // (last chunk of a packed sequence only)
