@@ -258,9 +258,17 @@ def run_ours(args, rank, world, dist_ctx):
         st_outs = gdn.chunk_state_output(Qs, inp.K, Wg, Ug, inp.g, C, inp.d_k ** -0.5)
         st_args = (Qs, Wg, Ug, st_outs)
 
+    mn_args = None
+    if method == "model-native":  # token-major tensors, raw gates, fused key normalisation, gated W (what a model passes)
+        mn_in = tuple(x.transpose(1, 2).contiguous() for x in (inp.K, inp.V, inp.beta, inp.g))
+        mn_flags = gdn.GDN_FLAG_LAYOUT_BTHD | gdn.GDN_FLAG_G_RAW | gdn.GDN_FLAG_K_L2NORM | gdn.GDN_FLAG_W_GATED
+        mn_args = (mn_in, gdn.alloc_outputs(mn_in[0], mn_in[1], C, True, True), mn_flags)
+
     def step():
         if method == "neumann":
             gdn.chunk_prepare(inp.K, inp.V, inp.beta, inp.g, C, outputs=outs)
+        elif method == "model-native":
+            gdn.chunk_prepare(*mn_args[0], C, outputs=mn_args[1], flags=mn_args[2])
         elif method == "int8":
             gdn.chunk_prepare_int8(q8, outputs=q8_outs)
         elif method == "state":
@@ -543,7 +551,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--method", default="neumann", choices=["neumann", "fwdsubst", "fwdsubst-blocked", "int8", "state"])
+    ap.add_argument("--method", default="neumann", choices=["neumann", "fwdsubst", "fwdsubst-blocked", "int8", "state", "model-native"])
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extras", action="store_true")
