@@ -120,3 +120,39 @@ def test_repeated_int8_launches_are_bit_identical():
         for a, b in zip(out, ref):
             assert torch.equal(a, b), f"launch {rep} differs from the first"
     assert gdn.gdn_device_status() == gdn.GDN_OK
+
+
+def test_packed_sequences_at_full_size():
+    """The prefill shapes as 201 packed sequences of ragged lengths (the benchmark's extra): sampled chunk slots,
+    short ones included, against the oracle; every row finite; a second launch agrees bit for bit."""
+    inp = gen.make_workload("prefill_gqa", device="cuda")
+    C, T = inp.C, inp.T
+    cuts = np.sort(np.random.default_rng(0).choice(np.arange(1, T), size=200, replace=False))
+    cu = [0] + cuts.tolist() + [T]
+    K, V, beta, g = inp.K[0], inp.V[0], inp.beta[0], inp.g[0]
+    # the workload's cumulative gates restart every 64 tokens of the dense axis; packed chunks start elsewhere, so the
+    # raw gates are recovered and passed as such
+    graw = g.view(inp.H_v, T // C, C).diff(dim=-1, prepend=torch.zeros(inp.H_v, T // C, 1, device="cuda")).reshape(inp.H_v, T).contiguous()
+    W, U, Tinv, cs, cl = gdn.chunk_prepare_varlen(K, V, beta, graw, cu, C, flags=gdn.GDN_FLAG_G_RAW)
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+    W2, U2, T2, _, _ = gdn.chunk_prepare_varlen(K, V, beta, graw, cu, C, flags=gdn.GDN_FLAG_G_RAW)
+    assert torch.equal(W, W2) and torch.equal(U, U2) and torch.equal(Tinv, T2)
+    assert bool(torch.isfinite(W).all()) and bool(torch.isfinite(U).all()) and bool(torch.isfinite(Tinv).all())
+    start, length = cs.cpu().tolist(), cl.cpu().tolist()
+    rng = np.random.default_rng(9)
+    short = [i for i, n in enumerate(length) if n < C]
+    pick = sorted(set([0, len(start) - 1] + rng.choice(short, size=12, replace=False).tolist() +
+                      rng.choice(len(start), size=12, replace=False).tolist()))
+    group = inp.H_v // inp.H_k
+    for hv in (0, inp.H_v - 1):
+        for c in pick:
+            a, L = start[c], length[c]
+            Kc = np.zeros((C, 128)); Vc = np.zeros((C, 128)); bc = np.zeros(C); gc = np.zeros(C)
+            Kc[:L] = K[hv // group, a:a + L].double().cpu().numpy(); Vc[:L] = V[hv, a:a + L].double().cpu().numpy()
+            bc[:L] = beta[hv, a:a + L].double().cpu().numpy(); gc[:L] = graw[hv, a:a + L].double().cpu().numpy()
+            Wo, Uo, To = orc.chunk_prepare(Kc, Vc, bc, gc, g_raw=True)
+            for label, got, ref in (("W", W[hv, a:a + L], Wo[:L]), ("U", U[hv, a:a + L], Uo[:L]), ("Tinv", Tinv[hv, c], To)):
+                err = orc.rel_frobenius(got.double().cpu().numpy()[None], ref[None])[0]
+                floor = orc.rel_frobenius(_bf16_round(ref)[None], ref[None])[0]
+                bound = max(TOL_BF16, floor + 2e-4) if floor > 0.9 * TOL_BF16 else TOL_BF16
+                assert err <= bound, f"{label} head {hv} chunk slot {c} (len {L}): rel-F {err:.3e} > {bound:.3e}"
