@@ -61,7 +61,10 @@ constexpr int kSmemTotal = kOffG + 3 * kTab * 4;
 #ifdef GDN_TRACE
 __device__ long long g_trace_s[4096];
 // slot, clock pairs of block 0: compute thread 0 at [0, 2048), the issuing warp's lane 0 at [2048, 4096)
-#define STAMPS(slot_) do { if (blockIdx.x == 0 && (tid == 0 || tid == kThreads) && trace_n < 500) { \
+#ifndef GDN_TRACE_SO
+#define GDN_TRACE_SO false
+#endif
+#define STAMPS(slot_) do { if (SO == GDN_TRACE_SO && blockIdx.x == 0 && (tid == 0 || tid == kThreads) && trace_n < 500) { \
     g_trace_s[(tid == 0 ? 0 : 2048) + trace_n * 2] = (slot_); g_trace_s[(tid == 0 ? 0 : 2048) + trace_n * 2 + 1] = clock64(); ++trace_n; } } while (0)
 #else
 #define STAMPS(slot_) do { } while (0)
