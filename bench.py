@@ -291,6 +291,24 @@ def run_ours(args, rank, world, dist_ctx):
     total_ms, per = device_time_steps(step, args.steps, 0, dist_ctx)
     clocks = sampler.stop()
     launches = gdn.gdn_launch_count() - launches0 - 2  # the two queue-priming launches sit before the first event
+    # a timed region that saw a thermal or hardware slowdown, or clocks far below maximum with no reason given (a leftover
+    # clock lock), is not a measurement: take it once more and say so
+    bad = {"hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown"} & set(clocks.get("reasons") or [])
+    stuck = (clocks.get("sm_mhz") and clocks.get("sm_max_mhz") and not clocks.get("reasons")
+             and clocks["sm_mhz"] < 0.8 * clocks["sm_max_mhz"])
+    remeasured = False
+    again = 1.0 if (bad or stuck) else 0.0
+    again = max_over_ranks(again, dev, dist_ctx) > 0.0  # every rank takes the same decision
+    if again:
+        time.sleep(2.0)
+        sampler = ClockSampler(torch.cuda.current_device())
+        launches0 = gdn.gdn_launch_count()
+        sampler.start()
+        total_ms, per = device_time_steps(step, args.steps, 0, dist_ctx)
+        first, clocks = clocks, sampler.stop()
+        clocks["first_attempt"] = first
+        launches = gdn.gdn_launch_count() - launches0 - 2
+        remeasured = True
     status = gdn.gdn_device_status()
     if status != gdn.GDN_OK:
         raise RuntimeError(f"kernel status {status}")
@@ -339,6 +357,8 @@ def run_ours(args, rank, world, dist_ctx):
         "effective_tflops": world * n_chunks * flops_chunk / (ms_per_step * 1e-3) / 1e12,
         "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline,
     }
+    if remeasured:
+        line["remeasured"] = True
 
     if rank == 0 and not args.no_e2e and method == "neumann":
         line["e2e"] = run_e2e(inp, outs, gdn, args, world, n_chunks)
