@@ -21,8 +21,14 @@
 //     O^T = scale (exp(g_i) O1 + O2)  -> transposed through shared memory -> bulk tensor store
 // Two MMA groups per chunk; Q, K, W, U tiles of the next chunk are in flight (two stages) while a chunk is worked on.
 // All operand layouts are the ones the chunk-prepare kernel uses.
-// Packed variable-length sequences (second instantiation): one CTA per (sequence, value head), starting at the
-// sequence's first token; the tokens a short last chunk lacks decay nothing and write nothing.
+// Warps: 16 compute warps (four threads per TMEM lane), one that issues every MMA, one that issues the TMA loads and
+// the output stores. The chain of a sequence is thread work (every phase runs on all 16 warps at once, so its
+// instruction count is what it costs); hand-offs to the issuing warp are hardware barriers, completions come back
+// through mbarriers (a poll costs ~200 cycles, so as few as possible are waited for).
+// Instantiations: packed variable-length sequences (one CTA per (sequence, value head), starting at the sequence's
+// first token; the tokens a short last chunk lacks decay nothing and write nothing); state only (no queries, no
+// output: the first pass of the segmented call for few long sequences, see launch_chunk_state_segmented); keys and
+// queries L2-normalised here (GDN_FLAG_K_L2NORM).
 #include <cuda.h>
 
 #include "common.cuh"
@@ -127,8 +133,9 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     float* gtab = reinterpret_cast<float*>(smem + kOffG);  // per buffer: exp(g_i), exp(g_C - g_j), g_i, 1/||k||, 1/||q|| (64 each)
 
-    // One mbarrier per MMA group (never two pending phases on one barrier), two per-stage TMA barriers, and two
-    // barriers on which the 256 compute threads tell the issuing warp that operands are in place.
+    // One mbarrier per MMA group that is waited for (never two pending phases on one barrier), two per-stage TMA
+    // barriers, and two on which the storing warp releases the output staging buffers. The hand-offs from the 512
+    // compute threads to the issuing and the storing warp go over hardware barriers 4, 5 and 6 (handoff_arrive / _wait).
     __shared__ uint64_t bar_full[2], bar_pre, bar_d1, bar_o2, bar_g2, bar_stg[2];
     __shared__ uint32_t tmem_base_s;
     __shared__ int s_fail;
