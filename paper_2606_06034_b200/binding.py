@@ -407,6 +407,12 @@ def gated_delta_layer(Q, K, V, beta, g_raw, C=64, scale=None, S_in=None, *, cu_s
         W, U, _, _, _ = chunk_prepare_varlen(K, V, beta, g_raw, cu_seqlens, C, flags=flags | GDN_FLAG_W_GATED, want_tinv=False)
         return chunk_state_output_varlen(Q, K, W, U, g_raw, cu_seqlens, C, scale, S_in, want_state=want_state, flags=flags)
     W, U, _ = chunk_prepare(K, V, beta, g_raw, C, flags=flags | GDN_FLAG_W_GATED, want_tinv=False)
+    H_v = V.shape[2] if token_major else V.shape[1]
+    if K.shape[0] == 1 and int(load_library().gdn_chunk_state_segments(H_v)) > 1:
+        # one long sequence per head and fewer heads than SMs: the segments of a sequence run in parallel
+        O, S = chunk_state_output_segmented(Q[0], K[0], W[0], U[0], g_raw[0], C, scale, None if S_in is None else S_in[0],
+                                            want_state=want_state, flags=flags)
+        return O[None], (None if S is None else S[None])
     return chunk_state_output(Q, K, W, U, g_raw, C, scale, S_in, want_state=want_state, flags=flags)
 
 

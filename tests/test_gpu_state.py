@@ -250,3 +250,30 @@ def test_model_native_layer_from_raw_projections(token_major):
         assert eO.max() <= 1e-2, f"O rel-F {eO.max():.3e} at chunk {eO.argmax()} of head {hv}"
         eS = orc.rel_frobenius(S[0, hv].double().cpu().numpy()[None], So[None])
         assert eS.max() <= 1e-2, f"S rel-F {eS.max():.3e} of head {hv}"
+
+
+def test_layer_wrapper_one_long_sequence_per_head_takes_the_segmented_path():
+    """B = 1 with few heads: `gated_delta_layer` runs the segments of every sequence in parallel (raw projections,
+    token-major tensors, raw gates); against the token-by-token rule."""
+    C, T = 64, 1536
+    inp = gen.make_inputs(1, 1, 2, T, C, 128, 128, seed=490)
+    gq = torch.Generator().manual_seed(491)
+    Qun = (1.3 * torch.randn(1, 1, T, 128, generator=gq)).to(torch.bfloat16)
+    Kun = (inp.K.float() * (0.5 + torch.rand(1, 1, T, 1, generator=gq))).to(torch.bfloat16)
+    graw = inp.g.view(1, 2, T // C, C).diff(dim=-1, prepend=torch.zeros(1, 2, T // C, 1)).reshape(1, 2, T).contiguous()
+    S0 = 0.1 * torch.randn(1, 2, 128, 128, generator=torch.Generator().manual_seed(492))
+    tm = lambda x: x.transpose(1, 2).contiguous().cuda()
+    assert gdn.load_library().gdn_chunk_state_segments(2) > 1
+    O, S = gdn.gated_delta_layer(tm(Qun), tm(Kun), tm(inp.V), tm(inp.beta), tm(graw), C, S_in=S0.cuda())
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+    O = O.transpose(1, 2)
+    Kn = Kun.double() / Kun.double().norm(dim=-1, keepdim=True)
+    Qn = Qun.double() / Qun.double().norm(dim=-1, keepdim=True)
+    for hv in range(2):
+        Oo, So = orc.gated_delta_rule(Qn[0, 0].numpy(), Kn[0, 0].numpy(), inp.V[0, hv].double().numpy(),
+                                      inp.beta[0, hv].double().numpy(), graw[0, hv].double().numpy(), 128 ** -0.5,
+                                      S0[0, hv].double().numpy())
+        eO = orc.rel_frobenius(O[0, hv].double().cpu().numpy().reshape(T // C, C, 128), Oo.reshape(T // C, C, 128))
+        assert eO.max() <= 1e-2, f"O rel-F {eO.max():.3e} at chunk {eO.argmax()} of head {hv}"
+        eS = orc.rel_frobenius(S[0, hv].double().cpu().numpy()[None], So[None])
+        assert eS.max() <= 1e-2, f"S rel-F {eS.max():.3e} of head {hv}"
