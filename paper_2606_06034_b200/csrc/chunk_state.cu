@@ -597,9 +597,12 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             }
 
             if (!SO) {
-                // the bulk store of chunk c - 2 has finished reading this chunk's staging buffer (polled here, in the shadow of
-                // the output product)
-                if (c >= 2 && !wait_bar(&bar_stg[c & 1], ((c - 2) >> 1) & 1)) { *fail = 1; ok = false; break; }
+                // The storing warp has released the PREVIOUS chunk's staging buffer (polled here, in the shadow of the
+                // output product; the store was issued most of a chunk ago). That is one chunk later than this chunk's
+                // own buffer needs (chunk c - 2 used it, and the stores are read in order), but it also says that the
+                // storing warp has taken the previous chunk's hand-off: the threads must not arrive on that hardware
+                // barrier a second time before it has, however long a store may be held up.
+                if (c >= 1 && !wait_bar(&bar_stg[(c - 1) & 1], ((c - 1) >> 1) & 1)) { *fail = 1; ok = false; break; }
                 // ---- exp(g_i) O1 (complete with O2: products finish in the order they were issued)
                 if (!wait_group(&bar_o2, par_o2)) { ok = false; break; }
                 STAMPS(8);
