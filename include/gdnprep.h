@@ -44,6 +44,7 @@
 #ifndef GDNPREP_H_
 #define GDNPREP_H_
 
+#include <stddef.h>
 #include <stdint.h>
 
 #ifdef __cplusplus

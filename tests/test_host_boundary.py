@@ -122,3 +122,18 @@ def test_chunk_table_of_packed_sequences():
     with pytest.raises(ValueError):
         gdn.chunk_table([0, 10, 5], 64)
 
+
+
+def test_public_header_compiles_on_its_own_as_c_and_cpp(tmp_path):
+    """include/gdnprep.h is the boundary: plain C (no torch, no CUDA headers), usable from C99 and C++."""
+    import shutil
+    import subprocess
+    inc = os.path.join(ROOT, "include")
+    for compiler, std, ext in (("gcc", "-std=c99", "c"), ("g++", "-std=c++17", "cpp")):
+        if shutil.which(compiler) is None:
+            pytest.skip(f"{compiler} not available")
+        src = tmp_path / f"t.{ext}"
+        src.write_text('#include "gdnprep.h"\nint main(void) { return gdn_default_order(64) == 0; }\n')
+        r = subprocess.run([compiler, std, "-Wall", "-Wextra", "-pedantic", "-I", inc, "-c", str(src), "-o", str(tmp_path / "t.o")],
+                           capture_output=True, text=True)
+        assert r.returncode == 0, r.stderr
