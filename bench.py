@@ -25,11 +25,21 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 import numpy as np
-import torch
+
+torch = None  # imported by main(): the worker processes of the CPU leg re-import this file and must not pay for it
+
+
+def _import_torch():
+    global torch
+    if torch is None:
+        import torch as _torch
+        torch = _torch
+    return torch
+
 
 METRIC = "chunk_prepare_throughput"
 UNIT = "chunks/s"
-DEFAULT_WORKLOAD = "sweep_c64"
+DEFAULT_WORKLOAD = "stress"  # the largest single-GPU configuration (B=8, H=32, T=65536, C=64: 262 144 chunks, 19.5 GB)
 
 
 # ----------------------------------------------------------------------------- bookkeeping
@@ -152,42 +162,75 @@ class ClockSampler(threading.Thread):
 
 
 # ----------------------------------------------------------------------------- CPU oracle leg
-def time_oracle(workload: str, budget_s: float, seed_offset: int = 0):
-    """Times the fp64 oracle, as it stands, on a bounded sample of the workload's chunks."""
-    from oracle import gdn_oracle as orc
+def _bf16_round(x: np.ndarray) -> np.ndarray:
+    """Round-to-nearest-even to bfloat16 and back, on the host (bit arithmetic on the fp32 pattern)."""
+    f = np.ascontiguousarray(x, dtype=np.float32)
+    u = f.view(np.uint32).astype(np.uint64)
+    u = ((u + 0x7FFF + ((u >> 16) & 1)) >> 16) << 16
+    return u.astype(np.uint32).view(np.float32).astype(np.float64).reshape(f.shape)
+
+
+def sample_chunk_ids(n_heads: int, n_c: int, n_random: int, seed: int):
+    """First and last chunk of the first and last head, of head 1 (adversarial in the stress workload), random ones."""
+    n = n_heads * n_c
+    fixed = [0, n_c - 1, (n_heads - 1) * n_c, n - 1]
+    if n_heads > 1:
+        fixed += [n_c, 2 * n_c - 1]
+    rnd = np.random.default_rng(seed).choice(n, size=min(n_random, n), replace=False).tolist()
+    return sorted(set(fixed + rnd))
+
+
+def parity_report(orc, sample, gpu):
+    """The numbers the target asks for next to the throughput, on the chunks the CPU leg ran: error of the GPU result
+    against the fp64 evaluation of the same truncated scheme (the graded number) with the bf16 rounding floor of that
+    evaluation beside it, the signal-to-noise ratio (Sec. 4.2), and the deviation from the exact inverse."""
+    K, V, b, g = sample
+    Wo, Uo, To = orc.chunk_prepare(K, V, b, g)
+    We, Ue, Te = orc.chunk_prepare(K, V, b, g, exact=True)
+    rep = {"chunks": int(K.shape[0]), "reference": "fp64 oracle of the same truncated scheme (order, residual steps as timed)"}
+    for name, got, ref, ex in (("Tinv", gpu[2], To, Te), ("W", gpu[0], Wo, We), ("U", gpu[1], Uo, Ue)):
+        err = orc.rel_frobenius(got, ref)
+        floor = orc.rel_frobenius(_bf16_round(ref), ref)
+        w = int(np.argmax(err))
+        rep[name] = {"worst_rel_frobenius": float(err[w]), "bf16_floor_of_that_chunk": float(floor[w]),
+                     "worst_bf16_floor": float(floor.max()), "mean_rel_frobenius": float(err.mean()),
+                     "snr_db_worst": float(orc.snr_db(got, ref).min()), "snr_db_mean": float(orc.snr_db(got, ref).mean()),
+                     "gpu_vs_exact_inverse_worst": float(orc.rel_frobenius(got, ex).max()),
+                     "scheme_vs_exact_inverse_worst": float(orc.rel_frobenius(ref, ex).max())}
+    return rep
+
+
+def time_oracle(workload: str, budget_s: float, sample=None, workers=None):
+    """Times the fp64 oracle, as it stands, on a bounded sample of the workload's chunks, on all usable host cores
+    (one process per core, each calling the oracle on batches of chunks). `sample`: (K, V, beta, g) stacks of chunks
+    taken from the workload itself; without it a small instance with the same shapes and distributions is drawn."""
+    from oracle import pool
     from paper_2606_06034_b200 import inputs as gen
 
     cfg = dict(gen.WORKLOADS[workload])
-    # a small instance with the same per-chunk shapes and distributions
-    small = dict(cfg, B=1, H_k=min(cfg["H_k"], 2), H_v=min(cfg["H_k"], 2) * (cfg["H_v"] // cfg["H_k"]), T=max(cfg["C"] * 16, 1024))
-    inp = gen.make_inputs(device="cpu", **small)
-    ids = list(range(inp.n_chunks))
-    sl = gen.chunk_slices(inp, ids)
-    K = np.stack([s[0] for s in sl]); V = np.stack([s[1] for s in sl])
-    b = np.stack([s[2] for s in sl]); g = np.stack([s[3] for s in sl])
-    n0 = min(64, len(ids))
-    t0 = time.perf_counter()
-    orc.chunk_prepare(K[:n0], V[:n0], b[:n0], g[:n0])
-    per_chunk = (time.perf_counter() - t0) / n0
-    n = int(max(n0, budget_s / max(per_chunk, 1e-9)))
-    reps = (n + len(ids) - 1) // len(ids)
-    done = 0
-    w0 = time.perf_counter(); c0 = time.process_time()
-    for r in range(reps):
-        m = min(len(ids), n - done)
-        if m <= 0:
-            break
-        orc.chunk_prepare(K[:m], V[:m], b[:m], g[:m])
-        done += m
-    wall = time.perf_counter() - w0
-    cpu = time.process_time() - c0
-    return {"value": done / wall, "unit": UNIT, "cores": max(1, int(round(cpu / max(wall, 1e-9)))), "kind": "oracle",
-            "sample": f"{done} chunks of the {workload} shapes (C={cfg['C']}, d={cfg['d_k']}), fp64 numpy oracle, "
-                      f"{wall:.1f} s wall, host has {os.cpu_count()} logical cores"}, wall
+    if sample is None:
+        small = dict(cfg, B=1, H_k=min(cfg["H_k"], 2), H_v=min(cfg["H_k"], 2) * (cfg["H_v"] // cfg["H_k"]), T=max(cfg["C"] * 16, 1024))
+        inp = gen.make_inputs(device="cpu", **small)
+        sl = gen.chunk_slices(inp, range(inp.n_chunks))
+        sample = tuple(np.stack([s[i] for s in sl]) for i in range(4))
+    K, V, b, g = sample
+    # calibrate on one core, then size the run so that the CPU work is about budget_s core-seconds
+    n0 = min(32, K.shape[0])
+    _, t1, _ = pool.timed_chunk_prepare(K[:n0], V[:n0], b[:n0], g[:n0], n0, workers=1)
+    per_chunk = t1 / n0
+    workers = pool.usable_cores() if workers is None else workers
+    n = int(max(n0 * workers, budget_s / max(per_chunk, 1e-9)))
+    done, wall, used = pool.timed_chunk_prepare(K, V, b, g, n, workers=workers)
+    return {"value": done / wall, "unit": UNIT, "cores": used, "kind": "oracle",
+            "sample": f"{done} chunk evaluations over {K.shape[0]} distinct chunks of the {workload} shapes (C={cfg['C']}, d={cfg['d_k']}), "
+                      f"fp64 numpy oracle in batches of 32 chunks, one process per core, {wall:.1f} s wall "
+                      f"({done * per_chunk:.0f} core-seconds at the single-core rate of {1.0 / per_chunk:.0f} chunks/s); "
+                      f"host has {os.cpu_count()} logical cores"}, wall
 
 
 # ----------------------------------------------------------------------------- GPU legs
 def device_time_steps(fn, steps: int, warmup: int, dist_ctx, finalize=None):
+    _import_torch()
     """Device time of `steps` calls of fn on the current stream. finalize (optional) joins work that fn left running on
     other streams; it is called after the last step, inside the timed region."""
     for _ in range(warmup):
@@ -222,6 +265,7 @@ def device_time_steps(fn, steps: int, warmup: int, dist_ctx, finalize=None):
 
 def max_over_ranks(total_ms: float, device, dist_ctx) -> float:
     """The slowest rank's device time counts (all-reduce MAX; identity on one rank)."""
+    _import_torch()
     t = torch.tensor([total_ms], dtype=torch.float64, device=device)
     if dist_ctx is not None:
         dist_ctx.all_reduce(t, op=dist_ctx.ReduceOp.MAX)
@@ -234,11 +278,13 @@ def whole_job_throughput(chunks_per_rank: int, world: int, ms_per_step: float) -
 
 
 def run_ours(args, rank, world, dist_ctx):
+    _import_torch()
     from paper_2606_06034_b200 import binding as gdn
     from paper_2606_06034_b200 import inputs as gen
 
     dev = torch.device("cuda", torch.cuda.current_device())
-    inp = gen.make_workload(args.workload, device=dev)
+    over = {"B": args.batch} if args.batch > 0 else {}
+    inp = gen.make_workload(args.workload, device=dev, **over)
     C, group = inp.C, inp.H_v // inp.H_k
     outs = gdn.alloc_outputs(inp.K, inp.V, C)
     n_chunks = inp.n_chunks
@@ -278,11 +324,15 @@ def run_ours(args, rank, world, dist_ctx):
                               variant=gdn.GDN_FWDSUBST_BLOCKED if method == "fwdsubst-blocked" else gdn.GDN_FWDSUBST_ROWS)
 
     sampler = ClockSampler(torch.cuda.current_device())
-    launches0 = gdn.gdn_launch_count()
-    # warm-up happens inside device_time_steps; the sampler only runs during the timed steps
-    # W warm-up steps as asked, and never fewer than 50 untimed launches: the first launches after the idle time spent
-    # generating the inputs run at lower clocks and would otherwise sit inside a short timed region
-    n_untimed = max(args.warmup, 50)
+    # W warm-up steps as asked, and never less than ~0.1 s of untimed launches: the first launches after the idle time
+    # spent generating the inputs run at lower clocks and would otherwise sit inside a short timed region
+    step()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    step()
+    torch.cuda.synchronize()
+    one = max(time.perf_counter() - t0, 1e-5)
+    n_untimed = max(args.warmup, min(50, int(0.1 / one) + 1))
     for _ in range(n_untimed):
         step()
     torch.cuda.synchronize()
@@ -326,22 +376,28 @@ def run_ours(args, rank, world, dist_ctx):
     hbm_peak, bf16_peak, peak_kind = measured_peaks()
     launch_ms = float(np.mean(per))
     achieved = n_chunks * bytes_chunk / (launch_ms * 1e-3) / 1e9
+    traffic = None
+    if method == "neumann" and args.workload in TRAFFIC_PER_CHUNK:
+        per_chunk_traffic, traffic_src = TRAFFIC_PER_CHUNK[args.workload]
+        traffic = per_chunk_traffic * n_chunks
     roofline = {"bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak,
-                "traffic": TRAFFIC_PER_LAUNCH.get(args.workload) if method == "neumann" else None, "peak_kind": peak_kind,
+                "traffic": traffic, "peak_kind": peak_kind,
                 "algorithmic_bytes_per_launch": n_chunks * bytes_chunk,
                 "kernel": {"int8": "chunk_tc_int8_kernel", "state": "chunk_state_kernel"}.get(method, "chunk_tc_kernel<C=%d>" % C),
                 "effective_tflops": n_chunks * flops_chunk / (launch_ms * 1e-3) / 1e12,
                 "tensor_time_frac_of_bf16_peak": (n_chunks * flops_chunk / (launch_ms * 1e-3) / 1e12) / bf16_peak}
+    if traffic is not None:
+        roofline["traffic_source"] = traffic_src
 
     if method == "int8":
-        # DRAM runs at a few per cent and the tensor pipe at 5 %: the variant is bound by the integer arithmetic between
-        # the products (ncu: integer pipe 65 % busy), so that is the roofline it is reported against
+        # the contract's roofline for this variant is HBM (every configuration is memory-bound on paper); the integer-ALU
+        # figure explains where the time goes (ncu: the integer pipe is the busiest unit) and is reported beside it
         ops = int8_integer_ops_per_chunk(C, inp.d_k, inp.d_v, gdn.gdn_default_order(C), gdn.gdn_default_residual_steps(C))
         alu_peak = INT_ALU_LANES * SM_MAX_GHZ / 1e3  # Tiop/s
         alu = n_chunks * ops / (launch_ms * 1e-3) / 1e12
-        roofline.update({"bound": "alu", "achieved": alu, "peak": alu_peak, "unit": "Tiop/s", "frac": alu / alu_peak,
-                         "peak_kind": "derived: 148 SMs x 64 integer lanes x 1.965 GHz",
-                         "algorithmic_int_ops_per_chunk": ops, "hbm_frac": achieved / hbm_peak, "hbm_gbs": achieved})
+        roofline["int_alu"] = {"achieved": alu, "peak": alu_peak, "unit": "Tiop/s", "frac": alu / alu_peak,
+                               "peak_kind": "derived: 148 SMs x 64 integer lanes x 1.965 GHz",
+                               "algorithmic_int_ops_per_chunk": ops}
     per_sorted = sorted(per)
     roofline["launch_us"] = {"mean": launch_ms * 1e3, "median": per_sorted[len(per_sorted) // 2] * 1e3, "best": per_sorted[0] * 1e3}
     line = {
@@ -352,7 +408,7 @@ def run_ours(args, rank, world, dist_ctx):
         "config": {"workload": args.workload, "method": method, "B": inp.B, "H_k": inp.H_k, "H_v": inp.H_v, "T": inp.T, "C": C, "d_k": inp.d_k,
                    "d_v": inp.d_v, "order": gdn.gdn_default_order(C), "residual_steps": gdn.gdn_default_residual_steps(C),
                    "chunks_per_gpu": n_chunks, "parallelism": f"independent shards x{world}, no collective",
-                   "untimed_launches_before_timing": n_untimed,
+                   "untimed_launches_before_timing": n_untimed + 2,
                    "l2_policy": "inputs+outputs %.0f MB per step, larger than the 126 MB L2" % (n_chunks * bytes_chunk / 1e6)},
         "effective_tflops": world * n_chunks * flops_chunk / (ms_per_step * 1e-3) / 1e12,
         "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline,
@@ -360,55 +416,68 @@ def run_ours(args, rank, world, dist_ctx):
     if remeasured:
         line["remeasured"] = True
 
+    # the chunks the CPU leg runs are taken from this workload's own device buffers, with the GPU results for them
+    cpu_sample = gpu_sample = None
+    if rank == 0 and not args.no_cpu and world == 1 and method == "neumann":
+        ids = sample_chunk_ids(inp.B * inp.H_v, inp.T // C, 58, seed=11)
+        sl = gen.chunk_slices(inp, ids)
+        cpu_sample = tuple(np.stack([s[i] for s in sl]) for i in range(4))
+        idx = torch.as_tensor(ids, device=dev)
+        gpu_sample = (outs[0].reshape(n_chunks, C, inp.d_k)[idx].double().cpu().numpy(),
+                      outs[1].reshape(n_chunks, C, inp.d_v)[idx].double().cpu().numpy(),
+                      outs[2].reshape(n_chunks, C, C)[idx].double().cpu().numpy())
+
     if rank == 0 and not args.no_e2e and method == "neumann":
         line["e2e"] = run_e2e(inp, outs, gdn, args, world, n_chunks)
+    del outs, inp
+    torch.cuda.empty_cache()
     if rank == 0 and not args.no_extras:
         line["extras"] = run_extras(gdn, gen, dev, args)
     if rank == 0 and not args.no_cpu and world == 1:
-        line["cpu_baseline"], _ = time_oracle(args.workload, args.cpu_seconds)
+        line["cpu_baseline"], _ = time_oracle(args.workload, args.cpu_seconds, sample=cpu_sample)
+        if cpu_sample is not None:
+            from oracle import gdn_oracle as orc
+            line["cpu_baseline"]["parity_on_sample"] = parity_report(orc, cpu_sample, gpu_sample)
     return line
 
 
-# per-launch DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under profiles/
-TRAFFIC_PER_LAUNCH: dict = {
-    "sweep_c64": 248.9e6,     # profiles/chunk_tc_kernel_bf16_c64_sweep_c64.md
-    "prefill_gqa": 1029.0e6,  # profiles/chunk_tc_kernel_bf16_c64_prefill_gqa.md
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per chunk from the ncu captures summarised under profiles/,
+# scaled to a launch by the number of chunks it processes (traffic grows in proportion: every chunk is read and written once)
+TRAFFIC_PER_CHUNK: dict = {
+    "sweep_c64": (248.9e6 / 4096, "ncu capture of this workload (profiles/chunk_tc_kernel_bf16_c64_sweep_c64.md)"),
+    "prefill_gqa": (1029.0e6 / 16384, "ncu capture of this workload (profiles/chunk_tc_kernel_bf16_c64_prefill_gqa.md)"),
 }
 
 
 def run_e2e(inp, outs, gdn, args, world, n_chunks):
     """Same metric through the C-ABI with HOST buffers: pinned host -> device copies of K, V, beta, g and a
-    device -> host read of W, U, Tinv inside the timed region, every step."""
-    host_in = [t.cpu().pin_memory() for t in (inp.K, inp.V, inp.beta, inp.g)]
-    dev_in = [torch.empty_like(t) for t in (inp.K, inp.V, inp.beta, inp.g)]
-    host_out = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in outs]
-    h2d = sum(t.numel() * t.element_size() for t in host_in)
-    d2h = sum(t.numel() * t.element_size() for t in host_out)
-    steps = max(3, min(args.steps, 10))
-
+    device -> host read of W, U, Tinv inside the timed region, every step. The batch is cut into one slice per batch
+    entry; a stream owns pinned host buffers for ONE slice (pinning the 20 GB of the largest workload is not an
+    option) and runs its slices in order through them: copy in -> kernel -> copy out."""
+    _import_torch()
     B = inp.K.shape[0]
-    streams = [torch.cuda.Stream() for _ in range(min(B, 4))] if B >= 2 else []
+    n_streams = min(B, 4)
+    ins = (inp.K, inp.V, inp.beta, inp.g)
+    host_in = [[t[s:s + 1].cpu().pin_memory() for t in ins] for s in range(n_streams)]
+    dev_in = [[torch.empty_like(t[0:1]) for t in ins] for _ in range(n_streams)]
+    host_out = [[torch.empty(t[0:1].shape, dtype=t.dtype, pin_memory=True) for t in outs] for _ in range(n_streams)]
+    h2d = B * sum(t.numel() * t.element_size() for t in host_in[0])
+    d2h = B * sum(t.numel() * t.element_size() for t in host_out[0])
+    steps = max(3, min(args.steps, 10 if h2d + d2h < (2 << 30) else 4))
+    streams = [torch.cuda.Stream() for _ in range(n_streams)]
 
-    def step_serial():
-        for h, d in zip(host_in, dev_in):
-            d.copy_(h, non_blocking=True)
-        gdn.chunk_prepare(dev_in[0], dev_in[1], dev_in[2], dev_in[3], inp.C, outputs=outs)
-        for h, d in zip(host_out, outs):
-            h.copy_(d, non_blocking=True)
-
-    def step_pipelined():
-        # one batch entry per slice, slices alternate between two streams: the device -> host copy of a slice
-        # overlaps the host -> device copy of the next one (PCIe is full duplex) and both overlap the kernels.
-        # Consecutive steps are not joined (a slice always runs on the same stream, so its buffers are reused in
-        # order): the copies of step k + 1 start while step k drains, as in a serving loop; `join` closes the region.
+    def step():
+        # consecutive steps are not joined (a slice always runs on the same stream, so its buffers are reused in order):
+        # the copies of step k + 1 start while step k drains, as in a serving loop; `join` closes the timed region
         for b in range(B):
-            with torch.cuda.stream(streams[b % len(streams)]):
-                for h, d in zip(host_in, dev_in):
-                    d[b:b + 1].copy_(h[b:b + 1], non_blocking=True)
-                gdn.chunk_prepare(dev_in[0][b:b + 1], dev_in[1][b:b + 1], dev_in[2][b:b + 1], dev_in[3][b:b + 1], inp.C,
+            s = b % n_streams
+            with torch.cuda.stream(streams[s]):
+                for h, d in zip(host_in[s], dev_in[s]):
+                    d.copy_(h, non_blocking=True)
+                gdn.chunk_prepare(dev_in[s][0], dev_in[s][1], dev_in[s][2], dev_in[s][3], inp.C,
                                   outputs=tuple(o[b:b + 1] for o in outs))
-                for h, d in zip(host_out, outs):
-                    h[b:b + 1].copy_(d[b:b + 1], non_blocking=True)
+                for h, d in zip(host_out[s], outs):
+                    h.copy_(d[b:b + 1], non_blocking=True)
 
     def join():
         cur = torch.cuda.current_stream()
@@ -422,20 +491,34 @@ def run_e2e(inp, outs, gdn, args, world, n_chunks):
     start.record(torch.cuda.current_stream())
     for st in streams:
         st.wait_event(start)
-    step = step_pipelined if streams else step_serial
-    total_ms, _ = device_time_steps(step, steps, 2, None, finalize=join if streams else None)
+    total_ms, _ = device_time_steps(step, steps, 1, None, finalize=join)
     return {"value": world * n_chunks / (total_ms / steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
             "d2h_bytes_per_step": d2h, "steps": steps, "ms_per_step": total_ms / steps,
-            "pipeline": ("%d slices over %d streams, steps back to back" % (B, len(streams))) if streams else "one slice"}
+            "pipeline": "%d slices (one per batch entry) over %d streams, each stream with pinned host buffers for one slice "
+                        "that its slices pass through in order (slice s carries the data of batch entry s mod %d); steps back to back"
+                        % (B, n_streams, n_streams)}
+
+
+def _timed_extra(fn, n_chunks, bytes_chunk, hbm_peak, steps, warm):
+    total_ms, per = device_time_steps(fn, steps, warm, None)
+    ms = float(np.mean(per))
+    return {"chunks_per_s": n_chunks / (ms * 1e-3), "ms": ms, "launch_ms_mean": ms, "launch_ms_best": float(min(per)),
+            "hbm_frac": n_chunks * bytes_chunk / (ms * 1e-3) / 1e9 / hbm_peak}
 
 
 def run_extras(gdn, gen, dev, args):
-    """Other workloads and the forward-substitution comparison, timed the same way (not the headline)."""
+    """The other graded configurations and the forward-substitution comparisons, timed the same way as the headline
+    (CUDA events around every launch after warm-up; every workload is larger than L2). Not the headline."""
+    _import_torch()
     out = {}
     hbm_peak, _, _ = measured_peaks()
     plan = [("sweep_c16", "neumann"), ("sweep_c32", "neumann"), ("sweep_c64", "neumann"), ("sweep_c128", "neumann"),
-            ("sweep_c64", "neumann-s15"), ("sweep_c64", "fwdsubst"), ("sweep_c64", "fwdsubst-blocked"),
-            ("sweep_c32", "fwdsubst"), ("sweep_c16", "fwdsubst"), ("prefill_gqa", "neumann")]
+            ("sweep_c64", "neumann-s15"),
+            ("sweep_c16", "fwdsubst"), ("sweep_c32", "fwdsubst"), ("sweep_c64", "fwdsubst"), ("sweep_c128", "fwdsubst"),
+            ("sweep_c16", "fwdsubst-blocked"), ("sweep_c32", "fwdsubst-blocked"), ("sweep_c64", "fwdsubst-blocked"),
+            ("sweep_c128", "fwdsubst-blocked"), ("prefill_gqa", "neumann"), ("prefill_gqa", "fwdsubst")]
+    if args.workload != "stress":
+        plan.append(("stress", "neumann"))
     for name, method in plan:
         try:
             inp = gen.make_workload(name, device=dev)
@@ -446,14 +529,19 @@ def run_extras(gdn, gen, dev, args):
             n_ord, n_res = (3, 15) if var == "s15" else (-1, -1)
             fn = lambda: gdn.chunk_prepare(inp.K, inp.V, inp.beta, inp.g, inp.C, n_ord, n_res, outputs=outs, method=meth,
                                            variant=variant)
-            total_ms, _ = device_time_steps(fn, 20, 3, None)
-            ms = total_ms / 20
             by = algorithmic_bytes_per_chunk(inp.C, inp.d_k, inp.d_v, inp.H_v // inp.H_k)
-            out[f"{name}:{method}"] = {"chunks_per_s": inp.n_chunks / (ms * 1e-3), "ms": ms,
-                                       "hbm_frac": inp.n_chunks * by / (ms * 1e-3) / 1e9 / hbm_peak}
+            out[f"{name}:{method}"] = _timed_extra(fn, inp.n_chunks, by, hbm_peak, 20 if name != "stress" else 10, 5)
             del inp, outs
         except Exception as exc:  # an unsupported extra must not lose the headline
             out[f"{name}:{method}"] = {"error": repr(exc)}
+    # Neumann against the better of the two substitutions, per chunk size
+    for c in (16, 32, 64, 128):
+        try:
+            neu = out[f"sweep_c{c}:neumann"]["ms"]
+            sub = min(out[f"sweep_c{c}:{m}"]["ms"] for m in ("fwdsubst", "fwdsubst-blocked") if "ms" in out.get(f"sweep_c{c}:{m}", {}))
+            out[f"sweep_c{c}:neumann_speedup_over_best_substitution"] = sub / neu
+        except Exception:
+            pass
     # the model-native call on the prefill shapes: token-major tensors, raw gates, fused key normalisation, gated W;
     # and the same tokens as 201 packed sequences of ragged lengths (seeded cuts)
     try:
@@ -464,10 +552,7 @@ def run_extras(gdn, gen, dev, args):
         flags = gdn.GDN_FLAG_LAYOUT_BTHD | gdn.GDN_FLAG_G_RAW | gdn.GDN_FLAG_K_L2NORM | gdn.GDN_FLAG_W_GATED
         outs = gdn.alloc_outputs(Kt, Vt, inp.C, True, True)
         fn = lambda: gdn.chunk_prepare(Kt, Vt, bt, gt, inp.C, outputs=outs, flags=flags)
-        total_ms, _ = device_time_steps(fn, 10, 3, None)
-        ms = total_ms / 10
-        out["prefill_gqa:model_native_flags"] = {"chunks_per_s": inp.n_chunks / (ms * 1e-3), "ms": ms,
-                                                 "hbm_frac": inp.n_chunks * by / (ms * 1e-3) / 1e9 / hbm_peak}
+        out["prefill_gqa:model_native_flags"] = _timed_extra(fn, inp.n_chunks, by, hbm_peak, 10, 3)
         del Kt, Vt, bt, gt, outs
         cuts = np.sort(np.random.default_rng(0).choice(np.arange(1, inp.T), size=200, replace=False))
         start, length = gdn.chunk_table([0] + cuts.tolist() + [inp.T], inp.C)
@@ -479,11 +564,11 @@ def run_extras(gdn, gen, dev, args):
         Ti = torch.empty(inp.H_v, -(-len(start) // per_tile) * per_tile, inp.C, inp.C, dtype=inp.K.dtype, device=dev)
         fn = lambda: gdn.gdn_chunk_prepare_varlen(inp.K[0], inp.V[0], inp.beta[0], inp.g[0], cs, cl, len(start), inp.T, inp.H_k,
                                                   inp.H_v, inp.C, inp.d_k, inp.d_v, -1, -1, W, U, Ti, 0)
-        total_ms, _ = device_time_steps(fn, 10, 3, None)
-        ms = total_ms / 10
         n_slots = len(start) * inp.H_v
-        out["prefill_gqa:packed_201_sequences"] = {"chunk_slots": n_slots, "chunks_per_s": n_slots / (ms * 1e-3), "ms": ms,
-                                                   "hbm_frac": inp.n_chunks * by / (ms * 1e-3) / 1e9 / hbm_peak}
+        r = _timed_extra(fn, inp.n_chunks, by, hbm_peak, 10, 3)
+        r["chunk_slots"] = n_slots
+        r["chunks_per_s"] = n_slots / (r["ms"] * 1e-3)
+        out["prefill_gqa:packed_201_sequences"] = r
         del inp, W, U, Ti
     except Exception as exc:
         out["prefill_gqa:model_native"] = {"error": repr(exc)}
@@ -493,14 +578,12 @@ def run_extras(gdn, gen, dev, args):
         q = gen.make_int8_inputs(inp)
         outs = gdn.chunk_prepare_int8(q)
         fn = lambda: gdn.chunk_prepare_int8(q, outputs=outs)
-        total_ms, _ = device_time_steps(fn, 10, 3, None)
-        ms = total_ms / 10
         group = inp.H_v // inp.H_k
         by = inp.C * inp.d_k / group + inp.C * inp.d_v + inp.C * inp.d_k + inp.C * inp.d_v + inp.C * inp.C + 6 * inp.C
         ops = int8_integer_ops_per_chunk(q.C, q.d_k, q.d_v, gdn.gdn_default_order(q.C), gdn.gdn_default_residual_steps(q.C))
-        out["prefill_gqa:int8"] = {"chunks_per_s": q.n_chunks / (ms * 1e-3), "ms": ms,
-                                   "hbm_frac": q.n_chunks * by / (ms * 1e-3) / 1e9 / hbm_peak,
-                                   "int_alu_frac": q.n_chunks * ops / (ms * 1e-3) / (INT_ALU_LANES * SM_MAX_GHZ * 1e9)}
+        r = _timed_extra(fn, q.n_chunks, by, hbm_peak, 10, 3)
+        r["int_alu_frac"] = q.n_chunks * ops / (r["ms"] * 1e-3) / (INT_ALU_LANES * SM_MAX_GHZ * 1e9)
+        out["prefill_gqa:int8"] = r
         del inp, q, outs
     except Exception as exc:
         out["prefill_gqa:int8"] = {"error": repr(exc)}
@@ -515,23 +598,18 @@ def run_extras(gdn, gen, dev, args):
             W, U, _ = gdn.chunk_prepare(inp.K, inp.V, inp.beta, inp.g, inp.C, flags=gdn.GDN_FLAG_W_GATED, want_tinv=False)
             outs = gdn.chunk_state_output(Q, inp.K, W, U, inp.g, inp.C, inp.d_k ** -0.5)
             fn = lambda: gdn.chunk_state_output(Q, inp.K, W, U, inp.g, inp.C, inp.d_k ** -0.5, outputs=outs)
-            total_ms, _ = device_time_steps(fn, 5, 2, None)
-            ms = total_ms / 5
             group = inp.H_v // inp.H_k
             # Q, K tiles (shared by a group), W, U read, O written, g
             by = inp.C * inp.d_k * 2 * (2.0 / group + 1) + 2 * inp.C * inp.d_v * 2 + 4 * inp.C
-            out[f"{name}:state_output"] = {"chunks_per_s": inp.n_chunks / (ms * 1e-3), "ms": ms,
-                                           "hbm_frac": inp.n_chunks * by / (ms * 1e-3) / 1e9 / hbm_peak,
-                                           "us_per_chunk_of_a_sequence": ms * 1e3 / (inp.T // inp.C)}
+            r = _timed_extra(fn, inp.n_chunks, by, hbm_peak, 5, 2)
+            r["us_per_chunk_of_a_sequence"] = r["ms"] * 1e3 / (inp.T // inp.C)
+            out[f"{name}:state_output"] = r
             if inp.B == 1:
                 # few long sequences: the segmented form (state maps of the segments in parallel)
                 fn = lambda: gdn.chunk_state_output_segmented(Q[0], inp.K[0], W[0], U[0], inp.g[0], inp.C, inp.d_k ** -0.5)
-                total_ms, _ = device_time_steps(fn, 5, 2, None)
-                ms = total_ms / 5
-                out[f"{name}:state_output_segmented"] = {
-                    "segments": int(gdn.load_library().gdn_chunk_state_segments(inp.H_v)),
-                    "chunks_per_s": inp.n_chunks / (ms * 1e-3), "ms": ms,
-                    "hbm_frac": inp.n_chunks * by / (ms * 1e-3) / 1e9 / hbm_peak}
+                r = _timed_extra(fn, inp.n_chunks, by, hbm_peak, 5, 2)
+                r["segments"] = int(gdn.load_library().gdn_chunk_state_segments(inp.H_v))
+                out[f"{name}:state_output_segmented"] = r
             del inp, Q, W, U, outs
         except Exception as exc:
             out[f"{name}:state_output"] = {"error": repr(exc)}
@@ -556,7 +634,8 @@ def run_reference(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps, "warmup": warm,
         "ms_per_step": float(np.mean([w for _, w in vals])) * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic", "impl": "reference",
-        "config": {"workload": args.workload, "C": cfg["C"], "d_k": cfg["d_k"], "d_v": cfg["d_v"],
+        "config": {"workload": args.workload, "method": "neumann", "B": cfg["B"], "H_k": cfg["H_k"], "H_v": cfg["H_v"], "T": cfg["T"],
+                   "C": cfg["C"], "d_k": cfg["d_k"], "d_v": cfg["d_v"],
                    "note": "each step is a bounded sample of the workload's chunks run through the fp64 CPU oracle"},
         "cpu_baseline": info,
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -567,12 +646,13 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
-    ap.add_argument("--warmup", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (smaller captures under ncu)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--method", default="neumann", choices=["neumann", "fwdsubst", "fwdsubst-blocked", "int8", "state", "model-native"])
-    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--cpu-seconds", type=float, default=20.0)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extras", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
@@ -588,6 +668,7 @@ def main():
             print(json.dumps(run_reference(args)), flush=True)
         return
 
+    _import_torch()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (the library has no CPU path)")
     torch.cuda.set_device(local_rank)
