@@ -59,7 +59,9 @@ typedef enum {
     GDN_ERR_ALIGN = -4,       /* a pointer is not 16-byte aligned */
     GDN_ERR_LAUNCH = -5,      /* the CUDA runtime refused the launch or a set-up call */
     GDN_ERR_TIMEOUT = -6,     /* a bounded wait inside a kernel ran out (reported by gdn_device_status) */
-    GDN_ERR_ARCH = -7         /* the current device is not sm_100 */
+    GDN_ERR_ARCH = -7,        /* the current device is not sm_100 */
+    GDN_ERR_SCRATCH = -8      /* gdn_chunk_state_output_segmented_noalloc: the problem needs more scratch memory than the
+                                 library's built-in array holds */
 } gdn_status;
 
 enum { GDN_DTYPE_FP32 = 0, GDN_DTYPE_BF16 = 1 };
@@ -229,6 +231,31 @@ int gdn_chunk_state_output_segmented(const void* Q, const void* K, const void* W
                                      int H_k, int H_v, int T, int C, int d_k, int d_v, float scale,
                                      const float* S_in, void* O_out, float* S_out, int segments,
                                      void* workspace, size_t workspace_bytes, unsigned flags, gdn_stream_t stream);
+
+/*
+ * gdn_chunk_state_output_segmented without a workspace argument (the paper has no counterpart: this is a
+ * convenience of the library). It is meant for callers that must not, or cannot, allocate device memory around
+ * the call: code running inside an inference engine that handed out all of the GPU's memory at start-up, a plug-in
+ * with no allocator of its own, a real-time loop in which cudaMalloc's implicit synchronisation is not acceptable.
+ * The scratch memory the segmented form needs (the segments' state maps and initial states) is a fixed array of
+ * device memory built into the library, 8 MB + 4 KB, which every GPU that loads the library holds until the
+ * process exits. The call allocates and frees nothing, neither directly nor through another library.
+ *   Arguments, layouts, flags and results: exactly those of gdn_chunk_state_output_segmented (the same kernels run).
+ *   Limit: H_v * (6 * segments - 6) <= 128 (the number of 128 x 128 fp32 state blocks the array holds; e.g. 8 value
+ *   heads in 3 segments, 4 in 6, 16 in 2), where segments is first clamped to the number of chunks. A larger problem
+ *   returns GDN_ERR_SCRATCH and launches nothing: use the variant with a workspace there. segments = 1 needs no
+ *   scratch and is always accepted.
+ *   First call on a device: the library looks up the device address of its array (with that device current, once
+ *   per device). Make that first call outside any stream capture.
+ *   Sharing: all calls on a device use the same array, and the array keeps what the last call left in it. Every
+ *   call writes all the scratch it later reads, so nothing has to be cleared between calls, but two calls that
+ *   overlap on the GPU (different streams, or different host threads) race on it: keep calls of this entry point
+ *   on one stream, or order them with events.
+ */
+int gdn_chunk_state_output_segmented_noalloc(const void* Q, const void* K, const void* W_gated, const void* U,
+                                             const float* g, int H_k, int H_v, int T, int C, int d_k, int d_v,
+                                             float scale, const float* S_in, void* O_out, float* S_out, int segments,
+                                             unsigned flags, gdn_stream_t stream);
 
 /* Checksum of the 256-entry gate-decay table round(2^15 * 2^(-f/256)) the INT8 kernel uses
  * (sum_f: s = (31 s + table[f] + f) mod 1000000007), so that a CPU evaluation can confirm it holds the same table. */

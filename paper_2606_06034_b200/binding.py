@@ -23,6 +23,7 @@ GDN_ERR_ALIGN = -4
 GDN_ERR_LAUNCH = -5
 GDN_ERR_TIMEOUT = -6
 GDN_ERR_ARCH = -7
+GDN_ERR_SCRATCH = -8
 GDN_DTYPE_FP32 = 0
 GDN_DTYPE_BF16 = 1
 GDN_FLAG_G_RAW = 1
@@ -37,6 +38,7 @@ EXPORTS = (
     "gdn_chunk_prepare", "gdn_chunk_prepare_gqa", "gdn_chunk_prepare_ex", "gdn_chunk_prepare_varlen",
     "gdn_chunk_prepare_fwdsubst",
     "gdn_chunk_prepare_int8", "gdn_chunk_state_output", "gdn_chunk_state_output_varlen", "gdn_chunk_state_output_segmented",
+    "gdn_chunk_state_output_segmented_noalloc",
     "gdn_chunk_state_segments", "gdn_chunk_state_segmented_workspace", "gdn_selftest_bounded_wait",
     "gdn_int8_lut_checksum",
     "gdn_device_status", "gdn_default_order", "gdn_default_residual_steps",
@@ -89,6 +91,9 @@ def load_library() -> ctypes.CDLL:
     lib.gdn_chunk_state_output_segmented.argtypes = [vp, vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ctypes.c_float, vp, vp, vp, ip,
                                                      vp, ctypes.c_size_t, ctypes.c_uint, vp]
     lib.gdn_chunk_state_output_segmented.restype = ip
+    lib.gdn_chunk_state_output_segmented_noalloc.argtypes = [vp, vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ctypes.c_float, vp, vp, vp,
+                                                             ip, ctypes.c_uint, vp]
+    lib.gdn_chunk_state_output_segmented_noalloc.restype = ip
     lib.gdn_selftest_bounded_wait.argtypes = [vp]
     lib.gdn_selftest_bounded_wait.restype = ip
     lib.gdn_int8_lut_checksum.argtypes = []
@@ -357,6 +362,22 @@ def chunk_state_output_segmented(Q, K, W_gated, U, g, C, scale=1.0, S_in=None, *
     if rc != GDN_OK:
         raise GdnError(rc, "gdn_chunk_state_output_segmented")
     return O, S_out
+
+
+def gdn_chunk_state_output_segmented_noalloc(Q, K, W_gated, U, g, H_k, H_v, T, C, d_k, d_v, scale, S_in, O_out, S_out, segments,
+                                             flags=0, *, check=True):
+    """Raw call of the segmented state passing on the library's built-in scratch array: for callers that cannot
+    allocate device memory around the call. The caller passes every input and output tensor; this wrapper and the
+    entry point allocate nothing. Returns the status (GDN_ERR_SCRATCH when H_v * (6 * segments - 6) > 128)."""
+    for t in (Q, K, W_gated, U, g, S_in, O_out, S_out):
+        if t is not None and (not t.is_cuda or not t.is_contiguous()):
+            raise ValueError("all tensors must be contiguous CUDA tensors (there is no CPU path)")
+    rc = load_library().gdn_chunk_state_output_segmented_noalloc(_ptr(Q), _ptr(K), _ptr(W_gated), _ptr(U), _ptr(g), H_k, H_v, T, C,
+                                                                 d_k, d_v, ctypes.c_float(scale), _ptr(S_in), _ptr(O_out),
+                                                                 _ptr(S_out), segments, flags, _stream())
+    if check and rc != GDN_OK:
+        raise GdnError(rc, "gdn_chunk_state_output_segmented_noalloc")
+    return rc
 
 
 def chunk_state_output_varlen(Q, K, W_gated, U, g, cu_seqlens, C, scale=1.0, S_in=None, *, want_state=True, flags=0):

@@ -871,6 +871,35 @@ int launch_chunk_state_segmented(const ProblemS& q, int P, void* workspace, cuda
     return cudaGetLastError() == cudaSuccess ? GDN_OK : GDN_ERR_LAUNCH;
 }
 
+// ---- the segmented call on built-in scratch memory (for callers that cannot allocate device memory)
+// The scratch lives in this file-scope device array: every GPU that loads the library holds it until the process
+// exits. In host code the array's name is only a handle; the device address comes from cudaGetSymbolAddress, once per
+// device, with that device current.
+namespace {
+constexpr size_t kBuiltinStateBlocks = 128;  // state-sized blocks of 128 x 128 fp32 (64 KB each): 8 MB
+constexpr size_t kBuiltinScratchBytes = kBuiltinStateBlocks * kD * kD * sizeof(float) + 4096;
+static __device__ __align__(256) unsigned char g_builtin_scratch[kBuiltinScratchBytes];
+constexpr int kMaxDev = 64;
+void* g_builtin_scratch_addr[kMaxDev] = {nullptr};
+}  // namespace
+
+int launch_chunk_state_segmented_builtin(const ProblemS& q, int P, cudaStream_t stream) {
+    const int n_chunks = q.T / kC;
+    const int p_eff = P > n_chunks ? n_chunks : P;
+    if (p_eff >= 2 && chunk_state_segmented_workspace(q.H_v, p_eff) > kBuiltinScratchBytes) return GDN_ERR_SCRATCH;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) return GDN_ERR_LAUNCH;
+    if (g_builtin_scratch_addr[dev] == nullptr) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_builtin_scratch) != cudaSuccess || ptr == nullptr) {
+            cudaGetLastError();
+            return GDN_ERR_LAUNCH;
+        }
+        g_builtin_scratch_addr[dev] = ptr;
+    }
+    return launch_chunk_state_segmented(q, P, g_builtin_scratch_addr[dev], stream);
+}
+
 #ifdef GDN_TRACE
 extern "C" int gdn_debug_read_trace_state(long long* host_out) {
     return cudaMemcpyFromSymbol(host_out, g_trace_s, sizeof(long long) * 4096) == cudaSuccess ? 0 : -1;

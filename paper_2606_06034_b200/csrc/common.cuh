@@ -85,6 +85,8 @@ int launch_chunk_state(const ProblemS& p, cudaStream_t stream);
 // the segmented form for few long sequences (B = 1): P segments per sequence, workspace of chunk_state_segmented_workspace bytes
 int launch_chunk_state_segmented(const ProblemS& q, int P, void* workspace, cudaStream_t stream);
 size_t chunk_state_segmented_workspace(int H_v, int P);
+// the same on the library's built-in scratch array (GDN_ERR_SCRATCH when the problem needs more than it holds)
+int launch_chunk_state_segmented_builtin(const ProblemS& q, int P, cudaStream_t stream);
 int chunk_state_auto_segments(long long H_v);
 int launch_tc_int8(const ProblemI8& p, cudaStream_t stream);
 void int8_decay_lut(uint16_t* out256);  // table of round(2^15 * 2^(-f/256))

@@ -218,6 +218,22 @@ int gdn_chunk_state_output_segmented(const void* Q, const void* K, const void* W
     return launch_chunk_state_segmented(q, segments, workspace, static_cast<cudaStream_t>(stream));
 }
 
+int gdn_chunk_state_output_segmented_noalloc(const void* Q, const void* K, const void* W_gated, const void* U, const float* g,
+                                             int H_k, int H_v, int T, int C, int d_k, int d_v, float scale, const float* S_in,
+                                             void* O_out, float* S_out, int segments, unsigned flags, gdn_stream_t stream) {
+    if (flags & ~static_cast<unsigned>(GDN_FLAG_G_RAW | GDN_FLAG_LAYOUT_BTHD | GDN_FLAG_K_L2NORM)) return GDN_ERR_INVALID_ARG;
+    if (Q == nullptr || K == nullptr || W_gated == nullptr || U == nullptr || g == nullptr || O_out == nullptr) return GDN_ERR_NULL;
+    if (H_k <= 0 || H_v <= 0 || T < 0 || C < 2 || d_k <= 0 || d_v <= 0 || segments < 1 || segments > 64) return GDN_ERR_INVALID_ARG;
+    if (H_v % H_k != 0 || T % C != 0) return GDN_ERR_INVALID_ARG;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(W_gated) || !aligned16(U) || !aligned16(g) || !aligned16(S_in) ||
+        !aligned16(O_out) || !aligned16(S_out))
+        return GDN_ERR_ALIGN;
+    const int rc = check_arch();
+    if (rc != GDN_OK) return rc;
+    ProblemS q{Q, K, W_gated, U, g, S_in, O_out, S_out, 1, H_k, H_v, T, C, d_k, d_v, scale, flags};
+    return launch_chunk_state_segmented_builtin(q, segments, static_cast<cudaStream_t>(stream));
+}
+
 int gdn_chunk_state_output_varlen(const void* Q, const void* K, const void* W_gated, const void* U, const float* g,
                                   const int32_t* cu_seqlens, int n_seq, int T_total, int H_k, int H_v, int C, int d_k, int d_v,
                                   float scale, const float* S_in, void* O_out, float* S_out, unsigned flags,
@@ -297,6 +313,7 @@ const char* gdn_status_string(int status) {
         case GDN_ERR_LAUNCH: return "CUDA launch or set-up failed";
         case GDN_ERR_TIMEOUT: return "bounded wait inside a kernel ran out";
         case GDN_ERR_ARCH: return "device is not sm_100";
+        case GDN_ERR_SCRATCH: return "problem needs more scratch memory than the library's built-in array holds";
         default: return "unknown status";
     }
 }
