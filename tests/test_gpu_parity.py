@@ -29,6 +29,16 @@ def _bf16_round(x):
     return torch.from_numpy(np.ascontiguousarray(x)).to(torch.bfloat16).double().numpy()
 
 
+def _bound(ref, tol, bf16_out=True):
+    """Per-chunk bar: `tol`, or, for bf16 outputs, the bf16 rounding floor of the fp64 result + 2e-4 where that floor
+    is within 10 % of `tol` or above it (rounding the exact result already costs ~1.7e-3, up to 2.2e-3 on a few
+    chunks of strongly correlated keys)."""
+    if not bf16_out:
+        return np.full(ref.shape[0], tol)
+    floor = orc.rel_frobenius(_bf16_round(ref), ref)
+    return np.where(floor > 0.9 * tol, np.maximum(tol, floor + 2e-4), tol)
+
+
 def _gpu_chunks(W, U, Tinv, inp, chunk_ids=None):
     C = inp.C
     n = inp.n_chunks
@@ -98,6 +108,36 @@ def test_bf16_other_orders_and_steps(C, N, S):
     _check(inp, TOL_BF16, N, S)
 
 
+@pytest.mark.parametrize("C,N,S,beta", [(64, 3, 2, 0.3), (64, 3, 1, 0.3), (64, 5, 3, 0.3), (64, 7, 2, 0.3), (64, 2, 5, 0.7),
+                                        (32, 4, 3, 0.3), (16, 3, 2, 0.3), (16, 2, 1, 0.3)])
+def test_bf16_orders_and_steps_where_every_term_counts(C, N, S, beta):
+    """Inputs on which the result depends visibly on N and on S: strongly correlated keys, no decay, and a write
+    strength low enough for the truncated series to stay bounded. The fp64 evaluations with N - 1 or S - 1 differ from
+    the one asked for by far more than the bar, so a kernel that clamped the order, ran one round too few or got the
+    band recursion wrong beyond distance 3 fails here. fp32 outputs, so that the bar is not hidden by bf16 output
+    rounding. These inputs lie outside the workload regimes (the series has not converged, E and the far part of T
+    are not small, so their single-bf16 tensor-core operands cost up to 1e-3 on Tinv and, through the cancellation in
+    T diag(beta) K on correlated keys, up to 1e-2 on W): the bar per output is a fifth of the distance to the nearest
+    neighbouring (N, S), at most 1e-2, and that distance must be at least 5e-3."""
+    inp = gen.make_inputs(1, 2, 2, 512, C, 128, 128, seed=40 + C + N + S, adversarial_heads="all")
+    inp.beta.fill_(beta)
+    ref = _oracle(inp, N, S)
+    dist = [np.inf, np.inf, np.inf]
+    for n2, s2 in ((N - 1, S), (N, S - 1)):
+        if n2 >= 1 and s2 >= 0:
+            other = _oracle(inp, n2, s2)
+            dist = [min(d, float(orc.rel_frobenius(o, r).min())) for d, o, r in zip(dist, other, ref)]
+    assert min(dist) >= 5e-3, dist
+    K, V, b, g = _to_dev(inp)
+    W, U, Tinv = gdn.chunk_prepare(K, V, b, g, C, N, S, flags=gdn.GDN_FLAG_OUT_FP32)
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+    got = _gpu_chunks(W, U, Tinv, inp)
+    for name, x, r, d in zip(("W", "U", "Tinv"), got, ref, dist):
+        err = orc.rel_frobenius(x, r)
+        bar = min(1e-2, d / 5)
+        assert err.max() <= bar, f"{name} rel-F {err.max():.3e} > {bar:.3e} at chunk {err.argmax()} (nearest neighbour {d:.3e})"
+
+
 @pytest.mark.parametrize("adv", ["none", "all"])
 def test_bf16_full_residual_sum_is_the_exact_inverse(adv):
     """S = 15 at N = 3, C = 64 keeps every term (E^16 = 0): the kernel's four-level doubling form of the sum must
@@ -113,10 +153,24 @@ def test_bf16_chunk_128_block_merge(N, S, adv):
     """C = 128: two 64-blocks by the scheme plus the block formula of App. E for the lower-left block. On strongly
     correlated keys both products of the merge cancel (A21 has entries near 1, A21 T11 is small): the kernel's
     hi + lo operands must keep the result at the bf16 rounding floor there too."""
-    if adv == "odd" and S in (2, 4):
-        pytest.skip("few residual terms on adversarial blocks: the truncated series itself has not converged")
     inp = gen.make_inputs(2, 2, 4, 512, 128, 128, 128, seed=45 + N + S, adversarial_heads=adv)
-    _check(inp, TOL_BF16, N, S)
+    if adv == "odd" and S in (2, 4):
+        # few residual terms on adversarial blocks: the truncated series has not converged and its entries are
+        # orders of magnitude larger than those of the inverse. Parity is still against the same truncated scheme:
+        # the result must be far closer to it than the exact inverse is (the bar of test_bf16_truncation_is_honoured).
+        K, V, beta, g = _to_dev(inp)
+        W, U, Tinv = gdn.chunk_prepare(K, V, beta, g, 128, N, S)
+        assert gdn.gdn_device_status() == gdn.GDN_OK
+        Wg, Ug, Tg = _gpu_chunks(W, U, Tinv, inp)
+        Wo, Uo, To = _oracle(inp, N, S)
+        We, Ue, Te = _oracle(inp, exact=True)
+        for got, ref, ex in ((Tg, To, Te), (Wg, Wo, We), (Ug, Uo, Ue)):
+            gap = orc.rel_frobenius(ref, ex)
+            err = orc.rel_frobenius(got, ref)
+            floor = orc.rel_frobenius(_bf16_round(ref), ref)
+            assert np.all(err <= np.maximum(np.maximum(TOL_BF16, floor + 2e-4), gap / 5))
+    else:
+        _check(inp, TOL_BF16, N, S)
     inp = gen.make_inputs(1, 1, 2, 128, 128, 128, 128, seed=46)
     _check(inp, TOL_BF16, N, S)
 
@@ -256,7 +310,9 @@ def _check_ex(inp, graw, flags, tol, N=-1, S=-1):
                                    w_gated=bool(flags & gdn.GDN_FLAG_W_GATED))
     for name, got, ref in (("Tinv", Tg, To), ("W", Wg, Wo), ("U", Ug, Uo)):
         err = orc.rel_frobenius(got, ref)
-        assert err.max() <= tol, f"{name} rel-F {err.max():.3e} at chunk {err.argmax()} (flags {flags})"
+        bound = _bound(ref, tol, bf16_out=inp.K.dtype == torch.bfloat16 and not (flags & gdn.GDN_FLAG_OUT_FP32))
+        worst = int(np.argmax(err - bound))
+        assert np.all(err <= bound), f"{name} rel-F {err[worst]:.3e} > {bound[worst]:.3e} at chunk {worst} (flags {flags})"
 
 
 @pytest.mark.parametrize("C", [16, 32, 64, 128])
@@ -282,7 +338,7 @@ def test_bf16_gated_w(C, flags):
     inp, graw = _raw_inputs(1, 2, 2, 4 * C, C, seed=300 + C + flags, adv="odd" if C <= 64 else "none")
     if not (flags & gdn.GDN_FLAG_K_L2NORM):
         inp = gen.make_inputs(1, 2, 2, 4 * C, C, 128, 128, seed=300 + C + flags, adversarial_heads="odd" if C <= 64 else "none")
-    _check_ex(inp, graw, flags, 5e-4 if (flags & gdn.GDN_FLAG_OUT_FP32) else TOL_BF16 + 3e-4)
+    _check_ex(inp, graw, flags, 5e-4 if (flags & gdn.GDN_FLAG_OUT_FP32) else TOL_BF16)
 
 
 @pytest.mark.parametrize("C", [16, 64, 128])
@@ -322,7 +378,7 @@ def test_bf16_token_major_layout(C, extra):
         W0, U0, T0 = gdn.chunk_prepare(K, V, beta, g, C, flags=extra)
     else:
         W0, U0, T0 = gdn.chunk_prepare(K, V, beta, g, C)
-    assert torch.equal(tm(W0) if W0.dtype == W.dtype else tm(W0), W)
+    assert torch.equal(tm(W0), W)
     assert torch.equal(tm(U0), U)
     assert torch.equal(T0, Tinv)
     # and against the oracle
@@ -331,10 +387,12 @@ def test_bf16_token_major_layout(C, extra):
     Kc = np.stack([s[0] for s in sl]); Vc = np.stack([s[1] for s in sl]); bc = np.stack([s[2] for s in sl])
     gc = g_src.double().numpy().reshape(inp.n_chunks, C)
     Wo, Uo, To = orc.chunk_prepare(Kc, Vc, bc, gc, None, None, g_raw=bool(extra & 1), k_l2norm=bool(extra & 2))
-    tol = 5e-4 if (extra & gdn.GDN_FLAG_OUT_FP32) else TOL_BF16 + 3e-4
+    fp32_out = bool(extra & gdn.GDN_FLAG_OUT_FP32)
     for name, got, ref in (("Tinv", Tg, To), ("W", Wg, Wo), ("U", Ug, Uo)):
         err = orc.rel_frobenius(got, ref)
-        assert err.max() <= tol, f"{name} rel-F {err.max():.3e} at chunk {err.argmax()}"
+        bound = _bound(ref, 5e-4 if fp32_out else TOL_BF16, bf16_out=not fp32_out)
+        worst = int(np.argmax(err - bound))
+        assert np.all(err <= bound), f"{name} rel-F {err[worst]:.3e} > {bound[worst]:.3e} at chunk {worst}"
 
 
 def test_token_major_layout_is_bf16_only():
