@@ -98,12 +98,7 @@ def test_identical_keys_closed_form_in_integers():
     assert np.abs(W[:, 0] - expect).max() <= 2.0 ** float(out["w_exp"][0]) * 1.5 + 2 * step
 
 
-@pytest.mark.parametrize("adv,lo_T,lo_WU", [("none", 25.0, 28.0), ("all", 20.0, 20.0)])
-def test_dequantised_result_tracks_the_fp64_definition(adv, lo_T, lo_WU):
-    """Sanity band: the integer pipeline, dequantised, stays within an 8-bit SNR band of the fp64 inverse of the
-    same (dequantised) inputs. Guards against a wrong exponent or a dropped term, not a precision claim."""
-    inp, q, (Kq, Vq, ke, ve, bq, dq) = _int8_chunks(64, n_heads=2, T=128, seed=9, adversarial=adv, d=64)
-    out = orq.chunk_prepare_int8(Kq, Vq, ke, ve, bq, dq, 3, 8)
+def _dequantised_snr(out, Kq, Vq, ke, ve, bq, dq):
     K = Kq * np.exp2(ke.astype(float))[:, None, None]
     V = Vq * np.exp2(ve.astype(float))[:, None, None]
     beta = bq / 32768.0
@@ -112,10 +107,42 @@ def test_dequantised_result_tracks_the_fp64_definition(adv, lo_T, lo_WU):
     T = orq.dequantise(out["Toffq"], out["t_exp"])
     W = orq.dequantise(out["Wq"], out["w_exp"])
     U = orq.dequantise(out["Uq"], out["u_exp"])
-    eye = np.eye(64)
-    assert orc.snr_db(T, Te - eye).min() > lo_T
-    assert orc.snr_db(W, We).min() > lo_WU
-    assert orc.snr_db(U, Ue).min() > lo_WU
+    return orc.snr_db(T, Te - np.eye(Te.shape[-1])), orc.snr_db(W, We), orc.snr_db(U, Ue)
+
+
+@pytest.mark.parametrize("adv,lo_T,lo_W,lo_U", [("none", 26.0, 33.0, 33.0), ("all", 28.0, 22.0, 30.0)])
+def test_dequantised_result_tracks_the_fp64_definition(adv, lo_T, lo_W, lo_U):
+    """Sanity band: the integer pipeline, dequantised, stays within an 8-bit SNR band of the fp64 inverse of the
+    same (dequantised) inputs. The floors sit within 3 dB of what these inputs give (benign: T - I 28.3..33.7 dB,
+    W 35.1..36.1, U 35.3..36.2; adversarial: 30.6..33.2, 23.9..27.6, 32.1..33.6), so that a dropped term or a wrong
+    exponent cannot hide below them. Not a precision claim about the paper's INT8."""
+    for seed in (9, 10):
+        inp, q, (Kq, Vq, ke, ve, bq, dq) = _int8_chunks(64, n_heads=2, T=128, seed=seed, adversarial=adv, d=64)
+        out = orq.chunk_prepare_int8(Kq, Vq, ke, ve, bq, dq, 3, 8)
+        sT, sW, sU = _dequantised_snr(out, Kq, Vq, ke, ve, bq, dq)
+        assert sT.min() > lo_T and sW.min() > lo_W and sU.min() > lo_U, (sT, sW, sU)
+
+
+@pytest.mark.parametrize("adv", ["none", "all"])
+def test_alignment_window_of_8_bits_loses_nothing_against_24(adv, monkeypatch):
+    """An aligned sum keeps 8 bits below its largest term (which makes every sum fit 32 bits). The reading's claim
+    is that this costs nothing against a 24-bit window: every sum is requantised to 8 bits right afterwards, so
+    bits more than 8 below the largest term can only move the rounding of the last place. Both evaluators read the
+    window from the module, so each is run with both widths on the cases of the evaluator comparison: the quality
+    against the fp64 definition must agree within 0.2 dB chunk by chunk, and the two evaluators must still agree
+    bit for bit at either width."""
+    for C, N, S, seed in ((64, 3, 8, 9), (64, 3, 8, 10), (32, 3, 4, 11), (16, 2, 3, 12)):
+        inp, q, (Kq, Vq, ke, ve, bq, dq) = _int8_chunks(C, n_heads=2, T=2 * C, seed=seed, adversarial=adv, d=64)
+        snr = {}
+        for window in (8, 24):
+            monkeypatch.setattr(orq, "ALIGN_WINDOW", window)
+            out = orq.chunk_prepare_int8(Kq, Vq, ke, ve, bq, dq, N, S)
+            snr[window] = _dequantised_snr(out, Kq, Vq, ke, ve, bq, dq)
+            ref = orq.chunk_prepare_int8_ref(Kq[0].tolist(), Vq[0].tolist(), int(ke[0]), int(ve[0]), bq[0].tolist(), dq[0].tolist(), N, S)
+            assert np.array_equal(np.asarray(ref["Wq"]), out["Wq"][0]) and int(ref["w_exp"]) == int(out["w_exp"][0])
+            assert np.array_equal(np.asarray(ref["Toffq"]), out["Toffq"][0]) and int(ref["t_exp"]) == int(out["t_exp"][0])
+        for a, b in zip(snr[8], snr[24]):
+            assert np.abs(a - b).max() < 0.2, (a, b)
 
 
 def test_int8_input_recipe():
