@@ -89,7 +89,7 @@ typedef void* gdn_stream_t;
  * truncated Neumann series, residual power sum, W and U.
  *   dtype GDN_DTYPE_BF16: bf16 K, V, W, U, Tinv; tensor-core kernel; C in {16, 32, 64, 128},
  *                         d_k, d_v = 128, 1 <= order <= 7. fp32 accumulation.
- *   dtype GDN_DTYPE_FP32: fp32 everywhere, plain FMA kernel; 2 <= C <= 128, d_k, d_v <= 256.
+ *   dtype GDN_DTYPE_FP32: fp32 everywhere, plain FMA kernel; 2 <= C <= 64 or C = 128 (two 64-blocks), d_k, d_v <= 256.
  * Tinv_out may be NULL (the store is skipped). H = H_k = H_v.
  */
 int gdn_chunk_prepare(const void* K, const void* V, const float* beta, const float* g,
@@ -120,7 +120,10 @@ int gdn_chunk_prepare_ex(const void* K, const void* V, const float* beta, const 
  * The comparison the paper's speed-up is measured against: the same A-build, W
  * and U, with T computed exactly by forward substitution (Eq. 2-3;
  * variant GDN_FWDSUBST_ROWS) or by 16 x 16 diagonal blocks merged with the
- * block recursion of App. E (Eq. 25-27; variant GDN_FWDSUBST_BLOCKED).
+ * block recursion of App. E (Eq. 25-27; variant GDN_FWDSUBST_BLOCKED). Same dtypes, sizes and layouts as
+ * gdn_chunk_prepare_gqa. For C = 128 on the bf16 path both variants invert the two 64 x 64 diagonal blocks by
+ * their substitution and obtain the lower-left block from the block formula of App. E (Eq. 28), as the Neumann
+ * path does.
  */
 int gdn_chunk_prepare_fwdsubst(const void* K, const void* V, const float* beta, const float* g,
                                int B, int H_k, int H_v, int T, int C, int d_k, int d_v,

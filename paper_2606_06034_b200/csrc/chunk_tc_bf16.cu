@@ -435,7 +435,7 @@ __global__ void __launch_bounds__(kThreads, 2)
 chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                 const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmU,
                 const __grid_constant__ CUtensorMap tmT, const Params p) {
-    static_assert(!MERGE || (C == 64 && MODE == INV_NEUMANN), "the block merge is built for 64-blocks of the Neumann scheme");
+    static_assert(!MERGE || C == 64, "the block merge is built for 64-blocks");
     static_assert(DBL == 0 || ((DBL == 8 || DBL == 15) && C == 64 && MODE == INV_NEUMANN), "the doubling scheme is built for 64-blocks");
     using L = Smem<C, NB>;
     using SP = Split<C>;
@@ -1622,7 +1622,7 @@ int launch_wait_selftest(cudaStream_t stream) {
 
 int launch_tc_bf16(const Problem& p, InverseMode mode, cudaStream_t stream) {
     if (p.d_k != kD || p.d_v != kD) return GDN_ERR_UNSUPPORTED;
-    if (!(p.C == 16 || p.C == 32 || p.C == 64 || (p.C == 128 && mode == INV_NEUMANN))) return GDN_ERR_UNSUPPORTED;
+    if (!(p.C == 16 || p.C == 32 || p.C == 64 || p.C == 128)) return GDN_ERR_UNSUPPORTED;
     if (mode == INV_NEUMANN && (p.order < 1 || p.order > 7)) return GDN_ERR_UNSUPPORTED;
     if ((long long)p.B * p.H_v * p.T == 0) return GDN_OK;
     const bool varlen = p.chunk_start != nullptr;
@@ -1685,12 +1685,14 @@ int launch_tc_bf16(const Problem& p, InverseMode mode, cudaStream_t stream) {
         switch (p.C) {
             case 16: return launch_c<16, INV_FWDSUBST_BLOCKED>(m, prm, stream);
             case 32: return launch_c<32, INV_FWDSUBST_BLOCKED>(m, prm, stream);
+            case 128: return launch_c<64, INV_FWDSUBST_BLOCKED, true>(m, prm, stream);
             default: return launch_c<64, INV_FWDSUBST_BLOCKED>(m, prm, stream);
         }
     }
     switch (p.C) {
         case 16: return launch_c<16, INV_FWDSUBST_ROWS>(m, prm, stream);
         case 32: return launch_c<32, INV_FWDSUBST_ROWS>(m, prm, stream);
+        case 128: return launch_c<64, INV_FWDSUBST_ROWS, true>(m, prm, stream);  // 64-blocks by substitution, merged by App. E
         default: return launch_c<64, INV_FWDSUBST_ROWS>(m, prm, stream);
     }
 }

@@ -218,13 +218,14 @@ def test_bf16_without_tinv_and_determinism():
     assert torch.equal(W1, W3) and torch.equal(U1, U3) and torch.equal(T1, T3)
 
 
-@pytest.mark.parametrize("C", [16, 32, 64])
+@pytest.mark.parametrize("C", [16, 32, 64, 128])
 def test_bf16_forward_substitution_kernel(C):
+    # C = 128: the two 64-blocks by substitution, the lower-left block by the block formula of App. E
     inp = gen.make_inputs(1, 2, 4, 512, C, 128, 128, seed=80 + C, adversarial_heads="odd")
     _check(inp, TOL_BF16, method="fwdsubst", exact=True)
 
 
-@pytest.mark.parametrize("C", [16, 32, 64])
+@pytest.mark.parametrize("C", [16, 32, 64, 128])
 def test_bf16_blocked_forward_substitution_kernel(C):
     inp = gen.make_inputs(1, 2, 4, 512, C, 128, 128, seed=85 + C, adversarial_heads="odd")
     K, V, beta, g = _to_dev(inp)
