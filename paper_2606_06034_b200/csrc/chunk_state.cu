@@ -64,17 +64,6 @@ constexpr int kTab = 5 * 64;  // floats per table buffer: exp(g_i), exp(g_C - g_
 constexpr int kOffG = kOffO + 2 * kTileBytes;  // three table buffers
 constexpr int kSmemTotal = kOffG + 3 * kTab * 4;
 
-#ifdef GDN_TRACE
-__device__ long long g_trace_s[4096];
-// slot, clock pairs of block 0: compute thread 0 at [0, 2048), the issuing warp's lane 0 at [2048, 4096)
-#ifndef GDN_TRACE_SO
-#define GDN_TRACE_SO false
-#endif
-#define STAMPS(slot_) do { if (SO == GDN_TRACE_SO && blockIdx.x == 0 && (tid == 0 || tid == kThreads) && trace_n < 500) { \
-    g_trace_s[(tid == 0 ? 0 : 2048) + trace_n * 2] = (slot_); g_trace_s[(tid == 0 ? 0 : 2048) + trace_n * 2 + 1] = clock64(); ++trace_n; } } while (0)
-#else
-#define STAMPS(slot_) do { } while (0)
-#endif
 
 struct ParamsS {
     const float* g;
@@ -142,9 +131,6 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
-#ifdef GDN_TRACE
-    int trace_n = 0;
-#endif
     const int t = tid & 127;  // TMEM lane: value feature (state rows, output columns); token j for PT
     const int h = (tid >> 7) & 3;  // column quarter: 16 of the 64 columns of a product, 32 of the 128 state columns
     const int wq = warp & 3;
@@ -283,9 +269,7 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         for (int c = 0; c < n_c && *fail == 0; ++c) {
             const uint32_t st_a = smem_a + (c & 1) * kStageBytes;
             // the state copies (and, for the first chunk, the constant operand) are in place
-            STAMPS(100);
             handoff_wait<4>();
-            STAMPS(101);
             tc_fence_after_sync();
             if (c == 0) issue_pre(0);
             if (*fail == 0 && elect_one()) {
@@ -315,10 +299,8 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 // costs the threads ~200 cycles even on a completed phase)
             }
             __syncwarp();
-            STAMPS(102);
             // U_new^T (hi, lo; plain, scaled), P (hi, lo) and the decayed accumulator are in place
             handoff_wait<5>();
-            STAMPS(103);
             tc_fence_after_sync();
             if (*fail == 0 && elect_one()) {
                 if (!SO) {
@@ -350,9 +332,7 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             __syncwarp();
             // D1 and PT are only read by the products just issued, which the tensor pipe runs first: the
             // state-independent products of the next chunk follow them directly
-            STAMPS(104);
             if (c + 1 < n_c) issue_pre(c + 1);
-            STAMPS(105);
         }
     } else {
         // ================= compute threads (512): four per TMEM lane
@@ -491,9 +471,7 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             const int left = len - c * kC;
             const bool short_chunk = VAR && left < kC;
             if (c + 1 < n_c && tabler) g_reg = (!VAR || (c + 1) * kC + tt < len) ? __ldg(gseq + ((c + 1) * kC + tt) * gstep) : 0.f;
-            STAMPS(1);
 
-            STAMPS(2);
             // ---- decay of the accumulator, S <- exp(g_C) S0 (the products of this chunk read the bf16 copies)
             {
                 const float dec = fast_exp2(gC * kLog2e);
@@ -511,9 +489,7 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 tmem_st16(lane_base + kSD + h * 32 + 16, w16);
             }
             // ---- P_ij = exp(g_i - g_j) PT_ji for j <= i (hi + lo): token j = lane (rows 0..63 only), this thread's 16 columns i
-            STAMPS(3);
             if (!SO && !wait_group(&bar_pre, par_pre)) { ok = false; break; }
-            STAMPS(4);
             if (!SO && wq < 2) {
                 uint32_t d[16];
                 tmem_ld16(lane_base + kPT + h * 16, d);
@@ -555,7 +531,6 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             // products that consume them: the hi halves are written over its own D1 columns (plain -> 16 h .. 16 h + 7,
             // scaled -> 16 h + 8 ..), the lo halves at the same offsets of the PT region (read above by this thread).
             if (!wait_group(&bar_d1, par_d1)) { ok = false; break; }
-            STAMPS(6);
             {
                 uint32_t d[16];
                 tmem_ld16(lane_base + kD1 + h * 16, d);
@@ -588,7 +563,6 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             tmem_wait_st();
             tc_fence_before_sync();
             handoff_arrive<5>();
-            STAMPS(7);
             // with the norms of the next chunk's keys and queries in the tables, both are formed here instead: the next
             // chunk's tiles are still on their way while P is formed, and the threads idle now anyway
             if (c + 1 < n_c && f_nrm) {
@@ -605,7 +579,6 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 if (c >= 1 && !wait_bar(&bar_stg[(c - 1) & 1], ((c - 1) >> 1) & 1)) { *fail = 1; ok = false; break; }
                 // ---- exp(g_i) O1 (complete with O2: products finish in the order they were issued)
                 if (!wait_group(&bar_o2, par_o2)) { ok = false; break; }
-                STAMPS(8);
                 float o[16];
                 {
                     uint32_t d[16];
@@ -620,7 +593,6 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                         o[i4 * 4 + 3] = __uint_as_float(d[i4 * 4 + 3]) * e4.w;
                     }
                 }
-                STAMPS(10);
                 // ---- O^T = scale (exp(g_i) O1 + O2): element (token i, feature t) of the staged tile
                 {
                     uint32_t d[16];
@@ -642,7 +614,6 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             // ---- bf16 copies (hi, lo) of the new state for the next chunk's products; the lo half goes where O2 was
             // (this thread has read its O2 columns above)
             if (!wait_group(&bar_g2, par_g2)) { ok = false; break; }
-            STAMPS(12);
             {
                 uint32_t v[32], pk[16];
                 tmem_ld32(lane_base + kSD + h * 32, v);
@@ -658,7 +629,6 @@ chunk_state_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 tc_fence_before_sync();
                 handoff_arrive<4>();
             }
-            STAMPS(11);
             // With the norms in the tables, the next chunk's tables are written after this chunk's hand-off (see above),
             // so the hand-off -> product -> completion chain does not order them before their readers: one barrier.
             if (NRM && c + 1 < n_c) asm volatile("bar.sync 1, 512;" ::: "memory");
@@ -900,11 +870,6 @@ int launch_chunk_state_segmented_builtin(const ProblemS& q, int P, cudaStream_t 
     return launch_chunk_state_segmented(q, P, g_builtin_scratch_addr[dev], stream);
 }
 
-#ifdef GDN_TRACE
-extern "C" int gdn_debug_read_trace_state(long long* host_out) {
-    return cudaMemcpyFromSymbol(host_out, g_trace_s, sizeof(long long) * 4096) == cudaSuccess ? 0 : -1;
-}
-#endif
 
 int launch_chunk_state(const ProblemS& q, cudaStream_t stream) {
     if (q.d_k != kD || q.d_v != kD || q.C != kC) return GDN_ERR_UNSUPPORTED;

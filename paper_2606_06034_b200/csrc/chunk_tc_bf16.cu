@@ -45,12 +45,6 @@ constexpr float kLog2e = 1.4426950408889634f;
 //                         (high half, block diagonal)
 constexpr uint32_t kR0 = 0, kR2 = 128, kAS = 192, kTmemCols = 256;
 
-#ifdef GDN_TRACE
-__device__ long long g_trace[4096];
-#define STAMP(slot) do { if (blockIdx.x == 0 && (tid == 0 || tid == 160) && trace_n < 120) { g_trace[(tid == 0 ? 0 : 2048) + trace_n * 2] = (slot); g_trace[(tid == 0 ? 0 : 2048) + trace_n * 2 + 1] = clock64(); ++trace_n; } } while (0)
-#else
-#define STAMP(slot) do { } while (0)
-#endif
 
 // (New fields go at the END: the struct's layout decides which parameters ptxas fetches with one wide load, and a
 // field inserted in the middle moved the default instantiation from 36 to 96 bytes of spill, 10 % of its speed.)
@@ -472,9 +466,6 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
     const int lane = tid & 31;
-#ifdef GDN_TRACE
-    int trace_n = 0;
-#endif
 
     if (tid == 0) {
         mbar_init(&bar_k, 1);
@@ -618,7 +609,6 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         const uint32_t next = tile + gridDim.x;
         const bool has_next = next < n_tiles;
 
-        STAMP(1);
         const float bi = bi_next;  // loaded during the previous tile
         float gi_ = gi_next;
         const int gtok = gtok_next;
@@ -645,9 +635,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         }
         if (warp == 0) {
             // G = K K^T into R0..R1 (128 columns)
-            STAMP(20);
             if (!wait_bar(&bar_k, par_kv)) ok = false;
-            STAMP(21);
             if (ok) {
                 tc_fence_after_sync();
                 if (elect_one()) {
@@ -672,10 +660,8 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         }
         compute_barrier();
 
-        STAMP(2);
         // ---- A-build: this thread's part of the row of Abar, from the Gram block in TMEM
         if (!wait_mma()) { ok = false; break; }
-        STAMP(3);
         tc_fence_after_sync();
         float a[HC];
         if constexpr (MERGE) {
@@ -753,7 +739,6 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         if (has_next) fetch_row(pos_next, bi_next, gi_next, gtok_next);
         compute_barrier();  // both halves of every fp32 row are written
 
-        STAMP(4);
         float lb[NB + 1];  // lb[d] = L[i][i-d], the band of T0 - I (or of T - I after forward substitution)
 #pragma unroll
         for (int e = 0; e <= NB; ++e) lb[e] = 0.f;
@@ -796,7 +781,6 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             }
             compute_barrier();
 
-            STAMP(5);
             if (active) {
                 // ---- E = Abar + Abar L on i-j > N (in place over a[])
 #pragma unroll
@@ -938,7 +922,6 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             compute_barrier();  // the fp32 rows are dead; the packed rows may overwrite them
         }
 
-        STAMP(6);
         // ---- packed bf16 form of the band: I + L (the keep-mask, 0 on the band and diagonal, was built before the loop)
         uint32_t bpT[PCH];
         if (active) {
@@ -952,7 +935,6 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             for (int i = 0; i < PCH; ++i) bpT[i] = 0u;
         }
 
-        STAMP(7);
         if constexpr (MODE == INV_NEUMANN) {
             // ---- residual correction T = T0 sum_{s<=S} E^s (Eq. 13). With X_m = T0 sum_{s<=m} E^s:
             //   X_{m+1} = T0 + X_m E   and   X_{2m+1} = X_m + X_m E^{m+1}.
@@ -991,10 +973,8 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     tmem_wait_st();
 #pragma unroll
                     for (int lv = 0; lv < 4; ++lv) {
-                        STAMP(30 + lv);
                         tc_fence_before_sync();
                         compute_barrier();
-                        STAMP(40 + lv);
                         if (warp == 0) {
                             tc_fence_after_sync();
                             const uint32_t bb = (lv == 0 || (lv == 2 && !kFull)) ? sEB_a : sEB_a + 16384;
@@ -1012,7 +992,6 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                         }
                         if (!wait_mma()) { ok = false; break; }
                         tc_fence_after_sync();
-                        STAMP(50 + lv);
                         // in two halves of 16 columns, to keep the live registers down
 #pragma unroll
                         for (int hh = 0; hh < 2; ++hh) {
@@ -1073,10 +1052,8 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     fence_proxy_async_smem();
                     tmem_wait_st();
                 }
-                STAMP(60);
                 tc_fence_before_sync();
                 compute_barrier();
-                STAMP(61);
                 if (warp == 0) {
                     // [Z_1; Z_2; ...] <- [A_1; A_2; ...] [E_1 | E_2 | ...]: M = 128, N = 128, K = C; row t keeps
                     // the C columns of its own chunk
@@ -1090,10 +1067,8 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                         mma_commit(&bar_mma);
                     }
                 }
-                STAMP(62);
                 if (!wait_mma()) { ok = false; break; }
                 tc_fence_after_sync();
-                STAMP(63);
                 if (active) load_diag_block<C>(lane_base, kR0, t, h, a);
             }
             }
@@ -1279,7 +1254,6 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             }
         }
 
-        STAMP(9);
         // ---- A operands for W/U: T diag(scale) = hi + lo, hi over the whole row, lo only on band + diagonal.
         // scale = beta for U; for W it is beta / ||K|| when the keys are normalised on the fly, else beta as well
         if (active) {
@@ -1313,7 +1287,6 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             }
         }
 
-        STAMP(8);
         // ---- T row -> Tinv: each half-row goes to a staging line in the TMA swizzle layout (the band-row
         // region is free now); one bulk tensor store of 32 rows x HC columns per warp, overlapping the W products
         if (f_f32 && p.Tinv != nullptr && active) {
@@ -1395,14 +1368,12 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             }
         }
 
-        STAMP(10);
         // ---- W, then U: each thread reads 64 accumulator columns of its row -> bf16 -> swizzled staging
         // sub-tile of its warp -> one bulk tensor store (32 rows x 64 columns) per warp
 #pragma unroll 1
         for (int half = 0; half < 2; ++half) {
             if (!wait_mma()) { ok = false; break; }
             tc_fence_after_sync();
-            STAMP(11 + half * 3);
             if (warp == 0 && has_next && elect_one()) {
                 // the products that read this tile's K (half 0) or V (half 1) are complete: prefetch the next tile's
                 const TileCoord nc = tile_coord<EX>(pos_next, p);
@@ -1460,7 +1431,6 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     }
                 }
             }
-            STAMP(12 + half * 3);
             // variable-length sequences: a warp whose 32 rows are 32 consecutive real tokens stores them like the dense
             // path (token coordinate of its first row); otherwise (a short chunk, or two chunks that are not adjacent in
             // memory) every row of a real token goes out by itself, so that nothing reaches a neighbouring sequence
@@ -1493,7 +1463,6 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     tma_store_commit();
                 }
             }
-            STAMP(13 + half * 3);
         }
         par_kv ^= 1;
     }
@@ -1593,11 +1562,6 @@ int launch_c(const Maps& m, const Params& prm, cudaStream_t stream) {
 
 }  // namespace
 
-#ifdef GDN_TRACE
-extern "C" int gdn_debug_read_trace(long long* host_out) {
-    return cudaMemcpyFromSymbol(host_out, g_trace, sizeof(long long) * 4096) == cudaSuccess ? 0 : -1;
-}
-#endif
 
 namespace {
 // waits on an mbarrier that never completes: wait_bar must give up after its budget and report it

@@ -40,12 +40,6 @@ constexpr int kSMax = 8;   // largest number of residual terms held in registers
 constexpr int kAlignWindow = 8;  // bits kept below the largest term of an aligned sum: every such sum fits 32 bits
 constexpr uint32_t kR0 = 0, kAS = 128, kTmemCols = 256;
 
-#ifdef GDN_TRACE
-__device__ long long g_trace8[4096];
-#define STAMP8(slot_) do { if (blockIdx.x == 0 && tid == 32 && trace_n < 200) { g_trace8[trace_n * 2] = (slot_); g_trace8[trace_n * 2 + 1] = clock64(); ++trace_n; } } while (0)
-#else
-#define STAMP8(slot_) do { } while (0)
-#endif
 
 struct ParamsI8 {
     const int16_t* beta_q;
@@ -196,18 +190,17 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
 
     __shared__ uint64_t bar_k, bar_v, bar_mma;
     __shared__ uint32_t tmem_base_s;
+    __shared__ int s_fail;  // set by warp 0 when one of its bounded waits ran out
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
     const int lane = tid & 31;
-#ifdef GDN_TRACE
-    int trace_n = 0;
-#endif
 
     if (tid == 0) {
         mbar_init(&bar_k, 1);
         mbar_init(&bar_v, 1);
         mbar_init(&bar_mma, 1);
+        s_fail = 0;
         mbar_fence_init();
         tma_prefetch_desc(&tmK);
         tma_prefetch_desc(&tmV);
@@ -243,6 +236,16 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
     const uint32_t idesc_m = instr_desc(128, 128, 1, 1, 0, 1, 2);  // B MN-major
     uint32_t par_mma = 0, par_kv = 0;
     bool ok = true;
+    // Completion of the MMAs committed to bar_mma: warp 0 polls the mbarrier, the other warps sleep on a hardware
+    // barrier that warp 0 joins afterwards. A wait that ran out (here, or thread 0's waits for the K and V tiles) is
+    // published in s_fail, so that all 256 threads leave the tile loop at the same point.
+    auto wait_mma = [&]() -> bool {
+        if (warp == 0 && (*reinterpret_cast<volatile int*>(&s_fail) != 0 || !wait_bar(&bar_mma, par_mma)))
+            *reinterpret_cast<volatile int*>(&s_fail) = 1;
+        asm volatile("bar.sync 2, 256;" ::: "memory");
+        par_mma ^= 1;
+        return *reinterpret_cast<volatile int*>(&s_fail) == 0;
+    };
 
     // bit length of the OR of |values| over the chunk; `slot` is a fresh reduction slot of this tile
     auto chunk_bitlen = [&](unsigned long long m, int slot) -> int {
@@ -288,7 +291,6 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
         int32_t* dbg_row = (p.dbg != nullptr && row_valid)
                                ? p.dbg + (((long long)tc.bhv * n_c + chunk_in_head) * kC + il) * kDbgRow
                                : nullptr;
-        STAMP8(1);
         int bq = 0, dq = 0, kexp = 0, vexp = 0;
         if (row_valid) {
             bq = static_cast<int>(static_cast<uint16_t>(p.beta_q[grow]));
@@ -302,7 +304,10 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
         tc_fence_before_sync();
         cta_barrier();  // previous tile finished with shared arrays and accumulators
         if (tid == 0) {
-            if (!wait_bar(&bar_k, par_kv)) ok = false;
+            if (!wait_bar(&bar_k, par_kv)) {
+                ok = false;
+                *reinterpret_cast<volatile int*>(&s_fail) = 1;
+            }
             if (ok) {
                 tc_fence_after_sync();
 #pragma unroll
@@ -327,10 +332,8 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
         cta_barrier();
         int slot = 0;
 
-        STAMP8(2);
         // ---- I1-I3: Aq = Q8(-(G o c))
-        if (!wait_bar(&bar_mma, par_mma)) { ok = false; break; }
-        par_mma ^= 1;
+        if (!wait_mma()) { ok = false; break; }
         tc_fence_after_sync();
         int aq[kHC];
         int eA;
@@ -373,7 +376,6 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             }
             eA = 2 * kexp - 15 + r;
         }
-        STAMP8(3);
         // Aq bytes to the private row; entries next to the diagonal and right of this half come back from there
         uint8_t* rowa = sRowA + t * 64;
         {
@@ -405,7 +407,6 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
         }
         cta_barrier();
 
-        STAMP8(4);
         // ---- I4: P_2, P_3 (band only), I5: T0q
         int t0q1 = 0, t0q2 = 0, t0q3 = 0;  // T0q[i][i-1..i-3]
         int eT0;
@@ -456,7 +457,6 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             cta_barrier();
         }
 
-        STAMP8(5);
         // ---- I6: Eq = Q8(align(Aq, Aq T0q)) on i-j > N
         int eq[kHC];
         int eE;
@@ -484,7 +484,6 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             for (int jl = 0; jl < kHC; ++jl) eq[jl] = q8_32(acc[jl], rq);
             eE = eref + r;
         }
-        STAMP8(6);
         // packed rows of the powers R_s (R_1 = Eq) and their exponents
         uint32_t rpk[kSMax][kHC / 4];
         int er[kSMax];
@@ -530,8 +529,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 }
                 mma_commit(&bar_mma);
             }
-            if (!wait_bar(&bar_mma, par_mma)) { ok = false; break; }
-            par_mma ^= 1;
+            if (!wait_mma()) { ok = false; break; }
             tc_fence_after_sync();
             uint32_t dres[kHC];
             tmem_ld32(lane_base + kR0 + cb + col0, dres);
@@ -556,7 +554,6 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
         }
         if (!ok) break;
 
-        STAMP8(7);
         // ---- Sq = Q8(align(R_1..)): the exponents fall by several bits per power, so most terms are
         // shifted far to the right; a term whose right shift exceeds 7 rounds to zero and is skipped
         int sq[kHC];
@@ -595,7 +592,6 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
 #pragma unroll
             for (int jl = 0; jl < kHC; ++jl) sq[jl] = 0;
         }
-        STAMP8(8);
         // Sq bytes to the private rows (the rows above are needed for T0q Sq)
         {
             uint4 v0, v1;
@@ -608,7 +604,6 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
         }
         cta_barrier();
 
-        STAMP8(9);
         // ---- I8: Toffq = Q8(align(T0q, Sq, T0q Sq)) on i > j
         int toff[kHC];
         int eT;
@@ -655,7 +650,6 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             eT = eref + r;
         }
 
-        STAMP8(10);
         // ---- I9: Tbq = Q8(Toffq_ij beta_q_j); A operand of W/U (block diagonal, int8 in TMEM)
         int eTb;
         {
@@ -680,7 +674,6 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             tmem_st8(lane_base + kAS + (16 - cb / 4) + h * 8, r8);
             tmem_wait_st();
         }
-        STAMP8(11);
         // Toffq row -> staging (64-byte lines, 64-byte TMA swizzle) -> bulk tensor store of 32 rows per warp (h = 0 issues)
         uint8_t* stage = smem + kOffStage;
         if (p.Toff != nullptr) {
@@ -714,7 +707,6 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             mma_commit(&bar_mma);
         }
 
-        STAMP8(12);
         // ---- I10: W, then U
 #pragma unroll 1
         for (int half = 0; half < 2; ++half) {
@@ -727,8 +719,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 const uint4 v = *reinterpret_cast<const uint4*>(xtile + t * 128 + (((h * 4 + c) ^ (t & 7)) << 4));
                 xr[4 * c + 0] = v.x; xr[4 * c + 1] = v.y; xr[4 * c + 2] = v.z; xr[4 * c + 3] = v.w;
             }
-            if (!wait_bar(&bar_mma, par_mma)) { ok = false; break; }
-            par_mma ^= 1;
+            if (!wait_mma()) { ok = false; break; }
             tc_fence_after_sync();
             const int ep = eTb + xexp, ed = xexp - 15;
             const int eref = align_ref2(ep, ed);
@@ -799,7 +790,10 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 tc_fence_before_sync();
                 cta_barrier();  // every row of the W accumulator has been read
                 if (tid == 0) {
-                    if (!wait_bar(&bar_v, par_kv)) ok = false;
+                    if (!wait_bar(&bar_v, par_kv)) {
+                        ok = false;
+                        *reinterpret_cast<volatile int*>(&s_fail) = 1;
+                    }
                     if (ok) {
                         tc_fence_after_sync();
 #pragma unroll
@@ -818,7 +812,6 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 tma_store_commit();
             }
         }
-        STAMP8(13);
         par_kv ^= 1;
     }
     if (lane == 0) tma_store_wait_all<0>();
@@ -865,11 +858,6 @@ bool make_map(CUtensorMap* tm, const void* base, long long heads, int T, int col
 
 }  // namespace
 
-#ifdef GDN_TRACE
-extern "C" int gdn_debug_read_trace8(long long* host_out) {
-    return cudaMemcpyFromSymbol(host_out, g_trace8, sizeof(long long) * 4096) == cudaSuccess ? 0 : -1;
-}
-#endif
 
 void int8_decay_lut(uint16_t* out) {
     for (int f = 0; f < 256; ++f) out[f] = static_cast<uint16_t>(floor(32768.0 * exp2(-static_cast<double>(f) / 256.0) + 0.5));
