@@ -53,6 +53,30 @@ import numpy as np
 
 QMAX = 127
 ALIGN_WINDOW = 8  # bits kept below the largest term of an aligned sum
+# Width of the mantissas (8 here). `gdn_oracle_int16` evaluates the same steps with 16-bit mantissas by running
+# these evaluators under `mantissa_width(16)`: QMAX = 2^15 - 1, shifts from bitlen - 15, a 16-bit alignment window,
+# matrix products checked against 62 bits instead of 31.
+MANT_BITS = 8
+ACC_BITS = 31
+
+
+class mantissa_width:
+    """Context manager that switches both evaluators of this module to `bits`-bit mantissas (8 or 16)."""
+
+    def __init__(self, bits: int):
+        assert bits in (8, 16)
+        self.new = (bits, (1 << (bits - 1)) - 1, bits, 31 if bits == 8 else 62)
+
+    def __enter__(self):
+        global MANT_BITS, QMAX, ALIGN_WINDOW, ACC_BITS
+        self.old = (MANT_BITS, QMAX, ALIGN_WINDOW, ACC_BITS)
+        MANT_BITS, QMAX, ALIGN_WINDOW, ACC_BITS = self.new
+        return self
+
+    def __exit__(self, *exc):
+        global MANT_BITS, QMAX, ALIGN_WINDOW, ACC_BITS
+        MANT_BITS, QMAX, ALIGN_WINDOW, ACC_BITS = self.old
+        return False
 
 
 def decay_lut() -> list[int]:
@@ -81,7 +105,7 @@ def _q8(acc, e, support):
     m = 0
     for idx in support:
         m = max(m, abs(acc[idx]))
-    r = max(0, m.bit_length() - 7)
+    r = max(0, m.bit_length() - (MANT_BITS - 1))
     out = {}
     for idx in support:
         q = _rsr(acc[idx], r)
@@ -233,7 +257,7 @@ def _shift_np(x: np.ndarray, s: np.ndarray) -> np.ndarray:
 def _q8_np(acc: np.ndarray, e: np.ndarray, support: np.ndarray):
     acc = np.where(support, acc, 0).astype(np.int64)
     m = np.abs(acc).max(axis=(-1, -2))
-    r = np.maximum(0, _bitlen(m) - 7)
+    r = np.maximum(0, _bitlen(m) - (MANT_BITS - 1))
     q = np.clip(_rsr_np(acc, r[..., None, None]), -QMAX, QMAX)
     return np.where(support, q, 0).astype(np.int64), np.asarray(e, dtype=np.int64) + r
 
@@ -249,7 +273,7 @@ def _align_np(terms, support):
 
 def _mm_i32(a: np.ndarray, b: np.ndarray) -> np.ndarray:
     out = np.matmul(a.astype(np.int64), b.astype(np.int64))
-    assert np.abs(out).max(initial=0) < 2 ** 31, "an MMA accumulator would overflow int32"
+    assert np.abs(out).max(initial=0) < 2 ** ACC_BITS, "a matrix-product accumulator would overflow"
     return out
 
 
@@ -338,10 +362,11 @@ def chunk_prepare_int8(Kq, Vq, k_exp, v_exp, beta_q, decay_q, N: int, S: int):
             acc_all[:, :, (s_ - 1) * C:s_ * C] = prod_
     acc_all[:, :, 8 * C:8 * C + dk] = acc_W
     acc_all[:, :, 8 * C + dk:] = acc_U
+    mt = np.int8 if MANT_BITS == 8 else np.int16
     return {"acc": acc_all,
-            "Wq": Wq.astype(np.int8), "w_exp": eW, "Uq": Uq.astype(np.int8), "u_exp": eU,
-            "Toffq": Toffq.astype(np.int8), "t_exp": eT, "Aq": Aq.astype(np.int8), "a_exp": eA,
-            "Eq": Eq.astype(np.int8), "e_exp": eE, "T0q": T0q.astype(np.int8), "t0_exp": eT0}
+            "Wq": Wq.astype(mt), "w_exp": eW, "Uq": Uq.astype(mt), "u_exp": eU,
+            "Toffq": Toffq.astype(mt), "t_exp": eT, "Aq": Aq.astype(mt), "a_exp": eA,
+            "Eq": Eq.astype(mt), "e_exp": eE, "T0q": T0q.astype(mt), "t0_exp": eT0}
 
 
 def dequantise(q: np.ndarray, e: np.ndarray) -> np.ndarray:

@@ -171,24 +171,31 @@ class Int8Inputs:
         return self.B * self.H_v * (self.T // self.C)
 
 
-def _quantise_per_chunk(x: torch.Tensor, C: int):
-    """Symmetric int8 with the smallest power-of-two scale that keeps max|x| / 2^e <= 127 per chunk."""
+def _quantise_per_chunk(x: torch.Tensor, C: int, bits: int = 8):
+    """Symmetric `bits`-bit mantissas with the smallest power-of-two scale that keeps max|x| / 2^e <= qmax per chunk
+    (qmax = 127 or 32767)."""
     B, H, T, d = x.shape
+    qmax = float((1 << (bits - 1)) - 1)
     xf = x.float().view(B, H, T // C, C * d)
     m = xf.abs().amax(dim=-1).clamp_min(1e-30)
-    e = torch.ceil(torch.log2(m / 127.0)).to(torch.int32)
-    # guard against log2 rounding: raise e where the scaled maximum still exceeds 127
-    e = torch.where(m / torch.exp2(e.float()) > 127.0, e + 1, e)
-    q = torch.round(xf / torch.exp2(e.float()).unsqueeze(-1)).clamp_(-127, 127).to(torch.int8)
+    e = torch.ceil(torch.log2(m / qmax)).to(torch.int32)
+    # guard against log2 rounding: raise e where the scaled maximum still exceeds qmax
+    e = torch.where(m / torch.exp2(e.float()) > qmax, e + 1, e)
+    q = torch.round(xf / torch.exp2(e.float()).unsqueeze(-1)).clamp_(-qmax, qmax).to(torch.int8 if bits == 8 else torch.int16)
     return q.view(B, H, T, d).contiguous(), e.contiguous()
 
 
-def make_int8_inputs(inp: ChunkInputs) -> Int8Inputs:
-    Kq, k_exp = _quantise_per_chunk(inp.K, inp.C)
-    Vq, v_exp = _quantise_per_chunk(inp.V, inp.C)
+def make_int8_inputs(inp: ChunkInputs, bits: int = 8) -> Int8Inputs:
+    """Integer inputs of the INT8 entry point, or with bits = 16 of the INT16 entry point (Kq, Vq int16, the rest alike)."""
+    Kq, k_exp = _quantise_per_chunk(inp.K, inp.C, bits)
+    Vq, v_exp = _quantise_per_chunk(inp.V, inp.C, bits)
     beta_q = torch.round(inp.beta.float() * 32768.0).clamp_(0, 32767).to(torch.int16).contiguous()
     decay_q = torch.round(-inp.g.double() * (1.4426950408889634 * 256.0)).to(torch.int32).contiguous()
     return Int8Inputs(Kq, Vq, k_exp, v_exp, beta_q, decay_q, inp.B, inp.H_k, inp.H_v, inp.T, inp.C, inp.d_k, inp.d_v)
+
+
+def make_int16_inputs(inp: ChunkInputs) -> Int8Inputs:
+    return make_int8_inputs(inp, bits=16)
 
 
 def int8_chunk_slices(q: Int8Inputs, chunk_ids):
