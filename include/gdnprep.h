@@ -153,6 +153,28 @@ int gdn_chunk_prepare_int8(const int8_t* Kq, const int8_t* Vq, const int32_t* k_
                            int8_t* Toff_q_out, int32_t* t_exp_out, int32_t* dbg_acc_out, gdn_stream_t stream);
 
 /*
+ * INT16 variant: the paper's primary integer precision for the inverse (Sec. 4.2, Table 1: INT16 within 0.4 dB of
+ * FP16; App. G table, row "Matrix Inversion"; quantiser of App. G, Eq. 32). The same chain as
+ * gdn_chunk_prepare_int8 with 16-bit mantissas in [-32767, 32767], one power-of-two exponent per chunk, aligned sums
+ * that keep 16 bits below their largest term, requantisation after every product and sum with the structural mask
+ * applied first. B200 has no 16-bit integer tensor path: every matrix product runs on the 8-bit integer tensor cores
+ * over the high and low bytes of the mantissas (four byte-plane products, recombined exactly in 64 bits).
+ * The outputs are a pure function of the integer inputs (bit-exact against an exact-integer evaluation).
+ *   Kq [B,H_k,T,d_k], Vq [B,H_v,T,d_v] int16 with k_exp [B,H_k,T/C], v_exp [B,H_v,T/C]: value = q * 2^exp;
+ *   beta_q, decay_q as for gdn_chunk_prepare_int8.
+ *   Wq_out [B,H_v,T,d_k], Uq_out [B,H_v,T,d_v] int16 with w_exp_out, u_exp_out [B,H_v,T/C];
+ *   Toff_q_out [B,H_v,T/C,C,C] int16 (may be NULL) with t_exp_out [B,H_v,T/C]: T = I + Toff_q * 2^t_exp.
+ *   dbg_acc_out (may be NULL; meant for small cases): the exact matrix products of the chain as int64,
+ *   [B,H_v,T/C, C, 8*C + d_k + d_v], laid out as for gdn_chunk_prepare_int8.
+ * Supported: C = 64, d_k = d_v = 128, 1 <= order <= 3, residual_steps <= 8.
+ */
+int gdn_chunk_prepare_int16(const int16_t* Kq, const int16_t* Vq, const int32_t* k_exp, const int32_t* v_exp,
+                            const uint16_t* beta_q, const int32_t* decay_q,
+                            int B, int H_k, int H_v, int T, int C, int d_k, int d_v, int order, int residual_steps,
+                            int16_t* Wq_out, int16_t* Uq_out, int32_t* w_exp_out, int32_t* u_exp_out,
+                            int16_t* Toff_q_out, int32_t* t_exp_out, int64_t* dbg_acc_out, gdn_stream_t stream);
+
+/*
  * gdn_chunk_prepare_ex for packed variable-length sequences (one batch of sequences laid end to end along the token
  * axis, as model code passes them with cumulative sequence lengths). Every sequence is cut into chunks of C tokens from
  * its own first token; its last chunk may be shorter. A short chunk is the chunk of C tokens whose missing tokens

@@ -37,7 +37,7 @@ GDN_FWDSUBST_BLOCKED = 1
 EXPORTS = (
     "gdn_chunk_prepare", "gdn_chunk_prepare_gqa", "gdn_chunk_prepare_ex", "gdn_chunk_prepare_varlen",
     "gdn_chunk_prepare_fwdsubst",
-    "gdn_chunk_prepare_int8", "gdn_chunk_state_output", "gdn_chunk_state_output_varlen", "gdn_chunk_state_output_segmented",
+    "gdn_chunk_prepare_int8", "gdn_chunk_prepare_int16", "gdn_chunk_state_output", "gdn_chunk_state_output_varlen", "gdn_chunk_state_output_segmented",
     "gdn_chunk_state_output_segmented_noalloc",
     "gdn_chunk_state_segments", "gdn_chunk_state_segmented_workspace", "gdn_selftest_bounded_wait",
     "gdn_int8_lut_checksum",
@@ -77,6 +77,8 @@ def load_library() -> ctypes.CDLL:
     lib.gdn_chunk_prepare_fwdsubst.argtypes = [vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ip, ip, ip, vp, vp, vp, vp]
     lib.gdn_chunk_prepare_int8.restype = ip
     lib.gdn_chunk_prepare_int8.argtypes = [vp, vp, vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ip, ip, ip, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.gdn_chunk_prepare_int16.restype = ip
+    lib.gdn_chunk_prepare_int16.argtypes = [vp, vp, vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ip, ip, ip, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.gdn_int8_lut_checksum.restype = ctypes.c_uint
     lib.gdn_chunk_state_output.argtypes = [vp, vp, vp, vp, vp, ip, ip, ip, ip, ip, ip, ip, ctypes.c_float, vp, vp, vp,
                                            ctypes.c_uint, vp]
@@ -301,6 +303,43 @@ def chunk_prepare_int8(q, order=-1, residual_steps=-1, *, want_toff=True, output
     Wq, Uq, w_exp, u_exp, Toff, t_exp = outputs
     gdn_chunk_prepare_int8(q.Kq, q.Vq, q.k_exp, q.v_exp, q.beta_q, q.decay_q, q.B, q.H_k, q.H_v, q.T, q.C, q.d_k, q.d_v,
                            order, residual_steps, Wq, Uq, w_exp, u_exp, Toff, t_exp, dbg_acc)
+    return outputs
+
+
+def gdn_chunk_prepare_int16(Kq, Vq, k_exp, v_exp, beta_q, decay_q, B, H_k, H_v, T, C, d_k, d_v, order, residual_steps,
+                            Wq_out, Uq_out, w_exp_out, u_exp_out, Toff_q_out, t_exp_out, dbg_acc_out=None, *, check=True):
+    """Raw call of the INT16 entry point (tensors instead of pointers, torch's current stream)."""
+    for t in (Kq, Vq, k_exp, v_exp, beta_q, decay_q, Wq_out, Uq_out, w_exp_out, u_exp_out, t_exp_out):
+        if not t.is_cuda or not t.is_contiguous():
+            raise ValueError("all tensors must be contiguous CUDA tensors (there is no CPU path)")
+    rc = load_library().gdn_chunk_prepare_int16(_ptr(Kq), _ptr(Vq), _ptr(k_exp), _ptr(v_exp), _ptr(beta_q), _ptr(decay_q),
+                                                B, H_k, H_v, T, C, d_k, d_v, order, residual_steps, _ptr(Wq_out),
+                                                _ptr(Uq_out), _ptr(w_exp_out), _ptr(u_exp_out), _ptr(Toff_q_out),
+                                                _ptr(t_exp_out), _ptr(dbg_acc_out), _stream())
+    if check and rc != GDN_OK:
+        raise GdnError(rc, "gdn_chunk_prepare_int16")
+    return rc
+
+
+def chunk_prepare_int16(q, order=-1, residual_steps=-1, *, want_toff=True, outputs=None, dbg_acc=None):
+    """Convenience wrapper over 16-bit integer inputs (`inputs.make_int16_inputs`, tensors on the GPU).
+
+    Returns (Wq, Uq, w_exp, u_exp, Toff_q, t_exp), mantissas int16. `dbg_acc`: optional zeroed int64 tensor
+    [B, H_v, T/C, C, 8*C + d_k + d_v] that receives the exact matrix products (small cases).
+    """
+    dev = q.Kq.device
+    n_c = q.T // q.C
+    if outputs is None:
+        Wq = torch.empty(q.B, q.H_v, q.T, q.d_k, dtype=torch.int16, device=dev)
+        Uq = torch.empty(q.B, q.H_v, q.T, q.d_v, dtype=torch.int16, device=dev)
+        w_exp = torch.empty(q.B, q.H_v, n_c, dtype=torch.int32, device=dev)
+        u_exp = torch.empty_like(w_exp)
+        t_exp = torch.empty_like(w_exp)
+        Toff = torch.empty(q.B, q.H_v, n_c, q.C, q.C, dtype=torch.int16, device=dev) if want_toff else None
+        outputs = (Wq, Uq, w_exp, u_exp, Toff, t_exp)
+    Wq, Uq, w_exp, u_exp, Toff, t_exp = outputs
+    gdn_chunk_prepare_int16(q.Kq, q.Vq, q.k_exp, q.v_exp, q.beta_q, q.decay_q, q.B, q.H_k, q.H_v, q.T, q.C, q.d_k, q.d_v,
+                            order, residual_steps, Wq, Uq, w_exp, u_exp, Toff, t_exp, dbg_acc)
     return outputs
 
 

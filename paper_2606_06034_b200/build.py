@@ -13,7 +13,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libgdnprep.so")
-SOURCES = ["gdn_api.cu", "chunk_simt.cu", "chunk_tc_bf16.cu", "chunk_tc_int8.cu", "chunk_state.cu"]
+SOURCES = ["gdn_api.cu", "chunk_simt.cu", "chunk_tc_bf16.cu", "chunk_tc_int8.cu", "chunk_tc_int16.cu", "chunk_state.cu"]
 HEADERS = ["common.cuh", "sm100_ptx.cuh", os.path.join("..", "..", "include", "gdnprep.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]

@@ -49,6 +49,25 @@ struct ProblemI8 {
     int order, steps;
 };
 
+// INT16 entry point's problem description (the INT8 one with 16-bit mantissas and 64-bit debug accumulators)
+struct ProblemI16 {
+    const int16_t* Kq;
+    const int16_t* Vq;
+    const int32_t* k_exp;
+    const int32_t* v_exp;
+    const int16_t* beta_q;
+    const int32_t* decay_q;
+    int16_t* Wq;
+    int16_t* Uq;
+    int32_t* w_exp;
+    int32_t* u_exp;
+    int16_t* Toff;  // may be null
+    int32_t* t_exp;
+    long long* dbg;  // may be null: exact matrix products of the chain
+    int B, H_k, H_v, T, C, d_k, d_v;
+    int order, steps;
+};
+
 // State passing + output of the layer, given W (gated) and U of every chunk
 struct ProblemS {
     const void* Q;
@@ -89,6 +108,7 @@ size_t chunk_state_segmented_workspace(int H_v, int P);
 int launch_chunk_state_segmented_builtin(const ProblemS& q, int P, cudaStream_t stream);
 int chunk_state_auto_segments(long long H_v);
 int launch_tc_int8(const ProblemI8& p, cudaStream_t stream);
+int launch_tc_int16(const ProblemI16& p, cudaStream_t stream);
 void int8_decay_lut(uint16_t* out256);  // table of round(2^15 * 2^(-f/256))
 
 }  // namespace gdn

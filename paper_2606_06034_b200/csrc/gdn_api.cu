@@ -177,6 +177,29 @@ int gdn_chunk_prepare_int8(const int8_t* Kq, const int8_t* Vq, const int32_t* k_
     return launch_tc_int8(q, static_cast<cudaStream_t>(stream));
 }
 
+int gdn_chunk_prepare_int16(const int16_t* Kq, const int16_t* Vq, const int32_t* k_exp, const int32_t* v_exp,
+                            const uint16_t* beta_q, const int32_t* decay_q, int B, int H_k, int H_v, int T, int C, int d_k,
+                            int d_v, int order, int residual_steps, int16_t* Wq_out, int16_t* Uq_out, int32_t* w_exp_out,
+                            int32_t* u_exp_out, int16_t* Toff_q_out, int32_t* t_exp_out, int64_t* dbg_acc_out,
+                            gdn_stream_t stream) {
+    if (order == -1) order = gdn_default_order(C);
+    if (residual_steps == -1) residual_steps = gdn_default_residual_steps(C);
+    if (Kq == nullptr || Vq == nullptr || k_exp == nullptr || v_exp == nullptr || beta_q == nullptr || decay_q == nullptr ||
+        Wq_out == nullptr || Uq_out == nullptr || w_exp_out == nullptr || u_exp_out == nullptr || t_exp_out == nullptr)
+        return GDN_ERR_NULL;
+    if (B < 0 || H_k <= 0 || H_v <= 0 || T < 0 || C < 2 || d_k <= 0 || d_v <= 0) return GDN_ERR_INVALID_ARG;
+    if (H_v % H_k != 0 || T % C != 0) return GDN_ERR_INVALID_ARG;
+    if (order < 1 || order >= C || residual_steps < 0) return GDN_ERR_INVALID_ARG;
+    if (!aligned16(Kq) || !aligned16(Vq) || !aligned16(Wq_out) || !aligned16(Uq_out) || !aligned16(Toff_q_out) || !aligned16(dbg_acc_out))
+        return GDN_ERR_ALIGN;
+    const int rc = check_arch();
+    if (rc != GDN_OK) return rc;
+    ProblemI16 q{Kq, Vq, k_exp, v_exp, reinterpret_cast<const int16_t*>(beta_q), decay_q, Wq_out, Uq_out, w_exp_out, u_exp_out,
+                 Toff_q_out, t_exp_out, reinterpret_cast<long long*>(dbg_acc_out), B, H_k, H_v, T, C, d_k, d_v, order,
+                 residual_steps};
+    return launch_tc_int16(q, static_cast<cudaStream_t>(stream));
+}
+
 int gdn_chunk_state_output(const void* Q, const void* K, const void* W_gated, const void* U, const float* g, int B, int H_k,
                            int H_v, int T, int C, int d_k, int d_v, float scale, const float* S_in, void* O_out, float* S_out,
                            unsigned flags, gdn_stream_t stream) {
