@@ -295,6 +295,9 @@ def run_ours(args, rank, world, dist_ctx):
     if method == "int8":
         q8 = gen.make_int8_inputs(inp)
         q8_outs = gdn.chunk_prepare_int8(q8)
+    if method == "int16":
+        q8 = gen.make_int16_inputs(inp)
+        q8_outs = gdn.chunk_prepare_int16(q8)
     st_args = None
     if method == "state":  # state passing + output of the layer, given the gated W and U
         gq = torch.Generator(device=dev).manual_seed(99)
@@ -317,6 +320,8 @@ def run_ours(args, rank, world, dist_ctx):
             gdn.chunk_prepare(*mn_args[0], C, outputs=mn_args[1], flags=mn_args[2])
         elif method == "int8":
             gdn.chunk_prepare_int8(q8, outputs=q8_outs)
+        elif method == "int16":
+            gdn.chunk_prepare_int16(q8, outputs=q8_outs)
         elif method == "state":
             gdn.chunk_state_output(st_args[0], inp.K, st_args[1], st_args[2], inp.g, C, inp.d_k ** -0.5, outputs=st_args[3])
         else:
@@ -372,6 +377,8 @@ def run_ours(args, rank, world, dist_ctx):
         bytes_chunk = C * inp.d_k * 2 * (2.0 / group + 1) + 2 * C * inp.d_v * 2 + 4 * C
     if method == "int8":  # one byte per element, u16 beta + i32 decay per token
         bytes_chunk = C * inp.d_k / group + C * inp.d_v + C * inp.d_k + C * inp.d_v + C * C + 6 * C
+    if method == "int16":  # two bytes per element
+        bytes_chunk = 2 * (C * inp.d_k / group + C * inp.d_v + C * inp.d_k + C * inp.d_v + C * C) + 6 * C
     flops_chunk = nominal_flops_per_chunk(C, inp.d_k, inp.d_v)
     hbm_peak, bf16_peak, peak_kind = measured_peaks()
     launch_ms = float(np.mean(per))
@@ -383,7 +390,7 @@ def run_ours(args, rank, world, dist_ctx):
     roofline = {"bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak,
                 "traffic": traffic, "peak_kind": peak_kind,
                 "algorithmic_bytes_per_launch": n_chunks * bytes_chunk,
-                "kernel": {"int8": "chunk_tc_int8_kernel", "state": "chunk_state_kernel"}.get(method, "chunk_tc_kernel<C=%d>" % C),
+                "kernel": {"int8": "chunk_tc_int8_kernel", "int16": "chunk_tc_int16_kernel", "state": "chunk_state_kernel"}.get(method, "chunk_tc_kernel<C=%d>" % C),
                 "effective_tflops": n_chunks * flops_chunk / (launch_ms * 1e-3) / 1e12,
                 "tensor_time_frac_of_bf16_peak": (n_chunks * flops_chunk / (launch_ms * 1e-3) / 1e12) / bf16_peak}
     if traffic is not None:
@@ -403,7 +410,7 @@ def run_ours(args, rank, world, dist_ctx):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "s8" if method == "int8" else "bf16",
+        "dtype": {"int8": "s8", "int16": "s16"}.get(method, "bf16"),
         "data": "synthetic", "impl": "ours",
         "config": {"workload": args.workload, "method": method, "B": inp.B, "H_k": inp.H_k, "H_v": inp.H_v, "T": inp.T, "C": C, "d_k": inp.d_k,
                    "d_v": inp.d_v, "order": gdn.gdn_default_order(C), "residual_steps": gdn.gdn_default_residual_steps(C),
@@ -587,6 +594,18 @@ def run_extras(gdn, gen, dev, args):
         del inp, q, outs
     except Exception as exc:
         out["prefill_gqa:int8"] = {"error": repr(exc)}
+    # INT16 variant (the paper's primary integer precision) on the prefill shapes: two bytes per element
+    try:
+        inp = gen.make_workload("prefill_gqa", device=dev)
+        q = gen.make_int16_inputs(inp)
+        outs = gdn.chunk_prepare_int16(q)
+        fn = lambda: gdn.chunk_prepare_int16(q, outputs=outs)
+        group = inp.H_v // inp.H_k
+        by = 2 * (inp.C * inp.d_k / group + inp.C * inp.d_v + inp.C * inp.d_k + inp.C * inp.d_v + inp.C * inp.C) + 6 * inp.C
+        out["prefill_gqa:int16"] = _timed_extra(fn, q.n_chunks, by, hbm_peak, 5, 2)
+        del inp, q, outs
+    except Exception as exc:
+        out["prefill_gqa:int16"] = {"error": repr(exc)}
     # the rest of the layer (state passing + output, given the gated W and U) on the prefill and stress shapes; last,
     # because the stress shapes (20 GB, milliseconds per launch) push the GPU into its power cap
     for name in ("prefill_gqa", "stress"):
@@ -651,7 +670,7 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (smaller captures under ncu)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--method", default="neumann", choices=["neumann", "fwdsubst", "fwdsubst-blocked", "int8", "state", "model-native"])
+    ap.add_argument("--method", default="neumann", choices=["neumann", "fwdsubst", "fwdsubst-blocked", "int8", "int16", "state", "model-native"])
     ap.add_argument("--cpu-seconds", type=float, default=20.0)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extras", action="store_true")

@@ -89,6 +89,29 @@ def test_int8_prefill_shapes_at_full_size():
         assert bad.size == 0, f"{key}: {len(bad)} mismatches, first at {bad[0]}"
 
 
+def test_int16_prefill_shapes_at_full_size():
+    from oracle import gdn_oracle_int16 as orq16
+    inp = gen.make_workload("prefill_gqa", device="cuda")
+    q = gen.make_int16_inputs(inp)
+    Wq, Uq, w_exp, u_exp, Toff, t_exp = gdn.chunk_prepare_int16(q)
+    Wq2, Uq2, _, _, Toff2, _ = gdn.chunk_prepare_int16(q)
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+    assert torch.equal(Wq, Wq2) and torch.equal(Uq, Uq2) and torch.equal(Toff, Toff2)
+    ids = _sample_ids(inp, 24, seed=9)
+    Kq, Vq, ke, ve, bq, dq = gen.int8_chunk_slices(q, ids)
+    ref = orq16.chunk_prepare_int16(Kq, Vq, ke, ve, bq, dq, gdn.gdn_default_order(q.C), gdn.gdn_default_residual_steps(q.C))
+    n, C = q.n_chunks, q.C
+    idx = torch.as_tensor(ids, device="cuda")
+    got = {
+        "Wq": Wq.reshape(n, C, q.d_k)[idx].cpu().numpy(), "Uq": Uq.reshape(n, C, q.d_v)[idx].cpu().numpy(),
+        "Toffq": Toff.reshape(n, C, C)[idx].cpu().numpy(), "w_exp": w_exp.reshape(n)[idx].cpu().numpy(),
+        "u_exp": u_exp.reshape(n)[idx].cpu().numpy(), "t_exp": t_exp.reshape(n)[idx].cpu().numpy(),
+    }
+    for key in ("t_exp", "Toffq", "w_exp", "Wq", "u_exp", "Uq"):
+        bad = np.argwhere(got[key] != ref[key])
+        assert bad.size == 0, f"{key}: {len(bad)} mismatches, first at {bad[0]}"
+
+
 @pytest.mark.parametrize("name", ["sweep_c16", "sweep_c64", "sweep_c128", "prefill_gqa"])
 def test_repeated_launches_are_bit_identical(name):
     """The kernels have no atomics on data and a fixed evaluation order per chunk, so repeated launches must agree
