@@ -222,25 +222,14 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
     const uint32_t n_tiles = static_cast<uint32_t>(p.n_tiles);
     const int n_c = p.T / kC;  // chunks per head
 
-    const int t = tid & 127;        // tile row = TMEM lane = row of the K / V tile in shared memory
+    const int t = tid & 127;        // tile row
     const int h = tid >> 7;         // column half
     const int col0 = h * kHC;       // first chunk column of this thread
-    // Rows 32..63 of a chunk carry three quarters of its strictly lower triangle, and a TMEM lane quadrant is tied to a
-    // warp scheduler: with the natural row order the two heavy quadrants of both resident CTAs sit on the same two
-    // schedulers. The second CTA of an SM (told by the base of its TMEM allocation) therefore holds its tiles ROTATED by
-    // 32 rows: tile row t holds token row lt = (t + 32) mod 128, so its heavy quadrants are the other two. Everything
-    // below that speaks of rows and columns of a chunk uses lt; t stays the physical position (TMEM lane, row of the
-    // tiles in shared memory, K index of the block-diagonal operand of W / U).
-    const int rot = ((tmem & 0xFFFFu) >= 256u) ? 32 : 0;
-    const int lt = (t + rot) & 127; // token row of the tile held by this tile row
-    const int il = lt & (kC - 1);   // row inside the chunk
-    const int cb = lt - il;         // first token row of the chunk
-    const int ci = lt >> 6;         // chunk of the tile
-    const int pcol = (cb + col0 - rot) & 127;         // physical position of this thread's 32 columns (tile rows of those tokens)
-    const int pcol_o = ((cb ^ 64) + col0 - rot) & 127;  // the same 32 columns of the other chunk
+    const int il = t & (kC - 1);    // row inside the chunk
+    const int cb = t - il;          // first tile row of the chunk
+    const int ci = t >> 6;          // chunk of the tile
     const int wq = warp & 3;
     const int wrow0 = wq * 32;
-    const int lrow0 = (wrow0 + rot) & 127;  // first token row of this warp's 32 tile rows
     const uint32_t lane_base = tmem + (static_cast<uint32_t>(wq * 32) << 16);
     const uint32_t sK_a = smem_u32(sK), sV_a = smem_u32(sV), sEB_a = smem_u32(sEB);
     const uint32_t idesc_g = instr_desc(128, 128, 1, 1, 0, 0, 2);  // s8 x s8 -> s32, both K-major
@@ -280,24 +269,20 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
         return 32 - __clz(static_cast<int>(all));
     };
 
-    // a tile arrives as four boxes of 32 rows: tile rows [32 b, 32 b + 32) hold the token rows starting at (32 b + rot) mod 128
-    auto load_tile = [&](uint8_t* dst, const CUtensorMap* tm, uint64_t* bar, int t0, int z) {
-        mbar_arrive_expect_tx(bar, 16384);
-#pragma unroll
-        for (int b = 0; b < 4; ++b) tma_load_3d(dst + b * 4096, tm, bar, 0, t0 + ((32 * b + rot) & 127), z);
-    };
     if (tid == 0 && blockIdx.x < n_tiles) {
         const TileCoord c = decode_tile(blockIdx.x, p);
-        load_tile(sK, &tmK, &bar_k, c.t0, c.bhk);
-        load_tile(sV, &tmV, &bar_v, c.t0, c.bhv);
+        mbar_arrive_expect_tx(&bar_k, 16384);
+        tma_load_3d(sK, &tmK, &bar_k, 0, c.t0, c.bhk);
+        mbar_arrive_expect_tx(&bar_v, 16384);
+        tma_load_3d(sV, &tmV, &bar_v, 0, c.t0, c.bhv);
     }
 
     for (uint32_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
         const TileCoord tc = decode_tile(tile, p);
         const uint32_t next = tile + gridDim.x;
         const bool has_next = next < n_tiles;
-        const bool row_valid = (tc.t0 + lt) < p.T;
-        const long long grow = (long long)tc.bhv * p.T + tc.t0 + lt;
+        const bool row_valid = (tc.t0 + t) < p.T;
+        const long long grow = (long long)tc.bhv * p.T + tc.t0 + t;
         const int chunk_in_head = (tc.t0 + cb) / kC;
         const bool chunk_valid = (tc.t0 + cb) < p.T;
 
@@ -334,10 +319,10 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             }
         }
         if (h == 0) {
-            sbeta[lt] = bq;
-            sdecay[lt] = dq;
+            sbeta[t] = bq;
+            sdecay[t] = dq;
 #pragma unroll
-            for (int e = 0; e < 4; ++e) sSH[lt * 4 + e] = 0;
+            for (int e = 0; e < 4; ++e) sSH[t * 4 + e] = 0;
             if (t < 8) {
 #pragma unroll
                 for (int e = 0; e < 4; ++e) sSH[(kTile + t) * 4 + e] = 0;
@@ -354,7 +339,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
         int eA;
         {
             uint32_t g[kHC];
-            tmem_ld32(lane_base + kR0 + pcol, g);  // the Gram matrix is in the tile's physical order
+            tmem_ld32(lane_base + kR0 + cb + col0, g);
             tmem_wait_ld();
             if (dbg_row != nullptr) {
 #pragma unroll
@@ -392,7 +377,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             eA = 2 * kexp - 15 + r;
         }
         // Aq bytes to the private row; entries next to the diagonal and right of this half come back from there
-        uint8_t* rowa = sRowA + lt * 64;
+        uint8_t* rowa = sRowA + t * 64;
         {
             uint4 v0, v1;
             v0.x = pack4(aq[0], aq[1], aq[2], aq[3]);     v0.y = pack4(aq[4], aq[5], aq[6], aq[7]);
@@ -416,9 +401,9 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
         // P_1 = band of Aq: zero beyond distance N
         const int p11 = ab1, p12 = (N >= 2) ? ab2 : 0, p13 = (N >= 3) ? ab3 : 0;
         if (h == 0) {
-            sAB[lt * 8 + 1] = p11;
-            sAB[lt * 8 + 2] = p12;
-            sAB[lt * 8 + 3] = p13;
+            sAB[t * 8 + 1] = p11;
+            sAB[t * 8 + 2] = p12;
+            sAB[t * 8 + 3] = p13;
         }
         cta_barrier();
 
@@ -426,7 +411,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
         int t0q1 = 0, t0q2 = 0, t0q3 = 0;  // T0q[i][i-1..i-3]
         int eT0;
         {
-            const int r1 = (lt - 1) > 0 ? (lt - 1) : 0, r2 = (lt - 2) > 0 ? (lt - 2) : 0;
+            const int r1 = (t - 1) > 0 ? (t - 1) : 0, r2 = (t - 2) > 0 ? (t - 2) : 0;
             // P_2 on distances 2..N: sum over the intermediate row
             int acc22 = (N >= 2) ? p11 * sAB[r1 * 8 + 1] : 0;
             int acc23 = (N >= 3) ? p11 * sAB[r1 * 8 + 2] + p12 * sAB[r2 * 8 + 1] : 0;
@@ -465,9 +450,9 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             t0q3 = q8_32(a3, r);
             eT0 = eref + r;
             if (h == 0) {
-                if (il >= 1) sSH[(lt - 1) * 4 + 0] = t0q1;
-                if (il >= 2) sSH[(lt - 2) * 4 + 1] = t0q2;
-                if (il >= 3) sSH[(lt - 3) * 4 + 2] = t0q3;
+                if (il >= 1) sSH[(t - 1) * 4 + 0] = t0q1;
+                if (il >= 2) sSH[(t - 2) * 4 + 1] = t0q2;
+                if (il >= 3) sSH[(t - 3) * 4 + 2] = t0q3;
             }
             cta_barrier();
         }
@@ -628,7 +613,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             for (int jl = 0; jl < kHC; ++jl) prod[jl] = 0;
 #pragma unroll
             for (int e = 1; e <= 3; ++e) {
-                const int rr = (lt - e) > 0 ? (lt - e) : 0;
+                const int rr = (t - e) > 0 ? (t - e) : 0;
                 const int cf = (il - e >= 0) ? (e == 1 ? t0q1 : (e == 2 ? t0q2 : t0q3)) : 0;
                 const uint4 a0 = *reinterpret_cast<const uint4*>(sRowA + rr * 64 + col0);
                 const uint4 a1 = *reinterpret_cast<const uint4*>(sRowA + rr * 64 + col0 + 16);
@@ -682,12 +667,11 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             for (int w = 0; w < 8; ++w)
                 r8[w] = q8_pack4(acc[4 * w], acc[4 * w + 1], acc[4 * w + 2], acc[4 * w + 3], rq9);
             eTb = eT - 15 + r;
-            // the K index of this operand is the tile row of the key / value token: this thread's 32 columns sit at
-            // packed columns [pcol/4, pcol/4 + 8) of the 32-column operand; the same columns of the other chunk are zero
-            tmem_st8(lane_base + kAS + pcol / 4, r8);
+            // row t's block occupies packed columns [cb/4, cb/4 + 16) of a 32-column operand; the other 16 are zero
+            tmem_st8(lane_base + kAS + cb / 4 + h * 8, r8);
 #pragma unroll
             for (int w = 0; w < 8; ++w) r8[w] = 0u;
-            tmem_st8(lane_base + kAS + pcol_o / 4, r8);
+            tmem_st8(lane_base + kAS + (16 - cb / 4) + h * 8, r8);
             tmem_wait_st();
         }
         // Toffq row -> staging (64-byte lines, 64-byte TMA swizzle) -> bulk tensor store of 32 rows per warp (h = 0 issues)
@@ -709,7 +693,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
         tc_fence_before_sync();
         cta_barrier();
         if (p.Toff != nullptr && h == 0 && lane == 0) {
-            tma_store_3d(&tmT, stage + wrow0 * 64, 0, tc.t0 + lrow0, tc.bhv);
+            tma_store_3d(&tmT, stage + wrow0 * 64, 0, tc.t0 + wrow0, tc.bhv);
             tma_store_commit();
         }
         if (tid == 0) {
@@ -774,10 +758,13 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             // read the tile are complete: the next tile's K (V) may land
             if (tid == 0 && has_next) {
                 const TileCoord nc = decode_tile(next, p);
-                if (half == 0)
-                    load_tile(sK, &tmK, &bar_k, nc.t0, nc.bhk);
-                else
-                    load_tile(sV, &tmV, &bar_v, nc.t0, nc.bhv);
+                if (half == 0) {
+                    mbar_arrive_expect_tx(&bar_k, 16384);
+                    tma_load_3d(sK, &tmK, &bar_k, 0, nc.t0, nc.bhk);
+                } else {
+                    mbar_arrive_expect_tx(&bar_v, 16384);
+                    tma_load_3d(sV, &tmV, &bar_v, 0, nc.t0, nc.bhv);
+                }
             }
             if (row_valid && il == 0 && h == 0)
                 ((half == 0) ? p.w_exp : p.u_exp)[(long long)tc.bhv * n_c + chunk_in_head] = eref + rr;
@@ -821,7 +808,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) {
-                tma_store_3d((half == 0) ? &tmW : &tmU, sub, h * 64, tc.t0 + lrow0, tc.bhv);
+                tma_store_3d((half == 0) ? &tmW : &tmU, sub, h * 64, tc.t0 + wrow0, tc.bhv);
                 tma_store_commit();
             }
         }
@@ -886,8 +873,8 @@ int launch_tc_int8(const ProblemI8& q, cudaStream_t stream) {
     if (status == nullptr) return GDN_ERR_LAUNCH;
     const long long hk = (long long)q.B * q.H_k, hv = (long long)q.B * q.H_v;
     CUtensorMap mK, mV, mW, mU, mT;
-    if (!make_map(&mK, q.Kq, hk, q.T, kD, 128, 32, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
-    if (!make_map(&mV, q.Vq, hv, q.T, kD, 128, 32, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
+    if (!make_map(&mK, q.Kq, hk, q.T, kD, 128, 128, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
+    if (!make_map(&mV, q.Vq, hv, q.T, kD, 128, 128, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
     if (!make_map(&mW, q.Wq, hv, q.T, kD, 64, 32, CU_TENSOR_MAP_SWIZZLE_64B)) return GDN_ERR_LAUNCH;
     if (!make_map(&mU, q.Uq, hv, q.T, kD, 64, 32, CU_TENSOR_MAP_SWIZZLE_64B)) return GDN_ERR_LAUNCH;
     if (!make_map(&mT, q.Toff != nullptr ? q.Toff : q.Wq, hv, q.T, q.Toff != nullptr ? kC : kD, 64, 32, CU_TENSOR_MAP_SWIZZLE_64B))
