@@ -326,7 +326,8 @@ def run_ours(args, rank, world, dist_ctx):
             gdn.chunk_state_output(st_args[0], inp.K, st_args[1], st_args[2], inp.g, C, inp.d_k ** -0.5, outputs=st_args[3])
         else:
             gdn.chunk_prepare(inp.K, inp.V, inp.beta, inp.g, C, outputs=outs, method="fwdsubst",
-                              variant=gdn.GDN_FWDSUBST_BLOCKED if method == "fwdsubst-blocked" else gdn.GDN_FWDSUBST_ROWS)
+                              variant={"fwdsubst-blocked": gdn.GDN_FWDSUBST_BLOCKED,
+                                       "fwdsubst-tc": gdn.GDN_FWDSUBST_BLOCKED_TC}.get(method, gdn.GDN_FWDSUBST_ROWS))
 
     sampler = ClockSampler(torch.cuda.current_device())
     # W warm-up steps as asked, and never less than ~0.1 s of untimed launches: the first launches after the idle time
@@ -525,7 +526,8 @@ def run_extras(gdn, gen, dev, args):
             ("sweep_c64", "neumann-s15"),
             ("sweep_c16", "fwdsubst"), ("sweep_c32", "fwdsubst"), ("sweep_c64", "fwdsubst"), ("sweep_c128", "fwdsubst"),
             ("sweep_c16", "fwdsubst-blocked"), ("sweep_c32", "fwdsubst-blocked"), ("sweep_c64", "fwdsubst-blocked"),
-            ("sweep_c128", "fwdsubst-blocked"), ("prefill_gqa", "neumann"), ("prefill_gqa", "fwdsubst")]
+            ("sweep_c128", "fwdsubst-blocked"), ("sweep_c64", "fwdsubst-tc"), ("prefill_gqa", "neumann"), ("prefill_gqa", "fwdsubst"),
+            ("prefill_gqa", "fwdsubst-tc")]
     if args.workload != "stress":
         plan.append(("stress", "neumann"))
     for name, method in plan:
@@ -533,7 +535,7 @@ def run_extras(gdn, gen, dev, args):
             inp = gen.make_workload(name, device=dev)
             outs = gdn.alloc_outputs(inp.K, inp.V, inp.C)
             meth, var = (method.split("-") + ["rows"])[:2]
-            variant = gdn.GDN_FWDSUBST_BLOCKED if var == "blocked" else gdn.GDN_FWDSUBST_ROWS
+            variant = {"blocked": gdn.GDN_FWDSUBST_BLOCKED, "tc": gdn.GDN_FWDSUBST_BLOCKED_TC}.get(var, gdn.GDN_FWDSUBST_ROWS)
             # "neumann-s15": all 15 residual terms (the exact inverse at N = 3, C = 64) by the doubling scheme
             n_ord, n_res = (3, 15) if var == "s15" else (-1, -1)
             fn = lambda: gdn.chunk_prepare(inp.K, inp.V, inp.beta, inp.g, inp.C, n_ord, n_res, outputs=outs, method=meth,
@@ -547,7 +549,8 @@ def run_extras(gdn, gen, dev, args):
     for c in (16, 32, 64, 128):
         try:
             neu = out[f"sweep_c{c}:neumann"]["ms"]
-            sub = min(out[f"sweep_c{c}:{m}"]["ms"] for m in ("fwdsubst", "fwdsubst-blocked") if "ms" in out.get(f"sweep_c{c}:{m}", {}))
+            sub = min(out[f"sweep_c{c}:{m}"]["ms"] for m in ("fwdsubst", "fwdsubst-blocked", "fwdsubst-tc")
+                      if "ms" in out.get(f"sweep_c{c}:{m}", {}))
             out[f"sweep_c{c}:neumann_speedup_over_best_substitution"] = sub / neu
         except Exception:
             pass
@@ -672,7 +675,7 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (smaller captures under ncu)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--method", default="neumann", choices=["neumann", "fwdsubst", "fwdsubst-blocked", "int8", "int16", "state", "model-native"])
+    ap.add_argument("--method", default="neumann", choices=["neumann", "fwdsubst", "fwdsubst-blocked", "fwdsubst-tc", "int8", "int16", "state", "model-native"])
     ap.add_argument("--cpu-seconds", type=float, default=20.0)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extras", action="store_true")

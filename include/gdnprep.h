@@ -79,7 +79,7 @@ enum {
 };
 
 /* variants of the forward-substitution comparison kernel */
-enum { GDN_FWDSUBST_ROWS = 0, GDN_FWDSUBST_BLOCKED = 1 };
+enum { GDN_FWDSUBST_ROWS = 0, GDN_FWDSUBST_BLOCKED = 1, GDN_FWDSUBST_BLOCKED_TC = 2 };
 
 /* A CUDA stream handle (cudaStream_t) passed as an opaque pointer. */
 typedef void* gdn_stream_t;
@@ -120,7 +120,9 @@ int gdn_chunk_prepare_ex(const void* K, const void* V, const float* beta, const 
  * The comparison the paper's speed-up is measured against: the same A-build, W
  * and U, with T computed exactly by forward substitution (Eq. 2-3;
  * variant GDN_FWDSUBST_ROWS) or by 16 x 16 diagonal blocks merged with the
- * block recursion of App. E (Eq. 25-27; variant GDN_FWDSUBST_BLOCKED). Same dtypes, sizes and layouts as
+ * block recursion of App. E (Eq. 25-27; variant GDN_FWDSUBST_BLOCKED), or by the two 32 x 32 diagonal blocks of a
+ * 64-chunk with the lower-left block from the block formula (Eq. 28) evaluated on the tensor cores (variant
+ * GDN_FWDSUBST_BLOCKED_TC: bf16, C = 64 only). Same dtypes, sizes and layouts as
  * gdn_chunk_prepare_gqa. For C = 128 on the bf16 path both variants invert the two 64 x 64 diagonal blocks by
  * their substitution and obtain the lower-left block from the block formula of App. E (Eq. 28), as the Neumann
  * path does.

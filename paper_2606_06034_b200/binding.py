@@ -33,6 +33,7 @@ GDN_FLAG_LAYOUT_BTHD = 8
 GDN_FLAG_W_GATED = 16
 GDN_FWDSUBST_ROWS = 0
 GDN_FWDSUBST_BLOCKED = 1
+GDN_FWDSUBST_BLOCKED_TC = 2
 
 EXPORTS = (
     "gdn_chunk_prepare", "gdn_chunk_prepare_gqa", "gdn_chunk_prepare_ex", "gdn_chunk_prepare_varlen",

@@ -821,6 +821,161 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         } else {
             // ---- forward substitution (Eq. 2-3). The private fp32 rows hold Abar; thread (h = 0, t) solves
             // column il of its chunk, which has no dependence on other columns.
+            if constexpr (MODE == INV_FWDSUBST_TC) {
+                // Blocked form with the block merge on the tensor cores (App. E, Eq. 28 inside every 64-chunk): the two
+                // 32 x 32 diagonal blocks by substitution (32 sequential rows instead of 64, 128 column threads), then
+                // T21 = T22 Abar21 T11 (Abar = -A) as Y = Abar21 + Abar21 X11, T21 = Y + X22 Y with X = T - I: two products with hi + lo
+                // bf16 operands (they cancel on correlated keys, as in the C = 128 merge), identity parts in fp32, all 256
+                // threads taking part in the operand work. M = 128, N = 64, K = 32: rows 32..63 of both chunks are the
+                // A operands, [X11 of chunk 0 | X11 of chunk 1] (then Y) the B operand.
+                static_assert(C == 64 && !MERGE, "built for 64-chunks");
+                const int b0 = il >> 5;        // diagonal block of this row / column (uniform per warp)
+                const int ci2 = t >> 6;        // chunk of the tile
+                if (h == 0) {
+                    float xcol[32];  // xcol[r] = T[32 b0 + r][il]
+#pragma unroll
+                    for (int r = 0; r < 32; ++r) {
+                        const int i = 32 * b0 + r;
+                        float acc = 0.f;
+                        const uint32_t ri = scratch_a + (cb + i) * (4 * C);
+#pragma unroll
+                        for (int q4 = 0; q4 < (r + 3) / 4; ++q4) {
+                            const uint4 q = lds128(ri + (swz<CPRF>(i, 8 * b0 + q4) << 4));
+                            if (q4 * 4 + 0 < r) acc = fmaf(__uint_as_float(q.x), xcol[q4 * 4 + 0], acc);
+                            if (q4 * 4 + 1 < r) acc = fmaf(__uint_as_float(q.y), xcol[(q4 * 4 + 1 < 32) ? q4 * 4 + 1 : 0], acc);
+                            if (q4 * 4 + 2 < r) acc = fmaf(__uint_as_float(q.z), xcol[(q4 * 4 + 2 < 32) ? q4 * 4 + 2 : 0], acc);
+                            if (q4 * 4 + 3 < r) acc = fmaf(__uint_as_float(q.w), xcol[(q4 * 4 + 3 < 32) ? q4 * 4 + 3 : 0], acc);
+                        }
+                        xcol[r] = (i > il) ? acc : ((i == il) ? 1.f : 0.f);
+                    }
+                    compute_barrier();  // everyone has read Abar of the diagonal blocks
+#pragma unroll
+                    for (int r = 0; r < 32; ++r) {
+                        const int i = 32 * b0 + r;
+                        const uint32_t addr = scratch_a + (cb + i) * (4 * C) + (swz<CPRF>(i, il >> 2) << 4) + (il & 3) * 4;
+                        asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(xcol[r]) : "memory");
+                    }
+                    if (b0 == 1) {
+                        // rows above the second block: zeros (the entries above the diagonal were never masked)
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            const uint32_t addr = scratch_a + (cb + i) * (4 * C) + (swz<CPRF>(i, il >> 2) << 4) + (il & 3) * 4;
+                            asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(0.f) : "memory");
+                        }
+                    }
+                } else {
+                    compute_barrier();
+                }
+                compute_barrier();
+                // every thread takes its half row: T11 / zeros (first block), Abar21 / T22 (second block)
+#pragma unroll
+                for (int c = 0; c < CPTF; ++c) {
+                    const uint4 q = lds128(rowf + (swz<CPRF>(t, (col0 >> 2) + c) << 4));
+                    a[c * 4 + 0] = __uint_as_float(q.x);
+                    a[c * 4 + 1] = __uint_as_float(q.y);
+                    a[c * 4 + 2] = __uint_as_float(q.z);
+                    a[c * 4 + 3] = __uint_as_float(q.w);
+                }
+                compute_barrier();  // the fp32 rows are dead: the B operands overlay them
+                const uint32_t idesc_t = instr_desc(128, 64, 1, 1, 0, 1, 1);
+                // one B piece = 8 columns of one row (16 bytes) at n8 * 512 + k * 16, hi plane at 0, lo plane at 4 KB
+                auto store_b = [&](int krow) {
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t wh[4], wl[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const float v0 = a[8 * c + 2 * i], v1 = a[8 * c + 2 * i + 1];
+                            wh[i] = pack_bf16x2(v0, v1);
+                            wl[i] = pack_bf16x2(v0 - bf16_lo(wh[i]), v1 - bf16_hi(wh[i]));
+                        }
+                        const uint32_t off = (4 * ci2 + c) * 512 + krow * 16;
+                        *reinterpret_cast<uint4*>(sEB + off) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
+                        *reinterpret_cast<uint4*>(sEB + 4096 + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
+                    }
+                };
+                auto store_a = [&](uint32_t slot_cols) {
+                    uint32_t ph[16], pl[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        ph[i] = pack_bf16x2(a[2 * i], a[2 * i + 1]);
+                        pl[i] = pack_bf16x2(a[2 * i] - bf16_lo(ph[i]), a[2 * i + 1] - bf16_hi(ph[i]));
+                    }
+                    tmem_st16(lane_base + slot_cols, ph);
+                    tmem_st16(lane_base + slot_cols + 16, pl);
+                };
+                auto issue = [&](uint32_t slot_cols) {
+                    if (warp == 0) {
+                        tc_fence_after_sync();
+                        if (elect_one()) {
+#pragma unroll
+                            for (int part = 0; part < 3; ++part) {
+                                // hi*hi, lo*hi, hi*lo
+#pragma unroll
+                                for (int ks = 0; ks < 2; ++ks) {
+                                    const uint64_t bd = smem_desc(sEB_a + (part == 2 ? 4096 : 0) + ks * 256, 128, 512, SWZ_NONE);
+                                    mma_f16_ts(tmem + kR0, tmem + slot_cols + (part == 1 ? 16 : 0) + ks * 8, bd, idesc_t, part > 0 || ks > 0);
+                                }
+                            }
+                            mma_commit(&bar_mma);
+                        }
+                    }
+                };
+                if (b0 == 0) {
+                    if (h == 0) {
+                        // X11 = T11 - I: the B operand of the first product
+#pragma unroll
+                        for (int jl = 0; jl < HC; ++jl) a[jl] -= (jl == il) ? 1.f : 0.f;
+                        store_b(il);
+#pragma unroll
+                        for (int jl = 0; jl < HC; ++jl) a[jl] += (jl == il) ? 1.f : 0.f;
+                    }
+                } else if (h == 0) {
+                    store_a(kAS);  // Abar21 (hi, lo): A operand of the first product
+                } else {
+                    // X22 = T22 - I (hi, lo): A operand of the second product
+#pragma unroll
+                    for (int jl = 0; jl < HC; ++jl) a[jl] -= (col0 + jl == il) ? 1.f : 0.f;
+                    store_a(kR2);
+#pragma unroll
+                    for (int jl = 0; jl < HC; ++jl) a[jl] += (col0 + jl == il) ? 1.f : 0.f;
+                }
+                tmem_wait_st();
+                fence_proxy_async_smem();
+                tc_fence_before_sync();
+                compute_barrier();
+                issue(kAS);
+                if (!wait_mma()) { ok = false; break; }
+                tc_fence_after_sync();
+                if (b0 == 1 && h == 0) {
+                    // Y = Abar21 + Abar21 X11: the B operand of the second product
+                    uint32_t d[32];
+                    tmem_ld32(lane_base + kR0 + 32 * ci2, d);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int jl = 0; jl < HC; ++jl) a[jl] += __uint_as_float(d[jl]);
+                    store_b(il - 32);
+                }
+                fence_proxy_async_smem();
+                tc_fence_before_sync();
+                compute_barrier();
+                issue(kR2);
+                if (!wait_mma()) { ok = false; break; }
+                tc_fence_after_sync();
+                if (b0 == 1 && h == 0) {
+                    // T21 = Y + X22 Y
+                    uint32_t d[32];
+                    tmem_ld32(lane_base + kR0 + 32 * ci2, d);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int jl = 0; jl < HC; ++jl) a[jl] += __uint_as_float(d[jl]);
+                }
+                // the finished rows go back to the fp32 lines (the operand planes overlaid some of them)
+#pragma unroll
+                for (int c = 0; c < CPTF; ++c)
+                    sts128(rowf + (swz<CPRF>(t, (col0 >> 2) + c) << 4), __float_as_uint(a[c * 4 + 0]), __float_as_uint(a[c * 4 + 1]),
+                           __float_as_uint(a[c * 4 + 2]), __float_as_uint(a[c * 4 + 3]));
+            } else {
             if (h == 0) {
                 float xcol[C];  // xcol[k] = T[k][il]
                 if constexpr (MODE == INV_FWDSUBST_BLOCKED) {
@@ -899,6 +1054,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             } else {
                 if constexpr (MODE == INV_FWDSUBST_BLOCKED) compute_barrier();
                 compute_barrier();
+            }
             }
             compute_barrier();
             // back to rows: a[] = far part of this thread's columns, lb[] = band part
@@ -1644,6 +1800,10 @@ int launch_tc_bf16(const Problem& p, InverseMode mode, cudaStream_t stream) {
             case 128: return launch_c<64, INV_NEUMANN, true>(m, prm, stream);
             default: return launch_c<64, INV_NEUMANN>(m, prm, stream);
         }
+    }
+    if (mode == INV_FWDSUBST_TC) {
+        if (p.C != 64) return GDN_ERR_UNSUPPORTED;
+        return launch_c<64, INV_FWDSUBST_TC>(m, prm, stream);
     }
     if (mode == INV_FWDSUBST_BLOCKED) {
         switch (p.C) {

@@ -90,7 +90,7 @@ struct ProblemS {
     const int* seq_no_u = nullptr;
 };
 
-enum InverseMode { INV_NEUMANN = 0, INV_FWDSUBST_ROWS = 1, INV_FWDSUBST_BLOCKED = 2 };
+enum InverseMode { INV_NEUMANN = 0, INV_FWDSUBST_ROWS = 1, INV_FWDSUBST_BLOCKED = 2, INV_FWDSUBST_TC = 3 };
 
 // Status word written by kernels (one per device, static device memory).
 int* device_status_word();  // device address for the current device (nullptr on failure)

@@ -151,9 +151,16 @@ int gdn_chunk_prepare_varlen(const void* K, const void* V, const float* beta, co
 int gdn_chunk_prepare_fwdsubst(const void* K, const void* V, const float* beta, const float* g, int B, int H_k, int H_v, int T,
                                int C, int d_k, int d_v, int dtype, int variant, void* W_out, void* U_out, void* Tinv_out,
                                gdn_stream_t stream) {
-    if (variant != GDN_FWDSUBST_ROWS && variant != GDN_FWDSUBST_BLOCKED) return GDN_ERR_INVALID_ARG;
+    if (variant != GDN_FWDSUBST_ROWS && variant != GDN_FWDSUBST_BLOCKED && variant != GDN_FWDSUBST_BLOCKED_TC)
+        return GDN_ERR_INVALID_ARG;
     Problem p{K, V, beta, g, W_out, U_out, Tinv_out, B, H_k, H_v, T, C, d_k, d_v, 0, 0, dtype};
-    return run(p, variant == GDN_FWDSUBST_ROWS ? INV_FWDSUBST_ROWS : INV_FWDSUBST_BLOCKED, static_cast<cudaStream_t>(stream));
+    if (variant == GDN_FWDSUBST_BLOCKED_TC && (dtype != GDN_DTYPE_BF16 || C != 64)) {
+        const int rc = validate(p, false);
+        return rc != GDN_OK ? rc : GDN_ERR_UNSUPPORTED;
+    }
+    const InverseMode mode = variant == GDN_FWDSUBST_ROWS ? INV_FWDSUBST_ROWS
+                             : variant == GDN_FWDSUBST_BLOCKED ? INV_FWDSUBST_BLOCKED : INV_FWDSUBST_TC;
+    return run(p, mode, static_cast<cudaStream_t>(stream));
 }
 
 int gdn_chunk_prepare_int8(const int8_t* Kq, const int8_t* Vq, const int32_t* k_exp, const int32_t* v_exp, const uint16_t* beta_q,

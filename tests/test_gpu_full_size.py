@@ -69,6 +69,25 @@ def test_bf16_workload_at_full_size(name):
         assert np.all(err <= bound), f"{name} {label}: rel-F {err[worst]:.3e} > {bound[worst]:.3e} at chunk {ids[worst]}"
 
 
+def test_tensor_core_blocked_substitution_at_full_size():
+    """The strongest comparator (32-blocks by substitution, block merge on the tensor cores) on the stress shapes with
+    one batch entry (32 768 chunks, half the heads adversarial): sampled chunks against the exact inverse."""
+    inp = gen.make_workload("stress", device="cuda", B=1)
+    W, U, Tinv = gdn.chunk_prepare(inp.K, inp.V, inp.beta, inp.g, inp.C, method="fwdsubst", variant=gdn.GDN_FWDSUBST_BLOCKED_TC)
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+    C, n = inp.C, inp.n_chunks
+    ids = _sample_ids(inp, 40, seed=12)
+    sl = gen.chunk_slices(inp, ids)
+    Wo, Uo, To = orc.chunk_prepare(*[np.stack([s[i] for s in sl]) for i in range(4)], exact=True)
+    idx = torch.as_tensor(ids, device="cuda")
+    for label, got, ref in (("Tinv", Tinv.reshape(n, C, C)[idx], To), ("W", W.reshape(n, C, inp.d_k)[idx], Wo),
+                            ("U", U.reshape(n, C, inp.d_v)[idx], Uo)):
+        err = orc.rel_frobenius(got.double().cpu().numpy(), ref)
+        floor = orc.rel_frobenius(_bf16_round(ref), ref)
+        bound = np.where(floor > 0.9 * TOL_BF16, np.maximum(TOL_BF16, floor + 2e-4), TOL_BF16)
+        assert np.all(err <= bound), f"{label}: {err.max():.3e}"
+
+
 def test_int8_prefill_shapes_at_full_size():
     inp = gen.make_workload("prefill_gqa", device="cuda")
     q = gen.make_int8_inputs(inp)

@@ -241,6 +241,31 @@ def test_bf16_blocked_forward_substitution_kernel(C):
     assert (Tinv.float() - Tinv2.float()).abs().max() <= 1e-2
 
 
+@pytest.mark.parametrize("adv", ["none", "odd", "all"])
+def test_bf16_blocked_forward_substitution_with_tensor_core_merge(adv):
+    """32 x 32 diagonal blocks by substitution, lower-left block by the block formula of App. E on the tensor cores
+    (hi + lo operands): the exact inverse, at the bf16 floor also on strongly correlated keys; several tiles, grouped
+    heads and a ragged last tile."""
+    inp = gen.make_inputs(2, 2, 4, 448, 64, 128, 128, seed=180, adversarial_heads=adv)
+    K, V, beta, g = _to_dev(inp)
+    W, U, Tinv = gdn.chunk_prepare(K, V, beta, g, 64, method="fwdsubst", variant=gdn.GDN_FWDSUBST_BLOCKED_TC)
+    W2, U2, Tinv2 = gdn.chunk_prepare(K, V, beta, g, 64, method="fwdsubst", variant=gdn.GDN_FWDSUBST_BLOCKED_TC)
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+    assert torch.equal(W, W2) and torch.equal(U, U2) and torch.equal(Tinv, Tinv2)
+    Wg, Ug, Tg = _gpu_chunks(W, U, Tinv, inp)
+    Wo, Uo, To = _oracle(inp, exact=True)
+    for name, got, ref in (("Tinv", Tg, To), ("W", Wg, Wo), ("U", Ug, Uo)):
+        err = orc.rel_frobenius(got, ref)
+        bound = _bound(ref, TOL_BF16)
+        worst = int(np.argmax(err - bound))
+        assert np.all(err <= bound), f"{name} rel-F {err[worst]:.3e} > {bound[worst]:.3e} at chunk {worst}"
+    assert np.all(np.triu(Tg, 1) == 0) and np.all(np.diagonal(Tg, axis1=-2, axis2=-1) == 1)
+    # other chunk sizes are refused
+    rc = gdn.gdn_chunk_prepare_fwdsubst(K, V, beta, g, inp.B, inp.H_k, inp.H_v, inp.T, 32, 128, 128, gdn.GDN_DTYPE_BF16,
+                                        gdn.GDN_FWDSUBST_BLOCKED_TC, W, U, Tinv, check=False)
+    assert rc == gdn.GDN_ERR_UNSUPPORTED
+
+
 @pytest.mark.parametrize("C", [16, 32, 64, 128])
 def test_fp32_blocked_forward_substitution(C):
     inp = gen.make_inputs(1, 1, 2, 2 * C, C, 64, 64, seed=95 + C, dtype=torch.float32)
