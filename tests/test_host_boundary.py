@@ -43,7 +43,7 @@ def test_int8_decay_table_matches_the_oracle(lib):
 
 
 def test_status_strings(lib):
-    for code in range(0, -8, -1):
+    for code in range(0, -9, -1):
         assert lib.gdn_status_string(code)
     assert gdn.status_string(gdn.GDN_ERR_TIMEOUT).startswith("bounded wait")
 
@@ -94,6 +94,33 @@ def test_bad_arguments_are_rejected_without_a_device(lib):
     assert seg(T=100) == gdn.GDN_ERR_INVALID_ARG
     assert seg(flags=gdn.GDN_FLAG_W_GATED) == gdn.GDN_ERR_INVALID_ARG
     assert seg(ws=mis) == gdn.GDN_ERR_ALIGN
+    # the variant of the segmented call on built-in scratch: same checks, no workspace argument
+    na = lambda **kw: lib.gdn_chunk_state_output_segmented_noalloc(*[kw.get(k, d) for k, d in (
+        ("Q", p), ("K", p), ("W", p), ("U", p), ("g", p), ("Hk", 1), ("Hv", 1), ("T", 256), ("C", 64), ("dk", 128), ("dv", 128),
+        ("scale", ctypes.c_float(1.0)), ("S_in", None), ("O", p), ("S_out", None), ("segments", 2), ("flags", 0), ("stream", None))])
+    assert na(Q=None) == gdn.GDN_ERR_NULL
+    assert na(segments=0) == gdn.GDN_ERR_INVALID_ARG
+    assert na(T=100) == gdn.GDN_ERR_INVALID_ARG
+    assert na(flags=gdn.GDN_FLAG_W_GATED) == gdn.GDN_ERR_INVALID_ARG
+    assert na(O=mis) == gdn.GDN_ERR_ALIGN
+    # the integer entry points
+    i8 = lambda fn, **kw: fn(*[kw.get(k, d) for k, d in (
+        ("Kq", p), ("Vq", p), ("ke", p), ("ve", p), ("bq", p), ("dq", p), ("B", 1), ("Hk", 1), ("Hv", 1), ("T", 128), ("C", 64),
+        ("dk", 128), ("dv", 128), ("N", -1), ("S", -1), ("Wq", p), ("Uq", p), ("we", p), ("ue", p), ("Toff", p), ("te", p),
+        ("dbg", None), ("stream", None))])
+    for fn in (lib.gdn_chunk_prepare_int8, lib.gdn_chunk_prepare_int16):
+        assert i8(fn, Kq=None) == gdn.GDN_ERR_NULL
+        assert i8(fn, te=None) == gdn.GDN_ERR_NULL
+        assert i8(fn, T=100) == gdn.GDN_ERR_INVALID_ARG
+        assert i8(fn, Hk=2, Hv=3) == gdn.GDN_ERR_INVALID_ARG
+        assert i8(fn, N=0) == gdn.GDN_ERR_INVALID_ARG
+        assert i8(fn, S=-2) == gdn.GDN_ERR_INVALID_ARG
+        assert i8(fn, Wq=mis) == gdn.GDN_ERR_ALIGN
+        assert i8(fn, dbg=mis) == gdn.GDN_ERR_ALIGN
+    assert lib.gdn_chunk_prepare_fwdsubst(p, p, p, p, 1, 1, 1, 128, 32, 128, 128, 1, gdn.GDN_FWDSUBST_BLOCKED_TC, p, p, p, None) in (
+        gdn.GDN_ERR_UNSUPPORTED,)
+    assert lib.gdn_chunk_prepare_fwdsubst(p, p, p, p, 1, 1, 1, 128, 64, 128, 128, 0, gdn.GDN_FWDSUBST_BLOCKED_TC, p, p, p, None) == \
+        gdn.GDN_ERR_UNSUPPORTED  # bf16 only
     # valid arguments but no sm_100 device in this process: refused, nothing launched
     import torch
     if not torch.cuda.is_available():
