@@ -484,38 +484,39 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             for (int jl = 0; jl < kHC; ++jl) eq[jl] = q8_32(acc[jl], rq);
             eE = eref + r;
         }
-        // packed rows of the powers R_s (R_1 = Eq) and their exponents
-        uint32_t rpk[kSMax][kHC / 4];
+        // Rows of the powers R_s (R_1 = Eq) as packed bytes. The loops over the powers are NOT unrolled (the kernel is bound
+        // by instruction fetch: its straight-line code is larger than the instruction cache), so the rows cannot sit in
+        // registers indexed by s: R_1 stays in registers, R_2.. are parked in free TMEM columns of the row's own lane
+        // (columns 160..255 for s = 2..7; s = 8 and, for the sum, R_1 go to accumulator columns that are idle by then).
+        uint32_t r1[kHC / 4];   // R_1
+        uint32_t cur[kHC / 4];  // R_{s-1} inside the loop
         int er[kSMax];
 #pragma unroll
-        for (int s = 0; s < kSMax; ++s) {
-            er[s] = 0;
+        for (int s = 0; s < kSMax; ++s) er[s] = 0;
 #pragma unroll
-            for (int w = 0; w < kHC / 4; ++w) rpk[s][w] = 0u;
-        }
+        for (int w = 0; w < kHC / 4; ++w) r1[w] = cur[w] = 0u;
+        auto park_col = [&](int s) -> uint32_t {  // TMEM column of the parked row of R_s (s >= 1)
+            return (s >= 2 && s <= 7) ? static_cast<uint32_t>(160 + (s - 2) * 16 + h * 8)
+                                      : static_cast<uint32_t>(kR0 + (s == 1 ? 0 : 16) + h * 8);
+        };
         int n_terms = 0;
         if (S >= 1) {
 #pragma unroll
-            for (int w = 0; w < kHC / 4; ++w) rpk[0][w] = pack4(eq[4 * w], eq[4 * w + 1], eq[4 * w + 2], eq[4 * w + 3]);
+            for (int w = 0; w < kHC / 4; ++w) r1[w] = cur[w] = pack4(eq[4 * w], eq[4 * w + 1], eq[4 * w + 2], eq[4 * w + 3]);
             er[0] = eE;
             n_terms = 1;
             // B operand [E_1 | E_2] (64 x 128 int8, MN-major, no swizzle): 16 columns of chunk-row il per 16-byte piece
 #pragma unroll
             for (int c = 0; c < kHC / 16; ++c) {
-                const uint4 v = make_uint4(rpk[0][4 * c], rpk[0][4 * c + 1], rpk[0][4 * c + 2], rpk[0][4 * c + 3]);
+                const uint4 v = make_uint4(r1[4 * c], r1[4 * c + 1], r1[4 * c + 2], r1[4 * c + 3]);
                 *reinterpret_cast<uint4*>(sEB + (((cb + col0) >> 4) + c) * (16 * kC) + il * 16) = v;
             }
         }
         // ---- I7: R_s = Q8(R_{s-1} Eq) while s (N+1) < C
-#pragma unroll
+#pragma unroll 1
         for (int s = 2; s <= kSMax; ++s) {
             if (s > S || s * (N + 1) >= kC) break;
-            {
-                uint32_t r8[8];
-#pragma unroll
-                for (int w = 0; w < 8; ++w) r8[w] = rpk[s - 2][w];
-                tmem_st8(lane_base + kAS + h * 8, r8);
-            }
+            tmem_st8(lane_base + kAS + h * 8, cur);
             fence_proxy_async_smem();
             tmem_wait_st();
             tc_fence_before_sync();
@@ -543,12 +544,13 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             // for i - j < s (N + 1), no mask needed
 #pragma unroll
             for (int jl = 0; jl < kHC; ++jl) m |= abs32(static_cast<int>(dres[jl]));
-            const int r = q8_shift(chunk_bitlen32(m, slot++));
+            const int r = q8_shift(chunk_bitlen32(m, slot++));  // (its barrier: every thread has read the accumulator)
             const Rnd rq = make_rnd(r);
 #pragma unroll
             for (int w = 0; w < kHC / 4; ++w)
-                rpk[s - 1][w] = q8_pack4(static_cast<int>(dres[4 * w]), static_cast<int>(dres[4 * w + 1]),
-                                         static_cast<int>(dres[4 * w + 2]), static_cast<int>(dres[4 * w + 3]), rq);
+                cur[w] = q8_pack4(static_cast<int>(dres[4 * w]), static_cast<int>(dres[4 * w + 1]),
+                                  static_cast<int>(dres[4 * w + 2]), static_cast<int>(dres[4 * w + 3]), rq);
+            tmem_st8(lane_base + park_col(s), cur);
             er[s - 1] = er[s - 2] + eE + r;
             n_terms = s;
         }
@@ -564,20 +566,24 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             for (int s = 1; s < kSMax; ++s)
                 if (s < n_terms) { emin = min(emin, er[s]); emax = max(emax, er[s]); }
             const int eref = max(emin, emax - kAlignWindow);
-            int sh[kSMax];
-#pragma unroll
-            for (int s = 0; s < kSMax; ++s) sh[s] = (s < n_terms) ? er[s] - eref : -64;
             int acc[kHC];
 #pragma unroll
             for (int jl = 0; jl < kHC; ++jl) acc[jl] = 0;
+            tmem_st8(lane_base + park_col(1), r1);
+            tmem_wait_st();
+#pragma unroll 1
+            for (int s = 1; s <= n_terms; ++s) {
+                const int sh = er[s - 1] - eref;
+                if (sh < -7) continue;
+                uint32_t w[kHC / 4];
+                tmem_ld8(lane_base + park_col(s), w);
+                tmem_wait_ld();
+                if (sh >= 0) {
 #pragma unroll
-            for (int s = 0; s < kSMax; ++s) {
-                if (sh[s] >= 0) {
+                    for (int jl = 0; jl < kHC; ++jl) acc[jl] += byte_at(w[jl >> 2], jl & 3) << sh;
+                } else {
 #pragma unroll
-                    for (int jl = 0; jl < kHC; ++jl) acc[jl] += byte_at(rpk[s][jl >> 2], jl & 3) << sh[s];
-                } else if (sh[s] >= -7) {
-#pragma unroll
-                    for (int jl = 0; jl < kHC; ++jl) acc[jl] += rsr32(byte_at(rpk[s][jl >> 2], jl & 3), -sh[s]);
+                    for (int jl = 0; jl < kHC; ++jl) acc[jl] += rsr32(byte_at(w[jl >> 2], jl & 3), -sh);
                 }
             }
             uint32_t m = 0;
