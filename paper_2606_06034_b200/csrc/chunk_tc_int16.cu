@@ -74,7 +74,8 @@ constexpr int kOffDecay = kOffBeta + 512;
 constexpr int kOffLut = kOffDecay + 512;
 constexpr int kOffRed = kOffLut + 512;     // OR-reduction slots: [24][2 chunks][2 words]
 constexpr int kNumRed = 24;
-constexpr int kSmemTotal = kOffRed + kNumRed * 16;
+constexpr int kOffPark = (kOffRed + kNumRed * 16 + 1023) / 1024 * 1024;  // 80 KB: parked rows of R_4..R_8 (see the kernel)
+constexpr int kSmemTotal = kOffPark + 5 * 16384;
 
 __device__ __forceinline__ void cta_barrier() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
@@ -88,21 +89,24 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity) {
     return true;
 }
 
-// rounded right shift, half away from zero (r >= 0)
+// rounded right shift, half away from zero (0 <= r <= 62), without branches: for x < 0 the rounded shift of the
+// magnitude equals the arithmetic shift of x + half - 1 (floor((x + h - 1) / 2^r) = -floor((|x| + h) / 2^r) because
+// 2^r - h = h); r = 0 gives x. r is uniform over a chunk, so the constants are computed once per stage.
 __device__ __forceinline__ long long rsr64(long long x, int r) {
-    if (r == 0) return x;
-    const unsigned long long a = static_cast<unsigned long long>(x < 0 ? -x : x);
-    const long long q = static_cast<long long>((a + (1ull << (r - 1))) >> r);
-    return x < 0 ? -q : q;
+    const long long half = static_cast<long long>((1ull << r) >> 1);
+    const long long neg1 = (r > 0) ? (x >> 63) : 0;
+    return (x + half + neg1) >> r;
 }
 // one term of an aligned sum: x 2^s for s >= 0, rounded right shift otherwise
 __device__ __forceinline__ long long term64(long long x, int s) {
-    if (s >= 0) return x << s;
-    return rsr64(x, (-s) < 62 ? (-s) : 62);
+    const int r = s >= 0 ? 0 : ((-s) < 62 ? (-s) : 62);
+    return rsr64(x, r) << (s >= 0 ? s : 0);
 }
+// clamp(rsr(x, r), +-kQ). r is the shift of the chunk's largest magnitude (q_shift of its bit length), so the shifted
+// value is at most 2^15 in magnitude and the clamp is done in 32 bits.
 __device__ __forceinline__ int q16(long long x, int r) {
-    const long long y = rsr64(x, r);
-    return static_cast<int>(y > kQ ? kQ : (y < -kQ ? -kQ : y));
+    const int y = static_cast<int>(rsr64(x, r));
+    return max(min(y, kQ), -kQ);
 }
 __device__ __forceinline__ unsigned long long abs64(long long x) { return static_cast<unsigned long long>(x < 0 ? -x : x); }
 __device__ __forceinline__ int q_shift(int bitlen) { return bitlen > 15 ? bitlen - 15 : 0; }
@@ -302,10 +306,6 @@ chunk_tc_int16_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
         tc_fence_before_sync();
         cta_barrier();  // the previous tile is finished with the shared arrays, the V tile and the accumulators
         if (tid == 0) {
-            // the V tile of this tile (its buffer was read until the end of the previous tile)
-            mbar_arrive_expect_tx(&bar_v, 32768);
-            tma_load_3d(sV16, &tmV, &bar_v, 0, tc.t0, tc.bhv);
-            tma_load_3d(sV16 + 16384, &tmV, &bar_v, 64, tc.t0, tc.bhv);
             if (!wait_bar(&bar_k, par_kv)) set_fail();
         }
         if (h == 0) {
@@ -480,26 +480,35 @@ chunk_tc_int16_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
             for (int jl = 0; jl < kHC; ++jl) eq[jl] = q16(acc[jl], r);
             eE = eref + r;
         }
-        // rows of the powers R_s (R_1 = Eq) as int16 pairs, and their exponents
-        uint32_t rpk[kSMax][kHC / 2];
+        // Rows of the powers R_s (R_1 = Eq) as int16 pairs. The loops over the powers are NOT unrolled (the kernel is bound
+        // by instruction fetch), so the rows cannot sit in registers indexed by s: every thread parks its 64 bytes of R_s
+        // in shared memory and reads them back for the sum. The parked rows are private to the thread (no barrier):
+        // R_1 in its private row (the Aq row there is dead), R_2 and R_3 in the V tile's buffer (V is loaded after the
+        // sum), R_4..R_8 in a region of their own.
+        auto park = [&](int s) -> uint8_t* {
+            uint8_t* base = (s == 1) ? sRow : (s <= 3 ? sV16 + (s - 2) * 16384 : smem + kOffPark + (s - 4) * 16384);
+            return base + t * 128 + h * 64;
+        };
+        uint32_t cur[kHC / 2];  // R_{s-1} inside the loop
         int er[kSMax];
 #pragma unroll
-        for (int s = 0; s < kSMax; ++s) {
-            er[s] = 0;
+        for (int s = 0; s < kSMax; ++s) er[s] = 0;
 #pragma unroll
-            for (int w = 0; w < kHC / 2; ++w) rpk[s][w] = 0u;
-        }
+        for (int w = 0; w < kHC / 2; ++w) cur[w] = 0u;
         int n_terms = 0;
         if (S >= 1) {
 #pragma unroll
-            for (int w = 0; w < kHC / 2; ++w) rpk[0][w] = pack2(eq[2 * w], eq[2 * w + 1]);
+            for (int w = 0; w < kHC / 2; ++w) cur[w] = pack2(eq[2 * w], eq[2 * w + 1]);
             er[0] = eE;
             n_terms = 1;
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                *reinterpret_cast<uint4*>(park(1) + c * 16) = make_uint4(cur[4 * c], cur[4 * c + 1], cur[4 * c + 2], cur[4 * c + 3]);
             // B operand [E_1 | E_2] as two byte planes (64 x 128 bytes each, MN-major, no swizzle): 16 columns of
             // chunk-row il per 16-byte piece
 #pragma unroll
             for (int c = 0; c < kHC / 16; ++c) {
-                const uint32_t* w = &rpk[0][8 * c];
+                const uint32_t* w = &cur[8 * c];
                 const uint32_t off = (((cb + col0) >> 4) + c) * (16 * kC) + il * 16;
                 *reinterpret_cast<uint4*>(sEl + off) = make_uint4(plane_lo(w[0], w[1]), plane_lo(w[2], w[3]), plane_lo(w[4], w[5]), plane_lo(w[6], w[7]));
                 *reinterpret_cast<uint4*>(sEh + off) = make_uint4(plane_hi(w[0], w[1]), plane_hi(w[2], w[3]), plane_hi(w[4], w[5]), plane_hi(w[6], w[7]));
@@ -507,17 +516,16 @@ chunk_tc_int16_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
         }
         // ---- I7: R_s = Q16(R_{s-1} Eq) while s (N+1) < C
         bool bad = false;
-#pragma unroll
+#pragma unroll 1
         for (int s = 2; s <= kSMax; ++s) {
             if (s > S || s * (N + 1) >= kC) break;
             {
                 // A operand: the rows of R_{s-1}, chunks stacked along M, as byte planes (64 bytes = 16 columns per plane)
-                const uint32_t* w = rpk[s - 2];
                 uint32_t lo8[8], hi8[8];
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
-                    lo8[i] = plane_lo(w[2 * i], w[2 * i + 1]);
-                    hi8[i] = plane_hi(w[2 * i], w[2 * i + 1]);
+                    lo8[i] = plane_lo(cur[2 * i], cur[2 * i + 1]);
+                    hi8[i] = plane_hi(cur[2 * i], cur[2 * i + 1]);
                 }
                 tmem_st8(lane_base + kAh + h * 8, hi8);
                 tmem_st8(lane_base + kAl + h * 8, lo8);
@@ -549,7 +557,10 @@ chunk_tc_int16_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
             }
             const int r = q_shift(chunk_bitlen(m, slot++));
 #pragma unroll
-            for (int w = 0; w < kHC / 2; ++w) rpk[s - 1][w] = pack2(q16(acc[2 * w], r), q16(acc[2 * w + 1], r));
+            for (int w = 0; w < kHC / 2; ++w) cur[w] = pack2(q16(acc[2 * w], r), q16(acc[2 * w + 1], r));
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                *reinterpret_cast<uint4*>(park(s) + c * 16) = make_uint4(cur[4 * c], cur[4 * c + 1], cur[4 * c + 2], cur[4 * c + 3]);
             er[s - 1] = er[s - 2] + eE + r;
             n_terms = s;
         }
@@ -567,20 +578,34 @@ chunk_tc_int16_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
             long long acc[kHC];
 #pragma unroll
             for (int jl = 0; jl < kHC; ++jl) acc[jl] = 0;
+#pragma unroll 1
+            for (int s = 1; s <= n_terms; ++s) {
+                const int sh = er[s - 1] - eref;
+                if (sh < -15) continue;
+                uint32_t w[kHC / 2];
 #pragma unroll
-            for (int s = 0; s < kSMax; ++s) {
-                const int sh = (s < n_terms) ? er[s] - eref : -64;
-                if (sh >= -15) {
+                for (int c = 0; c < 4; ++c) {
+                    const uint4 v = *reinterpret_cast<const uint4*>(park(s) + c * 16);
+                    w[4 * c] = v.x; w[4 * c + 1] = v.y; w[4 * c + 2] = v.z; w[4 * c + 3] = v.w;
+                }
+                if (sh >= 0) {
 #pragma unroll
-                    for (int w = 0; w < kHC / 2; ++w) {
-                        acc[2 * w] += term64(lo16(rpk[s][w]), sh);
-                        acc[2 * w + 1] += term64(hi16(rpk[s][w]), sh);
+                    for (int i = 0; i < kHC / 2; ++i) {
+                        acc[2 * i] += static_cast<long long>(lo16(w[i])) << sh;
+                        acc[2 * i + 1] += static_cast<long long>(hi16(w[i])) << sh;
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < kHC / 2; ++i) {
+                        acc[2 * i] += rsr64(lo16(w[i]), -sh);
+                        acc[2 * i + 1] += rsr64(hi16(w[i]), -sh);
                     }
                 }
             }
             unsigned long long m = 0;
 #pragma unroll
             for (int jl = 0; jl < kHC; ++jl) m |= abs64(acc[jl]);
+            fence_proxy_async_smem();  // the parked rows in the V buffer are overwritten by a bulk copy next
             const int r = q_shift(chunk_bitlen(m, slot++));
 #pragma unroll
             for (int jl = 0; jl < kHC; ++jl) sq[jl] = q16(acc[jl], r);
@@ -588,6 +613,14 @@ chunk_tc_int16_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
         } else {
 #pragma unroll
             for (int jl = 0; jl < kHC; ++jl) sq[jl] = 0;
+        }
+        // the V tile of this tile: its buffer held parked rows until the sum above (every thread is past its reads: the
+        // reduction of the sum is a barrier), and the previous tile's U stage is long finished
+        if (n_terms == 0) cta_barrier();
+        if (tid == 0) {
+            mbar_arrive_expect_tx(&bar_v, 32768);
+            tma_load_3d(sV16, &tmV, &bar_v, 0, tc.t0, tc.bhv);
+            tma_load_3d(sV16 + 16384, &tmV, &bar_v, 64, tc.t0, tc.bhv);
         }
         // Sq to the private rows (the rows above are needed for T0q Sq)
 #pragma unroll
@@ -694,9 +727,16 @@ chunk_tc_int16_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
 #pragma unroll 1
         for (int half = 0; half < 2; ++half) {
             const int xexp = (half == 0) ? kexp : vexp;
-            // diagonal term beta_q_i * Xq_i for this thread's 64 columns, from its own row of the int16 tile
-            uint32_t xr[32];
-            load_row16((half == 0) ? sK16 : sV16, xr);
+            // diagonal term beta_q_i * Xq_i for this thread's 64 columns, from its own row of the int16 tile (32 columns
+            // at a time: the loops over the column blocks are not unrolled)
+            const uint8_t* xtile = (half == 0) ? sK16 : sV16;
+            auto load_x32 = [&](int c0, uint32_t (&w)[16]) {
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const uint4 v = *reinterpret_cast<const uint4*>(xtile + h * 16384 + t * 128 + ((((c0 >> 3) + c) ^ (t & 7)) << 4));
+                    w[4 * c + 0] = v.x; w[4 * c + 1] = v.y; w[4 * c + 2] = v.z; w[4 * c + 3] = v.w;
+                }
+            };
             if (!wait_mma()) { bad2 = true; break; }
             tc_fence_after_sync();
             const int ep = eTb + xexp, ed = xexp - 15;
@@ -704,8 +744,10 @@ chunk_tc_int16_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
             const int sp = ep - eref, sd = ed - eref;
             // pass 1: the scale (bit length of the largest magnitude over the chunk's C x d block)
             unsigned long long m = 0;
-#pragma unroll
+#pragma unroll 1
             for (int c0 = 0; c0 < 64; c0 += 32) {
+                uint32_t xr[16];
+                load_x32(c0, xr);
                 uint32_t dhh[32], dmid[32], dll[32];
                 tmem_ld32(lane_base + kDhh + h * 64 + c0, dhh);
                 tmem_ld32(lane_base + kDmid + h * 64 + c0, dmid);
@@ -715,8 +757,8 @@ chunk_tc_int16_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
                 for (int i = 0; i < 32; ++i) {
                     const long long pr = combine(dhh[i], dmid[i], dll[i]);
                     if (dbg_row != nullptr) dbg_row[8 * kC + half * kD + h * 64 + c0 + i] = pr;
-                    const uint32_t xw = xr[(c0 + i) >> 1];
-                    const int x = ((c0 + i) & 1) ? hi16(xw) : lo16(xw);
+                    const uint32_t xw = xr[i >> 1];
+                    const int x = (i & 1) ? hi16(xw) : lo16(xw);
                     m |= abs64(term64(pr, sp) + term64((long long)bq * x, sd));
                 }
             }
@@ -724,8 +766,10 @@ chunk_tc_int16_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
             if (row_valid && il == 0 && h == 0) ((half == 0) ? p.w_exp : p.u_exp)[chunk_id] = eref + rr;
             // pass 2: mantissas, 64 int16 of this thread's row straight to global memory
             int16_t* out = ((half == 0) ? p.W : p.U) + grow * kD + h * 64;
-#pragma unroll
+#pragma unroll 1
             for (int c0 = 0; c0 < 64; c0 += 32) {
+                uint32_t xr[16];
+                load_x32(c0, xr);
                 uint32_t dhh[32], dmid[32], dll[32];
                 tmem_ld32(lane_base + kDhh + h * 64 + c0, dhh);
                 tmem_ld32(lane_base + kDmid + h * 64 + c0, dmid);
@@ -734,7 +778,7 @@ chunk_tc_int16_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
                 uint32_t o[16];
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
-                    const uint32_t xw = xr[(c0 >> 1) + i];
+                    const uint32_t xw = xr[i];
                     const long long v0 = term64(combine(dhh[2 * i], dmid[2 * i], dll[2 * i]), sp) + term64((long long)bq * lo16(xw), sd);
                     const long long v1 = term64(combine(dhh[2 * i + 1], dmid[2 * i + 1], dll[2 * i + 1]), sp) + term64((long long)bq * hi16(xw), sd);
                     o[i] = pack2(q16(v0, rr), q16(v1, rr));
