@@ -97,21 +97,37 @@ __device__ __forceinline__ int term32(int x, int s) {
     if (s >= 0) return x << s;
     return rsr32(x, (-s) < 31 ? (-s) : 31);
 }
-// Rounding constants of one requantisation (uniform over a chunk): shift, rounding half, and an all-ones mask when
+// Rounding constants of one requantisation (uniform over a chunk): shift, rounding half, and a flag that is 1 when
 // something is shifted out.
 struct Rnd {
-    int r, half, mask;
+    int r, half, flag;
 };
 __device__ __forceinline__ Rnd make_rnd(int r) {
     Rnd q;
     q.r = r;
     q.half = static_cast<int>((1u << r) >> 1);
-    q.mask = (r > 0) ? -1 : 0;
+    q.flag = (r > 0) ? 1 : 0;
     return q;
 }
 // rsr(x, r), branch-free: for x < 0 the rounded magnitude shift equals the arithmetic shift of x + half - 1
 // (floor((x + h - 1) / 2^r) = -floor((|x| + h) / 2^r) because 2^r - h = h); r = 0 gives x.
-__device__ __forceinline__ int rsr_rnd(int x, const Rnd& q) { return (x + q.half + ((x >> 31) & q.mask)) >> q.r; }
+// The correction term half - [x < 0] is one multiply-add on the (otherwise idle) multiplier pipe: the high word of
+// x * flag is -1 for x < 0 and 0 otherwise (flag = 1; flag = 0 when nothing is shifted out).
+__device__ __forceinline__ int mad_hi(int a, int b, int c) {
+    int d;
+    asm("mad.hi.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+__device__ __forceinline__ int rsr_rnd(int x, const Rnd& q) { return (x + mad_hi(x, q.flag, q.half)) >> q.r; }
+// largest magnitude of a set of values, two at a time with three-input min / max; only its bit length is used
+struct MaxMag {
+    int mx = 0, mn = 0;
+    __device__ __forceinline__ void add2(int a, int b) {
+        mx = __vimax3_s32(mx, a, b);
+        mn = __vimin3_s32(mn, a, b);
+    }
+    __device__ __forceinline__ uint32_t mag() const { return static_cast<uint32_t>(max(mx, -mn)); }
+};
 // clamp(rsr(x, r), +-127)
 __device__ __forceinline__ int q8_32(int x, const Rnd& q) { return max(min(rsr_rnd(x, q), 127), -127); }
 __device__ __forceinline__ int q8_32(int x, int r) { return q8_32(x, make_rnd(r)); }
@@ -476,8 +492,11 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 const int pr = a1 * c4.x + a2 * c4.y + a3 * c4.z;
                 const int v = on ? (left ? ((aq[jl] << sa) + (pr << sp)) : (term32(aq[jl], sa) + term32(pr, sp))) : 0;
                 acc[jl] = v;
-                m |= abs32(v);
             }
+            MaxMag mm;
+#pragma unroll
+            for (int jl = 0; jl < kHC; jl += 2) mm.add2(acc[jl], acc[jl + 1]);
+            m = mm.mag();
             const int r = q8_shift(chunk_bitlen32(m, slot++));
             const Rnd rq = make_rnd(r);
 #pragma unroll
@@ -542,8 +561,12 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             uint32_t m = 0;
             // R_{s-1} is zero for i - j < (s - 1)(N + 1) and Eq for i - j <= N: the integer product is exactly zero
             // for i - j < s (N + 1), no mask needed
+            {
+                MaxMag mm;
 #pragma unroll
-            for (int jl = 0; jl < kHC; ++jl) m |= abs32(static_cast<int>(dres[jl]));
+                for (int jl = 0; jl < kHC; jl += 2) mm.add2(static_cast<int>(dres[jl]), static_cast<int>(dres[jl + 1]));
+                m = mm.mag();
+            }
             const int r = q8_shift(chunk_bitlen32(m, slot++));  // (its barrier: every thread has read the accumulator)
             const Rnd rq = make_rnd(r);
 #pragma unroll
@@ -586,9 +609,10 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                     for (int jl = 0; jl < kHC; ++jl) acc[jl] += rsr32(byte_at(w[jl >> 2], jl & 3), -sh);
                 }
             }
-            uint32_t m = 0;
+            MaxMag mm;
 #pragma unroll
-            for (int jl = 0; jl < kHC; ++jl) m |= abs32(acc[jl]);
+            for (int jl = 0; jl < kHC; jl += 2) mm.add2(acc[jl], acc[jl + 1]);
+            const uint32_t m = mm.mag();
             const int r = q8_shift(chunk_bitlen32(m, slot++));
             const Rnd rq = make_rnd(r);
 #pragma unroll
@@ -647,7 +671,12 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                                               : (term32(v, (d <= N) ? s0 : s1) + term32(prod[jl], s2)))
                                       : 0;
                 acc[jl] = a;
-                m |= abs32(a);
+            }
+            {
+                MaxMag mm;
+#pragma unroll
+                for (int jl = 0; jl < kHC; jl += 2) mm.add2(acc[jl], acc[jl + 1]);
+                m = mm.mag();
             }
             const int r = q8_shift(chunk_bitlen32(m, slot++));
             const Rnd rq = make_rnd(r);
@@ -664,7 +693,12 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
 #pragma unroll
             for (int jl = 0; jl < kHC; ++jl) {
                 acc[jl] = toff[jl] * sbeta[cb + col0 + jl];
-                m |= abs32(acc[jl]);
+            }
+            {
+                MaxMag mm;
+#pragma unroll
+                for (int jl = 0; jl < kHC; jl += 2) mm.add2(acc[jl], acc[jl + 1]);
+                m = mm.mag();
             }
             const int r = q8_shift(chunk_bitlen32(m, slot++));
             const Rnd rq9 = make_rnd(r);
@@ -734,7 +768,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             // pass 1: the scale (bit length of the largest magnitude over the chunk's C x d block)
             const bool left = sp >= 0 && sd >= 0;  // the usual case: plain left shifts
             const int psc = left ? (1 << sp) : 0, bqs = left ? (bq << sd) : 0;
-            uint32_t m = 0;
+            MaxMag mmw;
             int sums[64];  // the aligned sums of this thread's 64 columns stay in registers between the two passes
 #pragma unroll
             for (int c0 = 0; c0 < 64; c0 += 32) {
@@ -756,9 +790,9 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                         sums[c0 + i] = term32(static_cast<int>(r[i]), sp) + term32(bq * byte_at(xr[(c0 + i) >> 2], (c0 + i) & 3), sd);
                 }
 #pragma unroll
-                for (int i = 0; i < 32; ++i) m |= abs32(sums[c0 + i]);
+                for (int i = 0; i < 32; i += 2) mmw.add2(sums[c0 + i], sums[c0 + i + 1]);
             }
-            const int rr = q8_shift(chunk_bitlen32(m, slot++));
+            const int rr = q8_shift(chunk_bitlen32(mmw.mag(), slot++));
             const Rnd rqw = make_rnd(rr);
             // after that barrier every thread holds its own row of the K (V) tile in registers, and the products that
             // read the tile are complete: the next tile's K (V) may land
