@@ -518,6 +518,16 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             return (s >= 2 && s <= 7) ? static_cast<uint32_t>(160 + (s - 2) * 16 + h * 8)
                                       : static_cast<uint32_t>(kR0 + (s == 1 ? 0 : 16) + h * 8);
         };
+        // Structural support: R_s is zero for i - j < s (N + 1), so of this thread's four blocks of eight columns only the
+        // first live_blocks(s) can hold a non-zero entry in any of the warp's 32 rows (a warp-uniform count; the warp
+        // with rows 0..31 and columns 32..63 has none at all). Dead blocks are skipped in the requantisation and in the
+        // sum. With the debug output every block is walked (the test reads every accumulator).
+        const int row_max = (wrow0 & (kC - 1)) + 31;
+        const bool walk_all = p.dbg != nullptr;
+        auto live_blocks = [&](int s) -> int {
+            const int x = row_max - col0 - s * (N + 1);
+            return walk_all ? 4 : (x < 0 ? 0 : min(4, (x >> 3) + 1));
+        };
         int n_terms = 0;
         if (S >= 1) {
 #pragma unroll
@@ -561,18 +571,30 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             uint32_t m = 0;
             // R_{s-1} is zero for i - j < (s - 1)(N + 1) and Eq for i - j <= N: the integer product is exactly zero
             // for i - j < s (N + 1), no mask needed
+            const int nb = live_blocks(s);
             {
                 MaxMag mm;
 #pragma unroll
-                for (int jl = 0; jl < kHC; jl += 2) mm.add2(static_cast<int>(dres[jl]), static_cast<int>(dres[jl + 1]));
+                for (int b = 0; b < 4; ++b) {
+                    if (b < nb) {
+#pragma unroll
+                        for (int jl = 8 * b; jl < 8 * b + 8; jl += 2) mm.add2(static_cast<int>(dres[jl]), static_cast<int>(dres[jl + 1]));
+                    }
+                }
                 m = mm.mag();
             }
             const int r = q8_shift(chunk_bitlen32(m, slot++));  // (its barrier: every thread has read the accumulator)
             const Rnd rq = make_rnd(r);
 #pragma unroll
-            for (int w = 0; w < kHC / 4; ++w)
-                cur[w] = q8_pack4(static_cast<int>(dres[4 * w]), static_cast<int>(dres[4 * w + 1]),
-                                  static_cast<int>(dres[4 * w + 2]), static_cast<int>(dres[4 * w + 3]), rq);
+            for (int b = 0; b < 4; ++b) {
+                cur[2 * b] = cur[2 * b + 1] = 0u;
+                if (b < nb) {
+#pragma unroll
+                    for (int w = 2 * b; w < 2 * b + 2; ++w)
+                        cur[w] = q8_pack4(static_cast<int>(dres[4 * w]), static_cast<int>(dres[4 * w + 1]),
+                                          static_cast<int>(dres[4 * w + 2]), static_cast<int>(dres[4 * w + 3]), rq);
+                }
+            }
             tmem_st8(lane_base + park_col(s), cur);
             er[s - 1] = er[s - 2] + eE + r;
             n_terms = s;
@@ -598,25 +620,50 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             for (int s = 1; s <= n_terms; ++s) {
                 const int sh = er[s - 1] - eref;
                 if (sh < -7) continue;
+                const int nb = live_blocks(s);
+                if (nb == 0) continue;
                 uint32_t w[kHC / 4];
                 tmem_ld8(lane_base + park_col(s), w);
                 tmem_wait_ld();
                 if (sh >= 0) {
 #pragma unroll
-                    for (int jl = 0; jl < kHC; ++jl) acc[jl] += byte_at(w[jl >> 2], jl & 3) << sh;
+                    for (int b = 0; b < 4; ++b) {
+                        if (b < nb) {
+#pragma unroll
+                            for (int jl = 8 * b; jl < 8 * b + 8; ++jl) acc[jl] += byte_at(w[jl >> 2], jl & 3) << sh;
+                        }
+                    }
                 } else {
 #pragma unroll
-                    for (int jl = 0; jl < kHC; ++jl) acc[jl] += rsr32(byte_at(w[jl >> 2], jl & 3), -sh);
+                    for (int b = 0; b < 4; ++b) {
+                        if (b < nb) {
+#pragma unroll
+                            for (int jl = 8 * b; jl < 8 * b + 8; ++jl) acc[jl] += rsr32(byte_at(w[jl >> 2], jl & 3), -sh);
+                        }
+                    }
                 }
             }
+            const int nb1 = live_blocks(1);  // the support of the sum is that of its first term
             MaxMag mm;
 #pragma unroll
-            for (int jl = 0; jl < kHC; jl += 2) mm.add2(acc[jl], acc[jl + 1]);
+            for (int b = 0; b < 4; ++b) {
+                if (b < nb1) {
+#pragma unroll
+                    for (int jl = 8 * b; jl < 8 * b + 8; jl += 2) mm.add2(acc[jl], acc[jl + 1]);
+                }
+            }
             const uint32_t m = mm.mag();
             const int r = q8_shift(chunk_bitlen32(m, slot++));
             const Rnd rq = make_rnd(r);
 #pragma unroll
-            for (int jl = 0; jl < kHC; ++jl) sq[jl] = q8_32(acc[jl], rq);
+            for (int b = 0; b < 4; ++b) {
+#pragma unroll
+                for (int jl = 8 * b; jl < 8 * b + 8; ++jl) sq[jl] = 0;
+                if (b < nb1) {
+#pragma unroll
+                    for (int jl = 8 * b; jl < 8 * b + 8; ++jl) sq[jl] = q8_32(acc[jl], rq);
+                }
+            }
             eS = eref + r;
         } else {
 #pragma unroll
