@@ -1,0 +1,91 @@
+"""Pins for the exact-integer INT8 oracle on chunks of 128 tokens (two 64-blocks and the block formula of App. E,
+Eq. 28): two separately written evaluators, reductions to the 64-token evaluator that the block structure forces,
+and a sanity band against the fp64 inverse of the same (dequantised) inputs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import gdn_oracle as orc
+from oracle import gdn_oracle_int8 as orq
+from paper_2606_06034_b200 import inputs as gen
+
+
+def _chunks128(n_heads=2, T=128, seed=0, adversarial="none", d=16):
+    inp = gen.make_inputs(1, n_heads, n_heads, T, 128, d, d, seed=seed, dtype=torch.float32, adversarial_heads=adversarial)
+    q = gen.make_int8_inputs(inp)
+    return gen.int8_chunk_slices(q, range(q.n_chunks))
+
+
+@pytest.mark.parametrize("adv,N,S,d", [("none", 3, 8, 16), ("all", 3, 8, 16), ("none", 2, 3, 8), ("none", 3, 8, 128)])
+def test_two_evaluators_agree_bit_for_bit(adv, N, S, d):
+    Kq, Vq, ke, ve, bq, dq = _chunks128(n_heads=1 if d == 128 else 2, seed=3 + N + S, adversarial=adv, d=d)
+    fast = orq.chunk_prepare_int8_c128(Kq, Vq, ke, ve, bq, dq, N, S)
+    for c in range(Kq.shape[0]):
+        ref = orq.chunk_prepare_int8_c128_ref(Kq[c].tolist(), Vq[c].tolist(), int(ke[c]), int(ve[c]), bq[c].tolist(), dq[c].tolist(), N, S)
+        for key in ("Wq", "Uq", "Toffq"):
+            assert np.array_equal(np.asarray(ref[key]), fast[key][c]), key
+        for key in ("w_exp", "u_exp", "t_exp"):
+            assert tuple(int(v) for v in ref[key]) == tuple(int(v) for v in fast[key][c]), key
+
+
+@pytest.mark.parametrize("adv", ["none", "all"])
+def test_structure_and_top_block_is_the_64_token_chunk(adv):
+    """Rows 0..63 of a 128-chunk do not see rows 64..127 (T is lower triangular): the first block, its exponent and
+    its rows of W and U are those of the 64-token evaluator on the first 64 tokens, bit for bit. The upper-right
+    block of Toffq is zero and every mantissa is within +-127."""
+    Kq, Vq, ke, ve, bq, dq = _chunks128(seed=11, adversarial=adv, d=32, T=256)
+    out = orq.chunk_prepare_int8_c128(Kq, Vq, ke, ve, bq, dq, 3, 8)
+    top = orq.chunk_prepare_int8(Kq[:, :64], Vq[:, :64], ke, ve, bq[:, :64], dq[:, :64], 3, 8)
+    assert np.array_equal(out["Toffq"][:, :64, :64], top["Toffq"]) and np.array_equal(out["t_exp"][:, 0], top["t_exp"])
+    assert np.array_equal(out["Wq"][:, :64], top["Wq"]) and np.array_equal(out["w_exp"][:, 0], top["w_exp"])
+    assert np.array_equal(out["Uq"][:, :64], top["Uq"]) and np.array_equal(out["u_exp"][:, 0], top["u_exp"])
+    assert not out["Toffq"][:, :64, 64:].any()
+    assert not np.triu(out["Toffq"]).any()
+    for key in ("Toffq", "Wq", "Uq"):
+        assert np.abs(out[key].astype(np.int64)).max() <= 127
+    assert np.abs(out["Toffq"][:, 64:, :64].astype(np.int64)).max() > 32  # the lower-left block is really there
+
+
+def test_closed_gate_between_the_blocks_decouples_them():
+    """When the gate closes at token 64 (decay difference of 16 octaves or more: Gamma = 0 across the blocks), A21 = 0:
+    the lower-left block of T vanishes and rows 64..127 are the 64-token evaluation of tokens 64..127, bit for bit
+    (mantissas and exponents)."""
+    Kq, Vq, ke, ve, bq, dq = _chunks128(seed=5, d=32, T=256)
+    dq = dq.copy()
+    dq[:, 64:] += 16 * 256
+    out = orq.chunk_prepare_int8_c128(Kq, Vq, ke, ve, bq, dq, 3, 8)
+    bot = orq.chunk_prepare_int8(Kq[:, 64:], Vq[:, 64:], ke, ve, bq[:, 64:], dq[:, 64:], 3, 8)
+    assert not out["Toffq"][:, 64:, :64].any()
+    assert np.array_equal(out["Toffq"][:, 64:, 64:], bot["Toffq"]) and np.array_equal(out["t_exp"][:, 2], bot["t_exp"])
+    assert np.array_equal(out["Wq"][:, 64:], bot["Wq"]) and np.array_equal(out["w_exp"][:, 1], bot["w_exp"])
+    assert np.array_equal(out["Uq"][:, 64:], bot["Uq"]) and np.array_equal(out["u_exp"][:, 1], bot["u_exp"])
+
+
+def _snr128(out, Kq, Vq, ke, ve, bq, dq):
+    K = Kq * np.exp2(ke.astype(float))[:, None, None]
+    V = Vq * np.exp2(ve.astype(float))[:, None, None]
+    beta = bq / 32768.0
+    g = -dq / (256.0 * 1.4426950408889634)
+    We, Ue, Te = orc.chunk_prepare(K, V, beta, g, exact=True)
+    T = orq.dequantise_c128(out["Toffq"], out["t_exp"])
+    rows = np.repeat(np.arange(2), 64)
+    W = out["Wq"] * np.exp2(out["w_exp"].astype(float))[:, rows, None]
+    U = out["Uq"] * np.exp2(out["u_exp"].astype(float))[:, rows, None]
+    X = Te - np.eye(128)
+    return (orc.snr_db(T, X), orc.snr_db(T[:, 64:, :64], X[:, 64:, :64]), orc.snr_db(W, We), orc.snr_db(U, Ue))
+
+
+@pytest.mark.parametrize("adv,lo_T,lo_21,lo_W,lo_U", [("none", 28.0, 28.0, 33.0, 29.0), ("all", 26.0, 8.0, 23.0, 28.0)])
+def test_dequantised_result_tracks_the_fp64_inverse(adv, lo_T, lo_21, lo_W, lo_U):
+    """Sanity band: the dequantised integer result stays within an 8-bit SNR band of the exact fp64 inverse (and W,
+    U) of the same dequantised inputs, for the whole of T - I and for the lower-left block alone (a wrong sign or a
+    dropped term of the block formula leaves that block at 0 dB or below: with the sign of Eq. 28 applied to blocks that
+    already hold -A it sits at -6.0 dB). The floors are within 3 dB of what these inputs give (benign: T - I 30.2..33.6,
+    lower-left block 30.6..39.3, W 35.3..35.8, U 31.6..35.9 dB; adversarial: 28.0..29.0, 10.1..11.4 (the block whose
+    terms cancel on correlated keys, at 8-bit operands), 25.0..26.8, 30.2..31.1). Not a precision claim about the
+    paper's INT8."""
+    for seed in (9, 10):
+        Kq, Vq, ke, ve, bq, dq = _chunks128(seed=seed, adversarial=adv, d=64, T=256)
+        out = orq.chunk_prepare_int8_c128(Kq, Vq, ke, ve, bq, dq, 3, 8)
+        sT, s21, sW, sU = _snr128(out, Kq, Vq, ke, ve, bq, dq)
+        assert sT.min() > lo_T and s21.min() > lo_21 and sW.min() > lo_W and sU.min() > lo_U, (sT, s21, sW, sU)
