@@ -341,12 +341,15 @@ def run_ours(args, rank, world, dist_ctx):
     n_untimed = max(args.warmup, min(50, int(0.1 / one) + 1))
     for _ in range(n_untimed):
         step()
+    lc = gdn.gdn_launch_count()
+    step()
+    per_call = gdn.gdn_launch_count() - lc  # kernels per call of the entry point (two for INT8 chunks of 128 tokens)
     torch.cuda.synchronize()
     launches0 = gdn.gdn_launch_count()
     sampler.start()
     total_ms, per = device_time_steps(step, args.steps, 0, dist_ctx)
     clocks = sampler.stop()
-    launches = gdn.gdn_launch_count() - launches0 - 2  # the two queue-priming launches sit before the first event
+    launches = gdn.gdn_launch_count() - launches0 - 2 * per_call  # the two queue-priming calls sit before the first event
     # a timed region that saw a thermal or hardware slowdown, or clocks far below maximum with no reason given (a leftover
     # clock lock), is not a measurement: take it once more and say so
     bad = {"hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown"} & set(clocks.get("reasons") or [])
@@ -363,7 +366,7 @@ def run_ours(args, rank, world, dist_ctx):
         total_ms, per = device_time_steps(step, args.steps, 0, dist_ctx)
         first, clocks = clocks, sampler.stop()
         clocks["first_attempt"] = first
-        launches = gdn.gdn_launch_count() - launches0 - 2
+        launches = gdn.gdn_launch_count() - launches0 - 2 * per_call
         remeasured = True
     status = gdn.gdn_device_status()
     if status != gdn.GDN_OK:
@@ -397,7 +400,7 @@ def run_ours(args, rank, world, dist_ctx):
     if traffic is not None:
         roofline["traffic_source"] = traffic_src
 
-    if method == "int8":
+    if method == "int8" and C == 64:
         # the contract's roofline for this variant is HBM (every configuration is memory-bound on paper); the integer-ALU
         # figure explains where the time goes (ncu: the integer pipe is the busiest unit) and is reported beside it
         ops = int8_integer_ops_per_chunk(C, inp.d_k, inp.d_v, gdn.gdn_default_order(C), gdn.gdn_default_residual_steps(C))
@@ -416,7 +419,7 @@ def run_ours(args, rank, world, dist_ctx):
         "config": {"workload": args.workload, "method": method, "B": inp.B, "H_k": inp.H_k, "H_v": inp.H_v, "T": inp.T, "C": C, "d_k": inp.d_k,
                    "d_v": inp.d_v, "order": gdn.gdn_default_order(C), "residual_steps": gdn.gdn_default_residual_steps(C),
                    "chunks_per_gpu": n_chunks, "parallelism": f"independent shards x{world}, no collective",
-                   "untimed_launches_before_timing": n_untimed + 2,
+                   "untimed_launches_before_timing": (n_untimed + 3) * per_call,
                    "l2_policy": "inputs+outputs %.0f MB per step, larger than the 126 MB L2" % (n_chunks * bytes_chunk / 1e6)},
         "effective_tflops": world * n_chunks * flops_chunk / (ms_per_step * 1e-3) / 1e12,
         "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline,
@@ -599,6 +602,18 @@ def run_extras(gdn, gen, dev, args):
         del inp, q, outs
     except Exception as exc:
         out["prefill_gqa:int8"] = {"error": repr(exc)}
+    # INT8 on chunks of 128 tokens (two 64-blocks and the block merge of App. E, Eq. 28: two launches per call)
+    try:
+        inp = gen.make_workload("sweep_c128", device=dev)
+        q = gen.make_int8_inputs(inp)
+        outs = gdn.chunk_prepare_int8(q)
+        fn = lambda: gdn.chunk_prepare_int8(q, outputs=outs)
+        group = inp.H_v // inp.H_k
+        by = inp.C * inp.d_k / group + inp.C * inp.d_v + inp.C * inp.d_k + inp.C * inp.d_v + inp.C * inp.C + 6 * inp.C
+        out["sweep_c128:int8"] = _timed_extra(fn, q.n_chunks, by, hbm_peak, 10, 3)
+        del inp, q, outs
+    except Exception as exc:
+        out["sweep_c128:int8"] = {"error": repr(exc)}
     # INT16 variant (the paper's primary integer precision) on the prefill shapes: two bytes per element
     try:
         inp = gen.make_workload("prefill_gqa", device=dev)

@@ -146,7 +146,16 @@ int gdn_chunk_prepare_fwdsubst(const void* K, const void* V, const float* beta, 
  *   [B,H_v,T/C, C, 8*C + d_k + d_v] int32. Row i of a chunk holds: columns [0, C) the Gram row Kq Kq^T;
  *   columns [(s-1)*C, s*C) for s = 2..8 the row of the power product R_{s-1} Eq (left untouched for powers
  *   that the parameters skip: the caller zeroes the buffer); then d_k columns of Tbq Kq and d_v of Tbq Vq.
- * Supported: C = 64, d_k = d_v = 128, 1 <= order <= 3 (the paper's low-bit limit), residual_steps <= 8.
+ * C = 128 (Sec. 4.3 and App. H: chunks of 128 tokens as 64 x 64 blocks; block formula of App. E, Eq. 28): the three
+ *   blocks of A (A11, A21, A22) are quantised separately from 2 k_exp - 15, the chain above runs on the two diagonal
+ *   blocks, and with the stored blocks holding -A the lower-left block is T21q = Q8(align(X, Toff22q X)),
+ *   X = Q8(align(A21q, A21q Toff11q)); W and U are requantised per 64 rows, the lower rows from the aligned sum of
+ *   T21b Kq_top, T22b Kq_bot and beta_q_i Kq_i (b = the block times beta_q_j, requantised). Shapes then:
+ *   k_exp [B,H_k,T/128], v_exp [B,H_v,T/128]; w_exp_out, u_exp_out [B,H_v,T/128,2] (rows 0..63, rows 64..127);
+ *   Toff_q_out [B,H_v,T/128,128,128] (required: the second of the call's two launches reads the diagonal blocks back
+ *   from it; the upper-right block is written as zeros) with t_exp_out [B,H_v,T/128,3] = exponents of the blocks
+ *   (11, 21, 22); dbg_acc_out must be NULL (GDN_ERR_UNSUPPORTED otherwise).
+ * Supported: C = 64 or 128, d_k = d_v = 128, 1 <= order <= 3 (the paper's low-bit limit), residual_steps <= 8.
  */
 int gdn_chunk_prepare_int8(const int8_t* Kq, const int8_t* Vq, const int32_t* k_exp, const int32_t* v_exp,
                            const uint16_t* beta_q, const int32_t* decay_q,

@@ -289,16 +289,24 @@ def chunk_prepare_int8(q, order=-1, residual_steps=-1, *, want_toff=True, output
     """Convenience wrapper over integer inputs (an `inputs.Int8Inputs` whose tensors live on the GPU).
 
     Returns (Wq, Uq, w_exp, u_exp, Toff_q, t_exp). `dbg_acc`: optional zeroed int32 tensor
-    [B, H_v, T/C, C, 8*C + d_k + d_v] that receives the tensor-core accumulators (small cases).
+    [B, H_v, T/C, C, 8*C + d_k + d_v] that receives the tensor-core accumulators (small cases, C = 64).
+    With C = 128 (two 64-blocks per chunk) w_exp, u_exp are [B, H_v, T/128, 2] (rows 0..63, rows 64..127) and t_exp is
+    [B, H_v, T/128, 3] (blocks 11, 21, 22); Toff_q is always produced.
     """
     dev = q.Kq.device
     n_c = q.T // q.C
     if outputs is None:
         Wq = torch.empty(q.B, q.H_v, q.T, q.d_k, dtype=torch.int8, device=dev)
         Uq = torch.empty(q.B, q.H_v, q.T, q.d_v, dtype=torch.int8, device=dev)
-        w_exp = torch.empty(q.B, q.H_v, n_c, dtype=torch.int32, device=dev)
-        u_exp = torch.empty_like(w_exp)
-        t_exp = torch.empty_like(w_exp)
+        if q.C == 128:
+            w_exp = torch.empty(q.B, q.H_v, n_c, 2, dtype=torch.int32, device=dev)
+            u_exp = torch.empty_like(w_exp)
+            t_exp = torch.empty(q.B, q.H_v, n_c, 3, dtype=torch.int32, device=dev)
+            want_toff = True
+        else:
+            w_exp = torch.empty(q.B, q.H_v, n_c, dtype=torch.int32, device=dev)
+            u_exp = torch.empty_like(w_exp)
+            t_exp = torch.empty_like(w_exp)
         Toff = torch.empty(q.B, q.H_v, n_c, q.C, q.C, dtype=torch.int8, device=dev) if want_toff else None
         outputs = (Wq, Uq, w_exp, u_exp, Toff, t_exp)
     Wq, Uq, w_exp, u_exp, Toff, t_exp = outputs

@@ -54,6 +54,9 @@ struct ParamsI8 {
     int* status;
     int H_k, H_v, T, group, n_tt;
     int N, S;
+    int merge;     // 1: the tile is one chunk of 128 tokens whose two 64-blocks this kernel treats as chunks (see below)
+    int8_t* Wq;    // raw output pointers (the block-merge kernel stores rows directly)
+    int8_t* Uq;
     long long n_tiles;
     uint16_t lut[256];
 };
@@ -313,8 +316,10 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             dq = p.decay_q[grow];
         }
         if (chunk_valid) {
-            kexp = p.k_exp[(long long)tc.bhk * n_c + chunk_in_head];
-            vexp = p.v_exp[(long long)tc.bhv * n_c + chunk_in_head];
+            // (chunks of 128 tokens: one input exponent per 128 tokens, shared by the two 64-blocks)
+            const int n_ce = p.merge ? (n_c >> 1) : n_c, ce = p.merge ? (chunk_in_head >> 1) : chunk_in_head;
+            kexp = p.k_exp[(long long)tc.bhk * n_ce + ce];
+            vexp = p.v_exp[(long long)tc.bhv * n_ce + ce];
         }
         if (lane == 0) tma_store_wait_read<0>();
         tc_fence_before_sync();
@@ -775,12 +780,17 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 *reinterpret_cast<uint4*>(line + ((cc ^ ((t >> 1) & 3)) << 4)) = v;
             }
         }
-        if (row_valid && il == 0 && h == 0) p.t_exp[(long long)tc.bhv * n_c + chunk_in_head] = eT;
+        if (row_valid && il == 0 && h == 0) {
+            // chunks of 128 tokens: three exponents per chunk (e11, e21, e22); this kernel writes the diagonal ones
+            const long long ti = p.merge ? (((long long)tc.bhv * (n_c >> 1) + (chunk_in_head >> 1)) * 3 + 2 * (chunk_in_head & 1))
+                                         : ((long long)tc.bhv * n_c + chunk_in_head);
+            p.t_exp[ti] = eT;
+        }
         fence_proxy_async_smem();
         tc_fence_before_sync();
         cta_barrier();
         if (p.Toff != nullptr && h == 0 && lane == 0) {
-            tma_store_3d(&tmT, stage + wrow0 * 64, 0, tc.t0 + wrow0, tc.bhv);
+            tma_store_3d(&tmT, stage + wrow0 * 64, p.merge ? ci * kC : 0, tc.t0 + wrow0, tc.bhv);
             tma_store_commit();
         }
         if (tid == 0) {
@@ -912,6 +922,415 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
     }
 }
 
+// ---------------------------------------------------------------------------------------------------------------
+// Chunks of 128 tokens, second kernel: the lower-left block of T and rows 64..127 of W and U (block formula of
+// App. E, Eq. 28, with this path's sign: T21 = -T22 A21 T11; the stored blocks hold Abar = -A, so T21 = T22 Abar21 T11).
+// The first kernel has treated the two 64-blocks of every chunk as chunks of their own (diagonal blocks of Toffq with
+// their exponents, rows 0..63 of W and U are final). Here, per chunk (one tile of 128 tokens, rows 64..127 do the
+// work: TMEM lanes 64..127):
+//
+//   G = Kq Kq^T (rows 64..127 x columns 0..63 used)                                   MMA
+//   A21q = Q8(-(G o c), 2 k_exp - 15) on the full 64 x 64 block                        integer ALU
+//   X    = Q8(align(A21q, A21q Toff11q));  T21q = Q8(align(X, Toff22q X))              MMA + ALU each
+//   T21b = Q8(T21q_ij beta_q_j), T22b = Q8(Toff22q_ij beta_q_j)                        integer ALU
+//   rows 64..127 of W: Q8(align(T21b Kq_top, T22b Kq_bot, beta_q_i Kq_i)), U likewise   two MMAs (two accumulators) + ALU
+//
+// One CTA per SM (512 TMEM columns: two accumulators of 128 columns and two A operands).
+constexpr uint32_t kMD1 = 0, kMD2 = 128, kMA1 = 256, kMA2 = 288, kMrgTmemCols = 512;
+constexpr int kMOffK = 0, kMOffV = 16384, kMOffEB = 32768, kMOffBeta = 40960, kMOffDecay = kMOffBeta + 512;
+constexpr int kMOffLut = kMOffDecay + 512, kMOffRed = kMOffLut + 512, kMrgSmemTotal = kMOffRed + 128;
+
+__global__ void __launch_bounds__(kThreads, 1)
+int8_merge128_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                     const __grid_constant__ ParamsI8 p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* sK = smem + kMOffK;
+    uint8_t* sV = smem + kMOffV;
+    uint8_t* sEB = smem + kMOffEB;
+    int* sbeta = reinterpret_cast<int*>(smem + kMOffBeta);
+    int* sdecay = reinterpret_cast<int*>(smem + kMOffDecay);
+    uint16_t* slut = reinterpret_cast<uint16_t*>(smem + kMOffLut);
+    uint32_t* sred = reinterpret_cast<uint32_t*>(smem + kMOffRed);
+
+    __shared__ uint64_t bar_k, bar_v, bar_mma;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int s_fail;
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    const int lane = tid & 31;
+    if (tid == 0) {
+        mbar_init(&bar_k, 1);
+        mbar_init(&bar_v, 1);
+        mbar_init(&bar_mma, 1);
+        s_fail = 0;
+        mbar_fence_init();
+        tma_prefetch_desc(&tmK);
+        tma_prefetch_desc(&tmV);
+    }
+    slut[tid] = p.lut[tid];
+    if (warp == 0) {
+        tmem_alloc(&tmem_base_s, kMrgTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = tmem_base_s;
+
+    const uint32_t n_tiles = static_cast<uint32_t>(p.n_tiles);
+    const int n128 = p.T / kTile;
+    const int t = tid & 127;        // tile row = token of the chunk
+    const int h = tid >> 7;         // column half of a 64-wide block
+    const int col0 = h * kHC;
+    const int il = t & (kC - 1);    // row inside its 64-block
+    const int ci = t >> 6;          // 0: rows of the first block, 1: rows of the second block (the workers)
+    const bool worker = ci == 1;
+    const int wq = warp & 3;
+    const uint32_t lane_base = tmem + (static_cast<uint32_t>(wq * 32) << 16);
+    const uint32_t sK_a = smem_u32(sK), sV_a = smem_u32(sV), sEB_a = smem_u32(sEB);
+    const uint32_t idesc_g = instr_desc(128, 128, 1, 1, 0, 0, 2);   // both K-major
+    const uint32_t idesc_b = instr_desc(128, 64, 1, 1, 0, 1, 2);    // B MN-major, N = 64
+    const uint32_t idesc_m = instr_desc(128, 128, 1, 1, 0, 1, 2);   // B MN-major, N = 128
+    uint32_t par_mma = 0, par_kv = 0;
+
+    auto failed = [&]() -> bool { return *reinterpret_cast<volatile int*>(&s_fail) != 0; };
+    auto set_fail = [&]() { *reinterpret_cast<volatile int*>(&s_fail) = 1; };
+    auto wait_mma = [&]() -> bool {
+        if (warp == 0 && (failed() || !wait_bar(&bar_mma, par_mma))) set_fail();
+        asm volatile("bar.sync 2, 256;" ::: "memory");
+        par_mma ^= 1;
+        return !failed();
+    };
+    // bit length of the OR of the workers' magnitudes (the one chunk of the tile); `slot` is fresh per use
+    auto block_bitlen = [&](unsigned long long m, int slot) -> int {
+        const uint32_t lo = __reduce_or_sync(0xFFFFFFFFu, static_cast<uint32_t>(m));
+        const uint32_t hi = __reduce_or_sync(0xFFFFFFFFu, static_cast<uint32_t>(m >> 32));
+        if (lane == 0) {
+            if (lo) atomicOr(&sred[slot * 2 + 0], lo);
+            if (hi) atomicOr(&sred[slot * 2 + 1], hi);
+        }
+        cta_barrier();
+        const unsigned long long all = (static_cast<unsigned long long>(sred[slot * 2 + 1]) << 32) | sred[slot * 2 + 0];
+        return all ? 64 - __clzll(static_cast<long long>(all)) : 0;
+    };
+    // this thread's 32 columns of a row as a piece pair of the B operand [64 x 64] (MN-major, no swizzle): 16 columns of
+    // row k per 16-byte piece, pieces of one column group 1024 bytes apart
+    auto store_b_row = [&](int k, const uint32_t (&w)[8]) {
+#pragma unroll
+        for (int c = 0; c < 2; ++c)
+            *reinterpret_cast<uint4*>(sEB + ((col0 >> 4) + c) * (16 * kC) + k * 16) =
+                make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
+    };
+    // D1 = A1 B with A1 = 64 bytes per row in TMEM, B the [64 x 64] operand above
+    auto issue_block_product = [&]() {
+#pragma unroll
+        for (int ks = 0; ks < kC / 32; ++ks) {
+            const uint64_t bd = smem_desc(sEB_a + ks * 512, 128, 16 * kC, SWZ_NONE);
+            mma_i8_ts(tmem + kMD1, tmem + kMA1 + ks * 8, bd, idesc_b, ks > 0);
+        }
+        mma_commit(&bar_mma);
+    };
+
+    for (uint32_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+        const TileCoord tc = decode_tile(tile, p);
+        const int c128 = tc.t0 / kTile;
+        const long long chunk = (long long)tc.bhv * n128 + c128;
+        const long long grow = (long long)tc.bhv * p.T + tc.t0 + t;
+
+        tc_fence_before_sync();
+        cta_barrier();  // the previous tile is finished with the shared arrays and the accumulators
+        if (tid == 0) {
+            mbar_arrive_expect_tx(&bar_k, 16384);
+            tma_load_3d(sK, &tmK, &bar_k, 0, tc.t0, tc.bhk);
+            mbar_arrive_expect_tx(&bar_v, 16384);
+            tma_load_3d(sV, &tmV, &bar_v, 0, tc.t0, tc.bhv);
+        }
+        const int bq = static_cast<int>(static_cast<uint16_t>(p.beta_q[grow]));
+        const int dq = p.decay_q[grow];
+        const int kexp = p.k_exp[(long long)tc.bhk * n128 + c128];
+        const int vexp = p.v_exp[chunk];
+        const int e11 = p.t_exp[chunk * 3 + 0], e22 = p.t_exp[chunk * 3 + 2];
+        // this row's 32 columns of its own diagonal block of Toffq (written by the first kernel)
+        uint32_t tw[8];
+        {
+            const uint4* src = reinterpret_cast<const uint4*>(p.Toff + (chunk * kTile + t) * kTile + ci * kC + col0);
+            const uint4 v0 = src[0], v1 = src[1];
+            tw[0] = v0.x; tw[1] = v0.y; tw[2] = v0.z; tw[3] = v0.w;
+            tw[4] = v1.x; tw[5] = v1.y; tw[6] = v1.z; tw[7] = v1.w;
+        }
+        if (h == 0) {
+            sbeta[t] = bq;
+            sdecay[t] = dq;
+        }
+        if (tid < 32) sred[tid] = 0u;
+        if (tid == 0) {
+            if (!wait_bar(&bar_k, par_kv)) set_fail();
+            if (!failed()) {
+                tc_fence_after_sync();
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) {
+                    const uint64_t d = smem_desc(sK_a + ks * 32, 16, 1024, SWZ_128B);
+                    mma_i8_ss(tmem + kMD1, d, d, idesc_g, ks > 0);
+                }
+                mma_commit(&bar_mma);
+            }
+        }
+        cta_barrier();
+        if (!wait_mma()) break;
+        tc_fence_after_sync();
+        int slot = 0;
+
+        // ---- A21q = Q8(-(G o c)) on the full block (rows of the second block, columns of the first)
+        int a21[kHC];
+        int eA21;
+        {
+            uint32_t g[kHC];
+            int cq[kHC];
+            uint32_t mlo = 0, mhi = 0;
+            if (worker) {
+                tmem_ld32(lane_base + kMD1 + col0, g);
+                tmem_wait_ld();
+#pragma unroll
+                for (int jl = 0; jl < kHC; ++jl) {
+                    const int dlt = dq - sdecay[col0 + jl];
+                    const int sh = dlt >> 8;
+                    const int gam = (sh >= 0 && sh < 16) ? (static_cast<int>(slut[dlt & 255]) >> sh) : 0;
+                    const int c = (bq * gam + (1 << 14)) >> 15;
+                    cq[jl] = c;
+                    const uint32_t ag = static_cast<uint32_t>(abs(static_cast<int>(g[jl])));
+                    mlo |= ag * static_cast<uint32_t>(c);
+                    mhi |= __umulhi(ag, static_cast<uint32_t>(c));
+                }
+            }
+            const int r = q8_shift(block_bitlen((static_cast<unsigned long long>(mhi) << 32) | mlo, slot++));
+            const uint32_t half = (1u << r) >> 1;
+#pragma unroll
+            for (int jl = 0; jl < kHC; ++jl) a21[jl] = 0;
+            if (worker) {
+                // |G| c needs up to 36 bits: (hi, lo) pair, the rounded shift (r < 32) is one funnel shift; Aq = -G c
+#pragma unroll
+                for (int jl = 0; jl < kHC; ++jl) {
+                    const int gv = static_cast<int>(g[jl]);
+                    const uint32_t ag = static_cast<uint32_t>(abs(gv)), c = static_cast<uint32_t>(cq[jl]);
+                    const uint32_t lo = ag * c, lo2 = lo + half;
+                    const uint32_t hi2 = __umulhi(ag, c) + (lo2 < lo ? 1u : 0u);
+                    const int q = static_cast<int>(min(__funnelshift_r(lo2, hi2, r), 127u));
+                    a21[jl] = (gv < 0) ? q : -q;
+                }
+            }
+            eA21 = 2 * kexp - 15 + r;
+        }
+        // ---- X = Q8(align(A21q, A21q Toff11q)): A operand = rows of A21q, B operand = Toff11q (rows of the first block)
+        {
+            uint32_t w[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) w[i] = worker ? pack4(a21[4 * i], a21[4 * i + 1], a21[4 * i + 2], a21[4 * i + 3]) : 0u;
+            tmem_st8(lane_base + kMA1 + h * 8, w);
+            if (!worker) store_b_row(il, tw);
+            fence_proxy_async_smem();
+            tmem_wait_st();
+            tc_fence_before_sync();
+            cta_barrier();
+            if (tid == 0) {
+                tc_fence_after_sync();
+                issue_block_product();
+            }
+        }
+        if (!wait_mma()) break;
+        tc_fence_after_sync();
+        int x[kHC];
+        int eX;
+        {
+            const int eref = align_ref2(eA21, eA21 + e11);
+            const int sa = eA21 - eref, sp = eA21 + e11 - eref;
+            int acc[kHC];
+            MaxMag mm;
+            if (worker) {
+                uint32_t d[kHC];
+                tmem_ld32(lane_base + kMD1 + col0, d);
+                tmem_wait_ld();
+#pragma unroll
+                for (int jl = 0; jl < kHC; ++jl) acc[jl] = term32(a21[jl], sa) + term32(static_cast<int>(d[jl]), sp);
+#pragma unroll
+                for (int jl = 0; jl < kHC; jl += 2) mm.add2(acc[jl], acc[jl + 1]);
+            }
+            const int r = q8_shift(block_bitlen(mm.mag(), slot++));
+#pragma unroll
+            for (int jl = 0; jl < kHC; ++jl) x[jl] = worker ? q8_32(acc[jl], r) : 0;
+            eX = eref + r;
+        }
+        // ---- T21q = Q8(align(X, Toff22q X)): A operand = rows of Toff22q, B operand = X (rows of the second block)
+        {
+            if (worker) {
+                uint32_t w[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) w[i] = pack4(x[4 * i], x[4 * i + 1], x[4 * i + 2], x[4 * i + 3]);
+                store_b_row(il, w);
+                tmem_st8(lane_base + kMA1 + h * 8, tw);
+            }
+            fence_proxy_async_smem();
+            tmem_wait_st();
+            tc_fence_before_sync();
+            cta_barrier();
+            if (tid == 0) {
+                tc_fence_after_sync();
+                issue_block_product();
+            }
+        }
+        if (!wait_mma()) break;
+        tc_fence_after_sync();
+        int t21[kHC];
+        int e21;
+        {
+            const int eref = align_ref2(eX, e22 + eX);
+            const int s0 = eX - eref, s1 = e22 + eX - eref;
+            int acc[kHC];
+            MaxMag mm;
+            if (worker) {
+                uint32_t d[kHC];
+                tmem_ld32(lane_base + kMD1 + col0, d);
+                tmem_wait_ld();
+#pragma unroll
+                for (int jl = 0; jl < kHC; ++jl) acc[jl] = term32(x[jl], s0) + term32(static_cast<int>(d[jl]), s1);
+#pragma unroll
+                for (int jl = 0; jl < kHC; jl += 2) mm.add2(acc[jl], acc[jl + 1]);
+            }
+            const int r = q8_shift(block_bitlen(mm.mag(), slot++));
+#pragma unroll
+            for (int jl = 0; jl < kHC; ++jl) t21[jl] = worker ? q8_32(acc[jl], r) : 0;
+            e21 = eref + r;
+        }
+        // the lower-left block of Toffq (rows 64..127) and zeros in the upper-right one (rows 0..63)
+        {
+            uint4* dst = reinterpret_cast<uint4*>(p.Toff + (chunk * kTile + t) * kTile + (worker ? 0 : kC) + col0);
+#pragma unroll
+            for (int c = 0; c < 2; ++c)
+                dst[c] = make_uint4(pack4(t21[16 * c + 0], t21[16 * c + 1], t21[16 * c + 2], t21[16 * c + 3]),
+                                    pack4(t21[16 * c + 4], t21[16 * c + 5], t21[16 * c + 6], t21[16 * c + 7]),
+                                    pack4(t21[16 * c + 8], t21[16 * c + 9], t21[16 * c + 10], t21[16 * c + 11]),
+                                    pack4(t21[16 * c + 12], t21[16 * c + 13], t21[16 * c + 14], t21[16 * c + 15]));
+            if (worker && il == 0 && h == 0) p.t_exp[chunk * 3 + 1] = e21;
+        }
+        // ---- T21b = Q8(T21q_ij beta_q_j) (columns of the first block), T22b = Q8(Toff22q_ij beta_q_j) (second block)
+        int e21b, e22b;
+        {
+            int acc1[kHC], acc2[kHC];
+            MaxMag m1, m2;
+            if (worker) {
+#pragma unroll
+                for (int jl = 0; jl < kHC; ++jl) {
+                    acc1[jl] = t21[jl] * sbeta[col0 + jl];
+                    acc2[jl] = byte_at(tw[jl >> 2], jl & 3) * sbeta[kC + col0 + jl];
+                }
+#pragma unroll
+                for (int jl = 0; jl < kHC; jl += 2) {
+                    m1.add2(acc1[jl], acc1[jl + 1]);
+                    m2.add2(acc2[jl], acc2[jl + 1]);
+                }
+            }
+            const int r1 = q8_shift(block_bitlen(m1.mag(), slot++));
+            const int r2 = q8_shift(block_bitlen(m2.mag(), slot++));
+            e21b = e21 - 15 + r1;
+            e22b = e22 - 15 + r2;
+            // A1 = [T21b | 0], A2 = [0 | T22b]: 128 bytes per row (the contraction runs over the 128 tokens of the tile)
+            uint32_t w1[8], w2[8], z[8];
+            const Rnd q1 = make_rnd(r1), q2 = make_rnd(r2);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                z[i] = 0u;
+                w1[i] = worker ? q8_pack4(acc1[4 * i], acc1[4 * i + 1], acc1[4 * i + 2], acc1[4 * i + 3], q1) : 0u;
+                w2[i] = worker ? q8_pack4(acc2[4 * i], acc2[4 * i + 1], acc2[4 * i + 2], acc2[4 * i + 3], q2) : 0u;
+            }
+            tmem_st8(lane_base + kMA1 + h * 8, w1);
+            tmem_st8(lane_base + kMA1 + 16 + h * 8, z);
+            tmem_st8(lane_base + kMA2 + h * 8, z);
+            tmem_st8(lane_base + kMA2 + 16 + h * 8, w2);
+            tmem_wait_st();
+        }
+        // ---- rows 64..127 of W, then of U
+        bool bad = false;
+#pragma unroll 1
+        for (int half = 0; half < 2; ++half) {
+            const int xexp = (half == 0) ? kexp : vexp;
+            const uint8_t* xtile = (half == 0) ? sK : sV;
+            const uint32_t xt_a = (half == 0) ? sK_a : sV_a;
+            tc_fence_before_sync();
+            cta_barrier();  // operands in place (half 0); the accumulators of W have been read (half 1)
+            if (tid == 0) {
+                if (half == 1 && !wait_bar(&bar_v, par_kv)) set_fail();
+                if (!failed()) {
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) {
+                        const uint64_t bd = smem_desc(xt_a + ks * 4096, 16384, 1024, SWZ_128B);
+                        mma_i8_ts(tmem + kMD1, tmem + kMA1 + ks * 8, bd, idesc_m, ks > 0);
+                    }
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) {
+                        const uint64_t bd = smem_desc(xt_a + ks * 4096, 16384, 1024, SWZ_128B);
+                        mma_i8_ts(tmem + kMD2, tmem + kMA2 + ks * 8, bd, idesc_m, ks > 0);
+                    }
+                    mma_commit(&bar_mma);
+                }
+            }
+            if (!wait_mma()) { bad = true; break; }
+            tc_fence_after_sync();
+            const int ep1 = e21b + xexp, ep2 = e22b + xexp, ed = xexp - 15;
+            const int emin = min(ep1, min(ep2, ed)), emax = max(ep1, max(ep2, ed));
+            const int eref = max(emin, emax - kAlignWindow);
+            const int s1 = ep1 - eref, s2 = ep2 - eref, sd = ed - eref;
+            // |T b X| <= 64 * 127^2 < 2^20, |beta_q X| < 2^22; a left shift is at most 8: the sum fits 32 bits
+            int sums[64];
+            MaxMag mm;
+            if (worker) {
+                uint32_t xr[16];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const uint4 v = *reinterpret_cast<const uint4*>(xtile + t * 128 + (((h * 4 + c) ^ (t & 7)) << 4));
+                    xr[4 * c + 0] = v.x; xr[4 * c + 1] = v.y; xr[4 * c + 2] = v.z; xr[4 * c + 3] = v.w;
+                }
+#pragma unroll
+                for (int c0 = 0; c0 < 64; c0 += 32) {
+                    uint32_t d1[32], d2[32];
+                    tmem_ld32(lane_base + kMD1 + h * 64 + c0, d1);
+                    tmem_ld32(lane_base + kMD2 + h * 64 + c0, d2);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        sums[c0 + i] = term32(static_cast<int>(d1[i]), s1) + term32(static_cast<int>(d2[i]), s2) +
+                                       term32(bq * byte_at(xr[(c0 + i) >> 2], (c0 + i) & 3), sd);
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) mm.add2(sums[c0 + i], sums[c0 + i + 1]);
+                }
+            }
+            const int rr = q8_shift(block_bitlen(mm.mag(), slot++));
+            if (worker) {
+                const Rnd rq = make_rnd(rr);
+                if (il == 0 && h == 0) ((half == 0) ? p.w_exp : p.u_exp)[chunk * 2 + 1] = eref + rr;
+                uint4* dst = reinterpret_cast<uint4*>(((half == 0) ? p.Wq : p.Uq) + grow * kD + h * 64);
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    dst[c] = make_uint4(q8_pack4(sums[16 * c + 0], sums[16 * c + 1], sums[16 * c + 2], sums[16 * c + 3], rq),
+                                        q8_pack4(sums[16 * c + 4], sums[16 * c + 5], sums[16 * c + 6], sums[16 * c + 7], rq),
+                                        q8_pack4(sums[16 * c + 8], sums[16 * c + 9], sums[16 * c + 10], sums[16 * c + 11], rq),
+                                        q8_pack4(sums[16 * c + 12], sums[16 * c + 13], sums[16 * c + 14], sums[16 * c + 15], rq));
+            }
+        }
+        if (bad) break;
+        par_kv ^= 1;
+    }
+    if (failed() && tid == 0) atomicExch(p.status, GDN_ERR_TIMEOUT);
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem, kMrgTmemCols);
+    }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -952,7 +1371,11 @@ void int8_decay_lut(uint16_t* out) {
 
 int launch_tc_int8(const ProblemI8& q, cudaStream_t stream) {
     if (q.d_k != kD || q.d_v != kD) return GDN_ERR_UNSUPPORTED;
-    if (q.C != kC) return GDN_ERR_UNSUPPORTED;
+    const bool merge = q.C == 2 * kC;  // chunks of 128 tokens: two 64-blocks, then the block-merge kernel
+    if (q.C != kC && !merge) return GDN_ERR_UNSUPPORTED;
+    if (merge && (q.Toff == nullptr || q.dbg != nullptr || q.T % (2 * kC) != 0)) return GDN_ERR_UNSUPPORTED;
+    if (merge && ((reinterpret_cast<uintptr_t>(q.Toff) | reinterpret_cast<uintptr_t>(q.Wq) | reinterpret_cast<uintptr_t>(q.Uq)) & 15) != 0)
+        return GDN_ERR_ALIGN;
     if (q.order < 1 || q.order > 3) return GDN_ERR_UNSUPPORTED;  // the paper limits the low-bit order to N <= 3
     if (q.steps > kSMax) return GDN_ERR_UNSUPPORTED;
     if ((long long)q.B * q.H_v * q.T == 0) return GDN_OK;
@@ -964,7 +1387,7 @@ int launch_tc_int8(const ProblemI8& q, cudaStream_t stream) {
     if (!make_map(&mV, q.Vq, hv, q.T, kD, 128, 128, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
     if (!make_map(&mW, q.Wq, hv, q.T, kD, 64, 32, CU_TENSOR_MAP_SWIZZLE_64B)) return GDN_ERR_LAUNCH;
     if (!make_map(&mU, q.Uq, hv, q.T, kD, 64, 32, CU_TENSOR_MAP_SWIZZLE_64B)) return GDN_ERR_LAUNCH;
-    if (!make_map(&mT, q.Toff != nullptr ? q.Toff : q.Wq, hv, q.T, q.Toff != nullptr ? kC : kD, 64, 32, CU_TENSOR_MAP_SWIZZLE_64B))
+    if (!make_map(&mT, q.Toff != nullptr ? q.Toff : q.Wq, hv, q.T, q.Toff != nullptr ? q.C : kD, 64, 32, CU_TENSOR_MAP_SWIZZLE_64B))
         return GDN_ERR_LAUNCH;
     ParamsI8 prm;
     prm.beta_q = q.beta_q;
@@ -984,6 +1407,9 @@ int launch_tc_int8(const ProblemI8& q, cudaStream_t stream) {
     prm.n_tt = (q.T + kTile - 1) / kTile;
     prm.N = q.order;
     prm.S = q.steps;
+    prm.merge = merge ? 1 : 0;
+    prm.Wq = q.Wq;
+    prm.Uq = q.Uq;
     prm.n_tiles = hv * prm.n_tt;
     if (prm.n_tiles >= (1LL << 31) - 4096) return GDN_ERR_UNSUPPORTED;
     int8_decay_lut(prm.lut);
@@ -993,6 +1419,15 @@ int launch_tc_int8(const ProblemI8& q, cudaStream_t stream) {
     const long long grid = prm.n_tiles < 2 * 148 ? prm.n_tiles : 2 * 148;
     chunk_tc_int8_kernel<<<static_cast<int>(grid), kThreads, smem, stream>>>(mK, mV, mW, mU, mT, prm);
     count_launch();
+    if (cudaGetLastError() != cudaSuccess) return GDN_ERR_LAUNCH;
+    if (merge) {
+        const int smem2 = kMrgSmemTotal + 1024;
+        if (cudaFuncSetAttribute(int8_merge128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem2) != cudaSuccess)
+            return GDN_ERR_LAUNCH;
+        const long long grid2 = prm.n_tiles < 148 ? prm.n_tiles : 148;
+        int8_merge128_kernel<<<static_cast<int>(grid2), kThreads, smem2, stream>>>(mK, mV, prm);
+        count_launch();
+    }
     return cudaGetLastError() == cudaSuccess ? GDN_OK : GDN_ERR_LAUNCH;
 }
 

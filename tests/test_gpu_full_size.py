@@ -108,6 +108,31 @@ def test_int8_prefill_shapes_at_full_size():
         assert bad.size == 0, f"{key}: {len(bad)} mismatches, first at {bad[0]}"
 
 
+def test_int8_chunks_of_128_at_full_size():
+    """The C = 128 sweep shapes through both launches of the INT8 call, sampled chunks against the integer oracle,
+    and a second call bit for bit."""
+    inp = gen.make_workload("sweep_c128", device="cuda")
+    q = gen.make_int8_inputs(inp)
+    Wq, Uq, w_exp, u_exp, Toff, t_exp = gdn.chunk_prepare_int8(q)
+    again = gdn.chunk_prepare_int8(q)
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+    for a, b in zip((Wq, Uq, w_exp, u_exp, Toff, t_exp), again):
+        assert torch.equal(a, b)
+    ids = _sample_ids(inp, 16, seed=9)
+    Kq, Vq, ke, ve, bq, dq = gen.int8_chunk_slices(q, ids)
+    ref = orq.chunk_prepare_int8_c128(Kq, Vq, ke, ve, bq, dq, gdn.gdn_default_order(q.C), gdn.gdn_default_residual_steps(q.C))
+    n, C = q.n_chunks, q.C
+    idx = torch.as_tensor(ids, device="cuda")
+    got = {
+        "Wq": Wq.reshape(n, C, q.d_k)[idx].cpu().numpy(), "Uq": Uq.reshape(n, C, q.d_v)[idx].cpu().numpy(),
+        "Toffq": Toff.reshape(n, C, C)[idx].cpu().numpy(), "w_exp": w_exp.reshape(n, 2)[idx].cpu().numpy(),
+        "u_exp": u_exp.reshape(n, 2)[idx].cpu().numpy(), "t_exp": t_exp.reshape(n, 3)[idx].cpu().numpy(),
+    }
+    for key in ("t_exp", "Toffq", "w_exp", "Wq", "u_exp", "Uq"):
+        bad = np.argwhere(got[key] != ref[key])
+        assert bad.size == 0, f"{key}: {len(bad)} mismatches, first at {bad[0]}"
+
+
 def test_int16_prefill_shapes_at_full_size():
     from oracle import gdn_oracle_int16 as orq16
     inp = gen.make_workload("prefill_gqa", device="cuda")

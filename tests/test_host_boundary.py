@@ -117,6 +117,8 @@ def test_bad_arguments_are_rejected_without_a_device(lib):
         assert i8(fn, S=-2) == gdn.GDN_ERR_INVALID_ARG
         assert i8(fn, Wq=mis) == gdn.GDN_ERR_ALIGN
         assert i8(fn, dbg=mis) == gdn.GDN_ERR_ALIGN
+    # INT8 on chunks of 128 tokens: T must be a multiple of 128 (the int16 entry point has no such form)
+    assert i8(lib.gdn_chunk_prepare_int8, C=128, T=192) == gdn.GDN_ERR_INVALID_ARG
     assert lib.gdn_chunk_prepare_fwdsubst(p, p, p, p, 1, 1, 1, 128, 32, 128, 128, 1, gdn.GDN_FWDSUBST_BLOCKED_TC, p, p, p, None) in (
         gdn.GDN_ERR_UNSUPPORTED,)
     assert lib.gdn_chunk_prepare_fwdsubst(p, p, p, p, 1, 1, 1, 128, 64, 128, 128, 0, gdn.GDN_FWDSUBST_BLOCKED_TC, p, p, p, None) == \
