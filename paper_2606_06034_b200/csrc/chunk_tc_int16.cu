@@ -742,6 +742,12 @@ chunk_tc_int16_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
             const int ep = eTb + xexp, ed = xexp - 15;
             const int eref = align_ref2(ep, ed);
             const int sp = ep - eref, sd = ed - eref;
+            // The usual case: both terms are shifted left (their exponents are within the 16-bit window of each other), by
+            // little enough that the shifts fold into 32-bit multipliers of the three accumulator words and of the key /
+            // value mantissa: four widening multiply-adds per element instead of the recombination and two general shifts.
+            const bool fold = sp >= 0 && sp <= 14 && sd >= 0 && sd <= 15;
+            const int m_hh = fold ? (1 << (16 + sp)) : 0, m_mid = fold ? (1 << (8 + sp)) : 0, m_ll = fold ? (1 << sp) : 0;
+            const int bqs = fold ? (bq << sd) : 0;
             // pass 1: the scale (bit length of the largest magnitude over the chunk's C x d block)
             unsigned long long m = 0;
 #pragma unroll 1
@@ -753,13 +759,27 @@ chunk_tc_int16_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
                 tmem_ld32(lane_base + kDmid + h * 64 + c0, dmid);
                 tmem_ld32(lane_base + kDll + h * 64 + c0, dll);
                 tmem_wait_ld();
+                if (dbg_row != nullptr) {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const long long pr = combine(dhh[i], dmid[i], dll[i]);
-                    if (dbg_row != nullptr) dbg_row[8 * kC + half * kD + h * 64 + c0 + i] = pr;
-                    const uint32_t xw = xr[i >> 1];
-                    const int x = (i & 1) ? hi16(xw) : lo16(xw);
-                    m |= abs64(term64(pr, sp) + term64((long long)bq * x, sd));
+                    for (int i = 0; i < 32; ++i) dbg_row[8 * kC + half * kD + h * 64 + c0 + i] = combine(dhh[i], dmid[i], dll[i]);
+                }
+                if (fold) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const uint32_t xw = xr[i >> 1];
+                        const int x = (i & 1) ? hi16(xw) : lo16(xw);
+                        const long long v = (long long)static_cast<int>(dhh[i]) * m_hh + (long long)static_cast<int>(dmid[i]) * m_mid +
+                                            (long long)static_cast<int>(dll[i]) * m_ll + (long long)x * bqs;
+                        m |= abs64(v);
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const long long pr = combine(dhh[i], dmid[i], dll[i]);
+                        const uint32_t xw = xr[i >> 1];
+                        const int x = (i & 1) ? hi16(xw) : lo16(xw);
+                        m |= abs64(term64(pr, sp) + term64((long long)bq * x, sd));
+                    }
                 }
             }
             const int rr = q_shift(chunk_bitlen(m, slot++));
@@ -776,12 +796,24 @@ chunk_tc_int16_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
                 tmem_ld32(lane_base + kDll + h * 64 + c0, dll);
                 tmem_wait_ld();
                 uint32_t o[16];
+                if (fold) {
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const uint32_t xw = xr[i];
-                    const long long v0 = term64(combine(dhh[2 * i], dmid[2 * i], dll[2 * i]), sp) + term64((long long)bq * lo16(xw), sd);
-                    const long long v1 = term64(combine(dhh[2 * i + 1], dmid[2 * i + 1], dll[2 * i + 1]), sp) + term64((long long)bq * hi16(xw), sd);
-                    o[i] = pack2(q16(v0, rr), q16(v1, rr));
+                    for (int i = 0; i < 16; ++i) {
+                        const uint32_t xw = xr[i];
+                        const long long v0 = (long long)static_cast<int>(dhh[2 * i]) * m_hh + (long long)static_cast<int>(dmid[2 * i]) * m_mid +
+                                             (long long)static_cast<int>(dll[2 * i]) * m_ll + (long long)lo16(xw) * bqs;
+                        const long long v1 = (long long)static_cast<int>(dhh[2 * i + 1]) * m_hh + (long long)static_cast<int>(dmid[2 * i + 1]) * m_mid +
+                                             (long long)static_cast<int>(dll[2 * i + 1]) * m_ll + (long long)hi16(xw) * bqs;
+                        o[i] = pack2(q16(v0, rr), q16(v1, rr));
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const uint32_t xw = xr[i];
+                        const long long v0 = term64(combine(dhh[2 * i], dmid[2 * i], dll[2 * i]), sp) + term64((long long)bq * lo16(xw), sd);
+                        const long long v1 = term64(combine(dhh[2 * i + 1], dmid[2 * i + 1], dll[2 * i + 1]), sp) + term64((long long)bq * hi16(xw), sd);
+                        o[i] = pack2(q16(v0, rr), q16(v1, rr));
+                    }
                 }
                 if (row_valid) {
                     uint4* dst = reinterpret_cast<uint4*>(out + c0);
