@@ -32,10 +32,14 @@ namespace {
 using namespace sm100;
 
 constexpr int kTile = 128;
-constexpr int kThreads = 256;
+constexpr int kNT = 2;                // threads per tile row (they split its 64 chunk columns and its 128 features); 4 also works
+constexpr int kThreads = 128 * kNT;
 constexpr int kD = 128;
-constexpr int kC = 64;     // chunk size handled by this kernel
-constexpr int kHC = 32;    // chunk columns per thread
+constexpr int kC = 64;                // chunk size handled by this kernel
+constexpr int kHC = kC / kNT;         // chunk columns per thread
+constexpr int kW = kHC / 4;           // packed int8 words of a thread's part of a chunk row
+constexpr int kFW = kD / kNT;         // features per thread in the W / U stage
+constexpr int kNB = kHC / 8;          // blocks of eight columns per thread
 constexpr int kSMax = 8;   // largest number of residual terms held in registers
 constexpr int kAlignWindow = 8;  // bits kept below the largest term of an aligned sum: every such sum fits 32 bits
 constexpr uint32_t kR0 = 0, kAS = 128, kTmemCols = 256;
@@ -76,7 +80,7 @@ constexpr int kOffRed = kOffLut + 512;     // OR-reduction slots: [24][2 chunks]
 constexpr int kNumRed = 24;
 constexpr int kSmemTotal = kOffRed + kNumRed * 16;
 
-__device__ __forceinline__ void cta_barrier() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+__device__ __forceinline__ void cta_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory"); }
 
 __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -227,7 +231,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
         tma_prefetch_desc(&tmU);
         tma_prefetch_desc(&tmT);
     }
-    slut[tid] = p.lut[tid];
+    if (tid < 256) slut[tid] = p.lut[tid];
     if (warp == 0) {
         tmem_alloc(&tmem_base_s, kTmemCols);
         tmem_relinquish();
@@ -242,7 +246,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
     const int n_c = p.T / kC;  // chunks per head
 
     const int t = tid & 127;        // tile row
-    const int h = tid >> 7;         // column half
+    const int h = tid >> 7;         // which of the row's kNT threads: columns [h kHC, (h + 1) kHC)
     const int col0 = h * kHC;       // first chunk column of this thread
     const int il = t & (kC - 1);    // row inside the chunk
     const int cb = t - il;          // first tile row of the chunk
@@ -261,7 +265,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
     auto wait_mma = [&]() -> bool {
         if (warp == 0 && (*reinterpret_cast<volatile int*>(&s_fail) != 0 || !wait_bar(&bar_mma, par_mma)))
             *reinterpret_cast<volatile int*>(&s_fail) = 1;
-        asm volatile("bar.sync 2, 256;" ::: "memory");
+        asm volatile("bar.sync 2, %0;" ::"n"(kThreads) : "memory");
         par_mma ^= 1;
         return *reinterpret_cast<volatile int*>(&s_fail) == 0;
     };
@@ -360,7 +364,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
         int eA;
         {
             uint32_t g[kHC];
-            tmem_ld32(lane_base + kR0 + cb + col0, g);
+            tmem_ldn(lane_base + kR0 + cb + col0, g);
             tmem_wait_ld();
             if (dbg_row != nullptr) {
 #pragma unroll
@@ -399,25 +403,23 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
         }
         // Aq bytes to the private row; entries next to the diagonal and right of this half come back from there
         uint8_t* rowa = sRowA + t * 64;
-        {
-            uint4 v0, v1;
-            v0.x = pack4(aq[0], aq[1], aq[2], aq[3]);     v0.y = pack4(aq[4], aq[5], aq[6], aq[7]);
-            v0.z = pack4(aq[8], aq[9], aq[10], aq[11]);   v0.w = pack4(aq[12], aq[13], aq[14], aq[15]);
-            v1.x = pack4(aq[16], aq[17], aq[18], aq[19]); v1.y = pack4(aq[20], aq[21], aq[22], aq[23]);
-            v1.z = pack4(aq[24], aq[25], aq[26], aq[27]); v1.w = pack4(aq[28], aq[29], aq[30], aq[31]);
-            *reinterpret_cast<uint4*>(rowa + col0) = v0;
-            *reinterpret_cast<uint4*>(rowa + col0 + 16) = v1;
-        }
+#pragma unroll
+        for (int c = 0; c < kHC / 16; ++c)
+            *reinterpret_cast<uint4*>(rowa + col0 + 16 * c) =
+                make_uint4(pack4(aq[16 * c + 0], aq[16 * c + 1], aq[16 * c + 2], aq[16 * c + 3]),
+                           pack4(aq[16 * c + 4], aq[16 * c + 5], aq[16 * c + 6], aq[16 * c + 7]),
+                           pack4(aq[16 * c + 8], aq[16 * c + 9], aq[16 * c + 10], aq[16 * c + 11]),
+                           pack4(aq[16 * c + 12], aq[16 * c + 13], aq[16 * c + 14], aq[16 * c + 15]));
         cta_barrier();
         int ab1 = 0, ab2 = 0, ab3 = 0;  // Aq[i][i-1..i-3]
         if (il >= 1) ab1 = static_cast<int>(static_cast<int8_t>(rowa[il - 1]));
         if (il >= 2) ab2 = static_cast<int>(static_cast<int8_t>(rowa[il - 2]));
         if (il >= 3) ab3 = static_cast<int>(static_cast<int8_t>(rowa[il - 3]));
-        int an0 = 0, an1 = 0, an2 = 0;  // Aq[i][32..34] for the left half: the entries right of its columns
-        if (h == 0) {
-            an0 = static_cast<int>(static_cast<int8_t>(rowa[kHC + 0]));
-            an1 = static_cast<int>(static_cast<int8_t>(rowa[kHC + 1]));
-            an2 = static_cast<int>(static_cast<int8_t>(rowa[kHC + 2]));
+        int an0 = 0, an1 = 0, an2 = 0;  // the three entries of the row right of this thread's columns
+        if (h < kNT - 1) {
+            an0 = static_cast<int>(static_cast<int8_t>(rowa[col0 + kHC + 0]));
+            an1 = static_cast<int>(static_cast<int8_t>(rowa[col0 + kHC + 1]));
+            an2 = static_cast<int>(static_cast<int8_t>(rowa[col0 + kHC + 2]));
         }
         // P_1 = band of Aq: zero beyond distance N
         const int p11 = ab1, p12 = (N >= 2) ? ab2 : 0, p13 = (N >= 3) ? ab3 : 0;
@@ -520,8 +522,8 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
 #pragma unroll
         for (int w = 0; w < kHC / 4; ++w) r1[w] = cur[w] = 0u;
         auto park_col = [&](int s) -> uint32_t {  // TMEM column of the parked row of R_s (s >= 1)
-            return (s >= 2 && s <= 7) ? static_cast<uint32_t>(160 + (s - 2) * 16 + h * 8)
-                                      : static_cast<uint32_t>(kR0 + (s == 1 ? 0 : 16) + h * 8);
+            return (s >= 2 && s <= 7) ? static_cast<uint32_t>(160 + (s - 2) * 16 + h * kW)
+                                      : static_cast<uint32_t>(kR0 + (s == 1 ? 0 : 16) + h * kW);
         };
         // Structural support: R_s is zero for i - j < s (N + 1), so of this thread's four blocks of eight columns only the
         // first live_blocks(s) can hold a non-zero entry in any of the warp's 32 rows (a warp-uniform count; the warp
@@ -531,7 +533,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
         const bool walk_all = p.dbg != nullptr;
         auto live_blocks = [&](int s) -> int {
             const int x = row_max - col0 - s * (N + 1);
-            return walk_all ? 4 : (x < 0 ? 0 : min(4, (x >> 3) + 1));
+            return walk_all ? kNB : (x < 0 ? 0 : min(kNB, (x >> 3) + 1));
         };
         int n_terms = 0;
         if (S >= 1) {
@@ -550,7 +552,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
 #pragma unroll 1
         for (int s = 2; s <= kSMax; ++s) {
             if (s > S || s * (N + 1) >= kC) break;
-            tmem_st8(lane_base + kAS + h * 8, cur);
+            tmem_stn(lane_base + kAS + h * kW, cur);
             fence_proxy_async_smem();
             tmem_wait_st();
             tc_fence_before_sync();
@@ -567,7 +569,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             if (!wait_mma()) { ok = false; break; }
             tc_fence_after_sync();
             uint32_t dres[kHC];
-            tmem_ld32(lane_base + kR0 + cb + col0, dres);
+            tmem_ldn(lane_base + kR0 + cb + col0, dres);
             tmem_wait_ld();
             if (dbg_row != nullptr) {
 #pragma unroll
@@ -580,7 +582,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             {
                 MaxMag mm;
 #pragma unroll
-                for (int b = 0; b < 4; ++b) {
+                for (int b = 0; b < kNB; ++b) {
                     if (b < nb) {
 #pragma unroll
                         for (int jl = 8 * b; jl < 8 * b + 8; jl += 2) mm.add2(static_cast<int>(dres[jl]), static_cast<int>(dres[jl + 1]));
@@ -591,7 +593,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             const int r = q8_shift(chunk_bitlen32(m, slot++));  // (its barrier: every thread has read the accumulator)
             const Rnd rq = make_rnd(r);
 #pragma unroll
-            for (int b = 0; b < 4; ++b) {
+            for (int b = 0; b < kNB; ++b) {
                 cur[2 * b] = cur[2 * b + 1] = 0u;
                 if (b < nb) {
 #pragma unroll
@@ -600,7 +602,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                                           static_cast<int>(dres[4 * w + 2]), static_cast<int>(dres[4 * w + 3]), rq);
                 }
             }
-            tmem_st8(lane_base + park_col(s), cur);
+            tmem_stn(lane_base + park_col(s), cur);
             er[s - 1] = er[s - 2] + eE + r;
             n_terms = s;
         }
@@ -619,7 +621,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             int acc[kHC];
 #pragma unroll
             for (int jl = 0; jl < kHC; ++jl) acc[jl] = 0;
-            tmem_st8(lane_base + park_col(1), r1);
+            tmem_stn(lane_base + park_col(1), r1);
             tmem_wait_st();
 #pragma unroll 1
             for (int s = 1; s <= n_terms; ++s) {
@@ -628,11 +630,11 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 const int nb = live_blocks(s);
                 if (nb == 0) continue;
                 uint32_t w[kHC / 4];
-                tmem_ld8(lane_base + park_col(s), w);
+                tmem_ldn(lane_base + park_col(s), w);
                 tmem_wait_ld();
                 if (sh >= 0) {
 #pragma unroll
-                    for (int b = 0; b < 4; ++b) {
+                    for (int b = 0; b < kNB; ++b) {
                         if (b < nb) {
 #pragma unroll
                             for (int jl = 8 * b; jl < 8 * b + 8; ++jl) acc[jl] += byte_at(w[jl >> 2], jl & 3) << sh;
@@ -640,7 +642,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                     }
                 } else {
 #pragma unroll
-                    for (int b = 0; b < 4; ++b) {
+                    for (int b = 0; b < kNB; ++b) {
                         if (b < nb) {
 #pragma unroll
                             for (int jl = 8 * b; jl < 8 * b + 8; ++jl) acc[jl] += rsr32(byte_at(w[jl >> 2], jl & 3), -sh);
@@ -651,7 +653,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             const int nb1 = live_blocks(1);  // the support of the sum is that of its first term
             MaxMag mm;
 #pragma unroll
-            for (int b = 0; b < 4; ++b) {
+            for (int b = 0; b < kNB; ++b) {
                 if (b < nb1) {
 #pragma unroll
                     for (int jl = 8 * b; jl < 8 * b + 8; jl += 2) mm.add2(acc[jl], acc[jl + 1]);
@@ -661,7 +663,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             const int r = q8_shift(chunk_bitlen32(m, slot++));
             const Rnd rq = make_rnd(r);
 #pragma unroll
-            for (int b = 0; b < 4; ++b) {
+            for (int b = 0; b < kNB; ++b) {
 #pragma unroll
                 for (int jl = 8 * b; jl < 8 * b + 8; ++jl) sq[jl] = 0;
                 if (b < nb1) {
@@ -675,15 +677,13 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             for (int jl = 0; jl < kHC; ++jl) sq[jl] = 0;
         }
         // Sq bytes to the private rows (the rows above are needed for T0q Sq)
-        {
-            uint4 v0, v1;
-            v0.x = pack4(sq[0], sq[1], sq[2], sq[3]);     v0.y = pack4(sq[4], sq[5], sq[6], sq[7]);
-            v0.z = pack4(sq[8], sq[9], sq[10], sq[11]);   v0.w = pack4(sq[12], sq[13], sq[14], sq[15]);
-            v1.x = pack4(sq[16], sq[17], sq[18], sq[19]); v1.y = pack4(sq[20], sq[21], sq[22], sq[23]);
-            v1.z = pack4(sq[24], sq[25], sq[26], sq[27]); v1.w = pack4(sq[28], sq[29], sq[30], sq[31]);
-            *reinterpret_cast<uint4*>(rowa + col0) = v0;
-            *reinterpret_cast<uint4*>(rowa + col0 + 16) = v1;
-        }
+#pragma unroll
+        for (int c = 0; c < kHC / 16; ++c)
+            *reinterpret_cast<uint4*>(rowa + col0 + 16 * c) =
+                make_uint4(pack4(sq[16 * c + 0], sq[16 * c + 1], sq[16 * c + 2], sq[16 * c + 3]),
+                           pack4(sq[16 * c + 4], sq[16 * c + 5], sq[16 * c + 6], sq[16 * c + 7]),
+                           pack4(sq[16 * c + 8], sq[16 * c + 9], sq[16 * c + 10], sq[16 * c + 11]),
+                           pack4(sq[16 * c + 12], sq[16 * c + 13], sq[16 * c + 14], sq[16 * c + 15]));
         cta_barrier();
 
         // ---- I8: Toffq = Q8(align(T0q, Sq, T0q Sq)) on i > j
@@ -697,9 +697,12 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             for (int e = 1; e <= 3; ++e) {
                 const int rr = (t - e) > 0 ? (t - e) : 0;
                 const int cf = (il - e >= 0) ? (e == 1 ? t0q1 : (e == 2 ? t0q2 : t0q3)) : 0;
-                const uint4 a0 = *reinterpret_cast<const uint4*>(sRowA + rr * 64 + col0);
-                const uint4 a1 = *reinterpret_cast<const uint4*>(sRowA + rr * 64 + col0 + 16);
-                const uint32_t w[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+                uint32_t w[kW];
+#pragma unroll
+                for (int c = 0; c < kHC / 16; ++c) {
+                    const uint4 a0 = *reinterpret_cast<const uint4*>(sRowA + rr * 64 + col0 + 16 * c);
+                    w[4 * c] = a0.x; w[4 * c + 1] = a0.y; w[4 * c + 2] = a0.z; w[4 * c + 3] = a0.w;
+                }
 #pragma unroll
                 for (int jl = 0; jl < kHC; ++jl) prod[jl] += cf * byte_at(w[jl >> 2], jl & 3);
             }
@@ -754,16 +757,16 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             }
             const int r = q8_shift(chunk_bitlen32(m, slot++));
             const Rnd rq9 = make_rnd(r);
-            uint32_t r8[8];
+            uint32_t r8[kW];
 #pragma unroll
-            for (int w = 0; w < 8; ++w)
+            for (int w = 0; w < kW; ++w)
                 r8[w] = q8_pack4(acc[4 * w], acc[4 * w + 1], acc[4 * w + 2], acc[4 * w + 3], rq9);
             eTb = eT - 15 + r;
             // row t's block occupies packed columns [cb/4, cb/4 + 16) of a 32-column operand; the other 16 are zero
-            tmem_st8(lane_base + kAS + cb / 4 + h * 8, r8);
+            tmem_stn(lane_base + kAS + cb / 4 + h * kW, r8);
 #pragma unroll
-            for (int w = 0; w < 8; ++w) r8[w] = 0u;
-            tmem_st8(lane_base + kAS + (16 - cb / 4) + h * 8, r8);
+            for (int w = 0; w < kW; ++w) r8[w] = 0u;
+            tmem_stn(lane_base + kAS + (16 - cb / 4) + h * kW, r8);
             tmem_wait_st();
         }
         // Toffq row -> staging (64-byte lines, 64-byte TMA swizzle) -> bulk tensor store of 32 rows per warp (h = 0 issues)
@@ -771,7 +774,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
         if (p.Toff != nullptr) {
             uint8_t* line = stage + t * 64;
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
+            for (int c = 0; c < kHC / 16; ++c) {
                 const int cc = (col0 >> 4) + c;
                 const uint4 v = make_uint4(pack4(toff[16 * c + 0], toff[16 * c + 1], toff[16 * c + 2], toff[16 * c + 3]),
                                            pack4(toff[16 * c + 4], toff[16 * c + 5], toff[16 * c + 6], toff[16 * c + 7]),
@@ -810,10 +813,10 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             const int xexp = (half == 0) ? kexp : vexp;
             const uint8_t* xtile = (half == 0) ? sK : sV;
             // diagonal term beta_q_i * Xq_i for this thread's 64 columns, from its own row of the int8 tile
-            uint32_t xr[16];
+            uint32_t xr[kFW / 4];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const uint4 v = *reinterpret_cast<const uint4*>(xtile + t * 128 + (((h * 4 + c) ^ (t & 7)) << 4));
+            for (int c = 0; c < kFW / 16; ++c) {
+                const uint4 v = *reinterpret_cast<const uint4*>(xtile + t * 128 + (((h * (kFW / 16) + c) ^ (t & 7)) << 4));
                 xr[4 * c + 0] = v.x; xr[4 * c + 1] = v.y; xr[4 * c + 2] = v.z; xr[4 * c + 3] = v.w;
             }
             if (!wait_mma()) { ok = false; break; }
@@ -826,15 +829,15 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             const bool left = sp >= 0 && sd >= 0;  // the usual case: plain left shifts
             const int psc = left ? (1 << sp) : 0, bqs = left ? (bq << sd) : 0;
             MaxMag mmw;
-            int sums[64];  // the aligned sums of this thread's 64 columns stay in registers between the two passes
+            int sums[kFW];  // the aligned sums of this thread's columns stay in registers between the two passes
 #pragma unroll
-            for (int c0 = 0; c0 < 64; c0 += 32) {
+            for (int c0 = 0; c0 < kFW; c0 += 32) {
                 uint32_t r[32];
-                tmem_ld32(lane_base + kR0 + h * 64 + c0, r);
+                tmem_ld32(lane_base + kR0 + h * kFW + c0, r);
                 tmem_wait_ld();
                 if (dbg_row != nullptr) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) dbg_row[8 * kC + half * kD + h * 64 + c0 + i] = static_cast<int>(r[i]);
+                    for (int i = 0; i < 32; ++i) dbg_row[8 * kC + half * kD + h * kFW + c0 + i] = static_cast<int>(r[i]);
                 }
                 if (left) {
                     // shifts folded into the multipliers: two multiply-adds per element
@@ -865,13 +868,16 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             }
             if (row_valid && il == 0 && h == 0)
                 ((half == 0) ? p.w_exp : p.u_exp)[(long long)tc.bhv * n_c + chunk_in_head] = eref + rr;
-            // pass 2: mantissas -> 32 rows x 64 int8 columns of this warp in the 64-byte TMA swizzle:
-            // 2 KB at stage + 8 KB + (wq * 2 + h) * 2 KB
-            uint8_t* sub = stage + 8192 + (wq * 2 + h) * 2048;
-            if (lane == 0) tma_store_wait_read<0>();
-            __syncwarp();
+            // pass 2: mantissas. Two threads per row: 32 rows x 64 int8 columns of this warp in the 64-byte TMA swizzle
+            // (2 KB at stage + 8 KB + (wq * 2 + h) * 2 KB), stored by a bulk tensor store below. Four threads per row:
+            // 32 bytes of the row straight to global memory (a whole 32-byte sector per thread).
+            uint8_t* sub = stage + 8192 + (wq * 2 + (h & 1)) * 2048;
+            if (kNT == 2) {
+                if (lane == 0) tma_store_wait_read<0>();
+                __syncwarp();
+            }
 #pragma unroll
-            for (int c0 = 0; c0 < 64; c0 += 32) {
+            for (int c0 = 0; c0 < kFW; c0 += 32) {
                 const int* qv = sums + c0;
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
@@ -880,7 +886,11 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                                                q8_pack4(qv[16 * c + 4], qv[16 * c + 5], qv[16 * c + 6], qv[16 * c + 7], rqw),
                                                q8_pack4(qv[16 * c + 8], qv[16 * c + 9], qv[16 * c + 10], qv[16 * c + 11], rqw),
                                                q8_pack4(qv[16 * c + 12], qv[16 * c + 13], qv[16 * c + 14], qv[16 * c + 15], rqw));
-                    *reinterpret_cast<uint4*>(sub + lane * 64 + ((cc ^ ((lane >> 1) & 3)) << 4)) = v;
+                    if (kNT == 2) {
+                        *reinterpret_cast<uint4*>(sub + lane * 64 + ((cc ^ ((lane >> 1) & 3)) << 4)) = v;
+                    } else if (row_valid) {
+                        *reinterpret_cast<uint4*>(((half == 0) ? p.Wq : p.Uq) + grow * kD + h * kFW + cc * 16) = v;
+                    }
                 }
             }
             if (half == 0) {
@@ -902,11 +912,13 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                     }
                 }
             }
-            fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) {
-                tma_store_3d((half == 0) ? &tmW : &tmU, sub, h * 64, tc.t0 + wrow0, tc.bhv);
-                tma_store_commit();
+            if (kNT == 2) {
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    tma_store_3d((half == 0) ? &tmW : &tmU, sub, h * 64, tc.t0 + wrow0, tc.bhv);
+                    tma_store_commit();
+                }
             }
         }
         par_kv ^= 1;
@@ -936,11 +948,14 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
 //   rows 64..127 of W: Q8(align(T21b Kq_top, T22b Kq_bot, beta_q_i Kq_i)), U likewise   two MMAs (two accumulators) + ALU
 //
 // One CTA per SM (512 TMEM columns: two accumulators of 128 columns and two A operands).
+constexpr int kMThreads = 256;  // two threads per tile row, 32 columns of a 64-wide block each
+constexpr int kMHC = 32;
+__device__ __forceinline__ void mrg_barrier() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 constexpr uint32_t kMD1 = 0, kMD2 = 128, kMA1 = 256, kMA2 = 288, kMrgTmemCols = 512;
 constexpr int kMOffK = 0, kMOffV = 16384, kMOffEB = 32768, kMOffBeta = 40960, kMOffDecay = kMOffBeta + 512;
 constexpr int kMOffLut = kMOffDecay + 512, kMOffRed = kMOffLut + 512, kMrgSmemTotal = kMOffRed + 128;
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kMThreads, 1)
 int8_merge128_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                      const __grid_constant__ ParamsI8 p) {
     extern __shared__ uint8_t smem_raw[];
@@ -983,7 +998,7 @@ int8_merge128_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
     const int n128 = p.T / kTile;
     const int t = tid & 127;        // tile row = token of the chunk
     const int h = tid >> 7;         // column half of a 64-wide block
-    const int col0 = h * kHC;
+    const int col0 = h * kMHC;
     const int il = t & (kC - 1);    // row inside its 64-block
     const int ci = t >> 6;          // 0: rows of the first block, 1: rows of the second block (the workers)
     const bool worker = ci == 1;
@@ -1011,7 +1026,7 @@ int8_merge128_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             if (lo) atomicOr(&sred[slot * 2 + 0], lo);
             if (hi) atomicOr(&sred[slot * 2 + 1], hi);
         }
-        cta_barrier();
+        mrg_barrier();
         const unsigned long long all = (static_cast<unsigned long long>(sred[slot * 2 + 1]) << 32) | sred[slot * 2 + 0];
         return all ? 64 - __clzll(static_cast<long long>(all)) : 0;
     };
@@ -1040,7 +1055,7 @@ int8_merge128_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
         const long long grow = (long long)tc.bhv * p.T + tc.t0 + t;
 
         tc_fence_before_sync();
-        cta_barrier();  // the previous tile is finished with the shared arrays and the accumulators
+        mrg_barrier();  // the previous tile is finished with the shared arrays and the accumulators
         if (tid == 0) {
             mbar_arrive_expect_tx(&bar_k, 16384);
             tma_load_3d(sK, &tmK, &bar_k, 0, tc.t0, tc.bhk);
@@ -1077,23 +1092,23 @@ int8_merge128_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 mma_commit(&bar_mma);
             }
         }
-        cta_barrier();
+        mrg_barrier();
         if (!wait_mma()) break;
         tc_fence_after_sync();
         int slot = 0;
 
         // ---- A21q = Q8(-(G o c)) on the full block (rows of the second block, columns of the first)
-        int a21[kHC];
+        int a21[kMHC];
         int eA21;
         {
-            uint32_t g[kHC];
-            int cq[kHC];
+            uint32_t g[kMHC];
+            int cq[kMHC];
             uint32_t mlo = 0, mhi = 0;
             if (worker) {
                 tmem_ld32(lane_base + kMD1 + col0, g);
                 tmem_wait_ld();
 #pragma unroll
-                for (int jl = 0; jl < kHC; ++jl) {
+                for (int jl = 0; jl < kMHC; ++jl) {
                     const int dlt = dq - sdecay[col0 + jl];
                     const int sh = dlt >> 8;
                     const int gam = (sh >= 0 && sh < 16) ? (static_cast<int>(slut[dlt & 255]) >> sh) : 0;
@@ -1107,11 +1122,11 @@ int8_merge128_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             const int r = q8_shift(block_bitlen((static_cast<unsigned long long>(mhi) << 32) | mlo, slot++));
             const uint32_t half = (1u << r) >> 1;
 #pragma unroll
-            for (int jl = 0; jl < kHC; ++jl) a21[jl] = 0;
+            for (int jl = 0; jl < kMHC; ++jl) a21[jl] = 0;
             if (worker) {
                 // |G| c needs up to 36 bits: (hi, lo) pair, the rounded shift (r < 32) is one funnel shift; Aq = -G c
 #pragma unroll
-                for (int jl = 0; jl < kHC; ++jl) {
+                for (int jl = 0; jl < kMHC; ++jl) {
                     const int gv = static_cast<int>(g[jl]);
                     const uint32_t ag = static_cast<uint32_t>(abs(gv)), c = static_cast<uint32_t>(cq[jl]);
                     const uint32_t lo = ag * c, lo2 = lo + half;
@@ -1132,7 +1147,7 @@ int8_merge128_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             fence_proxy_async_smem();
             tmem_wait_st();
             tc_fence_before_sync();
-            cta_barrier();
+            mrg_barrier();
             if (tid == 0) {
                 tc_fence_after_sync();
                 issue_block_product();
@@ -1140,25 +1155,25 @@ int8_merge128_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
         }
         if (!wait_mma()) break;
         tc_fence_after_sync();
-        int x[kHC];
+        int x[kMHC];
         int eX;
         {
             const int eref = align_ref2(eA21, eA21 + e11);
             const int sa = eA21 - eref, sp = eA21 + e11 - eref;
-            int acc[kHC];
+            int acc[kMHC];
             MaxMag mm;
             if (worker) {
-                uint32_t d[kHC];
+                uint32_t d[kMHC];
                 tmem_ld32(lane_base + kMD1 + col0, d);
                 tmem_wait_ld();
 #pragma unroll
-                for (int jl = 0; jl < kHC; ++jl) acc[jl] = term32(a21[jl], sa) + term32(static_cast<int>(d[jl]), sp);
+                for (int jl = 0; jl < kMHC; ++jl) acc[jl] = term32(a21[jl], sa) + term32(static_cast<int>(d[jl]), sp);
 #pragma unroll
-                for (int jl = 0; jl < kHC; jl += 2) mm.add2(acc[jl], acc[jl + 1]);
+                for (int jl = 0; jl < kMHC; jl += 2) mm.add2(acc[jl], acc[jl + 1]);
             }
             const int r = q8_shift(block_bitlen(mm.mag(), slot++));
 #pragma unroll
-            for (int jl = 0; jl < kHC; ++jl) x[jl] = worker ? q8_32(acc[jl], r) : 0;
+            for (int jl = 0; jl < kMHC; ++jl) x[jl] = worker ? q8_32(acc[jl], r) : 0;
             eX = eref + r;
         }
         // ---- T21q = Q8(align(X, Toff22q X)): A operand = rows of Toff22q, B operand = X (rows of the second block)
@@ -1173,7 +1188,7 @@ int8_merge128_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             fence_proxy_async_smem();
             tmem_wait_st();
             tc_fence_before_sync();
-            cta_barrier();
+            mrg_barrier();
             if (tid == 0) {
                 tc_fence_after_sync();
                 issue_block_product();
@@ -1181,25 +1196,25 @@ int8_merge128_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
         }
         if (!wait_mma()) break;
         tc_fence_after_sync();
-        int t21[kHC];
+        int t21[kMHC];
         int e21;
         {
             const int eref = align_ref2(eX, e22 + eX);
             const int s0 = eX - eref, s1 = e22 + eX - eref;
-            int acc[kHC];
+            int acc[kMHC];
             MaxMag mm;
             if (worker) {
-                uint32_t d[kHC];
+                uint32_t d[kMHC];
                 tmem_ld32(lane_base + kMD1 + col0, d);
                 tmem_wait_ld();
 #pragma unroll
-                for (int jl = 0; jl < kHC; ++jl) acc[jl] = term32(x[jl], s0) + term32(static_cast<int>(d[jl]), s1);
+                for (int jl = 0; jl < kMHC; ++jl) acc[jl] = term32(x[jl], s0) + term32(static_cast<int>(d[jl]), s1);
 #pragma unroll
-                for (int jl = 0; jl < kHC; jl += 2) mm.add2(acc[jl], acc[jl + 1]);
+                for (int jl = 0; jl < kMHC; jl += 2) mm.add2(acc[jl], acc[jl + 1]);
             }
             const int r = q8_shift(block_bitlen(mm.mag(), slot++));
 #pragma unroll
-            for (int jl = 0; jl < kHC; ++jl) t21[jl] = worker ? q8_32(acc[jl], r) : 0;
+            for (int jl = 0; jl < kMHC; ++jl) t21[jl] = worker ? q8_32(acc[jl], r) : 0;
             e21 = eref + r;
         }
         // the lower-left block of Toffq (rows 64..127) and zeros in the upper-right one (rows 0..63)
@@ -1216,16 +1231,16 @@ int8_merge128_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
         // ---- T21b = Q8(T21q_ij beta_q_j) (columns of the first block), T22b = Q8(Toff22q_ij beta_q_j) (second block)
         int e21b, e22b;
         {
-            int acc1[kHC], acc2[kHC];
+            int acc1[kMHC], acc2[kMHC];
             MaxMag m1, m2;
             if (worker) {
 #pragma unroll
-                for (int jl = 0; jl < kHC; ++jl) {
+                for (int jl = 0; jl < kMHC; ++jl) {
                     acc1[jl] = t21[jl] * sbeta[col0 + jl];
                     acc2[jl] = byte_at(tw[jl >> 2], jl & 3) * sbeta[kC + col0 + jl];
                 }
 #pragma unroll
-                for (int jl = 0; jl < kHC; jl += 2) {
+                for (int jl = 0; jl < kMHC; jl += 2) {
                     m1.add2(acc1[jl], acc1[jl + 1]);
                     m2.add2(acc2[jl], acc2[jl + 1]);
                 }
@@ -1257,7 +1272,7 @@ int8_merge128_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             const uint8_t* xtile = (half == 0) ? sK : sV;
             const uint32_t xt_a = (half == 0) ? sK_a : sV_a;
             tc_fence_before_sync();
-            cta_barrier();  // operands in place (half 0); the accumulators of W have been read (half 1)
+            mrg_barrier();  // operands in place (half 0); the accumulators of W have been read (half 1)
             if (tid == 0) {
                 if (half == 1 && !wait_bar(&bar_v, par_kv)) set_fail();
                 if (!failed()) {
@@ -1425,7 +1440,7 @@ int launch_tc_int8(const ProblemI8& q, cudaStream_t stream) {
         if (cudaFuncSetAttribute(int8_merge128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem2) != cudaSuccess)
             return GDN_ERR_LAUNCH;
         const long long grid2 = prm.n_tiles < 148 ? prm.n_tiles : 148;
-        int8_merge128_kernel<<<static_cast<int>(grid2), kThreads, smem2, stream>>>(mK, mV, prm);
+        int8_merge128_kernel<<<static_cast<int>(grid2), kMThreads, smem2, stream>>>(mK, mV, prm);
         count_launch();
     }
     return cudaGetLastError() == cudaSuccess ? GDN_OK : GDN_ERR_LAUNCH;
