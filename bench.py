@@ -414,7 +414,7 @@ def run_ours(args, rank, world, dist_ctx):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": {"int8": "s8", "int16": "s16"}.get(method, "bf16"),
+        "dtype": {"int8": "s8", "int16": "s16"}.get(method, "f32" if inp.K.dtype == torch.float32 else "bf16"),
         "data": "synthetic", "impl": "ours",
         "config": {"workload": args.workload, "method": method, "B": inp.B, "H_k": inp.H_k, "H_v": inp.H_v, "T": inp.T, "C": C, "d_k": inp.d_k,
                    "d_v": inp.d_v, "order": gdn.gdn_default_order(C), "residual_steps": gdn.gdn_default_residual_steps(C),

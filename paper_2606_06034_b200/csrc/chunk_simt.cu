@@ -2,9 +2,16 @@
 // every matrix of the chunk in shared memory, fp32 arithmetic throughout.
 //
 // It serves the fp32 configuration (tolerance 1e-5 against the fp64 definition), small and
-// odd chunk sizes, and the row-sequential forward-substitution comparison (Eq. 2-3). It follows
-// Alg. 1 step by step with dense products: T0 = mask(sum_{n<=N} Abar^n), E = I - (I - Abar) T0,
-// T = T0 * sum_{s<=S} E^s, and App. E's two-block formula for C = 128.
+// odd chunk sizes, and the forward-substitution comparisons (Eq. 2-3, App. E). The scheme of
+// Sec. 3 is evaluated through its structure rather than as dense products:
+//   * the band L = T0 - I (1 <= i-j <= N) by the distance recursion
+//       L_d[i] = Abar[i][i-d] + sum_{e<d} Abar[i][i-e] L_{d-e}[i-e],
+//     which equals the band of sum_{n<=N} Abar^n (a band entry at distance d only receives powers n <= d);
+//   * E = Abar + Abar L on i-j > N (Eq. 13 with T0 = I + L; exactly zero inside the band), N multiply-adds per entry;
+//   * X_0 = T0, X_{k+1} = T0 + X_k E for k < S (so X_S = T0 sum_{s<=S} E^s), every product summed over
+//     j+N+1 <= k <= i only (X is lower triangular, E vanishes for k-j <= N);
+//   * App. E's two-block formula for C = 128.
+// The Gram matrix is accumulated from slices of K staged in shared memory.
 #include "common.cuh"
 
 namespace gdn {
@@ -20,94 +27,65 @@ __device__ __forceinline__ void st(float* p, float v) { *p = v; }
 __device__ __forceinline__ void st(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
 
 constexpr int kThreads = 256;
+constexpr int kSlice = 32;  // features of K staged per step of the Gram accumulation
 
-// Inverse of (I - Abar) for one n x n diagonal block by the paper's scheme (Alg. 1, right product).
-// X: Abar block (ld = ldx); result written to Tout (ld = ldt). w0..w2: n x n work matrices (ld = ldw).
+// Inverse of (I - Abar) for one n x n diagonal block by the truncated scheme (order N, S residual terms).
+// X: Abar block (ld = ldx, strictly lower triangular); result written to Tout (ld = ldt).
+// w0..w2: n x n work matrices (ld = ldw).
 __device__ void neumann_block(const float* X, int ldx, float* Tout, int ldt, float* w0, float* w1, float* w2, int ldw, int n, int N,
                               int S) {
-    float* T0 = w0;
-    float* P = w1;
-    float* Q = w2;
-    // T0 = I + Abar, P = Abar
+    float* T0 = w0;  // I + L, zero outside the band
+    float* E = w1;
+    float* Y = w2;   // second buffer of the rounds
     for (int idx = threadIdx.x; idx < n * n; idx += kThreads) {
         const int i = idx / n, j = idx % n;
-        const float a = X[i * ldx + j];
-        P[i * ldw + j] = a;
-        T0[i * ldw + j] = a + (i == j ? 1.f : 0.f);
+        T0[i * ldw + j] = (i == j) ? 1.f : 0.f;
     }
     __syncthreads();
-    for (int p = 2; p <= N; ++p) {  // P <- P * Abar; T0 += P
-        for (int idx = threadIdx.x; idx < n * n; idx += kThreads) {
-            const int i = idx / n, j = idx % n;
-            float acc = 0.f;
-            for (int k = 0; k < n; ++k) acc = fmaf(P[i * ldw + k], X[k * ldx + j], acc);
-            Q[i * ldw + j] = acc;
-        }
-        __syncthreads();
-        for (int idx = threadIdx.x; idx < n * n; idx += kThreads) {
-            const int i = idx / n, j = idx % n;
-            T0[i * ldw + j] += Q[i * ldw + j];
-        }
-        float* t = P; P = Q; Q = t;
-        __syncthreads();
-    }
-    // band mask 0 <= i - j <= N (Eq. 10)
-    for (int idx = threadIdx.x; idx < n * n; idx += kThreads) {
-        const int i = idx / n, j = idx % n;
-        if (i - j < 0 || i - j > N) T0[i * ldw + j] = 0.f;
-    }
-    __syncthreads();
-    // E = I - (I - Abar) T0 = I - T0 + Abar T0   -> into P ; running power in Q ; sum in Tout
-    for (int idx = threadIdx.x; idx < n * n; idx += kThreads) {
-        const int i = idx / n, j = idx % n;
-        float acc = 0.f;
-        for (int k = 0; k < n; ++k) acc = fmaf(X[i * ldx + k], T0[k * ldw + j], acc);
-        const float e = (i == j ? 1.f : 0.f) - T0[i * ldw + j] + acc;
-        P[i * ldw + j] = e;
-    }
-    __syncthreads();
-    // power sum: Sum = I + E + ... + E^S, kept in Tout; running power R
-    // R lives in Q and a temporary in Tout is not possible, so use registers per element:
-    for (int idx = threadIdx.x; idx < n * n; idx += kThreads) {
-        const int i = idx / n, j = idx % n;
-        const float e = (S >= 1) ? P[i * ldw + j] : 0.f;
-        Q[i * ldw + j] = e;                               // R = E
-        Tout[i * ldt + j] = e + (i == j ? 1.f : 0.f);     // Sum = I + E
-    }
-    __syncthreads();
-    for (int s = 2; s <= S; ++s) {  // R <- R * E (in place needs a temp: compute rows to registers)
-        // each thread computes its elements from the old R, then all write after a barrier
-        float tmp[16];  // n <= 64: at most 64 * 64 / 256 elements per thread
-        int cnt = 0;
-        for (int idx = threadIdx.x; idx < n * n; idx += kThreads) {
-            const int i = idx / n, j = idx % n;
-            float acc = 0.f;
-            for (int k = 0; k < n; ++k) acc = fmaf(Q[i * ldw + k], P[k * ldw + j], acc);
-            tmp[cnt++] = acc;
-        }
-        __syncthreads();
-        cnt = 0;
-        for (int idx = threadIdx.x; idx < n * n; idx += kThreads) {
-            const int i = idx / n, j = idx % n;
-            const float v = tmp[cnt++];
-            Q[i * ldw + j] = v;
-            Tout[i * ldt + j] += v;
+    // band by distance: one row per thread, one barrier per distance (row i needs L_{d-e} of rows i-e)
+    for (int d = 1; d <= N && d < n; ++d) {
+        for (int i = d + threadIdx.x; i < n; i += kThreads) {
+            float acc = X[i * ldx + (i - d)];
+            for (int e = 1; e < d; ++e) acc = fmaf(X[i * ldx + (i - e)], T0[(i - e) * ldw + (i - d)], acc);
+            T0[i * ldw + (i - d)] = acc;
         }
         __syncthreads();
     }
-    // T = T0 * Sum  (Sum in Tout) -> needs a temp: P is free now (E no longer needed)
+    // E on i - j > N: Abar[i][j] + sum_{e=1..N} Abar[i][j+e] L[j+e][j]   (j + e < i always holds there)
     for (int idx = threadIdx.x; idx < n * n; idx += kThreads) {
         const int i = idx / n, j = idx % n;
-        float acc = 0.f;
-        for (int k = 0; k < n; ++k) acc = fmaf(T0[i * ldw + k], Tout[k * ldt + j], acc);
-        P[i * ldw + j] = acc;
+        float e_ij = 0.f;
+        if (i - j > N) {
+            e_ij = X[i * ldx + j];
+            for (int e = 1; e <= N; ++e) e_ij = fmaf(X[i * ldx + j + e], T0[(j + e) * ldw + j], e_ij);
+        }
+        E[i * ldw + j] = e_ij;
+        Tout[i * ldt + j] = T0[i * ldw + j];  // X_0 = T0
     }
     __syncthreads();
-    for (int idx = threadIdx.x; idx < n * n; idx += kThreads) {
-        const int i = idx / n, j = idx % n;
-        Tout[i * ldt + j] = P[i * ldw + j];
+    // X_{k+1} = T0 + X_k E: only entries with i - j > N change; the sum runs over j + N + 1 <= k <= i
+    float* cur = Tout;
+    int ldc = ldt;
+    float* nxt = Y;
+    int ldn = ldw;
+    for (int r = 0; r < S; ++r) {
+        for (int idx = threadIdx.x; idx < n * n; idx += kThreads) {
+            const int i = idx / n, j = idx % n;
+            float acc = T0[i * ldw + j];
+            for (int k = j + N + 1; k <= i; ++k) acc = fmaf(cur[i * ldc + k], E[k * ldw + j], acc);
+            nxt[i * ldn + j] = acc;
+        }
+        __syncthreads();
+        float* tp = cur; cur = nxt; nxt = tp;
+        const int tl = ldc; ldc = ldn; ldn = tl;
     }
-    __syncthreads();
+    if (cur != Tout) {
+        for (int idx = threadIdx.x; idx < n * n; idx += kThreads) {
+            const int i = idx / n, j = idx % n;
+            Tout[i * ldt + j] = cur[i * ldc + j];
+        }
+        __syncthreads();
+    }
 }
 
 template <typename IO>
@@ -128,6 +106,9 @@ __global__ void __launch_bounds__(kThreads) chunk_simt_kernel(const IO* __restri
     float* sbeta = w2 + blk * ldw;  // C
     float* sg = sbeta + C;          // C
     float* srn = sg + C;            // C: 1 / ||K_row|| (1 unless the keys are normalised here)
+    float* swsc = srn + C;          // C: column scale of the W operand (beta / ||K||, times exp(g) for the gated W)
+    float* sKs = swsc + C;          // C x (kSlice + 1): slice of K while the Gram matrix is accumulated
+    __shared__ float swt[kThreads / 32];
 
     const int n_c = T / C;
     const int group = H_v / H_k;
@@ -147,34 +128,58 @@ __global__ void __launch_bounds__(kThreads) chunk_simt_kernel(const IO* __restri
         for (int i = threadIdx.x; i < C; i += kThreads) {
             sbeta[i] = bc[i];
             sg[i] = gc[i];
-            float rn = 1.f;
-            if (flags & GDN_FLAG_K_L2NORM) {
-                float ss = 0.f;
-                for (int d = 0; d < d_k; ++d) {
-                    const float k = to_f32<IO>(Kc + (long long)i * d_k + d);
-                    ss = fmaf(k, k, ss);
-                }
-                rn = rsqrtf(fmaxf(ss, 1e-30f));
-            }
-            srn[i] = rn;
+            srn[i] = 0.f;  // (sum of squares first)
+        }
+        for (int idx = threadIdx.x; idx < C * C; idx += kThreads) {
+            sA[(idx / C) * ld + (idx % C)] = 0.f;
+            sT[(idx / C) * ld + (idx % C)] = 0.f;
         }
         __syncthreads();
-        if ((flags & GDN_FLAG_G_RAW) && threadIdx.x == 0) {
-            // raw log-gates: chunk-local inclusive prefix sum
-            for (int i = 1; i < C; ++i) sg[i] += sg[i - 1];
+        if (flags & GDN_FLAG_G_RAW) {
+            // raw log-gates: chunk-local inclusive prefix sum (C <= 128 <= kThreads): shuffles inside a warp, then the
+            // totals of the warps before it
+            const int i = threadIdx.x, lane = i & 31, wp = i >> 5;
+            float v = (i < C) ? sg[i] : 0.f;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const float u = __shfl_up_sync(0xFFFFFFFFu, v, off);
+                if (lane >= off) v += u;
+            }
+            if (lane == 31) swt[wp] = v;
+            __syncthreads();
+            for (int w = 0; w < wp; ++w) v += swt[w];
+            if (i < C) sg[i] = v;
+            __syncthreads();
+        }
+        // Gram matrix of the chunk's keys, lower triangle, from slices of kSlice features staged in shared memory
+        // (every element of K is read from global memory once); the diagonal gives the row norms
+        for (int d0 = 0; d0 < d_k; d0 += kSlice) {
+            const int dw = min(kSlice, d_k - d0);
+            for (int idx = threadIdx.x; idx < C * dw; idx += kThreads) {
+                const int i = idx / dw, d = idx % dw;
+                sKs[i * (kSlice + 1) + d] = to_f32<IO>(Kc + (long long)i * d_k + d0 + d);
+            }
+            __syncthreads();
+            for (int idx = threadIdx.x; idx < C * C; idx += kThreads) {
+                const int i = idx / C, j = idx % C;
+                if (j > i) continue;
+                float dot = 0.f;
+                for (int d = 0; d < dw; ++d) dot = fmaf(sKs[i * (kSlice + 1) + d], sKs[j * (kSlice + 1) + d], dot);
+                if (i == j) srn[i] += dot;
+                else sA[i * ld + j] += dot;
+            }
+            __syncthreads();
+        }
+        for (int i = threadIdx.x; i < C; i += kThreads) {
+            const float rn = (flags & GDN_FLAG_K_L2NORM) ? rsqrtf(fmaxf(srn[i], 1e-30f)) : 1.f;
+            srn[i] = rn;
+            swsc[i] = sbeta[i] * rn * ((flags & GDN_FLAG_W_GATED) ? expf(sg[i]) : 1.f);
         }
         __syncthreads();
         // Abar = -tril(diag(beta) (K K^T o Gamma), -1)
         for (int idx = threadIdx.x; idx < C * C; idx += kThreads) {
             const int i = idx / C, j = idx % C;
-            float a = 0.f;
-            if (i > j) {
-                float dot = 0.f;
-                for (int d = 0; d < d_k; ++d) dot = fmaf(to_f32<IO>(Kc + (long long)i * d_k + d), to_f32<IO>(Kc + (long long)j * d_k + d), dot);
-                a = -sbeta[i] * expf(sg[i] - sg[j]) * dot * srn[i] * srn[j];
-            }
-            sA[i * ld + j] = a;
-            sT[i * ld + j] = 0.f;
+            if (i > j) sA[i * ld + j] = -sbeta[i] * expf(sg[i] - sg[j]) * sA[i * ld + j] * srn[i] * srn[j];
         }
         __syncthreads();
 
@@ -249,9 +254,7 @@ __global__ void __launch_bounds__(kThreads) chunk_simt_kernel(const IO* __restri
         for (int idx = threadIdx.x; idx < C * d_k; idx += kThreads) {
             const int i = idx / d_k, d = idx % d_k;
             float acc = 0.f;
-            for (int j = 0; j <= i; ++j)
-                acc = fmaf(sT[i * ld + j] * sbeta[j] * srn[j] * ((flags & GDN_FLAG_W_GATED) ? expf(sg[j]) : 1.f),
-                           to_f32<IO>(Kc + (long long)j * d_k + d), acc);
+            for (int j = 0; j <= i; ++j) acc = fmaf(sT[i * ld + j] * swsc[j], to_f32<IO>(Kc + (long long)j * d_k + d), acc);
             st(Wc + (long long)i * d_k + d, acc);
         }
         for (int idx = threadIdx.x; idx < C * d_v; idx += kThreads) {
@@ -281,7 +284,8 @@ int launch_simt(const Problem& p, InverseMode mode, cudaStream_t stream) {
     const long long n_chunks = (long long)p.B * p.H_v * (p.T / C);
     if (n_chunks == 0) return GDN_OK;
     const int blk = (C == 128) ? 64 : C;
-    const size_t smem = sizeof(float) * (2 * (size_t)C * (C + 1) + 3 * (size_t)blk * (blk + 1) + 3 * (size_t)C);
+    const size_t smem = sizeof(float) * (2 * (size_t)C * (C + 1) + 3 * (size_t)blk * (blk + 1) + 4 * (size_t)C +
+                                         (size_t)C * (kSlice + 1));
     const int grid = (int)(n_chunks < 148LL * 8 ? n_chunks : 148LL * 8);
     cudaError_t e;
     if (p.dtype == GDN_DTYPE_FP32) {
