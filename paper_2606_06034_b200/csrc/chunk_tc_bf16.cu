@@ -289,7 +289,7 @@ __device__ __forceinline__ void load_diag_block(uint32_t lane_base, uint32_t col
 // hi (slot AS) = bf16(T diag(scale)) over the whole row, lo (slot R2) = bf16 of what hi loses on the diagonal and
 // the band, where entries are O(1). `sc` is the per-token scale in shared memory, `sc_i` the row's own scale;
 // a[] = far part of the row, lb[] = band, y[] = T21 part (second block of a 128-chunk).
-template <int C, int NB, bool MERGE, bool YPART = MERGE>
+template <int C, int NB, bool MERGE, bool YPART = MERGE, bool KEEP = true>
 __device__ __forceinline__ void build_wu_operands(uint32_t lane_base, uint32_t br_line, const uint32_t (&slot)[NB + 1], int t, int h,
                                                   int il, int cb, int col0, int wq, const float* sc, float sc_i,
                                                   const float (&a)[Split<C>::HC],
@@ -312,8 +312,9 @@ __device__ __forceinline__ void build_wu_operands(uint32_t lane_base, uint32_t b
 #pragma unroll
     for (int i = 0; i < PCH / 2; ++i) {
         const float4 bb = lds128f(sb_a + i * 16);
-        pk[2 * i] = (pack_bf16x2(a[4 * i] * bb.x, a[4 * i + 1] * bb.y) & keep[2 * i]) | bp[2 * i];
-        pk[2 * i + 1] = (pack_bf16x2(a[4 * i + 2] * bb.z, a[4 * i + 3] * bb.w) & keep[2 * i + 1]) | bp[2 * i + 1];
+        const uint32_t w0 = pack_bf16x2(a[4 * i] * bb.x, a[4 * i + 1] * bb.y), w1 = pack_bf16x2(a[4 * i + 2] * bb.z, a[4 * i + 3] * bb.w);
+        pk[2 * i] = (KEEP ? (w0 & keep[2 * i]) : w0) | bp[2 * i];
+        pk[2 * i + 1] = (KEEP ? (w1 & keep[2 * i + 1]) : w1) | bp[2 * i + 1];
     }
     bool plain = true;
     if constexpr (MERGE) {
@@ -526,11 +527,19 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         return *reinterpret_cast<volatile int*>(&s_fail) == 0;
     };
 
-    // tile-invariant per-thread band positions and keep-mask (0 on the band and the diagonal, ones elsewhere)
+    // tile-invariant per-thread band positions and keep-mask (0 on the band and the diagonal, ones elsewhere).
+    // The mask separates the far part of a row from its band where a[] holds the whole row (forward substitution). In
+    // the Neumann path at C = 64 it is not needed (and its 16 registers are): a[] only ever holds E and the sums of the
+    // products with E or its powers, which are exactly zero on the band, the diagonal and above (E is zero for
+    // i - j <= N, every left factor is lower triangular, and sums of exact zeros are zero).
+    constexpr bool kKeepMask = !(MODE == INV_NEUMANN && C == 64);
     uint32_t slot[NB + 1];
     uint32_t keep[PCH];
     band_slots<C, NB>(smem_u32(smem + L::kBR), smem_u32(smem + L::kDummy) + tid * 4, t, il, col0, n_band, slot);
-    if (active) {
+    if (!kKeepMask) {
+#pragma unroll
+        for (int i = 0; i < PCH; ++i) keep[i] = 0xFFFFFFFFu;
+    } else if (active) {
         uint16_t vals[NB + 1];
 #pragma unroll
         for (int e = 0; e <= NB; ++e) vals[e] = 0xFFFFu;
@@ -1167,7 +1176,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                                 for (int i = 0; i < 8; ++i) {
                                     const uint32_t w = (lv == 2 && !kFull) ? pack_bf16x2(__uint_as_float(d[2 * i]), __uint_as_float(d[2 * i + 1]))
                                                                  : pack_bf16x2(a[hh * 16 + 2 * i], a[hh * 16 + 2 * i + 1]);
-                                    pk[i] = (w & keep[hh * 8 + i]) | bpT[hh * 8 + i];
+                                    pk[i] = (kKeepMask ? (w & keep[hh * 8 + i]) : w) | bpT[hh * 8 + i];
                                 }
                                 tmem_st8(a_own + hh * 8, pk);
                             }
@@ -1202,7 +1211,10 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                         for (int i = 0; i < PCH; ++i) pk[i] = bpT[i];
                     } else {
 #pragma unroll
-                        for (int i = 0; i < PCH; ++i) pk[i] = (pack_bf16x2(a[2 * i], a[2 * i + 1]) & keep[i]) | bpT[i];
+                        for (int i = 0; i < PCH; ++i) {
+                            const uint32_t w = pack_bf16x2(a[2 * i], a[2 * i + 1]);
+                            pk[i] = (kKeepMask ? (w & keep[i]) : w) | bpT[i];
+                        }
                     }
                     store_stacked_operand<C>(lane_base + kAS, h, pk);
                     fence_proxy_async_smem();
@@ -1316,7 +1328,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                             const int k = hh * 8 + i;
                             uint32_t w = pack_bf16x2(a[2 * k], a[2 * k + 1]);
                             if (part == 1) w = pack_bf16x2(a[2 * k] - bf16_lo(w), a[2 * k + 1] - bf16_hi(w));
-                            x[i] = (w & keep[k]) | bp[k];
+                            x[i] = (kKeepMask ? (w & keep[k]) : w) | bp[k];
                         }
                         if (wq < 2) {
 #pragma unroll
@@ -1413,7 +1425,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         // ---- A operands for W/U: T diag(scale) = hi + lo, hi over the whole row, lo only on band + diagonal.
         // scale = beta for U; for W it is beta / ||K|| when the keys are normalised on the fly, else beta as well
         if (active) {
-            build_wu_operands<C, NB, MERGE, MERGE && !Y_EARLY>(lane_base, br_line, slot, t, h, il, cb, col0, wq, two_scales ? sbrn : sbeta,
+            build_wu_operands<C, NB, MERGE, MERGE && !Y_EARLY, kKeepMask>(lane_base, br_line, slot, t, h, il, cb, col0, wq, two_scales ? sbrn : sbeta,
                                             two_scales ? sbrn[t] : bi, a, keep, lb, y);
             if constexpr (MERGE) {
                 // I + L again for the Tinv rows: rebuilt here instead of being carried across the merge, where
@@ -1486,10 +1498,10 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 sts128(rowd + (swz<4>(t, c) << 4),
-                       (pack_bf16x2(a[c * 8 + 0], a[c * 8 + 1]) & keep[c * 4 + 0]) | bpT[c * 4 + 0],
-                       (pack_bf16x2(a[c * 8 + 2], a[c * 8 + 3]) & keep[c * 4 + 1]) | bpT[c * 4 + 1],
-                       (pack_bf16x2(a[c * 8 + 4], a[c * 8 + 5]) & keep[c * 4 + 2]) | bpT[c * 4 + 2],
-                       (pack_bf16x2(a[c * 8 + 6], a[c * 8 + 7]) & keep[c * 4 + 3]) | bpT[c * 4 + 3]);
+                       (kKeepMask ? (pack_bf16x2(a[c * 8 + 0], a[c * 8 + 1]) & keep[c * 4 + 0]) : pack_bf16x2(a[c * 8 + 0], a[c * 8 + 1])) | bpT[c * 4 + 0],
+                       (kKeepMask ? (pack_bf16x2(a[c * 8 + 2], a[c * 8 + 3]) & keep[c * 4 + 1]) : pack_bf16x2(a[c * 8 + 2], a[c * 8 + 3])) | bpT[c * 4 + 1],
+                       (kKeepMask ? (pack_bf16x2(a[c * 8 + 4], a[c * 8 + 5]) & keep[c * 4 + 2]) : pack_bf16x2(a[c * 8 + 4], a[c * 8 + 5])) | bpT[c * 4 + 2],
+                       (kKeepMask ? (pack_bf16x2(a[c * 8 + 6], a[c * 8 + 7]) & keep[c * 4 + 3]) : pack_bf16x2(a[c * 8 + 6], a[c * 8 + 7])) | bpT[c * 4 + 3]);
                 if constexpr (Y_EARLY)
                     sts128(rowo + (swz<4>(t, c) << 4), yp[c * 4 + 0], yp[c * 4 + 1], yp[c * 4 + 2], yp[c * 4 + 3]);
                 else
@@ -1511,10 +1523,10 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 #pragma unroll
             for (int c = 0; c < CPT; ++c) {
                 sts128(trow + (swz<CPT>(t, c) << 4),
-                       (pack_bf16x2(a[c * 8 + 0], a[c * 8 + 1]) & keep[c * 4 + 0]) | bpT[c * 4 + 0],
-                       (pack_bf16x2(a[c * 8 + 2], a[c * 8 + 3]) & keep[c * 4 + 1]) | bpT[c * 4 + 1],
-                       (pack_bf16x2(a[c * 8 + 4], a[c * 8 + 5]) & keep[c * 4 + 2]) | bpT[c * 4 + 2],
-                       (pack_bf16x2(a[c * 8 + 6], a[c * 8 + 7]) & keep[c * 4 + 3]) | bpT[c * 4 + 3]);
+                       (kKeepMask ? (pack_bf16x2(a[c * 8 + 0], a[c * 8 + 1]) & keep[c * 4 + 0]) : pack_bf16x2(a[c * 8 + 0], a[c * 8 + 1])) | bpT[c * 4 + 0],
+                       (kKeepMask ? (pack_bf16x2(a[c * 8 + 2], a[c * 8 + 3]) & keep[c * 4 + 1]) : pack_bf16x2(a[c * 8 + 2], a[c * 8 + 3])) | bpT[c * 4 + 1],
+                       (kKeepMask ? (pack_bf16x2(a[c * 8 + 4], a[c * 8 + 5]) & keep[c * 4 + 2]) : pack_bf16x2(a[c * 8 + 4], a[c * 8 + 5])) | bpT[c * 4 + 2],
+                       (kKeepMask ? (pack_bf16x2(a[c * 8 + 6], a[c * 8 + 7]) & keep[c * 4 + 3]) : pack_bf16x2(a[c * 8 + 6], a[c * 8 + 7])) | bpT[c * 4 + 3]);
             }
             fence_proxy_async_smem();
             __syncwarp();
@@ -1566,7 +1578,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 if (two_scales) {
                     // U uses beta where W used beta / ||K|| (or beta exp(g)): rebuild both A operands
                     if (active) {
-                        build_wu_operands<C, NB, MERGE, MERGE && !Y_EARLY>(lane_base, br_line, slot, t, h, il, cb, col0, wq, sbeta, bi, a, keep, lb, y);
+                        build_wu_operands<C, NB, MERGE, MERGE && !Y_EARLY, kKeepMask>(lane_base, br_line, slot, t, h, il, cb, col0, wq, sbeta, bi, a, keep, lb, y);
                         tmem_wait_st();
                     }
                     tc_fence_before_sync();
