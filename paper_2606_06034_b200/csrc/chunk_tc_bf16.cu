@@ -529,10 +529,10 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 
     // tile-invariant per-thread band positions and keep-mask (0 on the band and the diagonal, ones elsewhere).
     // The mask separates the far part of a row from its band where a[] holds the whole row (forward substitution). In
-    // the Neumann path at C = 64 it is not needed (and its 16 registers are): a[] only ever holds E and the sums of the
+    // the Neumann path at C >= 32 (every thread works on its row) it is not needed (and its 16 registers are): a[] only ever holds E and the sums of the
     // products with E or its powers, which are exactly zero on the band, the diagonal and above (E is zero for
     // i - j <= N, every left factor is lower triangular, and sums of exact zeros are zero).
-    constexpr bool kKeepMask = !(MODE == INV_NEUMANN && C == 64);
+    constexpr bool kKeepMask = !(MODE == INV_NEUMANN && C >= 32);
     uint32_t slot[NB + 1];
     uint32_t keep[PCH];
     band_slots<C, NB>(smem_u32(smem + L::kBR), smem_u32(smem + L::kDummy) + tid * 4, t, il, col0, n_band, slot);
@@ -641,6 +641,13 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         if (f_graw && kWarpsPerChunk > 1) {
             const int first = wq - (wq % kWarpsPerChunk);
             for (int w = first; w < wq; ++w) gi_ += swt[w];
+        }
+        if (C == 64 && warp == 0 && has_next && !(EX && f_var) && elect_one()) {
+            // The next tile's K can only land in shared memory once this tile's W products are done with the buffer,
+            // which leaves its load little time before the next Gram product wants it: ask for it in L2 now.
+            const TileCoord nc = tile_coord<EX>(pos_next, p);
+            tma_prefetch_l2_3d(&tmK, nc.kx, nc.t0, nc.kz);
+            tma_prefetch_l2_3d(&tmK, nc.kx + 64, nc.t0, nc.kz);
         }
         if (warp == 0) {
             // G = K K^T into R0..R1 (128 columns)
