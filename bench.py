@@ -455,9 +455,9 @@ def run_ours(args, rank, world, dist_ctx):
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per chunk from the ncu captures summarised under profiles/,
 # scaled to a launch by the number of chunks it processes (traffic grows in proportion: every chunk is read and written once)
 TRAFFIC_PER_CHUNK: dict = {
-    "stress": (2385.07e6 / 32768, "ncu capture of the same workload with one batch entry (32 768 chunks), scaled by the chunks "
+    "stress": (2378.12e6 / 32768, "ncu capture of the same workload with one batch entry (32 768 chunks), scaled by the chunks "
                                   "of the launch (profiles/chunk_tc_kernel_bf16_c64_stress.md)"),
-    "sweep_c64": (248.9e6 / 4096, "ncu capture of this workload (profiles/chunk_tc_kernel_bf16_c64_sweep_c64.md)"),
+    "sweep_c64": (247.93e6 / 4096, "ncu capture of this workload (profiles/chunk_tc_kernel_bf16_c64_sweep_c64.md)"),
     "prefill_gqa": (1029.0e6 / 16384, "ncu capture of this workload (profiles/chunk_tc_kernel_bf16_c64_prefill_gqa.md)"),
 }
 
