@@ -1348,6 +1348,15 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     }
                 }
             }
+            // The far part a[] is not needed during the two products: it is parked in accumulator columns 64..127 of the
+            // row's own lane (the products have N = 64) and comes back for the W / U operands, which frees 32 registers
+            // where the T21 part, its packed halves and the accumulator reads are live.
+            if constexpr (Y_EARLY) {
+                uint32_t pa[HC];
+#pragma unroll
+                for (int j = 0; j < HC; ++j) pa[j] = __float_as_uint(a[j]);
+                tmem_st32(lane_base + kR0 + 64 + h * 32, pa);
+            }
             tmem_wait_st();
 #pragma unroll 1
             for (int step = 0; step < 2; ++step) {
@@ -1429,6 +1438,13 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             }
         }
 
+        if constexpr (MERGE && !EX) {
+            uint32_t pa[HC];
+            tmem_ld32(lane_base + kR0 + 64 + h * 32, pa);
+            tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < HC; ++j) a[j] = __uint_as_float(pa[j]);
+        }
         // ---- A operands for W/U: T diag(scale) = hi + lo, hi over the whole row, lo only on band + diagonal.
         // scale = beta for U; for W it is beta / ||K|| when the keys are normalised on the fly, else beta as well
         if (active) {
