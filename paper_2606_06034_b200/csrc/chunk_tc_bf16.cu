@@ -528,11 +528,12 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     };
 
     // tile-invariant per-thread band positions and keep-mask (0 on the band and the diagonal, ones elsewhere).
-    // The mask separates the far part of a row from its band where a[] holds the whole row (forward substitution). In
-    // the Neumann path at C >= 32 (every thread works on its row) it is not needed (and its 16 registers are): a[] only ever holds E and the sums of the
-    // products with E or its powers, which are exactly zero on the band, the diagonal and above (E is zero for
-    // i - j <= N, every left factor is lower triangular, and sums of exact zeros are zero).
-    constexpr bool kKeepMask = !(MODE == INV_NEUMANN && C >= 32);
+    // The mask cuts the band out of the packed far part of a row before the band words are OR-ed in. At C >= 32 (every
+    // thread works on its row) it is not needed, and its 16 registers are: in the Neumann path a[] only ever holds E and
+    // sums of products with E or its powers, which are exactly zero on the band, the diagonal and above (E is zero for
+    // i - j <= N, every left factor is lower triangular, sums of exact zeros are zero); after a forward substitution
+    // a[] is zeroed there when the rows are read back. At C = 16 it also blanks the rows of the idle half.
+    constexpr bool kKeepMask = C < 32;
     uint32_t slot[NB + 1];
     uint32_t keep[PCH];
     band_slots<C, NB>(smem_u32(smem + L::kBR), smem_u32(smem + L::kDummy) + tid * 4, t, il, col0, n_band, slot);
