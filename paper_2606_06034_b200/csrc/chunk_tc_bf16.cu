@@ -1132,6 +1132,10 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     const uint32_t b_oth = ((co + col0) >> 3) * 1024 + il * 16;
                     const uint32_t idesc_h = instr_desc(128, 64, 1, 1, 0, 1, 1);
                     tmem_st16(a_own, bpT);
+                    // the band words are parked in the idle R2 columns of the row's own lane during the levels (they come
+                    // back 8 at a time with the accumulator reads, and as a whole afterwards): 16 registers less there
+                    constexpr bool kParkBand = !MERGE && EX != 0;  // (in the default instantiation, which has no spills, the extra TMEM reads cost more than they save)
+                    if constexpr (kParkBand) tmem_st16(lane_base + kR2 + h * 16, bpT);
                     compute_barrier();  // E of every row is in shared memory
                     {
                         uint32_t r16[16];
@@ -1168,8 +1172,14 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                         // in two halves of 16 columns, to keep the live registers down
 #pragma unroll
                         for (int hh = 0; hh < 2; ++hh) {
-                            uint32_t d[16];
+                            uint32_t d[16], bph[8];
                             tmem_ld16(d_own + hh * 16, d);
+                            if constexpr (kParkBand) {
+                                if (lv < 3) tmem_ld8(lane_base + kR2 + h * 16 + hh * 8, bph);
+                            } else {
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) bph[i] = bpT[hh * 8 + i];
+                            }
                             tmem_wait_ld();
                             if (lv == 0) {
 #pragma unroll
@@ -1184,7 +1194,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                                 for (int i = 0; i < 8; ++i) {
                                     const uint32_t w = (lv == 2 && !kFull) ? pack_bf16x2(__uint_as_float(d[2 * i]), __uint_as_float(d[2 * i + 1]))
                                                                  : pack_bf16x2(a[hh * 16 + 2 * i], a[hh * 16 + 2 * i + 1]);
-                                    pk[i] = (kKeepMask ? (w & keep[hh * 8 + i]) : w) | bpT[hh * 8 + i];
+                                    pk[i] = (kKeepMask ? (w & keep[hh * 8 + i]) : w) | bph[i];
                                 }
                                 tmem_st8(a_own + hh * 8, pk);
                             }
@@ -1208,6 +1218,10 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                         if (lv < 3) tmem_wait_st();
                     }
                     if (!ok) break;
+                    if constexpr (kParkBand) {
+                        tmem_ld16(lane_base + kR2 + h * 16, bpT);
+                        tmem_wait_ld();
+                    }
                 }
             } else {
             // one product per term: A_k = T0 + Z_k (bf16, TMEM), Z_{k+1} = A_k E, T = T0 + Z_S
