@@ -727,12 +727,12 @@ chunk_tc_int16_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
 #pragma unroll 1
         for (int half = 0; half < 2; ++half) {
             const int xexp = (half == 0) ? kexp : vexp;
-            // diagonal term beta_q_i * Xq_i for this thread's 64 columns, from its own row of the int16 tile (32 columns
+            // diagonal term beta_q_i * Xq_i for this thread's 64 columns, from its own row of the int16 tile (16 columns
             // at a time: the loops over the column blocks are not unrolled)
             const uint8_t* xtile = (half == 0) ? sK16 : sV16;
-            auto load_x32 = [&](int c0, uint32_t (&w)[16]) {
+            auto load_x16 = [&](int c0, uint32_t (&w)[8]) {
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
+                for (int c = 0; c < 2; ++c) {
                     const uint4 v = *reinterpret_cast<const uint4*>(xtile + h * 16384 + t * 128 + ((((c0 >> 3) + c) ^ (t & 7)) << 4));
                     w[4 * c + 0] = v.x; w[4 * c + 1] = v.y; w[4 * c + 2] = v.z; w[4 * c + 3] = v.w;
                 }
@@ -751,21 +751,21 @@ chunk_tc_int16_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
             // pass 1: the scale (bit length of the largest magnitude over the chunk's C x d block)
             unsigned long long m = 0;
 #pragma unroll 1
-            for (int c0 = 0; c0 < 64; c0 += 32) {
-                uint32_t xr[16];
-                load_x32(c0, xr);
-                uint32_t dhh[32], dmid[32], dll[32];
-                tmem_ld32(lane_base + kDhh + h * 64 + c0, dhh);
-                tmem_ld32(lane_base + kDmid + h * 64 + c0, dmid);
-                tmem_ld32(lane_base + kDll + h * 64 + c0, dll);
+            for (int c0 = 0; c0 < 64; c0 += 16) {
+                uint32_t xr[8];
+                load_x16(c0, xr);
+                uint32_t dhh[16], dmid[16], dll[16];
+                tmem_ld16(lane_base + kDhh + h * 64 + c0, dhh);
+                tmem_ld16(lane_base + kDmid + h * 64 + c0, dmid);
+                tmem_ld16(lane_base + kDll + h * 64 + c0, dll);
                 tmem_wait_ld();
                 if (dbg_row != nullptr) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) dbg_row[8 * kC + half * kD + h * 64 + c0 + i] = combine(dhh[i], dmid[i], dll[i]);
+                    for (int i = 0; i < 16; ++i) dbg_row[8 * kC + half * kD + h * 64 + c0 + i] = combine(dhh[i], dmid[i], dll[i]);
                 }
                 if (fold) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
+                    for (int i = 0; i < 16; ++i) {
                         const uint32_t xw = xr[i >> 1];
                         const int x = (i & 1) ? hi16(xw) : lo16(xw);
                         const long long v = (long long)static_cast<int>(dhh[i]) * m_hh + (long long)static_cast<int>(dmid[i]) * m_mid +
@@ -774,7 +774,7 @@ chunk_tc_int16_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
                     }
                 } else {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
+                    for (int i = 0; i < 16; ++i) {
                         const long long pr = combine(dhh[i], dmid[i], dll[i]);
                         const uint32_t xw = xr[i >> 1];
                         const int x = (i & 1) ? hi16(xw) : lo16(xw);
@@ -787,18 +787,18 @@ chunk_tc_int16_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
             // pass 2: mantissas, 64 int16 of this thread's row straight to global memory
             int16_t* out = ((half == 0) ? p.W : p.U) + grow * kD + h * 64;
 #pragma unroll 1
-            for (int c0 = 0; c0 < 64; c0 += 32) {
-                uint32_t xr[16];
-                load_x32(c0, xr);
-                uint32_t dhh[32], dmid[32], dll[32];
-                tmem_ld32(lane_base + kDhh + h * 64 + c0, dhh);
-                tmem_ld32(lane_base + kDmid + h * 64 + c0, dmid);
-                tmem_ld32(lane_base + kDll + h * 64 + c0, dll);
+            for (int c0 = 0; c0 < 64; c0 += 16) {
+                uint32_t xr[8];
+                load_x16(c0, xr);
+                uint32_t dhh[16], dmid[16], dll[16];
+                tmem_ld16(lane_base + kDhh + h * 64 + c0, dhh);
+                tmem_ld16(lane_base + kDmid + h * 64 + c0, dmid);
+                tmem_ld16(lane_base + kDll + h * 64 + c0, dll);
                 tmem_wait_ld();
-                uint32_t o[16];
+                uint32_t o[8];
                 if (fold) {
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) {
+                    for (int i = 0; i < 8; ++i) {
                         const uint32_t xw = xr[i];
                         const long long v0 = (long long)static_cast<int>(dhh[2 * i]) * m_hh + (long long)static_cast<int>(dmid[2 * i]) * m_mid +
                                              (long long)static_cast<int>(dll[2 * i]) * m_ll + (long long)lo16(xw) * bqs;
@@ -808,7 +808,7 @@ chunk_tc_int16_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
                     }
                 } else {
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) {
+                    for (int i = 0; i < 8; ++i) {
                         const uint32_t xw = xr[i];
                         const long long v0 = term64(combine(dhh[2 * i], dmid[2 * i], dll[2 * i]), sp) + term64((long long)bq * lo16(xw), sd);
                         const long long v1 = term64(combine(dhh[2 * i + 1], dmid[2 * i + 1], dll[2 * i + 1]), sp) + term64((long long)bq * hi16(xw), sd);
@@ -818,7 +818,7 @@ chunk_tc_int16_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
                 if (row_valid) {
                     uint4* dst = reinterpret_cast<uint4*>(out + c0);
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) dst[c] = make_uint4(o[4 * c], o[4 * c + 1], o[4 * c + 2], o[4 * c + 3]);
+                    for (int c = 0; c < 2; ++c) dst[c] = make_uint4(o[4 * c], o[4 * c + 1], o[4 * c + 2], o[4 * c + 3]);
                 }
             }
             if (half == 0) {
