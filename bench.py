@@ -458,7 +458,7 @@ TRAFFIC_PER_CHUNK: dict = {
     "stress": (2378.12e6 / 32768, "ncu capture of the same workload with one batch entry (32 768 chunks), scaled by the chunks "
                                   "of the launch (profiles/chunk_tc_kernel_bf16_c64_stress.md)"),
     "sweep_c64": (247.93e6 / 4096, "ncu capture of this workload (profiles/chunk_tc_kernel_bf16_c64_sweep_c64.md)"),
-    "prefill_gqa": (1029.0e6 / 16384, "ncu capture of this workload (profiles/chunk_tc_kernel_bf16_c64_prefill_gqa.md)"),
+    "prefill_gqa": (1024.84e6 / 16384, "ncu capture of this workload (profiles/chunk_tc_kernel_bf16_c64_prefill_gqa.md)"),
 }
 
 
