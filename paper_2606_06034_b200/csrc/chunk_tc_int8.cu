@@ -194,6 +194,8 @@ __device__ __forceinline__ TileCoord decode_tile(uint32_t tile, const ParamsI8& 
     return c;
 }
 
+// DBG: the instantiation that also dumps every tensor-core accumulator (small cases); the normal one carries none of it
+template <bool DBG>
 __global__ void __launch_bounds__(kThreads, 2)
 chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                      const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmU,
@@ -311,7 +313,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
 
         // row of the accumulator dump (debugging aid of small cases; null in normal use)
         constexpr int kDbgRow = 8 * kC + 2 * kD;
-        int32_t* dbg_row = (p.dbg != nullptr && row_valid)
+        int32_t* dbg_row = (DBG && p.dbg != nullptr && row_valid)
                                ? p.dbg + (((long long)tc.bhv * n_c + chunk_in_head) * kC + il) * kDbgRow
                                : nullptr;
         int bq = 0, dq = 0, kexp = 0, vexp = 0;
@@ -366,7 +368,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             uint32_t g[kHC];
             tmem_ldn(lane_base + kR0 + cb + col0, g);
             tmem_wait_ld();
-            if (dbg_row != nullptr) {
+            if (DBG && dbg_row != nullptr) {
 #pragma unroll
                 for (int jl = 0; jl < kHC; ++jl) dbg_row[col0 + jl] = static_cast<int>(g[jl]);
             }
@@ -530,7 +532,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
         // with rows 0..31 and columns 32..63 has none at all). Dead blocks are skipped in the requantisation and in the
         // sum. With the debug output every block is walked (the test reads every accumulator).
         const int row_max = (wrow0 & (kC - 1)) + 31;
-        const bool walk_all = p.dbg != nullptr;
+        const bool walk_all = DBG && p.dbg != nullptr;
         auto live_blocks = [&](int s) -> int {
             const int x = row_max - col0 - s * (N + 1);
             return walk_all ? kNB : (x < 0 ? 0 : min(kNB, (x >> 3) + 1));
@@ -571,7 +573,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             uint32_t dres[kHC];
             tmem_ldn(lane_base + kR0 + cb + col0, dres);
             tmem_wait_ld();
-            if (dbg_row != nullptr) {
+            if (DBG && dbg_row != nullptr) {
 #pragma unroll
                 for (int jl = 0; jl < kHC; ++jl) dbg_row[(s - 1) * kC + col0 + jl] = static_cast<int>(dres[jl]);
             }
@@ -835,7 +837,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 uint32_t r[32];
                 tmem_ld32(lane_base + kR0 + h * kFW + c0, r);
                 tmem_wait_ld();
-                if (dbg_row != nullptr) {
+                if (DBG && dbg_row != nullptr) {
 #pragma unroll
                     for (int i = 0; i < 32; ++i) dbg_row[8 * kC + half * kD + h * kFW + c0 + i] = static_cast<int>(r[i]);
                 }
@@ -1429,10 +1431,12 @@ int launch_tc_int8(const ProblemI8& q, cudaStream_t stream) {
     if (prm.n_tiles >= (1LL << 31) - 4096) return GDN_ERR_UNSUPPORTED;
     int8_decay_lut(prm.lut);
     const int smem = kSmemTotal + 1024;
-    if (cudaFuncSetAttribute(chunk_tc_int8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+    if (cudaFuncSetAttribute(chunk_tc_int8_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+        cudaFuncSetAttribute(chunk_tc_int8_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
         return GDN_ERR_LAUNCH;
     const long long grid = prm.n_tiles < 2 * 148 ? prm.n_tiles : 2 * 148;
-    chunk_tc_int8_kernel<<<static_cast<int>(grid), kThreads, smem, stream>>>(mK, mV, mW, mU, mT, prm);
+    if (q.dbg != nullptr) chunk_tc_int8_kernel<true><<<static_cast<int>(grid), kThreads, smem, stream>>>(mK, mV, mW, mU, mT, prm);
+    else chunk_tc_int8_kernel<false><<<static_cast<int>(grid), kThreads, smem, stream>>>(mK, mV, mW, mU, mT, prm);
     count_launch();
     if (cudaGetLastError() != cudaSuccess) return GDN_ERR_LAUNCH;
     if (merge) {

@@ -183,7 +183,7 @@ def test_hot_kernels_are_built_without_register_spills():
         assert hits[0]["spill_stores"] == 0 and hits[0]["spill_loads"] == 0, (key, hits[0])
         assert hits[0]["registers"] <= 128
     res = gdn_build.kernel_resources("chunk_tc_int8.cu")
-    main = [v for k, v in res.items() if "chunk_tc_int8_kernel" in k]
-    assert len(main) == 1 and main[0]["spill_stores"] == 0 and main[0]["registers"] <= 128
+    main = [v for k, v in res.items() if "chunk_tc_int8_kernel" in k]  # with and without the accumulator dump
+    assert len(main) == 2 and all(v["spill_stores"] == 0 and v["registers"] <= 128 for v in main)
     res = gdn_build.kernel_resources("chunk_state.cu")
     assert all(v["spill_stores"] == 0 for k, v in res.items() if "chunk_state_kernel" in k)
