@@ -689,7 +689,8 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
         cta_barrier();
 
         // ---- I8: Toffq = Q8(align(T0q, Sq, T0q Sq)) on i > j
-        int toff[kHC];
+        int toff[kHC];   // far part of the row (zero on the band)
+        int tband[3];    // Toffq[i][i-1..i-3] (zero where the row or the order has no such entry)
         int eT;
         {
             int prod[kHC];
@@ -712,33 +713,37 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             const int emin = min(e0, min(e1, e2)), emax = max(e0, max(e1, e2));
             const int eref = max(emin, emax - kAlignWindow);
             const int s0 = e0 - eref, s1 = e1 - eref, s2 = e2 - eref;
-            // the band entry and Sq never share an element (band: distance <= N, Sq: distance > N): one value per
-            // element with its own shift; entries below 2^7, the product below 3 * 127^2 < 2^16
+            // The band entries and Sq never share an element (band: distance <= N, Sq: distance > N), and Sq and T0q Sq
+            // are exactly zero on the band, the diagonal and above (Sq by its support, the product because T0q is banded
+            // and lower triangular). So the row's 32 columns take the far formula without any mask, and the (at most
+            // three) band entries of the row are three scalars, T0q alone: entries below 2^7, the product below
+            // 3 * 127^2 < 2^16. The band values are put into the packed rows afterwards, through shared memory.
             const bool left = s0 >= 0 && s1 >= 0 && s2 >= 0;
             int acc[kHC];
             uint32_t m = 0;
+            if (left) {
 #pragma unroll
-            for (int jl = 0; jl < kHC; ++jl) {
-                const int d = il - (col0 + jl);
-                int v = sq[jl];
-                if (d == 1 && N >= 1) v = t0q1;
-                if (d == 2 && N >= 2) v = t0q2;
-                if (d == 3 && N >= 3) v = t0q3;
-                const int a = (d > 0) ? (left ? ((v << ((d <= N) ? s0 : s1)) + (prod[jl] << s2))
-                                              : (term32(v, (d <= N) ? s0 : s1) + term32(prod[jl], s2)))
-                                      : 0;
-                acc[jl] = a;
+                for (int jl = 0; jl < kHC; ++jl) acc[jl] = (sq[jl] << s1) + (prod[jl] << s2);
+            } else {
+#pragma unroll
+                for (int jl = 0; jl < kHC; ++jl) acc[jl] = term32(sq[jl], s1) + term32(prod[jl], s2);
             }
+            const int ab1 = term32(t0q1, s0), ab2 = term32(t0q2, s0), ab3 = term32(t0q3, s0);
             {
                 MaxMag mm;
 #pragma unroll
                 for (int jl = 0; jl < kHC; jl += 2) mm.add2(acc[jl], acc[jl + 1]);
+                mm.add2(ab1, ab2);
+                mm.add2(ab3, 0);
                 m = mm.mag();
             }
             const int r = q8_shift(chunk_bitlen32(m, slot++));
             const Rnd rq = make_rnd(r);
 #pragma unroll
             for (int jl = 0; jl < kHC; ++jl) toff[jl] = q8_32(acc[jl], rq);
+            tband[0] = q8_32(ab1, rq);
+            tband[1] = q8_32(ab2, rq);
+            tband[2] = q8_32(ab3, rq);
             eT = eref + r;
         }
 
@@ -751,10 +756,15 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             for (int jl = 0; jl < kHC; ++jl) {
                 acc[jl] = toff[jl] * sbeta[cb + col0 + jl];
             }
+            int accb[3];  // the band entries times beta of their columns
+#pragma unroll
+            for (int e = 1; e <= 3; ++e) accb[e - 1] = (il - e >= 0) ? tband[e - 1] * sbeta[t - e] : 0;
             {
                 MaxMag mm;
 #pragma unroll
                 for (int jl = 0; jl < kHC; jl += 2) mm.add2(acc[jl], acc[jl + 1]);
+                mm.add2(accb[0], accb[1]);
+                mm.add2(accb[2], 0);
                 m = mm.mag();
             }
             const int r = q8_shift(chunk_bitlen32(m, slot++));
@@ -763,6 +773,21 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
 #pragma unroll
             for (int w = 0; w < kW; ++w)
                 r8[w] = q8_pack4(acc[4 * w], acc[4 * w + 1], acc[4 * w + 2], acc[4 * w + 3], rq9);
+            // the band bytes go in through the row's private shared-memory line (free since the reduction above: every
+            // thread is past its reads of the Sq rows); a thread patches the columns it owns and reads its part back
+#pragma unroll
+            for (int c = 0; c < kHC / 16; ++c)
+                *reinterpret_cast<uint4*>(rowa + col0 + 16 * c) = make_uint4(r8[4 * c], r8[4 * c + 1], r8[4 * c + 2], r8[4 * c + 3]);
+#pragma unroll
+            for (int e = 1; e <= 3; ++e) {
+                const int c = il - e;
+                if (e <= N && c >= col0 && c < col0 + kHC) rowa[c] = static_cast<uint8_t>(q8_32(accb[e - 1], rq9) & 0xFF);
+            }
+#pragma unroll
+            for (int c = 0; c < kHC / 16; ++c) {
+                const uint4 v = *reinterpret_cast<const uint4*>(rowa + col0 + 16 * c);
+                r8[4 * c] = v.x; r8[4 * c + 1] = v.y; r8[4 * c + 2] = v.z; r8[4 * c + 3] = v.w;
+            }
             eTb = eT - 15 + r;
             // row t's block occupies packed columns [cb/4, cb/4 + 16) of a 32-column operand; the other 16 are zero
             tmem_stn(lane_base + kAS + cb / 4 + h * kW, r8);
@@ -783,6 +808,12 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                                            pack4(toff[16 * c + 8], toff[16 * c + 9], toff[16 * c + 10], toff[16 * c + 11]),
                                            pack4(toff[16 * c + 12], toff[16 * c + 13], toff[16 * c + 14], toff[16 * c + 15]));
                 *reinterpret_cast<uint4*>(line + ((cc ^ ((t >> 1) & 3)) << 4)) = v;
+            }
+#pragma unroll
+            for (int e = 1; e <= 3; ++e) {
+                const int c = il - e;
+                if (e <= N && c >= col0 && c < col0 + kHC)
+                    line[(((c >> 4) ^ ((t >> 1) & 3)) << 4) + (c & 15)] = static_cast<uint8_t>(tband[e - 1] & 0xFF);
             }
         }
         if (row_valid && il == 0 && h == 0) {
