@@ -177,6 +177,23 @@ __device__ __forceinline__ int byte_at(uint32_t w, int i) {
     return static_cast<int>(prmt(w, 0u, (sx << 12) | (sx << 8) | (sx << 4) | static_cast<uint32_t>(i)));
 }
 
+// shared-memory loads by 32-bit shared address (a load through a generic pointer pays a 64-bit address computation)
+__device__ __forceinline__ int lds_s32(uint32_t a) {
+    int v;
+    asm volatile("ld.shared.s32 %0, [%1];" : "=r"(v) : "r"(a) : "memory");
+    return v;
+}
+__device__ __forceinline__ int lds_u16(uint32_t a) {
+    uint32_t v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(a) : "memory");
+    return static_cast<int>(v);
+}
+__device__ __forceinline__ int4 lds_v4(uint32_t a) {
+    int4 v;
+    asm volatile("ld.shared.v4.s32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a) : "memory");
+    return v;
+}
+
 struct TileCoord {
     int bhk, bhv, t0;
 };
@@ -257,6 +274,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
     const int wrow0 = wq * 32;
     const uint32_t lane_base = tmem + (static_cast<uint32_t>(wq * 32) << 16);
     const uint32_t sK_a = smem_u32(sK), sV_a = smem_u32(sV), sEB_a = smem_u32(sEB);
+    const uint32_t sdecay_a = smem_u32(sdecay), slut_a = smem_u32(slut), sSH_a = smem_u32(sSH), sbeta_a = smem_u32(sbeta);
     const uint32_t idesc_g = instr_desc(128, 128, 1, 1, 0, 0, 2);  // s8 x s8 -> s32, both K-major
     const uint32_t idesc_m = instr_desc(128, 128, 1, 1, 0, 1, 2);  // B MN-major
     uint32_t par_mma = 0, par_kv = 0;
@@ -381,9 +399,9 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
 #pragma unroll
             for (int jl = 0; jl < kHC; ++jl) {
                 const int j = col0 + jl;
-                const int dlt = dq - sdecay[cb + j];
+                const int dlt = dq - lds_s32(sdecay_a + (cb + j) * 4);
                 const int sh = dlt >> 8;
-                const int gam = (sh >= 0 && sh < 16) ? (static_cast<int>(slut[dlt & 255]) >> sh) : 0;
+                const int gam = (sh >= 0 && sh < 16) ? (lds_u16(slut_a + (dlt & 255) * 2) >> sh) : 0;
                 const int c = (j < il) ? ((bq * gam + (1 << 14)) >> 15) : 0;
                 cq[jl] = c;
                 const uint32_t ag = static_cast<uint32_t>(abs(static_cast<int>(g[jl])));
@@ -493,7 +511,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             uint32_t m = 0;
 #pragma unroll
             for (int jl = 0; jl < kHC; ++jl) {
-                const int4 c4 = *reinterpret_cast<const int4*>(sSH + (cb + col0 + jl) * 4);
+                const int4 c4 = lds_v4(sSH_a + (cb + col0 + jl) * 16);
                 const int a1 = (jl + 1 < kHC) ? aq[(jl + 1 < kHC) ? jl + 1 : 0] : ((jl + 1 == kHC) ? an0 : (jl + 1 == kHC + 1 ? an1 : an2));
                 const int a2 = (jl + 2 < kHC) ? aq[(jl + 2 < kHC) ? jl + 2 : 0] : ((jl + 2 == kHC) ? an0 : (jl + 2 == kHC + 1 ? an1 : an2));
                 const int a3 = (jl + 3 < kHC) ? aq[(jl + 3 < kHC) ? jl + 3 : 0] : ((jl + 3 == kHC) ? an0 : (jl + 3 == kHC + 1 ? an1 : an2));
@@ -703,7 +721,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
                 uint32_t w[kW];
 #pragma unroll
                 for (int c = 0; c < kHC / 16; ++c) {
-                    const uint4 a0 = *reinterpret_cast<const uint4*>(sRowA + rr * 64 + col0 + 16 * c);
+                    const int4 a0 = lds_v4(smem_u32(sRowA) + rr * 64 + col0 + 16 * c);
                     w[4 * c] = a0.x; w[4 * c + 1] = a0.y; w[4 * c + 2] = a0.z; w[4 * c + 3] = a0.w;
                 }
 #pragma unroll
@@ -754,7 +772,7 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             uint32_t m = 0;
 #pragma unroll
             for (int jl = 0; jl < kHC; ++jl) {
-                acc[jl] = toff[jl] * sbeta[cb + col0 + jl];
+                acc[jl] = toff[jl] * lds_s32(sbeta_a + (cb + col0 + jl) * 4);
             }
             int accb[3];  // the band entries times beta of their columns
 #pragma unroll
@@ -844,12 +862,11 @@ chunk_tc_int8_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
 #pragma unroll 1
         for (int half = 0; half < 2; ++half) {
             const int xexp = (half == 0) ? kexp : vexp;
-            const uint8_t* xtile = (half == 0) ? sK : sV;
             // diagonal term beta_q_i * Xq_i for this thread's 64 columns, from its own row of the int8 tile
             uint32_t xr[kFW / 4];
 #pragma unroll
             for (int c = 0; c < kFW / 16; ++c) {
-                const uint4 v = *reinterpret_cast<const uint4*>(xtile + t * 128 + (((h * (kFW / 16) + c) ^ (t & 7)) << 4));
+                const int4 v = lds_v4(((half == 0) ? sK_a : sV_a) + t * 128 + (((h * (kFW / 16) + c) ^ (t & 7)) << 4));
                 xr[4 * c + 0] = v.x; xr[4 * c + 1] = v.y; xr[4 * c + 2] = v.z; xr[4 * c + 3] = v.w;
             }
             if (!wait_mma()) { ok = false; break; }
