@@ -628,7 +628,11 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     if (blockIdx.x < n_tiles) fetch_row(pos_next, bi_next, gi_next, gtok_next);
 
     for (uint32_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-        const TileCoord tc = tile_coord<EX>(pos_next, p);
+        // The tile's coordinates are only needed by the stores at its end. With the optional layouts they are six values:
+        // those instantiations keep the tile's position (three) and form the coordinates there.
+        const TilePos pos_cur = pos_next;
+        TileCoord tc;
+        if constexpr (EX == 0) tc = tile_coord<EX>(pos_next, p);
         tile_advance<EX>(pos_next, p);
         const uint32_t next = tile + gridDim.x;
         const bool has_next = next < n_tiles;
@@ -1507,6 +1511,17 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             }
         }
 
+        if constexpr (EX != 0) {
+            TilePos pc = pos_cur;
+            asm volatile("" : "+r"(pc.gi), "+r"(pc.tt), "+r"(pc.bhk));  // (formed here, not carried from the tile's top)
+            tc = tile_coord<EX>(pc, p);
+        }
+        // With the optional prologue the U operand can differ from the W operand (two_scales) and is rebuilt from the row.
+        // That happens right after the W product completes and BEFORE its accumulator is read, so that the row's
+        // registers are dead while the epilogue holds its 64; the band-row lines must survive until then, so the Tinv
+        // rows are staged in the E-operand region (dead since the last round) instead of over the band-row lines.
+        constexpr bool kEarlyU = EX != 0 && !MERGE;
+        constexpr int kTinvStage = kEarlyU ? L::kEB : L::kBR;
         // ---- T row -> Tinv: each half-row goes to a staging line in the TMA swizzle layout (the band-row
         // region is free now); one bulk tensor store of 32 rows x HC columns per warp, overlapping the W products
         if (f_f32 && p.Tinv != nullptr && active) {
@@ -1570,7 +1585,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
           }
         } else if (p.Tinv != nullptr && active) {
             constexpr int RB = HC * 2;  // bytes per staged half-row
-            const uint32_t stage = smem_u32(smem + L::kBR) + h * (kTile * RB);
+            const uint32_t stage = smem_u32(smem + kTinvStage) + h * (kTile * RB);
             const uint32_t trow = stage + t * RB;
 #pragma unroll
             for (int c = 0; c < CPT; ++c) {
@@ -1583,7 +1598,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) {
-                tma_store_3d(&tmT, smem + L::kBR + h * (kTile * RB) + wrow0 * RB, col0, tc.t0 + wrow0, tc.bhv);
+                tma_store_3d(&tmT, smem + kTinvStage + h * (kTile * RB) + wrow0 * RB, col0, tc.t0 + wrow0, tc.bhv);
                 tma_store_commit();
             }
         }
@@ -1601,6 +1616,14 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     load_tile(sK, &tmK, &bar_k, nc.kx, nc.t0, nc.kz);
                 else
                     load_tile(sV, &tmV, &bar_v, nc.vx, nc.t0, nc.vz);
+            }
+            if constexpr (kEarlyU) {
+                if (half == 0 && two_scales && active) {
+                    // U uses beta where W used beta / ||K|| (or beta exp(g)): both A operands again (the W product has
+                    // completed; the hand-over to the issuing thread is the barrier below)
+                    build_wu_operands<C, NB, MERGE, MERGE && !Y_EARLY, kKeepMask>(lane_base, br_line, slot, t, h, il, cb, col0, wq, sbeta, bi, a, keep, lb, y);
+                    tmem_wait_st();
+                }
             }
             uint32_t o[32];
 #pragma unroll
@@ -1627,7 +1650,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 if (lane == 0) tma_store_wait_read<0>();
                 tc_fence_before_sync();
                 compute_barrier();  // every row of the W accumulator has been read
-                if (two_scales) {
+                if (!kEarlyU && two_scales) {
                     // U uses beta where W used beta / ||K|| (or beta exp(g)): rebuild both A operands
                     if (active) {
                         build_wu_operands<C, NB, MERGE, MERGE && !Y_EARLY, kKeepMask>(lane_base, br_line, slot, t, h, il, cb, col0, wq, sbeta, bi, a, keep, lb, y);
