@@ -87,9 +87,11 @@ typedef void* gdn_stream_t;
 /*
  * The hot path (Sec. 3, Alg. 1, Eq. 7-13; App. E for C = 128): A-build, masked
  * truncated Neumann series, residual power sum, W and U.
- *   dtype GDN_DTYPE_BF16: bf16 K, V, W, U, Tinv; tensor-core kernel; C in {16, 32, 64, 128},
- *                         d_k, d_v = 128, 1 <= order <= 7. fp32 accumulation.
- *   dtype GDN_DTYPE_FP32: fp32 everywhere, plain FMA kernel; 2 <= C <= 64 or C = 128 (two 64-blocks), d_k, d_v <= 256.
+ *   dtype GDN_DTYPE_BF16: bf16 K, V, W, U, Tinv, fp32 accumulation. The tensor-core kernel takes C in {16, 32, 64, 128},
+ *                         d_k = d_v = 128, 1 <= order <= 7 (every configuration of the benchmark); any other shape
+ *                         within the fp32 limits below runs on the plain FMA kernel with bf16 tensors.
+ *   dtype GDN_DTYPE_FP32: fp32 everywhere, plain FMA kernel; 2 <= C <= 64 or C = 128 (two 64-blocks), d_k, d_v <= 256
+ *                         in multiples of 8.
  * Tinv_out may be NULL (the store is skipped). H = H_k = H_v.
  */
 int gdn_chunk_prepare(const void* K, const void* V, const float* beta, const float* g,

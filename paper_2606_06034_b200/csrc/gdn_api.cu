@@ -85,6 +85,16 @@ int run(Problem p, InverseMode mode, cudaStream_t stream) {
         if (p.flags & GDN_FLAG_LAYOUT_BTHD) return GDN_ERR_UNSUPPORTED;  // the token-major layout is built for bf16 only
         return launch_simt(p, mode, stream);
     }
+    // bf16: the tensor-core kernel is built for d_k = d_v = 128, C in {16, 32, 64, 128} and order <= 7. Other shapes
+    // (any 2 <= C <= 64, feature sizes up to 256 in multiples of 8, higher orders) run on the ALU kernel with bf16
+    // tensors and the same fp32 arithmetic; the token-major layout and packed sequences exist on the tensor-core
+    // kernel only.
+    const bool tc_shape = p.d_k == 128 && p.d_v == 128 && (p.C == 16 || p.C == 32 || p.C == 64 || p.C == 128) &&
+                          (!neumann || p.order <= 7);
+    if (!tc_shape) {
+        if ((p.flags & GDN_FLAG_LAYOUT_BTHD) != 0 || p.chunk_start != nullptr) return GDN_ERR_UNSUPPORTED;
+        return launch_simt(p, mode, stream);
+    }
     return launch_tc_bf16(p, mode, stream);
 }
 

@@ -101,6 +101,20 @@ def test_bf16_defaults(C, adv):
     _check(inp, TOL_BF16)
 
 
+@pytest.mark.parametrize("C,d_k,d_v,N,S,adv", [(64, 64, 64, -1, -1, "none"), (64, 256, 64, -1, -1, "all"), (64, 64, 128, 3, 8, "all"),
+                                              (48, 128, 128, 3, 4, "none"), (24, 72, 40, 2, 3, "none"), (64, 128, 128, 9, 2, "none"),
+                                              (128, 64, 64, -1, -1, "all")])
+def test_bf16_shapes_outside_the_tensor_core_kernel(C, d_k, d_v, N, S, adv):
+    """bf16 tensors with feature sizes other than 128, chunk sizes other than 16 / 32 / 64 / 128 or an order above 7
+    run on the plain FMA kernel (bf16 in and out, fp32 arithmetic): same bar as the tensor-core path, grouped heads."""
+    inp = gen.make_inputs(1, 1, 2, 4 * C, C, d_k, d_v, seed=90 + C + d_k, adversarial_heads=adv)
+    assert inp.K.dtype == torch.bfloat16
+    n0 = gdn.gdn_launch_count()
+    _check(inp, TOL_BF16, N, S)
+    assert gdn.gdn_launch_count() == n0 + 1
+    _check(inp, TOL_BF16, method="fwdsubst", exact=True)
+
+
 @pytest.mark.parametrize("C,N,S", [(64, 3, 2), (64, 3, 1), (64, 3, 0), (64, 2, 5), (64, 1, 8), (64, 5, 3), (64, 7, 2),
                                    (32, 4, 3), (32, 3, 7), (16, 3, 2), (16, 2, 1)])
 def test_bf16_other_orders_and_steps(C, N, S):
@@ -299,8 +313,11 @@ def test_argument_errors_on_device():
     args = dict(check=False)
     assert gdn.gdn_chunk_prepare(K, V, beta, g, 1, 1, 128, 48, 128, 128, -1, -1, 1, W, U, Tinv, **args) == gdn.GDN_ERR_INVALID_ARG
     assert gdn.gdn_chunk_prepare(K, V, beta, g, 1, 1, 128, 64, 128, 128, 0, 3, 1, W, U, Tinv, **args) == gdn.GDN_ERR_INVALID_ARG
-    assert gdn.gdn_chunk_prepare(K, V, beta, g, 1, 1, 128, 64, 128, 128, 9, 3, 1, W, U, Tinv, **args) == gdn.GDN_ERR_UNSUPPORTED
-    assert gdn.gdn_chunk_prepare(K, V, beta, g, 1, 1, 128, 64, 96, 128, -1, -1, 1, W, U, Tinv, **args) == gdn.GDN_ERR_UNSUPPORTED
+    # (orders above 7 and other feature sizes run on the plain FMA kernel; these are outside both kernels)
+    assert gdn.gdn_chunk_prepare(K, V, beta, g, 1, 1, 128, 64, 100, 128, -1, -1, 1, W, U, Tinv, **args) == gdn.GDN_ERR_UNSUPPORTED
+    assert gdn.gdn_chunk_prepare(K, V, beta, g, 1, 1, 128, 64, 264, 128, -1, -1, 1, W, U, Tinv, **args) == gdn.GDN_ERR_UNSUPPORTED
+    assert gdn.gdn_chunk_prepare_ex(K, V, beta, g, 1, 1, 1, 128, 64, 64, 64, -1, -1, 1, W, U, Tinv, gdn.GDN_FLAG_LAYOUT_BTHD,
+                                    **args) == gdn.GDN_ERR_UNSUPPORTED  # token-major: tensor-core kernel only
     buf = torch.zeros(129, device="cuda")
     g_misaligned = buf[1:]  # 4 bytes past a 16-byte boundary
     assert gdn.gdn_chunk_prepare(K, V, beta, g_misaligned, 1, 1, 128, 64, 128, 128, -1, -1, 1, W, U, Tinv, **args) == gdn.GDN_ERR_ALIGN
