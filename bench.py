@@ -196,7 +196,9 @@ def parity_report(orc, sample, gpu):
                      "worst_bf16_floor": float(floor.max()), "mean_rel_frobenius": float(err.mean()),
                      "snr_db_worst": float(orc.snr_db(got, ref).min()), "snr_db_mean": float(orc.snr_db(got, ref).mean()),
                      "gpu_vs_exact_inverse_worst": float(orc.rel_frobenius(got, ex).max()),
-                     "scheme_vs_exact_inverse_worst": float(orc.rel_frobenius(ref, ex).max())}
+                     "scheme_vs_exact_inverse_worst": float(orc.rel_frobenius(ref, ex).max()),
+                     # chunks whose bf16 rounding floor alone is above 2e-3, and chunks above 2e-3 whatever the cause
+                     "chunks_with_floor_above_2e-3": int((floor > 2e-3).sum()), "chunks_above_2e-3": int((err > 2e-3).sum())}
     return rep
 
 
