@@ -616,6 +616,9 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             g_out = __ldg(p.g + r);
         }
     };
+    // Token-major tensors: beta and g of consecutive tokens are H_v floats apart, one 32-byte sector per row and array.
+    // Only the thread of a row's first column half fetches them; the other takes them from the shared arrays.
+    constexpr bool kRowHalf = EX == 1 && C >= 32;
     TilePos pos_next = tile_pos<EX>(blockIdx.x, p);  // position of the tile after the one being worked on
     if (!kEarlyLoad && tid == 0 && blockIdx.x < n_tiles) {
         const TileCoord c = tile_coord<EX>(pos_next, p);
@@ -625,7 +628,8 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     // beta and g of the row are fetched one tile ahead
     float bi_next = 0.f, gi_next = 0.f;
     int gtok_next = -1;
-    if (blockIdx.x < n_tiles) fetch_row(pos_next, bi_next, gi_next, gtok_next);
+    if (blockIdx.x < n_tiles && !(kRowHalf && (p.flags & GDN_FLAG_LAYOUT_BTHD) && (threadIdx.x >> 7) == 1))
+        fetch_row(pos_next, bi_next, gi_next, gtok_next);
 
     for (uint32_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
         // The tile's coordinates are only needed by the stores at its end. With the optional layouts they are six values:
@@ -637,7 +641,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         const uint32_t next = tile + gridDim.x;
         const bool has_next = next < n_tiles;
 
-        const float bi = bi_next;  // loaded during the previous tile
+        float bi = bi_next;  // loaded during the previous tile
         float gi_ = gi_next;
         const int gtok = gtok_next;
         constexpr int kWarpsPerChunk = MERGE ? 4 : (C >= 32 ? C / 32 : 1);
@@ -694,6 +698,10 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             }
         }
         compute_barrier();
+        if (kRowHalf && (p.flags & GDN_FLAG_LAYOUT_BTHD) && h == 1) {
+            bi = sbeta[t];
+            gi_ = sg[t];
+        }
 
         // ---- A-build: this thread's part of the row of Abar, from the Gram block in TMEM
         if (!wait_mma()) { ok = false; break; }
@@ -771,7 +779,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         }
         bi_next = 0.f;
         gi_next = 0.f;
-        if (has_next) fetch_row(pos_next, bi_next, gi_next, gtok_next);
+        if (has_next && !(kRowHalf && (p.flags & GDN_FLAG_LAYOUT_BTHD) && h == 1)) fetch_row(pos_next, bi_next, gi_next, gtok_next);
         compute_barrier();  // both halves of every fp32 row are written
 
         float lb[NB + 1];  // lb[d] = L[i][i-d], the band of T0 - I (or of T - I after forward substitution)
