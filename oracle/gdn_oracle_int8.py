@@ -338,9 +338,13 @@ def _bitlen(m: np.ndarray) -> np.ndarray:
 def _rsr_np(x: np.ndarray, r: np.ndarray) -> np.ndarray:
     """Round-half-away right shift by r >= 0 (r broadcastable); r == 0 leaves x unchanged."""
     r = np.asarray(r, dtype=np.int64)
-    half = np.where(r > 0, np.int64(1) << np.maximum(r - 1, 0), 0)
-    a = (np.abs(x) + half) >> r
-    return np.where(x >= 0, a, -a)
+    # int64 cannot hold 2^(r-1) for r >= 64 and numpy's shifts by 64 or more are not the mathematical ones: there the
+    # result is 0, since every value that reaches this function is below 2^62 in magnitude (|x| + 2^(r-1) < 2^r).
+    big = r >= 63
+    rc = np.where(big, 1, r)
+    half = np.where(rc > 0, np.int64(1) << np.maximum(rc - 1, 0), 0)
+    a = (np.abs(x) + half) >> rc
+    return np.where(big, 0, np.where(x >= 0, a, -a))
 
 
 def _shift_np(x: np.ndarray, s: np.ndarray) -> np.ndarray:

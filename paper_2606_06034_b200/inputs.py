@@ -198,6 +198,43 @@ def make_int16_inputs(inp: ChunkInputs) -> Int8Inputs:
     return make_int8_inputs(inp, bits=16)
 
 
+INT_EDGE_CASES = ("all_max", "sign_max", "alt_rows", "one_hot", "max_k_slow_decay", "steep_decay", "exp_extremes",
+                  "zero_k", "zero_beta", "zero_all")
+
+
+def int_edge_inputs(q: Int8Inputs, case: str, bits: int = 8) -> Int8Inputs:
+    """Overwrites integer inputs in place with a saturating or degenerate pattern (edge cases of the integer entry
+    points: largest mantissas with the gate open and beta at its maximum, where the inverse grows by tens of octaves
+    and aligned sums meet shifts far beyond the word size; empty chunks; closed gates; extreme input exponents)."""
+    assert case in INT_EDGE_CASES
+    m = (1 << (bits - 1)) - 1
+    gen = torch.Generator().manual_seed(7)
+    ramp = (torch.arange(q.T) % q.C).to(torch.int32)
+    if case == "all_max":
+        q.Kq.fill_(m); q.Vq.fill_(-m); q.beta_q.fill_(32767); q.decay_q.zero_()
+    elif case == "sign_max":
+        q.Kq.copy_(((torch.randint(0, 2, q.Kq.shape, generator=gen) * 2 - 1) * m).to(q.Kq.dtype))
+        q.Vq.copy_(((torch.randint(0, 2, q.Vq.shape, generator=gen) * 2 - 1) * m).to(q.Vq.dtype))
+        q.beta_q.fill_(32767); q.decay_q.zero_()
+    elif case == "alt_rows":
+        q.Kq.fill_(m); q.Kq[:, :, 1::2] = -m; q.beta_q.fill_(32767); q.decay_q.zero_()
+    elif case == "one_hot":
+        q.Kq.zero_(); q.Kq[..., 0] = m; q.beta_q.fill_(32767); q.decay_q.zero_()
+    elif case == "max_k_slow_decay":
+        q.Kq.fill_(m); q.beta_q.fill_(32767); q.decay_q.copy_((ramp * 3).expand_as(q.decay_q))
+    elif case == "steep_decay":
+        q.decay_q.copy_((ramp * (17 * 256)).expand_as(q.decay_q))  # 17 octaves per token: the gate factor is 0
+    elif case == "exp_extremes":
+        q.k_exp.fill_(-40); q.v_exp.fill_(37)
+    elif case == "zero_k":
+        q.Kq.zero_()
+    elif case == "zero_beta":
+        q.beta_q.zero_()
+    elif case == "zero_all":
+        q.Kq.zero_(); q.Vq.zero_(); q.beta_q.zero_()
+    return q
+
+
 def int8_chunk_slices(q: Int8Inputs, chunk_ids):
     """Host numpy copies of selected chunks: (Kq, Vq, k_exp, v_exp, beta_q, decay_q) stacked over the chunks."""
     import numpy as np

@@ -15,8 +15,10 @@ def _to_dev(q):
                           q.B, q.H_k, q.H_v, q.T, q.C, q.d_k, q.d_v)
 
 
-def _check(inp, N=-1, S=-1, chunk_ids=None):
+def _check(inp, N=-1, S=-1, chunk_ids=None, mutate=None):
     q = gen.make_int16_inputs(inp)
+    if mutate is not None:
+        mutate(q)
     qd = _to_dev(q)
     Wq, Uq, w_exp, u_exp, Toff, t_exp = gdn.chunk_prepare_int16(qd, N, S)
     assert gdn.gdn_device_status() == gdn.GDN_OK
@@ -47,6 +49,15 @@ def test_int16_defaults_bit_exact(adv):
 def test_int16_other_orders_and_steps(N, S):
     inp = gen.make_inputs(1, 1, 2, 256, 64, 128, 128, seed=110 + N + S, adversarial_heads="odd")
     _check(inp, N, S)
+
+
+@pytest.mark.parametrize("case", gen.INT_EDGE_CASES)
+def test_int16_saturating_and_degenerate_inputs_bit_exact(case):
+    inp = gen.make_inputs(1, 2, 2, 256, 64, 128, 128, seed=5)
+    _check(inp, mutate=lambda q: gen.int_edge_inputs(q, case, bits=16))
+    if case == "sign_max":
+        for N, S in ((1, 8), (2, 5), (3, 0)):
+            _check(inp, N, S, mutate=lambda q: gen.int_edge_inputs(q, case, bits=16))
 
 
 def test_int16_gqa_ragged_and_many_tiles():

@@ -15,8 +15,10 @@ def _to_dev(q):
                           q.B, q.H_k, q.H_v, q.T, q.C, q.d_k, q.d_v)
 
 
-def _check(inp, N=-1, S=-1, chunk_ids=None):
+def _check(inp, N=-1, S=-1, chunk_ids=None, mutate=None):
     q = gen.make_int8_inputs(inp)
+    if mutate is not None:
+        mutate(q)
     qd = _to_dev(q)
     Wq, Uq, w_exp, u_exp, Toff, t_exp = gdn.chunk_prepare_int8(qd, N, S)
     assert gdn.gdn_device_status() == gdn.GDN_OK
@@ -60,6 +62,17 @@ def test_int8_gqa_ragged_and_many_tiles():
     inp = gen.make_inputs(2, 4, 8, 4096, 64, 128, 128, seed=121)
     ids = np.random.default_rng(0).choice(inp.n_chunks, size=96, replace=False)
     _check(inp, chunk_ids=sorted(ids.tolist()))
+
+
+@pytest.mark.parametrize("case", gen.INT_EDGE_CASES)
+def test_int8_saturating_and_degenerate_inputs_bit_exact(case):
+    """Largest mantissas with the gate open and beta at its maximum (the inverse grows by tens of octaves: shifts far
+    beyond the word size in the aligned sums), empty chunks, closed gates, extreme input exponents."""
+    inp = gen.make_inputs(1, 2, 2, 256, 64, 128, 128, seed=5)
+    _check(inp, mutate=lambda q: gen.int_edge_inputs(q, case))
+    if case == "sign_max":
+        for N, S in ((1, 8), (2, 5), (3, 0)):
+            _check(inp, N, S, mutate=lambda q: gen.int_edge_inputs(q, case))
 
 
 def test_int8_unsupported_configurations():

@@ -41,6 +41,12 @@ def _check(inp, N=-1, S=-1, chunk_ids=None, mutate=None):
     return got
 
 
+@pytest.mark.parametrize("case", gen.INT_EDGE_CASES)
+def test_int8_c128_saturating_and_degenerate_inputs_bit_exact(case):
+    inp = gen.make_inputs(1, 2, 2, 512, 128, 128, 128, seed=5)
+    _check(inp, mutate=lambda q: gen.int_edge_inputs(q, case))
+
+
 @pytest.mark.parametrize("adv", ["none", "all"])
 def test_int8_c128_defaults_bit_exact(adv):
     inp = gen.make_inputs(1, 2, 2, 512, 128, 128, 128, seed=201, adversarial_heads=adv)

@@ -52,6 +52,19 @@ def test_two_evaluators_agree_bit_for_bit(C, N, S, adv):
             assert int(ref[key]) == int(fast[key][c]), key
 
 
+@pytest.mark.parametrize("case", gen.INT_EDGE_CASES)
+def test_two_evaluators_agree_on_saturating_and_degenerate_inputs(case):
+    inp = gen.make_inputs(1, 1, 1, 64, 64, 16, 16, seed=5, dtype=torch.float32)
+    q = gen.int_edge_inputs(gen.make_int16_inputs(inp), case, bits=16)
+    Kq, Vq, ke, ve, bq, dq = gen.int8_chunk_slices(q, range(q.n_chunks))
+    fast = orq.chunk_prepare_int16(Kq, Vq, ke, ve, bq, dq, 3, 8)
+    ref = orq.chunk_prepare_int16_ref(Kq[0].tolist(), Vq[0].tolist(), int(ke[0]), int(ve[0]), bq[0].tolist(), dq[0].tolist(), 3, 8)
+    for key in ("Wq", "Uq", "Toffq", "Aq", "Eq", "T0q"):
+        assert np.array_equal(np.asarray(ref[key]), fast[key][0]), key
+    for key in ("w_exp", "u_exp", "t_exp", "a_exp", "e_exp", "t0_exp"):
+        assert int(ref[key]) == int(fast[key][0]), key
+
+
 def test_structure_and_ranges():
     inp, q, (Kq, Vq, ke, ve, bq, dq) = _int16_chunks(64, seed=5, adversarial="all", d=32)
     out = orq.chunk_prepare_int16(Kq, Vq, ke, ve, bq, dq, 3, 8)

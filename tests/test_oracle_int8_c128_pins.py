@@ -28,6 +28,19 @@ def test_two_evaluators_agree_bit_for_bit(adv, N, S, d):
             assert tuple(int(v) for v in ref[key]) == tuple(int(v) for v in fast[key][c]), key
 
 
+@pytest.mark.parametrize("case", gen.INT_EDGE_CASES)
+def test_two_evaluators_agree_on_saturating_and_degenerate_inputs(case):
+    inp = gen.make_inputs(1, 1, 1, 128, 128, 16, 16, seed=5, dtype=torch.float32)
+    q = gen.int_edge_inputs(gen.make_int8_inputs(inp), case)
+    Kq, Vq, ke, ve, bq, dq = gen.int8_chunk_slices(q, range(q.n_chunks))
+    fast = orq.chunk_prepare_int8_c128(Kq, Vq, ke, ve, bq, dq, 3, 8)
+    ref = orq.chunk_prepare_int8_c128_ref(Kq[0].tolist(), Vq[0].tolist(), int(ke[0]), int(ve[0]), bq[0].tolist(), dq[0].tolist(), 3, 8)
+    for key in ("Wq", "Uq", "Toffq"):
+        assert np.array_equal(np.asarray(ref[key]), fast[key][0]), key
+    for key in ("w_exp", "u_exp", "t_exp"):
+        assert tuple(int(v) for v in ref[key]) == tuple(int(v) for v in fast[key][0]), key
+
+
 @pytest.mark.parametrize("adv", ["none", "all"])
 def test_structure_and_top_block_is_the_64_token_chunk(adv):
     """Rows 0..63 of a 128-chunk do not see rows 64..127 (T is lower triangular): the first block, its exponent and

@@ -62,6 +62,51 @@ def test_two_evaluators_agree_bit_for_bit(C, N, S, adv):
             assert int(ref[key]) == int(fast[key][c]), key
 
 
+def test_rounded_shift_beyond_the_word_size():
+    """Aligned sums shift a term right by the distance of its exponent from the reference, which on saturating inputs
+    exceeds 64: the result is 0 there (|x| < 2^(r-1)), in both evaluators' shift routines."""
+    x = np.array([-4161409, 4161409, 5, -1, 0, -(2 ** 61), 2 ** 61 - 1])
+    for r in (62, 63, 64, 65, 100, 1000):
+        want = [orq._rsr(int(v), r) for v in x]
+        assert list(orq._rsr_np(x, np.array(r))) == want, r
+        if r >= 63:
+            assert want == [0] * len(x)
+    assert list(orq._rsr_np(np.array([-4161409, 2 ** 61]), np.array(62))) == [orq._rsr(-4161409, 62), orq._rsr(2 ** 61, 62)] == [0, 1]
+
+
+@pytest.mark.parametrize("case", gen.INT_EDGE_CASES)
+def test_two_evaluators_agree_on_saturating_and_degenerate_inputs(case):
+    inp = gen.make_inputs(1, 1, 1, 64, 64, 16, 16, seed=5, dtype=torch.float32)
+    q = gen.int_edge_inputs(gen.make_int8_inputs(inp), case)
+    Kq, Vq, ke, ve, bq, dq = gen.int8_chunk_slices(q, range(q.n_chunks))
+    fast = orq.chunk_prepare_int8(Kq, Vq, ke, ve, bq, dq, 3, 8)
+    ref = orq.chunk_prepare_int8_ref(Kq[0].tolist(), Vq[0].tolist(), int(ke[0]), int(ve[0]), bq[0].tolist(), dq[0].tolist(), 3, 8)
+    for key in ("Wq", "Uq", "Toffq", "Aq", "Eq", "T0q"):
+        assert np.array_equal(np.asarray(ref[key]), fast[key][0]), key
+    for key in ("w_exp", "u_exp", "t_exp", "a_exp", "e_exp", "t0_exp"):
+        assert int(ref[key]) == int(fast[key][0]), key
+    if case in ("all_max", "sign_max", "alt_rows"):
+        assert int(ref["t_exp"]) > 20  # the inverse really grows by tens of octaves here
+    if case in ("zero_k", "zero_all", "steep_decay", "one_hot") and case != "one_hot":
+        assert not np.asarray(ref["Toffq"]).any()
+
+
+def test_two_evaluators_agree_where_a_term_is_shifted_out_entirely():
+    """Full feature size, largest mantissas with random signs: in the last chunk of the second head the diagonal term
+    of U sits 64 octaves below the reference exponent of its aligned sum and must contribute exactly 0 (an evaluator
+    that lets it contribute -1 moves one mantissa of U across a rounding boundary)."""
+    inp = gen.make_inputs(1, 2, 2, 256, 64, 128, 128, seed=5)
+    q = gen.int_edge_inputs(gen.make_int8_inputs(inp), "sign_max")
+    Kq, Vq, ke, ve, bq, dq = gen.int8_chunk_slices(q, [7])
+    fast = orq.chunk_prepare_int8(Kq, Vq, ke, ve, bq, dq, 3, 8)
+    ref = orq.chunk_prepare_int8_ref(Kq[0].tolist(), Vq[0].tolist(), int(ke[0]), int(ve[0]), bq[0].tolist(), dq[0].tolist(), 3, 8)
+    assert int(ref["u_exp"]) - int(ve[0]) > 60
+    for key in ("Wq", "Uq", "Toffq"):
+        assert np.array_equal(np.asarray(ref[key]), fast[key][0]), key
+    for key in ("w_exp", "u_exp", "t_exp"):
+        assert int(ref[key]) == int(fast[key][0]), key
+
+
 def test_structure_and_ranges():
     inp, q, (Kq, Vq, ke, ve, bq, dq) = _int8_chunks(64, seed=5, adversarial="all", d=32)
     out = orq.chunk_prepare_int8(Kq, Vq, ke, ve, bq, dq, 3, 8)
