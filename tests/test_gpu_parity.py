@@ -292,6 +292,41 @@ def test_fp32_blocked_forward_substitution(C):
     assert orc.rel_frobenius(Ug, Uo).max() <= TOL_FP32
 
 
+@pytest.mark.parametrize("C,dtype", [(64, torch.bfloat16), (128, torch.bfloat16), (32, torch.bfloat16), (16, torch.bfloat16),
+                                     (64, torch.float32), (24, torch.float32)])
+@pytest.mark.parametrize("case", ["zero_k", "zero_beta", "closed_gate", "open_gate_beta_one"])
+def test_degenerate_inputs(C, dtype, case):
+    """Degenerate chunks: no keys, no writes (beta = 0), a gate that closes between any two tokens (A = 0: T = I exactly,
+    W = diag(beta) K, U = diag(beta) V), and the other end, the ungated delta rule with beta = 1 (g = 0: no decay inside
+    a chunk, the far part of T is as large as its band), against the oracle of the same scheme."""
+    inp = gen.make_inputs(1, 1, 2, 4 * C, C, 128, 128, seed=77 + C, dtype=dtype)
+    if case == "zero_k":
+        inp.K.zero_()
+    elif case == "zero_beta":
+        inp.beta.zero_()
+    elif case == "closed_gate":
+        inp.g = (-200.0 * (torch.arange(inp.T) % C).float()).expand_as(inp.g).contiguous()
+    else:
+        inp.g.zero_()
+        inp.beta.fill_(1.0)
+    bf16 = dtype == torch.bfloat16
+    # Without decay the far entries of T are O(0.1) each instead of vanishing with the distance, and they enter the
+    # W / U products as single bf16 operands (the low halves cover the diagonal and the band): that adds ~1.2e-3 to the
+    # 1.7e-3 of the output rounding on 64-row blocks (measured 2.03e-3 .. 2.12e-3). Outside the paper's gated workloads;
+    # the bar for this case is 2.5e-3.
+    tol = (2.5e-3 if case == "open_gate_beta_one" and C >= 64 else TOL_BF16) if bf16 else TOL_FP32
+    _check(inp, tol)
+    if case == "open_gate_beta_one":
+        return
+    K, V, beta, g = _to_dev(inp)
+    W, U, Tinv = gdn.chunk_prepare(K, V, beta, g, inp.C)
+    assert torch.equal(Tinv, torch.eye(C, device="cuda", dtype=dtype).expand_as(Tinv))
+    if case == "zero_k":
+        assert not W.any()
+    if case == "zero_beta":
+        assert not W.any() and not U.any()
+
+
 def test_empty_batch_is_a_no_op():
     K = torch.empty(0, 2, 128, 128, dtype=torch.bfloat16, device="cuda")
     V = torch.empty(0, 2, 128, 128, dtype=torch.bfloat16, device="cuda")
