@@ -396,12 +396,14 @@ def chunk_state_output(Q, K, W_gated, U, g, C: int, scale: float = 1.0, S0=None)
     assert T % C == 0
     S = np.zeros((dv, K.shape[1])) if S0 is None else np.array(S0, dtype=np.float64)
     O = np.zeros((T, dv))
-    causal = np.tril(np.ones((C, C)))
+    causal = np.tril(np.ones((C, C), dtype=bool))
     for c in range(T // C):
         sl = slice(c * C, (c + 1) * C)
         q, k, w, u, gc = Q[sl], K[sl], W_gated[sl], U[sl], g[sl]
         u_new = u - w @ S.T
-        P = (q @ k.T) * np.exp(gc[:, None] - gc[None, :]) * causal
+        # the sum runs over j <= i only: the decay factor is not evaluated above the diagonal (g_i - g_j > 0 there, and a
+        # gate that closes fast would overflow the exponential and leave 0 * inf)
+        P = (q @ k.T) * np.exp(np.where(causal, gc[:, None] - gc[None, :], -np.inf))
         O[sl] = scale * (np.exp(gc)[:, None] * (q @ S.T) + P @ u_new)
         S = math.exp(gc[-1]) * S + (u_new * np.exp(gc[-1] - gc)[:, None]).T @ k
     return O, S

@@ -61,6 +61,48 @@ def test_state_output_matches_oracle(B, H_k, H_v, T, with_state):
             assert eS.max() <= TOL_S, f"S rel-F {eS.max():.3e} of head ({b},{hv})"
 
 
+@pytest.mark.parametrize("case", ["closed_gate", "open_gate", "zero_u", "large_state"])
+def test_state_output_on_degenerate_inputs(case):
+    """A gate that closes by 30 nats per token (every token forgets the state: the decay factors above the diagonal
+    of a chunk would overflow if they were formed), no decay at all, U = 0 (the state only decays and is corrected by
+    W S0), and an initial state a hundred times the usual size."""
+    C, B, H_k, H_v, T = 64, 2, 1, 2, 320
+    inp = gen.make_inputs(B, H_k, H_v, T, C, 128, 128, seed=430, adversarial_heads="odd")
+    if case == "closed_gate":
+        inp.g = (-30.0 * (1 + torch.arange(T) % C).float()).expand_as(inp.g).contiguous()
+    if case == "open_gate":
+        inp.g.zero_()
+    Q = _queries(inp, 431)
+    scale = 128 ** -0.5
+    S0 = (10.0 if case == "large_state" else 0.1) * torch.randn(B, H_v, 128, 128, generator=torch.Generator().manual_seed(432))
+    K, V, beta, g = inp.K.cuda(), inp.V.cuda(), inp.beta.cuda(), inp.g.cuda()
+    W, U, _ = gdn.chunk_prepare(K, V, beta, g, C, flags=gdn.GDN_FLAG_W_GATED)
+    if case == "zero_u":
+        U.zero_()
+    O, S = gdn.chunk_state_output(Q.cuda(), K, W, U, g, C, scale, S0.cuda())
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+    assert torch.isfinite(O.float()).all() and torch.isfinite(S).all()
+    for b in range(B):
+        for hv in range(H_v):
+            Oo, So = orc.chunk_state_output(Q[b, 0].double().numpy(), inp.K[b, 0].double().numpy(), W[b, hv].double().cpu().numpy(),
+                                            U[b, hv].double().cpu().numpy(), inp.g[b, hv].double().numpy(), C, scale,
+                                            S0[b, hv].double().numpy())
+            assert np.isfinite(Oo).all()
+            Og, Or = O[b, hv].double().cpu().numpy().reshape(T // C, C, 128), Oo.reshape(T // C, C, 128)
+            # (with U = 0 the state only decays, by e^-50 per chunk on these gates: from the third chunk on the output
+            # is below the fp32 range, where the kernel's zeros are the right answer and a relative error means nothing)
+            live = np.sqrt((Or ** 2).sum(axis=(-1, -2))) > 1e-30
+            assert live[:2].all() and np.abs(Og[~live]).max(initial=0.0) < 1e-30
+            eO = orc.rel_frobenius(Og[live], Or[live])
+            assert eO.max() <= TOL_O, f"O rel-F {eO.max():.3e} at chunk {eO.argmax()} of head ({b},{hv})"
+            Sg = S[b, hv].double().cpu().numpy()
+            if np.abs(So).max() > 1e-30:
+                eS = orc.rel_frobenius(Sg[None], So[None])
+                assert eS.max() <= TOL_S, f"S rel-F {eS.max():.3e} of head ({b},{hv})"
+            else:
+                assert np.abs(Sg).max() < 1e-30
+
+
 def test_whole_layer_matches_the_token_recurrence():
     """chunk-prepare (gated W, U) + state passing/output on the GPU against the token-by-token gated delta rule."""
     C, T = 64, 512

@@ -135,6 +135,35 @@ def test_chunkwise_state_passing_and_output_equal_the_token_recurrence():
     assert not np.allclose(O_bad2, O_ref, atol=1e-6)
 
 
+def test_chunkwise_output_with_a_gate_that_closes_fast_is_finite_and_equals_the_token_recurrence():
+    """A gate that closes by 30 nats per token: g_i - g_j reaches +1890 above the diagonal of a 64-token chunk, where
+    the sum over j <= i has no term. The chunk-wise evaluation must not touch those entries (exp would overflow and
+    0 * inf would poison the output) and still equal the token-by-token rule, where each token forgets the state."""
+    rng = np.random.default_rng(12)
+    C, n_chunks, dk, dv = 64, 2, 4, 3
+    T = C * n_chunks
+    K = rng.normal(size=(T, dk))
+    K /= np.linalg.norm(K, axis=1, keepdims=True)
+    Q = rng.normal(size=(T, dk))
+    V = rng.normal(size=(T, dv))
+    beta = np.full(T, 0.5)
+    graw = np.full(T, -30.0)
+    S0 = rng.normal(size=(dv, dk))
+    O_ref, S_ref = orc.gated_delta_rule(Q, K, V, beta, graw, scale=1.0, S0=S0)
+    g_local = np.cumsum(graw.reshape(n_chunks, C), axis=1).reshape(T)
+    W = np.zeros((T, dk)); U = np.zeros((T, dv))
+    for c in range(n_chunks):
+        sl = slice(c * C, (c + 1) * C)
+        W[sl], U[sl], _ = orc.chunk_prepare(K[sl], V[sl], beta[sl], g_local[sl], exact=True, w_gated=True)
+    with np.errstate(over="raise", invalid="raise"):
+        O, S = orc.chunk_state_output(Q, K, W, U, g_local, C, scale=1.0, S0=S0)
+    assert np.isfinite(O).all() and np.isfinite(S).all()
+    assert np.allclose(O, O_ref, atol=1e-12) and np.allclose(S, S_ref, atol=1e-12)
+    # every token sees (almost) only its own write: o_i = beta_i <k_i, q_i> v_i up to e^-30
+    own = 0.5 * np.einsum("td,td->t", K, Q)[:, None] * V
+    assert np.allclose(O, own, atol=1e-10)
+
+
 def test_variable_length_sequences_equal_the_token_recurrence_per_sequence():
     """Packed sequences of ragged lengths: the chunk quantities of `chunk_prepare_varlen` (chunks counted from each
     sequence's first token, the last one short) carried through the chunk-wise state passing reproduce the
