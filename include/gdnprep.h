@@ -316,7 +316,7 @@ int gdn_device_status(gdn_stream_t stream);
  */
 int gdn_selftest_bounded_wait(gdn_stream_t stream);
 
-/* Paper's parameters per chunk size: N = 3; S = 8 for C = 64 (Sec. 4.1) and for the
+/* Paper's parameters per chunk size: N = 3 (C - 1 for chunks of 2 or 3 tokens); S = 8 for C = 64 (Sec. 4.1) and for the
  * 64-blocks of C = 128 (App. H), S = 4 for C = 32 (Sec. 4.3); C = 16 is not in the
  * paper: S = 3, which makes the result exact. Other C: S = ceil(C/4) - 1. */
 int gdn_default_order(int C);

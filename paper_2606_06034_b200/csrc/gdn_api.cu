@@ -326,8 +326,7 @@ int gdn_device_status(gdn_stream_t stream) {
 }
 
 int gdn_default_order(int C) {
-    (void)C;
-    return 3;
+    return C > 3 ? 3 : (C > 1 ? C - 1 : 1);  // (the order must stay below the chunk size: C = 2, 3 get C - 1, which is exact)
 }
 
 int gdn_default_residual_steps(int C) {

@@ -34,6 +34,7 @@ def test_library_exports_every_declared_symbol(lib):
 
 def test_defaults_follow_the_paper(lib):
     assert [lib.gdn_default_order(c) for c in (16, 32, 64, 128)] == [3, 3, 3, 3]
+    assert [lib.gdn_default_order(c) for c in (2, 3, 4)] == [1, 2, 3]  # below the chunk size
     assert [lib.gdn_default_residual_steps(c) for c in (16, 32, 64, 128)] == [3, 4, 8, 8]
 
 
