@@ -1,0 +1,219 @@
+"""Every entry point on seeded random configurations (batch, grouped heads, ragged token counts, regimes, orders, flag
+subsets, length mixes, segment counts) against the oracles, with the bars of the targeted tests. The fixed cases of the
+other files pin known edges; these runs look for what nobody thought of."""
+import random
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import gdn_oracle as orc
+from oracle import gdn_oracle_int8 as o8
+from oracle import gdn_oracle_int16 as o16
+from paper_2606_06034_b200 import binding as gdn
+from paper_2606_06034_b200 import inputs as gen
+
+import test_gpu_parity as tp
+import test_gpu_state as ts
+import test_gpu_varlen as tv
+
+pytestmark = pytest.mark.gpu
+
+
+def _exact_check(inp, variant, tol):
+    K, V, beta, g = tp._to_dev(inp)
+    W, U, Tinv = gdn.chunk_prepare(K, V, beta, g, inp.C, method="fwdsubst", variant=variant)
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+    Wg, Ug, Tg = tp._gpu_chunks(W, U, Tinv, inp)
+    Wo, Uo, To = tp._oracle(inp, exact=True)
+    for name, got, ref in (("Tinv", Tg, To), ("W", Wg, Wo), ("U", Ug, Uo)):
+        err = orc.rel_frobenius(got, ref)
+        bound = tp._bound(ref, tol, bf16_out=inp.K.dtype == torch.bfloat16)
+        assert np.all(err <= bound), f"{name} {err.max():.3e} > {bound[np.argmax(err - bound)]:.3e}"
+
+
+def test_tensor_core_kernel_on_random_configurations():
+    rng = random.Random(1234)
+    for it in range(100):
+        C = rng.choice([16, 32, 64, 64, 64, 128])
+        B, Hk, grp = rng.choice([1, 2, 3]), rng.choice([1, 2, 3]), rng.choice([1, 1, 2, 3, 4])
+        Hv, T = Hk * grp, C * rng.choice([1, 2, 3, 5, 7, 9])
+        adv = rng.choice(["none", "odd", "all"])
+        mode = rng.choice(["plain", "plain", "flags", "rows", "blocked", "token_major"])
+        seed = 5000 + it
+        what = f"#{it} C={C} B={B} H_k={Hk} H_v={Hv} T={T} adv={adv} {mode}"
+        try:
+            if mode == "plain":
+                inp = gen.make_inputs(B, Hk, Hv, T, C, 128, 128, seed=seed, adversarial_heads=adv)
+                N, S = rng.choice([(-1, -1), (-1, -1), (3, 8), (2, 4), (3, 15), (1, 2)])
+                if C < 64 and S == 15:
+                    S = 3
+                if adv != "none" and (N, S) not in ((-1, -1), (3, 8)):
+                    N, S = -1, -1  # (truncated orders on correlated keys are graded by their own test)
+                tp._check(inp, tp.TOL_BF16, N, S)
+            elif mode in ("rows", "blocked"):
+                inp = gen.make_inputs(B, Hk, Hv, T, C, 128, 128, seed=seed, adversarial_heads=adv)
+                _exact_check(inp, gdn.GDN_FWDSUBST_BLOCKED if mode == "blocked" else gdn.GDN_FWDSUBST_ROWS, tp.TOL_BF16)
+            else:
+                flags = rng.choice([1, 2, 3, 16, 17, 18, 19] if mode == "flags" else [0, 1, 2, 3, 16, 19])
+                a = adv if C <= 64 else "none"
+                inp, graw = tp._raw_inputs(B, Hk, Hv, T, C, seed=seed, adv=a)
+                if not (flags & gdn.GDN_FLAG_K_L2NORM):
+                    inp = gen.make_inputs(B, Hk, Hv, T, C, 128, 128, seed=seed, adversarial_heads=a)
+                if mode == "flags":
+                    tp._check_ex(inp, graw, flags, tp.TOL_BF16)
+                else:
+                    g_src = graw if (flags & gdn.GDN_FLAG_G_RAW) else inp.g
+                    K, V, beta, g = inp.K.cuda(), inp.V.cuda(), inp.beta.cuda(), g_src.cuda()
+                    tm = lambda x: x.transpose(1, 2).contiguous()
+                    W, U, Tinv = gdn.chunk_prepare(tm(K), tm(V), tm(beta), tm(g), C, flags=flags | gdn.GDN_FLAG_LAYOUT_BTHD)
+                    W0, U0, T0 = gdn.chunk_prepare(K, V, beta, g, C, flags=flags) if flags else gdn.chunk_prepare(K, V, beta, g, C)
+                    assert gdn.gdn_device_status() == gdn.GDN_OK
+                    assert torch.equal(tm(W0), W) and torch.equal(tm(U0), U) and torch.equal(T0, Tinv)
+        except AssertionError as e:
+            raise AssertionError(f"{what}: {e}") from e
+
+
+def test_plain_fma_kernel_on_random_configurations():
+    rng = random.Random(2468)
+    for it in range(150):
+        dtype = rng.choice([torch.bfloat16, torch.float32])
+        C = rng.choice([2, 3, 5, 8, 12, 16, 24, 32, 40, 48, 64, 128])
+        dk, dv = rng.choice([8, 16, 40, 64, 72, 128, 192, 256]), rng.choice([8, 32, 64, 104, 128, 256])
+        if dtype == torch.bfloat16 and dk == 128 and dv == 128 and C in (16, 32, 64, 128):
+            dk = 64  # (that shape belongs to the tensor-core kernel)
+        B, Hk, grp = rng.choice([1, 2]), rng.choice([1, 2]), rng.choice([1, 2, 3])
+        T = C * rng.choice([1, 2, 3])
+        blk = 64 if C == 128 else C
+        N, S = max(1, min(rng.choice([1, 2, 3, 5, 9]), blk - 1)), rng.choice([0, 1, 3, 8])
+        mode = rng.choice(["neumann", "neumann", "rows", "blocked"])
+        adv = rng.choice(["none", "all"])
+        what = f"#{it} {dtype} C={C} d_k={dk} d_v={dv} B={B} H_k={Hk} group={grp} T={T} N={N} S={S} {mode} adv={adv}"
+        inp = gen.make_inputs(B, Hk, Hk * grp, T, C, dk, dv, seed=15000 + it, dtype=dtype, adversarial_heads=adv)
+        tol = tp.TOL_BF16 if dtype == torch.bfloat16 else tp.TOL_FP32
+        try:
+            if mode == "neumann":
+                if adv == "all":
+                    N, S = -1, -1
+                tp._check(inp, tol, N, S)
+            else:
+                blocked = mode == "blocked" and C % 16 == 0
+                _exact_check(inp, gdn.GDN_FWDSUBST_BLOCKED if blocked else gdn.GDN_FWDSUBST_ROWS, tol)
+        except AssertionError as e:
+            raise AssertionError(f"{what}: {e}") from e
+
+
+def test_integer_kernels_on_random_configurations():
+    rng = random.Random(31337)
+    for it in range(100):
+        kind = rng.choice(["i8", "i8", "i8c128", "i16"])
+        C, bits = (128 if kind == "i8c128" else 64), (16 if kind == "i16" else 8)
+        B, Hk, grp = rng.choice([1, 2]), rng.choice([1, 2, 3]), rng.choice([1, 2, 3])
+        T = C * rng.choice([1, 2, 3, 5])
+        N, S = rng.choice([(3, 8), (3, 8), (2, 8), (1, 5), (3, 3), (3, 0), (2, 1)])
+        adv = rng.choice(["none", "odd", "all"])
+        case = rng.choice([None, None, None] + list(gen.INT_EDGE_CASES))
+        what = f"#{it} {kind} B={B} H_k={Hk} group={grp} T={T} N={N} S={S} adv={adv} pattern={case}"
+        inp = gen.make_inputs(B, Hk, Hk * grp, T, C, 128, 128, seed=12000 + it, adversarial_heads=adv)
+        q = gen.make_int8_inputs(inp, bits)
+        if case:
+            gen.int_edge_inputs(q, case, bits)
+        qd = gen.Int8Inputs(q.Kq.cuda(), q.Vq.cuda(), q.k_exp.cuda(), q.v_exp.cuda(), q.beta_q.cuda(), q.decay_q.cuda(),
+                            q.B, q.H_k, q.H_v, q.T, q.C, q.d_k, q.d_v)
+        Wq, Uq, w_exp, u_exp, Toff, t_exp = (gdn.chunk_prepare_int16 if kind == "i16" else gdn.chunk_prepare_int8)(qd, N, S)
+        assert gdn.gdn_device_status() == gdn.GDN_OK
+        ids = list(range(q.n_chunks))
+        if len(ids) > 24:
+            ids = sorted(rng.sample(ids, 24))
+        sl = gen.int8_chunk_slices(q, ids)
+        if kind == "i8":
+            ref, ne, nt = o8.chunk_prepare_int8(*sl, N, S), (), ()
+        elif kind == "i8c128":
+            ref, ne, nt = o8.chunk_prepare_int8_c128(*sl, N, S), (2,), (3,)
+        else:
+            ref, ne, nt = o16.chunk_prepare_int16(*sl, N, S), (), ()
+        n, idx = q.n_chunks, torch.as_tensor(ids, device="cuda")
+        got = {"Wq": Wq.reshape(n, C, 128)[idx], "Uq": Uq.reshape(n, C, 128)[idx], "Toffq": Toff.reshape(n, C, C)[idx],
+               "w_exp": w_exp.reshape((n,) + ne)[idx], "u_exp": u_exp.reshape((n,) + ne)[idx], "t_exp": t_exp.reshape((n,) + nt)[idx]}
+        for key, val in got.items():
+            assert np.array_equal(val.cpu().numpy(), ref[key]), f"{what}: {key} differs"
+
+
+def test_state_passing_on_random_configurations():
+    rng = random.Random(99)
+    C = 64
+    for it in range(60):
+        B, Hk, grp = rng.choice([1, 2, 3]), rng.choice([1, 2, 3]), rng.choice([1, 2, 3])
+        Hv, n = Hk * grp, rng.choice([1, 2, 3, 5, 8, 13])
+        T = C * n
+        adv = rng.choice(["none", "odd", "all"])
+        case = rng.choice(["plain", "state", "open_gate", "large_state", "segments"])
+        what = f"#{it} B={B} H_k={Hk} H_v={Hv} T={T} adv={adv} {case}"
+        inp = gen.make_inputs(B, Hk, Hv, T, C, 128, 128, seed=7000 + it, adversarial_heads=adv)
+        if case == "open_gate":
+            inp.g.zero_()
+        Q = ts._queries(inp, 7001 + it)
+        scale = 128 ** -0.5
+        S0 = None
+        if case in ("state", "large_state", "segments"):
+            S0 = (10.0 if case == "large_state" else 0.1) * torch.randn(B, Hv, 128, 128, generator=torch.Generator().manual_seed(3))
+        K, V, beta, g = inp.K.cuda(), inp.V.cuda(), inp.beta.cuda(), inp.g.cuda()
+        W, U, _ = gdn.chunk_prepare(K, V, beta, g, C, flags=gdn.GDN_FLAG_W_GATED)
+        S0d = None if S0 is None else S0.cuda()
+        if case == "segments" and n >= 2 and B == 1:
+            P = min(rng.choice([2, 3, 5]), n)
+            Os, Ss = gdn.chunk_state_output_segmented(Q.cuda()[0], K[0], W[0], U[0], g[0], C, scale, S0d[0], segments=P)
+            O, S = Os[None], Ss[None]
+        else:
+            O, S = gdn.chunk_state_output(Q.cuda(), K, W, U, g, C, scale, S0d)
+        assert gdn.gdn_device_status() == gdn.GDN_OK
+        for b in range(B):
+            for hv in range(Hv):
+                Oo, So = orc.chunk_state_output(Q[b, hv // grp].double().numpy(), inp.K[b, hv // grp].double().numpy(),
+                                                W[b, hv].double().cpu().numpy(), U[b, hv].double().cpu().numpy(),
+                                                inp.g[b, hv].double().numpy(), C, scale, None if S0 is None else S0[b, hv].double().numpy())
+                eO = orc.rel_frobenius(O[b, hv].double().cpu().numpy().reshape(n, C, 128), Oo.reshape(n, C, 128))
+                eS = orc.rel_frobenius(S[b, hv].double().cpu().numpy()[None], So[None])
+                assert eO.max() <= ts.TOL_O and eS.max() <= ts.TOL_S, f"{what}: O {eO.max():.2e} S {eS.max():.2e} head ({b},{hv})"
+
+
+def test_packed_layer_on_random_length_mixes():
+    """Both packed calls back to back against the token-by-token rule, every sequence by itself (lengths 0, 1, C - 1, C,
+    C + 1, ...; up to 160 sequences; raw or cumulative gates; with and without initial states)."""
+    rng = random.Random(777)
+    C = 64
+    for it in range(50):
+        nseq = rng.choice([1, 2, 3, 5, 9, 33, 160])
+        kinds = [1, C - 1, C, C + 1, 2 * C, 3, rng.randint(1, 4 * C), rng.randint(1, 3 * C), 0]
+        lens = [rng.choice(kinds) for _ in range(nseq)]
+        if sum(lens) == 0:
+            lens[0] = 5
+        Hk, grp = rng.choice([1, 2]), rng.choice([1, 2])
+        Hv = Hk * grp
+        with_state, raw = rng.choice([False, True]), rng.choice([False, True])
+        what = f"#{it} sequences={nseq} T={sum(lens)} H_k={Hk} H_v={Hv} state={with_state} raw={raw}"
+        K, V, beta, g, graw, cu = tv._packed_inputs(lens, Hk, Hv, C, seed=9500 + it)
+        Q = tv._queries(Hk, int(cu[-1]), 9600 + it)
+        scale = 128 ** -0.5
+        S0 = 0.1 * torch.randn(len(lens), Hv, 128, 128, generator=torch.Generator().manual_seed(5)) if with_state else None
+        gates = graw if raw else g
+        flags = gdn.GDN_FLAG_W_GATED | (gdn.GDN_FLAG_G_RAW if raw else 0)
+        W, U, _, _, _ = gdn.chunk_prepare_varlen(K.cuda(), V.cuda(), beta.cuda(), gates.cuda(), cu, C, flags=flags, want_tinv=False)
+        O, S = gdn.chunk_state_output_varlen(Q.cuda(), K.cuda(), W, U, gates.cuda(), cu, C, scale, None if S0 is None else S0.cuda(),
+                                             flags=gdn.GDN_FLAG_G_RAW if raw else 0)
+        assert gdn.gdn_device_status() == gdn.GDN_OK
+        assert bool(torch.isfinite(O).all()) and bool(torch.isfinite(S).all()), what
+        for s_ in (range(len(lens)) if len(lens) <= 12 else rng.sample(range(len(lens)), 12)):
+            L, a = lens[s_], int(cu[s_])
+            for hv in range(Hv):
+                init = None if S0 is None else S0[s_, hv].double().numpy()
+                if L == 0:  # an empty sequence hands its initial state on
+                    want = np.zeros((128, 128)) if init is None else init
+                    assert np.abs(S[s_, hv].double().cpu().numpy() - want).max() <= 1e-6, what
+                    continue
+                Oo, So = orc.gated_delta_rule(Q[hv // grp, a:a + L].double().numpy(), K[hv // grp, a:a + L].double().numpy(),
+                                              V[hv, a:a + L].double().numpy(), beta[hv, a:a + L].double().numpy(),
+                                              graw[hv, a:a + L].double().numpy(), scale, init)
+                eO = orc.rel_frobenius(O[hv, a:a + L].double().cpu().numpy()[None], Oo[None])
+                eS = orc.rel_frobenius(S[s_, hv].double().cpu().numpy()[None], So[None])
+                assert eO.max() <= 1e-2 and eS.max() <= 1e-2, f"{what}: sequence {s_} (len {L}) head {hv}: O {eO.max():.2e} S {eS.max():.2e}"
