@@ -228,6 +228,7 @@ int gdn_chunk_prepare_varlen(const void* K, const void* V, const float* beta, co
  *   (zero state);
  *   O_out [B,H_v,T,d_v] bf16; S_out [B,H_v,d_v,d_k] fp32 or NULL.
  * Supported: C = 64, d_k = d_v = 128, T a multiple of C. fp32 state, bf16 tensor-core operands.
+ * B = 0 is a no-op; with T = 0 nothing is launched and S_out receives S_in (zeros without one).
  */
 int gdn_chunk_state_output(const void* Q, const void* K, const void* W_gated, const void* U, const float* g,
                            int B, int H_k, int H_v, int T, int C, int d_k, int d_v, float scale,

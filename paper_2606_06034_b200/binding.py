@@ -138,8 +138,21 @@ def _dtype_code(t: torch.Tensor) -> int:
     raise TypeError(f"unsupported dtype {t.dtype}")
 
 
+_EMPTY = {}  # per device: a small allocation whose address stands in for tensors without elements
+
+
 def _ptr(t):
-    return None if t is None else ctypes.c_void_p(t.data_ptr())
+    """Address of a tensor's data. torch gives tensors without elements a null data pointer, which the library would
+    report as a missing argument; an empty batch or zero tokens is a valid (empty) problem, so such tensors are passed
+    as the address of a small allocation that is never read or written."""
+    if t is None:
+        return None
+    if t.numel() == 0 and t.is_cuda:
+        key = t.device.index
+        if key not in _EMPTY:
+            _EMPTY[key] = torch.zeros(64, dtype=torch.float32, device=t.device)
+        return ctypes.c_void_p(_EMPTY[key].data_ptr())
+    return ctypes.c_void_p(t.data_ptr())
 
 
 def _stream():

@@ -878,7 +878,17 @@ int launch_chunk_state(const ProblemS& q, cudaStream_t stream) {
     if (q.state_only && !var) return GDN_ERR_UNSUPPORTED;
     const long long hk = var ? q.H_k : (long long)q.B * q.H_k, hv = var ? q.H_v : (long long)q.B * q.H_v;
     const long long n_cta = (long long)q.B * q.H_v;
-    if (n_cta == 0 || q.T == 0) return GDN_OK;
+    if (n_cta == 0) return GDN_OK;
+    if (q.T == 0) {
+        // no tokens: every sequence hands its initial state on (zeros without one)
+        if (q.S_out != nullptr && !q.state_only) {
+            const size_t bytes = static_cast<size_t>(n_cta) * kD * kD * sizeof(float);
+            const cudaError_t e = (q.S_in != nullptr) ? cudaMemcpyAsync(q.S_out, q.S_in, bytes, cudaMemcpyDeviceToDevice, stream)
+                                                      : cudaMemsetAsync(q.S_out, 0, bytes, stream);
+            if (e != cudaSuccess) return GDN_ERR_LAUNCH;
+        }
+        return GDN_OK;
+    }
     if (n_cta >= (1LL << 31)) return GDN_ERR_UNSUPPORTED;
     if (hv >= (1LL << 31)) return GDN_ERR_UNSUPPORTED;
     int* status = device_status_word();

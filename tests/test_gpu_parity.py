@@ -341,6 +341,30 @@ def test_empty_batch_is_a_no_op():
     assert rc == gdn.GDN_OK
 
 
+def test_empty_tensors_through_the_binding():
+    """torch gives tensors without elements a null data pointer; the binding passes a stand-in address, so an empty
+    batch or zero tokens is an empty problem on every entry point, not a missing argument."""
+    K = torch.zeros(0, 2, 128, 128, dtype=torch.bfloat16, device="cuda")
+    b = torch.zeros(0, 2, 128, device="cuda")
+    n0 = gdn.gdn_launch_count()
+    W, U, Tinv = gdn.chunk_prepare(K, K, b, b, 64)
+    assert W.shape == K.shape and Tinv.shape == (0, 2, 2, 64, 64)
+    K0 = torch.zeros(1, 2, 0, 128, dtype=torch.bfloat16, device="cuda")
+    b0 = torch.zeros(1, 2, 0, device="cuda")
+    W, U, Tinv = gdn.chunk_prepare(K0, K0, b0, b0, 64, method="fwdsubst")
+    assert W.shape == K0.shape
+    Kf = torch.zeros(0, 1, 48, 40, device="cuda")
+    W, U, Tinv = gdn.chunk_prepare(Kf, Kf, torch.zeros(0, 1, 48, device="cuda"), torch.zeros(0, 1, 48, device="cuda"), 24)
+    assert W.shape == Kf.shape
+    for bits, fn in ((8, gdn.chunk_prepare_int8), (16, gdn.chunk_prepare_int16)):
+        q = gen.make_int8_inputs(gen.make_inputs(1, 1, 1, 64, 64, 128, 128, seed=1), bits)
+        e = gen.Int8Inputs(q.Kq[:0].cuda(), q.Vq[:0].cuda(), q.k_exp[:0].cuda(), q.v_exp[:0].cuda(), q.beta_q[:0].cuda(),
+                           q.decay_q[:0].cuda(), 0, 1, 1, 64, 64, 128, 128)
+        out = fn(e)
+        assert out[0].shape == (0, 1, 64, 128)
+    assert gdn.gdn_device_status() == gdn.GDN_OK and gdn.gdn_launch_count() == n0
+
+
 def test_argument_errors_on_device():
     inp = gen.make_inputs(1, 1, 1, 128, 64, 128, 128, seed=90)
     K, V, beta, g = _to_dev(inp)

@@ -103,6 +103,20 @@ def test_state_output_on_degenerate_inputs(case):
                 assert np.abs(Sg).max() < 1e-30
 
 
+def test_zero_tokens_hand_the_initial_state_on():
+    K = torch.zeros(2, 3, 0, 128, dtype=torch.bfloat16, device="cuda")
+    g = torch.zeros(2, 3, 0, device="cuda")
+    S0 = torch.randn(2, 3, 128, 128, device="cuda")
+    O, S = gdn.chunk_state_output(K, K, K, K, g, 64, 1.0, S0)
+    assert O.shape == K.shape and torch.equal(S, S0)
+    O, S = gdn.chunk_state_output(K, K, K, K, g, 64, 1.0, None)
+    assert not S.any()
+    Ke = torch.zeros(0, 3, 64, 128, dtype=torch.bfloat16, device="cuda")
+    O, S = gdn.chunk_state_output(Ke, Ke, Ke, Ke, torch.zeros(0, 3, 64, device="cuda"), 64, 1.0, None)
+    assert O.shape == Ke.shape and S.shape == (0, 3, 128, 128)
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+
+
 def test_whole_layer_matches_the_token_recurrence():
     """chunk-prepare (gated W, U) + state passing/output on the GPU against the token-by-token gated delta rule."""
     C, T = 64, 512
