@@ -523,3 +523,34 @@ def test_bounded_wait_gives_up_and_reports():
     assert gdn.gdn_device_status() == gdn.GDN_OK
     inp = gen.make_inputs(1, 1, 1, 256, 64, 128, 128, seed=290)
     _check(inp, TOL_BF16)
+
+
+def test_host_threads_on_their_own_streams_do_not_disturb_each_other():
+    """Four host threads, each on its own stream, 100 calls each on its own problem: every result equals the one a
+    single-threaded call gives (the library keeps no per-call state on the host or the device)."""
+    import threading
+    problems = [gen.make_inputs(2, 2, 4, 64 * (3 + i), 64, 128, 128, seed=700 + i) for i in range(4)]
+    dev = [tuple(x.cuda() for x in (p.K, p.V, p.beta, p.g)) for p in problems]
+    want = [gdn.chunk_prepare(*d, 64) for d in dev]
+    torch.cuda.synchronize()
+    errors = []
+
+    def work(k):
+        stream = torch.cuda.Stream()
+        try:
+            with torch.cuda.stream(stream):
+                for _ in range(100):
+                    got = gdn.chunk_prepare(*dev[k], 64)
+                stream.synchronize()
+            if not all(torch.equal(a, b) for a, b in zip(got, want[k])):
+                errors.append(f"thread {k}: results differ")
+        except Exception as exc:  # a failure in a thread must fail the test
+            errors.append(f"thread {k}: {exc!r}")
+
+    threads = [threading.Thread(target=work, args=(k,)) for k in range(4)]
+    for th in threads:
+        th.start()
+    for th in threads:
+        th.join()
+    torch.cuda.synchronize()
+    assert not errors and gdn.gdn_device_status() == gdn.GDN_OK

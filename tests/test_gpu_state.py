@@ -103,6 +103,36 @@ def test_state_output_on_degenerate_inputs(case):
                 assert np.abs(Sg).max() < 1e-30
 
 
+def test_both_calls_can_be_captured_in_a_cuda_graph():
+    """The entry points launch kernels only (no allocation, no synchronisation; tensor maps travel as kernel arguments),
+    so a model can capture the layer in a CUDA graph and replay it on the same buffers."""
+    inp = gen.make_inputs(1, 2, 4, 1024, 64, 128, 128, seed=440)
+    K, V, beta, g = inp.K.cuda(), inp.V.cuda(), inp.beta.cuda(), inp.g.cuda()
+    Q = _queries(inp, 441).cuda()
+    outs = gdn.alloc_outputs(K, V, 64, True, False)
+    O, S = torch.empty_like(V), torch.empty(1, 4, 128, 128, device="cuda")
+
+    def step():
+        W, U, _ = gdn.chunk_prepare(K, V, beta, g, 64, outputs=outs, flags=gdn.GDN_FLAG_W_GATED)
+        gdn.chunk_state_output(Q, K, W, U, g, 64, 0.1, None, outputs=(O, S))
+
+    step()
+    torch.cuda.synchronize()
+    want = [t.clone() for t in (*outs, O, S)]
+    for t in (*outs, O, S):
+        t.zero_()
+    graph, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            step()
+    torch.cuda.synchronize()
+    assert not outs[0].any()  # captured, not run
+    graph.replay()
+    torch.cuda.synchronize()
+    assert all(torch.equal(a, b) for a, b in zip((*outs, O, S), want))
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+
+
 def test_zero_tokens_hand_the_initial_state_on():
     K = torch.zeros(2, 3, 0, 128, dtype=torch.bfloat16, device="cuda")
     g = torch.zeros(2, 3, 0, device="cuda")
