@@ -149,6 +149,9 @@ __device__ __forceinline__ TileCoord decode_tile(uint32_t tile, const ParamsI16&
     return c;
 }
 
+// DBG: the instantiation that also writes every exact matrix product (tests of small cases); the normal one carries
+// none of its tests and stores.
+template <bool DBG>
 __global__ void __launch_bounds__(kThreads, 1)
 chunk_tc_int16_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                       const __grid_constant__ ParamsI16 p) {
@@ -292,7 +295,7 @@ chunk_tc_int16_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
         const bool chunk_valid = (tc.t0 + cb) < p.T;
         const long long chunk_id = (long long)tc.bhv * n_c + chunk_in_head;
         constexpr int kDbgRow = 8 * kC + 2 * kD;
-        long long* dbg_row = (p.dbg != nullptr && row_valid) ? p.dbg + (chunk_id * kC + il) * kDbgRow : nullptr;
+        long long* dbg_row = (DBG && p.dbg != nullptr && row_valid) ? p.dbg + (chunk_id * kC + il) * kDbgRow : nullptr;
 
         int bq = 0, dq = 0, kexp = 0, vexp = 0;
         if (row_valid) {
@@ -365,7 +368,7 @@ chunk_tc_int16_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
 #pragma unroll
             for (int jl = 0; jl < kHC; ++jl) {
                 const long long G = combine(ghh[jl], gmid[jl], gll[jl]);
-                if (dbg_row != nullptr) dbg_row[col0 + jl] = G;
+                if (DBG && dbg_row != nullptr) dbg_row[col0 + jl] = G;
                 const int j = col0 + jl;
                 const int dlt = dq - sdecay[cb + j];
                 const int sh = dlt >> 8;
@@ -552,7 +555,7 @@ chunk_tc_int16_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
 #pragma unroll
             for (int jl = 0; jl < kHC; ++jl) {
                 acc[jl] = combine(dhh[jl], dmid[jl], dll[jl]);
-                if (dbg_row != nullptr) dbg_row[(s - 1) * kC + col0 + jl] = acc[jl];
+                if (DBG && dbg_row != nullptr) dbg_row[(s - 1) * kC + col0 + jl] = acc[jl];
                 m |= abs64(acc[jl]);
             }
             const int r = q_shift(chunk_bitlen(m, slot++));
@@ -759,7 +762,7 @@ chunk_tc_int16_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
                 tmem_ld16(lane_base + kDmid + h * 64 + c0, dmid);
                 tmem_ld16(lane_base + kDll + h * 64 + c0, dll);
                 tmem_wait_ld();
-                if (dbg_row != nullptr) {
+                if (DBG && dbg_row != nullptr) {
 #pragma unroll
                     for (int i = 0; i < 16; ++i) dbg_row[8 * kC + half * kD + h * 64 + c0 + i] = combine(dhh[i], dmid[i], dll[i]);
                 }
@@ -923,10 +926,10 @@ int launch_tc_int16(const ProblemI16& q, cudaStream_t stream) {
     if (prm.n_tiles >= (1LL << 31) - 4096) return GDN_ERR_UNSUPPORTED;
     int8_decay_lut(prm.lut);
     const int smem = kSmemTotal + 1024;
-    if (cudaFuncSetAttribute(chunk_tc_int16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
-        return GDN_ERR_LAUNCH;
+    auto kern = (prm.dbg != nullptr) ? chunk_tc_int16_kernel<true> : chunk_tc_int16_kernel<false>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return GDN_ERR_LAUNCH;
     const long long grid = prm.n_tiles < 148 ? prm.n_tiles : 148;
-    chunk_tc_int16_kernel<<<static_cast<int>(grid), kThreads, smem, stream>>>(mK, mV, prm);
+    kern<<<static_cast<int>(grid), kThreads, smem, stream>>>(mK, mV, prm);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? GDN_OK : GDN_ERR_LAUNCH;
 }
