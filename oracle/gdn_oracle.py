@@ -269,6 +269,13 @@ def exact_inverse(A: np.ndarray) -> np.ndarray:
     return forward_substitution_inverse(-np.asarray(A, dtype=np.float64))
 
 
+def l2_normalise_rows(K: np.ndarray) -> np.ndarray:
+    """Rows of K divided by their Euclidean norm (Sec. 2.1). The paper does not say what a zero key becomes: it stays
+    zero here (a token that writes nothing), as the usual normalise-with-epsilon routines leave it."""
+    norm = np.sqrt((K * K).sum(axis=-1, keepdims=True))
+    return np.divide(K, norm, out=np.zeros_like(K), where=norm > 0)
+
+
 def chunk_prepare(K, V, beta, g, N: int | None = None, S: int | None = None, *,
                   exact: bool = False, g_raw: bool = False, k_l2norm: bool = False, w_gated: bool = False):
     """One chunk or a stack of chunks: returns (W, U, T), all fp64.
@@ -292,7 +299,7 @@ def chunk_prepare(K, V, beta, g, N: int | None = None, S: int | None = None, *,
         g = np.cumsum(g, axis=-1)
     if k_l2norm:
         # keys are l2-normalised before the path (Sec. 2.1)
-        K = K / np.sqrt((K * K).sum(axis=-1, keepdims=True))
+        K = l2_normalise_rows(K)
     A = build_A(K, beta, g)
     if exact:
         T = exact_inverse(A)
@@ -334,7 +341,7 @@ def chunk_prepare_varlen(K, V, beta, g, cu_seqlens, C: int, N: int | None = None
     beta = np.asarray(beta, dtype=np.float64)
     g = np.asarray(g, dtype=np.float64)
     if k_l2norm:
-        K = K / np.sqrt((K * K).sum(axis=-1, keepdims=True))
+        K = l2_normalise_rows(K)
     start, length = chunk_table(cu_seqlens, C)
     W = np.zeros_like(K)
     U = np.zeros_like(V)

@@ -449,6 +449,18 @@ def test_fp32_gated_w(C):
     _check_ex(inp, graw, 16 + 3, TOL_FP32 * 3)
 
 
+@pytest.mark.parametrize("C,dtype", [(64, torch.bfloat16), (128, torch.bfloat16), (16, torch.bfloat16), (64, torch.float32)])
+def test_key_normalisation_with_zero_keys(C, dtype):
+    """GDN_FLAG_K_L2NORM on keys with a few all-zero rows (tokens that write nothing): such a key stays zero, the result
+    is finite and meets the usual bars against the oracle (which defines the same)."""
+    inp, graw = _raw_inputs(1, 1, 2, 2 * C, C, seed=330 + C, dtype=dtype)
+    inp.K[0, 0, [0, 7, C - 1, C + 3]] = 0
+    W, U, Tinv = gdn.chunk_prepare(inp.K.cuda(), inp.V.cuda(), inp.beta.cuda(), graw.cuda(), C, flags=3)
+    assert bool(torch.isfinite(W.float()).all() and torch.isfinite(U.float()).all() and torch.isfinite(Tinv.float()).all())
+    assert not W[0, :, [0, 7, C - 1, C + 3]].any()
+    _check_ex(inp, graw, 3, TOL_BF16 if dtype == torch.bfloat16 else TOL_FP32 * 3)
+
+
 def test_bf16_all_flags_together_gqa_ragged():
     inp, graw = _raw_inputs(2, 1, 3, 192, 64, seed=250, adv="odd")
     _check_ex(inp, graw, 7, 5e-4)

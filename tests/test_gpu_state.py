@@ -133,6 +133,32 @@ def test_both_calls_can_be_captured_in_a_cuda_graph():
     assert gdn.gdn_device_status() == gdn.GDN_OK
 
 
+def test_layer_with_zero_key_and_query_rows_under_in_kernel_normalisation():
+    """Raw projections with a few all-zero key and query rows, normalised in the kernels: a zero row stays zero (the
+    token writes nothing / reads nothing), nothing is NaN, and the layer equals the token-by-token rule on rows
+    normalised the same way."""
+    gq = torch.Generator().manual_seed(450)
+    T, C = 256, 64
+    Q, K = torch.randn(1, T, 1, 128, generator=gq), torch.randn(1, T, 1, 128, generator=gq)
+    K[0, [0, 5, 63, 64, 200]] = 0
+    Q[0, [1, 5, 130]] = 0
+    V = torch.randn(1, T, 2, 128, generator=gq)
+    beta = torch.sigmoid(torch.randn(1, T, 2, generator=gq))
+    graw = -torch.nn.functional.softplus(torch.randn(1, T, 2, generator=gq))
+    Qb, Kb, Vb = Q.to(torch.bfloat16), K.to(torch.bfloat16), V.to(torch.bfloat16)
+    O, S = gdn.gated_delta_layer(Qb.cuda(), Kb.cuda(), Vb.cuda(), beta.cuda(), graw.cuda(), C)
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+    assert bool(torch.isfinite(O.float()).all()) and bool(torch.isfinite(S).all())
+    assert not O[0, [1, 5, 130]].any()  # a zero query reads nothing
+    q, k = orc.l2_normalise_rows(Qb[0, :, 0].double().numpy()), orc.l2_normalise_rows(Kb[0, :, 0].double().numpy())
+    for hv in range(2):
+        Oo, So = orc.gated_delta_rule(q, k, Vb[0, :, hv].double().numpy(), beta[0, :, hv].double().numpy(),
+                                      graw[0, :, hv].double().numpy(), 128 ** -0.5)
+        eO = orc.rel_frobenius(O[0, :, hv].double().cpu().numpy().reshape(T // C, C, 128), Oo.reshape(T // C, C, 128))
+        eS = orc.rel_frobenius(S[0, hv].double().cpu().numpy()[None], So[None])
+        assert eO.max() <= 1e-2 and eS.max() <= 1e-2, (eO.max(), eS.max())
+
+
 def test_zero_tokens_hand_the_initial_state_on():
     K = torch.zeros(2, 3, 0, 128, dtype=torch.bfloat16, device="cuda")
     g = torch.zeros(2, 3, 0, device="cuda")

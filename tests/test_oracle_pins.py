@@ -164,6 +164,28 @@ def test_chunkwise_output_with_a_gate_that_closes_fast_is_finite_and_equals_the_
     assert np.allclose(O, own, atol=1e-10)
 
 
+def test_key_normalisation_leaves_a_zero_key_zero():
+    """Normalised keys: every non-zero row has unit norm and the result equals the plain call on rows normalised by
+    hand; a zero key stays zero, so its token neither reads nor writes (row and column of A vanish, its row of T is
+    the unit row and W_i = 0), and nothing is NaN."""
+    rng = np.random.default_rng(21)
+    C, d = 16, 8
+    K = rng.normal(size=(C, d)) * rng.uniform(0.2, 5.0, size=(C, 1))
+    K[5] = 0.0
+    V = rng.normal(size=(C, d))
+    beta = rng.uniform(0.2, 0.9, size=C)
+    g = np.cumsum(-rng.uniform(0.01, 0.3, size=C))
+    Kn = K.copy()
+    nz = np.arange(C) != 5
+    Kn[nz] /= np.linalg.norm(K[nz], axis=1, keepdims=True)
+    assert np.allclose(np.linalg.norm(orc.l2_normalise_rows(K)[nz], axis=1), 1.0) and not orc.l2_normalise_rows(K)[5].any()
+    with np.errstate(invalid="raise", divide="raise"):
+        W, U, T = orc.chunk_prepare(K, V, beta, g, exact=True, k_l2norm=True)
+    W0, U0, T0 = orc.chunk_prepare(Kn, V, beta, g, exact=True)
+    assert np.isfinite(W).all() and np.allclose(W, W0, atol=1e-14) and np.allclose(U, U0, atol=1e-14) and np.allclose(T, T0, atol=1e-14)
+    assert not T[5, :5].any() and not T[6:, 5].any() and not W[5].any() and np.allclose(U[5], beta[5] * V[5])
+
+
 def test_variable_length_sequences_equal_the_token_recurrence_per_sequence():
     """Packed sequences of ragged lengths: the chunk quantities of `chunk_prepare_varlen` (chunks counted from each
     sequence's first token, the last one short) carried through the chunk-wise state passing reproduce the
