@@ -29,7 +29,12 @@
  *     Tinv [B, H_v, T/C, C, C] (the full matrix, unit diagonal included, zeros
  *     above it). K, V, W, U, Tinv have the element type selected by `dtype`.
  *   - g is the CUMULATIVE log-gate. Only differences inside a chunk are used,
- *     so a chunk-local or a global prefix sum give the same result.
+ *     so a chunk-local or a global prefix sum give the same result. Gates are at most 1: g must not increase inside
+ *     a chunk (raw log-gates <= 0). The decay factor exp(g_i - g_j), i > j, is evaluated with its exponent clamped at
+ *     +64 octaves, so an increasing g gives finite but unspecified results; any rate of decrease is fine (the factor
+ *     underflows to 0 for a gate that closes).
+ *   - Degenerate inputs are well defined: a zero key or beta = 0 is a token that writes nothing (T keeps its unit row
+ *     there); with GDN_FLAG_K_L2NORM a zero key stays zero; B = 0 or T = 0 launches nothing.
  *   - Value head h reads key head h / (H_v / H_k); H_v must be a multiple of H_k.
  *   - order = N >= 1 and residual_steps = S >= 0; -1 selects the paper's value
  *     for the chunk size (gdn_default_order, gdn_default_residual_steps).
