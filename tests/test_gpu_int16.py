@@ -60,6 +60,16 @@ def test_int16_saturating_and_degenerate_inputs_bit_exact(case):
             _check(inp, N, S, mutate=lambda q: gen.int_edge_inputs(q, case, bits=16))
 
 
+def test_int16_without_the_t_output_gives_the_same_w_and_u():
+    inp = gen.make_inputs(1, 2, 2, 256, 64, 128, 128, seed=140, adversarial_heads="odd")
+    qd = _to_dev(gen.make_int16_inputs(inp))
+    full = gdn.chunk_prepare_int16(qd)
+    part = gdn.chunk_prepare_int16(qd, want_toff=False)
+    assert gdn.gdn_device_status() == gdn.GDN_OK and part[4] is None
+    for i in (0, 1, 2, 3, 5):
+        assert torch.equal(full[i], part[i])
+
+
 def test_int16_gqa_ragged_and_many_tiles():
     inp = gen.make_inputs(2, 2, 6, 192, 64, 128, 128, seed=120, adversarial_heads="odd")
     _check(inp)

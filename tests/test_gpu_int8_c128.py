@@ -97,3 +97,18 @@ def test_int8_c128_unsupported_configurations():
     with pytest.raises(gdn.GdnError) as e:
         gdn.chunk_prepare_int8(qd, outputs=(Wq, Uq, w_exp, u_exp, Toff, t_exp), dbg_acc=dbg)
     assert e.value.status == gdn.GDN_ERR_UNSUPPORTED
+
+
+def test_int8_c128_needs_the_t_output():
+    """The second launch reads the diagonal blocks of T back from Toff_q_out: the C ABI refuses a null pointer there
+    (the binding always allocates it for chunks of 128 tokens)."""
+    inp = gen.make_inputs(1, 1, 1, 256, 128, 128, 128, seed=260)
+    qd = _to_dev(gen.make_int8_inputs(inp))
+    out = gdn.chunk_prepare_int8(qd, want_toff=False)
+    assert out[4] is not None
+    W, U = torch.empty_like(qd.Kq), torch.empty_like(qd.Vq)
+    we = torch.empty(1, 1, 2, 2, dtype=torch.int32, device="cuda")
+    ue, te = torch.empty_like(we), torch.empty(1, 1, 2, 3, dtype=torch.int32, device="cuda")
+    rc = gdn.gdn_chunk_prepare_int8(qd.Kq, qd.Vq, qd.k_exp, qd.v_exp, qd.beta_q, qd.decay_q, 1, 1, 1, 256, 128, 128, 128, -1, -1,
+                                    W, U, we, ue, None, te, None, check=False)
+    assert rc == gdn.GDN_ERR_UNSUPPORTED
