@@ -74,6 +74,18 @@ def test_tensor_core_kernel_on_random_configurations():
             raise AssertionError(f"{what}: {e}") from e
 
 
+def test_blocked_substitution_with_tensor_core_merge_on_random_configurations():
+    rng = random.Random(8)
+    for it in range(30):
+        B, Hk, grp = rng.choice([1, 2, 3]), rng.choice([1, 2, 3]), rng.choice([1, 2, 4])
+        T, adv = 64 * rng.choice([1, 2, 3, 5, 9]), rng.choice(["none", "odd", "all"])
+        inp = gen.make_inputs(B, Hk, Hk * grp, T, 64, 128, 128, seed=30000 + it, adversarial_heads=adv)
+        try:
+            _exact_check(inp, gdn.GDN_FWDSUBST_BLOCKED_TC, tp.TOL_BF16)
+        except AssertionError as e:
+            raise AssertionError(f"#{it} B={B} H_k={Hk} group={grp} T={T} adv={adv}: {e}") from e
+
+
 def test_plain_fma_kernel_on_random_configurations():
     rng = random.Random(2468)
     for it in range(150):
