@@ -24,6 +24,7 @@
 // The forward-substitution comparisons (Eq. 2-3; App. E for the blocked form) replace the L / E / residual steps by a
 // column-parallel substitution in shared memory and reuse everything else.
 #include <cuda.h>
+#include <cstdlib>
 
 #include "common.cuh"
 #include "sm100_ptx.cuh"
@@ -289,7 +290,7 @@ __device__ __forceinline__ void load_diag_block(uint32_t lane_base, uint32_t col
 // hi (slot AS) = bf16(T diag(scale)) over the whole row, lo (slot R2) = bf16 of what hi loses on the diagonal and
 // the band, where entries are O(1). `sc` is the per-token scale in shared memory, `sc_i` the row's own scale;
 // a[] = far part of the row, lb[] = band, y[] = T21 part (second block of a 128-chunk).
-template <int C, int NB, bool MERGE, bool YPART = MERGE, bool KEEP = true>
+template <int C, int NB, bool MERGE, bool YPART = MERGE, bool KEEP = true, bool PERM = false>
 __device__ __forceinline__ void build_wu_operands(uint32_t lane_base, uint32_t br_line, const uint32_t (&slot)[NB + 1], int t, int h,
                                                   int il, int cb, int col0, int wq, const float* sc, float sc_i,
                                                   const float (&a)[Split<C>::HC],
@@ -336,6 +337,13 @@ __device__ __forceinline__ void build_wu_operands(uint32_t lane_base, uint32_t b
                 store_stacked_operand<C>(lane_base + kR2, h, pl);
             }
         }
+    }
+    if constexpr (PERM) {
+        // (M = 64 products per chunk: no zero columns of the other chunk to fill, columns 0..31 for both chunks)
+        store_a_operand<C, false>(lane_base + kAS, 0, h, pk);
+        build_band_row<C, NB>(br_line, slot, lo, bp);
+        store_a_operand<C, false>(lane_base + kR2, 0, h, bp);
+        return;
     }
     if (plain) store_a_operand<C, true>(lane_base + kAS, t, h, pk);
     build_band_row<C, NB>(br_line, slot, lo, bp);
@@ -425,7 +433,7 @@ __device__ __forceinline__ TileCoord tile_coord(const TilePos& c, const Params& 
 // last two cost registers, so each has its own code.
 // DBL: 8 or 15 = the residual sum for that S is evaluated by the four-level doubling scheme (C = 64 only); 0 = one
 // product per term.
-template <int C, int NB, int MODE, bool MERGE, int EX, int DBL>
+template <int C, int NB, int MODE, bool MERGE, int EX, int DBL, bool PERM = false>
 __global__ void __launch_bounds__(kThreads, 2)
 chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                 const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmU,
@@ -512,7 +520,22 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     // [h * HC, (h + 1) * HC) when C >= 32; for C = 16 only h = 0 works on the row (h = 1 joins for W/U).
     // One elected lane of warp 0 also issues every TMA load and every tcgen05.mma, right after the CTA barrier
     // that says all rows of the operand are in place.
-    const int t = tid & 127;
+    // kPerm (PERM instantiations of the default 64-chunk path): every tensor-core product is an M = 64 instruction on ONE chunk, so
+    // that none multiplies the structural zeros an M = 128 instruction spanning both chunks of the tile would (half of
+    // the Gram product, half of the K steps of the block-diagonal W / U operands; that work is what drives the launch
+    // into the power cap). An M = 64 accumulator (and A operand) occupies 16 lanes of every lane quadrant: rows
+    // 16 q .. 16 q + 15 on lanes 32 q .. 32 q + 15, and with a lane offset of 16 the other half-lanes. So chunk 0 lives on
+    // the lanes [0, 16) of every quadrant and chunk 1 on the lanes [16, 32): the thread on TMEM lane l works on tile row
+    // t = 64 ((l / 16) % 2) + 16 (l / 32) + l % 16 instead of t = l. Everything indexed by a token (shared arrays, global
+    // rows, B operands) keeps using t; TMEM columns no longer depend on the chunk (the two chunks sit on different
+    // lanes of the same columns); a warp holds two groups of 16 consecutive rows, which leave as two bulk stores.
+    // M = 64 instructions take as long as M = 128 ones (and the doubling levels need twice as many of them), so at full
+    // clocks this form is ~10 % slower; it draws less power, and a launch long enough to run into the power cap is
+    // faster with it. The host picks it for large launches (launch_tc_bf16).
+    static_assert(!PERM || (C == 64 && !MERGE && MODE == INV_NEUMANN && EX == 0 && DBL != 0), "built for the default 64-chunk path");
+    constexpr bool kPerm = PERM;
+    const int lrow = tid & 127;  // TMEM lane of this thread's row
+    const int t = kPerm ? ((((lrow >> 4) & 1) << 6) + ((lrow >> 5) << 4) + (lrow & 15)) : lrow;
     const int h = tid >> 7;
     const bool active = SP::kSplit || (h == 0);
     const int col0 = SP::kSplit ? h * HC : 0;  // first chunk-local column of this thread
@@ -534,6 +557,19 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     // Completion of the MMAs committed to bar_mma: warp 0 polls the mbarrier, the other warps sleep on a hardware
     // barrier that warp 0 joins afterwards (no polling instructions from 7 of the 8 warps). A timeout is published
     // in s_fail, so that every thread leaves the tile loop at the same point.
+    // kPerm: W (or U) of chunk m = (hi + lo operand of the chunk, 4 + 4 K steps of its own 64 tokens) x (the chunk's rows
+    // of the K (V) tile), an M = 64, N = 128 product on the chunk's half-lanes
+    auto issue_wu64 = [&](uint32_t tile_a) {
+#pragma unroll
+        for (int m = 0; m < 2; ++m) {
+            const uint32_t lm = static_cast<uint32_t>(16 * m) << 16;
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                const uint64_t bd = smem_desc(tile_a + (4 * m + (ks & 3)) * 2048, 16384, 1024, SWZ_128B);
+                mma_f16_ts(tmem + kR0 + lm, tmem + ((ks < 4) ? kAS : kR2) + (ks & 3) * 8 + lm, bd, instr_desc(64, 128, 1, 1, 0, 1, 1), ks > 0);
+            }
+        }
+    };
     auto wait_mma = [&]() -> bool {
         if (warp == 0 && !wait_bar(&bar_mma, par_mma)) *reinterpret_cast<volatile int*>(&s_fail) = 1;
         asm volatile("bar.sync 2, 256;" ::: "memory");
@@ -679,9 +715,22 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 tc_fence_after_sync();
                 if (elect_one()) {
 #pragma unroll
+                    if constexpr (kPerm) {
+                        // one 64 x 64 Gram block per chunk, on the chunk's half-lanes, both in columns 0..63
+#pragma unroll
+                        for (int m = 0; m < 2; ++m) {
+#pragma unroll
+                            for (int ks = 0; ks < 8; ++ks) {
+                                const uint64_t d = smem_desc(sK_a + (ks >> 2) * 16384 + m * 8192 + (ks & 3) * 32, 16, 1024, SWZ_128B);
+                                mma_f16_ss(tmem + kR0 + (static_cast<uint32_t>(16 * m) << 16), d, d, instr_desc(64, 64, 1, 1, 0, 0, 1), ks > 0);
+                            }
+                        }
+                    } else {
+#pragma unroll
                     for (int ks = 0; ks < 8; ++ks) {
                         const uint64_t d = smem_desc(sK_a + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024, SWZ_128B);
                         mma_f16_ss(tmem + kR0, d, d, idesc_g, ks > 0);
+                    }
                     }
                     mma_commit(&bar_mma);
                 }
@@ -723,7 +772,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 tmem_wait_st();
             }
         }
-        if (active) load_diag_block<C>(lane_base, kR0, t, h, a);
+        if (active) load_diag_block<C>(lane_base, kR0, kPerm ? (t & 63) : t, h, a);
         float rni = 1.f;
         if (f_l2) {
             // keys are normalised on the fly: 1 / ||K_i|| from the diagonal of the Gram matrix
@@ -1150,10 +1199,10 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     // (E_m, E_m^2 or E_m^4) comes out of the same instruction. A thread therefore owns, besides its
                     // part of row il of X of its chunk, the same part of row il of the powers of the OTHER chunk's E.
                     const int co = cb ^ 64;  // first tile row of the other chunk
-                    const uint32_t a_own = lane_base + kAS + (cb >> 1) + h * 16;
-                    const uint32_t a_oth = lane_base + kAS + (co >> 1) + h * 16;
-                    const uint32_t d_own = lane_base + kR0 + cb + h * 32;
-                    const uint32_t d_oth = lane_base + kR0 + co + h * 32;
+                    const uint32_t a_own = lane_base + kAS + (kPerm ? 0 : (cb >> 1)) + h * 16;
+                    const uint32_t a_oth = lane_base + kAS + (kPerm ? 32 : (co >> 1)) + h * 16;
+                    const uint32_t d_own = lane_base + kR0 + (kPerm ? 0 : cb) + h * 32;
+                    const uint32_t d_oth = lane_base + kR0 + (kPerm ? 64 : co) + h * 32;
                     uint8_t* sQB = sEB + 16384;  // powers of E as B operand, same layout as E
                     const uint32_t b_oth = ((co + col0) >> 3) * 1024 + il * 16;
                     const uint32_t idesc_h = instr_desc(128, 64, 1, 1, 0, 1, 1);
@@ -1182,6 +1231,30 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                             tc_fence_after_sync();
                             const uint32_t bb = (lv == 0 || (lv == 2 && !kFull)) ? sEB_a : sEB_a + 16384;
                             if (elect_one()) {
+                            if constexpr (kPerm) {
+                                // with B_m (E_m or one of its powers): the X rows of chunk m, on that chunk's half-lanes
+                                // (operand columns 0..31 -> accumulator columns 0..63), and the rows of the power of E_m,
+                                // which the threads of the OTHER chunk hold (columns 32..63 -> 64..127), while a power is
+                                // still needed
+                                constexpr uint32_t idesc_p = instr_desc(64, 64, 1, 1, 0, 1, 1);
+                                const bool powers = lv < (kFull ? 3 : 2);
+#pragma unroll
+                                for (int m = 0; m < 2; ++m) {
+                                    const uint32_t lm = static_cast<uint32_t>(16 * m) << 16, lo = static_cast<uint32_t>(16 * (1 - m)) << 16;
+#pragma unroll
+                                    for (int ks = 0; ks < 4; ++ks) {
+                                        const uint64_t bd = smem_desc(bb + m * 8192 + ks * 256, 128, 1024, SWZ_NONE);
+                                        mma_f16_ts(tmem + kR0 + lm, tmem + kAS + ks * 8 + lm, bd, idesc_p, ks > 0);
+                                    }
+                                    if (powers) {
+#pragma unroll
+                                        for (int ks = 0; ks < 4; ++ks) {
+                                            const uint64_t bd = smem_desc(bb + m * 8192 + ks * 256, 128, 1024, SWZ_NONE);
+                                            mma_f16_ts(tmem + kR0 + 64 + lo, tmem + kAS + 32 + ks * 8 + lo, bd, idesc_p, ks > 0);
+                                        }
+                                    }
+                                }
+                            } else {
 #pragma unroll
                             for (int m = 0; m < 2; ++m) {
 #pragma unroll
@@ -1189,6 +1262,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                                     const uint64_t bd = smem_desc(bb + m * 8192 + ks * 256, 128, 1024, SWZ_NONE);
                                     mma_f16_ts(tmem + kR0 + 64 * m, tmem + kAS + 32 * m + ks * 8, bd, idesc_h, ks > 0);
                                 }
+                            }
                             }
                             mma_commit(&bar_mma);
                             }
@@ -1489,7 +1563,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         // ---- A operands for W/U: T diag(scale) = hi + lo, hi over the whole row, lo only on band + diagonal.
         // scale = beta for U; for W it is beta / ||K|| when the keys are normalised on the fly, else beta as well
         if (active) {
-            build_wu_operands<C, NB, MERGE, MERGE && !Y_EARLY, kKeepMask>(lane_base, br_line, slot, t, h, il, cb, col0, wq, two_scales ? sbrn : sbeta,
+            build_wu_operands<C, NB, MERGE, MERGE && !Y_EARLY, kKeepMask, kPerm>(lane_base, br_line, slot, t, h, il, cb, col0, wq, two_scales ? sbrn : sbeta,
                                             two_scales ? sbrn[t] : bi, a, keep, lb, y);
             if constexpr (MERGE) {
                 // I + L again for the Tinv rows: rebuilt here instead of being carried across the merge, where
@@ -1511,10 +1585,11 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             tc_fence_after_sync();
             if (elect_one()) {
 #pragma unroll
-                for (int ks = 0; ks < 16; ++ks) {
+                for (int ks = 0; ks < (kPerm ? 0 : 16); ++ks) {
                     const uint64_t bd = smem_desc(sK_a + (ks & 7) * 2048, 16384, 1024, SWZ_128B);
                     mma_f16_ts(tmem + kR0, tmem + ((ks < 8) ? kAS : kR2) + (ks & 7) * 8, bd, idesc_w, ks > 0);
                 }
+                if constexpr (kPerm) issue_wu64(sK_a);
                 mma_commit(&bar_mma);
             }
         }
@@ -1594,10 +1669,11 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         } else if (p.Tinv != nullptr && active) {
             constexpr int RB = HC * 2;  // bytes per staged half-row
             const uint32_t stage = smem_u32(smem + kTinvStage) + h * (kTile * RB);
-            const uint32_t trow = stage + t * RB;
+            const int srow = kPerm ? lrow : t;  // (kPerm: a warp's 32 lanes hold 16 rows of each chunk; staged in lane order)
+            const uint32_t trow = stage + srow * RB;
 #pragma unroll
             for (int c = 0; c < CPT; ++c) {
-                sts128(trow + (swz<CPT>(t, c) << 4),
+                sts128(trow + (swz<CPT>(srow, c) << 4),
                        (kKeepMask ? (pack_bf16x2(a[c * 8 + 0], a[c * 8 + 1]) & keep[c * 4 + 0]) : pack_bf16x2(a[c * 8 + 0], a[c * 8 + 1])) | bpT[c * 4 + 0],
                        (kKeepMask ? (pack_bf16x2(a[c * 8 + 2], a[c * 8 + 3]) & keep[c * 4 + 1]) : pack_bf16x2(a[c * 8 + 2], a[c * 8 + 3])) | bpT[c * 4 + 1],
                        (kKeepMask ? (pack_bf16x2(a[c * 8 + 4], a[c * 8 + 5]) & keep[c * 4 + 2]) : pack_bf16x2(a[c * 8 + 4], a[c * 8 + 5])) | bpT[c * 4 + 2],
@@ -1606,7 +1682,13 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) {
-                tma_store_3d(&tmT, smem + kTinvStage + h * (kTile * RB) + wrow0 * RB, col0, tc.t0 + wrow0, tc.bhv);
+                if constexpr (kPerm) {
+#pragma unroll
+                    for (int m = 0; m < 2; ++m)
+                        tma_store_3d(&tmT, smem + kTinvStage + h * (kTile * RB) + (wrow0 + 16 * m) * RB, col0, tc.t0 + 64 * m + 16 * wq, tc.bhv);
+                } else {
+                    tma_store_3d(&tmT, smem + kTinvStage + h * (kTile * RB) + wrow0 * RB, col0, tc.t0 + wrow0, tc.bhv);
+                }
                 tma_store_commit();
             }
         }
@@ -1629,7 +1711,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 if (half == 0 && two_scales && active) {
                     // U uses beta where W used beta / ||K|| (or beta exp(g)): both A operands again (the W product has
                     // completed; the hand-over to the issuing thread is the barrier below)
-                    build_wu_operands<C, NB, MERGE, MERGE && !Y_EARLY, kKeepMask>(lane_base, br_line, slot, t, h, il, cb, col0, wq, sbeta, bi, a, keep, lb, y);
+                    build_wu_operands<C, NB, MERGE, MERGE && !Y_EARLY, kKeepMask, kPerm>(lane_base, br_line, slot, t, h, il, cb, col0, wq, sbeta, bi, a, keep, lb, y);
                     tmem_wait_st();
                 }
             }
@@ -1661,7 +1743,7 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 if (!kEarlyU && two_scales) {
                     // U uses beta where W used beta / ||K|| (or beta exp(g)): rebuild both A operands
                     if (active) {
-                        build_wu_operands<C, NB, MERGE, MERGE && !Y_EARLY, kKeepMask>(lane_base, br_line, slot, t, h, il, cb, col0, wq, sbeta, bi, a, keep, lb, y);
+                        build_wu_operands<C, NB, MERGE, MERGE && !Y_EARLY, kKeepMask, kPerm>(lane_base, br_line, slot, t, h, il, cb, col0, wq, sbeta, bi, a, keep, lb, y);
                         tmem_wait_st();
                     }
                     tc_fence_before_sync();
@@ -1673,10 +1755,11 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                         tc_fence_after_sync();
                         if (elect_one()) {
 #pragma unroll
-                            for (int ks = 0; ks < 16; ++ks) {
+                            for (int ks = 0; ks < (kPerm ? 0 : 16); ++ks) {
                                 const uint64_t bd = smem_desc(sV_a + (ks & 7) * 2048, 16384, 1024, SWZ_128B);
                                 mma_f16_ts(tmem + kR0, tmem + ((ks < 8) ? kAS : kR2) + (ks & 7) * 8, bd, idesc_w, ks > 0);
                             }
+                            if constexpr (kPerm) issue_wu64(sV_a);
                             mma_commit(&bar_mma);
                         }
                     }
@@ -1710,7 +1793,14 @@ chunk_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) {
-                    tma_store_3d((half == 0) ? &tmW : &tmU, smem + L::kEB + wq * 8192 + h * 4096, tc.vx + h * 64, tok0, tc.vz);
+                    if constexpr (kPerm) {
+#pragma unroll
+                        for (int m = 0; m < 2; ++m)
+                            tma_store_3d((half == 0) ? &tmW : &tmU, smem + L::kEB + wq * 8192 + h * 4096 + m * 2048, tc.vx + h * 64,
+                                         tc.t0 + 64 * m + 16 * wq, tc.vz);
+                    } else {
+                        tma_store_3d((half == 0) ? &tmW : &tmU, smem + L::kEB + wq * 8192 + h * 4096, tc.vx + h * 64, tok0, tc.vz);
+                    }
                     tma_store_commit();
                 }
             }
@@ -1763,11 +1853,11 @@ struct Maps {
     CUtensorMap K, V, W, U, T;
 };
 
-template <int C, int NB, int MODE, bool MERGE, int EX, int DBL>
+template <int C, int NB, int MODE, bool MERGE, int EX, int DBL, bool PERM = false>
 int launch_ex(const Maps& m, const Params& prm, cudaStream_t stream) {
     using L = Smem<C, NB>;
     const int smem = L::kTotal + 1024;
-    auto kern = chunk_tc_kernel<C, NB, MODE, MERGE, EX, DBL>;
+    auto kern = chunk_tc_kernel<C, NB, MODE, MERGE, EX, DBL, PERM>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return GDN_ERR_LAUNCH;
     long long grid = prm.n_tiles < 2 * 148 ? prm.n_tiles : 2 * 148;
     Params q = prm;
@@ -1781,7 +1871,7 @@ int launch_ex(const Maps& m, const Params& prm, cudaStream_t stream) {
 }
 
 template <int C, int NB, int MODE, bool MERGE>
-int launch_one(const Maps& m, const Params& prm, cudaStream_t stream) {
+int launch_one(const Maps& m, const Params& prm, cudaStream_t stream, bool perm) {
     constexpr bool kNeu = (MODE == INV_NEUMANN);
     constexpr bool kDbl = kNeu && C == 64;
     const int dbl = !kDbl ? 0 : (prm.S == 8 ? 8 : (prm.S == 15 ? 15 : 0));
@@ -1800,21 +1890,28 @@ int launch_one(const Maps& m, const Params& prm, cudaStream_t stream) {
         if (dbl == 15) return launch_ex<C, NB, MODE, MERGE, kNeu ? 1 : 0, kDbl ? 15 : 0>(m, prm, stream);
         return launch_ex<C, NB, MODE, MERGE, kNeu ? 1 : 0, 0>(m, prm, stream);
     }
+    if constexpr (kDbl && !MERGE) {
+        // (the tensor maps of W, U and Tinv were built with 16-row boxes when `perm` is set: see launch_tc_bf16)
+        if (perm && dbl == 8) return launch_ex<C, NB, MODE, MERGE, 0, 8, true>(m, prm, stream);
+        if (perm && dbl == 15) return launch_ex<C, NB, MODE, MERGE, 0, 15, true>(m, prm, stream);
+    }
+    if (perm) return GDN_ERR_LAUNCH;  // (not reached: `perm` is only set for the cases above)
     if (dbl == 8) return launch_ex<C, NB, MODE, MERGE, 0, kDbl ? 8 : 0>(m, prm, stream);
     if (dbl == 15) return launch_ex<C, NB, MODE, MERGE, 0, kDbl ? 15 : 0>(m, prm, stream);
     return launch_ex<C, NB, MODE, MERGE, 0, 0>(m, prm, stream);
 }
 
 template <int C, int MODE, bool MERGE = false>
-int launch_c(const Maps& m, const Params& prm, cudaStream_t stream) {
-    if (MODE != INV_NEUMANN || prm.N <= 3) return launch_one<C, 3, MODE, MERGE>(m, prm, stream);
-    return launch_one<C, 7, MODE, MERGE>(m, prm, stream);
+int launch_c(const Maps& m, const Params& prm, cudaStream_t stream, bool perm = false) {
+    if (MODE != INV_NEUMANN || prm.N <= 3) return launch_one<C, 3, MODE, MERGE>(m, prm, stream, perm);
+    return launch_one<C, 7, MODE, MERGE>(m, prm, stream, perm);
 }
 
 }  // namespace
 
 
 namespace {
+constexpr long long kM64MinTiles = 32768;  // 65 536 chunks of 64 tokens: a launch of about 1.2 ms
 // waits on an mbarrier that never completes: wait_bar must give up after its budget and report it
 __global__ void wait_selftest_kernel(int* status) {
     __shared__ uint64_t bar;
@@ -1860,10 +1957,22 @@ int launch_tc_bf16(const Problem& p, InverseMode mode, cudaStream_t stream) {
     const int in_rows = varlen ? p.C : 128;
     if (!make_map(&m.K, p.K, zk, t_in, ck, 64, in_rows, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
     if (!make_map(&m.V, p.V, zv, t_in, cv, 64, in_rows, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
-    if (!make_map(&m.W, p.W, zv, t_in, cv, 64, 32, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
-    if (!make_map(&m.U, p.U, zv, t_in, cv, 64, 32, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
+    // Large launches of the default 64-chunk path (no flags, S = 8 or 15) run the form whose tensor-core products are
+    // M = 64 instructions per chunk (kPerm in the kernel): it draws less power, and a launch of a millisecond or more
+    // runs into the power cap, where that is worth more than the ~10 % it costs at full clocks. Its warps hold 16 rows
+    // of each of a tile's two chunks, so its W, U and Tinv rows leave in boxes of 16 rows. (GDN_FORCE_M64 = 1 / 0 in the
+    // environment forces the choice: the tests run both forms on small cases.)
+    const long long n_tiles_all = (long long)p.B * p.H_v * ((p.T + kTile - 1) / kTile);
+    bool perm = p.C == 64 && mode == INV_NEUMANN && p.flags == 0 && !varlen && (p.steps == 8 || p.steps == 15);
+    if (perm) {
+        const char* force = getenv("GDN_FORCE_M64");
+        perm = (force != nullptr) ? (force[0] == '1') : (n_tiles_all >= kM64MinTiles);
+    }
+    const int obox = perm ? 16 : 32;
+    if (!make_map(&m.W, p.W, zv, t_in, cv, 64, obox, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
+    if (!make_map(&m.U, p.U, zv, t_in, cv, 64, obox, CU_TENSOR_MAP_SWIZZLE_128B)) return GDN_ERR_LAUNCH;
     // Tinv rows are C wide; without a Tinv output the map points at W (never used by the kernel then)
-    if (!make_map(&m.T, p.Tinv != nullptr ? p.Tinv : p.W, hv, p.T, p.Tinv != nullptr ? p.C : kD, p.Tinv != nullptr ? tbox : 64, 32,
+    if (!make_map(&m.T, p.Tinv != nullptr ? p.Tinv : p.W, hv, p.T, p.Tinv != nullptr ? p.C : kD, p.Tinv != nullptr ? tbox : 64, obox,
                   p.Tinv != nullptr ? tsw : CU_TENSOR_MAP_SWIZZLE_128B))
         return GDN_ERR_LAUNCH;
     Params prm;
@@ -1893,7 +2002,7 @@ int launch_tc_bf16(const Problem& p, InverseMode mode, cudaStream_t stream) {
             case 16: return launch_c<16, INV_NEUMANN>(m, prm, stream);
             case 32: return launch_c<32, INV_NEUMANN>(m, prm, stream);
             case 128: return launch_c<64, INV_NEUMANN, true>(m, prm, stream);
-            default: return launch_c<64, INV_NEUMANN>(m, prm, stream);
+            default: return launch_c<64, INV_NEUMANN>(m, prm, stream, perm);
         }
     }
     if (mode == INV_FWDSUBST_TC) {

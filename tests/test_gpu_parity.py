@@ -566,3 +566,29 @@ def test_host_threads_on_their_own_streams_do_not_disturb_each_other():
         th.join()
     torch.cuda.synchronize()
     assert not errors and gdn.gdn_device_status() == gdn.GDN_OK
+
+
+@pytest.mark.parametrize("adv", ["none", "all"])
+@pytest.mark.parametrize("N,S", [(-1, -1), (3, 15), (5, 8)])
+def test_bf16_large_launch_form_on_small_cases(adv, N, S, monkeypatch):
+    """Large launches of the default 64-chunk path run a second form of the kernel (every tensor-core product an M = 64
+    instruction on one chunk, the rows of the two chunks interleaved over the lanes; the library picks it by launch
+    size). GDN_FORCE_M64 selects it here on small cases: grouped heads, a ragged last tile, benign and adversarial
+    heads, the exact inverse (S = 15), a wider band (N = 5), with and without the Tinv output; same bars against the
+    oracle, and W, U, Tinv within one bf16 rounding of the other form (the two differ in the order of fp32 sums)."""
+    inp = gen.make_inputs(2, 2, 4, 64 * 7, 64, 128, 128, seed=800, adversarial_heads=adv)
+    K, V, beta, g = _to_dev(inp)
+    monkeypatch.setenv("GDN_FORCE_M64", "0")
+    ref = gdn.chunk_prepare(K, V, beta, g, 64, N, S)
+    monkeypatch.setenv("GDN_FORCE_M64", "1")
+    _check(inp, TOL_BF16, N, S)
+    got = gdn.chunk_prepare(K, V, beta, g, 64, N, S)
+    again = gdn.chunk_prepare(K, V, beta, g, 64, N, S)
+    no_t = gdn.chunk_prepare(K, V, beta, g, 64, N, S, want_tinv=False)
+    assert gdn.gdn_device_status() == gdn.GDN_OK
+    for a, b in zip(got, again):
+        assert torch.equal(a, b)  # bit-identical repeats
+    assert torch.equal(no_t[0], got[0]) and torch.equal(no_t[1], got[1]) and no_t[2] is None
+    for a, b in zip(got, ref):
+        d = (a.float() - b.float()).abs()
+        assert bool((d <= 2.0 ** -7 * b.float().abs() + 1e-6).all())

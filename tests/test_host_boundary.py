@@ -176,11 +176,13 @@ def test_hot_kernels_are_built_without_register_spills():
     from paper_2606_06034_b200 import build as gdn_build
     gdn_build.build()
     res = gdn_build.kernel_resources("chunk_tc_bf16.cu")
-    # <C, NB, MODE, MERGE, EX, DBL>: the default C = 64 instantiation, the C = 128 one, C = 32 and C = 16, and the
-    # C = 64 instantiations with the optional prologue / layouts (EX = 1) and for packed sequences (EX = 3)
-    for key in ("chunk_tc_kernelILi64ELi3ELi0ELb0ELi0ELi8E", "chunk_tc_kernelILi64ELi3ELi0ELb1ELi0ELi8E",
-                "chunk_tc_kernelILi32ELi3ELi0ELb0ELi0ELi0E", "chunk_tc_kernelILi16ELi3ELi0ELb0ELi0ELi0E",
-                "chunk_tc_kernelILi64ELi3ELi0ELb0ELi1ELi8E", "chunk_tc_kernelILi64ELi3ELi0ELb0ELi3ELi8E"):
+    # <C, NB, MODE, MERGE, EX, DBL, PERM>: the default C = 64 instantiation in both forms (M = 128 products; M = 64
+    # products per chunk for large launches), the C = 128 one, C = 32 and C = 16, and the C = 64 instantiations with
+    # the optional prologue / layouts (EX = 1) and for packed sequences (EX = 3)
+    for key in ("chunk_tc_kernelILi64ELi3ELi0ELb0ELi0ELi8ELb0E", "chunk_tc_kernelILi64ELi3ELi0ELb0ELi0ELi8ELb1E",
+                "chunk_tc_kernelILi64ELi3ELi0ELb1ELi0ELi8ELb0E",
+                "chunk_tc_kernelILi32ELi3ELi0ELb0ELi0ELi0ELb0E", "chunk_tc_kernelILi16ELi3ELi0ELb0ELi0ELi0ELb0E",
+                "chunk_tc_kernelILi64ELi3ELi0ELb0ELi1ELi8ELb0E", "chunk_tc_kernelILi64ELi3ELi0ELb0ELi3ELi8ELb0E"):
         hits = [v for k, v in res.items() if key in k]
         assert len(hits) == 1, key
         assert hits[0]["spill_stores"] == 0 and hits[0]["spill_loads"] == 0, (key, hits[0])
